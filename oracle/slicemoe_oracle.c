@@ -1,0 +1,446 @@
+/*
+ * fp64 CPU oracle of the SliceMoE layer forward.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain statement of what the layer computes, written
+ * from the paper's Section 3 / 3.1 / 3.4 and Eq. 1.  It shares no code with
+ * the CUDA library and must never be called from the product path: only the
+ * tests, the smoke check and the bench's CPU-baseline leg may use it.
+ *
+ * Everything is row by row, in double precision, in the paper's order:
+ *   slice (Section 3)  ->  router MLP + softmax + top-k (Section 3.1)
+ *   -> weight the slice by its routing probability (Eq. 1)
+ *   -> group by expert (Section 3.4), with an optional hard capacity
+ *   -> two-layer expert FFN (Section 3.1)  -> sum the k outputs of a slice
+ *   and write it back at the slice's position in h' (Section 3.1).
+ *
+ * A row is one slice: row n = t*S + s is columns [s*ds, (s+1)*ds) of token t,
+ * which in a row-major h[T, d] is simply elements [n*ds, (n+1)*ds).
+ *
+ * Parallelism: an OpenMP `for` over independent rows only; the capacity walk
+ * is serial, so results do not depend on the thread count.
+ *
+ * Pins (tests/test_oracle_pins.py): brute-force per-slice loop on tiny
+ * inputs, a hand-worked example, identity experts, E = 1, zero router,
+ * Zipf-bias capacity closed form, reshape (S = 1) equivalence, permutation
+ * equivariance, an affine special case and a dense-MLP special case checked
+ * against numpy matmul.  No function here is unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int32_t T, d, S, E, k, Hr, F;
+    int32_t act;       /* 0 = ReLU, 1 = GELU (tanh form) */
+    int64_t capacity;  /* 0 = unlimited */
+} oracle_cfg;
+
+enum { ORACLE_OK = 0, ORACLE_BAD_SHAPE = 1, ORACLE_NO_MEMORY = 2 };
+
+int slicemoe_oracle_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+static int check_cfg(const oracle_cfg *c) {
+    if (c->T < 0 || c->d < 1 || c->S < 1 || c->E < 1 || c->k < 1 || c->Hr < 1 || c->F < 1) return ORACLE_BAD_SHAPE;
+    if (c->d % c->S != 0) return ORACLE_BAD_SHAPE;
+    if (c->k > c->E) return ORACLE_BAD_SHAPE;
+    if (c->capacity < 0) return ORACLE_BAD_SHAPE;
+    return ORACLE_OK;
+}
+
+/* Section 3.1: expert activation.  ReLU, or GELU in its tanh form. */
+static double activation(double z, int act) {
+    if (act == 0) return z > 0.0 ? z : 0.0;
+    const double c = 0.7978845608028654; /* sqrt(2/pi) */
+    return 0.5 * z * (1.0 + tanh(c * (z + 0.044715 * z * z * z)));
+}
+
+/* Section 3.1: router MLP Linear(ds->Hr), ReLU, Linear(Hr->E), then softmax.
+ * x[ds] -> p[E].  a[Hr] is scratch. */
+static void router_probs_row(const oracle_cfg *c, const double *x,
+                             const double *Wr1, const double *br1,
+                             const double *Wr2, const double *br2,
+                             double *a, double *p) {
+    const int ds = c->d / c->S;
+    for (int i = 0; i < c->Hr; ++i) {
+        double z = br1 ? br1[i] : 0.0;
+        for (int q = 0; q < ds; ++q) z += Wr1[(size_t)i * ds + q] * x[q];
+        a[i] = z > 0.0 ? z : 0.0;
+    }
+    double m = -INFINITY;
+    for (int e = 0; e < c->E; ++e) {
+        double g = br2 ? br2[e] : 0.0;
+        for (int i = 0; i < c->Hr; ++i) g += Wr2[(size_t)e * c->Hr + i] * a[i];
+        p[e] = g;
+        if (g > m) m = g;
+    }
+    double sum = 0.0;
+    for (int e = 0; e < c->E; ++e) { p[e] = exp(p[e] - m); sum += p[e]; }
+    for (int e = 0; e < c->E; ++e) p[e] /= sum;
+}
+
+/* Section 3.1: the k most probable experts of one slice, most probable first;
+ * equal probabilities go to the lower expert id.  gap = p_(k) - p_(k+1). */
+static void topk_row(const oracle_cfg *c, const double *p, int32_t *idx, double *pk, double *gap) {
+    for (int j = 0; j < c->k; ++j) {
+        int best = -1;
+        for (int e = 0; e < c->E; ++e) {
+            int taken = 0;
+            for (int i = 0; i < j; ++i) taken |= (idx[i] == e);
+            if (taken) continue;
+            if (best < 0 || p[e] > p[best]) best = e;
+        }
+        idx[j] = best;
+        pk[j] = p[best];
+    }
+    if (gap) {
+        if (c->k == c->E) { *gap = INFINITY; return; }
+        double next = -INFINITY;
+        for (int e = 0; e < c->E; ++e) {
+            int taken = 0;
+            for (int i = 0; i < c->k; ++i) taken |= (idx[i] == e);
+            if (!taken && p[e] > next) next = p[e];
+        }
+        *gap = pk[c->k - 1] - next;
+    }
+}
+
+/* Section 3.1: one expert's two-layer FFN on one (already weighted) slice.
+ * xt[ds] -> y[ds]; u[F] is scratch.  W1[E,F,ds], b1[E,F], W2[E,ds,F], b2[E,ds]. */
+static void expert_ffn_row(const oracle_cfg *c, int e, const double *xt,
+                           const double *W1, const double *b1,
+                           const double *W2, const double *b2,
+                           double *u, double *y) {
+    const int ds = c->d / c->S, F = c->F;
+    const double *W1e = W1 + (size_t)e * F * ds;
+    const double *W2e = W2 + (size_t)e * ds * F;
+    for (int f = 0; f < F; ++f) {
+        double z = b1 ? b1[(size_t)e * F + f] : 0.0;
+        for (int q = 0; q < ds; ++q) z += W1e[(size_t)f * ds + q] * xt[q];
+        u[f] = activation(z, c->act);
+    }
+    for (int q = 0; q < ds; ++q) {
+        double z = b2 ? b2[(size_t)e * ds + q] : 0.0;
+        for (int f = 0; f < F; ++f) z += W2e[(size_t)q * F + f] * u[f];
+        y[q] = z;
+    }
+}
+
+/*
+ * Route every slice (Section 3.1).
+ * in : h[T*d]; Wr1[Hr*ds], br1[Hr] or NULL, Wr2[E*Hr], br2[E] or NULL
+ * out: probs[N*E] (or NULL), topk_idx[N*k], topk_p[N*k], gap[N] (or NULL),
+ *      assigned[E] = how many (slice, j) pairs chose each expert (Section 3.2's counts).
+ */
+int slicemoe_oracle_route(const oracle_cfg *c, const double *h,
+                          const double *Wr1, const double *br1,
+                          const double *Wr2, const double *br2,
+                          double *probs, int32_t *topk_idx, double *topk_p,
+                          double *gap, int64_t *assigned) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int ds = c->d / c->S;
+    const int64_t N = (int64_t)c->T * c->S;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *a = (double *)malloc(sizeof(double) * (size_t)c->Hr);
+        double *p = (double *)malloc(sizeof(double) * (size_t)c->E);
+        if (!a || !p) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for schedule(static)
+            for (int64_t n = 0; n < N; ++n) {
+                router_probs_row(c, h + n * ds, Wr1, br1, Wr2, br2, a, p);
+                if (probs) memcpy(probs + n * c->E, p, sizeof(double) * (size_t)c->E);
+                topk_row(c, p, topk_idx + n * c->k, topk_p + n * c->k, gap ? gap + n : NULL);
+            }
+        }
+        free(a);
+        free(p);
+    }
+    if (failed) return ORACLE_NO_MEMORY;
+    if (assigned) {
+        for (int e = 0; e < c->E; ++e) assigned[e] = 0;
+        for (int64_t i = 0; i < N * c->k; ++i) assigned[topk_idx[i]] += 1;
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Group the routed (slice, j) pairs by expert (Section 3.4), with the hard
+ * per-expert capacity of the skewed-routing workload: pairs are ranked inside
+ * their expert in ascending (n, j) order; a pair whose rank reaches the
+ * capacity is dropped (dest = -1).
+ * in : topk_idx[N*k]
+ * out: assigned[E], kept[E] = min(assigned, capacity), offsets[E+1] = exclusive
+ *      scan of kept, dest[N*k] = offsets[e] + rank or -1, perm[sum kept] =
+ *      the flat pair index n*k + j stored at each destination row.
+ */
+int slicemoe_oracle_dispatch(const oracle_cfg *c, const int32_t *topk_idx,
+                             int64_t *assigned, int64_t *kept, int64_t *offsets,
+                             int64_t *dest, int64_t *perm) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int64_t R = (int64_t)c->T * c->S * c->k;
+    for (int e = 0; e < c->E; ++e) assigned[e] = 0;
+    for (int64_t i = 0; i < R; ++i) {
+        if (topk_idx[i] < 0 || topk_idx[i] >= c->E) return ORACLE_BAD_SHAPE;
+        assigned[topk_idx[i]] += 1;
+    }
+    offsets[0] = 0;
+    for (int e = 0; e < c->E; ++e) {
+        kept[e] = (c->capacity > 0 && assigned[e] > c->capacity) ? c->capacity : assigned[e];
+        offsets[e + 1] = offsets[e] + kept[e];
+    }
+    int64_t *running = (int64_t *)calloc((size_t)c->E, sizeof(int64_t));
+    if (!running) return ORACLE_NO_MEMORY;
+    for (int64_t i = 0; i < R; ++i) {
+        const int e = topk_idx[i];
+        const int64_t rank = running[e]++;
+        if (c->capacity == 0 || rank < c->capacity) {
+            dest[i] = offsets[e] + rank;
+            if (perm) perm[dest[i]] = i;
+        } else {
+            dest[i] = -1;
+        }
+    }
+    free(running);
+    return ORACLE_OK;
+}
+
+/* Eq. 1: every kept (slice, j) pair contributes the row p_j * x at its
+ * destination.  xperm[sum kept, ds]. */
+int slicemoe_oracle_weight_slices(const oracle_cfg *c, const double *h,
+                                  const double *topk_p, const int64_t *dest,
+                                  double *xperm) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int ds = c->d / c->S;
+    const int64_t N = (int64_t)c->T * c->S;
+    for (int64_t n = 0; n < N; ++n)
+        for (int j = 0; j < c->k; ++j) {
+            const int64_t r = dest[n * c->k + j];
+            if (r < 0) continue;
+            for (int q = 0; q < ds; ++q) xperm[r * ds + q] = topk_p[n * c->k + j] * h[n * ds + q];
+        }
+    return ORACLE_OK;
+}
+
+/* Section 3.1 / 3.4: each expert's FFN over its stacked rows.
+ * xperm[Rk, ds], offsets[E+1] -> yperm[Rk, ds]. */
+int slicemoe_oracle_expert_ffn(const oracle_cfg *c, const double *xperm, const int64_t *offsets,
+                               const double *W1, const double *b1,
+                               const double *W2, const double *b2, double *yperm) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int ds = c->d / c->S;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *u = (double *)malloc(sizeof(double) * (size_t)c->F);
+        if (!u) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+            for (int e = 0; e < c->E; ++e) {
+#pragma omp for schedule(static) nowait
+                for (int64_t r = offsets[e]; r < offsets[e + 1]; ++r)
+                    expert_ffn_row(c, e, xperm + r * ds, W1, b1, W2, b2, u, yperm + r * ds);
+            }
+        }
+        free(u);
+    }
+    return failed ? ORACLE_NO_MEMORY : ORACLE_OK;
+}
+
+/* Section 3.1: the k expert outputs of a slice are summed (dropped pairs add
+ * nothing; a slice with no kept pair becomes zero) and the sum is written at
+ * the slice's own columns of h'. */
+int slicemoe_oracle_combine(const oracle_cfg *c, const double *yperm, const int64_t *dest,
+                            double *h_out) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int ds = c->d / c->S;
+    const int64_t N = (int64_t)c->T * c->S;
+    for (int64_t n = 0; n < N; ++n)
+        for (int q = 0; q < ds; ++q) {
+            double acc = 0.0;
+            for (int j = 0; j < c->k; ++j) {
+                const int64_t r = dest[n * c->k + j];
+                if (r >= 0) acc += yperm[r * ds + q];
+            }
+            h_out[n * ds + q] = acc;
+        }
+    return ORACLE_OK;
+}
+
+/*
+ * The whole layer: the five steps above in order.
+ * forced_idx == NULL : experts are the router's own top-k.
+ * forced_idx != NULL : the expert ids [N*k] are taken from the caller while the
+ *   gate values are still the router's probabilities of those ids; used to
+ *   grade outputs where another implementation legitimately resolved a
+ *   near-tie differently.
+ * Optional outputs may be NULL: probs[N*E], topk_idx[N*k], topk_p[N*k],
+ * gap[N], assigned[E], kept[E], offsets[E+1], dest[N*k].
+ */
+int slicemoe_oracle_forward(const oracle_cfg *c, const double *h,
+                            const double *Wr1, const double *br1,
+                            const double *Wr2, const double *br2,
+                            const double *W1, const double *b1,
+                            const double *W2, const double *b2,
+                            const int32_t *forced_idx,
+                            double *h_out, double *probs_out,
+                            int32_t *topk_idx_out, double *topk_p_out, double *gap_out,
+                            int64_t *assigned_out, int64_t *kept_out,
+                            int64_t *offsets_out, int64_t *dest_out) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int ds = c->d / c->S;
+    const int64_t N = (int64_t)c->T * c->S, R = N * c->k;
+    const size_t E = (size_t)c->E;
+    double *probs = (double *)malloc(sizeof(double) * (size_t)(N > 0 ? N : 1) * E);
+    int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
+    double *pk = (double *)malloc(sizeof(double) * (size_t)(R > 0 ? R : 1));
+    int64_t *assigned = (int64_t *)malloc(sizeof(int64_t) * E);
+    int64_t *kept = (int64_t *)malloc(sizeof(int64_t) * E);
+    int64_t *offsets = (int64_t *)malloc(sizeof(int64_t) * (E + 1));
+    int64_t *dest = (int64_t *)malloc(sizeof(int64_t) * (size_t)(R > 0 ? R : 1));
+    double *xperm = NULL, *yperm = NULL;
+    rc = ORACLE_NO_MEMORY;
+    if (!probs || !idx || !pk || !assigned || !kept || !offsets || !dest) goto done;
+
+    rc = slicemoe_oracle_route(c, h, Wr1, br1, Wr2, br2, probs, idx, pk, gap_out, assigned);
+    if (rc) goto done;
+    if (forced_idx) {
+        for (int64_t i = 0; i < R; ++i) {
+            if (forced_idx[i] < 0 || forced_idx[i] >= c->E) { rc = ORACLE_BAD_SHAPE; goto done; }
+            idx[i] = forced_idx[i];
+            pk[i] = probs[(i / c->k) * c->E + forced_idx[i]];
+        }
+    }
+    rc = slicemoe_oracle_dispatch(c, idx, assigned, kept, offsets, dest, NULL);
+    if (rc) goto done;
+    {
+        const size_t rows = (size_t)(offsets[c->E] > 0 ? offsets[c->E] : 1);
+        xperm = (double *)malloc(sizeof(double) * rows * (size_t)ds);
+        yperm = (double *)malloc(sizeof(double) * rows * (size_t)ds);
+        if (!xperm || !yperm) { rc = ORACLE_NO_MEMORY; goto done; }
+    }
+    rc = slicemoe_oracle_weight_slices(c, h, pk, dest, xperm);
+    if (rc) goto done;
+    rc = slicemoe_oracle_expert_ffn(c, xperm, offsets, W1, b1, W2, b2, yperm);
+    if (rc) goto done;
+    rc = slicemoe_oracle_combine(c, yperm, dest, h_out);
+    if (rc) goto done;
+
+    if (probs_out) memcpy(probs_out, probs, sizeof(double) * (size_t)N * E);
+    if (topk_idx_out) memcpy(topk_idx_out, idx, sizeof(int32_t) * (size_t)R);
+    if (topk_p_out) memcpy(topk_p_out, pk, sizeof(double) * (size_t)R);
+    if (assigned_out) memcpy(assigned_out, assigned, sizeof(int64_t) * E);
+    if (kept_out) memcpy(kept_out, kept, sizeof(int64_t) * E);
+    if (offsets_out) memcpy(offsets_out, offsets, sizeof(int64_t) * (E + 1));
+    if (dest_out) memcpy(dest_out, dest, sizeof(int64_t) * (size_t)R);
+done:
+    free(probs); free(idx); free(pk); free(assigned); free(kept); free(offsets); free(dest);
+    free(xperm); free(yperm);
+    return rc;
+}
+
+/*
+ * Outputs of a chosen subset of slices, one by one (for full-size workloads
+ * where only sampled rows are graded).  For sampled row i: n = rows[i]; its
+ * experts are idx[i*k + j]; pair j contributes only if keep[i*k + j] != 0
+ * (the caller gets keep from slicemoe_oracle_dispatch on the full routing).
+ * Gate values are this oracle's router probabilities of those experts (Eq. 1).
+ * out: y[nrows*ds]; p_out[nrows*k] (or NULL).
+ */
+int slicemoe_oracle_rows(const oracle_cfg *c, const double *h,
+                         const double *Wr1, const double *br1,
+                         const double *Wr2, const double *br2,
+                         const double *W1, const double *b1,
+                         const double *W2, const double *b2,
+                         int64_t nrows, const int64_t *rows, const int32_t *idx,
+                         const int32_t *keep, double *y, double *p_out) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int ds = c->d / c->S;
+    const int64_t N = (int64_t)c->T * c->S;
+    for (int64_t i = 0; i < nrows; ++i)
+        if (rows[i] < 0 || rows[i] >= N) return ORACLE_BAD_SHAPE;
+    for (int64_t i = 0; i < nrows * c->k; ++i)
+        if (idx[i] < 0 || idx[i] >= c->E) return ORACLE_BAD_SHAPE;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *a = (double *)malloc(sizeof(double) * (size_t)c->Hr);
+        double *p = (double *)malloc(sizeof(double) * (size_t)c->E);
+        double *u = (double *)malloc(sizeof(double) * (size_t)c->F);
+        double *xt = (double *)malloc(sizeof(double) * (size_t)ds);
+        double *yj = (double *)malloc(sizeof(double) * (size_t)ds);
+        if (!a || !p || !u || !xt || !yj) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for schedule(dynamic, 16)
+            for (int64_t i = 0; i < nrows; ++i) {
+                const double *x = h + rows[i] * ds;
+                router_probs_row(c, x, Wr1, br1, Wr2, br2, a, p);
+                for (int q = 0; q < ds; ++q) y[i * ds + q] = 0.0;
+                for (int j = 0; j < c->k; ++j) {
+                    const int e = idx[i * c->k + j];
+                    if (p_out) p_out[i * c->k + j] = p[e];
+                    if (!keep[i * c->k + j]) continue;
+                    for (int q = 0; q < ds; ++q) xt[q] = p[e] * x[q];
+                    expert_ffn_row(c, e, xt, W1, b1, W2, b2, u, yj);
+                    for (int q = 0; q < ds; ++q) y[i * ds + q] += yj[q];
+                }
+            }
+        }
+        free(a); free(p); free(u); free(xt); free(yj);
+    }
+    return failed ? ORACLE_NO_MEMORY : ORACLE_OK;
+}
+
+/*
+ * Balance statistics of the per-expert counts.
+ * Eq. 2: L_cap = alpha * (std(counts) / mean(counts))^2 with the population
+ * standard deviation.  Section 4 (Metrics): ELE = -sum_e load_e log load_e / log E
+ * with load_e the fraction of routed slices on expert e (0 log 0 = 0; E = 1 gives 1).
+ */
+int slicemoe_oracle_load_stats(const int64_t *counts, int32_t E, double alpha,
+                               double *l_cap, double *ele) {
+    if (E < 1) return ORACLE_BAD_SHAPE;
+    double total = 0.0;
+    for (int e = 0; e < E; ++e) total += (double)counts[e];
+    if (total <= 0.0) { *l_cap = 0.0; *ele = 0.0; return ORACLE_OK; }
+    const double mean = total / E;
+    double var = 0.0;
+    for (int e = 0; e < E; ++e) var += ((double)counts[e] - mean) * ((double)counts[e] - mean);
+    var /= E;
+    *l_cap = alpha * var / (mean * mean);
+    double ent = 0.0;
+    for (int e = 0; e < E; ++e) {
+        const double load = (double)counts[e] / total;
+        if (load > 0.0) ent -= load * log(load);
+    }
+    *ele = (E == 1) ? 1.0 : ent / log((double)E);
+    return ORACLE_OK;
+}

@@ -1,0 +1,195 @@
+"""Seeded synthetic inputs for the SliceMoE layer forward.
+
+This module only draws random tensors and rounds them to their storage type.
+It holds none of the layer's arithmetic (no router, no softmax, no expert FFN),
+so the CUDA path and the CPU oracle can both be fed from it without sharing
+any code of the method itself.
+
+Every tensor has its own counter-based sub-stream: Philox keyed by
+(seed, tensor id).  Values are rounded to the storage dtype (bf16
+round-to-nearest-even, or fp32) *before* anyone reads them and are returned as
+float32 arrays that hold exactly those stored values.
+
+Shapes follow the paper's notation (Section 3): a token vector h in R^d is cut
+into S contiguous slices of ds = d/S; the shared router MLP is
+Linear(ds -> H_r) -> ReLU -> Linear(H_r -> E); each of the E experts is a
+two-layer FFN ds -> F -> ds; k experts are chosen per slice.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, replace
+
+import numpy as np
+
+ACT_RELU = 0
+ACT_GELU_TANH = 1
+
+_TENSOR_IDS = {"h": 0, "Wr1": 1, "br1": 2, "Wr2": 3, "br2": 4,
+               "W1": 5, "b1": 6, "W2": 7, "b2": 8}
+
+
+@dataclass(frozen=True)
+class LayerConfig:
+    """Shape and input recipe of one synthetic workload."""
+    name: str
+    T: int
+    d: int
+    S: int
+    E: int
+    k: int
+    F: int
+    Hr: int = 256
+    dtype: str = "bf16"          # storage type: "bf16" or "f32"
+    act: int = ACT_GELU_TANH
+    capacity: int = 0            # 0 = unlimited
+    init: str = "normal"         # "normal": N(0, 0.02) weights, zero biases
+                                 # "kaiming": He-uniform weights, uniform biases
+    zipf_s: float = 0.0          # > 0: router output bias 1.5*log(Zipf(s) weight)
+    wr2_gain: float = 1.0        # multiplies the std of Wr2 (calibrated-skew variant)
+
+    @property
+    def ds(self) -> int:
+        return self.d // self.S
+
+    @property
+    def N(self) -> int:
+        return self.T * self.S
+
+    @property
+    def R(self) -> int:
+        return self.T * self.S * self.k
+
+    def with_tokens(self, T: int) -> "LayerConfig":
+        cap = self.capacity
+        if cap:
+            cap = capacity_for(T, self.S, self.k, self.E)
+        return replace(self, T=T, capacity=cap)
+
+
+def capacity_for(T: int, S: int, k: int, E: int, factor: float = 1.25) -> int:
+    """Per-expert capacity ceil(factor * T*S*k / E) of the skewed-routing workload."""
+    return int(math.ceil(factor * T * S * k / E))
+
+
+CONFIGS = {
+    # Tiny fp32 layer, all four Linears carry biases, ReLU experts.
+    "cfg0": LayerConfig("cfg0", T=512, d=256, S=4, E=8, k=2, F=256, dtype="f32",
+                        act=ACT_RELU, init="kaiming"),
+    # LM-layer shape (batch 32 x seq 512).
+    "cfg1": LayerConfig("cfg1", T=16384, d=512, S=8, E=16, k=2, F=256),
+    # Wider layer (batch 64 x seq 1024).
+    "cfg2": LayerConfig("cfg2", T=65536, d=1024, S=16, E=32, k=2, F=256),
+    # Skewed routing with a hard capacity and overflow drop.
+    "cfg3": LayerConfig("cfg3", T=32768, d=2048, S=8, E=64, k=1, F=1024,
+                        capacity=capacity_for(32768, 8, 1, 64), zipf_s=1.2),
+    # Same, with the router's output layer scaled so that data, not only the
+    # bias, decides the expert: several experts overflow instead of one.
+    "cfg3b": LayerConfig("cfg3b", T=32768, d=2048, S=8, E=64, k=1, F=1024,
+                         capacity=capacity_for(32768, 8, 1, 64), zipf_s=1.2,
+                         wr2_gain=100.0),
+    # Decode-shaped, weight-bandwidth-bound.
+    "cfg4": LayerConfig("cfg4", T=128, d=4096, S=32, E=64, k=2, F=512),
+    # Same-E token-level MoE comparison (S = 1).
+    "cfg4b": LayerConfig("cfg4b", T=128, d=4096, S=1, E=64, k=2, F=16384),
+}
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest bf16 (ties to even); result stays float32."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32)
+    rounded = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return rounded.view(np.float32)
+
+
+def bf16_bits(x: np.ndarray) -> np.ndarray:
+    """The uint16 bit patterns of float32 values that are already bf16-representable."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    return (x.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+def round_to_storage(x: np.ndarray, dtype: str) -> np.ndarray:
+    if dtype == "bf16":
+        return round_to_bf16(x)
+    if dtype == "f32":
+        return np.ascontiguousarray(x, dtype=np.float32)
+    raise ValueError(f"unknown storage dtype {dtype!r}")
+
+
+def _rng(seed: int, tensor: str) -> np.random.Generator:
+    key = np.array([seed, _TENSOR_IDS[tensor]], dtype=np.uint64)
+    return np.random.Generator(np.random.Philox(key=key))
+
+
+def _normal(seed, tensor, shape, std, dtype):
+    g = _rng(seed, tensor)
+    x = g.standard_normal(size=shape, dtype=np.float32)
+    if std != 1.0:
+        x *= np.float32(std)
+    return round_to_storage(x, dtype)
+
+
+def _uniform(seed, tensor, shape, bound, dtype):
+    g = _rng(seed, tensor)
+    x = g.random(size=shape, dtype=np.float32)
+    x = (x * np.float32(2.0) - np.float32(1.0)) * np.float32(bound)
+    return round_to_storage(x, dtype)
+
+
+def zipf_router_bias(E: int, s: float) -> np.ndarray:
+    """1.5 * log(w_e) with w_e = (e+1)^-s / sum_j (j+1)^-s (float64)."""
+    w = np.arange(1, E + 1, dtype=np.float64) ** (-s)
+    w /= w.sum()
+    return 1.5 * np.log(w)
+
+
+def make_tokens(cfg: LayerConfig, seed: int = 0) -> np.ndarray:
+    """h[T, d] ~ N(0, 1), rounded to the storage dtype."""
+    return _normal(seed, "h", (cfg.T, cfg.d), 1.0, cfg.dtype)
+
+
+def make_weights(cfg: LayerConfig, seed: int = 0) -> dict:
+    """Router and expert weights, nn.Linear layout [out, in] (in contiguous).
+
+    Returns float32 arrays (exact stored values):
+      Wr1[Hr, ds], br1[Hr], Wr2[E, Hr], br2[E],
+      W1[E, F, ds], b1[E, F], W2[E, ds, F], b2[E, ds].
+    """
+    ds, Hr, E, F, dt = cfg.ds, cfg.Hr, cfg.E, cfg.F, cfg.dtype
+    w = {}
+    if cfg.init == "kaiming":
+        def wt(name, shape, fan_in):
+            return _uniform(seed, name, shape, math.sqrt(6.0 / fan_in), dt)
+
+        def bs(name, shape, fan_in):
+            return _uniform(seed, name, shape, 1.0 / math.sqrt(fan_in), dt)
+
+        w["Wr1"] = wt("Wr1", (Hr, ds), ds)
+        w["br1"] = bs("br1", (Hr,), ds)
+        w["Wr2"] = wt("Wr2", (E, Hr), Hr)
+        w["br2"] = bs("br2", (E,), Hr)
+        w["W1"] = wt("W1", (E, F, ds), ds)
+        w["b1"] = bs("b1", (E, F), ds)
+        w["W2"] = wt("W2", (E, ds, F), F)
+        w["b2"] = bs("b2", (E, ds), F)
+    elif cfg.init == "normal":
+        std = 0.02
+        w["Wr1"] = _normal(seed, "Wr1", (Hr, ds), std, dt)
+        w["br1"] = np.zeros((Hr,), dtype=np.float32)
+        w["Wr2"] = _normal(seed, "Wr2", (E, Hr), std * cfg.wr2_gain, dt)
+        w["br2"] = np.zeros((E,), dtype=np.float32)
+        w["W1"] = _normal(seed, "W1", (E, F, ds), std, dt)
+        w["b1"] = np.zeros((E, F), dtype=np.float32)
+        w["W2"] = _normal(seed, "W2", (E, ds, F), std, dt)
+        w["b2"] = np.zeros((E, ds), dtype=np.float32)
+    else:
+        raise ValueError(f"unknown init {cfg.init!r}")
+    if cfg.zipf_s > 0.0:
+        w["br2"] = round_to_storage(zipf_router_bias(E, cfg.zipf_s).astype(np.float32), dt)
+    return w
+
+
+def make_layer_inputs(cfg: LayerConfig, seed: int = 0):
+    """(h, weights) for one workload."""
+    return make_tokens(cfg, seed), make_weights(cfg, seed)

@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Throughput of the SliceMoE layer forward on B200, one JSON line per run.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl ours|reference]
+
+A step is one whole layer forward (route -> dispatch -> expert FFN -> combine) over one batch of
+seeded synthetic tokens.  `value` is tokens/s with the inputs already in HBM; `e2e` is the same
+through slicemoe_forward_host with pinned host buffers (copies inside the timed region).  The
+path does not shard: with --gpus N every rank runs an independent replica on its own batch
+(weak scaling, no data-path collective) and `value` is the sum over ranks / max time.
+
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+L2_BYTES = 126e6
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (kernel -> workload -> bytes); None where no capture exists.
+NCU_TRAFFIC = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------------------------
+# workload arithmetic (algorithmic FLOPs / bytes; the design doc derives them)
+# --------------------------------------------------------------------------------------------
+def layer_work(lc, kept_rows, touched_experts):
+    b = 2 if lc.dtype == "bf16" else 4
+    ds = lc.ds
+    router_flops = 2.0 * lc.N * (ds * lc.Hr + lc.Hr * lc.E)
+    expert_flops = 4.0 * kept_rows * ds * lc.F
+    io_bytes = 2.0 * lc.T * lc.d * b
+    router_w = (lc.Hr * ds + lc.Hr + lc.E * lc.Hr + lc.E) * b
+    expert_w = touched_experts * (2 * ds * lc.F + lc.F + ds) * b
+    return dict(router_flops=router_flops, expert_flops=expert_flops,
+                total_flops=router_flops + expert_flops,
+                compulsory_bytes=io_bytes + router_w + expert_w,
+                # per-stage algorithmic figures of the staged pipeline
+                stage_flops=dict(route=router_flops, expert_ffn=expert_flops),
+                stage_bytes=dict(
+                    route=lc.T * lc.d * b + router_w + lc.R * 8,
+                    dispatch=lc.R * 8 + lc.R * 8 + kept_rows * ds * b * 2,      # idx+p in, dest+perm out, row read+write
+                    expert_ffn=2.0 * kept_rows * ds * b + expert_w,
+                    combine=kept_rows * ds * b + lc.R * 4 + lc.T * lc.d * b))
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True,
+                                     timeout=5).stdout.strip()
+                if out:
+                    self.samples.append([x.strip() for x in out.split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        mhz, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for s in self.samples:
+            try:
+                mhz.append(float(s[0]))
+                mx = float(s[1])
+                for name, v in zip(names, s[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                continue
+        mhz.sort()
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(mhz)}
+
+
+def shard_tokens(T_per_rank, world):
+    """Replicas only: every rank processes its own batch of T tokens (weak scaling)."""
+    return [T_per_rank] * world
+
+
+def aggregate(tokens_per_rank_per_step, steps, seconds_per_rank):
+    """Whole-job tokens/s: all ranks' tokens over the slowest rank's time."""
+    return sum(tokens_per_rank_per_step) * steps / max(seconds_per_rank)
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle leg (also the `--impl reference` arm)
+# --------------------------------------------------------------------------------------------
+def time_oracle(lc, target_s=12.0, steps=1, warmup=0):
+    """Times oracle.forward on the first T_s tokens of the workload; T_s is sized from a short
+    calibration run so that one call takes about target_s seconds."""
+    import oracle
+    from paper_2510_04286_b200 import synth
+    probe_T = min(lc.T, 64)
+    sub = lc.with_tokens(probe_T)
+    h, w = synth.make_layer_inputs(sub)
+    ocfg = oracle.OracleConfig(T=sub.T, d=sub.d, S=sub.S, E=sub.E, k=sub.k, Hr=sub.Hr, F=sub.F,
+                               act=sub.act, capacity=sub.capacity)
+    oracle.forward(ocfg, h, w)
+    t0 = time.perf_counter()
+    oracle.forward(ocfg, h, w)
+    rate = probe_T / max(time.perf_counter() - t0, 1e-6)
+    T_s = int(max(probe_T, min(lc.T, rate * target_s)))
+    sub = lc.with_tokens(T_s)
+    h, w = synth.make_layer_inputs(sub)
+    ocfg = oracle.OracleConfig(T=sub.T, d=sub.d, S=sub.S, E=sub.E, k=sub.k, Hr=sub.Hr, F=sub.F,
+                               act=sub.act, capacity=sub.capacity)
+    for _ in range(warmup):
+        oracle.forward(ocfg, h, w)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.forward(ocfg, h, w)
+    dt = time.perf_counter() - t0
+    return dict(value=T_s * steps / dt, unit="tokens/s", cores=oracle.threads(), kind="oracle",
+                sample=f"first {T_s} of {lc.T} tokens of {lc.name}, {steps} call(s), fp64, OpenMP over rows",
+                seconds=dt, tokens=T_s)
+
+
+def run_reference(args, lc):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    per_call = max(0.5, min(12.0, 120.0 / (steps + warmup)))
+    r = time_oracle(lc, target_s=per_call, steps=steps, warmup=warmup)
+    line = {
+        "impl": "reference", "metric": "SliceMoE layer fwd tokens/s", "value": r["value"],
+        "unit": "tokens/s", "n_gpus": args.gpus, "steps": steps, "warmup": warmup,
+        "ms_per_step": 1e3 * r["seconds"] / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(lc, sets=1),
+        "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": r["value"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(lc, sets):
+    return {"workload": lc.name, "T": lc.T, "d": lc.d, "S": lc.S, "E": lc.E, "k": lc.k, "F": lc.F,
+            "Hr": lc.Hr, "act": "gelu_tanh" if lc.act else "relu", "capacity": lc.capacity,
+            "l2": f"rotating {sets} distinct token/output buffer sets between steps "
+                  f"(larger than the 126 MB L2)" if sets > 1 else "single buffer set"}
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+def run_ours(args, lc):
+    import numpy as np
+    import torch
+    import paper_2510_04286_b200 as sm
+    from paper_2510_04286_b200 import synth, tensors
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = tensors.config_from_synth(lc)
+    tdt = sm.torch_dtype(cfg)
+    b = 2 if lc.dtype == "bf16" else 4
+    set_bytes = 2 * lc.T * lc.d * b
+    sets = int(max(2, min(64, -(-2.2 * L2_BYTES // set_bytes)))) if set_bytes < 2.2 * L2_BYTES else 2
+    # distinct seeded batches: rank r, set s draws seed 1000*r + s
+    w_np = synth.make_weights(lc)
+    w = tensors.weights_to_torch(w_np, lc.dtype)
+    hs = [tensors.to_torch(synth.make_tokens(lc, seed=1000 * rank + s), lc.dtype) for s in range(sets)]
+    outs = [torch.empty((lc.T, lc.d), dtype=tdt, device="cuda") for _ in range(sets)]
+    ws = sm.alloc_workspace(cfg)
+    assigned = torch.empty((lc.E,), dtype=torch.int32, device="cuda")
+    kept = torch.empty((lc.E,), dtype=torch.int32, device="cuda")
+
+    def step(i):
+        sm.slicemoe_forward(cfg, w, hs[i % sets], outs[i % sets], ws, assigned, kept)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    torch.cuda.synchronize()
+    if sm.slicemoe_last_status(ws) != 0:
+        raise RuntimeError(f"device status {sm.slicemoe_last_status(ws)} after warm-up")
+    kept_rows = int(kept.sum().item())
+    touched = int((kept > 0).sum().item())
+
+    # ---- timed region 1: device-resident inputs -------------------------------------------
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    launches0 = sm.slicemoe_launch_count()
+    with ClockSampler(local) as clocks:
+        start.record()
+        for i in range(args.steps):
+            step(i)
+        stop.record()
+        barrier()
+    launches = sm.slicemoe_launch_count() - launches0
+    t_dev = start.elapsed_time(stop) / 1e3
+
+    # ---- timed region 2: host buffers through the C ABI -----------------------------------
+    h_host = [tensors.to_torch(synth.make_tokens(lc, seed=1000 * rank + s), lc.dtype, "cpu", pin=True)
+              for s in range(min(sets, 4))]
+    o_host = [torch.empty_like(x).pin_memory() for x in h_host]
+    for i in range(3):
+        sm.slicemoe_forward_host(cfg, w, h_host[i % len(h_host)], o_host[i % len(h_host)], ws, assigned, kept)
+    barrier()
+    start.record()
+    for i in range(args.steps):
+        sm.slicemoe_forward_host(cfg, w, h_host[i % len(h_host)], o_host[i % len(h_host)], ws, assigned, kept)
+    stop.record()
+    barrier()
+    t_e2e = start.elapsed_time(stop) / 1e3
+
+    # ---- timed region 3: per-stage CUDA events (recorded by the library on its stream) ----
+    ev = [sm.StageEvents() for _ in range(min(args.steps, 64))]
+    barrier()
+    for i in range(len(ev)):
+        sm.slicemoe_forward_profiled(cfg, w, hs[i % sets], outs[i % sets], ws, ev[i], assigned, kept)
+    torch.cuda.synchronize()
+    stage_ms = np.mean([e.stage_ms() for e in ev], axis=0)
+
+    times = torch.tensor([t_dev, t_e2e], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    t_dev, t_e2e = (float(x) for x in times.cpu())
+
+    if rank == 0:
+        peaks, peak_src = load_peaks()
+        work = layer_work(lc, kept_rows, touched)
+        stages = dict(zip(sm.STAGES, (float(x) for x in stage_ms)))
+        dom = max(stages, key=stages.get)
+        if dom in work["stage_flops"]:
+            achieved = work["stage_flops"][dom] / (stages[dom] * 1e-3) / 1e12
+            roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+        else:
+            achieved = work["stage_bytes"][dom] / (stages[dom] * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roof.update(frac=roof["achieved"] / roof["peak"], traffic=NCU_TRAFFIC.get(dom, {}).get(lc.name),
+                    kernel=dom, kernel_ms=stages[dom], peak_source=f"of {peak_src}")
+        t_step = t_dev / args.steps
+        t_tensor = work["total_flops"] / (peaks["bf16_tflops"] * 1e12)
+        t_hbm = work["compulsory_bytes"] / (peaks["hbm_gbs"] * 1e9)
+        line = {
+            "metric": "SliceMoE layer fwd tokens/s", "value": aggregate(shard_tokens(lc.T, world), args.steps, [t_dev]),
+            "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": 1e3 * t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": lc.dtype, "data": "synthetic", "config": workload_config(lc, sets),
+            "routed_slices_per_s": world * lc.R / t_step,
+            "e2e": {"value": world * lc.T * args.steps / t_e2e, "unit": "tokens/s",
+                    "h2d_bytes_per_step": lc.T * lc.d * b, "d2h_bytes_per_step": lc.T * lc.d * b},
+            "gpu_launches": int(launches),
+            "clocks": clocks.summary(),
+            "roofline": roof,
+            "stage_ms": stages,
+            "layer_roofline": {"t_tensor_us": 1e6 * t_tensor, "t_hbm_us": 1e6 * t_hbm,
+                               "bound": "tensor" if t_tensor >= t_hbm else "hbm",
+                               "frac": max(t_tensor, t_hbm) / t_step, "kept_rows": kept_rows,
+                               "touched_experts": touched, "peak_source": f"of {peak_src}"},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            r = time_oracle(lc)
+            line["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="cfg1")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2510_04286_b200 import synth
+    lc = synth.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, lc)
+    else:
+        run_ours(args, lc)
+
+
+if __name__ == "__main__":
+    main()

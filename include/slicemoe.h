@@ -1,0 +1,204 @@
+/*
+ * slicemoe.h -- C ABI of the B200 (sm_100a) SliceMoE layer forward.
+ *
+ * The layer (paper Section 3): a token vector h in R^d is cut into S contiguous
+ * slices of ds = d/S elements.  A router MLP shared by all slices
+ * (Linear ds->H_r, ReLU, Linear H_r->E) scores each slice, a softmax turns the
+ * scores into probabilities and the k most probable experts are chosen per
+ * slice (Section 3.1).  Each chosen expert e_j runs its two-layer FFN on the
+ * slice scaled by its probability (Eq. 1); slices bound for the same expert
+ * are stacked so that an expert works on one contiguous batch (Section 3.4);
+ * the k outputs of a slice are summed and written at the slice's own columns
+ * of h' (Section 3.1).
+ *
+ * Rows.  With h row-major [T, d], slice s of token t is the contiguous run of
+ * ds elements starting at (t*S + s)*ds.  The library therefore works on the
+ * matrix X[N, ds], N = T*S, which is the same memory as h; row n = t*S + s.
+ * "Pair" (n, j) is the j-th chosen expert of row n, flat index n*k + j;
+ * R = N*k pairs.
+ *
+ * Conventions for every call below
+ *   - All pointers are CUDA DEVICE pointers unless the comment says HOST.
+ *     `cfg` and `w` themselves are HOST structs (read during the call).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls only enqueue work on it: no allocation, no host
+ *     synchronisation, unless stated.
+ *   - The caller owns every buffer, including the workspace `ws`
+ *     (slicemoe_workspace_bytes(), 256-byte aligned).  The library keeps no
+ *     device memory of its own.
+ *   - Tensors are dense row-major, 16-byte aligned, of cfg->dtype
+ *     (bf16 or fp32) unless a type is written.  Weights use the nn.Linear
+ *     layout [out, in] with `in` contiguous.  Bias pointers may be NULL (= 0).
+ *   - Return value: 0 (SLICEMOE_OK) or a slicemoe_status error; on an error
+ *     found by argument checking nothing has been launched.  Nothing throws.
+ *   - Routing arithmetic (logits, softmax, top-k) is fp32 in both dtypes; with
+ *     bf16 storage the GEMMs take bf16 operands and accumulate in fp32.
+ *   - Ties between equal router scores go to the lower expert id; the k
+ *     experts of a row are listed most probable first.
+ */
+#ifndef SLICEMOE_H_
+#define SLICEMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SLICEMOE_OK = 0,
+    SLICEMOE_ERR_NULL = 1,           /* a required pointer is NULL */
+    SLICEMOE_ERR_SHAPE = 2,          /* d % S != 0, k > E, k < 1, E < 1, T < 0, sizes overflow int32 ... */
+    SLICEMOE_ERR_UNSUPPORTED = 3,    /* shape, dtype or activation outside the built set */
+    SLICEMOE_ERR_ALIGN = 4,          /* a tensor pointer is not 16-byte aligned */
+    SLICEMOE_ERR_WORKSPACE = 5,      /* ws is NULL or smaller than slicemoe_workspace_bytes() */
+    SLICEMOE_ERR_ALIAS = 6,          /* h_out overlaps h */
+    SLICEMOE_ERR_CUDA = 7,           /* a CUDA runtime call failed (see slicemoe_last_cuda_error) */
+    SLICEMOE_ERR_DEVICE_TIMEOUT = 8, /* a bounded wait inside a kernel ran out (slicemoe_last_status) */
+    SLICEMOE_ERR_NO_DEVICE = 9       /* no usable sm_100 device */
+} slicemoe_status;
+
+typedef enum { SLICEMOE_BF16 = 0, SLICEMOE_F32 = 1 } slicemoe_dtype;
+typedef enum { SLICEMOE_ACT_RELU = 0, SLICEMOE_ACT_GELU_TANH = 1 } slicemoe_act;
+
+/* Shape of one layer (paper notation).  Limits of the built set:
+ * ds = d/S a multiple of 8 (bf16) or 4 (fp32); 1 <= k <= 8; E <= 256;
+ * T*S*k < 2^31. */
+typedef struct {
+    int32_t T;        /* tokens in the batch */
+    int32_t d;        /* hidden size */
+    int32_t S;        /* slices per token (Section 3) */
+    int32_t E;        /* experts */
+    int32_t k;        /* experts per slice (Section 3.1) */
+    int32_t Hr;       /* router hidden width (256 in the paper, Appendix A) */
+    int32_t F;        /* expert FFN hidden width */
+    int32_t dtype;    /* slicemoe_dtype: storage type of h, h', weights and stacked rows */
+    int32_t act;      /* slicemoe_act: activation between the two expert layers */
+    int64_t capacity; /* hard per-expert limit on kept pairs; 0 = unlimited */
+} slicemoe_config;
+
+/* Caller-owned weights, dtype = cfg->dtype. */
+typedef struct {
+    const void *Wr1; /* [Hr, ds]   router layer 1 (Section 3.1) */
+    const void *br1; /* [Hr]       or NULL */
+    const void *Wr2; /* [E, Hr]    router layer 2 */
+    const void *br2; /* [E]        or NULL */
+    const void *W1;  /* [E, F, ds] expert layer 1 */
+    const void *b1;  /* [E, F]     or NULL */
+    const void *W2;  /* [E, ds, F] expert layer 2 */
+    const void *b2;  /* [E, ds]    or NULL */
+} slicemoe_weights;
+
+/* Bytes of workspace that any call below needs for `cfg` (the maximum over the
+ * calls, slicemoe_forward_host's device staging included).  `bytes` is a HOST
+ * out-pointer. */
+int slicemoe_workspace_bytes(const slicemoe_config *cfg, size_t *bytes);
+
+/*
+ * Section 3.1, router: for every row n of X[N, ds]
+ *   a = relu(Wr1 x + br1),  g = Wr2 a + br2,  p = softmax(g),
+ *   topk_idx[n, :] = the k experts with the largest p (ties: lower id first),
+ *   topk_p[n, :]   = their probabilities, descending.
+ * out: topk_idx int32 [N, k]; topk_p float [N, k]; assigned int32 [E] =
+ *      number of pairs that chose each expert (the counts of Section 3.2);
+ *      probs_opt float [N, E] (NULL to skip).
+ */
+int slicemoe_route(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
+                   int32_t *topk_idx, float *topk_p, int32_t *assigned, float *probs_opt,
+                   void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Eq. 1 and Section 3.4, dispatch: group the pairs by expert and stack their
+ * probability-weighted rows.  Inside an expert, pairs keep ascending (n, j)
+ * order (a stable counting sort, so the result is unique and deterministic).
+ * With cfg->capacity = C > 0 a pair whose rank inside its expert is >= C is
+ * dropped.
+ * in : h [T, d]; topk_idx int32 [N, k]; topk_p float [N, k]
+ * out: kept int32 [E]      = min(assigned, C) (= assigned when C = 0);
+ *      offsets int32 [E+1] = exclusive scan of kept;
+ *      dest int32 [N, k]   = offsets[e] + rank, or -1 if dropped;
+ *      perm int32 [R]      = perm[dest(n, j)] = n*k + j (first offsets[E] entries are written);
+ *      xperm [R, ds]       = xperm[dest(n, j), :] = dtype(topk_p[n, j] * X[n, :])
+ *                            (first offsets[E] rows are written; NULL to skip).
+ * An expert id outside [0, E) in topk_idx is treated as a dropped pair.
+ */
+int slicemoe_dispatch(const slicemoe_config *cfg, const void *h, const int32_t *topk_idx,
+                      const float *topk_p, int32_t *kept, int32_t *offsets, int32_t *dest,
+                      int32_t *perm, void *xperm, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Section 3.1 / 3.4, experts: for every expert e and every stacked row r in
+ * [offsets[e], offsets[e+1])
+ *   yperm[r, :] = W2_e act(W1_e xperm[r, :] + b1_e) + b2_e
+ * The row ranges are read from `offsets` on the device (no host sync); rows at
+ * or beyond offsets[E] are not touched.
+ */
+int slicemoe_expert_ffn(const slicemoe_config *cfg, const slicemoe_weights *w, const void *xperm,
+                        const int32_t *offsets, void *yperm, void *ws, size_t ws_bytes,
+                        void *stream);
+
+/*
+ * Section 3.1, combine: Y[n, :] = sum over j with dest[n, j] >= 0 of
+ * yperm[dest[n, j], :], added in j order in fp32 and rounded once; a row whose
+ * pairs were all dropped becomes zero.  h_out [T, d] is the same memory as
+ * Y[N, ds], so every slice lands at its own columns of its token.
+ */
+int slicemoe_combine(const slicemoe_config *cfg, const void *yperm, const int32_t *dest,
+                     void *h_out, void *stream);
+
+/*
+ * The whole layer forward, h [T, d] -> h_out [T, d], equal to
+ * route -> dispatch -> expert_ffn -> combine up to rounding, and bit-equal on
+ * topk_idx / assigned / kept.  h_out must not overlap h.
+ * Optional outputs (NULL to skip): assigned_opt int32 [E], kept_opt int32 [E],
+ * topk_idx_opt int32 [N, k], topk_p_opt float [N, k].
+ */
+int slicemoe_forward(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
+                     void *h_out, int32_t *assigned_opt, int32_t *kept_opt,
+                     int32_t *topk_idx_opt, float *topk_p_opt, void *ws, size_t ws_bytes,
+                     void *stream);
+
+/*
+ * slicemoe_forward with HOST tokens: h_host and h_out_host are HOST buffers
+ * (pinned memory makes the copies asynchronous).  Enqueues the host->device
+ * copy of h into the workspace, the forward, and the device->host copy of h'.
+ * Weights and the optional outputs stay DEVICE pointers.  The caller
+ * synchronises the stream before reading h_out_host.
+ */
+int slicemoe_forward_host(const slicemoe_config *cfg, const slicemoe_weights *w,
+                          const void *h_host, void *h_out_host, int32_t *assigned_opt,
+                          int32_t *kept_opt, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * slicemoe_forward that also records CUDA events at its stage boundaries, for
+ * measurement.  `events` is a HOST array of SLICEMOE_N_STAGE_EVENTS
+ * cudaEvent_t handles (as void*) created by slicemoe_event_create(): event i is
+ * recorded before stage i and event i+1 after it, stages being
+ * 0 route, 1 dispatch, 2 expert FFN, 3 combine.
+ */
+#define SLICEMOE_N_STAGE_EVENTS 5
+int slicemoe_forward_profiled(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
+                              void *h_out, int32_t *assigned_opt, int32_t *kept_opt,
+                              int32_t *topk_idx_opt, float *topk_p_opt, void *ws, size_t ws_bytes,
+                              void *stream, void *const *events);
+int slicemoe_event_create(void **event /* HOST out */);
+int slicemoe_event_destroy(void *event);
+/* Milliseconds between two recorded events; synchronises on `stop`.  `ms` is a HOST out-pointer. */
+int slicemoe_event_elapsed_ms(void *start, void *stop, float *ms);
+
+/* Device status word of the last kernels that used `ws` (0 = fine, else a
+ * slicemoe_status such as SLICEMOE_ERR_DEVICE_TIMEOUT).  Synchronises `stream`. */
+int slicemoe_last_status(const void *ws, void *stream);
+
+/* Number of kernels this library has launched in this process so far (HOST counter). */
+int64_t slicemoe_launch_count(void);
+
+/* Text of the last CUDA runtime error seen by this library on this thread (HOST string). */
+const char *slicemoe_last_cuda_error(void);
+const char *slicemoe_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLICEMOE_H_ */

@@ -1,0 +1,349 @@
+// C ABI of the SliceMoE layer forward: argument checking, workspace layout and the sequencing of
+// the stage kernels on the caller's stream.  No step of the layer is computed here.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace slicemoe {
+
+static std::atomic<long long> g_launches{0};
+static thread_local char g_cuda_error[256] = "";
+
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void note_cuda_error(cudaError_t e) {
+    std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    (void)cudaGetLastError();  // clear the sticky-less error state
+}
+
+static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+Workspace workspace_layout(const Dims& D) {
+    Workspace W;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + (bytes ? bytes : 1)); return at; };
+    const size_t R = (size_t)D.R, E = (size_t)D.E, b = elem_bytes(D);
+    W.status = take(sizeof(int32_t) * 64);
+    W.topk_idx = take(sizeof(int32_t) * R);
+    W.topk_p = take(sizeof(float) * R);
+    W.assigned = take(sizeof(int32_t) * E);
+    W.kept = take(sizeof(int32_t) * E);
+    W.offsets = take(sizeof(int32_t) * (E + 1));
+    W.dest = take(sizeof(int32_t) * R);
+    W.perm = take(sizeof(int32_t) * R);
+    W.gate = take(sizeof(float) * R);
+    W.chunk_hist = take(sizeof(int32_t) * (size_t)num_chunks(D) * E);
+    W.tiles = take(sizeof(int32_t) * (4 + 2 * (size_t)max_tiles(D)));
+    W.xperm = take(b * R * D.ds);
+    W.yperm = take(b * R * D.ds);
+    W.h_dev = take(b * (size_t)D.T * D.d);
+    W.hout_dev = take(b * (size_t)D.T * D.d);
+    W.total = off;
+    return W;
+}
+
+static int make_dims(const slicemoe_config* c, Dims& D) {
+    if (!c) return SLICEMOE_ERR_NULL;
+    if (c->T < 0 || c->d < 1 || c->S < 1 || c->E < 1 || c->k < 1 || c->Hr < 1 || c->F < 1 || c->capacity < 0)
+        return SLICEMOE_ERR_SHAPE;
+    if (c->d % c->S != 0 || c->k > c->E) return SLICEMOE_ERR_SHAPE;
+    if (c->dtype != SLICEMOE_BF16 && c->dtype != SLICEMOE_F32) return SLICEMOE_ERR_UNSUPPORTED;
+    if (c->act != SLICEMOE_ACT_RELU && c->act != SLICEMOE_ACT_GELU_TANH) return SLICEMOE_ERR_UNSUPPORTED;
+    const long long N = (long long)c->T * c->S, R = N * c->k;
+    const long long lim = 0x7fffffffLL;
+    if (R >= lim || (long long)c->T * c->d >= lim) return SLICEMOE_ERR_SHAPE;
+    if ((long long)c->E * c->F * (c->d / c->S) >= lim) return SLICEMOE_ERR_SHAPE;
+    const int V = c->dtype == SLICEMOE_BF16 ? 8 : 4;
+    const int ds = c->d / c->S;
+    if (ds % V || c->Hr % V || c->F % V) return SLICEMOE_ERR_UNSUPPORTED;
+    if (c->k > 8 || c->E > 256) return SLICEMOE_ERR_UNSUPPORTED;
+    D.T = c->T; D.d = c->d; D.S = c->S; D.E = c->E; D.k = c->k; D.Hr = c->Hr; D.F = c->F;
+    D.ds = ds; D.N = (int)N; D.R = (int)R; D.dtype = c->dtype; D.act = c->act;
+    D.capacity = (int)(c->capacity > R ? R : c->capacity);
+    if (c->capacity > 0 && D.capacity == 0) D.capacity = 1;  // R == 0: keep "limited" semantics harmless
+    return SLICEMOE_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_weights(const slicemoe_weights* w, bool router, bool experts) {
+    if (!w) return SLICEMOE_ERR_NULL;
+    if (router) {
+        if (!w->Wr1 || !w->Wr2) return SLICEMOE_ERR_NULL;
+        if (!aligned16(w->Wr1) || !aligned16(w->Wr2) || !aligned16(w->br1) || !aligned16(w->br2))
+            return SLICEMOE_ERR_ALIGN;
+    }
+    if (experts) {
+        if (!w->W1 || !w->W2) return SLICEMOE_ERR_NULL;
+        if (!aligned16(w->W1) || !aligned16(w->W2) || !aligned16(w->b1) || !aligned16(w->b2))
+            return SLICEMOE_ERR_ALIGN;
+    }
+    return SLICEMOE_OK;
+}
+
+static int check_device() {
+    static std::atomic<int> state{0};  // 0 unknown, 1 ok, 2 bad
+    int s = state.load();
+    if (s == 0) {
+        int dev = 0, major = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            s = 2;
+        } else {
+            s = (major == 10) ? 1 : 2;
+        }
+        state.store(s);
+    }
+    return s == 1 ? SLICEMOE_OK : SLICEMOE_ERR_NO_DEVICE;
+}
+
+static int check_ws(const Dims& D, const void* ws, size_t ws_bytes, Workspace& W) {
+    W = workspace_layout(D);
+    if (!ws || ws_bytes < W.total) return SLICEMOE_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return SLICEMOE_ERR_ALIGN;
+    return SLICEMOE_OK;
+}
+
+template <typename U> static U* at(void* ws, size_t off) {
+    return reinterpret_cast<U*>(static_cast<char*>(ws) + off);
+}
+
+// Clears the device status word that kernels with bounded waits report into.
+static int reset_status(void* ws, const Workspace& W, cudaStream_t st) {
+    SLICEMOE_CUDA_TRY(cudaMemsetAsync(at<char>(ws, W.status), 0, sizeof(int32_t) * 64, st));
+    return SLICEMOE_OK;
+}
+
+static int route_any(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* idx, float* p,
+                     int32_t* assigned, float* probs, cudaStream_t st) {
+    return launch_route_simt(D, w, h, idx, p, assigned, probs, st);
+}
+
+static int ffn_any(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets,
+                   void* yperm, cudaStream_t st) {
+    return launch_ffn_simt(D, w, xperm, offsets, yperm, st);
+}
+
+static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out,
+                        int32_t* assigned_opt, int32_t* kept_opt, int32_t* idx_opt, float* p_opt,
+                        void* ws, const Workspace& W, cudaStream_t st, void* const* events) {
+    int32_t* idx = idx_opt ? idx_opt : at<int32_t>(ws, W.topk_idx);
+    float* p = p_opt ? p_opt : at<float>(ws, W.topk_p);
+    int32_t* assigned = assigned_opt ? assigned_opt : at<int32_t>(ws, W.assigned);
+    int32_t* kept = kept_opt ? kept_opt : at<int32_t>(ws, W.kept);
+    int32_t* offsets = at<int32_t>(ws, W.offsets);
+    int32_t* dest = at<int32_t>(ws, W.dest);
+    int32_t* perm = at<int32_t>(ws, W.perm);
+    void* xperm = at<char>(ws, W.xperm);
+    void* yperm = at<char>(ws, W.yperm);
+    auto mark = [&](int i) -> int {
+        if (events) SLICEMOE_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st));
+        return SLICEMOE_OK;
+    };
+    int rc;
+    if ((rc = reset_status(ws, W, st))) return rc;
+    if ((rc = mark(0))) return rc;
+    if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, st))) return rc;
+    if ((rc = mark(1))) return rc;
+    if ((rc = launch_dispatch(D, h, idx, p, kept, offsets, dest, perm, xperm, nullptr,
+                              at<int32_t>(ws, W.chunk_hist), st))) return rc;
+    if ((rc = mark(2))) return rc;
+    if ((rc = ffn_any(D, w, xperm, offsets, yperm, st))) return rc;
+    if ((rc = mark(3))) return rc;
+    if ((rc = launch_combine(D, yperm, dest, h_out, st))) return rc;
+    return mark(4);
+}
+
+static bool overlaps(const void* a, const void* b, size_t bytes) {
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + bytes && y < x + bytes;
+}
+
+}  // namespace slicemoe
+
+using namespace slicemoe;
+
+extern "C" {
+
+int slicemoe_workspace_bytes(const slicemoe_config* cfg, size_t* bytes) {
+    if (!bytes) return SLICEMOE_ERR_NULL;
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    *bytes = workspace_layout(D).total;
+    return SLICEMOE_OK;
+}
+
+int slicemoe_route(const slicemoe_config* cfg, const slicemoe_weights* w, const void* h,
+                   int32_t* topk_idx, float* topk_p, int32_t* assigned, float* probs_opt, void* ws,
+                   size_t ws_bytes, void* stream) {
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    if ((rc = check_weights(w, true, false))) return rc;
+    if (!h || !topk_idx || !topk_p || !assigned) return SLICEMOE_ERR_NULL;
+    if (!aligned16(h) || !aligned16(topk_idx) || !aligned16(topk_p) || !aligned16(probs_opt))
+        return SLICEMOE_ERR_ALIGN;
+    Workspace W;
+    if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
+    if ((rc = check_device())) return rc;
+    if ((rc = reset_status(ws, W, static_cast<cudaStream_t>(stream)))) return rc;
+    return route_any(D, *w, h, topk_idx, topk_p, assigned, probs_opt, static_cast<cudaStream_t>(stream));
+}
+
+int slicemoe_dispatch(const slicemoe_config* cfg, const void* h, const int32_t* topk_idx,
+                      const float* topk_p, int32_t* kept, int32_t* offsets, int32_t* dest,
+                      int32_t* perm, void* xperm, void* ws, size_t ws_bytes, void* stream) {
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    if (!topk_idx || !topk_p || !kept || !offsets || !dest || !perm) return SLICEMOE_ERR_NULL;
+    if (xperm && !h) return SLICEMOE_ERR_NULL;
+    if (!aligned16(h) || !aligned16(xperm)) return SLICEMOE_ERR_ALIGN;
+    Workspace W;
+    if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
+    if ((rc = check_device())) return rc;
+    if ((rc = reset_status(ws, W, static_cast<cudaStream_t>(stream)))) return rc;
+    return launch_dispatch(D, h, topk_idx, topk_p, kept, offsets, dest, perm, xperm, nullptr,
+                           at<int32_t>(ws, W.chunk_hist), static_cast<cudaStream_t>(stream));
+}
+
+int slicemoe_expert_ffn(const slicemoe_config* cfg, const slicemoe_weights* w, const void* xperm,
+                        const int32_t* offsets, void* yperm, void* ws, size_t ws_bytes, void* stream) {
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    if ((rc = check_weights(w, false, true))) return rc;
+    if (!xperm || !offsets || !yperm) return SLICEMOE_ERR_NULL;
+    if (!aligned16(xperm) || !aligned16(yperm)) return SLICEMOE_ERR_ALIGN;
+    Workspace W;
+    if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
+    if ((rc = check_device())) return rc;
+    if ((rc = reset_status(ws, W, static_cast<cudaStream_t>(stream)))) return rc;
+    return ffn_any(D, *w, xperm, offsets, yperm, static_cast<cudaStream_t>(stream));
+}
+
+int slicemoe_combine(const slicemoe_config* cfg, const void* yperm, const int32_t* dest, void* h_out,
+                     void* stream) {
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    if (!yperm || !dest || !h_out) return SLICEMOE_ERR_NULL;
+    if (!aligned16(yperm) || !aligned16(h_out)) return SLICEMOE_ERR_ALIGN;
+    if ((rc = check_device())) return rc;
+    return launch_combine(D, yperm, dest, h_out, static_cast<cudaStream_t>(stream));
+}
+
+static int forward_checked(const slicemoe_config* cfg, const slicemoe_weights* w, const void* h,
+                           void* h_out, int32_t* assigned_opt, int32_t* kept_opt, int32_t* topk_idx_opt,
+                           float* topk_p_opt, void* ws, size_t ws_bytes, void* stream,
+                           void* const* events) {
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    if ((rc = check_weights(w, true, true))) return rc;
+    if (!h || !h_out) return SLICEMOE_ERR_NULL;
+    if (!aligned16(h) || !aligned16(h_out) || !aligned16(topk_idx_opt) || !aligned16(topk_p_opt))
+        return SLICEMOE_ERR_ALIGN;
+    if (overlaps(h, h_out, elem_bytes(D) * (size_t)D.T * D.d)) return SLICEMOE_ERR_ALIAS;
+    Workspace W;
+    if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
+    if ((rc = check_device())) return rc;
+    return forward_impl(D, *w, h, h_out, assigned_opt, kept_opt, topk_idx_opt, topk_p_opt, ws, W,
+                        static_cast<cudaStream_t>(stream), events);
+}
+
+int slicemoe_forward(const slicemoe_config* cfg, const slicemoe_weights* w, const void* h, void* h_out,
+                     int32_t* assigned_opt, int32_t* kept_opt, int32_t* topk_idx_opt, float* topk_p_opt,
+                     void* ws, size_t ws_bytes, void* stream) {
+    return forward_checked(cfg, w, h, h_out, assigned_opt, kept_opt, topk_idx_opt, topk_p_opt, ws,
+                           ws_bytes, stream, nullptr);
+}
+
+int slicemoe_forward_profiled(const slicemoe_config* cfg, const slicemoe_weights* w, const void* h,
+                              void* h_out, int32_t* assigned_opt, int32_t* kept_opt,
+                              int32_t* topk_idx_opt, float* topk_p_opt, void* ws, size_t ws_bytes,
+                              void* stream, void* const* events) {
+    if (!events) return SLICEMOE_ERR_NULL;
+    for (int i = 0; i < SLICEMOE_N_STAGE_EVENTS; ++i)
+        if (!events[i]) return SLICEMOE_ERR_NULL;
+    return forward_checked(cfg, w, h, h_out, assigned_opt, kept_opt, topk_idx_opt, topk_p_opt, ws,
+                           ws_bytes, stream, events);
+}
+
+int slicemoe_forward_host(const slicemoe_config* cfg, const slicemoe_weights* w, const void* h_host,
+                          void* h_out_host, int32_t* assigned_opt, int32_t* kept_opt, void* ws,
+                          size_t ws_bytes, void* stream) {
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    if ((rc = check_weights(w, true, true))) return rc;
+    if (!h_host || !h_out_host) return SLICEMOE_ERR_NULL;
+    Workspace W;
+    if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
+    if ((rc = check_device())) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = elem_bytes(D) * (size_t)D.T * D.d;
+    void* h_dev = at<char>(ws, W.h_dev);
+    void* hout_dev = at<char>(ws, W.hout_dev);
+    if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_dev, h_host, bytes, cudaMemcpyHostToDevice, st));
+    if ((rc = forward_impl(D, *w, h_dev, hout_dev, assigned_opt, kept_opt, nullptr, nullptr, ws, W, st,
+                           nullptr)))
+        return rc;
+    if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_out_host, hout_dev, bytes, cudaMemcpyDeviceToHost, st));
+    return SLICEMOE_OK;
+}
+
+int slicemoe_event_create(void** event) {
+    if (!event) return SLICEMOE_ERR_NULL;
+    cudaEvent_t ev;
+    SLICEMOE_CUDA_TRY(cudaEventCreate(&ev));
+    *event = ev;
+    return SLICEMOE_OK;
+}
+
+int slicemoe_event_destroy(void* event) {
+    if (!event) return SLICEMOE_ERR_NULL;
+    SLICEMOE_CUDA_TRY(cudaEventDestroy(static_cast<cudaEvent_t>(event)));
+    return SLICEMOE_OK;
+}
+
+int slicemoe_event_elapsed_ms(void* start, void* stop, float* ms) {
+    if (!start || !stop || !ms) return SLICEMOE_ERR_NULL;
+    SLICEMOE_CUDA_TRY(cudaEventSynchronize(static_cast<cudaEvent_t>(stop)));
+    SLICEMOE_CUDA_TRY(cudaEventElapsedTime(ms, static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop)));
+    return SLICEMOE_OK;
+}
+
+int slicemoe_last_status(const void* ws, void* stream) {
+    if (!ws) return SLICEMOE_ERR_NULL;
+    int32_t word = 0;
+    SLICEMOE_CUDA_TRY(cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost,
+                                      static_cast<cudaStream_t>(stream)));
+    SLICEMOE_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    return word;
+}
+
+int64_t slicemoe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* slicemoe_last_cuda_error(void) { return g_cuda_error; }
+
+const char* slicemoe_status_string(int status) {
+    switch (status) {
+        case SLICEMOE_OK: return "ok";
+        case SLICEMOE_ERR_NULL: return "a required pointer is NULL";
+        case SLICEMOE_ERR_SHAPE: return "inconsistent shape";
+        case SLICEMOE_ERR_UNSUPPORTED: return "shape, dtype or activation outside the built set";
+        case SLICEMOE_ERR_ALIGN: return "a pointer is not aligned as required";
+        case SLICEMOE_ERR_WORKSPACE: return "workspace missing or too small";
+        case SLICEMOE_ERR_ALIAS: return "h_out overlaps h";
+        case SLICEMOE_ERR_CUDA: return "a CUDA runtime call failed";
+        case SLICEMOE_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case SLICEMOE_ERR_NO_DEVICE: return "no usable sm_100 device";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

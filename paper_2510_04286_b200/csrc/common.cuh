@@ -1,0 +1,142 @@
+// Shared declarations of the SliceMoE CUDA library (internal; the public ABI is include/slicemoe.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "slicemoe.h"
+
+namespace slicemoe {
+
+typedef __nv_bfloat16 bf16;
+
+// Derived sizes of one layer call (paper notation; rows are slices, pairs are (row, j)).
+struct Dims {
+    int T, d, S, E, k, Hr, F;
+    int ds;   // slice width d/S
+    int N;    // rows  = T*S
+    int R;    // pairs = N*k
+    int dtype, act;
+    int capacity;  // 0 = unlimited; clamped to R
+};
+
+// Pairs handled by one dispatch chunk (one CTA of the histogram / scatter kernels).
+constexpr int kDispatchChunk = 2048;
+// Rows per CTA tile of the tensor-core kernels.
+constexpr int kTileM = 128;
+
+// Sub-buffers of the caller's workspace (byte offsets, each 256-byte aligned).
+struct Workspace {
+    size_t status;      // int32[64]: [0] device status word
+    size_t topk_idx;    // int32[R]
+    size_t topk_p;      // float[R]
+    size_t assigned;    // int32[E]
+    size_t kept;        // int32[E]
+    size_t offsets;     // int32[E+1]
+    size_t dest;        // int32[R]
+    size_t perm;        // int32[R]
+    size_t gate;        // float[R]   gate value of each stacked row (fused forward)
+    size_t chunk_hist;  // int32[nchunks*E]
+    size_t tiles;       // int32[4 + 2*max_tiles]  tile list of the grouped expert kernel
+    size_t xperm;       // dtype[R*ds]
+    size_t yperm;       // dtype[R*ds]
+    size_t h_dev;       // dtype[T*d]  staging of slicemoe_forward_host
+    size_t hout_dev;    // dtype[T*d]
+    size_t total;
+};
+
+Workspace workspace_layout(const Dims& D);
+inline int num_chunks(const Dims& D) { return (D.R + kDispatchChunk - 1) / kDispatchChunk; }
+inline int max_tiles(const Dims& D) { return (D.R + kTileM - 1) / kTileM + D.E; }
+inline size_t elem_bytes(const Dims& D) { return D.dtype == SLICEMOE_BF16 ? 2 : 4; }
+
+void count_launches(int n);
+void note_cuda_error(cudaError_t e);
+
+#define SLICEMOE_CUDA_TRY(expr)                          \
+    do {                                                 \
+        cudaError_t _e = (expr);                         \
+        if (_e != cudaSuccess) {                         \
+            ::slicemoe::note_cuda_error(_e);             \
+            return SLICEMOE_ERR_CUDA;                    \
+        }                                                \
+    } while (0)
+
+// Checks the launch that was just enqueued.
+#define SLICEMOE_LAUNCH_CHECK(nlaunches)                 \
+    do {                                                 \
+        ::slicemoe::count_launches(nlaunches);           \
+        SLICEMOE_CUDA_TRY(cudaGetLastError());           \
+    } while (0)
+
+// ---- per-stage launchers (each returns a slicemoe_status) ---------------------------------
+
+// Router on CUDA cores, fp32 arithmetic in both storage types.
+int launch_route_simt(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx,
+                      float* topk_p, int32_t* assigned, float* probs_opt, cudaStream_t st);
+
+// Stable counting sort of the pairs by expert + optional row gather.
+// xperm may be NULL (no gather); gate_opt (float[R], gate of each stacked row) may be NULL.
+int launch_dispatch(const Dims& D, const void* h, const int32_t* topk_idx, const float* topk_p,
+                    int32_t* kept, int32_t* offsets, int32_t* dest, int32_t* perm, void* xperm,
+                    float* gate_opt, int32_t* chunk_hist, cudaStream_t st);
+
+// Grouped expert FFN on CUDA cores.
+int launch_ffn_simt(const Dims& D, const slicemoe_weights& w, const void* xperm,
+                    const int32_t* offsets, void* yperm, cudaStream_t st);
+
+int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
+                   cudaStream_t st);
+
+// ---- storage-type helpers ---------------------------------------------------------------------
+
+template <typename T> struct Vec;  // 16-byte vector of T
+template <> struct Vec<float> { static constexpr int n = 4; };
+template <> struct Vec<bf16> { static constexpr int n = 8; };
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// Unpacks one 16-byte vector into Vec<T>::n floats.
+template <typename T> __device__ __forceinline__ void unpack16(const uint4& raw, float* out);
+template <> __device__ __forceinline__ void unpack16<float>(const uint4& raw, float* out) {
+    out[0] = __uint_as_float(raw.x); out[1] = __uint_as_float(raw.y);
+    out[2] = __uint_as_float(raw.z); out[3] = __uint_as_float(raw.w);
+}
+template <> __device__ __forceinline__ void unpack16<bf16>(const uint4& raw, float* out) {
+    const uint32_t u[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        out[2 * i] = __uint_as_float(u[i] << 16);
+        out[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+    }
+}
+template <typename T> __device__ __forceinline__ uint4 pack16(const float* in);
+template <> __device__ __forceinline__ uint4 pack16<float>(const float* in) {
+    return make_uint4(__float_as_uint(in[0]), __float_as_uint(in[1]), __float_as_uint(in[2]),
+                      __float_as_uint(in[3]));
+}
+template <> __device__ __forceinline__ uint4 pack16<bf16>(const float* in) {
+    uint32_t u[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 v = __floats2bfloat162_rn(in[2 * i], in[2 * i + 1]);
+        u[i] = *reinterpret_cast<uint32_t*>(&v);
+    }
+    return make_uint4(u[0], u[1], u[2], u[3]);
+}
+
+// GELU in its tanh form, fp32.
+__device__ __forceinline__ float gelu_tanh_f32(float z) {
+    const float c = 0.7978845608028654f;
+    return 0.5f * z * (1.0f + tanhf(c * (z + 0.044715f * z * z * z)));
+}
+__device__ __forceinline__ float apply_act(float z, int act) {
+    return act == SLICEMOE_ACT_RELU ? fmaxf(z, 0.0f) : gelu_tanh_f32(z);
+}
+
+}  // namespace slicemoe

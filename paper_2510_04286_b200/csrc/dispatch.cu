@@ -1,0 +1,188 @@
+// Dispatch of Section 3.4 / Eq. 1: a stable counting sort of the (row, j) pairs by expert, with
+// the optional hard capacity, followed by the gather of the probability-weighted rows into
+// contiguous per-expert tiles.  Three kernels, no host synchronisation, no atomics on the
+// positions (ranks come from prefix sums, so the order inside an expert is ascending (n, j) and
+// the result is the same on every run).
+//
+//   1. histogram : per chunk of kDispatchChunk pairs, how many go to each expert
+//   2. scan      : per expert, exclusive prefix over chunks; kept = min(total, C); offsets
+//   3. scatter   : per chunk, the stable rank of each pair -> dest / perm, then a coalesced
+//                  16-byte-vector copy of p * X[n, :] to its destination row
+#include "common.cuh"
+
+namespace slicemoe {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kPairsPerWarp = kDispatchChunk / kWarps;  // 256
+constexpr int kIters = kPairsPerWarp / 32;              // 8
+
+__global__ void __launch_bounds__(kThreads)
+dispatch_hist_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
+                     int32_t* __restrict__ chunk_hist) {
+    extern __shared__ int cnt[];  // [E]
+    for (int e = threadIdx.x; e < E; e += kThreads) cnt[e] = 0;
+    __syncthreads();
+    const int base = blockIdx.x * kDispatchChunk;
+    for (int i = threadIdx.x; i < kDispatchChunk; i += kThreads) {
+        const int pair = base + i;
+        if (pair < R) {
+            const int e = topk_idx[pair];
+            if (e >= 0 && e < E) atomicAdd(&cnt[e], 1);
+        }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += kThreads) chunk_hist[(size_t)blockIdx.x * E + e] = cnt[e];
+}
+
+// One CTA.  Warp w scans experts w, w+32, ... over the chunks; chunk_hist becomes the exclusive
+// prefix (the rank of the chunk's first pair inside its expert).
+__global__ void __launch_bounds__(1024)
+dispatch_scan_kernel(int32_t* __restrict__ chunk_hist, int nchunks, int E, int capacity,
+                     int32_t* __restrict__ kept, int32_t* __restrict__ offsets) {
+    extern __shared__ int total[];  // [E]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int e = warp; e < E; e += 32) {
+        int carry = 0;
+        for (int c0 = 0; c0 < nchunks; c0 += 32) {
+            const int c = c0 + lane;
+            const int v = c < nchunks ? chunk_hist[(size_t)c * E + e] : 0;
+            int incl = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (c < nchunks) chunk_hist[(size_t)c * E + e] = carry + incl - v;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) total[e] = carry;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int e = 0; e < E; ++e) {
+            const int kp = (capacity > 0 && total[e] > capacity) ? capacity : total[e];
+            kept[e] = kp;
+            offsets[e] = run;
+            run += kp;
+        }
+        offsets[E] = run;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+dispatch_scatter_kernel(const T* __restrict__ X, const int32_t* __restrict__ topk_idx,
+                        const float* __restrict__ topk_p, const int32_t* __restrict__ chunk_base,
+                        const int32_t* __restrict__ offsets, int R, int E, int k, int ds, int capacity,
+                        int32_t* __restrict__ dest, int32_t* __restrict__ perm, T* __restrict__ xperm,
+                        float* __restrict__ gate) {
+    extern __shared__ int wcnt[];  // [kWarps][E]
+    constexpr int V = Vec<T>::n;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int chunk = blockIdx.x;
+    const int warp_base = chunk * kDispatchChunk + warp * kPairsPerWarp;
+    int* mine = wcnt + warp * E;
+
+    for (int e = lane; e < E; e += 32) mine[e] = 0;
+    __syncwarp();
+    // pass A: this warp's count per expert
+    for (int it = 0; it < kIters; ++it) {
+        const int pair = warp_base + it * 32 + lane;
+        if (pair < R) {
+            const int e = topk_idx[pair];
+            if (e >= 0 && e < E) atomicAdd(&mine[e], 1);
+        }
+    }
+    __syncthreads();
+    // exclusive prefix over the warps, seeded with the chunk's base rank
+    for (int e = threadIdx.x; e < E; e += kThreads) {
+        int run = chunk_base[(size_t)chunk * E + e];
+        for (int w = 0; w < kWarps; ++w) {
+            const int t = wcnt[w * E + e];
+            wcnt[w * E + e] = run;
+            run += t;
+        }
+    }
+    __syncthreads();
+    // pass B: stable rank of each pair, then the row copy
+    const int vec_per_row = ds / V;
+    for (int it = 0; it < kIters; ++it) {
+        const int pair = warp_base + it * 32 + lane;
+        int e = -1;
+        float p = 0.0f;
+        if (pair < R) {
+            e = topk_idx[pair];
+            p = topk_p[pair];
+            if (e < 0 || e >= E) e = -1;
+        }
+        // lanes with the same expert form a group; invalid lanes get private keys
+        const int key = e >= 0 ? e : -1 - lane;
+        const unsigned grp = __match_any_sync(0xffffffffu, key);
+        const int before = __popc(grp & ((1u << lane) - 1u));
+        int d = -1;
+        if (e >= 0) {
+            const int rank = mine[e] + before;
+            if (capacity == 0 || rank < capacity) d = offsets[e] + rank;
+        }
+        __syncwarp();
+        if (e >= 0 && before == 0) mine[e] += __popc(grp);
+        __syncwarp();
+        if (pair < R) {
+            dest[pair] = d;
+            if (d >= 0) {
+                perm[d] = pair;
+                if (gate) gate[d] = p;
+            }
+        }
+        if (xperm != nullptr) {
+            const int total = 32 * vec_per_row;
+            for (int v = lane; v < total; v += 32) {
+                const int item = v / vec_per_row, col = v - item * vec_per_row;
+                const int d_i = __shfl_sync(0xffffffffu, d, item);
+                const float p_i = __shfl_sync(0xffffffffu, p, item);
+                const int pair_i = warp_base + it * 32 + item;
+                if (d_i >= 0) {
+                    const int n = pair_i / k;
+                    float f[V];
+                    unpack16<T>(*reinterpret_cast<const uint4*>(X + (size_t)n * ds + (size_t)col * V), f);
+#pragma unroll
+                    for (int i = 0; i < V; ++i) f[i] *= p_i;
+                    *reinterpret_cast<uint4*>(xperm + (size_t)d_i * ds + (size_t)col * V) = pack16<T>(f);
+                }
+            }
+        }
+    }
+}
+
+}  // namespace
+
+int launch_dispatch(const Dims& D, const void* h, const int32_t* topk_idx, const float* topk_p,
+                    int32_t* kept, int32_t* offsets, int32_t* dest, int32_t* perm, void* xperm,
+                    float* gate_opt, int32_t* chunk_hist, cudaStream_t st) {
+    const int nchunks = num_chunks(D);
+    if (nchunks > 0) {
+        dispatch_hist_kernel<<<nchunks, kThreads, sizeof(int) * D.E, st>>>(topk_idx, D.R, D.E, chunk_hist);
+        SLICEMOE_LAUNCH_CHECK(1);
+    }
+    dispatch_scan_kernel<<<1, 1024, sizeof(int) * D.E, st>>>(chunk_hist, nchunks, D.E, D.capacity, kept,
+                                                            offsets);
+    SLICEMOE_LAUNCH_CHECK(1);
+    if (nchunks > 0) {
+        const size_t smem = sizeof(int) * kWarps * D.E;
+        if (D.dtype == SLICEMOE_BF16)
+            dispatch_scatter_kernel<bf16><<<nchunks, kThreads, smem, st>>>(
+                (const bf16*)h, topk_idx, topk_p, chunk_hist, offsets, D.R, D.E, D.k, D.ds, D.capacity,
+                dest, perm, (bf16*)xperm, gate_opt);
+        else
+            dispatch_scatter_kernel<float><<<nchunks, kThreads, smem, st>>>(
+                (const float*)h, topk_idx, topk_p, chunk_hist, offsets, D.R, D.E, D.k, D.ds, D.capacity,
+                dest, perm, (float*)xperm, gate_opt);
+        SLICEMOE_LAUNCH_CHECK(1);
+    }
+    return SLICEMOE_OK;
+}
+
+}  // namespace slicemoe

@@ -1,0 +1,206 @@
+"""GPU parity: every C-ABI call against the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2510_04286_b200 import binding, synth, tensors
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+C = synth.CONFIGS
+LC = synth.LayerConfig
+
+# Small shapes that still span several row tiles, dispatch chunks and ragged tails.
+SMALL = {
+    "f32_tiny": C["cfg0"].with_tokens(77),
+    "f32_cfg0": C["cfg0"],
+    "bf16_lm": C["cfg1"].with_tokens(333),                       # N = 2664, R = 5328
+    "bf16_wide": C["cfg2"].with_tokens(150),                     # N = 2400, E = 32
+    "bf16_skew_cap": C["cfg3b"].with_tokens(96),                 # ds = 256, F = 1024, k = 1, capacity
+    "bf16_skew_literal": C["cfg3"].with_tokens(64),              # everything to expert 0, most dropped
+    "bf16_decode": C["cfg4"].with_tokens(16),                    # ds = 128, F = 512, E = 64
+    "bf16_paper_slice96": LC("s96", T=40, d=768, S=8, E=16, k=2, F=384),   # the paper's own ds = 96
+    "bf16_k3": LC("k3", T=50, d=256, S=4, E=8, k=3, F=256),
+    "f32_gelu_cap": LC("f32cap", T=90, d=128, S=2, E=4, k=2, F=128, dtype="f32", capacity=50, init="kaiming"),
+    "bf16_one_expert": LC("e1", T=20, d=128, S=2, E=1, k=1, F=256),
+    "bf16_k_equals_E": LC("kE", T=20, d=128, S=2, E=2, k=2, F=256),
+    "bf16_single_row": LC("one", T=1, d=64, S=1, E=16, k=2, F=256),
+}
+
+
+def inputs(lc, seed=0):
+    return synth.make_layer_inputs(lc, seed)
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_route(name):
+    import torch
+    lc = SMALL[name]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    idx, p, assigned, probs = gpu.route()
+    torch.cuda.synchronize()
+    ref = oracle.route(pu.oracle_config(lc), h, w)
+    idx_np = idx.cpu().numpy()
+    pu.check_routing(ref["probs"], ref["gap"], ref["topk_idx"], idx_np, p.cpu().numpy().astype(np.float64))
+    assert np.abs(probs.cpu().numpy() - ref["probs"]).max() <= 2e-4
+    np.testing.assert_array_equal(assigned.cpu().numpy(), np.bincount(idx_np.ravel(), minlength=lc.E))
+    assert assigned.sum().item() == lc.R
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_dispatch(name):
+    import torch
+    lc = SMALL[name]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    ocfg = pu.oracle_config(lc)
+    # routing input: the oracle's own top-k (dispatch is graded on its own)
+    ref_route = oracle.route(ocfg, h, w)
+    idx = torch.from_numpy(ref_route["topk_idx"]).cuda()
+    p = torch.from_numpy(ref_route["topk_p"].astype(np.float32)).cuda()
+    kept, offsets, dest, perm, xperm = gpu.dispatch(idx, p)
+    torch.cuda.synchronize()
+    ref = oracle.dispatch(ocfg, ref_route["topk_idx"])
+    np.testing.assert_array_equal(kept.cpu().numpy(), ref["kept"])
+    np.testing.assert_array_equal(offsets.cpu().numpy(), ref["offsets"])
+    np.testing.assert_array_equal(dest.cpu().numpy(), ref["dest"])
+    n_kept = int(ref["offsets"][-1])
+    np.testing.assert_array_equal(perm.cpu().numpy()[:n_kept], ref["perm"])
+    assert np.all(perm.cpu().numpy()[n_kept:] == -1)            # nothing written past the kept rows
+    want = oracle.weight_slices(ocfg, h, p.cpu().numpy().astype(np.float64), ref["dest"], n_kept)
+    got = tensors.to_numpy_f32(xperm)[:n_kept]
+    # Eq. 1 with one rounding to the storage type
+    tol = 2.0 ** -8 if lc.dtype == "bf16" else 2.0 ** -23
+    assert np.all(np.abs(got - want) <= tol * np.abs(want) + 1e-30)
+    assert not tensors.to_numpy_f32(xperm)[n_kept:].any()
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_expert_ffn_and_combine(name):
+    import torch
+    lc = SMALL[name]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    ocfg = pu.oracle_config(lc)
+    ref_route = oracle.route(ocfg, h, w)
+    idx = torch.from_numpy(ref_route["topk_idx"]).cuda()
+    p = torch.from_numpy(ref_route["topk_p"].astype(np.float32)).cuda()
+    kept, offsets, dest, perm, xperm = gpu.dispatch(idx, p)
+    yperm = gpu.expert_ffn(xperm, offsets)
+    h_out = gpu.combine(yperm, dest)
+    torch.cuda.synchronize()
+    assert gpu.status() == 0
+    n_kept = int(offsets[-1].item())
+    x_in = tensors.to_numpy_f32(xperm)[:n_kept].astype(np.float64)
+    want_y = oracle.expert_ffn(ocfg, x_in, offsets.cpu().numpy(), w)
+    got_y = tensors.to_numpy_f32(yperm)
+    pu.assert_outputs_close(got_y[:n_kept], want_y, lc.dtype, "yperm")
+    assert not got_y[n_kept:].any()                               # rows past offsets[E] untouched
+    want_h = oracle.combine(ocfg, got_y[:max(n_kept, 1)].astype(np.float64), dest.cpu().numpy())
+    got_h = tensors.to_numpy_f32(h_out)
+    tol = 2.0 ** -8 if lc.dtype == "bf16" else 2.0 ** -22
+    assert np.all(np.abs(got_h - want_h) <= tol * np.abs(want_h) + 1e-30)
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_forward_small(name):
+    rep = pu.check_forward_against_oracle(SMALL[name])
+    print(name, rep)
+
+
+def test_forward_equals_staged_calls_and_is_deterministic():
+    import torch
+    lc = SMALL["bf16_lm"]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    h1, a1, k1, i1, p1 = gpu.forward()
+    h2, a2, k2, i2, p2 = gpu.forward()
+    idx, p, assigned, _ = gpu.route(want_probs=False)
+    kept, offsets, dest, perm, xperm = gpu.dispatch(idx, p)
+    h3 = gpu.combine(gpu.expert_ffn(xperm, offsets), dest)
+    torch.cuda.synchronize()
+    assert torch.equal(h1, h2) and torch.equal(i1, i2) and torch.equal(p1, p2) and torch.equal(a1, a2)
+    assert torch.equal(i1, idx) and torch.equal(a1, assigned) and torch.equal(k1, kept)
+    pu.assert_outputs_close(tensors.to_numpy_f32(h1), tensors.to_numpy_f32(h3), lc.dtype)
+
+
+def test_empty_batch():
+    import torch
+    lc = C["cfg1"].with_tokens(0)
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    h_out, assigned, kept, idx, p = gpu.forward()
+    torch.cuda.synchronize()
+    assert h_out.numel() == 0 and not assigned.any() and not kept.any()
+
+
+def test_forward_host_matches_forward():
+    import torch
+    lc = SMALL["bf16_lm"]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    h_dev = gpu.forward()[0]
+    h_host = tensors.to_torch(h, lc.dtype, "cpu", pin=True)
+    out_host = torch.empty_like(h_host).pin_memory()
+    binding.slicemoe_forward_host(gpu.cfg, gpu.w, h_host, out_host, gpu.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out_host, h_dev.cpu())
+
+
+def test_profiled_forward_records_stage_times():
+    import torch
+    lc = SMALL["bf16_lm"]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    ev = binding.StageEvents()
+    h_out = gpu.empty((lc.T, lc.d), gpu.tdtype)
+    before = binding.slicemoe_launch_count()
+    binding.slicemoe_forward_profiled(gpu.cfg, gpu.w, gpu.h, h_out, gpu.ws, ev)
+    ms = ev.stage_ms()
+    assert len(ms) == 4 and all(m > 0 for m in ms)
+    assert binding.slicemoe_launch_count() - before >= 4
+    assert torch.equal(h_out, gpu.forward()[0])
+
+
+def test_dispatch_drops_out_of_range_ids():
+    import torch
+    lc = SMALL["bf16_lm"]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    rng = np.random.default_rng(3)
+    idx_np = rng.integers(0, lc.E, (lc.N, lc.k)).astype(np.int32)
+    idx_np[::7, 0] = -1
+    idx_np[::11, 1] = lc.E + 3
+    p = torch.rand((lc.N, lc.k), device="cuda")
+    kept, offsets, dest, perm, xperm = gpu.dispatch(torch.from_numpy(idx_np).cuda(), p)
+    torch.cuda.synchronize()
+    valid = (idx_np >= 0) & (idx_np < lc.E)
+    d = dest.cpu().numpy()
+    assert np.all(d[~valid] == -1) and np.all(d[valid] >= 0)
+    np.testing.assert_array_equal(kept.cpu().numpy(), np.bincount(idx_np[valid], minlength=lc.E))
+
+
+# ---- full-size workloads, in the launch configuration the bench times ------------------------
+
+def test_forward_full_cfg1():
+    rep = pu.check_forward_against_oracle(C["cfg1"])
+    print("cfg1", rep)
+
+
+def test_forward_full_cfg4_decode():
+    rep = pu.check_forward_against_oracle(C["cfg4"])
+    print("cfg4", rep)
+
+
+def test_forward_full_cfg3_capacity():
+    for name in ("cfg3", "cfg3b"):
+        rep = pu.check_forward_against_oracle(C[name], sample_rows=4096)
+        print(name, rep)
+
+
+def test_forward_full_cfg2_sampled_rows():
+    rep = pu.check_forward_against_oracle(C["cfg2"], sample_rows=8192)
+    print("cfg2", rep)

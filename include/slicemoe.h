@@ -29,6 +29,7 @@
  *   - Tensors are dense row-major, 16-byte aligned, of cfg->dtype
  *     (bf16 or fp32) unless a type is written.  Weights use the nn.Linear
  *     layout [out, in] with `in` contiguous.  Bias pointers may be NULL (= 0).
+ *   - With T = 0 the token-sized buffers may be NULL; the per-expert outputs are still written.
  *   - Return value: 0 (SLICEMOE_OK) or a slicemoe_status error; on an error
  *     found by argument checking nothing has been launched.  Nothing throws.
  *   - Routing arithmetic (logits, softmax, top-k) is fp32 in both dtypes; with

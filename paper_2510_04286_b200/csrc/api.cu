@@ -244,10 +244,10 @@ static int forward_checked(const slicemoe_config* cfg, const slicemoe_weights* w
     int rc = make_dims(cfg, D);
     if (rc) return rc;
     if ((rc = check_weights(w, true, true))) return rc;
-    if (!h || !h_out) return SLICEMOE_ERR_NULL;
+    if (D.T > 0 && (!h || !h_out)) return SLICEMOE_ERR_NULL;
     if (!aligned16(h) || !aligned16(h_out) || !aligned16(topk_idx_opt) || !aligned16(topk_p_opt))
         return SLICEMOE_ERR_ALIGN;
-    if (overlaps(h, h_out, elem_bytes(D) * (size_t)D.T * D.d)) return SLICEMOE_ERR_ALIAS;
+    if (D.T > 0 && overlaps(h, h_out, elem_bytes(D) * (size_t)D.T * D.d)) return SLICEMOE_ERR_ALIAS;
     Workspace W;
     if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
     if ((rc = check_device())) return rc;

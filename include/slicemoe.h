@@ -57,7 +57,8 @@ typedef enum {
     SLICEMOE_ERR_ALIAS = 6,          /* h_out overlaps h */
     SLICEMOE_ERR_CUDA = 7,           /* a CUDA runtime call failed (see slicemoe_last_cuda_error) */
     SLICEMOE_ERR_DEVICE_TIMEOUT = 8, /* a bounded wait inside a kernel ran out (slicemoe_last_status) */
-    SLICEMOE_ERR_NO_DEVICE = 9       /* no usable sm_100 device */
+    SLICEMOE_ERR_NO_DEVICE = 9,      /* no usable sm_100 device */
+    SLICEMOE_ERR_STATIC_SCRATCH = 10 /* too large for slicemoe_dispatch_static's fixed scratch */
 } slicemoe_status;
 
 typedef enum { SLICEMOE_BF16 = 0, SLICEMOE_F32 = 1 } slicemoe_dtype;
@@ -127,6 +128,37 @@ int slicemoe_route(const slicemoe_config *cfg, const slicemoe_weights *w, const 
 int slicemoe_dispatch(const slicemoe_config *cfg, const void *h, const int32_t *topk_idx,
                       const float *topk_p, int32_t *kept, int32_t *offsets, int32_t *dest,
                       int32_t *perm, void *xperm, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * slicemoe_dispatch for callers that cannot allocate device memory.  (The paper
+ * has no counterpart; this is a deployment variant of the call above.)
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where they
+ * need a dispatch: a plugin running inside another runtime's memory arena, a
+ * real-time serving loop whose memory was pinned down at start-up, code that
+ * runs after the process has handed all free HBM to a caching allocator.  The
+ * ordinary call needs a workspace for its per-chunk histogram table; this one
+ * keeps that table in a fixed array inside the library's own device image, so
+ * the caller passes only inputs and outputs and nothing is allocated or freed,
+ * by this call or by anything it calls.
+ *
+ * Limit: ceil(T*S*k / 2048) * E <= SLICEMOE_STATIC_SCRATCH_INTS (65536 int32 =
+ * 256 KiB, held by every GPU that loads the library until the process exits).
+ * Larger problems return SLICEMOE_ERR_STATIC_SCRATCH and launch nothing.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  All calls
+ * share the one array, which keeps whatever the last call left in it: every
+ * entry a call reads is first written by that same call, so nothing needs
+ * clearing, but two calls that overlap on the GPU (different streams, or
+ * different threads) race on it -- serialise them.
+ *
+ * Arguments and results are exactly those of slicemoe_dispatch.
+ */
+#define SLICEMOE_STATIC_SCRATCH_INTS 65536
+int slicemoe_dispatch_static(const slicemoe_config *cfg, const void *h, const int32_t *topk_idx,
+                             const float *topk_p, int32_t *kept, int32_t *offsets, int32_t *dest,
+                             int32_t *perm, void *xperm, void *stream);
 
 /*
  * Section 3.1 / 3.4, experts: for every expert e and every stacked row r in

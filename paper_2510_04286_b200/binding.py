@@ -19,7 +19,8 @@ N_STAGE_EVENTS = 5
 STAGES = ("route", "dispatch", "expert_ffn", "combine")
 
 EXPORTS = (
-    "slicemoe_workspace_bytes", "slicemoe_route", "slicemoe_dispatch", "slicemoe_expert_ffn",
+    "slicemoe_workspace_bytes", "slicemoe_route", "slicemoe_dispatch", "slicemoe_dispatch_static",
+    "slicemoe_expert_ffn",
     "slicemoe_combine", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
     "slicemoe_event_create", "slicemoe_event_destroy", "slicemoe_event_elapsed_ms",
     "slicemoe_last_status", "slicemoe_launch_count", "slicemoe_last_cuda_error",
@@ -156,6 +157,20 @@ def slicemoe_dispatch(cfg, h, topk_idx, topk_p, kept, offsets, dest, perm, xperm
     _check(_lib().slicemoe_dispatch(ctypes.byref(c), _ptr(h), _ptr(topk_idx), _ptr(topk_p), _ptr(kept),
                                     _ptr(offsets), _ptr(dest), _ptr(perm), _ptr(xperm), _ptr(ws),
                                     ctypes.c_size_t(ws.numel()), _stream(stream)), "slicemoe_dispatch")
+
+
+STATIC_SCRATCH_INTS = 65536
+
+
+def slicemoe_dispatch_static(cfg, h, topk_idx, topk_p, kept, offsets, dest, perm, xperm, stream=None):
+    """slicemoe_dispatch without a workspace, for callers that may not allocate device memory:
+    the histogram table sits in a fixed 256 KiB array inside the library.  Calls share that array,
+    so do not let two of them overlap on the GPU; problems with
+    ceil(R / 2048) * E > STATIC_SCRATCH_INTS are refused (status 10)."""
+    c = cfg.c()
+    _check(_lib().slicemoe_dispatch_static(ctypes.byref(c), _ptr(h), _ptr(topk_idx), _ptr(topk_p),
+                                           _ptr(kept), _ptr(offsets), _ptr(dest), _ptr(perm), _ptr(xperm),
+                                           _stream(stream)), "slicemoe_dispatch_static")
 
 
 def slicemoe_expert_ffn(cfg, w, xperm, offsets, yperm, ws, stream=None):

@@ -43,7 +43,7 @@ Workspace workspace_layout(const Dims& D) {
     return W;
 }
 
-static int make_dims(const slicemoe_config* c, Dims& D) {
+int make_dims(const slicemoe_config* c, Dims& D) {
     if (!c) return SLICEMOE_ERR_NULL;
     if (c->T < 0 || c->d < 1 || c->S < 1 || c->E < 1 || c->k < 1 || c->Hr < 1 || c->F < 1 || c->capacity < 0)
         return SLICEMOE_ERR_SHAPE;
@@ -82,7 +82,7 @@ static int check_weights(const slicemoe_weights* w, bool router, bool experts) {
     return SLICEMOE_OK;
 }
 
-static int check_device() {
+int check_device() {
     static std::atomic<int> state{0};  // 0 unknown, 1 ok, 2 bad
     int s = state.load();
     if (s == 0) {
@@ -342,6 +342,7 @@ const char* slicemoe_status_string(int status) {
         case SLICEMOE_ERR_CUDA: return "a CUDA runtime call failed";
         case SLICEMOE_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
         case SLICEMOE_ERR_NO_DEVICE: return "no usable sm_100 device";
+        case SLICEMOE_ERR_STATIC_SCRATCH: return "problem too large for the fixed scratch of the allocation-free call";
         default: return "unknown status";
     }
 }

@@ -51,6 +51,10 @@ inline int num_chunks(const Dims& D) { return (D.R + kDispatchChunk - 1) / kDisp
 inline int max_tiles(const Dims& D) { return (D.R + kTileM - 1) / kTileM + D.E; }
 inline size_t elem_bytes(const Dims& D) { return D.dtype == SLICEMOE_BF16 ? 2 : 4; }
 
+// Checks a config and derives the sizes (SLICEMOE_OK or an error status).
+int make_dims(const slicemoe_config* c, Dims& D);
+// SLICEMOE_OK if the current device is an sm_100 part.
+int check_device();
 void count_launches(int n);
 void note_cuda_error(cudaError_t e);
 

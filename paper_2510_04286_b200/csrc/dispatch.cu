@@ -8,10 +8,17 @@
 //   2. scan      : per expert, exclusive prefix over chunks; kept = min(total, C); offsets
 //   3. scatter   : per chunk, the stable rank of each pair -> dest / perm, then a coalesced
 //                  16-byte-vector copy of p * X[n, :] to its destination row
+#include <mutex>
+
 #include "common.cuh"
 
 namespace slicemoe {
 namespace {
+
+// Histogram table of slicemoe_dispatch_static: lives in the library's device image, so that the
+// call needs no workspace.  Host code must not use this name as a pointer; it asks the runtime
+// for the device address once per device (static_scratch_address below).
+static __device__ __align__(256) int32_t g_static_chunk_hist[SLICEMOE_STATIC_SCRATCH_INTS];
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
@@ -186,3 +193,53 @@ int launch_dispatch(const Dims& D, const void* h, const int32_t* topk_idx, const
 }
 
 }  // namespace slicemoe
+
+// ---- allocation-free dispatch ------------------------------------------------------------------
+
+namespace slicemoe {
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+int32_t* g_scratch_addr[kMaxDevices] = {};
+
+// Device address of g_static_chunk_hist on the current device, looked up once per device.
+int static_scratch_address(int32_t** out) {
+    int dev = -1;
+    SLICEMOE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SLICEMOE_ERR_NO_DEVICE;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[dev]) {
+        void* p = nullptr;
+        SLICEMOE_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_chunk_hist));
+        if (!p) return SLICEMOE_ERR_CUDA;
+        g_scratch_addr[dev] = static_cast<int32_t*>(p);
+    }
+    *out = g_scratch_addr[dev];
+    return SLICEMOE_OK;
+}
+
+}  // namespace
+}  // namespace slicemoe
+
+extern "C" int slicemoe_dispatch_static(const slicemoe_config* cfg, const void* h,
+                                        const int32_t* topk_idx, const float* topk_p, int32_t* kept,
+                                        int32_t* offsets, int32_t* dest, int32_t* perm, void* xperm,
+                                        void* stream) {
+    using namespace slicemoe;
+    Dims D;
+    int rc = make_dims(cfg, D);
+    if (rc) return rc;
+    if (!topk_idx || !topk_p || !kept || !offsets || !dest || !perm) return SLICEMOE_ERR_NULL;
+    if (xperm && !h) return SLICEMOE_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(h) & 15u) || (reinterpret_cast<uintptr_t>(xperm) & 15u))
+        return SLICEMOE_ERR_ALIGN;
+    if ((long long)num_chunks(D) * D.E > SLICEMOE_STATIC_SCRATCH_INTS) return SLICEMOE_ERR_STATIC_SCRATCH;
+    if ((rc = check_device())) return rc;
+    int32_t* scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch))) return rc;
+    // The histogram kernel writes every entry of the table that the later kernels read, so the
+    // previous call's contents need no clearing.
+    return launch_dispatch(D, h, topk_idx, topk_p, kept, offsets, dest, perm, xperm, nullptr, scratch,
+                           static_cast<cudaStream_t>(stream));
+}

@@ -116,13 +116,17 @@ static int reset_status(void* ws, const Workspace& W, cudaStream_t st) {
     return SLICEMOE_OK;
 }
 
+// The tensor-core kernels take bf16 shapes inside their tile set; everything else (fp32 storage,
+// other widths) runs on the CUDA-core kernels.  Both are this library's own kernels.
 static int route_any(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* idx, float* p,
-                     int32_t* assigned, float* probs, cudaStream_t st) {
+                     int32_t* assigned, float* probs, int32_t* status, cudaStream_t st) {
+    if (tc_route_supported(D)) return launch_route_tc(D, w, h, idx, p, assigned, probs, status, st);
     return launch_route_simt(D, w, h, idx, p, assigned, probs, st);
 }
 
 static int ffn_any(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets,
-                   void* yperm, cudaStream_t st) {
+                   void* yperm, int32_t* status, cudaStream_t st) {
+    if (tc_ffn_supported(D)) return launch_ffn_tc(D, w, xperm, offsets, yperm, status, st);
     return launch_ffn_simt(D, w, xperm, offsets, yperm, st);
 }
 
@@ -145,12 +149,12 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     int rc;
     if ((rc = reset_status(ws, W, st))) return rc;
     if ((rc = mark(0))) return rc;
-    if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, st))) return rc;
+    if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, at<int32_t>(ws, W.status), st))) return rc;
     if ((rc = mark(1))) return rc;
     if ((rc = launch_dispatch(D, h, idx, p, kept, offsets, dest, perm, xperm, nullptr,
                               at<int32_t>(ws, W.chunk_hist), st))) return rc;
     if ((rc = mark(2))) return rc;
-    if ((rc = ffn_any(D, w, xperm, offsets, yperm, st))) return rc;
+    if ((rc = ffn_any(D, w, xperm, offsets, yperm, at<int32_t>(ws, W.status), st))) return rc;
     if ((rc = mark(3))) return rc;
     if ((rc = launch_combine(D, yperm, dest, h_out, st))) return rc;
     return mark(4);
@@ -190,7 +194,8 @@ int slicemoe_route(const slicemoe_config* cfg, const slicemoe_weights* w, const 
     if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
     if ((rc = check_device())) return rc;
     if ((rc = reset_status(ws, W, static_cast<cudaStream_t>(stream)))) return rc;
-    return route_any(D, *w, h, topk_idx, topk_p, assigned, probs_opt, static_cast<cudaStream_t>(stream));
+    return route_any(D, *w, h, topk_idx, topk_p, assigned, probs_opt, at<int32_t>(ws, W.status),
+                     static_cast<cudaStream_t>(stream));
 }
 
 int slicemoe_dispatch(const slicemoe_config* cfg, const void* h, const int32_t* topk_idx,
@@ -222,7 +227,7 @@ int slicemoe_expert_ffn(const slicemoe_config* cfg, const slicemoe_weights* w, c
     if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
     if ((rc = check_device())) return rc;
     if ((rc = reset_status(ws, W, static_cast<cudaStream_t>(stream)))) return rc;
-    return ffn_any(D, *w, xperm, offsets, yperm, static_cast<cudaStream_t>(stream));
+    return ffn_any(D, *w, xperm, offsets, yperm, at<int32_t>(ws, W.status), static_cast<cudaStream_t>(stream));
 }
 
 int slicemoe_combine(const slicemoe_config* cfg, const void* yperm, const int32_t* dest, void* h_out,

@@ -90,6 +90,14 @@ int launch_dispatch(const Dims& D, const void* h, const int32_t* topk_idx, const
 int launch_ffn_simt(const Dims& D, const slicemoe_weights& w, const void* xperm,
                     const int32_t* offsets, void* yperm, cudaStream_t st);
 
+// Tensor-core (tcgen05 / TMEM / TMA) router and grouped expert FFN, bf16 storage only.
+bool tc_route_supported(const Dims& D);
+bool tc_ffn_supported(const Dims& D);
+int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx,
+                    float* topk_p, int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st);
+int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets,
+                  void* yperm, int32_t* status, cudaStream_t st);
+
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);
 

@@ -5,17 +5,22 @@
 //                                                                                 one expert's rows)
 //
 // Both are the same kernel: GEMM-1 into a TMEM accumulator, an epilogue that applies bias +
-// activation and writes the hidden chunk as bf16 into shared memory in the K-major 128-byte
-// swizzled layout, GEMM-2 from that chunk into a second TMEM accumulator, and a final epilogue
-// (softmax + top-k + histogram for the router; bias + store for the experts).  The hidden layer is
-// processed in chunks of HC units and never leaves the SM.
+// activation and writes the hidden chunk as bf16 pairs back into TMEM (over the columns of the
+// accumulator it just read), GEMM-2 with that chunk as its TMEM-resident A operand into a second
+// TMEM accumulator, and a final epilogue (softmax + top-k + histogram for the router; bias +
+// store for the experts).  The hidden layer is processed in chunks of HC units and never leaves
+// tensor memory.
 //
 // One persistent CTA per SM walks a contiguous range of tiles (expert-major, so expert weights
 // stay in shared memory while the expert does not change).  Warp roles:
-//   warp 0        TMA producer (one lane): row tiles and weight chunks
-//   warp 1        TMEM allocation + MMA issue (one lane)
-//   warps 2..     epilogue warps (two warpgroups; a warp owns TMEM lanes 32*(warp_id % 4)..+31,
-//                 one row per thread; the warpgroups split the columns)
+//   warp 0            TMA producer (one lane): row tiles and weight chunks
+//   warp 1            TMEM allocation + MMA issue (one lane)
+//   warps 2, 3        idle (keep every warpgroup aligned to a multiple of four warps)
+//   2 warpgroups      activation: both work on the same hidden chunk, each on half of its
+//                     columns; GEMM-1 accumulators are double-buffered so that the next chunk
+//                     is already waiting when the current one is done
+//   last warpgroup    output: final accumulator -> softmax/top-k or bias + store
+// A warp reads TMEM lanes 32*(warp_id % 4)..+31: one tile row per thread.
 // All hand-offs are mbarriers; every wait is bounded and a run-out sets the status word and makes
 // all roles leave.
 #include <cuda.h>
@@ -48,6 +53,31 @@ struct TcParams {
     int32_t* status;
 };
 
+// Optional timeline tracing (development builds only: -DSLICEMOE_TC_TRACE).  CTA 0 stamps
+// (event code, SM clock) pairs per role into a caller-provided buffer.
+#ifdef SLICEMOE_TC_TRACE
+constexpr int kTraceSlots = 8, kTraceEvents = 2048, kTraceSmemEvents = 320;
+__device__ unsigned long long* g_trace_buf = nullptr;
+// Events go to shared memory (cheap) and are copied out at the end of the kernel.
+struct Tracer {
+    uint2* base;
+    int n;
+    __device__ Tracer(int slot) : base(nullptr), n(0) {
+        extern __shared__ uint8_t smem_raw[];
+        if (blockIdx.x == 0 && g_trace_buf && slot < 6)
+            base = reinterpret_cast<uint2*>(smem_raw + 200 * 1024) + slot * kTraceSmemEvents;
+    }
+    __device__ void operator()(int code) {
+        if (base && n < kTraceSmemEvents) { base[n] = make_uint2((unsigned)code, (unsigned)clock64()); ++n; }
+    }
+};
+#define TRACE_DECL(name, slot) Tracer name(slot)
+#define TRACE(name, code) name(code)
+#else
+#define TRACE_DECL(name, slot)
+#define TRACE(name, code)
+#endif
+
 constexpr int pow2_at_least(int x) {
     int p = 32;
     while (p < x) p <<= 1;
@@ -61,12 +91,33 @@ struct TcCfg {
     static constexpr int HC = (K1 == 64) ? 128 : 64;           // hidden units per chunk
     static constexpr int A_BUFS = (K1 <= 128) ? 2 : 1;
     static constexpr int W_STAGES = (K1 == 128) ? 3 : 2;
-    static constexpr int EPI_WG = 2;
-    static constexpr int EPI_WARPS = EPI_WG * 4;
-    static constexpr int EPI_THREADS = EPI_WG * 128;
-    static constexpr int THREADS = 64 + EPI_THREADS;
+    static constexpr int NWG = 2;                               // activation warpgroups (column split)
+    static constexpr int NBUF = 2;                              // GEMM-1 accumulator / hidden buffers
+    static constexpr int ACT_WARPS = NWG * 4;
+    static constexpr int THREADS = 128 + NWG * 128 + 128;
+    static constexpr int OUT_WARP0 = 4 + NWG * 4;               // first warp of the output warpgroup
     static constexpr int ACC2_BUFS = (N2 <= 128) ? 2 : 1;
-    static constexpr int TMEM_COLS = pow2_at_least(2 * HC + ACC2_BUFS * N2);
+    // The router keeps the hidden layer as a bf16 pair (hi + lo = 16 mantissa bits): GEMM-2 runs
+    // over both halves against the same weights, so that the logits carry fp32-level accuracy and
+    // the top-k decision does not depend on bf16 rounding of the hidden layer.
+    // The experts keep it as plain bf16; their activation math is packed 2-wide bf16.
+    // (A and B of one MMA must have the same 16-bit format: fp16 hidden x bf16 weights is an
+    // illegal instruction on sm_100a.)
+    static constexpr int H_PARTS = ROUTER_ ? 2 : 1;
+    static constexpr bool PACKED_ACT = !ROUTER_;
+    // TMEM columns:
+    //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w owns columns [w HC/2, (w+1) HC/2)
+    //                        of each.  Router: once a thread has read a 32-column piece it writes
+    //                        the piece's hi half (16 packed columns) over the start of its own
+    //                        column range, so the chunk's hi half ends up in two runs of HC/4.
+    //   [2 HC, 3 HC)         two hidden buffers of HC/2 packed columns: the experts' hidden chunk
+    //                        (so GEMM-1 of a later chunk need not wait for GEMM-2), or the
+    //                        router's lo half.
+    //   [3 HC, ...)          ACC2_BUFS final accumulators of N2 columns.
+    static constexpr int H_COL0 = NBUF * HC;
+    static constexpr int ACC2_COL0 = H_COL0 + NBUF * (HC / 2);
+    static constexpr int TMEM_COLS = pow2_at_least(ACC2_COL0 + ACC2_BUFS * N2);
+    static constexpr int KSTEPS_PER_WG = HC / 32;               // 16-element K steps in one warpgroup's half
     static constexpr int KP1 = K1 / 64;                         // 64-wide K panels of GEMM-1
     static constexpr int KP2 = HC / 64;                         // K panels of GEMM-2 per chunk
     static constexpr int A_PANEL = 128 * 128;                   // bytes: 128 rows x 128 B
@@ -76,23 +127,16 @@ struct TcCfg {
     static constexpr int W2_PANEL = N2 * 128;
     static constexpr int W2C_BYTES = KP2 * W2_PANEL;
     static constexpr int W_STAGE_BYTES = W1C_BYTES + W2C_BYTES;
-    static constexpr int H_PANEL = 128 * 128;
-    // The router keeps the hidden layer as a bf16 pair (hi + lo = 16 mantissa bits): GEMM-2 runs
-    // over both halves against the same weights, so that the logits carry fp32-level accuracy and
-    // the top-k decision does not depend on bf16 rounding of the hidden layer.
-    static constexpr int H_PARTS = ROUTER_ ? 2 : 1;
-    static constexpr int H_BYTES = H_PARTS * KP2 * H_PANEL;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_W = OFF_A + A_BUFS * A_BYTES;
-    static constexpr int OFF_H = OFF_W + W_STAGES * W_STAGE_BYTES;
-    static constexpr int SMEM_BYTES = OFF_H + 2 * H_BYTES;
-    static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;        // slack for the 1024-byte alignment
-    static constexpr int COLS1 = HC / EPI_WG;                   // hidden columns per epilogue thread
+    static constexpr int SMEM_BYTES = OFF_W + W_STAGES * W_STAGE_BYTES;
+    // at least 120 KiB is requested so that two CTAs never share an SM (each allocates most of TMEM)
+    static constexpr int SMEM_ALLOC = (SMEM_BYTES + 1024 > 120 * 1024) ? SMEM_BYTES + 1024 : 120 * 1024;
+    static constexpr int NPIECE = HC / (32 * NWG);              // 32-column pieces per thread and chunk
     static_assert(W_STAGE_BYTES % 1024 == 0 && W1C_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
     static_assert(N2 % 16 == 0 && N2 >= 16 && N2 <= 256, "MMA N");
-    static_assert(COLS1 % 32 == 0, "epilogue loads are 32 columns wide");
     static_assert(SMEM_ALLOC <= 232448, "shared memory budget");
-    static_assert(2 * HC + ACC2_BUFS * N2 <= 512, "TMEM budget");
+    static_assert(ACC2_COL0 + ACC2_BUFS * N2 <= 512, "TMEM budget");
 };
 
 // Barrier slots in shared memory.
@@ -102,11 +146,13 @@ struct Bars {
     static constexpr int A_EMPTY = A_FULL + C::A_BUFS;
     static constexpr int W_FULL = A_EMPTY + C::A_BUFS;
     static constexpr int W_EMPTY = W_FULL + C::W_STAGES;
-    static constexpr int ACC1_FULL = W_EMPTY + C::W_STAGES;
-    static constexpr int ACC1_EMPTY = ACC1_FULL + 2;
-    static constexpr int H_FULL = ACC1_EMPTY + 2;
-    static constexpr int H_EMPTY = H_FULL + 2;
-    static constexpr int ACC2_FULL = H_EMPTY + 2;
+    static constexpr int ACC1_FULL = W_EMPTY + C::W_STAGES;   // GEMM-1 done (MMA -> activation)
+    // accumulator may be overwritten: experts, all activation warps have read it;
+    // router (hidden chunk lives in it), GEMM-2 has consumed it
+    static constexpr int ACC1_EMPTY = ACC1_FULL + C::NBUF;
+    static constexpr int H_FULL = ACC1_EMPTY + C::NBUF;       // hidden chunk written (activation -> MMA)
+    static constexpr int H_EMPTY = H_FULL + C::NBUF;          // experts: GEMM-2 has consumed the hidden buffer
+    static constexpr int ACC2_FULL = H_EMPTY + C::NBUF;
     static constexpr int ACC2_EMPTY = ACC2_FULL + C::ACC2_BUFS;
     static constexpr int DRAIN = ACC2_EMPTY + C::ACC2_BUFS;
     static constexpr int COUNT = DRAIN + 1;
@@ -119,24 +165,69 @@ __device__ __forceinline__ void locate_tile(const int* tile_start, const int* of
     rows = min(kTileM, offs[e + 1] - row0);
 }
 
-__device__ __forceinline__ float tanh_approx(float x) {
-    float y;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-template <int ACT>
-__device__ __forceinline__ float activate(float z) {
-    if (ACT == SLICEMOE_ACT_RELU) return fmaxf(z, 0.0f);
-    // GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))
-    const float u = z * fmaf(0.0356774081f, z * z, 0.7978845608f);
-    const float hz = 0.5f * z;
-    return fmaf(hz, tanh_approx(u), hz);
-}
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// 32 fp32 pre-activations (one thread's piece of a row) -> 16 packed bf16 activation pairs, all
+// arithmetic 2-wide in bf16: one conversion, five packed multiply-adds and one packed tanh per
+// pair, written step by step over the whole piece (16 independent instructions per step).
+// GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))).  Where z^2 overflows, tanh
+// saturates to +-1 and the formula still returns z (z > 0) or 0 (z < 0).
+template <int ACT>
+__device__ __forceinline__ void activate_piece_bf16x2(const uint32_t* cur, uint32_t* out) {
+    __nv_bfloat162 z[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) z[i] = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+    if (ACT == SLICEMOE_ACT_RELU) {
+        const __nv_bfloat162 zero = __float2bfloat162_rn(0.0f);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 r = __hmax2(z[i], zero);
+            out[i] = *reinterpret_cast<const uint32_t*>(&r);
+        }
+        return;
+    }
+    const __nv_bfloat162 c0 = __float2bfloat162_rn(0.7978845608f), c1 = __float2bfloat162_rn(0.0356774081f);
+    const __nv_bfloat162 half = __float2bfloat162_rn(0.5f);
+    __nv_bfloat162 u[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) u[i] = __hmul2(z[i], z[i]);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) u[i] = __hfma2(u[i], c1, c0);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) u[i] = __hmul2(z[i], u[i]);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        uint32_t ur = *reinterpret_cast<const uint32_t*>(&u[i]), tr;
+        asm("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
+        u[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) z[i] = __hmul2(z[i], half);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const __nv_bfloat162 r = __hfma2(z[i], u[i], z[i]);
+        out[i] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+}
+
+// Router: ReLU in fp32, then each value as a bf16 pair, the rounded value (hi) and the rounded
+// remainder (lo); hi + lo carries 16 mantissa bits of the fp32 value.
+__device__ __forceinline__ void relu_split_piece(const uint32_t* cur, uint32_t* hi, uint32_t* lo) {
+    float a[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) a[i] = fmaxf(__uint_as_float(cur[i]), 0.0f);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) hi[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        a[2 * i] -= __uint_as_float(hi[i] << 16);
+        a[2 * i + 1] -= __uint_as_float(hi[i] & 0xFFFF0000u);
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) lo[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
 }
 
 template <class C>
@@ -154,26 +245,29 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile int* abort = &abort_flag;
     const int nchunks = p.HID / C::HC;
     const bool resident = nchunks <= C::W_STAGES;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
+#ifdef SLICEMOE_TC_TRACE
+    for (int i = threadIdx.x; i < 6 * kTraceSmemEvents * 2; i += C::THREADS)
+        reinterpret_cast<uint32_t*>(smem_raw + 200 * 1024)[i] = 0;
+#endif
     // ---- set-up ---------------------------------------------------------------------------
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), 1); mbar_init(bar(B::A_EMPTY + i), 1); }
         for (int i = 0; i < C::W_STAGES; ++i) { mbar_init(bar(B::W_FULL + i), 1); mbar_init(bar(B::W_EMPTY + i), 1); }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < C::NBUF; ++i) {
             mbar_init(bar(B::ACC1_FULL + i), 1);
-            mbar_init(bar(B::ACC1_EMPTY + i), C::EPI_WARPS);
-            mbar_init(bar(B::H_FULL + i), C::EPI_WARPS);
+            mbar_init(bar(B::ACC1_EMPTY + i), C::ROUTER ? 1 : C::ACT_WARPS);
+            mbar_init(bar(B::H_FULL + i), C::ACT_WARPS);
             mbar_init(bar(B::H_EMPTY + i), 1);
         }
         for (int i = 0; i < C::ACC2_BUFS; ++i) {
             mbar_init(bar(B::ACC2_FULL + i), 1);
-            mbar_init(bar(B::ACC2_EMPTY + i), C::EPI_WARPS);
+            mbar_init(bar(B::ACC2_EMPTY + i), 4);
         }
         mbar_init(bar(B::DRAIN), 1);
         fence_mbar_init();
@@ -205,37 +299,38 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
     const int t_end = min(total_tiles, t_begin + per_cta);
 
-    const uint32_t sA = smem_base + C::OFF_A, sW = smem_base + C::OFF_W, sH = smem_base + C::OFF_H;
+    const uint32_t sA = smem_base + C::OFF_A, sW = smem_base + C::OFF_W;
 
     if (warp == 0) {
         // ================= TMA producer =====================================================
         if (lane == 0 && t_begin < t_end) {
             int e = 0, prev_e = -1;
-            uint32_t g = 0;
-            uint32_t w_loads[C::W_STAGES];
-            uint32_t last_w_bar[C::W_STAGES], last_w_par[C::W_STAGES];
-            uint32_t last_a_bar[C::A_BUFS], last_a_par[C::A_BUFS];
-            for (int i = 0; i < C::W_STAGES; ++i) { w_loads[i] = 0; last_w_bar[i] = 0; last_w_par[i] = 0; }
-            for (int i = 0; i < C::A_BUFS; ++i) { last_a_bar[i] = 0; last_a_par[i] = 0; }
+            uint32_t g = 0, reloads = 0;             // chunks seen; tiles that (re)loaded weights
+            uint32_t last_a_bar = 0, last_a_par = 0, last_w_bar = 0, last_w_par = 0;
             bool ok = true;
+            TRACE_DECL(tr, 0);
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
                 int row0, rows;
                 locate_tile(tile_start, offs, t, e, row0, rows);
                 const int ab = ta % C::A_BUFS;
                 const uint32_t an = ta / C::A_BUFS;
+                TRACE(tr, 1);
                 if (!mbar_wait(bar(B::A_EMPTY + ab), (an & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                TRACE(tr, 2);
                 mbar_arrive_expect_tx(bar(B::A_FULL + ab), C::A_BYTES);
 #pragma unroll
                 for (int kp = 0; kp < C::KP1; ++kp)
                     tma_load_2d(sA + ab * C::A_BYTES + kp * C::A_PANEL, &tmA, kp * 64, row0, bar(B::A_FULL + ab));
-                last_a_bar[ab] = bar(B::A_FULL + ab);
-                last_a_par[ab] = an & 1u;
+                last_a_bar = bar(B::A_FULL + ab);
+                last_a_par = an & 1u;
                 const bool reload = !resident || (e != prev_e);
                 prev_e = e;
+                if (!reload) { g += nchunks; continue; }
                 for (int c = 0; c < nchunks && ok; ++c, ++g) {
-                    if (!reload) continue;
+                    // resident weights: slot = chunk, n-th load of the slot = n-th reloading tile;
+                    // streamed weights: slots in ring order
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
-                    const uint32_t n = w_loads[slot]++;
+                    const uint32_t n = resident ? reloads : g / C::W_STAGES;
                     if (!mbar_wait(bar(B::W_EMPTY + slot), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar(B::W_FULL + slot), C::W_STAGE_BYTES);
                     const uint32_t dst = sW + slot * C::W_STAGE_BYTES;
@@ -246,105 +341,141 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     for (int kp = 0; kp < C::KP2; ++kp)
                         tma_load_2d(dst + C::W1C_BYTES + kp * C::W2_PANEL, &tmW2, c * C::HC + kp * 64, e * C::N2,
                                     bar(B::W_FULL + slot));
-                    last_w_bar[slot] = bar(B::W_FULL + slot);
-                    last_w_par[slot] = n & 1u;
+                    last_w_bar = bar(B::W_FULL + slot);
+                    last_w_par = n & 1u;
                 }
+                ++reloads;
             }
             if (!ok || *abort) {
-                // leaving early: let this thread's copies in flight land first (bounded)
+                // leaving early: let this thread's last copies land first (bounded; the copies
+                // complete on their own, earlier ones were issued before these)
                 volatile int never = 0;
-                for (int i = 0; i < C::A_BUFS; ++i)
-                    if (last_a_bar[i]) mbar_wait(last_a_bar[i], last_a_par[i], &never, 10000000ull);
-                for (int i = 0; i < C::W_STAGES; ++i)
-                    if (last_w_bar[i]) mbar_wait(last_w_bar[i], last_w_par[i], &never, 10000000ull);
+                if (last_a_bar) mbar_wait(last_a_bar, last_a_par, &never, 10000000ull);
+                if (last_w_bar) mbar_wait(last_w_bar, last_w_par, &never, 10000000ull);
             }
         }
     } else if (warp == 1) {
         // ================= MMA issue =========================================================
         if (lane == 0 && t_begin < t_end) {
-            constexpr uint32_t idesc1 = make_idesc_bf16(128, C::HC);
-            constexpr uint32_t idesc2 = make_idesc_bf16(128, C::N2);
-            uint32_t w_uses[C::W_STAGES];
-            for (int i = 0; i < C::W_STAGES; ++i) w_uses[i] = 0;
+            constexpr uint32_t idesc1 = make_idesc(128, C::HC, kFmtBF16, kFmtBF16);
+            constexpr uint32_t idesc2 = make_idesc(128, C::N2, kFmtBF16, kFmtBF16);
+            const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
             bool ok = true;
+            TRACE_DECL(tr, 1);
 
-            struct Item { int t, ta, c, e; uint32_t g; bool valid, reload, release; };
-            auto enter_tile = [&](Item& it, int prev_e) {
-                int row0, rows;
-                locate_tile(tile_start, offs, it.t, it.e, row0, rows);
-                it.reload = !resident || (it.e != prev_e);
+            // Two cursors over the same (tile, chunk) sequence: `h*` issues GEMM-1, `q*` GEMM-2.
+            // All state is scalar (registers); weight-slot phases follow from counters.
+            int ht = t_begin, hta = 0, hc = 0, he = 0, h_prev_e = -1;
+            uint32_t hg = 0, h_reloads = 0;
+            bool h_valid = true, h_reload = false;
+            int qt = t_begin, qta = 0, qc = 0, qe = 0;
+            uint32_t qg = 0;
+            bool q_valid = true, q_release = false;
+            auto h_enter = [&]() {
+                int r0, rr;
+                locate_tile(tile_start, offs, ht, he, r0, rr);
+                h_reload = !resident || (he != h_prev_e);
+                h_prev_e = he;
+            };
+            auto q_enter = [&]() {
+                int r0, rr;
+                locate_tile(tile_start, offs, qt, qe, r0, rr);
                 bool rel = !resident;
-                if (resident && it.t + 1 < t_end) {
-                    int e2 = it.e, r0, rr;
-                    locate_tile(tile_start, offs, it.t + 1, e2, r0, rr);
-                    rel = (e2 != it.e);
+                if (resident && qt + 1 < t_end) {
+                    int e2 = qe;
+                    locate_tile(tile_start, offs, qt + 1, e2, r0, rr);
+                    rel = (e2 != qe);
                 }
-                it.release = rel;
+                q_release = rel;
             };
-            auto advance = [&](Item& it) {
-                ++it.c; ++it.g;
-                if (it.c == nchunks) {
-                    it.c = 0; ++it.t; ++it.ta;
-                    if (it.t < t_end) { const int pe = it.e; enter_tile(it, pe); } else it.valid = false;
-                }
-            };
-            auto issue_g1 = [&](const Item& it) -> bool {
-                const int ab = it.ta % C::A_BUFS;
-                if (it.c == 0 &&
-                    !mbar_wait(bar(B::A_FULL + ab), (uint32_t)(it.ta / C::A_BUFS) & 1u, abort, kWaitLimitNs)) return false;
-                const int slot = resident ? it.c : (int)(it.g % C::W_STAGES);
-                if (it.reload) {
-                    const uint32_t n = w_uses[slot]++;
+            h_enter();
+            q_enter();
+
+            auto issue_g1 = [&]() -> bool {
+                const int ab = hta % C::A_BUFS;
+                TRACE(tr, 10);
+                if (hc == 0 &&
+                    !mbar_wait(bar(B::A_FULL + ab), (uint32_t)(hta / C::A_BUFS) & 1u, abort, kWaitLimitNs)) return false;
+                TRACE(tr, 11);
+                const int slot = resident ? hc : (int)(hg % C::W_STAGES);
+                if (h_reload) {
+                    const uint32_t n = resident ? h_reloads : hg / C::W_STAGES;
                     if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) return false;
                 }
-                const uint32_t b = it.g & 1u, n1 = it.g >> 1;
+                const uint32_t b = hg % C::NBUF, n1 = hg / C::NBUF;
+                TRACE(tr, 12);
                 if (!mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs)) return false;
+                TRACE(tr, 13);
                 tc_fence_after_sync();
-                const uint32_t a0 = sA + ab * C::A_BYTES, w0 = sW + slot * C::W_STAGE_BYTES;
+                const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W_STAGE_BYTES) >> 4);
+                const uint32_t d = tmem_base + b * C::HC;
+                mma_ss<0>(d, a0, w0, idesc1);
+                TRACE(tr, 15);
 #pragma unroll
-                for (int kk = 0; kk < C::K1 / 16; ++kk) {
-                    const uint64_t ad = make_desc_sw128(a0 + (kk >> 2) * C::A_PANEL + (kk & 3) * 32);
-                    const uint64_t bd = make_desc_sw128(w0 + (kk >> 2) * C::W1_PANEL + (kk & 3) * 32);
-                    mma_bf16_ss(tmem_base + b * C::HC, ad, bd, idesc1, kk > 0 ? 1u : 0u);
+                for (int kk = 1; kk < C::K1 / 16; ++kk) {
+                    mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
+                              w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
+                    TRACE(tr, 15);
                 }
                 mma_commit(bar(B::ACC1_FULL + b));
-                if (it.c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
+                TRACE(tr, 16);
+                if (hc == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
+                TRACE(tr, 14);
+                // advance
+                ++hc; ++hg;
+                if (hc == nchunks) {
+                    if (h_reload) ++h_reloads;
+                    hc = 0; ++ht; ++hta;
+                    if (ht < t_end) h_enter(); else h_valid = false;
+                }
                 return true;
             };
-            auto issue_g2 = [&](const Item& it) -> bool {
-                const uint32_t b = it.g & 1u, n1 = it.g >> 1;
+            auto issue_g2 = [&]() -> bool {
+                const uint32_t b = qg % C::NBUF, n1 = qg / C::NBUF;
+                TRACE(tr, 20);
                 if (!mbar_wait(bar(B::H_FULL + b), n1 & 1u, abort, kWaitLimitNs)) return false;
-                const int buf = it.ta % C::ACC2_BUFS;
-                if (it.c == 0 && !mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(it.ta / C::ACC2_BUFS) & 1u) ^ 1u,
-                                            abort, kWaitLimitNs)) return false;
+                TRACE(tr, 21);
+                const int buf = qta % C::ACC2_BUFS;
+                if (qc == 0 && !mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(qta / C::ACC2_BUFS) & 1u) ^ 1u,
+                                          abort, kWaitLimitNs)) return false;
                 tc_fence_after_sync();
-                const int slot = resident ? it.c : (int)(it.g % C::W_STAGES);
-                const uint32_t h0 = sH + b * C::H_BYTES, w0 = sW + slot * C::W_STAGE_BYTES + C::W1C_BYTES;
+                const int slot = resident ? qc : (int)(qg % C::W_STAGES);
+                const uint32_t w0 = dW + ((slot * C::W_STAGE_BYTES + C::W1C_BYTES) >> 4);
+                const uint32_t d = tmem_base + C::ACC2_COL0 + buf * C::N2;
+                const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: chunk; router: lo half
+                const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi half, two runs
 #pragma unroll
                 for (int part = 0; part < C::H_PARTS; ++part) {
 #pragma unroll
                     for (int kk = 0; kk < C::HC / 16; ++kk) {
-                        const uint64_t ad = make_desc_sw128(h0 + (part * C::KP2 + (kk >> 2)) * C::H_PANEL + (kk & 3) * 32);
-                        const uint64_t bd = make_desc_sw128(w0 + (kk >> 2) * C::W2_PANEL + (kk & 3) * 32);
-                        mma_bf16_ss(tmem_base + 2 * C::HC + buf * C::N2, ad, bd, idesc2,
-                                    (it.c > 0 || kk > 0 || part > 0) ? 1u : 0u);
+                        uint32_t a;
+                        if (C::ROUTER && part == 0)
+                            a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / 2) + (kk % C::KSTEPS_PER_WG) * 8;
+                        else
+                            a = hbuf + kk * 8;
+                        const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
+                        if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, qc > 0 ? 1u : 0u);
+                        else mma_ts<1>(d, a, bd, idesc2);
                     }
                 }
-                mma_commit(bar(B::H_EMPTY + b));
-                if (it.release) mma_commit(bar(B::W_EMPTY + slot));
-                if (it.c == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
+                mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
+                if (q_release) mma_commit(bar(B::W_EMPTY + slot));
+                if (qc == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
+                TRACE(tr, 22);
+                ++qc; ++qg;
+                if (qc == nchunks) {
+                    qc = 0; ++qt; ++qta;
+                    if (qt < t_end) q_enter(); else q_valid = false;
+                }
                 return true;
             };
 
-            Item nxt;
-            nxt.t = t_begin; nxt.ta = 0; nxt.c = 0; nxt.e = 0; nxt.g = 0; nxt.valid = true;
-            enter_tile(nxt, -1);
-            ok = issue_g1(nxt);
-            while (ok && nxt.valid) {
-                const Item cur = nxt;
-                advance(nxt);
-                if (nxt.valid) ok = issue_g1(nxt);
-                if (ok) ok = issue_g2(cur);
+            // GEMM-1 runs one chunk ahead of GEMM-2: the next accumulator is ready when the
+            // activation warps finish the current chunk.
+            ok = issue_g1();
+            while (ok && q_valid) {
+                if (h_valid) ok = issue_g1();
+                if (ok) ok = issue_g2();
             }
             if (!ok || *abort) {
                 // make sure no MMA is still running before TMEM is released
@@ -353,165 +484,168 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 mbar_wait(bar(B::DRAIN), 0u, &never, 10000000ull);
             }
         }
-    } else {
-        // ================= epilogue warps ====================================================
-        const int ew = warp - 2;
-        const int wg = ew >> 2;                       // column split
-        const int lg = warp & 3;                      // TMEM lane group this warp may read
-        const int row = lg * 32 + lane;               // row of the tile owned by this thread
-        const uint32_t tmem_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
+    } else if (warp >= 4 && warp < C::OUT_WARP0) {
+        // ================= activation warpgroups =============================================
+        const int w = (warp - 4) >> 2;                // warpgroup = which half of the chunk's columns
+        const int lg = warp & 3;                      // TMEM lane group this warp may access
+        const uint32_t lane_base = tmem_base + ((uint32_t)(lg * 32) << 16);
+        constexpr int WCOLS = C::HC / C::NWG;         // accumulator columns per thread and chunk
         bool ok = true;
         int e = 0;
         uint32_t g = 0;
-        for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+        TRACE_DECL(tr, (lg == 0 && lane == 0) ? 2 + w : 7);
+        for (int t = t_begin; t < t_end && ok; ++t) {
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
             for (int c = 0; c < nchunks && ok; ++c, ++g) {
-                const uint32_t b = g & 1u, n1 = g >> 1;
+                const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
+                const uint32_t acc1 = lane_base + b * C::HC + w * WCOLS;               // my accumulator columns
+                const uint32_t hdst = lane_base + C::H_COL0 + b * (C::HC / 2) + w * (WCOLS / 2);
+                TRACE(tr, 30);
                 ok = mbar_wait(bar(B::ACC1_FULL + b), n1 & 1u, abort, kWaitLimitNs);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                TRACE(tr, 31);
                 tc_fence_after_sync();
-                uint32_t v[C::COLS1];
+                uint32_t v[2][32];
+                tmem_ld_x32(acc1, v[0]);
 #pragma unroll
-                for (int q = 0; q < C::COLS1 / 32; ++q)
-                    tmem_ld_x32(tmem_lane + b * C::HC + wg * C::COLS1 + q * 32, v + q * 32);
-                tmem_ld_wait();
+                for (int pc = 0; pc < C::NPIECE; ++pc) {
+                    uint32_t* cur = v[pc & 1];
+                    tmem_ld_wait();
+                    TRACE(tr, 32);
+                    if (pc + 1 < C::NPIECE) {
+                        tmem_ld_x32(acc1 + (pc + 1) * 32, v[(pc + 1) & 1]);   // overlaps the math below
+                    } else if constexpr (!C::ROUTER) {
+                        // the accumulator is in registers: GEMM-1 of a later chunk may overwrite it
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
+                    }
+                    if (p.bias1) {
+                        // same address for the whole warp: one broadcast load per 8 columns
+                        const bf16* gb = p.bias1 + (size_t)e * p.HID + c * C::HC + w * WCOLS + pc * 32;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            float bb[8];
+                            unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(gb + j)), bb);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) cur[j + i] = __float_as_uint(__uint_as_float(cur[j + i]) + bb[i]);
+                        }
+                    }
+                    // The 16 column pairs of the piece go through every step together, so that
+                    // each step is 16 independent instructions.
+                    uint32_t hi[16];
+                    if constexpr (C::PACKED_ACT) {
+                        activate_piece_bf16x2<C::ACT>(cur, hi);
+                        if (pc == 0) {
+                            // GEMM-2 of two chunks ago must be done with this hidden buffer
+                            ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
+                            ok = __all_sync(0xffffffffu, ok);
+                        }
+                        if (ok) tmem_st_x16(hdst + pc * 16, hi);
+                    } else {
+                        uint32_t lo[16];
+                        relu_split_piece(cur, hi, lo);
+                        tmem_st_x16(acc1 + pc * 16, hi);     // over columns this thread has already read
+                        tmem_st_x16(hdst + pc * 16, lo);
+                    }
+                    TRACE(tr, 33);
+                }
+                if (!ok) break;
+                tmem_st_wait();
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
-                // bias (same address for the whole warp: one broadcast load per 8 columns) +
-                // activation, packed to bf16 pairs
-                if (p.bias1) {
-                    const bf16* gb = p.bias1 + (size_t)e * p.HID + c * C::HC + wg * C::COLS1;
-#pragma unroll
-                    for (int j = 0; j < C::COLS1; j += 8) {
-                        float bb[8];
-                        unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(gb + j)), bb);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) v[j + i] = __float_as_uint(__uint_as_float(v[j + i]) + bb[i]);
-                    }
-                }
-                uint32_t packed[C::COLS1 / 2];
-#pragma unroll
-                for (int j = 0; j < C::COLS1; j += 2) {
-                    const float a0 = activate<C::ACT>(__uint_as_float(v[j]));
-                    const float a1 = activate<C::ACT>(__uint_as_float(v[j + 1]));
-                    packed[j / 2] = pack_bf16x2(a0, a1);
-                    if constexpr (C::H_PARTS == 2) {
-                        // remainder after the bf16 rounding, itself rounded to bf16 (reuses v)
-                        const float r0 = a0 - __uint_as_float(packed[j / 2] << 16);
-                        const float r1 = a1 - __uint_as_float(packed[j / 2] & 0xFFFF0000u);
-                        v[j / 2] = pack_bf16x2(r0, r1);
-                    }
-                }
-                ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                // hidden chunk -> shared memory, K-major rows of 64 bf16 with the 128-byte swizzle
-                uint8_t* hrow = smem_gen + C::OFF_H + b * C::H_BYTES + (row >> 3) * 1024 + (row & 7) * 128;
-#pragma unroll
-                for (int q = 0; q < C::COLS1 / 8; ++q) {
-                    const int col = wg * C::COLS1 + q * 8;
-                    const int panel = col >> 6, j16 = (col & 63) >> 3;
-                    uint4 val = make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
-                    *reinterpret_cast<uint4*>(hrow + panel * C::H_PANEL + ((j16 ^ (row & 7)) << 4)) = val;
-                    if constexpr (C::H_PARTS == 2) {
-                        uint4 lo = make_uint4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
-                        *reinterpret_cast<uint4*>(hrow + (C::KP2 + panel) * C::H_PANEL + ((j16 ^ (row & 7)) << 4)) = lo;
-                    }
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B::H_FULL + b));
+                TRACE(tr, 35);
             }
-            if (!ok) break;
-            // ---- final epilogue of the tile -----------------------------------------------
+        }
+    } else if (warp >= C::OUT_WARP0) {
+        // ================= output warpgroup ==================================================
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
+        bool ok = true;
+        int e = 0;
+        TRACE_DECL(tr, (lg == 0 && lane == 0) ? 5 : 7);
+        for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+            int row0, rows;
+            locate_tile(tile_start, offs, t, e, row0, rows);
             const int buf = ta % C::ACC2_BUFS;
+            TRACE(tr, 40);
             ok = mbar_wait(bar(B::ACC2_FULL + buf), (uint32_t)(ta / C::ACC2_BUFS) & 1u, abort, kWaitLimitNs);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            TRACE(tr, 41);
             tc_fence_after_sync();
-            const uint32_t acc2 = tmem_lane + 2 * C::HC + buf * C::N2;
+            const uint32_t acc2 = tmem_lane + C::ACC2_COL0 + buf * C::N2;
+            uint32_t v[C::N2];
+#pragma unroll
+            for (int q = 0; q < C::N2 / 16; ++q) tmem_ld_x16(acc2 + q * 16, v + q * 16);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
+            TRACE(tr, 42);
+            if (row >= rows) continue;
             if constexpr (C::ROUTER) {
                 constexpr int E = C::N2;
-                uint32_t v[E];
-                if (wg == 0) {
+                float gl[E];
 #pragma unroll
-                    for (int q = 0; q < E / 16; ++q) tmem_ld_x16(acc2 + q * 16, v + q * 16);
-                    tmem_ld_wait();
+                for (int i = 0; i < E; ++i)
+                    gl[i] = __uint_as_float(v[i]) + (p.bias2 ? __bfloat162float(__ldg(p.bias2 + i)) : 0.0f);
+                const int n = row0 + row;
+                // top-k by repeated arg-max over the logits; ties go to the lower id
+                unsigned long long taken = 0ull;
+                float m = 0.0f;
+                int sel[8];
+                float gsel[8];
+                for (int j = 0; j < p.k; ++j) {
+                    int best = -1;
+                    float bv = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < E; ++i) {
+                        const bool free_i = !((taken >> i) & 1ull);
+                        if (free_i && (best < 0 || gl[i] > bv)) { best = i; bv = gl[i]; }
+                    }
+                    taken |= 1ull << best;
+                    sel[j] = best;
+                    gsel[j] = bv;
+                    if (j == 0) m = bv;
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
-                if (wg == 0 && row < rows) {
-                    float gl[E];
+                float sum = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < E; ++i)
-                        gl[i] = __uint_as_float(v[i]) + (p.bias2 ? __bfloat162float(__ldg(p.bias2 + i)) : 0.0f);
-                    const int n = row0 + row;
-                    // top-k by repeated arg-max over the logits; ties go to the lower id
-                    unsigned long long taken = 0ull;
-                    float m = 0.0f;
-                    int sel[8];
-                    float gsel[8];
-                    for (int j = 0; j < p.k; ++j) {
-                        int best = -1;
-                        float bv = 0.0f;
+                for (int i = 0; i < E; ++i) sum += __expf(gl[i] - m);
+                const float inv = 1.0f / sum;
+                for (int j = 0; j < p.k; ++j) {
+                    p.topk_idx[(size_t)n * p.k + j] = sel[j];
+                    p.topk_p[(size_t)n * p.k + j] = __expf(gsel[j] - m) * inv;
+                    atomicAdd(&hist[sel[j]], 1);
+                }
+                if (p.probs) {
+                    float4* dst = reinterpret_cast<float4*>(p.probs + (size_t)n * E);
 #pragma unroll
-                        for (int i = 0; i < E; ++i) {
-                            const bool free_i = !((taken >> i) & 1ull);
-                            if (free_i && (best < 0 || gl[i] > bv)) { best = i; bv = gl[i]; }
-                        }
-                        taken |= 1ull << best;
-                        sel[j] = best;
-                        gsel[j] = bv;
-                        if (j == 0) m = bv;
-                    }
-                    float sum = 0.0f;
-#pragma unroll
-                    for (int i = 0; i < E; ++i) sum += __expf(gl[i] - m);
-                    const float inv = 1.0f / sum;
-                    for (int j = 0; j < p.k; ++j) {
-                        p.topk_idx[(size_t)n * p.k + j] = sel[j];
-                        p.topk_p[(size_t)n * p.k + j] = __expf(gsel[j] - m) * inv;
-                        atomicAdd(&hist[sel[j]], 1);
-                    }
-                    if (p.probs) {
-                        float4* dst = reinterpret_cast<float4*>(p.probs + (size_t)n * E);
-#pragma unroll
-                        for (int i = 0; i < E; i += 4)
-                            dst[i / 4] = make_float4(__expf(gl[i] - m) * inv, __expf(gl[i + 1] - m) * inv,
-                                                     __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
-                    }
+                    for (int i = 0; i < E; i += 4)
+                        dst[i / 4] = make_float4(__expf(gl[i] - m) * inv, __expf(gl[i + 1] - m) * inv,
+                                                 __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
                 }
             } else {
-                constexpr int COLS2 = C::N2 / C::EPI_WG;
-                uint32_t v[COLS2];
+                bf16* dst = p.yperm + (size_t)(row0 + row) * C::N2;
 #pragma unroll
-                for (int q = 0; q < COLS2 / 16; ++q) tmem_ld_x16(acc2 + wg * COLS2 + q * 16, v + q * 16);
-                tmem_ld_wait();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
-                if (row < rows) {
-                    bf16* dst = p.yperm + (size_t)(row0 + row) * C::N2 + wg * COLS2;
+                for (int q = 0; q < C::N2 / 8; ++q) {
+                    float bb[8];
+                    if (p.bias2) {
+                        unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.bias2 + (size_t)e * C::N2 + q * 8)), bb);
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < COLS2 / 8; ++q) {
-                        float bb[8];
-                        if (p.bias2) {
-                            unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.bias2 + (size_t)e * C::N2 + wg * COLS2 + q * 8)), bb);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) bb[i] = 0.0f;
-                        }
-                        uint32_t o[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            o[i] = pack_bf16x2(__uint_as_float(v[q * 8 + 2 * i]) + bb[2 * i],
-                                               __uint_as_float(v[q * 8 + 2 * i + 1]) + bb[2 * i + 1]);
-                        *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                        for (int i = 0; i < 8; ++i) bb[i] = 0.0f;
                     }
+                    uint32_t o[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        o[i] = pack_bf16x2(__uint_as_float(v[q * 8 + 2 * i]) + bb[2 * i],
+                                           __uint_as_float(v[q * 8 + 2 * i + 1]) + bb[2 * i + 1]);
+                    *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
         }
@@ -526,6 +660,16 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         for (int i = threadIdx.x; i < C::N2; i += C::THREADS)
             if (hist[i]) atomicAdd(&p.assigned[i], hist[i]);
     }
+#ifdef SLICEMOE_TC_TRACE
+    if (blockIdx.x == 0 && g_trace_buf) {
+        const uint2* src = reinterpret_cast<const uint2*>(smem_raw + 200 * 1024);
+        for (int i = threadIdx.x; i < 6 * kTraceSmemEvents; i += C::THREADS) {
+            const int slot = i / kTraceSmemEvents, n = i % kTraceSmemEvents;
+            g_trace_buf[((size_t)slot * kTraceEvents + n) * 2] = src[i].x;
+            g_trace_buf[((size_t)slot * kTraceEvents + n) * 2 + 1] = src[i].y;
+        }
+    }
+#endif
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();
@@ -576,6 +720,12 @@ int sm_count() {
     return n;
 }
 
+#ifdef SLICEMOE_TC_TRACE
+template <class C> constexpr int kSmemLaunch = 200 * 1024 + 6 * kTraceSmemEvents * 8;   // trace area after 200 KiB
+#else
+template <class C> constexpr int kSmemLaunch = C::SMEM_ALLOC;
+#endif
+
 template <class C>
 int launch_tc(const void* A, uint64_t a_rows, const void* W1, const void* W2, int n_experts, const TcParams& p,
               int max_tiles, cudaStream_t st) {
@@ -587,11 +737,11 @@ int launch_tc(const void* A, uint64_t a_rows, const void* W1, const void* W2, in
     auto kern = tc_mlp_kernel<C>;
     static bool attr_set = false;
     if (!attr_set) {
-        SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_ALLOC));
+        SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch<C>));
         attr_set = true;
     }
     const int grid = max_tiles < sm_count() ? max_tiles : sm_count();
-    kern<<<grid, C::THREADS, C::SMEM_ALLOC, st>>>(tmA, tmW1, tmW2, p);
+    kern<<<grid, C::THREADS, kSmemLaunch<C>, st>>>(tmA, tmW1, tmW2, p);
     SLICEMOE_LAUNCH_CHECK(1);
     return SLICEMOE_OK;
 }
@@ -620,13 +770,22 @@ int launch_route_k1(const Dims& D, const slicemoe_weights& w, const void* h, con
 
 }  // namespace
 
+#ifdef SLICEMOE_TC_TRACE
+// Development hook: where CTA 0 of the next tensor-core launches writes its timeline
+// (kTraceSlots * kTraceEvents * 2 uint64 values; NULL switches tracing off).
+extern "C" int slicemoe_debug_set_trace(void* device_buf) {
+    unsigned long long* ptr = static_cast<unsigned long long*>(device_buf);
+    return cudaMemcpyToSymbol(g_trace_buf, &ptr, sizeof(ptr)) == cudaSuccess ? 0 : SLICEMOE_ERR_CUDA;
+}
+#endif
+
 bool tc_route_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
     if (D.ds != 64 && D.ds != 128 && D.ds != 256) return false;
     if (D.E != 16 && D.E != 32 && D.E != 64) return false;
     const int hc = D.ds == 64 ? 128 : 64;
-    // at least two hidden chunks: the MMA warp issues GEMM-1 of the next chunk before GEMM-2 of the
-    // current one, and with resident weights that look-ahead must not need the slot it is still using
+    // at least two hidden chunks: GEMM-1 is issued ahead of GEMM-2, and with resident weights that
+    // look-ahead must not need the weight slot that the chunk in flight is still using
     return D.Hr % hc == 0 && D.Hr >= 2 * hc && D.Hr <= kMaxHid && D.k <= 8;
 }
 

@@ -151,10 +151,18 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     if ((rc = mark(0))) return rc;
     if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, at<int32_t>(ws, W.status), st))) return rc;
     if ((rc = mark(1))) return rc;
-    if ((rc = launch_dispatch(D, h, idx, p, kept, offsets, dest, perm, xperm, nullptr,
-                              at<int32_t>(ws, W.chunk_hist), st))) return rc;
+    // With the tensor-core expert kernel the stacked rows are never materialised: dispatch only
+    // ranks the pairs (dest, perm, gate) and the kernel gathers its rows from h.
+    const bool fused_gather = tc_ffn_supported(D);
+    float* gate = at<float>(ws, W.gate);
+    if ((rc = launch_dispatch(D, h, idx, p, kept, offsets, dest, perm, fused_gather ? nullptr : xperm,
+                              fused_gather ? gate : nullptr, at<int32_t>(ws, W.chunk_hist), st))) return rc;
     if ((rc = mark(2))) return rc;
-    if ((rc = ffn_any(D, w, xperm, offsets, yperm, at<int32_t>(ws, W.status), st))) return rc;
+    if (fused_gather) {
+        if ((rc = launch_ffn_tc(D, w, nullptr, offsets, yperm, at<int32_t>(ws, W.status), st, h, perm, gate))) return rc;
+    } else {
+        if ((rc = ffn_any(D, w, xperm, offsets, yperm, at<int32_t>(ws, W.status), st))) return rc;
+    }
     if ((rc = mark(3))) return rc;
     if ((rc = launch_combine(D, yperm, dest, h_out, st))) return rc;
     return mark(4);

@@ -95,8 +95,11 @@ bool tc_route_supported(const Dims& D);
 bool tc_ffn_supported(const Dims& D);
 int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx,
                     float* topk_p, int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st);
+// With gather_h != nullptr the rows are not read from xperm: row r of the stacked order is
+// bf16(gate[r] * X[perm[r] / k, :]) gathered from h inside the kernel (fused forward).
 int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets,
-                  void* yperm, int32_t* status, cudaStream_t st);
+                  void* yperm, int32_t* status, cudaStream_t st, const void* gather_h = nullptr,
+                  const int32_t* perm = nullptr, const float* gate = nullptr);
 
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);

@@ -14,12 +14,17 @@
 // One persistent CTA per SM walks a contiguous range of tiles (expert-major, so expert weights
 // stay in shared memory while the expert does not change).  Warp roles:
 //   warp 0            TMA producer (one lane): row tiles and weight chunks
-//   warp 1            TMEM allocation + MMA issue (one lane)
-//   warps 2, 3        idle (keep every warpgroup aligned to a multiple of four warps)
+//   warp 1            TMEM allocation + GEMM-1 issue (one lane)
+//   warp 2            GEMM-2 issue (one lane); two issuing threads because the small MMAs of this
+//                     layer (N <= 128) are issue-bound, not tensor-bound
+//   warp 3            idle (keeps every warpgroup aligned to a multiple of four warps)
 //   2 warpgroups      activation: both work on the same hidden chunk, each on half of its
 //                     columns; GEMM-1 accumulators are double-buffered so that the next chunk
 //                     is already waiting when the current one is done
-//   last warpgroup    output: final accumulator -> softmax/top-k or bias + store
+//   last warpgroup    output: final accumulator -> softmax/top-k or bias + store.  In the fused
+//                     forward it also builds the next tile's A operand: each thread gathers one
+//                     row of h through perm, applies the gate of Eq. 1 and writes it swizzled
+//                     (otherwise the A tile comes from the stacked rows by TMA)
 // A warp reads TMEM lanes 32*(warp_id % 4)..+31: one tile row per thread.
 // All hand-offs are mbarriers; every wait is bounded and a run-out sets the status word and makes
 // all roles leave.
@@ -45,6 +50,11 @@ struct TcParams {
     const bf16* bias1;        // [E, HID] or nullptr
     const bf16* bias2;        // [E, N2]  or nullptr
     bf16* yperm;              // experts: output rows [R, N2]
+    // experts, fused forward: A rows are gathered instead of read from stacked rows
+    const bf16* gather_src;   // h viewed as X[N, K1], or nullptr (A = stacked rows via TMA)
+    const int32_t* perm;      // [R] pair index n*k + j of each stacked row
+    const float* gate;        // [R] gate value of each stacked row
+    int gather_k;             // k (pairs per row)
     int32_t* topk_idx;        // router outputs
     float* topk_p;
     int32_t* assigned;
@@ -155,7 +165,7 @@ struct Bars {
     static constexpr int ACC2_FULL = H_EMPTY + C::NBUF;
     static constexpr int ACC2_EMPTY = ACC2_FULL + C::ACC2_BUFS;
     static constexpr int DRAIN = ACC2_EMPTY + C::ACC2_BUFS;
-    static constexpr int COUNT = DRAIN + 1;
+    static constexpr int COUNT = DRAIN + 2;
 };
 
 __device__ __forceinline__ void locate_tile(const int* tile_start, const int* offs, int t, int& e,
@@ -172,9 +182,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 // 32 fp32 pre-activations (one thread's piece of a row) -> 16 packed bf16 activation pairs, all
 // arithmetic 2-wide in bf16: one conversion, five packed multiply-adds and one packed tanh per
-// pair, written step by step over the whole piece (16 independent instructions per step).
-// GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))).  Where z^2 overflows, tanh
-// saturates to +-1 and the formula still returns z (z > 0) or 0 (z < 0).
+// pair.  GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))).  Where z^2 overflows,
+// tanh saturates to +-1 and the formula still returns z (z > 0) or 0 (z < 0).
+// The tanh unit (16 results per clock per SM) is the scarce resource, so the piece is processed
+// in groups of four pairs, staggered: while one group's tanh is in flight the multiply-adds
+// before the next group's tanh and after the previous group's are issued.
 template <int ACT>
 __device__ __forceinline__ void activate_piece_bf16x2(const uint32_t* cur, uint32_t* out) {
     __nv_bfloat162 z[16];
@@ -191,26 +203,33 @@ __device__ __forceinline__ void activate_piece_bf16x2(const uint32_t* cur, uint3
     }
     const __nv_bfloat162 c0 = __float2bfloat162_rn(0.7978845608f), c1 = __float2bfloat162_rn(0.0356774081f);
     const __nv_bfloat162 half = __float2bfloat162_rn(0.5f);
-    __nv_bfloat162 u[16];
+    __nv_bfloat162 t[16];
+    auto pre_tanh = [&](int g0) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) u[i] = __hmul2(z[i], z[i]);
+        for (int i = g0; i < g0 + 4; ++i) {
+            const __nv_bfloat162 inner = __hfma2(__hmul2(z[i], z[i]), c1, c0);
+            const __nv_bfloat162 u = __hmul2(z[i], inner);
+            uint32_t ur = *reinterpret_cast<const uint32_t*>(&u), tr;
+            asm volatile("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
+            t[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
+        }
+    };
+    auto post = [&](int g0) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) u[i] = __hfma2(u[i], c1, c0);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) u[i] = __hmul2(z[i], u[i]);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        uint32_t ur = *reinterpret_cast<const uint32_t*>(&u[i]), tr;
-        asm("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
-        u[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
-    }
-#pragma unroll
-    for (int i = 0; i < 16; ++i) z[i] = __hmul2(z[i], half);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const __nv_bfloat162 r = __hfma2(z[i], u[i], z[i]);
-        out[i] = *reinterpret_cast<const uint32_t*>(&r);
-    }
+        for (int i = g0; i < g0 + 4; ++i) {
+            const __nv_bfloat162 hz = __hmul2(z[i], half);
+            const __nv_bfloat162 r = __hfma2(hz, t[i], hz);
+            out[i] = *reinterpret_cast<const uint32_t*>(&r);
+        }
+    };
+    pre_tanh(0);
+    pre_tanh(4);
+    post(0);
+    pre_tanh(8);
+    post(4);
+    pre_tanh(12);
+    post(8);
+    post(12);
 }
 
 // Router: ReLU in fp32, then each value as a bf16 pair, the rounded value (hi) and the rounded
@@ -248,6 +267,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     volatile int* abort = &abort_flag;
     const int nchunks = p.HID / C::HC;
     const bool resident = nchunks <= C::W_STAGES;
+    const bool gather = !C::ROUTER && p.gather_src != nullptr;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
 #ifdef SLICEMOE_TC_TRACE
@@ -257,7 +277,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     // ---- set-up ---------------------------------------------------------------------------
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), 1); mbar_init(bar(B::A_EMPTY + i), 1); }
+        for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 4 : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
         for (int i = 0; i < C::W_STAGES; ++i) { mbar_init(bar(B::W_FULL + i), 1); mbar_init(bar(B::W_EMPTY + i), 1); }
         for (int i = 0; i < C::NBUF; ++i) {
             mbar_init(bar(B::ACC1_FULL + i), 1);
@@ -270,6 +290,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             mbar_init(bar(B::ACC2_EMPTY + i), 4);
         }
         mbar_init(bar(B::DRAIN), 1);
+        mbar_init(bar(B::DRAIN + 1), 1);
         fence_mbar_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmW1);
@@ -314,15 +335,17 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 locate_tile(tile_start, offs, t, e, row0, rows);
                 const int ab = ta % C::A_BUFS;
                 const uint32_t an = ta / C::A_BUFS;
-                TRACE(tr, 1);
-                if (!mbar_wait(bar(B::A_EMPTY + ab), (an & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
-                TRACE(tr, 2);
-                mbar_arrive_expect_tx(bar(B::A_FULL + ab), C::A_BYTES);
+                if (!gather) {
+                    TRACE(tr, 1);
+                    if (!mbar_wait(bar(B::A_EMPTY + ab), (an & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    TRACE(tr, 2);
+                    mbar_arrive_expect_tx(bar(B::A_FULL + ab), C::A_BYTES);
 #pragma unroll
-                for (int kp = 0; kp < C::KP1; ++kp)
-                    tma_load_2d(sA + ab * C::A_BYTES + kp * C::A_PANEL, &tmA, kp * 64, row0, bar(B::A_FULL + ab));
-                last_a_bar = bar(B::A_FULL + ab);
-                last_a_par = an & 1u;
+                    for (int kp = 0; kp < C::KP1; ++kp)
+                        tma_load_2d(sA + ab * C::A_BYTES + kp * C::A_PANEL, &tmA, kp * 64, row0, bar(B::A_FULL + ab));
+                    last_a_bar = bar(B::A_FULL + ab);
+                    last_a_par = an & 1u;
+                }
                 const bool reload = !resident || (e != prev_e);
                 prev_e = e;
                 if (!reload) { g += nchunks; continue; }
@@ -355,133 +378,120 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issue =========================================================
+        // ================= GEMM-1 issue ======================================================
         if (lane == 0 && t_begin < t_end) {
             constexpr uint32_t idesc1 = make_idesc(128, C::HC, kFmtBF16, kFmtBF16);
-            constexpr uint32_t idesc2 = make_idesc(128, C::N2, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
             bool ok = true;
             TRACE_DECL(tr, 1);
-
-            // Two cursors over the same (tile, chunk) sequence: `h*` issues GEMM-1, `q*` GEMM-2.
-            // All state is scalar (registers); weight-slot phases follow from counters.
-            int ht = t_begin, hta = 0, hc = 0, he = 0, h_prev_e = -1;
-            uint32_t hg = 0, h_reloads = 0;
-            bool h_valid = true, h_reload = false;
-            int qt = t_begin, qta = 0, qc = 0, qe = 0;
-            uint32_t qg = 0;
-            bool q_valid = true, q_release = false;
-            auto h_enter = [&]() {
+            int e = 0, prev_e = -1;
+            uint32_t g = 0, reloads = 0;
+            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
                 int r0, rr;
-                locate_tile(tile_start, offs, ht, he, r0, rr);
-                h_reload = !resident || (he != h_prev_e);
-                h_prev_e = he;
-            };
-            auto q_enter = [&]() {
-                int r0, rr;
-                locate_tile(tile_start, offs, qt, qe, r0, rr);
-                bool rel = !resident;
-                if (resident && qt + 1 < t_end) {
-                    int e2 = qe;
-                    locate_tile(tile_start, offs, qt + 1, e2, r0, rr);
-                    rel = (e2 != qe);
-                }
-                q_release = rel;
-            };
-            h_enter();
-            q_enter();
-
-            auto issue_g1 = [&]() -> bool {
-                const int ab = hta % C::A_BUFS;
+                locate_tile(tile_start, offs, t, e, r0, rr);
+                const bool reload = !resident || (e != prev_e);
+                prev_e = e;
+                const int ab = ta % C::A_BUFS;
                 TRACE(tr, 10);
-                if (hc == 0 &&
-                    !mbar_wait(bar(B::A_FULL + ab), (uint32_t)(hta / C::A_BUFS) & 1u, abort, kWaitLimitNs)) return false;
+                if (!mbar_wait(bar(B::A_FULL + ab), (uint32_t)(ta / C::A_BUFS) & 1u, abort, kWaitLimitNs)) { ok = false; break; }
                 TRACE(tr, 11);
-                const int slot = resident ? hc : (int)(hg % C::W_STAGES);
-                if (h_reload) {
-                    const uint32_t n = resident ? h_reloads : hg / C::W_STAGES;
-                    if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) return false;
-                }
-                const uint32_t b = hg % C::NBUF, n1 = hg / C::NBUF;
-                TRACE(tr, 12);
-                if (!mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs)) return false;
-                TRACE(tr, 13);
-                tc_fence_after_sync();
-                const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W_STAGE_BYTES) >> 4);
-                const uint32_t d = tmem_base + b * C::HC;
-                mma_ss<0>(d, a0, w0, idesc1);
-                TRACE(tr, 15);
-#pragma unroll
-                for (int kk = 1; kk < C::K1 / 16; ++kk) {
-                    mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
-                              w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
-                    TRACE(tr, 15);
-                }
-                mma_commit(bar(B::ACC1_FULL + b));
-                TRACE(tr, 16);
-                if (hc == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
-                TRACE(tr, 14);
-                // advance
-                ++hc; ++hg;
-                if (hc == nchunks) {
-                    if (h_reload) ++h_reloads;
-                    hc = 0; ++ht; ++hta;
-                    if (ht < t_end) h_enter(); else h_valid = false;
-                }
-                return true;
-            };
-            auto issue_g2 = [&]() -> bool {
-                const uint32_t b = qg % C::NBUF, n1 = qg / C::NBUF;
-                TRACE(tr, 20);
-                if (!mbar_wait(bar(B::H_FULL + b), n1 & 1u, abort, kWaitLimitNs)) return false;
-                TRACE(tr, 21);
-                const int buf = qta % C::ACC2_BUFS;
-                if (qc == 0 && !mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(qta / C::ACC2_BUFS) & 1u) ^ 1u,
-                                          abort, kWaitLimitNs)) return false;
-                tc_fence_after_sync();
-                const int slot = resident ? qc : (int)(qg % C::W_STAGES);
-                const uint32_t w0 = dW + ((slot * C::W_STAGE_BYTES + C::W1C_BYTES) >> 4);
-                const uint32_t d = tmem_base + C::ACC2_COL0 + buf * C::N2;
-                const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: chunk; router: lo half
-                const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi half, two runs
-#pragma unroll
-                for (int part = 0; part < C::H_PARTS; ++part) {
-#pragma unroll
-                    for (int kk = 0; kk < C::HC / 16; ++kk) {
-                        uint32_t a;
-                        if (C::ROUTER && part == 0)
-                            a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / 2) + (kk % C::KSTEPS_PER_WG) * 8;
-                        else
-                            a = hbuf + kk * 8;
-                        const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
-                        if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, qc > 0 ? 1u : 0u);
-                        else mma_ts<1>(d, a, bd, idesc2);
+                for (int c = 0; c < nchunks; ++c, ++g) {
+                    const int slot = resident ? c : (int)(g % C::W_STAGES);
+                    if (reload) {
+                        const uint32_t n = resident ? reloads : g / C::W_STAGES;
+                        if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
                     }
+                    const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
+                    TRACE(tr, 12);
+                    if (!mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    TRACE(tr, 13);
+                    tc_fence_after_sync();
+                    const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W_STAGE_BYTES) >> 4);
+                    const uint32_t d = tmem_base + b * C::HC;
+                    mma_ss<0>(d, a0, w0, idesc1);
+#pragma unroll
+                    for (int kk = 1; kk < C::K1 / 16; ++kk)
+                        mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
+                                  w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
+                    mma_commit(bar(B::ACC1_FULL + b));
+                    if (c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
+                    TRACE(tr, 14);
                 }
-                mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
-                if (q_release) mma_commit(bar(B::W_EMPTY + slot));
-                if (qc == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
-                TRACE(tr, 22);
-                ++qc; ++qg;
-                if (qc == nchunks) {
-                    qc = 0; ++qt; ++qta;
-                    if (qt < t_end) q_enter(); else q_valid = false;
-                }
-                return true;
-            };
-
-            // GEMM-1 runs one chunk ahead of GEMM-2: the next accumulator is ready when the
-            // activation warps finish the current chunk.
-            ok = issue_g1();
-            while (ok && q_valid) {
-                if (h_valid) ok = issue_g1();
-                if (ok) ok = issue_g2();
+                if (reload) ++reloads;
             }
             if (!ok || *abort) {
-                // make sure no MMA is still running before TMEM is released
+                // make sure no MMA of this thread is still running before TMEM is released
                 volatile int never = 0;
                 mma_commit(bar(B::DRAIN));
                 mbar_wait(bar(B::DRAIN), 0u, &never, 10000000ull);
+            }
+        }
+    } else if (warp == 2) {
+        // ================= GEMM-2 issue ======================================================
+        if (lane == 0 && t_begin < t_end) {
+            constexpr uint32_t idesc2 = make_idesc(128, C::N2, kFmtBF16, kFmtBF16);
+            const uint32_t dW = desc_lo_sw128(sW);
+            bool ok = true;
+            TRACE_DECL(tr, 4);
+            int e = 0, prev_e = -1;
+            uint32_t g = 0, reloads = 0;
+            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+                int r0, rr;
+                locate_tile(tile_start, offs, t, e, r0, rr);
+                const bool reload = !resident || (e != prev_e);
+                prev_e = e;
+                // resident weights are handed back only when the next tile brings another expert
+                bool release = !resident;
+                if (resident && t + 1 < t_end) {
+                    int e2 = e;
+                    locate_tile(tile_start, offs, t + 1, e2, r0, rr);
+                    release = (e2 != e);
+                }
+                const int buf = ta % C::ACC2_BUFS;
+                for (int c = 0; c < nchunks; ++c, ++g) {
+                    const int slot = resident ? c : (int)(g % C::W_STAGES);
+                    if (reload) {
+                        // (already observed by the GEMM-1 thread; waited here too so that this
+                        // thread's reads of the weight tile are ordered after the copy)
+                        const uint32_t n = resident ? reloads : g / C::W_STAGES;
+                        if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    }
+                    const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
+                    TRACE(tr, 20);
+                    if (!mbar_wait(bar(B::H_FULL + b), n1 & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    TRACE(tr, 21);
+                    if (c == 0 && !mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(ta / C::ACC2_BUFS) & 1u) ^ 1u,
+                                             abort, kWaitLimitNs)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t w0 = dW + ((slot * C::W_STAGE_BYTES + C::W1C_BYTES) >> 4);
+                    const uint32_t d = tmem_base + C::ACC2_COL0 + buf * C::N2;
+                    const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: chunk; router: lo half
+                    const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi half, two runs
+#pragma unroll
+                    for (int part = 0; part < C::H_PARTS; ++part) {
+#pragma unroll
+                        for (int kk = 0; kk < C::HC / 16; ++kk) {
+                            uint32_t a;
+                            if (C::ROUTER && part == 0)
+                                a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / 2) + (kk % C::KSTEPS_PER_WG) * 8;
+                            else
+                                a = hbuf + kk * 8;
+                            const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
+                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, c > 0 ? 1u : 0u);
+                            else mma_ts<1>(d, a, bd, idesc2);
+                        }
+                    }
+                    mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
+                    if (release) mma_commit(bar(B::W_EMPTY + slot));
+                    if (c == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
+                    TRACE(tr, 22);
+                }
+                if (reload) ++reloads;
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                mma_commit(bar(B::DRAIN + 1));
+                mbar_wait(bar(B::DRAIN + 1), 0u, &never, 10000000ull);
             }
         }
     } else if (warp >= 4 && warp < C::OUT_WARP0) {
@@ -568,7 +578,49 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         bool ok = true;
         int e = 0;
         TRACE_DECL(tr, (lg == 0 && lane == 0) ? 5 : 7);
+        // Fused forward: row `row` of tile (tg, tga) is stacked row row0 + row = pair perm[.] = (n, j);
+        // its A row is bf16(gate * X[n, :]) (Eq. 1), written in the K-major 128-byte-swizzled layout.
+        int ge = 0;
+        auto gather_tile = [&](int tg, int tga) -> bool {
+            constexpr int CPR = C::K1 / 8;                       // 16-byte chunks per row
+            int row0, rows;
+            locate_tile(tile_start, offs, tg, ge, row0, rows);
+            const int ab = tga % C::A_BUFS;
+            uint4 raw[CPR];
+            float g = 0.0f;
+#pragma unroll
+            for (int i = 0; i < CPR; ++i) raw[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (row < rows) {
+                const int n = __ldg(p.perm + row0 + row) / p.gather_k;
+                g = __ldg(p.gate + row0 + row);
+                const uint4* src = reinterpret_cast<const uint4*>(p.gather_src + (size_t)n * C::K1);
+#pragma unroll
+                for (int i = 0; i < CPR; ++i) raw[i] = __ldg(src + i);
+            }
+            bool okg = mbar_wait(bar(B::A_EMPTY + ab), ((uint32_t)(tga / C::A_BUFS) & 1u) ^ 1u, abort, kWaitLimitNs);
+            okg = __all_sync(0xffffffffu, okg);
+            if (!okg) return false;
+            uint8_t* dst = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_A + ab * C::A_BYTES +
+                           (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+            for (int i = 0; i < CPR; ++i) {
+                float f[8];
+                unpack16<bf16>(raw[i], f);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) f[q] *= g;
+                *reinterpret_cast<uint4*>(dst + (i >> 3) * C::A_PANEL + (((i & 7) ^ (row & 7)) << 4)) = pack16<bf16>(f);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B::A_FULL + ab));
+            return true;
+        };
+        if (gather && t_begin < t_end) ok = gather_tile(t_begin, 0);
         for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+            if (gather && t + 1 < t_end) {
+                ok = gather_tile(t + 1, ta + 1);      // the next tile's A operand, while this tile computes
+                if (!ok) break;
+            }
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
             const int buf = ta % C::ACC2_BUFS;
@@ -749,7 +801,7 @@ int launch_tc(const void* A, uint64_t a_rows, const void* W1, const void* W2, in
 template <int K1, int ACT>
 int launch_ffn_k1(const Dims& D, const slicemoe_weights& w, const void* xperm, const TcParams& p, cudaStream_t st) {
     using C = TcCfg<K1, K1, false, ACT>;
-    return launch_tc<C>(xperm, (uint64_t)D.R, w.W1, w.W2, D.E, p, max_tiles(D), st);
+    return launch_tc<C>(xperm, (uint64_t)(p.gather_src ? D.N : D.R), w.W1, w.W2, D.E, p, max_tiles(D), st);
 }
 
 template <int K1, int E>
@@ -814,12 +866,14 @@ int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int
 }
 
 int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets, void* yperm,
-                  int32_t* status, cudaStream_t st) {
+                  int32_t* status, cudaStream_t st, const void* gather_h, const int32_t* perm, const float* gate) {
     if (D.R == 0) return SLICEMOE_OK;
     TcParams p{};
     p.offsets = offsets; p.n_rows = 0; p.E = D.E; p.HID = D.F;
     p.bias1 = (const bf16*)w.b1; p.bias2 = (const bf16*)w.b2;
     p.yperm = (bf16*)yperm; p.status = status;
+    p.gather_src = (const bf16*)gather_h; p.perm = perm; p.gate = gate; p.gather_k = D.k;
+    if (gather_h) xperm = gather_h;   // the A tensor map is not used in gather mode; any valid matrix will do
     const bool gelu = D.act == SLICEMOE_ACT_GELU_TANH;
     if (D.ds == 64)
         return gelu ? launch_ffn_k1<64, SLICEMOE_ACT_GELU_TANH>(D, w, xperm, p, st)

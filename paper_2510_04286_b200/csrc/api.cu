@@ -34,6 +34,7 @@ Workspace workspace_layout(const Dims& D) {
     W.perm = take(sizeof(int32_t) * R);
     W.gate = take(sizeof(float) * R);
     W.chunk_hist = take(sizeof(int32_t) * (size_t)num_chunks(D) * E);
+    W.cta_hist = take(sizeof(int32_t) * 256 * E);
     W.tiles = take(sizeof(int32_t) * (4 + 2 * (size_t)max_tiles(D)));
     W.xperm = take(b * R * D.ds);
     W.yperm = take(b * R * D.ds);
@@ -149,19 +150,33 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     int rc;
     if ((rc = reset_status(ws, W, st))) return rc;
     if ((rc = mark(0))) return rc;
-    if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, at<int32_t>(ws, W.status), st))) return rc;
-    if ((rc = mark(1))) return rc;
-    // With the tensor-core expert kernel the stacked rows are never materialised: dispatch only
-    // ranks the pairs (dest, perm, gate) and the kernel gathers its rows from h.
-    const bool fused_gather = tc_ffn_supported(D);
+    // With both tensor-core kernels available the stacked rows are never materialised: the router
+    // leaves its per-CTA expert counts, one dispatch kernel ranks the pairs (dest, perm, gate) and
+    // the expert kernel gathers its rows from h.
+    const bool fused = tc_route_supported(D) && tc_ffn_supported(D) && D.N > 0;
     float* gate = at<float>(ws, W.gate);
-    if ((rc = launch_dispatch(D, h, idx, p, kept, offsets, dest, perm, fused_gather ? nullptr : xperm,
-                              fused_gather ? gate : nullptr, at<int32_t>(ws, W.chunk_hist), st))) return rc;
-    if ((rc = mark(2))) return rc;
-    if (fused_gather) {
+    if (fused) {
+        int grid = 0, rows_per_cta = 0;
+        tc_route_grid(D, &grid, &rows_per_cta);
+        int32_t* cta_hist = at<int32_t>(ws, W.cta_hist);
+        if ((rc = launch_route_tc(D, w, h, idx, p, nullptr, nullptr, at<int32_t>(ws, W.status), st, cta_hist))) return rc;
+        if ((rc = mark(1))) return rc;
+        if ((rc = launch_dispatch_fused(D, idx, p, cta_hist, grid, rows_per_cta, assigned, kept, offsets, dest, perm,
+                                        gate, st))) return rc;
+        if ((rc = mark(2))) return rc;
         if ((rc = launch_ffn_tc(D, w, nullptr, offsets, yperm, at<int32_t>(ws, W.status), st, h, perm, gate))) return rc;
     } else {
-        if ((rc = ffn_any(D, w, xperm, offsets, yperm, at<int32_t>(ws, W.status), st))) return rc;
+        if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, at<int32_t>(ws, W.status), st))) return rc;
+        if ((rc = mark(1))) return rc;
+        const bool gather = tc_ffn_supported(D);
+        if ((rc = launch_dispatch(D, h, idx, p, kept, offsets, dest, perm, gather ? nullptr : xperm,
+                                  gather ? gate : nullptr, at<int32_t>(ws, W.chunk_hist), st))) return rc;
+        if ((rc = mark(2))) return rc;
+        if (gather) {
+            if ((rc = launch_ffn_tc(D, w, nullptr, offsets, yperm, at<int32_t>(ws, W.status), st, h, perm, gate))) return rc;
+        } else {
+            if ((rc = ffn_any(D, w, xperm, offsets, yperm, at<int32_t>(ws, W.status), st))) return rc;
+        }
     }
     if ((rc = mark(3))) return rc;
     if ((rc = launch_combine(D, yperm, dest, h_out, st))) return rc;

@@ -38,6 +38,7 @@ struct Workspace {
     size_t perm;        // int32[R]
     size_t gate;        // float[R]   gate value of each stacked row (fused forward)
     size_t chunk_hist;  // int32[nchunks*E]
+    size_t cta_hist;    // int32[256*E]  per-CTA expert counts of the tensor-core router (fused forward)
     size_t tiles;       // int32[4 + 2*max_tiles]  tile list of the grouped expert kernel
     size_t xperm;       // dtype[R*ds]
     size_t yperm;       // dtype[R*ds]
@@ -93,8 +94,18 @@ int launch_ffn_simt(const Dims& D, const slicemoe_weights& w, const void* xperm,
 // Tensor-core (tcgen05 / TMEM / TMA) router and grouped expert FFN, bf16 storage only.
 bool tc_route_supported(const Dims& D);
 bool tc_ffn_supported(const Dims& D);
+// assigned may be NULL (no global counts); cta_hist (int32[grid, E], see tc_route_grid) receives each
+// CTA's own counts for the fused dispatch.
 int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx,
-                    float* topk_p, int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st);
+                    float* topk_p, int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st,
+                    int32_t* cta_hist = nullptr);
+// Grid of the tensor-core router and the rows each of its CTAs routes (CTA c: rows [c*rows_per_cta, ...)).
+void tc_route_grid(const Dims& D, int* grid, int* rows_per_cta);
+// Fused dispatch after the tensor-core router: one kernel that turns the router's per-CTA counts into
+// assigned / kept / offsets and ranks every pair (dest, perm, gate); no stacked-row copy.
+int launch_dispatch_fused(const Dims& D, const int32_t* topk_idx, const float* topk_p, const int32_t* cta_hist,
+                          int grid, int rows_per_cta, int32_t* assigned, int32_t* kept, int32_t* offsets,
+                          int32_t* dest, int32_t* perm, float* gate, cudaStream_t st);
 // With gather_h != nullptr the rows are not read from xperm: row r of the stacked order is
 // bf16(gate[r] * X[perm[r] / k, :]) gathered from h inside the kernel (fused forward).
 int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets,

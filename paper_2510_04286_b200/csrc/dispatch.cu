@@ -164,6 +164,117 @@ dispatch_scatter_kernel(const T* __restrict__ X, const int32_t* __restrict__ top
     }
 }
 
+
+// Fused dispatch for the forward call.  Chunk c is the row range that CTA c of the tensor-core
+// router handled; `table[c][e]` is how many pairs of that chunk chose expert e (written by the
+// router).  Every CTA derives from the table (G x E, a few KB) the rank of its chunk's first pair
+// inside each expert, the totals, kept = min(total, C) and the offsets -- redundantly, which is
+// cheaper than a separate scan launch -- and then ranks its own pairs exactly as the scatter
+// kernel above does (per-warp counts, prefix over warps, match-any inside the warp).
+constexpr int kFusedThreads = 512;
+constexpr int kFusedWarps = kFusedThreads / 32;
+
+__global__ void __launch_bounds__(kFusedThreads)
+dispatch_fused_kernel(const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_p,
+                      const int32_t* __restrict__ table, int G, int R, int E, int k, int pairs_per_chunk,
+                      int capacity, int32_t* __restrict__ assigned, int32_t* __restrict__ kept,
+                      int32_t* __restrict__ offsets, int32_t* __restrict__ dest, int32_t* __restrict__ perm,
+                      float* __restrict__ gate) {
+    extern __shared__ int sm[];
+    int* base = sm;                  // [E]   rank of this chunk's first pair inside each expert
+    int* offs = base + E;            // [E+1]
+    int* wcnt = offs + E + 1;        // [kFusedWarps][E]
+    int* tab = wcnt + kFusedWarps * E;   // [G][E] copy of the table
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int chunk = blockIdx.x;
+
+    for (int i = threadIdx.x; i < G * E; i += kFusedThreads) tab[i] = table[i];   // coalesced
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += kFusedThreads) {
+        int before = 0, total = 0;
+        for (int c = 0; c < G; ++c) {
+            const int v = tab[c * E + e];
+            if (c < chunk) before += v;
+            total += v;
+        }
+        base[e] = before;
+        const int kp = (capacity > 0 && total > capacity) ? capacity : total;
+        wcnt[e] = kp;                // kept, scanned below
+        if (chunk == 0) {
+            if (assigned) assigned[e] = total;
+            kept[e] = kp;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int e = 0; e < E; ++e) { offs[e] = run; run += wcnt[e]; }
+        offs[E] = run;
+    }
+    __syncthreads();
+    if (chunk == 0)
+        for (int e = threadIdx.x; e <= E; e += kFusedThreads) offsets[e] = offs[e];
+    __syncthreads();
+
+    const long long chunk_begin = (long long)chunk * pairs_per_chunk;
+    long long chunk_end = chunk_begin + pairs_per_chunk;
+    if (chunk_end > R) chunk_end = R;
+    if (chunk_begin >= chunk_end) return;
+    const int npairs = (int)(chunk_end - chunk_begin);
+    const int per_warp = ((npairs + kFusedWarps - 1) / kFusedWarps + 31) / 32 * 32;   // multiple of 32
+    const int warp_begin = (int)chunk_begin + warp * per_warp;
+    const int iters = per_warp / 32;
+    int* mine = wcnt + warp * E;
+
+    for (int e = lane; e < E; e += 32) mine[e] = 0;
+    __syncthreads();                 // wcnt[0..E) was the scan scratch
+    for (int it = 0; it < iters; ++it) {
+        const int pair = warp_begin + it * 32 + lane;
+        if (pair < chunk_end) {
+            const int e = topk_idx[pair];
+            if (e >= 0 && e < E) atomicAdd(&mine[e], 1);
+        }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += kFusedThreads) {
+        int run = base[e];
+        for (int w = 0; w < kFusedWarps; ++w) {
+            const int t = wcnt[w * E + e];
+            wcnt[w * E + e] = run;
+            run += t;
+        }
+    }
+    __syncthreads();
+    for (int it = 0; it < iters; ++it) {
+        const int pair = warp_begin + it * 32 + lane;
+        int e = -1;
+        float p = 0.0f;
+        if (pair < chunk_end) {
+            e = topk_idx[pair];
+            p = topk_p[pair];
+            if (e < 0 || e >= E) e = -1;
+        }
+        const int key = e >= 0 ? e : -1 - lane;
+        const unsigned grp = __match_any_sync(0xffffffffu, key);
+        const int before = __popc(grp & ((1u << lane) - 1u));
+        int d = -1;
+        if (e >= 0) {
+            const int rank = mine[e] + before;
+            if (capacity == 0 || rank < capacity) d = offs[e] + rank;
+        }
+        __syncwarp();
+        if (e >= 0 && before == 0) mine[e] += __popc(grp);
+        __syncwarp();
+        if (pair < chunk_end) {
+            dest[pair] = d;
+            if (d >= 0) {
+                perm[d] = pair;
+                gate[d] = p;
+            }
+        }
+    }
+}
+
 }  // namespace
 
 int launch_dispatch(const Dims& D, const void* h, const int32_t* topk_idx, const float* topk_p,
@@ -189,6 +300,20 @@ int launch_dispatch(const Dims& D, const void* h, const int32_t* topk_idx, const
                 dest, perm, (float*)xperm, gate_opt);
         SLICEMOE_LAUNCH_CHECK(1);
     }
+    return SLICEMOE_OK;
+}
+
+int launch_dispatch_fused(const Dims& D, const int32_t* topk_idx, const float* topk_p, const int32_t* cta_hist,
+                          int grid, int rows_per_cta, int32_t* assigned, int32_t* kept, int32_t* offsets,
+                          int32_t* dest, int32_t* perm, float* gate, cudaStream_t st) {
+    if (grid <= 0) return SLICEMOE_ERR_SHAPE;
+    const size_t smem = sizeof(int) * ((size_t)D.E * (kFusedWarps + 2 + grid) + 1);
+    if (smem > 48 * 1024)
+        SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(dispatch_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dispatch_fused_kernel<<<grid, kFusedThreads, smem, st>>>(topk_idx, topk_p, cta_hist, grid, D.R, D.E, D.k,
+                                                            rows_per_cta * D.k, D.capacity, assigned, kept, offsets,
+                                                            dest, perm, gate);
+    SLICEMOE_LAUNCH_CHECK(1);
     return SLICEMOE_OK;
 }
 

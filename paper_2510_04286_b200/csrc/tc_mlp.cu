@@ -57,7 +57,8 @@ struct TcParams {
     int gather_k;             // k (pairs per row)
     int32_t* topk_idx;        // router outputs
     float* topk_p;
-    int32_t* assigned;
+    int32_t* assigned;        // global counts, added atomically (or nullptr)
+    int32_t* cta_hist;        // [gridDim.x, N2] this CTA's counts (or nullptr): input of the fused dispatch
     float* probs;             // or nullptr
     int k;
     int32_t* status;
@@ -709,8 +710,10 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     if (threadIdx.x == 0 && abort_flag) atomicExch(p.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
     if constexpr (C::ROUTER) {
         // per-CTA histogram -> global counts (Section 3.2's per-expert counts)
-        for (int i = threadIdx.x; i < C::N2; i += C::THREADS)
-            if (hist[i]) atomicAdd(&p.assigned[i], hist[i]);
+        for (int i = threadIdx.x; i < C::N2; i += C::THREADS) {
+            if (p.assigned && hist[i]) atomicAdd(&p.assigned[i], hist[i]);
+            if (p.cta_hist) p.cta_hist[(size_t)blockIdx.x * C::N2 + i] = hist[i];
+        }
     }
 #ifdef SLICEMOE_TC_TRACE
     if (blockIdx.x == 0 && g_trace_buf) {
@@ -848,14 +851,21 @@ bool tc_ffn_supported(const Dims& D) {
     return D.F % hc == 0 && D.F >= 2 * hc && D.F <= kMaxHid;
 }
 
+void tc_route_grid(const Dims& D, int* grid, int* rows_per_cta) {
+    const int tiles = (D.N + kTileM - 1) / kTileM;
+    const int g = tiles < sm_count() ? tiles : sm_count();
+    *grid = g;
+    *rows_per_cta = g > 0 ? ((tiles + g - 1) / g) * kTileM : 0;
+}
+
 int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx, float* topk_p,
-                    int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st) {
-    SLICEMOE_CUDA_TRY(cudaMemsetAsync(assigned, 0, sizeof(int32_t) * D.E, st));
+                    int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st, int32_t* cta_hist) {
+    if (assigned) SLICEMOE_CUDA_TRY(cudaMemsetAsync(assigned, 0, sizeof(int32_t) * D.E, st));
     if (D.N == 0) return SLICEMOE_OK;
     TcParams p{};
     p.offsets = nullptr; p.n_rows = D.N; p.E = 1; p.HID = D.Hr;
     p.bias1 = (const bf16*)w.br1; p.bias2 = (const bf16*)w.br2;
-    p.topk_idx = topk_idx; p.topk_p = topk_p; p.assigned = assigned; p.probs = probs_opt; p.k = D.k;
+    p.topk_idx = topk_idx; p.topk_p = topk_p; p.assigned = assigned; p.cta_hist = cta_hist; p.probs = probs_opt; p.k = D.k;
     p.status = status;
     switch (D.ds) {
         case 64: return launch_route_k1<64>(D, w, h, p, st);

@@ -208,7 +208,10 @@ int slicemoe_forward_host(const slicemoe_config *cfg, const slicemoe_weights *w,
  * measurement.  `events` is a HOST array of SLICEMOE_N_STAGE_EVENTS
  * cudaEvent_t handles (as void*) created by slicemoe_event_create(): event i is
  * recorded before stage i and event i+1 after it, stages being
- * 0 route, 1 dispatch, 2 expert FFN, 3 combine.
+ * 0 route, 1 dispatch, 2 expert FFN, 3 combine.  Where the library folds a
+ * stage into its neighbour (bf16 with k <= 2: the experts add their outputs
+ * straight into h', so stage 3 is empty) the two events are recorded back to
+ * back.
  */
 #define SLICEMOE_N_STAGE_EVENTS 5
 int slicemoe_forward_profiled(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,

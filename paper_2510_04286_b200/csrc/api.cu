@@ -159,12 +159,21 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
         int grid = 0, rows_per_cta = 0;
         tc_route_grid(D, &grid, &rows_per_cta);
         int32_t* cta_hist = at<int32_t>(ws, W.cta_hist);
-        if ((rc = launch_route_tc(D, w, h, idx, p, nullptr, nullptr, at<int32_t>(ws, W.status), st, cta_hist))) return rc;
+        // k <= 2: the experts add their rows straight into h' (zeroed by the router), so there is no
+        // stacked output and no combine kernel; the two-term bf16 sum is order-independent.
+        const bool scatter = D.k <= 2;
+        if ((rc = launch_route_tc(D, w, h, idx, p, nullptr, nullptr, at<int32_t>(ws, W.status), st, cta_hist,
+                                  scatter ? h_out : nullptr))) return rc;
         if ((rc = mark(1))) return rc;
         if ((rc = launch_dispatch_fused(D, idx, p, cta_hist, grid, rows_per_cta, assigned, kept, offsets, dest, perm,
                                         gate, st))) return rc;
         if ((rc = mark(2))) return rc;
-        if ((rc = launch_ffn_tc(D, w, nullptr, offsets, yperm, at<int32_t>(ws, W.status), st, h, perm, gate))) return rc;
+        if ((rc = launch_ffn_tc(D, w, nullptr, offsets, yperm, at<int32_t>(ws, W.status), st, h, perm, gate,
+                                scatter ? h_out : nullptr))) return rc;
+        if (scatter) {
+            if ((rc = mark(3))) return rc;
+            return mark(4);
+        }
     } else {
         if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, at<int32_t>(ws, W.status), st))) return rc;
         if ((rc = mark(1))) return rc;

@@ -98,7 +98,7 @@ bool tc_ffn_supported(const Dims& D);
 // CTA's own counts for the fused dispatch.
 int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx,
                     float* topk_p, int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st,
-                    int32_t* cta_hist = nullptr);
+                    int32_t* cta_hist = nullptr, void* zero_out = nullptr);
 // Grid of the tensor-core router and the rows each of its CTAs routes (CTA c: rows [c*rows_per_cta, ...)).
 void tc_route_grid(const Dims& D, int* grid, int* rows_per_cta);
 // Fused dispatch after the tensor-core router: one kernel that turns the router's per-CTA counts into
@@ -106,11 +106,15 @@ void tc_route_grid(const Dims& D, int* grid, int* rows_per_cta);
 int launch_dispatch_fused(const Dims& D, const int32_t* topk_idx, const float* topk_p, const int32_t* cta_hist,
                           int grid, int rows_per_cta, int32_t* assigned, int32_t* kept, int32_t* offsets,
                           int32_t* dest, int32_t* perm, float* gate, cudaStream_t st);
+// zero_out (router): each CTA also zeroes its rows of that [N, ds] matrix.
+// scatter_out (experts, with gather_h, k <= 2): expert outputs are added to row perm[r] / k of that
+// [N, ds] matrix (zeroed before) instead of being stored to yperm, which makes the combine step part
+// of the kernel; the sum of at most two bf16 values does not depend on the order of the additions.
 // With gather_h != nullptr the rows are not read from xperm: row r of the stacked order is
 // bf16(gate[r] * X[perm[r] / k, :]) gathered from h inside the kernel (fused forward).
 int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets,
                   void* yperm, int32_t* status, cudaStream_t st, const void* gather_h = nullptr,
-                  const int32_t* perm = nullptr, const float* gate = nullptr);
+                  const int32_t* perm = nullptr, const float* gate = nullptr, void* scatter_out = nullptr);
 
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);

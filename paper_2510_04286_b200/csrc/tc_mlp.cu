@@ -17,10 +17,12 @@
 //   warp 1            TMEM allocation + GEMM-1 issue (one lane)
 //   warp 2            GEMM-2 issue (one lane); two issuing threads because the small MMAs of this
 //                     layer (N <= 128) are issue-bound, not tensor-bound
-//   warp 3            idle (keeps every warpgroup aligned to a multiple of four warps)
-//   2 warpgroups      activation: both work on the same hidden chunk, each on half of its
-//                     columns; GEMM-1 accumulators are double-buffered so that the next chunk
-//                     is already waiting when the current one is done
+//   warp 3            router in the fused forward: zeroes this CTA's rows of h' (the experts add
+//                     into it); otherwise idle
+//   4 warpgroups      activation: all work on the same hidden chunk, each on a quarter of its
+//                     columns (16 warps hide each other's latencies); GEMM-1 accumulators are
+//                     double-buffered so that the next chunk is already waiting when the current
+//                     one is done
 //   last warpgroup    output: final accumulator -> softmax/top-k or bias + store.  In the fused
 //                     forward it also builds the next tile's A operand: each thread gathers one
 //                     row of h through perm, applies the gate of Eq. 1 and writes it swizzled
@@ -55,6 +57,11 @@ struct TcParams {
     const int32_t* perm;      // [R] pair index n*k + j of each stacked row
     const float* gate;        // [R] gate value of each stacked row
     int gather_k;             // k (pairs per row)
+    bf16* scatter_out;        // fused forward, k <= 2: h' viewed as Y[N, N2]; the row of pair (n, j) is added to
+                              // Y[n, :] (h' zeroed beforehand) instead of being stored to yperm; or nullptr
+    // router, fused forward: this CTA also zeroes the rows of zero_out that it routes
+    bf16* zero_out;           // h' viewed as Y[N, zero_cols], or nullptr
+    int zero_cols;
     int32_t* topk_idx;        // router outputs
     float* topk_p;
     int32_t* assigned;        // global counts, added atomically (or nullptr)
@@ -102,7 +109,7 @@ struct TcCfg {
     static constexpr int HC = (K1 == 64) ? 128 : 64;           // hidden units per chunk
     static constexpr int A_BUFS = (K1 <= 128) ? 2 : 1;
     static constexpr int W_STAGES = (K1 == 128) ? 3 : 2;
-    static constexpr int NWG = 2;                               // activation warpgroups (column split)
+    static constexpr int NWG = 4;                               // activation warpgroups (column split)
     static constexpr int NBUF = 2;                              // GEMM-1 accumulator / hidden buffers
     static constexpr int ACT_WARPS = NWG * 4;
     static constexpr int THREADS = 128 + NWG * 128 + 128;
@@ -117,10 +124,10 @@ struct TcCfg {
     static constexpr int H_PARTS = ROUTER_ ? 2 : 1;
     static constexpr bool PACKED_ACT = !ROUTER_;
     // TMEM columns:
-    //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w owns columns [w HC/2, (w+1) HC/2)
-    //                        of each.  Router: once a thread has read a 32-column piece it writes
-    //                        the piece's hi half (16 packed columns) over the start of its own
-    //                        column range, so the chunk's hi half ends up in two runs of HC/4.
+    //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w owns columns [w HC/4, (w+1) HC/4)
+    //                        of each.  Router: once a thread has read a 16-column piece it writes
+    //                        the piece's hi half (8 packed columns) over the start of its own
+    //                        column range, so the chunk's hi half ends up in four runs of HC/8.
     //   [2 HC, 3 HC)         two hidden buffers of HC/2 packed columns: the experts' hidden chunk
     //                        (so GEMM-1 of a later chunk need not wait for GEMM-2), or the
     //                        router's lo half.
@@ -128,7 +135,7 @@ struct TcCfg {
     static constexpr int H_COL0 = NBUF * HC;
     static constexpr int ACC2_COL0 = H_COL0 + NBUF * (HC / 2);
     static constexpr int TMEM_COLS = pow2_at_least(ACC2_COL0 + ACC2_BUFS * N2);
-    static constexpr int KSTEPS_PER_WG = HC / 32;               // 16-element K steps in one warpgroup's half
+    static constexpr int KSTEPS_PER_WG = HC / (16 * NWG);       // 16-element K steps in one warpgroup's columns
     static constexpr int KP1 = K1 / 64;                         // 64-wide K panels of GEMM-1
     static constexpr int KP2 = HC / 64;                         // K panels of GEMM-2 per chunk
     static constexpr int A_PANEL = 128 * 128;                   // bytes: 128 rows x 128 B
@@ -143,7 +150,9 @@ struct TcCfg {
     static constexpr int SMEM_BYTES = OFF_W + W_STAGES * W_STAGE_BYTES;
     // at least 120 KiB is requested so that two CTAs never share an SM (each allocates most of TMEM)
     static constexpr int SMEM_ALLOC = (SMEM_BYTES + 1024 > 120 * 1024) ? SMEM_BYTES + 1024 : 120 * 1024;
-    static constexpr int NPIECE = HC / (32 * NWG);              // 32-column pieces per thread and chunk
+    static constexpr int PIECE = 16;                            // accumulator columns per piece
+    static constexpr int NPIECE = HC / (PIECE * NWG);           // pieces per thread and chunk
+    static_assert(NPIECE >= 1, "hidden chunk too narrow for the activation warpgroups");
     static_assert(W_STAGE_BYTES % 1024 == 0 && W1C_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
     static_assert(N2 % 16 == 0 && N2 >= 16 && N2 <= 256, "MMA N");
     static_assert(SMEM_ALLOC <= 232448, "shared memory budget");
@@ -181,22 +190,26 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// 32 fp32 pre-activations (one thread's piece of a row) -> 16 packed bf16 activation pairs, all
+// 16 fp32 pre-activations (one thread's piece of a row) -> 8 packed bf16 activation pairs, all
 // arithmetic 2-wide in bf16: one conversion, five packed multiply-adds and one packed tanh per
 // pair.  GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))).  Where z^2 overflows,
 // tanh saturates to +-1 and the formula still returns z (z > 0) or 0 (z < 0).
-// The tanh unit (16 results per clock per SM) is the scarce resource, so the piece is processed
-// in groups of four pairs, staggered: while one group's tanh is in flight the multiply-adds
-// before the next group's tanh and after the previous group's are issued.
+// The tanh unit (16 results per clock per SM) is the scarce resource; 16 activation warps keep it
+// fed while the others convert, multiply and store.
 template <int ACT>
 __device__ __forceinline__ void activate_piece_bf16x2(const uint32_t* cur, uint32_t* out) {
-    __nv_bfloat162 z[16];
+    constexpr int P = 8;   // column pairs per piece
+    __nv_bfloat162 z[P];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) z[i] = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+    for (int i = 0; i < P; ++i) z[i] = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+#ifdef SLICEMOE_TC_SKELETON   // development: time the pipeline without the activation math
+    if (true) {
+#else
     if (ACT == SLICEMOE_ACT_RELU) {
+#endif
         const __nv_bfloat162 zero = __float2bfloat162_rn(0.0f);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < P; ++i) {
             const __nv_bfloat162 r = __hmax2(z[i], zero);
             out[i] = *reinterpret_cast<const uint32_t*>(&r);
         }
@@ -204,50 +217,39 @@ __device__ __forceinline__ void activate_piece_bf16x2(const uint32_t* cur, uint3
     }
     const __nv_bfloat162 c0 = __float2bfloat162_rn(0.7978845608f), c1 = __float2bfloat162_rn(0.0356774081f);
     const __nv_bfloat162 half = __float2bfloat162_rn(0.5f);
-    __nv_bfloat162 t[16];
-    auto pre_tanh = [&](int g0) {
+    __nv_bfloat162 t[P];
 #pragma unroll
-        for (int i = g0; i < g0 + 4; ++i) {
-            const __nv_bfloat162 inner = __hfma2(__hmul2(z[i], z[i]), c1, c0);
-            const __nv_bfloat162 u = __hmul2(z[i], inner);
-            uint32_t ur = *reinterpret_cast<const uint32_t*>(&u), tr;
-            asm volatile("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
-            t[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
-        }
-    };
-    auto post = [&](int g0) {
+    for (int i = 0; i < P; ++i) {
+        const __nv_bfloat162 inner = __hfma2(__hmul2(z[i], z[i]), c1, c0);
+        const __nv_bfloat162 u = __hmul2(z[i], inner);
+        uint32_t ur = *reinterpret_cast<const uint32_t*>(&u), tr;
+        asm("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
+        t[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
+    }
 #pragma unroll
-        for (int i = g0; i < g0 + 4; ++i) {
-            const __nv_bfloat162 hz = __hmul2(z[i], half);
-            const __nv_bfloat162 r = __hfma2(hz, t[i], hz);
-            out[i] = *reinterpret_cast<const uint32_t*>(&r);
-        }
-    };
-    pre_tanh(0);
-    pre_tanh(4);
-    post(0);
-    pre_tanh(8);
-    post(4);
-    pre_tanh(12);
-    post(8);
-    post(12);
+    for (int i = 0; i < P; ++i) {
+        const __nv_bfloat162 hz = __hmul2(z[i], half);
+        const __nv_bfloat162 r = __hfma2(hz, t[i], hz);
+        out[i] = *reinterpret_cast<const uint32_t*>(&r);
+    }
 }
 
 // Router: ReLU in fp32, then each value as a bf16 pair, the rounded value (hi) and the rounded
 // remainder (lo); hi + lo carries 16 mantissa bits of the fp32 value.
 __device__ __forceinline__ void relu_split_piece(const uint32_t* cur, uint32_t* hi, uint32_t* lo) {
-    float a[32];
+    constexpr int P = 8;
+    float a[2 * P];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) a[i] = fmaxf(__uint_as_float(cur[i]), 0.0f);
+    for (int i = 0; i < 2 * P; ++i) a[i] = fmaxf(__uint_as_float(cur[i]), 0.0f);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) hi[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+    for (int i = 0; i < P; ++i) hi[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < P; ++i) {
         a[2 * i] -= __uint_as_float(hi[i] << 16);
         a[2 * i + 1] -= __uint_as_float(hi[i] & 0xFFFF0000u);
     }
 #pragma unroll
-    for (int i = 0; i < 16; ++i) lo[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+    for (int i = 0; i < P; ++i) lo[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
 }
 
 template <class C>
@@ -474,7 +476,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         for (int kk = 0; kk < C::HC / 16; ++kk) {
                             uint32_t a;
                             if (C::ROUTER && part == 0)
-                                a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / 2) + (kk % C::KSTEPS_PER_WG) * 8;
+                                a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / C::NWG) + (kk % C::KSTEPS_PER_WG) * 8;
                             else
                                 a = hbuf + kk * 8;
                             const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
@@ -493,6 +495,19 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 volatile int never = 0;
                 mma_commit(bar(B::DRAIN + 1));
                 mbar_wait(bar(B::DRAIN + 1), 0u, &never, 10000000ull);
+            }
+        }
+    } else if (warp == 3) {
+        // ================= zero this CTA's rows of h' (router, fused forward) ================
+        if constexpr (C::ROUTER) {
+            if (p.zero_out != nullptr && t_begin < t_end) {
+                const long long row_lo = (long long)t_begin * kTileM;
+                long long row_hi = (long long)t_end * kTileM;
+                if (row_hi > p.n_rows) row_hi = p.n_rows;
+                uint4* dst = reinterpret_cast<uint4*>(p.zero_out + row_lo * p.zero_cols);
+                const long long nvec = (row_hi - row_lo) * p.zero_cols / 8;
+                const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                for (long long i = lane; i < nvec; i += 32) dst[i] = z;
             }
         }
     } else if (warp >= 4 && warp < C::OUT_WARP0) {
@@ -518,15 +533,15 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (!ok) break;
                 TRACE(tr, 31);
                 tc_fence_after_sync();
-                uint32_t v[2][32];
-                tmem_ld_x32(acc1, v[0]);
+                uint32_t v[2][C::PIECE];
+                tmem_ld_x16(acc1, v[0]);
 #pragma unroll
                 for (int pc = 0; pc < C::NPIECE; ++pc) {
                     uint32_t* cur = v[pc & 1];
                     tmem_ld_wait();
                     TRACE(tr, 32);
                     if (pc + 1 < C::NPIECE) {
-                        tmem_ld_x32(acc1 + (pc + 1) * 32, v[(pc + 1) & 1]);   // overlaps the math below
+                        tmem_ld_x16(acc1 + (pc + 1) * C::PIECE, v[(pc + 1) & 1]);   // overlaps the math below
                     } else if constexpr (!C::ROUTER) {
                         // the accumulator is in registers: GEMM-1 of a later chunk may overwrite it
                         tc_fence_before_sync();
@@ -535,18 +550,16 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     }
                     if (p.bias1) {
                         // same address for the whole warp: one broadcast load per 8 columns
-                        const bf16* gb = p.bias1 + (size_t)e * p.HID + c * C::HC + w * WCOLS + pc * 32;
+                        const bf16* gb = p.bias1 + (size_t)e * p.HID + c * C::HC + w * WCOLS + pc * C::PIECE;
 #pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
+                        for (int j = 0; j < C::PIECE; j += 8) {
                             float bb[8];
                             unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(gb + j)), bb);
 #pragma unroll
                             for (int i = 0; i < 8; ++i) cur[j + i] = __float_as_uint(__uint_as_float(cur[j + i]) + bb[i]);
                         }
                     }
-                    // The 16 column pairs of the piece go through every step together, so that
-                    // each step is 16 independent instructions.
-                    uint32_t hi[16];
+                    uint32_t hi[C::PIECE / 2];
                     if constexpr (C::PACKED_ACT) {
                         activate_piece_bf16x2<C::ACT>(cur, hi);
                         if (pc == 0) {
@@ -554,12 +567,12 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
                             ok = __all_sync(0xffffffffu, ok);
                         }
-                        if (ok) tmem_st_x16(hdst + pc * 16, hi);
+                        if (ok) tmem_st_x8(hdst + pc * (C::PIECE / 2), hi);
                     } else {
-                        uint32_t lo[16];
+                        uint32_t lo[C::PIECE / 2];
                         relu_split_piece(cur, hi, lo);
-                        tmem_st_x16(acc1 + pc * 16, hi);     // over columns this thread has already read
-                        tmem_st_x16(hdst + pc * 16, lo);
+                        tmem_st_x8(acc1 + pc * (C::PIECE / 2), hi);     // over columns this thread has already read
+                        tmem_st_x8(hdst + pc * (C::PIECE / 2), lo);
                     }
                     TRACE(tr, 33);
                 }
@@ -582,6 +595,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         // Fused forward: row `row` of tile (tg, tga) is stacked row row0 + row = pair perm[.] = (n, j);
         // its A row is bf16(gate * X[n, :]) (Eq. 1), written in the K-major 128-byte-swizzled layout.
         int ge = 0;
+        int n_next = -1, n_cur = -1;          // source row (of X / Y) of this thread's row: next tile, current tile
         auto gather_tile = [&](int tg, int tga) -> bool {
             constexpr int CPR = C::K1 / 8;                       // 16-byte chunks per row
             int row0, rows;
@@ -589,10 +603,12 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             const int ab = tga % C::A_BUFS;
             uint4 raw[CPR];
             float g = 0.0f;
+            n_next = -1;
 #pragma unroll
             for (int i = 0; i < CPR; ++i) raw[i] = make_uint4(0u, 0u, 0u, 0u);
             if (row < rows) {
                 const int n = __ldg(p.perm + row0 + row) / p.gather_k;
+                n_next = n;
                 g = __ldg(p.gate + row0 + row);
                 const uint4* src = reinterpret_cast<const uint4*>(p.gather_src + (size_t)n * C::K1);
 #pragma unroll
@@ -618,6 +634,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         };
         if (gather && t_begin < t_end) ok = gather_tile(t_begin, 0);
         for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+            n_cur = n_next;
             if (gather && t + 1 < t_end) {
                 ok = gather_tile(t + 1, ta + 1);      // the next tile's A operand, while this tile computes
                 if (!ok) break;
@@ -683,7 +700,8 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                                  __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
                 }
             } else {
-                bf16* dst = p.yperm + (size_t)(row0 + row) * C::N2;
+                const bool scatter = gather && p.scatter_out != nullptr;
+                bf16* dst = scatter ? p.scatter_out + (size_t)n_cur * C::N2 : p.yperm + (size_t)(row0 + row) * C::N2;
 #pragma unroll
                 for (int q = 0; q < C::N2 / 8; ++q) {
                     float bb[8];
@@ -698,7 +716,8 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     for (int i = 0; i < 4; ++i)
                         o[i] = pack_bf16x2(__uint_as_float(v[q * 8 + 2 * i]) + bb[2 * i],
                                            __uint_as_float(v[q * 8 + 2 * i + 1]) + bb[2 * i + 1]);
-                    *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                    if (scatter) red_add_bf16x8(dst + q * 8, o[0], o[1], o[2], o[3]);   // sum over the row's k experts
+                    else *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
         }
@@ -859,7 +878,8 @@ void tc_route_grid(const Dims& D, int* grid, int* rows_per_cta) {
 }
 
 int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx, float* topk_p,
-                    int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st, int32_t* cta_hist) {
+                    int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st, int32_t* cta_hist,
+                    void* zero_out) {
     if (assigned) SLICEMOE_CUDA_TRY(cudaMemsetAsync(assigned, 0, sizeof(int32_t) * D.E, st));
     if (D.N == 0) return SLICEMOE_OK;
     TcParams p{};
@@ -867,6 +887,7 @@ int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int
     p.bias1 = (const bf16*)w.br1; p.bias2 = (const bf16*)w.br2;
     p.topk_idx = topk_idx; p.topk_p = topk_p; p.assigned = assigned; p.cta_hist = cta_hist; p.probs = probs_opt; p.k = D.k;
     p.status = status;
+    p.zero_out = (bf16*)zero_out; p.zero_cols = D.ds;
     switch (D.ds) {
         case 64: return launch_route_k1<64>(D, w, h, p, st);
         case 128: return launch_route_k1<128>(D, w, h, p, st);
@@ -876,13 +897,15 @@ int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int
 }
 
 int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets, void* yperm,
-                  int32_t* status, cudaStream_t st, const void* gather_h, const int32_t* perm, const float* gate) {
+                  int32_t* status, cudaStream_t st, const void* gather_h, const int32_t* perm, const float* gate,
+                  void* scatter_out) {
     if (D.R == 0) return SLICEMOE_OK;
     TcParams p{};
     p.offsets = offsets; p.n_rows = 0; p.E = D.E; p.HID = D.F;
     p.bias1 = (const bf16*)w.b1; p.bias2 = (const bf16*)w.b2;
     p.yperm = (bf16*)yperm; p.status = status;
     p.gather_src = (const bf16*)gather_h; p.perm = perm; p.gate = gate; p.gather_k = D.k;
+    p.scatter_out = gather_h ? (bf16*)scatter_out : nullptr;
     if (gather_h) xperm = gather_h;   // the A tensor map is not used in gather mode; any valid matrix will do
     const bool gelu = D.act == SLICEMOE_ACT_GELU_TANH;
     if (D.ds == 64)

@@ -160,8 +160,10 @@ def test_profiled_forward_records_stage_times():
     before = binding.slicemoe_launch_count()
     binding.slicemoe_forward_profiled(gpu.cfg, gpu.w, gpu.h, h_out, gpu.ws, ev)
     ms = ev.stage_ms()
-    assert len(ms) == 4 and all(m > 0 for m in ms)
-    assert binding.slicemoe_launch_count() - before >= 4
+    # route, dispatch and the expert kernel always run; with k <= 2 on the tensor-core path the
+    # combine step is folded into the expert kernel and its stage is empty
+    assert len(ms) == 4 and all(m > 0 for m in ms[:3]) and ms[3] >= 0
+    assert binding.slicemoe_launch_count() - before >= 3
     assert torch.equal(h_out, gpu.forward()[0])
 
 

@@ -24,7 +24,7 @@ Workspace workspace_layout(const Dims& D) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + (bytes ? bytes : 1)); return at; };
     const size_t R = (size_t)D.R, E = (size_t)D.E, b = elem_bytes(D);
-    W.status = take(sizeof(int32_t) * 64);
+    W.status = take(sizeof(int32_t) * 256);
     W.topk_idx = take(sizeof(int32_t) * R);
     W.topk_p = take(sizeof(float) * R);
     W.assigned = take(sizeof(int32_t) * E);

@@ -28,7 +28,7 @@ constexpr int kTileM = 128;
 
 // Sub-buffers of the caller's workspace (byte offsets, each 256-byte aligned).
 struct Workspace {
-    size_t status;      // int32[64]: [0] device status word
+    size_t status;      // int32[256]: [0] device status word (the rest is spare, used by development builds)
     size_t topk_idx;    // int32[R]
     size_t topk_p;      // float[R]
     size_t assigned;    // int32[E]

@@ -107,7 +107,7 @@ struct TcCfg {
     static constexpr int K1 = K1_, N2 = N2_, ACT = ACT_;
     static constexpr bool ROUTER = ROUTER_;
     static constexpr int HC = (K1 == 64) ? 128 : 64;           // hidden units per chunk
-    static constexpr int A_BUFS = (K1 <= 128) ? 2 : 1;
+    static constexpr int A_BUFS = (K1 <= 128) ? 3 : 1;          // three: the fused forward gathers two tiles ahead
     static constexpr int W_STAGES = (K1 == 128) ? 3 : 2;
     static constexpr int NWG = 4;                               // activation warpgroups (column split)
     static constexpr int NBUF = 2;                              // GEMM-1 accumulator / hidden buffers
@@ -412,10 +412,12 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W_STAGE_BYTES) >> 4);
                     const uint32_t d = tmem_base + b * C::HC;
                     mma_ss<0>(d, a0, w0, idesc1);
+#ifndef SLICEMOE_DEV_G1_ONE   // development: time the pipeline with a single GEMM-1 MMA per chunk
 #pragma unroll
                     for (int kk = 1; kk < C::K1 / 16; ++kk)
                         mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
                                   w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
+#endif
                     mma_commit(bar(B::ACC1_FULL + b));
                     if (c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
                     TRACE(tr, 14);
@@ -481,7 +483,9 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 a = hbuf + kk * 8;
                             const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
                             if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, c > 0 ? 1u : 0u);
+#ifndef SLICEMOE_DEV_G2_ONE   // development: time the pipeline with a single GEMM-2 MMA per chunk
                             else mma_ts<1>(d, a, bd, idesc2);
+#endif
                         }
                     }
                     mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
@@ -520,6 +524,14 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         int e = 0;
         uint32_t g = 0;
         TRACE_DECL(tr, (lg == 0 && lane == 0) ? 2 + w : 7);
+#ifdef SLICEMOE_TC_ACCT   // development: where do the activation warps spend their cycles?
+        long long acct_wait_acc1 = 0, acct_wait_hempty = 0, acct_stwait = 0, acct_t0 = clock64(), acct_mark;
+#define ACCT_BEGIN() acct_mark = clock64()
+#define ACCT_END(var) var += clock64() - acct_mark
+#else
+#define ACCT_BEGIN()
+#define ACCT_END(var)
+#endif
         for (int t = t_begin; t < t_end && ok; ++t) {
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
@@ -528,8 +540,10 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const uint32_t acc1 = lane_base + b * C::HC + w * WCOLS;               // my accumulator columns
                 const uint32_t hdst = lane_base + C::H_COL0 + b * (C::HC / 2) + w * (WCOLS / 2);
                 TRACE(tr, 30);
+                ACCT_BEGIN();
                 ok = mbar_wait(bar(B::ACC1_FULL + b), n1 & 1u, abort, kWaitLimitNs);
                 ok = __all_sync(0xffffffffu, ok);
+                ACCT_END(acct_wait_acc1);
                 if (!ok) break;
                 TRACE(tr, 31);
                 tc_fence_after_sync();
@@ -564,8 +578,10 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         activate_piece_bf16x2<C::ACT>(cur, hi);
                         if (pc == 0) {
                             // GEMM-2 of two chunks ago must be done with this hidden buffer
+                            ACCT_BEGIN();
                             ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
                             ok = __all_sync(0xffffffffu, ok);
+                            ACCT_END(acct_wait_hempty);
                         }
                         if (ok) tmem_st_x8(hdst + pc * (C::PIECE / 2), hi);
                     } else {
@@ -577,13 +593,21 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     TRACE(tr, 33);
                 }
                 if (!ok) break;
+                ACCT_BEGIN();
                 tmem_st_wait();
+                ACCT_END(acct_stwait);
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B::H_FULL + b));
                 TRACE(tr, 35);
             }
         }
+#ifdef SLICEMOE_TC_ACCT
+        if (lane == 0 && p.status != nullptr && blockIdx.x == 0) {
+            long long* out = reinterpret_cast<long long*>(p.status + 16) + (warp - 4) * 4;   // status area: int32[64] -> spill past it
+            out[0] = clock64() - acct_t0; out[1] = acct_wait_acc1; out[2] = acct_wait_hempty; out[3] = acct_stwait;
+        }
+#endif
     } else if (warp >= C::OUT_WARP0) {
         // ================= output warpgroup ==================================================
         const int lg = warp & 3;
@@ -595,7 +619,8 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         // Fused forward: row `row` of tile (tg, tga) is stacked row row0 + row = pair perm[.] = (n, j);
         // its A row is bf16(gate * X[n, :]) (Eq. 1), written in the K-major 128-byte-swizzled layout.
         int ge = 0;
-        int n_next = -1, n_cur = -1;          // source row (of X / Y) of this thread's row: next tile, current tile
+        // source row (of X / Y) of this thread's row in the tile being output and the two gathered ahead
+        int n_cur = -1, n_ahead1 = -1, n_ahead2 = -1, n_next = -1;
         auto gather_tile = [&](int tg, int tga) -> bool {
             constexpr int CPR = C::K1 / 8;                       // 16-byte chunks per row
             int row0, rows;
@@ -632,12 +657,20 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             if (lane == 0) mbar_arrive(bar(B::A_FULL + ab));
             return true;
         };
-        if (gather && t_begin < t_end) ok = gather_tile(t_begin, 0);
+        constexpr int AHEAD = C::A_BUFS - 1;   // tiles gathered ahead of the one being output
+        if (gather) {
+            for (int i = 0; i < AHEAD && ok && t_begin + i < t_end; ++i) {
+                ok = gather_tile(t_begin + i, i);
+                if (i == 0) n_ahead1 = n_next; else n_ahead2 = n_next;
+            }
+        }
         for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
-            n_cur = n_next;
-            if (gather && t + 1 < t_end) {
-                ok = gather_tile(t + 1, ta + 1);      // the next tile's A operand, while this tile computes
+            n_cur = n_ahead1;
+            n_ahead1 = n_ahead2;
+            if (gather && t + AHEAD < t_end) {
+                ok = gather_tile(t + AHEAD, ta + AHEAD);      // a later tile's A operand, while this one computes
                 if (!ok) break;
+                if (AHEAD == 1) n_ahead1 = n_next; else n_ahead2 = n_next;
             }
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
@@ -700,6 +733,9 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                                  __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
                 }
             } else {
+#ifdef SLICEMOE_DEV_NO_OUT    // development: time the pipeline without the output stores
+                if (true) continue;
+#endif
                 const bool scatter = gather && p.scatter_out != nullptr;
                 bf16* dst = scatter ? p.scatter_out + (size_t)n_cur * C::N2 : p.yperm + (size_t)(row0 + row) * C::N2;
 #pragma unroll

@@ -107,9 +107,14 @@ struct TcCfg {
     static constexpr int K1 = K1_, N2 = N2_, ACT = ACT_;
     static constexpr bool ROUTER = ROUTER_;
     static constexpr int HC = (K1 == 64) ? 128 : 64;           // hidden units per chunk
-    static constexpr int A_BUFS = (K1 <= 128) ? 3 : 1;          // three: the fused forward gathers two tiles ahead
+    // row-tile buffers: three where they fit (the fused forward gathers two tiles ahead); with
+    // 256-wide rows (64 KB per tile) the router gets two and the experts, whose weight stages are
+    // larger, one
+    static constexpr int A_BUFS = (K1 <= 128) ? 3 : (ROUTER_ ? 2 : 1);
     static constexpr int W_STAGES = (K1 == 128) ? 3 : 2;
-    static constexpr int NWG = 4;                               // activation warpgroups (column split)
+    // activation warpgroups (column split); two for 256-wide rows, whose wide output epilogue needs
+    // the larger register budget of a 512-thread CTA
+    static constexpr int NWG = (K1 == 256) ? 2 : 4;
     static constexpr int NBUF = 2;                              // GEMM-1 accumulator / hidden buffers
     static constexpr int ACT_WARPS = NWG * 4;
     static constexpr int THREADS = 128 + NWG * 128 + 128;
@@ -532,6 +537,13 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #define ACCT_BEGIN()
 #define ACCT_END(var)
 #endif
+#ifdef SLICEMOE_TC_PROBE   // development: clock stamps inside one chunk (g == 12) of one warp
+        unsigned probe[16];
+        for (int i = 0; i < 16; ++i) probe[i] = 0;
+#define PROBE(i) do { if (g == 12) probe[i] = (unsigned)clock(); } while (0)
+#else
+#define PROBE(i)
+#endif
         for (int t = t_begin; t < t_end && ok; ++t) {
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
@@ -540,19 +552,23 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const uint32_t acc1 = lane_base + b * C::HC + w * WCOLS;               // my accumulator columns
                 const uint32_t hdst = lane_base + C::H_COL0 + b * (C::HC / 2) + w * (WCOLS / 2);
                 TRACE(tr, 30);
+                PROBE(0);
                 ACCT_BEGIN();
                 ok = mbar_wait(bar(B::ACC1_FULL + b), n1 & 1u, abort, kWaitLimitNs);
                 ok = __all_sync(0xffffffffu, ok);
                 ACCT_END(acct_wait_acc1);
                 if (!ok) break;
                 TRACE(tr, 31);
+                PROBE(1);
                 tc_fence_after_sync();
                 uint32_t v[2][C::PIECE];
                 tmem_ld_x16(acc1, v[0]);
+                PROBE(2);
 #pragma unroll
                 for (int pc = 0; pc < C::NPIECE; ++pc) {
                     uint32_t* cur = v[pc & 1];
                     tmem_ld_wait();
+                    PROBE(3 + pc * 5);
                     TRACE(tr, 32);
                     if (pc + 1 < C::NPIECE) {
                         tmem_ld_x16(acc1 + (pc + 1) * C::PIECE, v[(pc + 1) & 1]);   // overlaps the math below
@@ -562,6 +578,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
                     }
+                    PROBE(4 + pc * 5);
                     if (p.bias1) {
                         // same address for the whole warp: one broadcast load per 8 columns
                         const bf16* gb = p.bias1 + (size_t)e * p.HID + c * C::HC + w * WCOLS + pc * C::PIECE;
@@ -576,6 +593,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     uint32_t hi[C::PIECE / 2];
                     if constexpr (C::PACKED_ACT) {
                         activate_piece_bf16x2<C::ACT>(cur, hi);
+                        PROBE(5 + pc * 5);
                         if (pc == 0) {
                             // GEMM-2 of two chunks ago must be done with this hidden buffer
                             ACCT_BEGIN();
@@ -583,7 +601,9 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             ok = __all_sync(0xffffffffu, ok);
                             ACCT_END(acct_wait_hempty);
                         }
+                        PROBE(6 + pc * 5);
                         if (ok) tmem_st_x8(hdst + pc * (C::PIECE / 2), hi);
+                        PROBE(7 + pc * 5);
                     } else {
                         uint32_t lo[C::PIECE / 2];
                         relu_split_piece(cur, hi, lo);
@@ -596,12 +616,20 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 ACCT_BEGIN();
                 tmem_st_wait();
                 ACCT_END(acct_stwait);
+                PROBE(13);
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B::H_FULL + b));
+                PROBE(14);
                 TRACE(tr, 35);
             }
         }
+#ifdef SLICEMOE_TC_PROBE
+        if (lane == 0 && p.status != nullptr && blockIdx.x == 0 && !C::ROUTER) {
+            unsigned* out = reinterpret_cast<unsigned*>(p.status + 16) + (warp - 4) * 16;
+            for (int i = 0; i < 16; ++i) out[i] = probe[i];
+        }
+#endif
 #ifdef SLICEMOE_TC_ACCT
         if (lane == 0 && p.status != nullptr && blockIdx.x == 0) {
             long long* out = reinterpret_cast<long long*>(p.status + 16) + (warp - 4) * 4;   // status area: int32[64] -> spill past it
@@ -619,38 +647,45 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         // Fused forward: row `row` of tile (tg, tga) is stacked row row0 + row = pair perm[.] = (n, j);
         // its A row is bf16(gate * X[n, :]) (Eq. 1), written in the K-major 128-byte-swizzled layout.
         int ge = 0;
-        // source row (of X / Y) of this thread's row in the tile being output and the two gathered ahead
-        int n_cur = -1, n_ahead1 = -1, n_ahead2 = -1, n_next = -1;
+        int n_of[3] = {-1, -1, -1};           // source row (of X / Y) of this thread's row, per tile in flight
         auto gather_tile = [&](int tg, int tga) -> bool {
             constexpr int CPR = C::K1 / 8;                       // 16-byte chunks per row
+            constexpr int GB = 8;                                // chunks per block (registers)
             int row0, rows;
             locate_tile(tile_start, offs, tg, ge, row0, rows);
             const int ab = tga % C::A_BUFS;
-            uint4 raw[CPR];
             float g = 0.0f;
-            n_next = -1;
-#pragma unroll
-            for (int i = 0; i < CPR; ++i) raw[i] = make_uint4(0u, 0u, 0u, 0u);
+            int n = -1;
             if (row < rows) {
-                const int n = __ldg(p.perm + row0 + row) / p.gather_k;
-                n_next = n;
+                n = __ldg(p.perm + row0 + row) / p.gather_k;
                 g = __ldg(p.gate + row0 + row);
-                const uint4* src = reinterpret_cast<const uint4*>(p.gather_src + (size_t)n * C::K1);
-#pragma unroll
-                for (int i = 0; i < CPR; ++i) raw[i] = __ldg(src + i);
             }
+            n_of[tga % 3] = n;
+            const uint4* src = reinterpret_cast<const uint4*>(p.gather_src + (size_t)(n < 0 ? 0 : n) * C::K1);
+            uint4 raw[GB];
+#pragma unroll
+            for (int i = 0; i < GB; ++i) raw[i] = (n >= 0) ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
             bool okg = mbar_wait(bar(B::A_EMPTY + ab), ((uint32_t)(tga / C::A_BUFS) & 1u) ^ 1u, abort, kWaitLimitNs);
             okg = __all_sync(0xffffffffu, okg);
             if (!okg) return false;
             uint8_t* dst = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_A + ab * C::A_BYTES +
                            (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
-            for (int i = 0; i < CPR; ++i) {
-                float f[8];
-                unpack16<bf16>(raw[i], f);
+            for (int blk = 0; blk < CPR / GB; ++blk) {
 #pragma unroll
-                for (int q = 0; q < 8; ++q) f[q] *= g;
-                *reinterpret_cast<uint4*>(dst + (i >> 3) * C::A_PANEL + (((i & 7) ^ (row & 7)) << 4)) = pack16<bf16>(f);
+                for (int i = 0; i < GB; ++i) {
+                    float f[8];
+                    unpack16<bf16>(raw[i], f);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) f[q] *= g;
+                    // chunk blk*8 + i of the row lives in panel blk (64 columns), 16-byte slot i
+                    *reinterpret_cast<uint4*>(dst + blk * C::A_PANEL + ((i ^ (row & 7)) << 4)) = pack16<bf16>(f);
+                }
+                if (blk + 1 < CPR / GB) {
+#pragma unroll
+                    for (int i = 0; i < GB; ++i)
+                        raw[i] = (n >= 0) ? __ldg(src + (blk + 1) * GB + i) : make_uint4(0u, 0u, 0u, 0u);
+                }
             }
             fence_proxy_async_smem();
             __syncwarp();
@@ -659,19 +694,14 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         };
         constexpr int AHEAD = C::A_BUFS - 1;   // tiles gathered ahead of the one being output
         if (gather) {
-            for (int i = 0; i < AHEAD && ok && t_begin + i < t_end; ++i) {
-                ok = gather_tile(t_begin + i, i);
-                if (i == 0) n_ahead1 = n_next; else n_ahead2 = n_next;
-            }
+            for (int i = 0; i < AHEAD && ok && t_begin + i < t_end; ++i) ok = gather_tile(t_begin + i, i);
         }
         for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
-            n_cur = n_ahead1;
-            n_ahead1 = n_ahead2;
             if (gather && t + AHEAD < t_end) {
-                ok = gather_tile(t + AHEAD, ta + AHEAD);      // a later tile's A operand, while this one computes
-                if (!ok) break;
-                if (AHEAD == 1) n_ahead1 = n_next; else n_ahead2 = n_next;
+                ok = gather_tile(t + AHEAD, ta + AHEAD);      // a later tile's A operand (this tile's when there
+                if (!ok) break;                               // is only one buffer), while the tensor core works
             }
+            const int n_cur = n_of[ta % 3];
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
             const int buf = ta % C::ACC2_BUFS;
@@ -682,17 +712,17 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             TRACE(tr, 41);
             tc_fence_after_sync();
             const uint32_t acc2 = tmem_lane + C::ACC2_COL0 + buf * C::N2;
-            uint32_t v[C::N2];
-#pragma unroll
-            for (int q = 0; q < C::N2 / 16; ++q) tmem_ld_x16(acc2 + q * 16, v + q * 16);
-            tmem_ld_wait();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
-            TRACE(tr, 42);
-            if (row >= rows) continue;
             if constexpr (C::ROUTER) {
                 constexpr int E = C::N2;
+                uint32_t v[E];
+#pragma unroll
+                for (int q = 0; q < E / 16; ++q) tmem_ld_x16(acc2 + q * 16, v + q * 16);
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
+                TRACE(tr, 42);
+                if (row >= rows) continue;
                 float gl[E];
 #pragma unroll
                 for (int i = 0; i < E; ++i)
@@ -733,27 +763,46 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                                  __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
                 }
             } else {
-#ifdef SLICEMOE_DEV_NO_OUT    // development: time the pipeline without the output stores
-                if (true) continue;
-#endif
+                // 64 output columns at a time: accumulator -> registers -> bias -> bf16 -> global
+                constexpr int OB = 64;
                 const bool scatter = gather && p.scatter_out != nullptr;
-                bf16* dst = scatter ? p.scatter_out + (size_t)n_cur * C::N2 : p.yperm + (size_t)(row0 + row) * C::N2;
+                const bool live = row < rows;
+                bf16* dst = nullptr;
+                if (live) dst = scatter ? p.scatter_out + (size_t)n_cur * C::N2 : p.yperm + (size_t)(row0 + row) * C::N2;
+#pragma unroll 1
+                for (int cb = 0; cb < C::N2; cb += OB) {
+                    uint32_t v[OB];
 #pragma unroll
-                for (int q = 0; q < C::N2 / 8; ++q) {
-                    float bb[8];
-                    if (p.bias2) {
-                        unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.bias2 + (size_t)e * C::N2 + q * 8)), bb);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) bb[i] = 0.0f;
+                    for (int q = 0; q < OB / 16; ++q) tmem_ld_x16(acc2 + cb + q * 16, v + q * 16);
+                    tmem_ld_wait();
+                    if (cb + OB >= C::N2) {
+                        // the accumulator is in registers: GEMM-2 of a later tile may overwrite it
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
+                        TRACE(tr, 42);
                     }
-                    uint32_t o[4];
+#ifdef SLICEMOE_DEV_NO_OUT    // development: time the pipeline without the output stores
+                    if (true) continue;
+#endif
+                    if (!live) continue;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        o[i] = pack_bf16x2(__uint_as_float(v[q * 8 + 2 * i]) + bb[2 * i],
-                                           __uint_as_float(v[q * 8 + 2 * i + 1]) + bb[2 * i + 1]);
-                    if (scatter) red_add_bf16x8(dst + q * 8, o[0], o[1], o[2], o[3]);   // sum over the row's k experts
-                    else *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                    for (int q = 0; q < OB / 8; ++q) {
+                        float bb[8];
+                        if (p.bias2) {
+                            unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.bias2 + (size_t)e * C::N2 + cb + q * 8)), bb);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) bb[i] = 0.0f;
+                        }
+                        uint32_t o[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            o[i] = pack_bf16x2(__uint_as_float(v[q * 8 + 2 * i]) + bb[2 * i],
+                                               __uint_as_float(v[q * 8 + 2 * i + 1]) + bb[2 * i + 1]);
+                        if (scatter) red_add_bf16x8(dst + cb + q * 8, o[0], o[1], o[2], o[3]);   // sum over the row's k experts
+                        else *reinterpret_cast<uint4*>(dst + cb + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
                 }
             }
         }
@@ -901,7 +950,7 @@ bool tc_route_supported(const Dims& D) {
 
 bool tc_ffn_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
-    if (D.ds != 64 && D.ds != 128) return false;
+    if (D.ds != 64 && D.ds != 128 && D.ds != 256) return false;
     const int hc = D.ds == 64 ? 128 : 64;
     return D.F % hc == 0 && D.F >= 2 * hc && D.F <= kMaxHid;
 }
@@ -950,6 +999,9 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
     if (D.ds == 128)
         return gelu ? launch_ffn_k1<128, SLICEMOE_ACT_GELU_TANH>(D, w, xperm, p, st)
                     : launch_ffn_k1<128, SLICEMOE_ACT_RELU>(D, w, xperm, p, st);
+    if (D.ds == 256)
+        return gelu ? launch_ffn_k1<256, SLICEMOE_ACT_GELU_TANH>(D, w, xperm, p, st)
+                    : launch_ffn_k1<256, SLICEMOE_ACT_RELU>(D, w, xperm, p, st);
     return SLICEMOE_ERR_UNSUPPORTED;
 }
 

@@ -28,9 +28,25 @@ if ROOT not in sys.path:
 L2_BYTES = 126e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (kernel -> workload -> bytes); None where no capture exists.
-NCU_TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+# profiles/forward_kernels_cfg1_cfg2.md (taken on cfg2, whose tokens exceed L2).  The other workloads of
+# the same slice width scale it by the rows one launch processes (traffic is proportional to rows:
+# every row is read once per chosen expert and written once).
+NCU_TRAFFIC_CFG2 = {"route": 134.328064e6 + 142.558720e6, "dispatch": 17.735168e6 + 0.924928e6,
+                    "expert_ffn": 451.720704e6 + 175.928320e6}
+NCU_TRAFFIC_ROWS_CFG2 = 65536 * 16
+
+
+def ncu_traffic(stage, lc):
+    if stage not in NCU_TRAFFIC_CFG2 or lc.ds != 64 or lc.k != 2:
+        return None
+    return NCU_TRAFFIC_CFG2[stage] * lc.N / NCU_TRAFFIC_ROWS_CFG2
+
+
+# tanh.approx results per clock per SM (measured, profiles/microbenchmarks_b200.md): the GELU(tanh) experts
+# cannot go faster than R_kept * F / (148 * 16) cycles, whatever the tensor pipe does.
+TANH_PER_CLK_PER_SM = 16.0
+N_SM = 148
 
 
 def load_peaks():
@@ -144,6 +160,9 @@ def time_oracle(lc, target_s=12.0, steps=1, warmup=0):
     oracle.forward(ocfg, h, w)
     rate = probe_T / max(time.perf_counter() - t0, 1e-6)
     T_s = int(max(probe_T, min(lc.T, rate * target_s)))
+    if steps == 1 and T_s == lc.T:
+        # the whole workload takes less than the target: repeat it to reach about target_s of CPU work
+        steps = int(max(1, min(64, round(target_s * rate / lc.T))))
     sub = lc.with_tokens(T_s)
     h, w = synth.make_layer_inputs(sub)
     ocfg = oracle.OracleConfig(T=sub.T, d=sub.d, S=sub.S, E=sub.E, k=sub.k, Hr=sub.Hr, F=sub.F,
@@ -240,12 +259,13 @@ def run_ours(args, lc):
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     launches0 = sm.slicemoe_launch_count()
-    with ClockSampler(local) as clocks:
-        start.record()
-        for i in range(args.steps):
-            step(i)
-        stop.record()
-        barrier()
+    clocks = ClockSampler(local)          # samples through all three timed regions below
+    clocks.__enter__()
+    start.record()
+    for i in range(args.steps):
+        step(i)
+    stop.record()
+    barrier()
     launches = sm.slicemoe_launch_count() - launches0
     t_dev = start.elapsed_time(stop) / 1e3
 
@@ -269,6 +289,7 @@ def run_ours(args, lc):
     for i in range(len(ev)):
         sm.slicemoe_forward_profiled(cfg, w, hs[i % sets], outs[i % sets], ws, ev[i], assigned, kept)
     torch.cuda.synchronize()
+    clocks.__exit__(None, None, None)
     stage_ms = np.mean([e.stage_ms() for e in ev], axis=0)
 
     times = torch.tensor([t_dev, t_e2e], dtype=torch.float64, device="cuda")
@@ -287,7 +308,7 @@ def run_ours(args, lc):
         else:
             achieved = work["stage_bytes"][dom] / (stages[dom] * 1e-3) / 1e9
             roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-        roof.update(frac=roof["achieved"] / roof["peak"], traffic=NCU_TRAFFIC.get(dom, {}).get(lc.name),
+        roof.update(frac=roof["achieved"] / roof["peak"], traffic=ncu_traffic(dom, lc),
                     kernel=dom, kernel_ms=stages[dom], peak_source=f"of {peak_src}")
         t_step = t_dev / args.steps
         t_tensor = work["total_flops"] / (peaks["bf16_tflops"] * 1e12)
@@ -304,6 +325,10 @@ def run_ours(args, lc):
             "clocks": clocks.summary(),
             "roofline": roof,
             "stage_ms": stages,
+            "activation_bound": {
+                "what": "tanh unit: R_kept*F GELU(tanh) evaluations at 16 per clock per SM",
+                "t_us": (1e6 * kept_rows * lc.F / (N_SM * TANH_PER_CLK_PER_SM) / (clocks.summary()["sm_max_mhz"] or 1965.0) / 1e6
+                         if lc.act else 0.0)},
             "layer_roofline": {"t_tensor_us": 1e6 * t_tensor, "t_hbm_us": 1e6 * t_hbm,
                                "bound": "tensor" if t_tensor >= t_hbm else "hbm",
                                "frac": max(t_tensor, t_hbm) / t_step, "kept_rows": kept_rows,

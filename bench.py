@@ -142,6 +142,15 @@ def aggregate(tokens_per_rank_per_step, steps, seconds_per_rank):
     return sum(tokens_per_rank_per_step) * steps / max(seconds_per_rank)
 
 
+def max_over_ranks(times, dist=None, device="cpu"):
+    """Element-wise maximum of a list of per-rank timings over all ranks (identity without a group)."""
+    import torch
+    t = torch.tensor(list(times), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
 # --------------------------------------------------------------------------------------------
 # CPU oracle leg (also the `--impl reference` arm)
 # --------------------------------------------------------------------------------------------
@@ -292,10 +301,7 @@ def run_ours(args, lc):
     clocks.__exit__(None, None, None)
     stage_ms = np.mean([e.stage_ms() for e in ev], axis=0)
 
-    times = torch.tensor([t_dev, t_e2e], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_dev, t_e2e = (float(x) for x in times.cpu())
+    t_dev, t_e2e = max_over_ranks([t_dev, t_e2e], dist, device="cuda")
 
     if rank == 0:
         peaks, peak_src = load_peaks()

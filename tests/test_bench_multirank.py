@@ -1,0 +1,53 @@
+"""The N > 1 host logic of bench.py on CPU: two gloo ranks, replicas only (no data-path collective)."""
+import os
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def _worker(rank, world, port, out):
+    import torch.distributed as dist
+    import bench
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    # rank r "measures" (r + 1) seconds on the device-resident arm and (r + 2) on the host arm
+    t_dev, t_e2e = bench.max_over_ranks([rank + 1.0, rank + 2.0], dist)
+    dist.barrier()
+    if rank == 0:
+        tokens = bench.shard_tokens(1000, world)
+        out.put((t_dev, t_e2e, tokens, bench.aggregate(tokens, 10, [t_dev])))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_take_the_slowest_time_and_sum_the_tokens():
+    torch = pytest.importorskip("torch")
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    t_dev, t_e2e, tokens, value = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert (t_dev, t_e2e) == (2.0, 3.0)              # max over ranks
+    assert tokens == [1000, 1000]                    # weak scaling: every rank its own batch
+    assert value == 2 * 1000 * 10 / 2.0              # whole-job tokens / slowest rank
+
+
+def test_single_rank_helpers():
+    import bench
+    assert bench.max_over_ranks([0.5, 0.25]) == [0.5, 0.25]
+    assert bench.aggregate([100], 4, [2.0]) == 200.0
+    from paper_2510_04286_b200 import synth
+    w = bench.layer_work(synth.CONFIGS["cfg1"], kept_rows=262144, touched_experts=16)
+    assert abs(w["total_flops"] - 22.55e9) < 0.01e9          # router 5.37 G + experts 17.18 G
+    assert abs(w["compulsory_bytes"] - 34.7e6) < 0.1e6
+    assert bench.ncu_traffic("expert_ffn", synth.CONFIGS["cfg1"]) == pytest.approx(627.649024e6 / 8)
+    assert bench.ncu_traffic("expert_ffn", synth.CONFIGS["cfg3"]) is None

@@ -202,16 +202,33 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // The tanh unit (16 results per clock per SM) is the scarce resource; 16 activation warps keep it
 // fed while the others convert, multiply and store.
 template <int ACT>
-__device__ __forceinline__ void activate_piece_bf16x2(const uint32_t* cur, uint32_t* out) {
+__device__ __forceinline__ void activate_pre_bf16x2(const uint32_t* cur, __nv_bfloat162* z, __nv_bfloat162* t) {
     constexpr int P = 8;   // column pairs per piece
-    __nv_bfloat162 z[P];
 #pragma unroll
     for (int i = 0; i < P; ++i) z[i] = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
 #ifdef SLICEMOE_TC_SKELETON   // development: time the pipeline without the activation math
-    if (true) {
-#else
-    if (ACT == SLICEMOE_ACT_RELU) {
+    return;
 #endif
+    if (ACT == SLICEMOE_ACT_RELU) return;
+    const __nv_bfloat162 c0 = __float2bfloat162_rn(0.7978845608f), c1 = __float2bfloat162_rn(0.0356774081f);
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+        const __nv_bfloat162 inner = __hfma2(__hmul2(z[i], z[i]), c1, c0);
+        const __nv_bfloat162 u = __hmul2(z[i], inner);
+        uint32_t ur = *reinterpret_cast<const uint32_t*>(&u), tr;
+        asm volatile("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
+        t[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
+    }
+}
+template <int ACT>
+__device__ __forceinline__ void activate_post_bf16x2(const __nv_bfloat162* z, const __nv_bfloat162* t, uint32_t* out) {
+    constexpr int P = 8;
+#ifdef SLICEMOE_TC_SKELETON
+    const bool relu = true;
+#else
+    const bool relu = ACT == SLICEMOE_ACT_RELU;
+#endif
+    if (relu) {
         const __nv_bfloat162 zero = __float2bfloat162_rn(0.0f);
 #pragma unroll
         for (int i = 0; i < P; ++i) {
@@ -220,17 +237,7 @@ __device__ __forceinline__ void activate_piece_bf16x2(const uint32_t* cur, uint3
         }
         return;
     }
-    const __nv_bfloat162 c0 = __float2bfloat162_rn(0.7978845608f), c1 = __float2bfloat162_rn(0.0356774081f);
     const __nv_bfloat162 half = __float2bfloat162_rn(0.5f);
-    __nv_bfloat162 t[P];
-#pragma unroll
-    for (int i = 0; i < P; ++i) {
-        const __nv_bfloat162 inner = __hfma2(__hmul2(z[i], z[i]), c1, c0);
-        const __nv_bfloat162 u = __hmul2(z[i], inner);
-        uint32_t ur = *reinterpret_cast<const uint32_t*>(&u), tr;
-        asm("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
-        t[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
-    }
 #pragma unroll
     for (int i = 0; i < P; ++i) {
         const __nv_bfloat162 hz = __hmul2(z[i], half);
@@ -284,6 +291,9 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #endif
     // ---- set-up ---------------------------------------------------------------------------
     if (threadIdx.x == 0) {
+#ifdef SLICEMOE_TC_TRACE
+        { TRACE_DECL(tr0, 5); TRACE(tr0, 99); }
+#endif
         abort_flag = 0;
         for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 4 : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
         for (int i = 0; i < C::W_STAGES; ++i) { mbar_init(bar(B::W_FULL + i), 1); mbar_init(bar(B::W_EMPTY + i), 1); }
@@ -329,6 +339,9 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int t_end = min(total_tiles, t_begin + per_cta);
 
     const uint32_t sA = smem_base + C::OFF_A, sW = smem_base + C::OFF_W;
+#ifdef SLICEMOE_TC_TRACE
+    if (threadIdx.x == 0) { Tracer tr1(5); tr1.n = 1; tr1(98); }   // set-up finished
+#endif
 
     if (warp == 0) {
         // ================= TMA producer =====================================================
@@ -561,24 +574,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 TRACE(tr, 31);
                 PROBE(1);
                 tc_fence_after_sync();
-                uint32_t v[2][C::PIECE];
-                tmem_ld_x16(acc1, v[0]);
-                PROBE(2);
-#pragma unroll
-                for (int pc = 0; pc < C::NPIECE; ++pc) {
-                    uint32_t* cur = v[pc & 1];
-                    tmem_ld_wait();
-                    PROBE(3 + pc * 5);
-                    TRACE(tr, 32);
-                    if (pc + 1 < C::NPIECE) {
-                        tmem_ld_x16(acc1 + (pc + 1) * C::PIECE, v[(pc + 1) & 1]);   // overlaps the math below
-                    } else if constexpr (!C::ROUTER) {
-                        // the accumulator is in registers: GEMM-1 of a later chunk may overwrite it
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
-                    }
-                    PROBE(4 + pc * 5);
+                auto add_bias = [&](uint32_t* cur, int pc) {
                     if (p.bias1) {
                         // same address for the whole warp: one broadcast load per 8 columns
                         const bf16* gb = p.bias1 + (size_t)e * p.HID + c * C::HC + w * WCOLS + pc * C::PIECE;
@@ -590,27 +586,63 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             for (int i = 0; i < 8; ++i) cur[j + i] = __float_as_uint(__uint_as_float(cur[j + i]) + bb[i]);
                         }
                     }
-                    uint32_t hi[C::PIECE / 2];
-                    if constexpr (C::PACKED_ACT) {
-                        activate_piece_bf16x2<C::ACT>(cur, hi);
-                        PROBE(5 + pc * 5);
-                        if (pc == 0) {
-                            // GEMM-2 of two chunks ago must be done with this hidden buffer
-                            ACCT_BEGIN();
-                            ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
-                            ok = __all_sync(0xffffffffu, ok);
-                            ACCT_END(acct_wait_hempty);
+                };
+                if constexpr (C::PACKED_ACT) {
+                    // Experts.  All pieces of the chunk are loaded at once; every piece's conversion,
+                    // multiply-adds and tanh are issued before the first piece's tail, so that the tanh
+                    // unit (the scarce resource) has a queue to work on while the tails and stores run.
+                    uint32_t v[C::NPIECE][C::PIECE];
+#pragma unroll
+                    for (int pc = 0; pc < C::NPIECE; ++pc) tmem_ld_x16(acc1 + pc * C::PIECE, v[pc]);
+                    tmem_ld_wait();
+                    PROBE(3);
+#ifdef SLICEMOE_TC_PROBE
+                    asm volatile("mov.b32 %0, %0;" : "+r"(v[0][0]));                       // first use of loaded data
+                    PROBE(4);
+                    asm volatile("mov.b32 %0, %0;" : "+r"(v[C::NPIECE - 1][C::PIECE - 1])); // last register of the last piece
+                    PROBE(8);
+#endif
+                    // the accumulator is in registers: GEMM-1 of a later chunk may overwrite it
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
+                    PROBE(9);
+                    __nv_bfloat162 z[C::NPIECE][C::PIECE / 2], th[C::NPIECE][C::PIECE / 2];
+#pragma unroll
+                    for (int pc = 0; pc < C::NPIECE; ++pc) {
+                        add_bias(v[pc], pc);
+                        activate_pre_bf16x2<C::ACT>(v[pc], z[pc], th[pc]);
+                    }
+                    PROBE(5);
+                    // GEMM-2 of two chunks ago must be done with this hidden buffer
+                    ACCT_BEGIN();
+                    ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
+                    ok = __all_sync(0xffffffffu, ok);
+                    ACCT_END(acct_wait_hempty);
+                    PROBE(6);
+                    if (ok) {
+#pragma unroll
+                        for (int pc = 0; pc < C::NPIECE; ++pc) {
+                            uint32_t hi[C::PIECE / 2];
+                            activate_post_bf16x2<C::ACT>(z[pc], th[pc], hi);
+                            tmem_st_x8(hdst + pc * (C::PIECE / 2), hi);
                         }
-                        PROBE(6 + pc * 5);
-                        if (ok) tmem_st_x8(hdst + pc * (C::PIECE / 2), hi);
-                        PROBE(7 + pc * 5);
-                    } else {
-                        uint32_t lo[C::PIECE / 2];
+                    }
+                    PROBE(12);
+                } else {
+                    uint32_t v[2][C::PIECE];
+                    tmem_ld_x16(acc1, v[0]);
+#pragma unroll
+                    for (int pc = 0; pc < C::NPIECE; ++pc) {
+                        uint32_t* cur = v[pc & 1];
+                        tmem_ld_wait();
+                        if (pc + 1 < C::NPIECE) tmem_ld_x16(acc1 + (pc + 1) * C::PIECE, v[(pc + 1) & 1]);   // overlaps the math below
+                        add_bias(cur, pc);
+                        uint32_t hi[C::PIECE / 2], lo[C::PIECE / 2];
                         relu_split_piece(cur, hi, lo);
                         tmem_st_x8(acc1 + pc * (C::PIECE / 2), hi);     // over columns this thread has already read
                         tmem_st_x8(hdst + pc * (C::PIECE / 2), lo);
                     }
-                    TRACE(tr, 33);
                 }
                 if (!ok) break;
                 ACCT_BEGIN();

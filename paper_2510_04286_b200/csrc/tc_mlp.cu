@@ -43,10 +43,15 @@ using namespace ptx;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that takes 2 s is a bug, not load
 constexpr int kMaxHid = 1024;
 constexpr int kMaxE = 256;
+// Depth of the per-tile metadata ring.  An entry is rewritten once GEMM-1 of the tile kMetaRing - 3
+// tiles later has finished (three A buffers), by which time the activation warps have read their
+// accumulators for the old tile and the output warps, at most two accumulators and one tile of
+// GEMM-1 run-ahead behind, have stored it.
+constexpr int kMetaRing = 8;
 
 struct TcParams {
     const int32_t* offsets;   // experts: [E+1] device row ranges; router: nullptr
-    int n_rows;               // router: N
+    int n_rows;               // router: N; experts: R (length of the stacked-row arrays)
     int E;                    // experts: E; router: 1
     int HID;                  // Hr or F
     const bf16* bias1;        // [E, HID] or nullptr
@@ -112,11 +117,16 @@ struct TcCfg {
     // larger, one
     static constexpr int A_BUFS = (K1 <= 128) ? 3 : (ROUTER_ ? 2 : 1);
     static constexpr int W_STAGES = (K1 == 128) ? 3 : 2;
-    // activation warpgroups (column split); two for 256-wide rows, whose wide output epilogue needs
-    // the larger register budget of a 512-thread CTA
-    static constexpr int NWG = (K1 == 256) ? 2 : 4;
+    // Activation warps: NGRP groups that take the hidden chunks in turn (chunk g goes to group
+    // g mod NGRP), each group GWG warpgroups that split the chunk's columns.  With two groups one
+    // group's accumulator loads, tails and stores run while the other group's tanh work occupies
+    // the tanh unit.  256-wide rows get one group: their wide output epilogue needs the larger
+    // register budget of a 512-thread CTA.
+    static constexpr int NGRP = (K1 == 256) ? 1 : 2;
+    static constexpr int GWG = 2;
+    static constexpr int NWG = NGRP * GWG;
     static constexpr int NBUF = 2;                              // GEMM-1 accumulator / hidden buffers
-    static constexpr int ACT_WARPS = NWG * 4;
+    static constexpr int GRP_WARPS = GWG * 4;                   // warps that work on one chunk
     static constexpr int THREADS = 128 + NWG * 128 + 128;
     static constexpr int OUT_WARP0 = 4 + NWG * 4;               // first warp of the output warpgroup
     static constexpr int ACC2_BUFS = (N2 <= 128) ? 2 : 1;
@@ -129,10 +139,11 @@ struct TcCfg {
     static constexpr int H_PARTS = ROUTER_ ? 2 : 1;
     static constexpr bool PACKED_ACT = !ROUTER_;
     // TMEM columns:
-    //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w owns columns [w HC/4, (w+1) HC/4)
-    //                        of each.  Router: once a thread has read a 16-column piece it writes
-    //                        the piece's hi half (8 packed columns) over the start of its own
-    //                        column range, so the chunk's hi half ends up in four runs of HC/8.
+    //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w of the group that has the chunk
+    //                        owns columns [w HC/GWG, (w+1) HC/GWG).  Router: once a thread has
+    //                        read a 16-column piece it writes the piece's hi half (8 packed
+    //                        columns) over the start of its own column range, so the chunk's hi
+    //                        half ends up in GWG runs of HC/(2 GWG) columns.
     //   [2 HC, 3 HC)         two hidden buffers of HC/2 packed columns: the experts' hidden chunk
     //                        (so GEMM-1 of a later chunk need not wait for GEMM-2), or the
     //                        router's lo half.
@@ -140,7 +151,7 @@ struct TcCfg {
     static constexpr int H_COL0 = NBUF * HC;
     static constexpr int ACC2_COL0 = H_COL0 + NBUF * (HC / 2);
     static constexpr int TMEM_COLS = pow2_at_least(ACC2_COL0 + ACC2_BUFS * N2);
-    static constexpr int KSTEPS_PER_WG = HC / (16 * NWG);       // 16-element K steps in one warpgroup's columns
+    static constexpr int KSTEPS_PER_WG = HC / (16 * GWG);       // 16-element K steps in one warpgroup's columns
     static constexpr int KP1 = K1 / 64;                         // 64-wide K panels of GEMM-1
     static constexpr int KP2 = HC / 64;                         // K panels of GEMM-2 per chunk
     static constexpr int A_PANEL = 128 * 128;                   // bytes: 128 rows x 128 B
@@ -152,11 +163,15 @@ struct TcCfg {
     static constexpr int W_STAGE_BYTES = W1C_BYTES + W2C_BYTES;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_W = OFF_A + A_BUFS * A_BYTES;
-    static constexpr int SMEM_BYTES = OFF_W + W_STAGES * W_STAGE_BYTES;
+    static constexpr int B1_BYTES = HC * 2;                     // one chunk of the first layer's bias, per weight stage
+    static constexpr int OFF_B1 = OFF_W + W_STAGES * W_STAGE_BYTES;
+    static constexpr int SMEM_BYTES = OFF_B1 + W_STAGES * B1_BYTES;
     // at least 120 KiB is requested so that two CTAs never share an SM (each allocates most of TMEM)
     static constexpr int SMEM_ALLOC = (SMEM_BYTES + 1024 > 120 * 1024) ? SMEM_BYTES + 1024 : 120 * 1024;
     static constexpr int PIECE = 16;                            // accumulator columns per piece
-    static constexpr int NPIECE = HC / (PIECE * NWG);           // pieces per thread and chunk
+    static constexpr int NPIECE = HC / (PIECE * GWG);           // pieces per thread and chunk
+    static constexpr int SUB = (NPIECE > 2) ? 2 : NPIECE;       // pieces held in registers at once (experts)
+    static_assert(NBUF % NGRP == 0 && NPIECE % SUB == 0, "chunk-to-group and piece-to-batch maps");
     static_assert(NPIECE >= 1, "hidden chunk too narrow for the activation warpgroups");
     static_assert(W_STAGE_BYTES % 1024 == 0 && W1C_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
     static_assert(N2 % 16 == 0 && N2 >= 16 && N2 <= 256, "MMA N");
@@ -195,17 +210,32 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// 16 fp32 pre-activations (one thread's piece of a row) -> 8 packed bf16 activation pairs, all
-// arithmetic 2-wide in bf16: one conversion, five packed multiply-adds and one packed tanh per
-// pair.  GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))).  Where z^2 overflows,
-// tanh saturates to +-1 and the formula still returns z (z > 0) or 0 (z < 0).
-// The tanh unit (16 results per clock per SM) is the scarce resource; 16 activation warps keep it
-// fed while the others convert, multiply and store.
-template <int ACT>
-__device__ __forceinline__ void activate_pre_bf16x2(const uint32_t* cur, __nv_bfloat162* z, __nv_bfloat162* t) {
-    constexpr int P = 8;   // column pairs per piece
+// Expert activation, all arithmetic 2-wide in bf16 on one thread's 16-column piece of a row:
+//   convert   z = bf16(acc) * gate + bias             one conversion, two multiply-adds per pair (the gate
+//                                                     as a bf16 pair hi + lo: rounding it to one bf16
+//                                                     would tilt a whole row's pre-activations together)
+//   pre       t = tanh(z (c0 + c1 z^2))               three multiply-adds and one packed tanh per pair
+//   post      2 gelu(z) = z t + z                     one multiply-add per pair
+// GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))); the factor 0.5 is applied to
+// the GEMM-2 accumulator in the output epilogue (exact: a power of two).  Where z^2 overflows, tanh
+// saturates to +-1 and the formula still returns 2z (z > 0) or 0 (z < 0).
+// The tanh unit (16 results per clock per SM) is the scarce resource; the instruction count around
+// it is kept low enough that the issue slots are not the next one.
+__device__ __forceinline__ void convert_piece_bf16x2(const uint32_t* cur, __nv_bfloat162 gate_hi, __nv_bfloat162 gate_lo,
+                                                     const uint4* bias8, bool has_bias, __nv_bfloat162* z) {
+    uint4 braw[2];
+    if (has_bias) { braw[0] = bias8[0]; braw[1] = bias8[1]; }      // 16 packed bf16, warp-wide broadcast
+    else braw[0] = braw[1] = make_uint4(0u, 0u, 0u, 0u);
+    const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(braw);
 #pragma unroll
-    for (int i = 0; i < P; ++i) z[i] = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+    for (int i = 0; i < 8; ++i) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+        z[i] = __hfma2(a, gate_hi, __hfma2(a, gate_lo, b2[i]));
+    }
+}
+template <int ACT>
+__device__ __forceinline__ void activate_pre_bf16x2(const __nv_bfloat162* z, __nv_bfloat162* t) {
+    constexpr int P = 8;   // column pairs per piece
 #ifdef SLICEMOE_TC_SKELETON   // development: time the pipeline without the activation math
     return;
 #endif
@@ -237,14 +267,20 @@ __device__ __forceinline__ void activate_post_bf16x2(const __nv_bfloat162* z, co
         }
         return;
     }
-    const __nv_bfloat162 half = __float2bfloat162_rn(0.5f);
 #pragma unroll
     for (int i = 0; i < P; ++i) {
-        const __nv_bfloat162 hz = __hmul2(z[i], half);
-        const __nv_bfloat162 r = __hfma2(hz, t[i], hz);
+        const __nv_bfloat162 r = __hfma2(z[i], t[i], z[i]);
         out[i] = *reinterpret_cast<const uint32_t*>(&r);
     }
 }
+// factor the output epilogue applies to the GEMM-2 accumulator (see above)
+template <int ACT>
+constexpr float kOutScale =
+#ifdef SLICEMOE_TC_SKELETON
+    1.0f;
+#else
+    (ACT == SLICEMOE_ACT_RELU) ? 1.0f : 0.5f;
+#endif
 
 // Router: ReLU in fp32, then each value as a bf16 pair, the rounded value (hi) and the rounded
 // remainder (lo); hi + lo carries 16 mantissa bits of the fp32 value.
@@ -276,6 +312,10 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     __shared__ int hist[kMaxE];
     __shared__ uint32_t tmem_base_smem;
     __shared__ int abort_flag;
+    // fused forward: per-row gate (Eq. 1) and pair index of the tiles in flight, copied in by the
+    // gather warp with the rows themselves (ring over the CTA's tile counter)
+    __shared__ float gate_s[kMetaRing][kTileM];
+    __shared__ int pair_s[kMetaRing][kTileM];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -295,12 +335,12 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         { TRACE_DECL(tr0, 5); TRACE(tr0, 99); }
 #endif
         abort_flag = 0;
-        for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 4 : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
+        for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 32 : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
         for (int i = 0; i < C::W_STAGES; ++i) { mbar_init(bar(B::W_FULL + i), 1); mbar_init(bar(B::W_EMPTY + i), 1); }
         for (int i = 0; i < C::NBUF; ++i) {
             mbar_init(bar(B::ACC1_FULL + i), 1);
-            mbar_init(bar(B::ACC1_EMPTY + i), C::ROUTER ? 1 : C::ACT_WARPS);
-            mbar_init(bar(B::H_FULL + i), C::ACT_WARPS);
+            mbar_init(bar(B::ACC1_EMPTY + i), C::ROUTER ? 1 : C::GRP_WARPS);
+            mbar_init(bar(B::H_FULL + i), C::GRP_WARPS);
             mbar_init(bar(B::H_EMPTY + i), 1);
         }
         for (int i = 0; i < C::ACC2_BUFS; ++i) {
@@ -376,8 +416,11 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
                     const uint32_t n = resident ? reloads : g / C::W_STAGES;
                     if (!mbar_wait(bar(B::W_EMPTY + slot), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
-                    mbar_arrive_expect_tx(bar(B::W_FULL + slot), C::W_STAGE_BYTES);
+                    mbar_arrive_expect_tx(bar(B::W_FULL + slot), C::W_STAGE_BYTES + (p.bias1 ? C::B1_BYTES : 0));
                     const uint32_t dst = sW + slot * C::W_STAGE_BYTES;
+                    if (p.bias1)
+                        bulk_load(smem_base + C::OFF_B1 + slot * C::B1_BYTES, p.bias1 + (size_t)e * p.HID + c * C::HC,
+                                  C::B1_BYTES, bar(B::W_FULL + slot));
 #pragma unroll
                     for (int kp = 0; kp < C::KP1; ++kp)
                         tma_load_2d(dst + kp * C::W1_PANEL, &tmW1, kp * 64, e * p.HID + c * C::HC, bar(B::W_FULL + slot));
@@ -416,6 +459,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 TRACE(tr, 10);
                 if (!mbar_wait(bar(B::A_FULL + ab), (uint32_t)(ta / C::A_BUFS) & 1u, abort, kWaitLimitNs)) { ok = false; break; }
                 TRACE(tr, 11);
+                if (gather) fence_proxy_async_smem();   // rows written by cp.async -> visible to the MMA's reads
                 for (int c = 0; c < nchunks; ++c, ++g) {
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
                     if (reload) {
@@ -496,7 +540,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         for (int kk = 0; kk < C::HC / 16; ++kk) {
                             uint32_t a;
                             if (C::ROUTER && part == 0)
-                                a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / C::NWG) + (kk % C::KSTEPS_PER_WG) * 8;
+                                a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / C::GWG) + (kk % C::KSTEPS_PER_WG) * 8;
                             else
                                 a = hbuf + kk * 8;
                             const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
@@ -520,8 +564,8 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             }
         }
     } else if (warp == 3) {
-        // ================= zero this CTA's rows of h' (router, fused forward) ================
         if constexpr (C::ROUTER) {
+            // ============= zero this CTA's rows of h' (router, fused forward) ================
             if (p.zero_out != nullptr && t_begin < t_end) {
                 const long long row_lo = (long long)t_begin * kTileM;
                 long long row_hi = (long long)t_end * kTileM;
@@ -531,17 +575,88 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const uint4 z = make_uint4(0u, 0u, 0u, 0u);
                 for (long long i = lane; i < nvec; i += 32) dst[i] = z;
             }
+        } else if (gather && t_begin < t_end) {
+            // ============= gather warp (experts, fused forward) ===============================
+            // Row r of a tile is stacked row row0 + r = pair perm[row0 + r] = (n, j); its A row is
+            // X[n, :], copied asynchronously (no registers) into the K-major 128-byte-swizzled
+            // layout.  The gate of Eq. 1 multiplies the GEMM-1 accumulator instead of the row.
+            // The warp runs ahead of the MMAs by as many tiles as there are A buffers.
+            constexpr int CPR = C::K1 / 8;            // 16-byte chunks per row
+            constexpr int RPI = 32 / CPR;             // rows covered by one warp-wide copy
+            const int ch = lane % CPR, rsub = lane / CPR;
+            int ge = 0, gm = 0;
+            bool ok = true;
+            int nrow[4], nnext[4];                    // source rows of tile rows lane + 32 q
+            // (the loaded pair index is left untouched until the next tile, so that the load's latency
+            // is not waited for here)
+            auto load_rows = [&](int t, int* out) {
+                int row0, rows;
+                locate_tile(tile_start, offs, t, ge, row0, rows);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int r = lane + 32 * q;
+                    out[q] = (r < rows) ? __ldg(p.perm + row0 + r) : -1;
+                }
+            };
+            load_rows(t_begin, nnext);
+            TRACE_DECL(tr, lane == 0 ? 0 : 7);
+            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+                TRACE(tr, 1);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) nrow[q] = nnext[q] < 0 ? -1 : nnext[q] / p.gather_k;
+#ifdef SLICEMOE_TC_TRACE
+#pragma unroll
+                for (int q = 0; q < 4; ++q) asm volatile("mov.b32 %0, %0;" : "+r"(nrow[q]));
+                TRACE(tr, 4);
+#endif
+                if (t + 1 < t_end) load_rows(t + 1, nnext);
+                TRACE(tr, 5);
+                const int ab = ta % C::A_BUFS;
+                ok = mbar_wait(bar(B::A_EMPTY + ab), ((uint32_t)(ta / C::A_BUFS) & 1u) ^ 1u, abort, kWaitLimitNs);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                TRACE(tr, 2);
+                const uint32_t dst0 = sA + ab * C::A_BYTES + (ch >> 3) * C::A_PANEL;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+#pragma unroll 8
+                    for (int i = 0; i < 32 / RPI; ++i) {
+                        const int r32 = i * RPI + rsub;                 // row within this block of 32
+                        const int r = q * 32 + r32;
+                        const int n = __shfl_sync(0xffffffffu, nrow[q], r32);
+                        const bf16* src = p.gather_src + (size_t)(n < 0 ? 0 : n) * C::K1 + ch * 8;
+                        cp_async_16(dst0 + (r >> 3) * 1024 + (r & 7) * 128 + (((ch & 7) ^ (r & 7)) << 4), src,
+                                    n < 0 ? 0u : 16u);
+                    }
+                }
+                {
+                    int row0, rows;
+                    locate_tile(tile_start, offs, t, gm, row0, rows);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        // rows past the tile's end take a neighbour's values: their A rows are zero and
+                        // they are never stored
+                        const int r = lane + 32 * q, src = min(row0 + r, p.n_rows - 1);
+                        cp_async_4(smem_u32(&gate_s[ta % kMetaRing][r]), p.gate + src);
+                        cp_async_4(smem_u32(&pair_s[ta % kMetaRing][r]), p.perm + src);
+                    }
+                }
+                cp_async_mbar_arrive_noinc(bar(B::A_FULL + ab));
+                TRACE(tr, 3);
+            }
+            cp_async_wait_all();
         }
     } else if (warp >= 4 && warp < C::OUT_WARP0) {
         // ================= activation warpgroups =============================================
-        const int w = (warp - 4) >> 2;                // warpgroup = which half of the chunk's columns
+        const int grp = (warp - 4) / C::GRP_WARPS;    // which chunks: g mod NGRP == grp
+        const int w = ((warp - 4) >> 2) % C::GWG;     // warpgroup within the group = which part of the chunk's columns
         const int lg = warp & 3;                      // TMEM lane group this warp may access
         const uint32_t lane_base = tmem_base + ((uint32_t)(lg * 32) << 16);
-        constexpr int WCOLS = C::HC / C::NWG;         // accumulator columns per thread and chunk
+        constexpr int WCOLS = C::HC / C::GWG;         // accumulator columns per thread and chunk
         bool ok = true;
         int e = 0;
         uint32_t g = 0;
-        TRACE_DECL(tr, (lg == 0 && lane == 0) ? 2 + w : 7);
+        TRACE_DECL(tr, (lg == 0 && lane == 0 && w == 0) ? 2 + grp : 7);
 #ifdef SLICEMOE_TC_ACCT   // development: where do the activation warps spend their cycles?
         long long acct_wait_acc1 = 0, acct_wait_hempty = 0, acct_stwait = 0, acct_t0 = clock64(), acct_mark;
 #define ACCT_BEGIN() acct_mark = clock64()
@@ -560,7 +675,11 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         for (int t = t_begin; t < t_end && ok; ++t) {
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
+            TRACE(tr, 36);
+            float gs = 1.0f;                          // Eq. 1's gate of this thread's row (fused forward; the
+                                                      // staged call's rows arrive weighted), read per chunk
             for (int c = 0; c < nchunks && ok; ++c, ++g) {
+                if (C::NGRP > 1 && (int)(g % C::NGRP) != grp) continue;               // the other group's chunk
                 const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
                 const uint32_t acc1 = lane_base + b * C::HC + w * WCOLS;               // my accumulator columns
                 const uint32_t hdst = lane_base + C::H_COL0 + b * (C::HC / 2) + w * (WCOLS / 2);
@@ -571,61 +690,71 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 ok = __all_sync(0xffffffffu, ok);
                 ACCT_END(acct_wait_acc1);
                 if (!ok) break;
+                // (the tile's A rows, and with them its ring entry, landed before GEMM-1 could run)
+                if (gather) gs = gate_s[(t - t_begin) % kMetaRing][lg * 32 + lane];
                 TRACE(tr, 31);
                 PROBE(1);
                 tc_fence_after_sync();
+                // this chunk's bias came into shared memory with its weights (same stage, same barrier)
+                const int slot = resident ? c : (int)(g % C::W_STAGES);
+                const uint8_t* sb1 = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_B1 + slot * C::B1_BYTES + w * WCOLS * 2;
                 auto add_bias = [&](uint32_t* cur, int pc) {
                     if (p.bias1) {
-                        // same address for the whole warp: one broadcast load per 8 columns
-                        const bf16* gb = p.bias1 + (size_t)e * p.HID + c * C::HC + w * WCOLS + pc * C::PIECE;
 #pragma unroll
                         for (int j = 0; j < C::PIECE; j += 8) {
                             float bb[8];
-                            unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(gb + j)), bb);
+                            unpack16<bf16>(*reinterpret_cast<const uint4*>(sb1 + (pc * C::PIECE + j) * 2), bb);   // warp-wide broadcast
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) cur[j + i] = __float_as_uint(__uint_as_float(cur[j + i]) + bb[i]);
+                            for (int i = 0; i < 8; ++i) cur[j + i] = __float_as_uint(fmaf(__uint_as_float(cur[j + i]), gs, bb[i]));
                         }
+                    } else if (gather) {
+#pragma unroll
+                        for (int i = 0; i < C::PIECE; ++i) cur[i] = __float_as_uint(__uint_as_float(cur[i]) * gs);
                     }
                 };
                 if constexpr (C::PACKED_ACT) {
-                    // Experts.  All pieces of the chunk are loaded at once; every piece's conversion,
-                    // multiply-adds and tanh are issued before the first piece's tail, so that the tanh
-                    // unit (the scarce resource) has a queue to work on while the tails and stores run.
-                    uint32_t v[C::NPIECE][C::PIECE];
+                    // Experts.  The whole accumulator chunk is brought into registers as packed bf16
+                    // (SUB pieces at a time) and handed back at once, so that GEMM-1 of this group's
+                    // next chunk runs under this chunk's activation.  Then piece by piece: the argument
+                    // and tanh of piece pc, and behind them the tail and the store of piece pc - 1,
+                    // whose tanh results have arrived by then.
+                    __nv_bfloat162 z[C::NPIECE][C::PIECE / 2];
+                    const __nv_bfloat16 gs_hi = __float2bfloat16_rn(gs);
+                    const __nv_bfloat162 gate_hi = __bfloat162bfloat162(gs_hi);
+                    const __nv_bfloat162 gate_lo = __float2bfloat162_rn(gs - __bfloat162float(gs_hi));
 #pragma unroll
-                    for (int pc = 0; pc < C::NPIECE; ++pc) tmem_ld_x16(acc1 + pc * C::PIECE, v[pc]);
-                    tmem_ld_wait();
+                    for (int s0 = 0; s0 < C::NPIECE; s0 += C::SUB) {
+                        uint32_t v[C::SUB][C::PIECE];
+#pragma unroll
+                        for (int i = 0; i < C::SUB; ++i) tmem_ld_x16(acc1 + (s0 + i) * C::PIECE, v[i]);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < C::SUB; ++i)
+                            convert_piece_bf16x2(v[i], gate_hi, gate_lo, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
+                                                 p.bias1 != nullptr, z[s0 + i]);
+                    }
                     PROBE(3);
-#ifdef SLICEMOE_TC_PROBE
-                    asm volatile("mov.b32 %0, %0;" : "+r"(v[0][0]));                       // first use of loaded data
-                    PROBE(4);
-                    asm volatile("mov.b32 %0, %0;" : "+r"(v[C::NPIECE - 1][C::PIECE - 1])); // last register of the last piece
-                    PROBE(8);
-#endif
-                    // the accumulator is in registers: GEMM-1 of a later chunk may overwrite it
+                    TRACE(tr, 32);
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
-                    PROBE(9);
-                    __nv_bfloat162 z[C::NPIECE][C::PIECE / 2], th[C::NPIECE][C::PIECE / 2];
+                    __nv_bfloat162 th[2][C::PIECE / 2];
 #pragma unroll
-                    for (int pc = 0; pc < C::NPIECE; ++pc) {
-                        add_bias(v[pc], pc);
-                        activate_pre_bf16x2<C::ACT>(v[pc], z[pc], th[pc]);
-                    }
-                    PROBE(5);
-                    // GEMM-2 of two chunks ago must be done with this hidden buffer
-                    ACCT_BEGIN();
-                    ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
-                    ok = __all_sync(0xffffffffu, ok);
-                    ACCT_END(acct_wait_hempty);
-                    PROBE(6);
-                    if (ok) {
-#pragma unroll
-                        for (int pc = 0; pc < C::NPIECE; ++pc) {
+                    for (int pc = 0; pc <= C::NPIECE; ++pc) {
+                        if (pc < C::NPIECE) activate_pre_bf16x2<C::ACT>(z[pc], th[pc & 1]);
+                        if (pc == 0) {
+                            TRACE(tr, 33);
+                            // GEMM-2 of two chunks ago must be done with this hidden buffer
+                            ACCT_BEGIN();
+                            ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
+                            ok = __all_sync(0xffffffffu, ok);
+                            ACCT_END(acct_wait_hempty);
+                            if (!ok) break;
+                            TRACE(tr, 34);
+                        } else {
                             uint32_t hi[C::PIECE / 2];
-                            activate_post_bf16x2<C::ACT>(z[pc], th[pc], hi);
-                            tmem_st_x8(hdst + pc * (C::PIECE / 2), hi);
+                            activate_post_bf16x2<C::ACT>(z[pc - 1], th[(pc - 1) & 1], hi);
+                            tmem_st_x8(hdst + (pc - 1) * (C::PIECE / 2), hi);
                         }
                     }
                     PROBE(12);
@@ -647,6 +776,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (!ok) break;
                 ACCT_BEGIN();
                 tmem_st_wait();
+                TRACE(tr, 37);
                 ACCT_END(acct_stwait);
                 PROBE(13);
                 tc_fence_before_sync();
@@ -676,64 +806,9 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         bool ok = true;
         int e = 0;
         TRACE_DECL(tr, (lg == 0 && lane == 0) ? 5 : 7);
-        // Fused forward: row `row` of tile (tg, tga) is stacked row row0 + row = pair perm[.] = (n, j);
-        // its A row is bf16(gate * X[n, :]) (Eq. 1), written in the K-major 128-byte-swizzled layout.
-        int ge = 0;
-        int n_of[3] = {-1, -1, -1};           // source row (of X / Y) of this thread's row, per tile in flight
-        auto gather_tile = [&](int tg, int tga) -> bool {
-            constexpr int CPR = C::K1 / 8;                       // 16-byte chunks per row
-            constexpr int GB = 8;                                // chunks per block (registers)
-            int row0, rows;
-            locate_tile(tile_start, offs, tg, ge, row0, rows);
-            const int ab = tga % C::A_BUFS;
-            float g = 0.0f;
-            int n = -1;
-            if (row < rows) {
-                n = __ldg(p.perm + row0 + row) / p.gather_k;
-                g = __ldg(p.gate + row0 + row);
-            }
-            n_of[tga % 3] = n;
-            const uint4* src = reinterpret_cast<const uint4*>(p.gather_src + (size_t)(n < 0 ? 0 : n) * C::K1);
-            uint4 raw[GB];
-#pragma unroll
-            for (int i = 0; i < GB; ++i) raw[i] = (n >= 0) ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
-            bool okg = mbar_wait(bar(B::A_EMPTY + ab), ((uint32_t)(tga / C::A_BUFS) & 1u) ^ 1u, abort, kWaitLimitNs);
-            okg = __all_sync(0xffffffffu, okg);
-            if (!okg) return false;
-            uint8_t* dst = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_A + ab * C::A_BYTES +
-                           (row >> 3) * 1024 + (row & 7) * 128;
-#pragma unroll
-            for (int blk = 0; blk < CPR / GB; ++blk) {
-#pragma unroll
-                for (int i = 0; i < GB; ++i) {
-                    float f[8];
-                    unpack16<bf16>(raw[i], f);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) f[q] *= g;
-                    // chunk blk*8 + i of the row lives in panel blk (64 columns), 16-byte slot i
-                    *reinterpret_cast<uint4*>(dst + blk * C::A_PANEL + ((i ^ (row & 7)) << 4)) = pack16<bf16>(f);
-                }
-                if (blk + 1 < CPR / GB) {
-#pragma unroll
-                    for (int i = 0; i < GB; ++i)
-                        raw[i] = (n >= 0) ? __ldg(src + (blk + 1) * GB + i) : make_uint4(0u, 0u, 0u, 0u);
-                }
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B::A_FULL + ab));
-            return true;
-        };
-        constexpr int AHEAD = C::A_BUFS - 1;   // tiles gathered ahead of the one being output
-        if (gather) {
-            for (int i = 0; i < AHEAD && ok && t_begin + i < t_end; ++i) ok = gather_tile(t_begin + i, i);
-        }
+        // Fused forward: this thread's row of a tile is pair perm[row0 + row] = (n, j); its output is
+        // added into row n of Y.
         for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
-            if (gather && t + AHEAD < t_end) {
-                ok = gather_tile(t + AHEAD, ta + AHEAD);      // a later tile's A operand (this tile's when there
-                if (!ok) break;                               // is only one buffer), while the tensor core works
-            }
-            const int n_cur = n_of[ta % 3];
             int row0, rows;
             locate_tile(tile_start, offs, t, e, row0, rows);
             const int buf = ta % C::ACC2_BUFS;
@@ -743,6 +818,7 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             if (!ok) break;
             TRACE(tr, 41);
             tc_fence_after_sync();
+            const int pair_cur = gather ? pair_s[ta % kMetaRing][row] : 0;
             const uint32_t acc2 = tmem_lane + C::ACC2_COL0 + buf * C::N2;
             if constexpr (C::ROUTER) {
                 constexpr int E = C::N2;
@@ -800,7 +876,8 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const bool scatter = gather && p.scatter_out != nullptr;
                 const bool live = row < rows;
                 bf16* dst = nullptr;
-                if (live) dst = scatter ? p.scatter_out + (size_t)n_cur * C::N2 : p.yperm + (size_t)(row0 + row) * C::N2;
+                if (live) dst = scatter ? p.scatter_out + (size_t)(pair_cur / p.gather_k) * C::N2
+                                        : p.yperm + (size_t)(row0 + row) * C::N2;
 #pragma unroll 1
                 for (int cb = 0; cb < C::N2; cb += OB) {
                     uint32_t v[OB];
@@ -830,12 +907,13 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         uint32_t o[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            o[i] = pack_bf16x2(__uint_as_float(v[q * 8 + 2 * i]) + bb[2 * i],
-                                               __uint_as_float(v[q * 8 + 2 * i + 1]) + bb[2 * i + 1]);
+                            o[i] = pack_bf16x2(fmaf(__uint_as_float(v[q * 8 + 2 * i]), kOutScale<C::ACT>, bb[2 * i]),
+                                               fmaf(__uint_as_float(v[q * 8 + 2 * i + 1]), kOutScale<C::ACT>, bb[2 * i + 1]));
                         if (scatter) red_add_bf16x8(dst + cb + q * 8, o[0], o[1], o[2], o[3]);   // sum over the row's k experts
                         else *reinterpret_cast<uint4*>(dst + cb + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
+                TRACE(tr, 43);
             }
         }
     }
@@ -852,7 +930,12 @@ tc_mlp_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
     }
 #ifdef SLICEMOE_TC_TRACE
-    if (blockIdx.x == 0 && g_trace_buf) {
+#ifdef SLICEMOE_TRACE_EXPERTS_ONLY
+    constexpr bool dump_trace = !C::ROUTER;
+#else
+    constexpr bool dump_trace = true;
+#endif
+    if (dump_trace && blockIdx.x == 0 && g_trace_buf) {
         const uint2* src = reinterpret_cast<const uint2*>(smem_raw + 200 * 1024);
         for (int i = threadIdx.x; i < 6 * kTraceSmemEvents; i += C::THREADS) {
             const int slot = i / kTraceSmemEvents, n = i % kTraceSmemEvents;
@@ -1018,7 +1101,7 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
                   void* scatter_out) {
     if (D.R == 0) return SLICEMOE_OK;
     TcParams p{};
-    p.offsets = offsets; p.n_rows = 0; p.E = D.E; p.HID = D.F;
+    p.offsets = offsets; p.n_rows = (int)D.R; p.E = D.E; p.HID = D.F;
     p.bias1 = (const bf16*)w.b1; p.bias2 = (const bf16*)w.b2;
     p.yperm = (bf16*)yperm; p.status = status;
     p.gather_src = (const bf16*)gather_h; p.perm = perm; p.gate = gate; p.gather_k = D.k;

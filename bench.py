@@ -293,7 +293,10 @@ def run_ours(args, lc):
     t_e2e = start.elapsed_time(stop) / 1e3
 
     # ---- timed region 3: per-stage CUDA events (recorded by the library on its stream) ----
+    # (the stage-timed call keeps one launch per stage; the forward timed above is one launch)
     ev = [sm.StageEvents() for _ in range(min(args.steps, 64))]
+    for i in range(3):
+        sm.slicemoe_forward_profiled(cfg, w, hs[i % sets], outs[i % sets], ws, ev[0], assigned, kept)
     barrier()
     for i in range(len(ev)):
         sm.slicemoe_forward_profiled(cfg, w, hs[i % sets], outs[i % sets], ws, ev[i], assigned, kept)
@@ -308,7 +311,16 @@ def run_ours(args, lc):
         work = layer_work(lc, kept_rows, touched)
         stages = dict(zip(sm.STAGES, (float(x) for x in stage_ms)))
         dom = max(stages, key=stages.get)
-        if dom in work["stage_flops"]:
+        t_step = t_dev / args.steps
+        single_launch = launches == args.steps
+        if single_launch:
+            # the timed forward is ONE kernel (router, dispatch and expert phases): its launch
+            # duration is the step time measured by the events around the timed region
+            dom = "fused_forward"
+            achieved = work["total_flops"] / t_step / 1e12
+            roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+            stages = dict(stages, fused_forward=1e3 * t_step)
+        elif dom in work["stage_flops"]:
             achieved = work["stage_flops"][dom] / (stages[dom] * 1e-3) / 1e12
             roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
         else:
@@ -316,7 +328,6 @@ def run_ours(args, lc):
             roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
         roof.update(frac=roof["achieved"] / roof["peak"], traffic=ncu_traffic(dom, lc),
                     kernel=dom, kernel_ms=stages[dom], peak_source=f"of {peak_src}")
-        t_step = t_dev / args.steps
         t_tensor = work["total_flops"] / (peaks["bf16_tflops"] * 1e12)
         t_hbm = work["compulsory_bytes"] / (peaks["hbm_gbs"] * 1e9)
         line = {
@@ -330,7 +341,7 @@ def run_ours(args, lc):
             "gpu_launches": int(launches),
             "clocks": clocks.summary(),
             "roofline": roof,
-            "stage_ms": stages,
+            "stage_ms_one_launch_per_stage": {k: v for k, v in stages.items() if k != "fused_forward"},
             "activation_bound": {
                 "what": "tanh unit: R_kept*F GELU(tanh) evaluations at 16 per clock per SM",
                 "t_us": (1e6 * kept_rows * lc.F / (N_SM * TANH_PER_CLK_PER_SM) / (clocks.summary()["sm_max_mhz"] or 1965.0) / 1e6

@@ -186,6 +186,12 @@ int slicemoe_combine(const slicemoe_config *cfg, const void *yperm, const int32_
  * topk_idx / assigned / kept.  h_out must not overlap h.
  * Optional outputs (NULL to skip): assigned_opt int32 [E], kept_opt int32 [E],
  * topk_idx_opt int32 [N, k], topk_p_opt float [N, k].
+ * For bf16 layers with ds in {64, 128, 256}, E in {16, 32, 64}, k <= 2 and
+ * hidden widths that are multiples of the chunk width, the whole forward is ONE
+ * kernel launch (router, dispatch and expert phases separated by grid-wide
+ * barriers, one CTA per SM); other shapes run one kernel per step.  Every wait
+ * inside is bounded: a run-out leaves SLICEMOE_ERR_DEVICE_TIMEOUT in the status
+ * word (slicemoe_last_status) and the call's outputs undefined.
  */
 int slicemoe_forward(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
                      void *h_out, int32_t *assigned_opt, int32_t *kept_opt,
@@ -224,7 +230,9 @@ int slicemoe_event_destroy(void *event);
 int slicemoe_event_elapsed_ms(void *start, void *stop, float *ms);
 
 /* Device status word of the last kernels that used `ws` (0 = fine, else a
- * slicemoe_status such as SLICEMOE_ERR_DEVICE_TIMEOUT).  Synchronises `stream`. */
+ * slicemoe_status such as SLICEMOE_ERR_DEVICE_TIMEOUT).  Synchronises `stream`.
+ * After a time-out it also puts the device's grid-barrier words, which the
+ * aborted launch may have left half-counted, back to zero. */
 int slicemoe_last_status(const void *ws, void *stream);
 
 /* Number of kernels this library has launched in this process so far (HOST counter). */

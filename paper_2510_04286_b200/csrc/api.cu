@@ -4,6 +4,8 @@
 #include <cstdio>
 #include <cstring>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace slicemoe {
@@ -148,13 +150,19 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
         return SLICEMOE_OK;
     };
     int rc;
-    if ((rc = reset_status(ws, W, st))) return rc;
+    const bool one_launch = !events && fused_forward_supported(D);
+    if (!one_launch && (rc = reset_status(ws, W, st))) return rc;     // (the single kernel clears it itself)
     if ((rc = mark(0))) return rc;
     // With both tensor-core kernels available the stacked rows are never materialised: the router
     // leaves its per-CTA expert counts, one dispatch kernel ranks the pairs (dest, perm, gate) and
     // the expert kernel gathers its rows from h.
     const bool fused = tc_route_supported(D) && tc_ffn_supported(D) && D.N > 0;
     float* gate = at<float>(ws, W.gate);
+    // One cooperative launch does all of it; the stage-timed call keeps the three launches so that
+    // the stages stay separable.
+    if (one_launch)
+        return launch_forward_fused(D, w, h, h_out, idx, p, assigned, kept, offsets, dest, perm, gate,
+                                    at<int32_t>(ws, W.cta_hist), at<int32_t>(ws, W.status), st);
     if (fused) {
         int grid = 0, rows_per_cta = 0;
         tc_route_grid(D, &grid, &rows_per_cta);
@@ -360,6 +368,11 @@ int slicemoe_last_status(const void* ws, void* stream) {
     SLICEMOE_CUDA_TRY(cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost,
                                       static_cast<cudaStream_t>(stream)));
     SLICEMOE_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    if (word == SLICEMOE_ERR_DEVICE_TIMEOUT) {
+        // a launch gave up inside a grid barrier: put the barrier words back in order
+        const int rc = slicemoe::fused_forward_reset_sync(static_cast<cudaStream_t>(stream));
+        if (rc) return rc;
+    }
     return word;
 }
 

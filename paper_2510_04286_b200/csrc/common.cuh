@@ -116,6 +116,18 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
                   void* yperm, int32_t* status, cudaStream_t st, const void* gather_h = nullptr,
                   const int32_t* perm = nullptr, const float* gate = nullptr, void* scatter_out = nullptr);
 
+// The whole forward as one cooperative launch (router phase, dispatch phase, expert phase with grid
+// barriers between them): bf16 shapes that both tensor-core kernels take, k <= 2.  The kernel clears
+// the status word itself (no memset before it).  topk_idx/topk_p/dest/perm/gate/cta_hist as in the
+// three-launch path; assigned/kept/offsets are written by CTA 0.
+// fused_forward_reset_sync: puts the device's grid-barrier words back to zero (after a launch whose
+// bounded waits ran out).
+bool fused_forward_supported(const Dims& D);
+int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
+                         float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
+                         int32_t* perm, float* gate, int32_t* cta_hist, int32_t* status, cudaStream_t st);
+int fused_forward_reset_sync(cudaStream_t st);
+
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);
 

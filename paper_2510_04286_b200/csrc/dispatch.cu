@@ -11,6 +11,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "dispatch_body.cuh"
 
 namespace slicemoe {
 namespace {
@@ -165,165 +166,17 @@ dispatch_scatter_kernel(const T* __restrict__ X, const int32_t* __restrict__ top
 }
 
 
-// Fused dispatch for the forward call.  Chunk c is the row range that CTA c of the tensor-core
-// router handled; `table[c][e]` is how many pairs of that chunk chose expert e (written by the
-// router).  Every CTA derives from the table (G x E, a few KB) the rank of its chunk's first pair
-// inside each expert, the totals, kept = min(total, C) and the offsets -- redundantly, which is
-// cheaper than a separate scan launch -- and then ranks its own pairs in stable (n, j) order.
-// The chunk is taken in segments of kSegPairs pairs: a segment's expert ids and probabilities are
-// brought into shared memory with all loads in flight at once (the ranking loop itself is a chain
-// of dependent warp votes and would otherwise pay the memory latency once per 32 pairs), then
-// counted per warp, prefixed over warps, and ranked with match-any inside the warp.
 constexpr int kFusedThreads = 512;
-constexpr int kFusedWarps = kFusedThreads / 32;
-constexpr int kSegPairs = 8192;
 
 __global__ void __launch_bounds__(kFusedThreads)
 dispatch_fused_kernel(const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_p,
-                      const int32_t* __restrict__ table, int G, int R, int E, int k, int pairs_per_chunk,
+                      const int32_t* __restrict__ table, int G, int R, int E, int pairs_per_chunk,
                       int capacity, int32_t* __restrict__ assigned, int32_t* __restrict__ kept,
                       int32_t* __restrict__ offsets, int32_t* __restrict__ dest, int32_t* __restrict__ perm,
                       float* __restrict__ gate) {
     extern __shared__ __align__(16) int sm[];
-    int* seg_e = sm;                               // [kSegPairs]  (16-byte aligned: first)
-    float* seg_p = reinterpret_cast<float*>(seg_e + kSegPairs);   // [kSegPairs]
-    int* base = seg_e + 2 * kSegPairs;             // [E]   rank of the next segment's first pair inside each expert
-    int* total = base + E;                         // [E]
-    int* offs = total + E;                         // [E+1]
-    int* wcnt = offs + E + 1;                      // [kFusedWarps][E]
-    int* tab = wcnt + kFusedWarps * E;             // [G][E] copy of the table
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int chunk = blockIdx.x;
-    const long long chunk_begin = (long long)chunk * pairs_per_chunk;
-    long long chunk_end = chunk_begin + pairs_per_chunk;
-    if (chunk_end > R) chunk_end = R;
-
-    // Segment loader.  chunk_begin and kSegPairs are multiples of 4, both arrays 16-byte aligned.
-    auto load_segment = [&](long long seg_begin, int n) {
-        const int nvec = n >> 2;
-        const int4* gi = reinterpret_cast<const int4*>(topk_idx + seg_begin);
-        const float4* gp = reinterpret_cast<const float4*>(topk_p + seg_begin);
-#pragma unroll 4
-        for (int v = threadIdx.x; v < nvec; v += kFusedThreads) {
-            reinterpret_cast<int4*>(seg_e)[v] = __ldg(gi + v);
-            reinterpret_cast<float4*>(seg_p)[v] = __ldg(gp + v);
-        }
-        for (int i = (nvec << 2) + threadIdx.x; i < n; i += kFusedThreads) {
-            seg_e[i] = topk_idx[seg_begin + i];
-            seg_p[i] = topk_p[seg_begin + i];
-        }
-    };
-    // the first segment's loads go out before the table work
-    const bool has_pairs = chunk_begin < chunk_end;
-    if (has_pairs) load_segment(chunk_begin, (int)min((long long)kSegPairs, chunk_end - chunk_begin));
-
-    for (int i = threadIdx.x; i < G * E; i += kFusedThreads) tab[i] = table[i];   // coalesced
-    for (int e = threadIdx.x; e < 2 * E; e += kFusedThreads) base[e] = 0;        // base and total
-    __syncthreads();
-    {
-        // thread (part, e) sums the table rows c = part, part + parts, ... of expert e
-        const int parts = kFusedThreads / E > 0 ? kFusedThreads / E : 1;
-        for (int idx = threadIdx.x; idx < parts * E; idx += kFusedThreads) {
-            const int e = idx % E, part = idx / E;
-            int before = 0, tot = 0;
-            for (int c = part; c < G; c += parts) {
-                const int v = tab[c * E + e];
-                if (c < chunk) before += v;
-                tot += v;
-            }
-            if (before) atomicAdd(&base[e], before);
-            if (tot) atomicAdd(&total[e], tot);
-        }
-    }
-    __syncthreads();
-    if (warp == 0) {
-        // kept = min(total, C) and its exclusive scan over the experts
-        int run = 0;
-        for (int e0 = 0; e0 < E; e0 += 32) {
-            const int e = e0 + lane;
-            const int tot = e < E ? total[e] : 0;
-            const int kp = (capacity > 0 && tot > capacity) ? capacity : tot;
-            int incl = kp;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, d);
-                if (lane >= d) incl += up;
-            }
-            if (e < E) {
-                offs[e] = run + incl - kp;
-                if (chunk == 0) {
-                    if (assigned) assigned[e] = tot;
-                    kept[e] = kp;
-                    offsets[e] = run + incl - kp;
-                }
-            }
-            run += __shfl_sync(0xffffffffu, incl, 31);
-        }
-        if (lane == 0) {
-            offs[E] = run;
-            if (chunk == 0) offsets[E] = run;
-        }
-    }
-    __syncthreads();
-    if (!has_pairs) return;
-
-    int* mine = wcnt + warp * E;
-    for (long long seg_begin = chunk_begin; seg_begin < chunk_end; seg_begin += kSegPairs) {
-        const int n = (int)min((long long)kSegPairs, chunk_end - seg_begin);
-        if (seg_begin != chunk_begin) {
-            __syncthreads();             // everyone is done with the previous segment's staging
-            load_segment(seg_begin, n);
-        }
-        for (int e = lane; e < E; e += 32) mine[e] = 0;
-        __syncthreads();
-        const int per_warp = ((n + kFusedWarps - 1) / kFusedWarps + 31) / 32 * 32;   // multiple of 32
-        const int w_begin = warp * per_warp;
-        const int w_end = min(n, w_begin + per_warp);
-        for (int i = w_begin + lane; i < w_end; i += 32) {
-            const int e = seg_e[i];
-            if (e >= 0 && e < E) atomicAdd(&mine[e], 1);
-        }
-        __syncthreads();
-        for (int e = threadIdx.x; e < E; e += kFusedThreads) {
-            int run = base[e];
-            for (int w = 0; w < kFusedWarps; ++w) {
-                const int t = wcnt[w * E + e];
-                wcnt[w * E + e] = run;
-                run += t;
-            }
-            base[e] = run;               // rank of the next segment's first pair
-        }
-        __syncthreads();
-        for (int i0 = w_begin; i0 < w_end; i0 += 32) {
-            const int i = i0 + lane;
-            int e = -1;
-            float p = 0.0f;
-            if (i < w_end) {
-                e = seg_e[i];
-                p = seg_p[i];
-                if (e < 0 || e >= E) e = -1;
-            }
-            const int key = e >= 0 ? e : -1 - lane;
-            const unsigned grp = __match_any_sync(0xffffffffu, key);
-            const int before = __popc(grp & ((1u << lane) - 1u));
-            int d = -1;
-            if (e >= 0) {
-                const int rank = mine[e] + before;
-                if (capacity == 0 || rank < capacity) d = offs[e] + rank;
-            }
-            __syncwarp();
-            if (e >= 0 && before == 0) mine[e] += __popc(grp);
-            __syncwarp();
-            if (i < w_end) {
-                const long long pair = seg_begin + i;
-                dest[pair] = d;
-                if (d >= 0) {
-                    perm[d] = (int)pair;
-                    gate[d] = p;
-                }
-            }
-        }
-    }
+    dispatch_fused_body<kFusedThreads, false>(topk_idx, topk_p, table, G, (int)blockIdx.x, R, E, pairs_per_chunk,
+                                              capacity, assigned, kept, offsets, dest, perm, gate, sm);
 }
 
 }  // namespace
@@ -358,11 +211,11 @@ int launch_dispatch_fused(const Dims& D, const int32_t* topk_idx, const float* t
                           int grid, int rows_per_cta, int32_t* assigned, int32_t* kept, int32_t* offsets,
                           int32_t* dest, int32_t* perm, float* gate, cudaStream_t st) {
     if (grid <= 0) return SLICEMOE_ERR_SHAPE;
-    const size_t smem = sizeof(int) * (2 * (size_t)kSegPairs + (size_t)D.E * (kFusedWarps + 3 + grid) + 1);
+    const size_t smem = dispatch_fused_smem_bytes(D.E, grid, kFusedThreads);
     if (smem > 227 * 1024) return SLICEMOE_ERR_UNSUPPORTED;
     if (smem > 48 * 1024)
         SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(dispatch_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    dispatch_fused_kernel<<<grid, kFusedThreads, smem, st>>>(topk_idx, topk_p, cta_hist, grid, D.R, D.E, D.k,
+    dispatch_fused_kernel<<<grid, kFusedThreads, smem, st>>>(topk_idx, topk_p, cta_hist, grid, D.R, D.E,
                                                             rows_per_cta * D.k, D.capacity, assigned, kept, offsets,
                                                             dest, perm, gate);
     SLICEMOE_LAUNCH_CHECK(1);

@@ -1,0 +1,1018 @@
+// Tensor-core path (sm_100a: tcgen05 + TMEM + TMA) for the two MLPs of the layer, bf16 storage:
+//
+//   router  (Section 3.1): relu(X Wr1^T + br1) Wr2^T + br2 -> softmax -> top-k   (per 128-row tile)
+//   experts (Section 3.1 / 3.4): act(X~_e W1_e^T + b1_e) W2_e^T + b2_e           (per 128-row tile of
+//                                                                                 one expert's rows)
+//
+// Both are the same pipeline (tc_body): GEMM-1 into a TMEM accumulator, an epilogue that applies
+// gate, bias and activation and writes the hidden chunk as bf16 pairs back into TMEM, GEMM-2 with
+// that chunk as its TMEM-resident A operand into a second TMEM accumulator, and a final epilogue
+// (softmax + top-k + histogram for the router; bias + store or add for the experts).  The hidden
+// layer is processed in chunks of HC units and never leaves tensor memory.
+//
+// One persistent CTA per SM walks a contiguous range of tiles (expert-major, so expert weights
+// stay in shared memory while the expert does not change).  Warp roles:
+//   warp 0            TMA producer (one lane): weight chunks with their bias, and the row tiles
+//                     unless they are gathered
+//   warp 1            GEMM-1 issue (one lane)
+//   warp 2            GEMM-2 issue (one lane); two issuing threads because the small MMAs of this
+//                     layer (N <= 128) are issue-bound, not tensor-bound
+//   warp 3            fused forward only.  Router: zeroes this CTA's rows of h' (the experts add
+//                     into it).  Experts: gathers the next tiles' rows of h through perm with
+//                     asynchronous 16-byte copies into the swizzled A buffers, together with the
+//                     rows' gates and pair indices
+//   activation warps  two groups that take the hidden chunks in turn, each two warpgroups that
+//                     split a chunk's columns; GEMM-1 accumulators are double-buffered
+//   last warpgroup    output: final accumulator -> softmax/top-k, or bias + store / add into h'
+// A warp reads TMEM lanes 32*(warp_id % 4)..+31: one tile row per thread.
+// All hand-offs are mbarriers; every wait is bounded and a run-out sets the status word and makes
+// all roles leave.
+//
+// This header holds the device code and the launch helpers; tc_mlp.cu wraps tc_body in the router
+// and expert kernels, fused_forward.cu in the single-kernel forward.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace slicemoe {
+namespace {
+
+using namespace ptx;
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that takes 2 s is a bug, not load
+constexpr int kMaxHid = 1024;
+constexpr int kMaxE = 256;
+// Depth of the per-tile metadata ring.  An entry is rewritten once GEMM-1 of the tile kMetaRing - 3
+// tiles later has finished (three A buffers), by which time the activation warps have read their
+// accumulators for the old tile and the output warps, at most two accumulators and one tile of
+// GEMM-1 run-ahead behind, have stored it.
+constexpr int kMetaRing = 8;
+constexpr int kMaxBars = 40;
+
+struct TcParams {
+    const int32_t* offsets;   // experts: [E+1] device row ranges; router: nullptr
+    int n_rows;               // router: N; experts: R (length of the stacked-row arrays)
+    int E;                    // experts: E; router: 1
+    int HID;                  // Hr or F
+    const bf16* bias1;        // [E, HID] or nullptr
+    const bf16* bias2;        // [E, N2]  or nullptr
+    bf16* yperm;              // experts: output rows [R, N2]
+    // experts, fused forward: A rows are gathered instead of read from stacked rows
+    const bf16* gather_src;   // h viewed as X[N, K1], or nullptr (A = stacked rows via TMA)
+    const int32_t* perm;      // [R] pair index n*k + j of each stacked row
+    const float* gate;        // [R] gate value of each stacked row
+    int gather_k;             // k (pairs per row)
+    bf16* scatter_out;        // fused forward, k <= 2: h' viewed as Y[N, N2]; the row of pair (n, j) is added to
+                              // Y[n, :] (h' zeroed beforehand) instead of being stored to yperm; or nullptr
+    // router, fused forward: this CTA also zeroes the rows of zero_out that it routes
+    bf16* zero_out;           // h' viewed as Y[N, zero_cols], or nullptr
+    int zero_cols;
+    int32_t* topk_idx;        // router outputs
+    float* topk_p;
+    int32_t* assigned;        // global counts, added atomically (or nullptr)
+    int32_t* cta_hist;        // [gridDim.x, N2] this CTA's counts (or nullptr): input of the fused dispatch
+    float* probs;             // or nullptr
+    int k;
+    int32_t* status;
+};
+
+// Optional timeline tracing (development builds only: -DSLICEMOE_TC_TRACE).  CTA 0 stamps
+// (event code, SM clock) pairs per role into a caller-provided buffer.
+#ifdef SLICEMOE_TC_TRACE
+constexpr int kTraceSlots = 8, kTraceEvents = 2048, kTraceSmemEvents = 320;
+__device__ unsigned long long* g_trace_buf = nullptr;
+// Events go to shared memory (cheap) and are copied out at the end of the kernel.
+struct Tracer {
+    uint2* base;
+    int n;
+    __device__ Tracer(int slot) : base(nullptr), n(0) {
+        extern __shared__ uint8_t smem_raw[];
+        if (blockIdx.x == 0 && g_trace_buf && slot < 6)
+            base = reinterpret_cast<uint2*>(smem_raw + 200 * 1024) + slot * kTraceSmemEvents;
+    }
+    __device__ void operator()(int code) {
+        if (base && n < kTraceSmemEvents) { base[n] = make_uint2((unsigned)code, (unsigned)clock64()); ++n; }
+    }
+};
+#define TRACE_DECL(name, slot) Tracer name(slot)
+#define TRACE(name, code) name(code)
+#else
+#define TRACE_DECL(name, slot)
+#define TRACE(name, code)
+#endif
+
+constexpr int pow2_at_least(int x) {
+    int p = 32;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+template <int K1_, int N2_, bool ROUTER_, int ACT_>
+struct TcCfg {
+    static constexpr int K1 = K1_, N2 = N2_, ACT = ACT_;
+    static constexpr bool ROUTER = ROUTER_;
+    static constexpr int HC = (K1 == 64) ? 128 : 64;           // hidden units per chunk
+    // row-tile buffers: three where they fit (the fused forward gathers two tiles ahead); with
+    // 256-wide rows (64 KB per tile) the router gets two and the experts, whose weight stages are
+    // larger, one
+    static constexpr int A_BUFS = (K1 <= 128) ? 3 : (ROUTER_ ? 2 : 1);
+    static constexpr int W_STAGES = (K1 == 128) ? 3 : 2;
+    // Activation warps: NGRP groups that take the hidden chunks in turn (chunk g goes to group
+    // g mod NGRP), each group GWG warpgroups that split the chunk's columns.  With two groups one
+    // group's accumulator loads, tails and stores run while the other group's tanh work occupies
+    // the tanh unit.  256-wide rows get one group: their wide output epilogue needs the larger
+    // register budget of a 512-thread CTA.
+    static constexpr int NGRP = (K1 == 256) ? 1 : 2;
+    static constexpr int GWG = 2;
+    static constexpr int NWG = NGRP * GWG;
+    static constexpr int NBUF = 2;                              // GEMM-1 accumulator / hidden buffers
+    static constexpr int GRP_WARPS = GWG * 4;                   // warps that work on one chunk
+    static constexpr int THREADS = 128 + NWG * 128 + 128;
+    static constexpr int OUT_WARP0 = 4 + NWG * 4;               // first warp of the output warpgroup
+    static constexpr int ACC2_BUFS = (N2 <= 128) ? 2 : 1;
+    // The router keeps the hidden layer as a bf16 pair (hi + lo = 16 mantissa bits): GEMM-2 runs
+    // over both halves against the same weights, so that the logits carry fp32-level accuracy and
+    // the top-k decision does not depend on bf16 rounding of the hidden layer.
+    // The experts keep it as plain bf16; their activation math is packed 2-wide bf16.
+    // (A and B of one MMA must have the same 16-bit format: fp16 hidden x bf16 weights is an
+    // illegal instruction on sm_100a.)
+    static constexpr int H_PARTS = ROUTER_ ? 2 : 1;
+    static constexpr bool PACKED_ACT = !ROUTER_;
+    // TMEM columns:
+    //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w of the group that has the chunk
+    //                        owns columns [w HC/GWG, (w+1) HC/GWG).  Router: once a thread has
+    //                        read a 16-column piece it writes the piece's hi half (8 packed
+    //                        columns) over the start of its own column range, so the chunk's hi
+    //                        half ends up in GWG runs of HC/(2 GWG) columns.
+    //   [2 HC, 3 HC)         two hidden buffers of HC/2 packed columns: the experts' hidden chunk
+    //                        (so GEMM-1 of a later chunk need not wait for GEMM-2), or the
+    //                        router's lo half.
+    //   [3 HC, ...)          ACC2_BUFS final accumulators of N2 columns.
+    static constexpr int H_COL0 = NBUF * HC;
+    static constexpr int ACC2_COL0 = H_COL0 + NBUF * (HC / 2);
+    static constexpr int TMEM_COLS = pow2_at_least(ACC2_COL0 + ACC2_BUFS * N2);
+    static constexpr int KSTEPS_PER_WG = HC / (16 * GWG);       // 16-element K steps in one warpgroup's columns
+    static constexpr int KP1 = K1 / 64;                         // 64-wide K panels of GEMM-1
+    static constexpr int KP2 = HC / 64;                         // K panels of GEMM-2 per chunk
+    static constexpr int A_PANEL = 128 * 128;                   // bytes: 128 rows x 128 B
+    static constexpr int A_BYTES = KP1 * A_PANEL;
+    static constexpr int W1_PANEL = HC * 128;
+    static constexpr int W1C_BYTES = KP1 * W1_PANEL;
+    static constexpr int W2_PANEL = N2 * 128;
+    static constexpr int W2C_BYTES = KP2 * W2_PANEL;
+    static constexpr int W_STAGE_BYTES = W1C_BYTES + W2C_BYTES;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_W = OFF_A + A_BUFS * A_BYTES;
+    static constexpr int B1_BYTES = HC * 2;                     // one chunk of the first layer's bias, per weight stage
+    static constexpr int OFF_B1 = OFF_W + W_STAGES * W_STAGE_BYTES;
+    static constexpr int SMEM_BYTES = OFF_B1 + W_STAGES * B1_BYTES;
+    // at least 120 KiB is requested so that two CTAs never share an SM (each allocates most of TMEM)
+    static constexpr int SMEM_ALLOC = (SMEM_BYTES + 1024 > 120 * 1024) ? SMEM_BYTES + 1024 : 120 * 1024;
+    static constexpr int PIECE = 16;                            // accumulator columns per piece
+    static constexpr int NPIECE = HC / (PIECE * GWG);           // pieces per thread and chunk
+    static constexpr int SUB = (NPIECE > 2) ? 2 : NPIECE;       // pieces held in registers at once (experts)
+    static_assert(NBUF % NGRP == 0 && NPIECE % SUB == 0, "chunk-to-group and piece-to-batch maps");
+    static_assert(NPIECE >= 1, "hidden chunk too narrow for the activation warpgroups");
+    static_assert(W_STAGE_BYTES % 1024 == 0 && W1C_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+    static_assert(N2 % 16 == 0 && N2 >= 16 && N2 <= 256, "MMA N");
+    static_assert(SMEM_ALLOC <= 232448, "shared memory budget");
+    static_assert(ACC2_COL0 + ACC2_BUFS * N2 <= 512, "TMEM budget");
+};
+
+// Barrier slots in shared memory.
+template <class C>
+struct Bars {
+    static constexpr int A_FULL = 0;
+    static constexpr int A_EMPTY = A_FULL + C::A_BUFS;
+    static constexpr int W_FULL = A_EMPTY + C::A_BUFS;
+    static constexpr int W_EMPTY = W_FULL + C::W_STAGES;
+    static constexpr int ACC1_FULL = W_EMPTY + C::W_STAGES;   // GEMM-1 done (MMA -> activation)
+    // accumulator may be overwritten: experts, all activation warps have read it;
+    // router (hidden chunk lives in it), GEMM-2 has consumed it
+    static constexpr int ACC1_EMPTY = ACC1_FULL + C::NBUF;
+    static constexpr int H_FULL = ACC1_EMPTY + C::NBUF;       // hidden chunk written (activation -> MMA)
+    static constexpr int H_EMPTY = H_FULL + C::NBUF;          // experts: GEMM-2 has consumed the hidden buffer
+    static constexpr int ACC2_FULL = H_EMPTY + C::NBUF;
+    static constexpr int ACC2_EMPTY = ACC2_FULL + C::ACC2_BUFS;
+    static constexpr int DRAIN = ACC2_EMPTY + C::ACC2_BUFS;
+    static constexpr int COUNT = DRAIN + 2;
+};
+
+__device__ __forceinline__ void locate_tile(const int* tile_start, const int* offs, int t, int& e,
+                                            int& row0, int& rows) {
+    while (t >= tile_start[e + 1]) ++e;
+    row0 = offs[e] + (t - tile_start[e]) * kTileM;
+    rows = min(kTileM, offs[e + 1] - row0);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Expert activation, all arithmetic 2-wide in bf16 on one thread's 16-column piece of a row:
+//   convert   z = bf16(acc) * gate + bias             one conversion, two multiply-adds per pair (the gate
+//                                                     as a bf16 pair hi + lo: rounding it to one bf16
+//                                                     would tilt a whole row's pre-activations together)
+//   pre       t = tanh(z (c0 + c1 z^2))               three multiply-adds and one packed tanh per pair
+//   post      2 gelu(z) = z t + z                     one multiply-add per pair
+// GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))); the factor 0.5 is applied to
+// the GEMM-2 accumulator in the output epilogue (exact: a power of two).  Where z^2 overflows, tanh
+// saturates to +-1 and the formula still returns 2z (z > 0) or 0 (z < 0).
+// The tanh unit (16 results per clock per SM) is the scarce resource; the instruction count around
+// it is kept low enough that the issue slots are not the next one.
+__device__ __forceinline__ void convert_piece_bf16x2(const uint32_t* cur, __nv_bfloat162 gate_hi, __nv_bfloat162 gate_lo,
+                                                     const uint4* bias8, bool has_bias, __nv_bfloat162* z) {
+    uint4 braw[2];
+    if (has_bias) { braw[0] = bias8[0]; braw[1] = bias8[1]; }      // 16 packed bf16, warp-wide broadcast
+    else braw[0] = braw[1] = make_uint4(0u, 0u, 0u, 0u);
+    const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(braw);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
+        z[i] = __hfma2(a, gate_hi, __hfma2(a, gate_lo, b2[i]));
+    }
+}
+template <int ACT>
+__device__ __forceinline__ void activate_pre_bf16x2(const __nv_bfloat162* z, __nv_bfloat162* t) {
+    constexpr int P = 8;   // column pairs per piece
+#ifdef SLICEMOE_TC_SKELETON   // development: time the pipeline without the activation math
+    return;
+#endif
+    if (ACT == SLICEMOE_ACT_RELU) return;
+    const __nv_bfloat162 c0 = __float2bfloat162_rn(0.7978845608f), c1 = __float2bfloat162_rn(0.0356774081f);
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+        const __nv_bfloat162 inner = __hfma2(__hmul2(z[i], z[i]), c1, c0);
+        const __nv_bfloat162 u = __hmul2(z[i], inner);
+        uint32_t ur = *reinterpret_cast<const uint32_t*>(&u), tr;
+        asm volatile("tanh.approx.bf16x2 %0, %1;" : "=r"(tr) : "r"(ur));
+        t[i] = *reinterpret_cast<__nv_bfloat162*>(&tr);
+    }
+}
+template <int ACT>
+__device__ __forceinline__ void activate_post_bf16x2(const __nv_bfloat162* z, const __nv_bfloat162* t, uint32_t* out) {
+    constexpr int P = 8;
+#ifdef SLICEMOE_TC_SKELETON
+    const bool relu = true;
+#else
+    const bool relu = ACT == SLICEMOE_ACT_RELU;
+#endif
+    if (relu) {
+        const __nv_bfloat162 zero = __float2bfloat162_rn(0.0f);
+#pragma unroll
+        for (int i = 0; i < P; ++i) {
+            const __nv_bfloat162 r = __hmax2(z[i], zero);
+            out[i] = *reinterpret_cast<const uint32_t*>(&r);
+        }
+        return;
+    }
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+        const __nv_bfloat162 r = __hfma2(z[i], t[i], z[i]);
+        out[i] = *reinterpret_cast<const uint32_t*>(&r);
+    }
+}
+// factor the output epilogue applies to the GEMM-2 accumulator (see above)
+template <int ACT>
+constexpr float kOutScale =
+#ifdef SLICEMOE_TC_SKELETON
+    1.0f;
+#else
+    (ACT == SLICEMOE_ACT_RELU) ? 1.0f : 0.5f;
+#endif
+
+// Router: ReLU in fp32, then each value as a bf16 pair, the rounded value (hi) and the rounded
+// remainder (lo); hi + lo carries 16 mantissa bits of the fp32 value.
+__device__ __forceinline__ void relu_split_piece(const uint32_t* cur, uint32_t* hi, uint32_t* lo) {
+    constexpr int P = 8;
+    float a[2 * P];
+#pragma unroll
+    for (int i = 0; i < 2 * P; ++i) a[i] = fmaxf(__uint_as_float(cur[i]), 0.0f);
+#pragma unroll
+    for (int i = 0; i < P; ++i) hi[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+        a[2 * i] -= __uint_as_float(hi[i] << 16);
+        a[2 * i + 1] -= __uint_as_float(hi[i] & 0xFFFF0000u);
+    }
+#pragma unroll
+    for (int i = 0; i < P; ++i) lo[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+}
+
+// Shared-memory state of one CTA besides the operand tiles.
+struct TcShared {
+    __align__(8) uint64_t bars[kMaxBars];
+    int tile_start[kMaxE + 1];
+    int offs[kMaxE + 1];
+    int hist[kMaxE];
+    uint32_t tmem_base;
+    int abort_flag;
+    // fused forward: per-row gate (Eq. 1) and pair index of the tiles in flight, copied in by the
+    // gather warp with the rows themselves (ring over the CTA's tile counter)
+    float gate_s[kMetaRing][kTileM];
+    int pair_s[kMetaRing][kTileM];
+};
+
+// Loads of data that an earlier phase of the same launch may have written (single-kernel forward)
+// must not take the non-coherent path.
+template <bool SAME_LAUNCH>
+__device__ __forceinline__ int ld_index(const int32_t* ptr) {
+    if (SAME_LAUNCH) return __ldcg(ptr);
+    return __ldg(ptr);
+}
+
+// One pass of the two-layer MLP pipeline over this CTA's share of the row tiles: the body of the
+// router and expert kernels, and of the router and expert phases of the single-kernel forward.
+// Called by all threads of the CTA; TMEM (sh.tmem_base, at least C::TMEM_COLS columns) is allocated
+// and freed by the caller.  SAME_LAUNCH: offsets / perm / gate were written earlier in this launch.
+template <class C, bool SAME_LAUNCH>
+__device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p,
+                                        const TcParams& p, TcShared& sh, uint8_t* smem_raw) {
+    using B = Bars<C>;
+    static_assert(B::COUNT <= kMaxBars, "barrier slots");
+    const CUtensorMap& tmA = *tmA_p;
+    const CUtensorMap& tmW1 = *tmW1_p;
+    const CUtensorMap& tmW2 = *tmW2_p;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    volatile int* abort = &sh.abort_flag;
+    const int nchunks = p.HID / C::HC;
+    const bool resident = nchunks <= C::W_STAGES;
+    const bool gather = !C::ROUTER && p.gather_src != nullptr;
+    auto bar = [&](int i) { return smem_u32(&sh.bars[i]); };
+
+#ifdef SLICEMOE_TC_TRACE
+    for (int i = threadIdx.x; i < 6 * kTraceSmemEvents * 2; i += C::THREADS)
+        reinterpret_cast<uint32_t*>(smem_raw + 200 * 1024)[i] = 0;
+#endif
+    // ---- set-up ---------------------------------------------------------------------------
+    if (threadIdx.x == 0) {
+#ifdef SLICEMOE_TC_TRACE
+        { TRACE_DECL(tr0, 5); TRACE(tr0, 99); }
+#endif
+        sh.abort_flag = 0;
+        for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 32 : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
+        for (int i = 0; i < C::W_STAGES; ++i) { mbar_init(bar(B::W_FULL + i), 1); mbar_init(bar(B::W_EMPTY + i), 1); }
+        for (int i = 0; i < C::NBUF; ++i) {
+            mbar_init(bar(B::ACC1_FULL + i), 1);
+            mbar_init(bar(B::ACC1_EMPTY + i), C::ROUTER ? 1 : C::GRP_WARPS);
+            mbar_init(bar(B::H_FULL + i), C::GRP_WARPS);
+            mbar_init(bar(B::H_EMPTY + i), 1);
+        }
+        for (int i = 0; i < C::ACC2_BUFS; ++i) {
+            mbar_init(bar(B::ACC2_FULL + i), 1);
+            mbar_init(bar(B::ACC2_EMPTY + i), 4);
+        }
+        mbar_init(bar(B::DRAIN), 1);
+        mbar_init(bar(B::DRAIN + 1), 1);
+        fence_mbar_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmW1);
+        prefetch_tensormap(&tmW2);
+    }
+    for (int e = threadIdx.x; e <= p.E; e += C::THREADS) sh.offs[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.n_rows);
+    for (int e = threadIdx.x; e < kMaxE; e += C::THREADS) sh.hist[e] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int e = 0; e < p.E; ++e) {
+            sh.tile_start[e] = run;
+            run += (sh.offs[e + 1] - sh.offs[e] + kTileM - 1) / kTileM;
+        }
+        sh.tile_start[p.E] = run;
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh.tmem_base;
+    const int total_tiles = sh.tile_start[p.E];
+    const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
+    const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
+    const int t_end = min(total_tiles, t_begin + per_cta);
+
+    const uint32_t sA = smem_base + C::OFF_A, sW = smem_base + C::OFF_W;
+#ifdef SLICEMOE_TC_TRACE
+    if (threadIdx.x == 0) { Tracer tr1(5); tr1.n = 1; tr1(98); }   // set-up finished
+#endif
+
+    if (warp == 0) {
+        // ================= TMA producer =====================================================
+        if (lane == 0 && t_begin < t_end) {
+            int e = 0, prev_e = -1;
+            uint32_t g = 0, reloads = 0;             // chunks seen; tiles that (re)loaded weights
+            uint32_t last_a_bar = 0, last_a_par = 0, last_w_bar = 0, last_w_par = 0;
+            bool ok = true;
+            TRACE_DECL(tr, 0);
+            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+                int row0, rows;
+                locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
+                const int ab = ta % C::A_BUFS;
+                const uint32_t an = ta / C::A_BUFS;
+                if (!gather) {
+                    TRACE(tr, 1);
+                    if (!mbar_wait(bar(B::A_EMPTY + ab), (an & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    TRACE(tr, 2);
+                    mbar_arrive_expect_tx(bar(B::A_FULL + ab), C::A_BYTES);
+#pragma unroll
+                    for (int kp = 0; kp < C::KP1; ++kp)
+                        tma_load_2d(sA + ab * C::A_BYTES + kp * C::A_PANEL, &tmA, kp * 64, row0, bar(B::A_FULL + ab));
+                    last_a_bar = bar(B::A_FULL + ab);
+                    last_a_par = an & 1u;
+                }
+                const bool reload = !resident || (e != prev_e);
+                prev_e = e;
+                if (!reload) { g += nchunks; continue; }
+                for (int c = 0; c < nchunks && ok; ++c, ++g) {
+                    // resident weights: slot = chunk, n-th load of the slot = n-th reloading tile;
+                    // streamed weights: slots in ring order
+                    const int slot = resident ? c : (int)(g % C::W_STAGES);
+                    const uint32_t n = resident ? reloads : g / C::W_STAGES;
+                    if (!mbar_wait(bar(B::W_EMPTY + slot), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(B::W_FULL + slot), C::W_STAGE_BYTES + (p.bias1 ? C::B1_BYTES : 0));
+                    const uint32_t dst = sW + slot * C::W_STAGE_BYTES;
+                    if (p.bias1)
+                        bulk_load(smem_base + C::OFF_B1 + slot * C::B1_BYTES, p.bias1 + (size_t)e * p.HID + c * C::HC,
+                                  C::B1_BYTES, bar(B::W_FULL + slot));
+#pragma unroll
+                    for (int kp = 0; kp < C::KP1; ++kp)
+                        tma_load_2d(dst + kp * C::W1_PANEL, &tmW1, kp * 64, e * p.HID + c * C::HC, bar(B::W_FULL + slot));
+#pragma unroll
+                    for (int kp = 0; kp < C::KP2; ++kp)
+                        tma_load_2d(dst + C::W1C_BYTES + kp * C::W2_PANEL, &tmW2, c * C::HC + kp * 64, e * C::N2,
+                                    bar(B::W_FULL + slot));
+                    last_w_bar = bar(B::W_FULL + slot);
+                    last_w_par = n & 1u;
+                }
+                ++reloads;
+            }
+            if (!ok || *abort) {
+                // leaving early: let this thread's last copies land first (bounded; the copies
+                // complete on their own, earlier ones were issued before these)
+                volatile int never = 0;
+                if (last_a_bar) mbar_wait(last_a_bar, last_a_par, &never, 10000000ull);
+                if (last_w_bar) mbar_wait(last_w_bar, last_w_par, &never, 10000000ull);
+            }
+        }
+    } else if (warp == 1) {
+        // ================= GEMM-1 issue ======================================================
+        if (lane == 0 && t_begin < t_end) {
+            constexpr uint32_t idesc1 = make_idesc(128, C::HC, kFmtBF16, kFmtBF16);
+            const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
+            bool ok = true;
+            TRACE_DECL(tr, 1);
+            int e = 0, prev_e = -1;
+            uint32_t g = 0, reloads = 0;
+            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+                int r0, rr;
+                locate_tile(sh.tile_start, sh.offs, t, e, r0, rr);
+                const bool reload = !resident || (e != prev_e);
+                prev_e = e;
+                const int ab = ta % C::A_BUFS;
+                TRACE(tr, 10);
+                if (!mbar_wait(bar(B::A_FULL + ab), (uint32_t)(ta / C::A_BUFS) & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                TRACE(tr, 11);
+                if (gather) fence_proxy_async_smem();   // rows written by cp.async -> visible to the MMA's reads
+                for (int c = 0; c < nchunks; ++c, ++g) {
+                    const int slot = resident ? c : (int)(g % C::W_STAGES);
+                    if (reload) {
+                        const uint32_t n = resident ? reloads : g / C::W_STAGES;
+                        if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    }
+                    const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
+                    TRACE(tr, 12);
+                    if (!mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    TRACE(tr, 13);
+                    tc_fence_after_sync();
+                    const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W_STAGE_BYTES) >> 4);
+                    const uint32_t d = tmem_base + b * C::HC;
+                    mma_ss<0>(d, a0, w0, idesc1);
+#ifndef SLICEMOE_DEV_G1_ONE   // development: time the pipeline with a single GEMM-1 MMA per chunk
+#pragma unroll
+                    for (int kk = 1; kk < C::K1 / 16; ++kk)
+                        mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
+                                  w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
+#endif
+                    mma_commit(bar(B::ACC1_FULL + b));
+                    if (c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
+                    TRACE(tr, 14);
+                }
+                if (reload) ++reloads;
+            }
+            if (!ok || *abort) {
+                // make sure no MMA of this thread is still running before TMEM is released
+                volatile int never = 0;
+                mma_commit(bar(B::DRAIN));
+                mbar_wait(bar(B::DRAIN), 0u, &never, 10000000ull);
+            }
+        }
+    } else if (warp == 2) {
+        // ================= GEMM-2 issue ======================================================
+        if (lane == 0 && t_begin < t_end) {
+            constexpr uint32_t idesc2 = make_idesc(128, C::N2, kFmtBF16, kFmtBF16);
+            const uint32_t dW = desc_lo_sw128(sW);
+            bool ok = true;
+            TRACE_DECL(tr, 4);
+            int e = 0, prev_e = -1;
+            uint32_t g = 0, reloads = 0;
+            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+                int r0, rr;
+                locate_tile(sh.tile_start, sh.offs, t, e, r0, rr);
+                const bool reload = !resident || (e != prev_e);
+                prev_e = e;
+                // resident weights are handed back only when the next tile brings another expert
+                bool release = !resident;
+                if (resident && t + 1 < t_end) {
+                    int e2 = e;
+                    locate_tile(sh.tile_start, sh.offs, t + 1, e2, r0, rr);
+                    release = (e2 != e);
+                }
+                const int buf = ta % C::ACC2_BUFS;
+                for (int c = 0; c < nchunks; ++c, ++g) {
+                    const int slot = resident ? c : (int)(g % C::W_STAGES);
+                    if (reload) {
+                        // (already observed by the GEMM-1 thread; waited here too so that this
+                        // thread's reads of the weight tile are ordered after the copy)
+                        const uint32_t n = resident ? reloads : g / C::W_STAGES;
+                        if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    }
+                    const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
+                    TRACE(tr, 20);
+                    if (!mbar_wait(bar(B::H_FULL + b), n1 & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    TRACE(tr, 21);
+                    if (c == 0 && !mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(ta / C::ACC2_BUFS) & 1u) ^ 1u,
+                                             abort, kWaitLimitNs)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t w0 = dW + ((slot * C::W_STAGE_BYTES + C::W1C_BYTES) >> 4);
+                    const uint32_t d = tmem_base + C::ACC2_COL0 + buf * C::N2;
+                    const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: chunk; router: lo half
+                    const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi half, two runs
+#pragma unroll
+                    for (int part = 0; part < C::H_PARTS; ++part) {
+#pragma unroll
+                        for (int kk = 0; kk < C::HC / 16; ++kk) {
+                            uint32_t a;
+                            if (C::ROUTER && part == 0)
+                                a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / C::GWG) + (kk % C::KSTEPS_PER_WG) * 8;
+                            else
+                                a = hbuf + kk * 8;
+                            const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
+                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, c > 0 ? 1u : 0u);
+#ifndef SLICEMOE_DEV_G2_ONE   // development: time the pipeline with a single GEMM-2 MMA per chunk
+                            else mma_ts<1>(d, a, bd, idesc2);
+#endif
+                        }
+                    }
+                    mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
+                    if (release) mma_commit(bar(B::W_EMPTY + slot));
+                    if (c == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
+                    TRACE(tr, 22);
+                }
+                if (reload) ++reloads;
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                mma_commit(bar(B::DRAIN + 1));
+                mbar_wait(bar(B::DRAIN + 1), 0u, &never, 10000000ull);
+            }
+        }
+    } else if (warp == 3) {
+        if constexpr (C::ROUTER) {
+            // ============= zero this CTA's rows of h' (router, fused forward) ================
+            if (p.zero_out != nullptr && t_begin < t_end) {
+                const long long row_lo = (long long)t_begin * kTileM;
+                long long row_hi = (long long)t_end * kTileM;
+                if (row_hi > p.n_rows) row_hi = p.n_rows;
+                uint4* dst = reinterpret_cast<uint4*>(p.zero_out + row_lo * p.zero_cols);
+                const long long nvec = (row_hi - row_lo) * p.zero_cols / 8;
+                const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                for (long long i = lane; i < nvec; i += 32) dst[i] = z;
+            }
+        } else if (gather && t_begin < t_end) {
+            // ============= gather warp (experts, fused forward) ===============================
+            // Row r of a tile is stacked row row0 + r = pair perm[row0 + r] = (n, j); its A row is
+            // X[n, :], copied asynchronously (no registers) into the K-major 128-byte-swizzled
+            // layout.  The gate of Eq. 1 multiplies the GEMM-1 accumulator instead of the row.
+            // The warp runs ahead of the MMAs by as many tiles as there are A buffers.
+            constexpr int CPR = C::K1 / 8;            // 16-byte chunks per row
+            constexpr int RPI = 32 / CPR;             // rows covered by one warp-wide copy
+            const int ch = lane % CPR, rsub = lane / CPR;
+            int ge = 0, gm = 0;
+            bool ok = true;
+            int nrow[4], nnext[4];                    // source rows of tile rows lane + 32 q
+            // (the loaded pair index is left untouched until the next tile, so that the load's latency
+            // is not waited for here)
+            auto load_rows = [&](int t, int* out) {
+                int row0, rows;
+                locate_tile(sh.tile_start, sh.offs, t, ge, row0, rows);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int r = lane + 32 * q;
+                    out[q] = (r < rows) ? ld_index<SAME_LAUNCH>(p.perm + row0 + r) : -1;
+                }
+            };
+            load_rows(t_begin, nnext);
+            TRACE_DECL(tr, lane == 0 ? 0 : 7);
+            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+                TRACE(tr, 1);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) nrow[q] = nnext[q] < 0 ? -1 : nnext[q] / p.gather_k;
+#ifdef SLICEMOE_TC_TRACE
+#pragma unroll
+                for (int q = 0; q < 4; ++q) asm volatile("mov.b32 %0, %0;" : "+r"(nrow[q]));
+                TRACE(tr, 4);
+#endif
+                if (t + 1 < t_end) load_rows(t + 1, nnext);
+                TRACE(tr, 5);
+                const int ab = ta % C::A_BUFS;
+                ok = mbar_wait(bar(B::A_EMPTY + ab), ((uint32_t)(ta / C::A_BUFS) & 1u) ^ 1u, abort, kWaitLimitNs);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                TRACE(tr, 2);
+                const uint32_t dst0 = sA + ab * C::A_BYTES + (ch >> 3) * C::A_PANEL;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+#pragma unroll 8
+                    for (int i = 0; i < 32 / RPI; ++i) {
+                        const int r32 = i * RPI + rsub;                 // row within this block of 32
+                        const int r = q * 32 + r32;
+                        const int n = __shfl_sync(0xffffffffu, nrow[q], r32);
+                        const bf16* src = p.gather_src + (size_t)(n < 0 ? 0 : n) * C::K1 + ch * 8;
+                        cp_async_16(dst0 + (r >> 3) * 1024 + (r & 7) * 128 + (((ch & 7) ^ (r & 7)) << 4), src,
+                                    n < 0 ? 0u : 16u);
+                    }
+                }
+                {
+                    int row0, rows;
+                    locate_tile(sh.tile_start, sh.offs, t, gm, row0, rows);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        // rows past the tile's end take a neighbour's values: their A rows are zero and
+                        // they are never stored
+                        const int r = lane + 32 * q, src = min(row0 + r, p.n_rows - 1);
+                        cp_async_4(smem_u32(&sh.gate_s[ta % kMetaRing][r]), p.gate + src);
+                        cp_async_4(smem_u32(&sh.pair_s[ta % kMetaRing][r]), p.perm + src);
+                    }
+                }
+                cp_async_mbar_arrive_noinc(bar(B::A_FULL + ab));
+                TRACE(tr, 3);
+            }
+            cp_async_wait_all();
+        }
+    } else if (warp >= 4 && warp < C::OUT_WARP0) {
+        // ================= activation warpgroups =============================================
+        const int grp = (warp - 4) / C::GRP_WARPS;    // which chunks: g mod NGRP == grp
+        const int w = ((warp - 4) >> 2) % C::GWG;     // warpgroup within the group = which part of the chunk's columns
+        const int lg = warp & 3;                      // TMEM lane group this warp may access
+        const uint32_t lane_base = tmem_base + ((uint32_t)(lg * 32) << 16);
+        constexpr int WCOLS = C::HC / C::GWG;         // accumulator columns per thread and chunk
+        bool ok = true;
+        int e = 0;
+        uint32_t g = 0;
+        TRACE_DECL(tr, (lg == 0 && lane == 0 && w == 0) ? 2 + grp : 7);
+#ifdef SLICEMOE_TC_ACCT   // development: where do the activation warps spend their cycles?
+        long long acct_wait_acc1 = 0, acct_wait_hempty = 0, acct_stwait = 0, acct_t0 = clock64(), acct_mark;
+#define ACCT_BEGIN() acct_mark = clock64()
+#define ACCT_END(var) var += clock64() - acct_mark
+#else
+#define ACCT_BEGIN()
+#define ACCT_END(var)
+#endif
+#ifdef SLICEMOE_TC_PROBE   // development: clock stamps inside one chunk (g == 12) of one warp
+        unsigned probe[16];
+        for (int i = 0; i < 16; ++i) probe[i] = 0;
+#define PROBE(i) do { if (g == 12) probe[i] = (unsigned)clock(); } while (0)
+#else
+#define PROBE(i)
+#endif
+        for (int t = t_begin; t < t_end && ok; ++t) {
+            int row0, rows;
+            locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
+            TRACE(tr, 36);
+            float gs = 1.0f;                          // Eq. 1's gate of this thread's row (fused forward; the
+                                                      // staged call's rows arrive weighted), read per chunk
+            for (int c = 0; c < nchunks && ok; ++c, ++g) {
+                if (C::NGRP > 1 && (int)(g % C::NGRP) != grp) continue;               // the other group's chunk
+                const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
+                const uint32_t acc1 = lane_base + b * C::HC + w * WCOLS;               // my accumulator columns
+                const uint32_t hdst = lane_base + C::H_COL0 + b * (C::HC / 2) + w * (WCOLS / 2);
+                TRACE(tr, 30);
+                PROBE(0);
+                ACCT_BEGIN();
+                ok = mbar_wait(bar(B::ACC1_FULL + b), n1 & 1u, abort, kWaitLimitNs);
+                ok = __all_sync(0xffffffffu, ok);
+                ACCT_END(acct_wait_acc1);
+                if (!ok) break;
+                // (the tile's A rows, and with them its ring entry, landed before GEMM-1 could run)
+                if (gather) gs = sh.gate_s[(t - t_begin) % kMetaRing][lg * 32 + lane];
+                TRACE(tr, 31);
+                PROBE(1);
+                tc_fence_after_sync();
+                // this chunk's bias came into shared memory with its weights (same stage, same barrier)
+                const int slot = resident ? c : (int)(g % C::W_STAGES);
+                const uint8_t* sb1 = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_B1 + slot * C::B1_BYTES + w * WCOLS * 2;
+                auto add_bias = [&](uint32_t* cur, int pc) {
+                    if (p.bias1) {
+#pragma unroll
+                        for (int j = 0; j < C::PIECE; j += 8) {
+                            float bb[8];
+                            unpack16<bf16>(*reinterpret_cast<const uint4*>(sb1 + (pc * C::PIECE + j) * 2), bb);   // warp-wide broadcast
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) cur[j + i] = __float_as_uint(fmaf(__uint_as_float(cur[j + i]), gs, bb[i]));
+                        }
+                    } else if (gather) {
+#pragma unroll
+                        for (int i = 0; i < C::PIECE; ++i) cur[i] = __float_as_uint(__uint_as_float(cur[i]) * gs);
+                    }
+                };
+                if constexpr (C::PACKED_ACT) {
+                    // Experts.  The whole accumulator chunk is brought into registers as packed bf16
+                    // (SUB pieces at a time) and handed back at once, so that GEMM-1 of this group's
+                    // next chunk runs under this chunk's activation.  Then piece by piece: the argument
+                    // and tanh of piece pc, and behind them the tail and the store of piece pc - 1,
+                    // whose tanh results have arrived by then.
+                    __nv_bfloat162 z[C::NPIECE][C::PIECE / 2];
+                    const __nv_bfloat16 gs_hi = __float2bfloat16_rn(gs);
+                    const __nv_bfloat162 gate_hi = __bfloat162bfloat162(gs_hi);
+                    const __nv_bfloat162 gate_lo = __float2bfloat162_rn(gs - __bfloat162float(gs_hi));
+#pragma unroll
+                    for (int s0 = 0; s0 < C::NPIECE; s0 += C::SUB) {
+                        uint32_t v[C::SUB][C::PIECE];
+#pragma unroll
+                        for (int i = 0; i < C::SUB; ++i) tmem_ld_x16(acc1 + (s0 + i) * C::PIECE, v[i]);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < C::SUB; ++i)
+                            convert_piece_bf16x2(v[i], gate_hi, gate_lo, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
+                                                 p.bias1 != nullptr, z[s0 + i]);
+                    }
+                    PROBE(3);
+                    TRACE(tr, 32);
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
+                    __nv_bfloat162 th[2][C::PIECE / 2];
+#pragma unroll
+                    for (int pc = 0; pc <= C::NPIECE; ++pc) {
+                        if (pc < C::NPIECE) activate_pre_bf16x2<C::ACT>(z[pc], th[pc & 1]);
+                        if (pc == 0) {
+                            TRACE(tr, 33);
+                            // GEMM-2 of two chunks ago must be done with this hidden buffer
+                            ACCT_BEGIN();
+                            ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
+                            ok = __all_sync(0xffffffffu, ok);
+                            ACCT_END(acct_wait_hempty);
+                            if (!ok) break;
+                            TRACE(tr, 34);
+                        } else {
+                            uint32_t hi[C::PIECE / 2];
+                            activate_post_bf16x2<C::ACT>(z[pc - 1], th[(pc - 1) & 1], hi);
+                            tmem_st_x8(hdst + (pc - 1) * (C::PIECE / 2), hi);
+                        }
+                    }
+                    PROBE(12);
+                } else {
+                    uint32_t v[2][C::PIECE];
+                    tmem_ld_x16(acc1, v[0]);
+#pragma unroll
+                    for (int pc = 0; pc < C::NPIECE; ++pc) {
+                        uint32_t* cur = v[pc & 1];
+                        tmem_ld_wait();
+                        if (pc + 1 < C::NPIECE) tmem_ld_x16(acc1 + (pc + 1) * C::PIECE, v[(pc + 1) & 1]);   // overlaps the math below
+                        add_bias(cur, pc);
+                        uint32_t hi[C::PIECE / 2], lo[C::PIECE / 2];
+                        relu_split_piece(cur, hi, lo);
+                        tmem_st_x8(acc1 + pc * (C::PIECE / 2), hi);     // over columns this thread has already read
+                        tmem_st_x8(hdst + pc * (C::PIECE / 2), lo);
+                    }
+                }
+                if (!ok) break;
+                ACCT_BEGIN();
+                tmem_st_wait();
+                TRACE(tr, 37);
+                ACCT_END(acct_stwait);
+                PROBE(13);
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B::H_FULL + b));
+                PROBE(14);
+                TRACE(tr, 35);
+            }
+        }
+#ifdef SLICEMOE_TC_PROBE
+        if (lane == 0 && p.status != nullptr && blockIdx.x == 0 && !C::ROUTER) {
+            unsigned* out = reinterpret_cast<unsigned*>(p.status + 16) + (warp - 4) * 16;
+            for (int i = 0; i < 16; ++i) out[i] = probe[i];
+        }
+#endif
+#ifdef SLICEMOE_TC_ACCT
+        if (lane == 0 && p.status != nullptr && blockIdx.x == 0) {
+            long long* out = reinterpret_cast<long long*>(p.status + 16) + (warp - 4) * 4;   // status area: int32[64] -> spill past it
+            out[0] = clock64() - acct_t0; out[1] = acct_wait_acc1; out[2] = acct_wait_hempty; out[3] = acct_stwait;
+        }
+#endif
+    } else if (warp >= C::OUT_WARP0) {
+        // ================= output warpgroup ==================================================
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
+        bool ok = true;
+        int e = 0;
+        TRACE_DECL(tr, (lg == 0 && lane == 0) ? 5 : 7);
+        // Fused forward: this thread's row of a tile is pair perm[row0 + row] = (n, j); its output is
+        // added into row n of Y.
+        for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+            int row0, rows;
+            locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
+            const int buf = ta % C::ACC2_BUFS;
+            TRACE(tr, 40);
+            ok = mbar_wait(bar(B::ACC2_FULL + buf), (uint32_t)(ta / C::ACC2_BUFS) & 1u, abort, kWaitLimitNs);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            TRACE(tr, 41);
+            tc_fence_after_sync();
+            const int pair_cur = gather ? sh.pair_s[ta % kMetaRing][row] : 0;
+            const uint32_t acc2 = tmem_lane + C::ACC2_COL0 + buf * C::N2;
+            if constexpr (C::ROUTER) {
+                constexpr int E = C::N2;
+                uint32_t v[E];
+#pragma unroll
+                for (int q = 0; q < E / 16; ++q) tmem_ld_x16(acc2 + q * 16, v + q * 16);
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
+                TRACE(tr, 42);
+                if (row >= rows) continue;
+                float gl[E];
+#pragma unroll
+                for (int i = 0; i < E; ++i)
+                    gl[i] = __uint_as_float(v[i]) + (p.bias2 ? __bfloat162float(__ldg(p.bias2 + i)) : 0.0f);
+                const int n = row0 + row;
+                // top-k by repeated arg-max over the logits; ties go to the lower id
+                unsigned long long taken = 0ull;
+                float m = 0.0f;
+                int sel[8];
+                float gsel[8];
+                for (int j = 0; j < p.k; ++j) {
+                    int best = -1;
+                    float bv = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < E; ++i) {
+                        const bool free_i = !((taken >> i) & 1ull);
+                        if (free_i && (best < 0 || gl[i] > bv)) { best = i; bv = gl[i]; }
+                    }
+                    taken |= 1ull << best;
+                    sel[j] = best;
+                    gsel[j] = bv;
+                    if (j == 0) m = bv;
+                }
+                float sum = 0.0f;
+#pragma unroll
+                for (int i = 0; i < E; ++i) sum += __expf(gl[i] - m);
+                const float inv = 1.0f / sum;
+                for (int j = 0; j < p.k; ++j) {
+                    p.topk_idx[(size_t)n * p.k + j] = sel[j];
+                    p.topk_p[(size_t)n * p.k + j] = __expf(gsel[j] - m) * inv;
+                    atomicAdd(&sh.hist[sel[j]], 1);
+                }
+                if (p.probs) {
+                    float4* dst = reinterpret_cast<float4*>(p.probs + (size_t)n * E);
+#pragma unroll
+                    for (int i = 0; i < E; i += 4)
+                        dst[i / 4] = make_float4(__expf(gl[i] - m) * inv, __expf(gl[i + 1] - m) * inv,
+                                                 __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
+                }
+            } else {
+                // 64 output columns at a time: accumulator -> registers -> bias -> bf16 -> global
+                constexpr int OB = 64;
+                const bool scatter = gather && p.scatter_out != nullptr;
+                const bool live = row < rows;
+                bf16* dst = nullptr;
+                if (live) dst = scatter ? p.scatter_out + (size_t)(pair_cur / p.gather_k) * C::N2
+                                        : p.yperm + (size_t)(row0 + row) * C::N2;
+#pragma unroll 1
+                for (int cb = 0; cb < C::N2; cb += OB) {
+                    uint32_t v[OB];
+#pragma unroll
+                    for (int q = 0; q < OB / 16; ++q) tmem_ld_x16(acc2 + cb + q * 16, v + q * 16);
+                    tmem_ld_wait();
+                    if (cb + OB >= C::N2) {
+                        // the accumulator is in registers: GEMM-2 of a later tile may overwrite it
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
+                        TRACE(tr, 42);
+                    }
+#ifdef SLICEMOE_DEV_NO_OUT    // development: time the pipeline without the output stores
+                    if (true) continue;
+#endif
+                    if (!live) continue;
+#pragma unroll
+                    for (int q = 0; q < OB / 8; ++q) {
+                        float bb[8];
+                        if (p.bias2) {
+                            unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.bias2 + (size_t)e * C::N2 + cb + q * 8)), bb);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) bb[i] = 0.0f;
+                        }
+                        uint32_t o[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            o[i] = pack_bf16x2(fmaf(__uint_as_float(v[q * 8 + 2 * i]), kOutScale<C::ACT>, bb[2 * i]),
+                                               fmaf(__uint_as_float(v[q * 8 + 2 * i + 1]), kOutScale<C::ACT>, bb[2 * i + 1]));
+                        if (scatter) red_add_bf16x8(dst + cb + q * 8, o[0], o[1], o[2], o[3]);   // sum over the row's k experts
+                        else *reinterpret_cast<uint4*>(dst + cb + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+                TRACE(tr, 43);
+            }
+        }
+    }
+
+    // ---- teardown -------------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh.abort_flag) atomicExch(p.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
+    if constexpr (C::ROUTER) {
+        // per-CTA histogram -> global counts (Section 3.2's per-expert counts)
+        for (int i = threadIdx.x; i < C::N2; i += C::THREADS) {
+            if (p.assigned && sh.hist[i]) atomicAdd(&p.assigned[i], sh.hist[i]);
+            if (p.cta_hist) p.cta_hist[(size_t)blockIdx.x * C::N2 + i] = sh.hist[i];
+        }
+    }
+#ifdef SLICEMOE_TC_TRACE
+#ifdef SLICEMOE_TRACE_EXPERTS_ONLY
+    constexpr bool dump_trace = !C::ROUTER;
+#else
+    constexpr bool dump_trace = true;
+#endif
+    if (dump_trace && blockIdx.x == 0 && g_trace_buf) {
+        const uint2* src = reinterpret_cast<const uint2*>(smem_raw + 200 * 1024);
+        for (int i = threadIdx.x; i < 6 * kTraceSmemEvents; i += C::THREADS) {
+            const int slot = i / kTraceSmemEvents, n = i % kTraceSmemEvents;
+            g_trace_buf[((size_t)slot * kTraceEvents + n) * 2] = src[i].x;
+            g_trace_buf[((size_t)slot * kTraceEvents + n) * 2 + 1] = src[i].y;
+        }
+    }
+#endif
+    tc_fence_before_sync();
+    __syncthreads();          // nothing of this pass is in flight any more: barriers and TMEM may be reused
+    tc_fence_after_sync();
+}
+
+// ---- host side --------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+// bf16 matrix [rows, cols] row-major; box = 64 columns (128 bytes) x box_rows, 128-byte swizzle.
+int make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SLICEMOE_ERR_CUDA;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SLICEMOE_OK : SLICEMOE_ERR_CUDA;
+}
+
+int sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            v = 148;
+        return v;
+    }();
+    return n;
+}
+
+#ifdef SLICEMOE_TC_TRACE
+template <class C> constexpr int kSmemLaunch = 200 * 1024 + 6 * kTraceSmemEvents * 8;   // trace area after 200 KiB
+#else
+template <class C> constexpr int kSmemLaunch = C::SMEM_ALLOC;
+#endif
+
+}  // namespace
+}  // namespace slicemoe

@@ -167,6 +167,49 @@ def test_profiled_forward_records_stage_times():
     assert torch.equal(h_out, gpu.forward()[0])
 
 
+@pytest.mark.parametrize("name", ["bf16_lm", "bf16_skew_cap", "bf16_decode", "bf16_single_row", "bf16_k3", "f32_cfg0"])
+def test_forward_launch_count_and_status(name):
+    """Supported bf16 shapes with k <= 2 run the whole forward as one launch; the others one
+    launch per step.  Either way the status word stays clear and repeated calls on two
+    workspaces give the same bits."""
+    import torch
+    lc = SMALL[name]
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    gpu2 = pu.GpuLayer(lc, h, w)
+    first = gpu.forward()
+    before = binding.slicemoe_launch_count()
+    again = gpu.forward()
+    launches = binding.slicemoe_launch_count() - before
+    other = gpu2.forward()
+    torch.cuda.synchronize()
+    one_launch = lc.dtype == "bf16" and lc.k <= 2 and lc.ds in (64, 128, 256) and lc.E in (16, 32, 64)
+    assert launches == 1 if one_launch else launches >= 3
+    assert gpu.status() == 0 and gpu2.status() == 0
+    for a, b, c in zip(first, again, other):
+        assert torch.equal(a, b) and torch.equal(a, c)
+
+
+def test_forward_back_to_back_on_two_streams():
+    """Launches of the single-kernel forward queued on two streams share the device's grid-barrier
+    words; each must still see its own barriers complete."""
+    import torch
+    lc = SMALL["bf16_lm"]
+    h, w = inputs(lc)
+    a, b = pu.GpuLayer(lc, h, w), pu.GpuLayer(lc, h, w)
+    want = a.forward()[0].clone()
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    outs = []
+    for i in range(6):
+        with torch.cuda.stream(s1 if i % 2 == 0 else s2):
+            outs.append((a if i % 2 == 0 else b).forward()[0].clone())
+    torch.cuda.synchronize()
+    assert a.status() == 0 and b.status() == 0
+    for o in outs:
+        assert torch.equal(o, want)
+
+
 def test_dispatch_drops_out_of_range_ids():
     import torch
     lc = SMALL["bf16_lm"]

@@ -28,12 +28,13 @@ if ROOT not in sys.path:
 L2_BYTES = 126e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-# profiles/forward_kernels_cfg1_cfg2.md (taken on cfg2, whose tokens exceed L2).  The other workloads of
-# the same slice width scale it by the rows one launch processes (traffic is proportional to rows:
-# every row is read once per chosen expert and written once).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised in
+# profiles/fused_forward_cfg1_cfg2.md and profiles/three_launch_forward_cfg1_cfg2.md (taken on cfg2,
+# whose tokens exceed L2).  The other workloads of the same slice width scale it by the rows one launch
+# processes (traffic is proportional to rows: every row is read once per chosen expert and written once).
 NCU_TRAFFIC_CFG2 = {"route": 134.328064e6 + 142.558720e6, "dispatch": 17.735168e6 + 0.924928e6,
-                    "expert_ffn": 451.720704e6 + 175.928320e6}
+                    "expert_ffn": 451.720704e6 + 175.928320e6,
+                    "fused_forward": 578.491648e6 + 350.857216e6}
 NCU_TRAFFIC_ROWS_CFG2 = 65536 * 16
 
 

@@ -264,6 +264,10 @@ def run_ours(args, lc):
         raise RuntimeError(f"device status {sm.slicemoe_last_status(ws)} after warm-up")
     kept_rows = int(kept.sum().item())
     touched = int((kept > 0).sum().item())
+    # routing balance of this batch (Eq. 2 with alpha = 0.1, Section 4's ELE), computed on the device
+    stats = torch.empty(2, dtype=torch.float64, device="cuda")
+    sm.slicemoe_load_stats(assigned, 0.1, stats)
+    l_cap, ele = (float(x) for x in stats.cpu())
 
     # ---- timed region 1: device-resident inputs -------------------------------------------
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -337,6 +341,7 @@ def run_ours(args, lc):
             "ms_per_step": 1e3 * t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": lc.dtype, "data": "synthetic", "config": workload_config(lc, sets),
             "routed_slices_per_s": world * lc.R / t_step,
+            "routing_stats": {"ele": ele, "l_cap_alpha_0.1": l_cap},
             "e2e": {"value": world * lc.T * args.steps / t_e2e, "unit": "tokens/s",
                     "h2d_bytes_per_step": lc.T * lc.d * b, "d2h_bytes_per_step": lc.T * lc.d * b},
             "gpu_launches": int(launches),

@@ -181,6 +181,18 @@ int slicemoe_combine(const slicemoe_config *cfg, const void *yperm, const int32_
                      void *h_out, void *stream);
 
 /*
+ * Routing statistics from per-expert counts (such as `assigned` of the forward):
+ *   out[0] = L_cap of Eq. 2 = alpha * (std(counts) / mean(counts))^2, with the
+ *            population standard deviation (divide by E) -- the paper does not
+ *            say which; alpha is the paper's coefficient (0.01 ... 0.2)
+ *   out[1] = ELE of Section 4 (Metrics) = -sum_e load_e log load_e / log E,
+ *            load_e = counts_e / sum(counts), 0 log 0 = 0; E = 1 gives 1
+ * Both are 0 when nothing was routed.  counts: DEVICE int32 [E]; out: DEVICE
+ * double [2], 8-byte aligned.  fp64, deterministic; asynchronous on `stream`.
+ */
+int slicemoe_load_stats(const int32_t *counts, int32_t E, double alpha, double *out, void *stream);
+
+/*
  * The whole layer forward, h [T, d] -> h_out [T, d], equal to
  * route -> dispatch -> expert_ffn -> combine up to rounding, and bit-equal on
  * topk_idx / assigned / kept.  h_out must not overlap h.

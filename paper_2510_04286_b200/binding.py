@@ -21,7 +21,7 @@ STAGES = ("route", "dispatch", "expert_ffn", "combine")
 EXPORTS = (
     "slicemoe_workspace_bytes", "slicemoe_route", "slicemoe_dispatch", "slicemoe_dispatch_static",
     "slicemoe_expert_ffn",
-    "slicemoe_combine", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
+    "slicemoe_combine", "slicemoe_load_stats", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
     "slicemoe_event_create", "slicemoe_event_destroy", "slicemoe_event_elapsed_ms",
     "slicemoe_last_status", "slicemoe_launch_count", "slicemoe_last_cuda_error",
     "slicemoe_status_string",
@@ -184,6 +184,12 @@ def slicemoe_combine(cfg, yperm, dest, h_out, stream=None):
     c = cfg.c()
     _check(_lib().slicemoe_combine(ctypes.byref(c), _ptr(yperm), _ptr(dest), _ptr(h_out), _stream(stream)),
            "slicemoe_combine")
+
+
+def slicemoe_load_stats(counts, alpha, out, stream=None):
+    """counts: cuda int32 [E]; out: cuda float64 [2] <- (L_cap of Eq. 2, ELE of Section 4)."""
+    _check(_lib().slicemoe_load_stats(_ptr(counts), ctypes.c_int32(counts.numel()), ctypes.c_double(alpha),
+                                      _ptr(out), _stream(stream)), "slicemoe_load_stats")
 
 
 def slicemoe_forward(cfg, w, h, h_out, ws, assigned=None, kept=None, topk_idx=None, topk_p=None,

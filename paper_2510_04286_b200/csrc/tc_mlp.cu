@@ -89,7 +89,7 @@ bool tc_route_supported(const Dims& D) {
 bool tc_ffn_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
     if (D.ds != 64 && D.ds != 128 && D.ds != 256) return false;
-    const int hc = D.ds == 64 ? 128 : 64;
+    const int hc = 64;
     return D.F % hc == 0 && D.F >= 2 * hc && D.F <= kMaxHid;
 }
 

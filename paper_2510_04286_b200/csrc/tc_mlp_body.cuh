@@ -113,21 +113,26 @@ template <int K1_, int N2_, bool ROUTER_, int ACT_>
 struct TcCfg {
     static constexpr int K1 = K1_, N2 = N2_, ACT = ACT_;
     static constexpr bool ROUTER = ROUTER_;
-    static constexpr int HC = (K1 == 64) ? 128 : 64;           // hidden units per chunk
+    // 64-wide expert rows: four narrow chunks in flight, one warpgroup each (see NGRP below)
+    static constexpr bool FOUR_GROUPS = (K1 == 64) && !ROUTER_;
+    static constexpr int HC = (K1 == 64 && ROUTER_) ? 128 : 64;   // hidden units per chunk
     // row-tile buffers: three where they fit (the fused forward gathers two tiles ahead); with
     // 256-wide rows (64 KB per tile) the router gets two and the experts, whose weight stages are
     // larger, one
     static constexpr int A_BUFS = (K1 <= 128) ? 3 : (ROUTER_ ? 2 : 1);
-    static constexpr int W_STAGES = (K1 == 128) ? 3 : 2;
+    static constexpr int W_STAGES = (K1 == 128) ? 3 : (FOUR_GROUPS ? 4 : 2);
     // Activation warps: NGRP groups that take the hidden chunks in turn (chunk g goes to group
     // g mod NGRP), each group GWG warpgroups that split the chunk's columns.  With two groups one
     // group's accumulator loads, tails and stores run while the other group's tanh work occupies
     // the tanh unit.  256-wide rows get one group: their wide output epilogue needs the larger
     // register budget of a 512-thread CTA.
-    static constexpr int NGRP = (K1 == 256) ? 1 : 2;
-    static constexpr int GWG = 2;
+    // 64-wide expert rows run four groups of one warpgroup on four 64-column chunks instead: the
+    // warps of a sub-partition are then in four different phases, and a warp in its tanh phase is
+    // more often there to use the unit while the others load, convert and store.
+    static constexpr int NGRP = (K1 == 256) ? 1 : (FOUR_GROUPS ? 4 : 2);
+    static constexpr int GWG = FOUR_GROUPS ? 1 : 2;
     static constexpr int NWG = NGRP * GWG;
-    static constexpr int NBUF = 2;                              // GEMM-1 accumulator / hidden buffers
+    static constexpr int NBUF = FOUR_GROUPS ? 4 : 2;            // GEMM-1 accumulator / hidden buffers
     static constexpr int GRP_WARPS = GWG * 4;                   // warps that work on one chunk
     static constexpr int THREADS = 128 + NWG * 128 + 128;
     static constexpr int OUT_WARP0 = 4 + NWG * 4;               // first warp of the output warpgroup
@@ -672,7 +677,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         bool ok = true;
         int e = 0;
         uint32_t g = 0;
-        TRACE_DECL(tr, (lg == 0 && lane == 0 && w == 0) ? 2 + grp : 7);
+        TRACE_DECL(tr, (lg == 0 && lane == 0 && w == 0 && grp < 2) ? 2 + grp : 7);
 #ifdef SLICEMOE_TC_ACCT   // development: where do the activation warps spend their cycles?
         long long acct_wait_acc1 = 0, acct_wait_hempty = 0, acct_stwait = 0, acct_t0 = clock64(), acct_mark;
 #define ACCT_BEGIN() acct_mark = clock64()

@@ -248,6 +248,9 @@ int fused_forward_reset_sync(cudaStream_t st) {
 }
 
 bool fused_forward_supported(const Dims& D) {
+#ifdef SLICEMOE_TC_TRACE   // the timeline tracer needs its own shared-memory area: one launch per stage only
+    return false;
+#endif
     return tc_route_supported(D) && tc_ffn_supported(D) && D.N > 0 && D.k <= 2 && cooperative_launch_available();
 }
 

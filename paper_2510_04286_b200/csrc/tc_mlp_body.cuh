@@ -49,7 +49,13 @@ constexpr int kMaxE = 256;
 // accumulators for the old tile and the output warps, at most two accumulators and one tile of
 // GEMM-1 run-ahead behind, have stored it.
 constexpr int kMetaRing = 8;
-constexpr int kMaxBars = 40;
+constexpr int kMaxBars = 48;
+// Slots of the first-layer bias ring, indexed by the running count of W1 chunk loads.  Slot q is
+// rewritten by load q + kBiasRing, which needs a free W1 slot, i.e. GEMM-1 of load q + kBiasRing -
+// W_STAGES done, i.e. (accumulator hand-back) the activation of the chunks before it, load q's among
+// them, finished; with resident weights a new expert's loads must not touch the previous expert's
+// slots, hence at least two full sets.
+constexpr int kBiasRing = 8;
 
 struct TcParams {
     const int32_t* offsets;   // experts: [E+1] device row ranges; router: nullptr
@@ -81,7 +87,14 @@ struct TcParams {
 // Optional timeline tracing (development builds only: -DSLICEMOE_TC_TRACE).  CTA 0 stamps
 // (event code, SM clock) pairs per role into a caller-provided buffer.
 #ifdef SLICEMOE_TC_TRACE
-constexpr int kTraceSlots = 8, kTraceEvents = 2048, kTraceSmemEvents = 320;
+#ifndef SLICEMOE_TRACE_EVENTS
+#define SLICEMOE_TRACE_EVENTS 320          // per role, in shared memory
+#endif
+#ifndef SLICEMOE_TRACE_OFFSET_KB
+#define SLICEMOE_TRACE_OFFSET_KB 200       // where the trace area starts; must lie past the operand tiles
+#endif
+constexpr int kTraceSlots = 8, kTraceEvents = 2048, kTraceSmemEvents = SLICEMOE_TRACE_EVENTS;
+constexpr int kTraceOffset = SLICEMOE_TRACE_OFFSET_KB * 1024;
 __device__ unsigned long long* g_trace_buf = nullptr;
 // Events go to shared memory (cheap) and are copied out at the end of the kernel.
 struct Tracer {
@@ -90,7 +103,7 @@ struct Tracer {
     __device__ Tracer(int slot) : base(nullptr), n(0) {
         extern __shared__ uint8_t smem_raw[];
         if (blockIdx.x == 0 && g_trace_buf && slot < 6)
-            base = reinterpret_cast<uint2*>(smem_raw + 200 * 1024) + slot * kTraceSmemEvents;
+            base = reinterpret_cast<uint2*>(smem_raw + kTraceOffset) + slot * kTraceSmemEvents;
     }
     __device__ void operator()(int code) {
         if (base && n < kTraceSmemEvents) { base[n] = make_uint2((unsigned)code, (unsigned)clock64()); ++n; }
@@ -167,12 +180,18 @@ struct TcCfg {
     static constexpr int W1C_BYTES = KP1 * W1_PANEL;
     static constexpr int W2_PANEL = N2 * 128;
     static constexpr int W2C_BYTES = KP2 * W2_PANEL;
-    static constexpr int W_STAGE_BYTES = W1C_BYTES + W2C_BYTES;
+    // W1 and W2 chunks live in two rings of W_STAGES slots each with their own barriers: a W1 slot
+    // is handed back as soon as GEMM-1 has read it, so the next chunk's W1 streams in under this
+    // chunk's activation and GEMM-2 instead of after them.
     static constexpr int OFF_A = 0;
     static constexpr int OFF_W = OFF_A + A_BUFS * A_BYTES;
-    static constexpr int B1_BYTES = HC * 2;                     // one chunk of the first layer's bias, per weight stage
-    static constexpr int OFF_B1 = OFF_W + W_STAGES * W_STAGE_BYTES;
-    static constexpr int SMEM_BYTES = OFF_B1 + W_STAGES * B1_BYTES;
+    static constexpr int OFF_W2 = OFF_W + W_STAGES * W1C_BYTES;
+    // The first layer's bias chunk arrives with W1 but is read after GEMM-1, by the activation
+    // warps, so it has a ring of its own, deep enough that a slot is rewritten only by a W1 load
+    // that cannot be issued before the old chunk's activation has finished (see kBiasRing).
+    static constexpr int B1_BYTES = HC * 2;
+    static constexpr int OFF_B1 = OFF_W2 + W_STAGES * W2C_BYTES;
+    static constexpr int SMEM_BYTES = OFF_B1 + kBiasRing * B1_BYTES;
     // at least 120 KiB is requested so that two CTAs never share an SM (each allocates most of TMEM)
     static constexpr int SMEM_ALLOC = (SMEM_BYTES + 1024 > 120 * 1024) ? SMEM_BYTES + 1024 : 120 * 1024;
     static constexpr int PIECE = 16;                            // accumulator columns per piece
@@ -180,7 +199,8 @@ struct TcCfg {
     static constexpr int SUB = (NPIECE > 2) ? 2 : NPIECE;       // pieces held in registers at once (experts)
     static_assert(NBUF % NGRP == 0 && NPIECE % SUB == 0, "chunk-to-group and piece-to-batch maps");
     static_assert(NPIECE >= 1, "hidden chunk too narrow for the activation warpgroups");
-    static_assert(W_STAGE_BYTES % 1024 == 0 && W1C_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+    static_assert(W2C_BYTES % 1024 == 0 && W1C_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+    static_assert(kBiasRing >= 2 * W_STAGES, "bias ring");
     static_assert(N2 % 16 == 0 && N2 >= 16 && N2 <= 256, "MMA N");
     static_assert(SMEM_ALLOC <= 232448, "shared memory budget");
     static_assert(ACC2_COL0 + ACC2_BUFS * N2 <= 512, "TMEM budget");
@@ -191,9 +211,11 @@ template <class C>
 struct Bars {
     static constexpr int A_FULL = 0;
     static constexpr int A_EMPTY = A_FULL + C::A_BUFS;
-    static constexpr int W_FULL = A_EMPTY + C::A_BUFS;
-    static constexpr int W_EMPTY = W_FULL + C::W_STAGES;
-    static constexpr int ACC1_FULL = W_EMPTY + C::W_STAGES;   // GEMM-1 done (MMA -> activation)
+    static constexpr int W1_FULL = A_EMPTY + C::A_BUFS;
+    static constexpr int W1_EMPTY = W1_FULL + C::W_STAGES;    // GEMM-1 has read the W1 slot
+    static constexpr int W2_FULL = W1_EMPTY + C::W_STAGES;
+    static constexpr int W2_EMPTY = W2_FULL + C::W_STAGES;    // GEMM-2 has read the W2 slot
+    static constexpr int ACC1_FULL = W2_EMPTY + C::W_STAGES;  // GEMM-1 done (MMA -> activation)
     // accumulator may be overwritten: experts, all activation warps have read it;
     // router (hidden chunk lives in it), GEMM-2 has consumed it
     static constexpr int ACC1_EMPTY = ACC1_FULL + C::NBUF;
@@ -352,7 +374,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 
 #ifdef SLICEMOE_TC_TRACE
     for (int i = threadIdx.x; i < 6 * kTraceSmemEvents * 2; i += C::THREADS)
-        reinterpret_cast<uint32_t*>(smem_raw + 200 * 1024)[i] = 0;
+        reinterpret_cast<uint32_t*>(smem_raw + kTraceOffset)[i] = 0;
 #endif
     // ---- set-up ---------------------------------------------------------------------------
     if (threadIdx.x == 0) {
@@ -361,7 +383,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #endif
         sh.abort_flag = 0;
         for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 32 : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
-        for (int i = 0; i < C::W_STAGES; ++i) { mbar_init(bar(B::W_FULL + i), 1); mbar_init(bar(B::W_EMPTY + i), 1); }
+        for (int i = 0; i < C::W_STAGES; ++i) {
+            mbar_init(bar(B::W1_FULL + i), 1); mbar_init(bar(B::W1_EMPTY + i), 1);
+            mbar_init(bar(B::W2_FULL + i), 1); mbar_init(bar(B::W2_EMPTY + i), 1);
+        }
         for (int i = 0; i < C::NBUF; ++i) {
             mbar_init(bar(B::ACC1_FULL + i), 1);
             mbar_init(bar(B::ACC1_EMPTY + i), C::ROUTER ? 1 : C::GRP_WARPS);
@@ -406,10 +431,17 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 
     if (warp == 0) {
         // ================= TMA producer =====================================================
+        // One thread, per tile: the row tile (unless rows are gathered), then per chunk W1 (with its
+        // bias) and W2, each into its own ring behind its own "slot free" barrier.  All waits park
+        // the thread (no polling).  W1 of chunk g waits for GEMM-1 of the chunk that had the slot;
+        // W2 of chunk g for GEMM-2 of the chunk that had its slot, which may come a little later
+        // than the next W1 slot frees up -- a short delay, against a full weight round trip on the
+        // critical path when both halves shared one slot.
         if (lane == 0 && t_begin < t_end) {
             int e = 0, prev_e = -1;
             uint32_t g = 0, reloads = 0;             // chunks seen; tiles that (re)loaded weights
-            uint32_t last_a_bar = 0, last_a_par = 0, last_w_bar = 0, last_w_par = 0;
+            uint32_t wq = 0;                         // W1 chunk loads issued (bias ring position)
+            uint32_t last_bar[3] = {0, 0, 0}, last_par[3] = {0, 0, 0};
             bool ok = true;
             TRACE_DECL(tr, 0);
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
@@ -425,8 +457,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #pragma unroll
                     for (int kp = 0; kp < C::KP1; ++kp)
                         tma_load_2d(sA + ab * C::A_BYTES + kp * C::A_PANEL, &tmA, kp * 64, row0, bar(B::A_FULL + ab));
-                    last_a_bar = bar(B::A_FULL + ab);
-                    last_a_par = an & 1u;
+                    last_bar[0] = bar(B::A_FULL + ab);
+                    last_par[0] = an & 1u;
                 }
                 const bool reload = !resident || (e != prev_e);
                 prev_e = e;
@@ -436,30 +468,35 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     // streamed weights: slots in ring order
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
                     const uint32_t n = resident ? reloads : g / C::W_STAGES;
-                    if (!mbar_wait(bar(B::W_EMPTY + slot), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
-                    mbar_arrive_expect_tx(bar(B::W_FULL + slot), C::W_STAGE_BYTES + (p.bias1 ? C::B1_BYTES : 0));
-                    const uint32_t dst = sW + slot * C::W_STAGE_BYTES;
+                    if (!mbar_wait(bar(B::W1_EMPTY + slot), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(B::W1_FULL + slot), C::W1C_BYTES + (p.bias1 ? C::B1_BYTES : 0));
                     if (p.bias1)
-                        bulk_load(smem_base + C::OFF_B1 + slot * C::B1_BYTES, p.bias1 + (size_t)e * p.HID + c * C::HC,
-                                  C::B1_BYTES, bar(B::W_FULL + slot));
+                        bulk_load(smem_base + C::OFF_B1 + (wq % kBiasRing) * C::B1_BYTES,
+                                  p.bias1 + (size_t)e * p.HID + c * C::HC, C::B1_BYTES, bar(B::W1_FULL + slot));
 #pragma unroll
                     for (int kp = 0; kp < C::KP1; ++kp)
-                        tma_load_2d(dst + kp * C::W1_PANEL, &tmW1, kp * 64, e * p.HID + c * C::HC, bar(B::W_FULL + slot));
+                        tma_load_2d(sW + slot * C::W1C_BYTES + kp * C::W1_PANEL, &tmW1, kp * 64, e * p.HID + c * C::HC,
+                                    bar(B::W1_FULL + slot));
+                    last_bar[1] = bar(B::W1_FULL + slot);
+                    last_par[1] = n & 1u;
+                    ++wq;
+                    if (!mbar_wait(bar(B::W2_EMPTY + slot), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(B::W2_FULL + slot), C::W2C_BYTES);
 #pragma unroll
                     for (int kp = 0; kp < C::KP2; ++kp)
-                        tma_load_2d(dst + C::W1C_BYTES + kp * C::W2_PANEL, &tmW2, c * C::HC + kp * 64, e * C::N2,
-                                    bar(B::W_FULL + slot));
-                    last_w_bar = bar(B::W_FULL + slot);
-                    last_w_par = n & 1u;
+                        tma_load_2d(smem_base + C::OFF_W2 + slot * C::W2C_BYTES + kp * C::W2_PANEL, &tmW2,
+                                    c * C::HC + kp * 64, e * C::N2, bar(B::W2_FULL + slot));
+                    last_bar[2] = bar(B::W2_FULL + slot);
+                    last_par[2] = n & 1u;
                 }
                 ++reloads;
             }
             if (!ok || *abort) {
                 // leaving early: let this thread's last copies land first (bounded; the copies
-                // complete on their own, earlier ones were issued before these)
+                // complete on their own, earlier ones of a stream were issued before its last)
                 volatile int never = 0;
-                if (last_a_bar) mbar_wait(last_a_bar, last_a_par, &never, 10000000ull);
-                if (last_w_bar) mbar_wait(last_w_bar, last_w_par, &never, 10000000ull);
+                for (int i = 0; i < 3; ++i)
+                    if (last_bar[i]) mbar_wait(last_bar[i], last_par[i], &never, 10000000ull);
             }
         }
     } else if (warp == 1) {
@@ -485,14 +522,14 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
                     if (reload) {
                         const uint32_t n = resident ? reloads : g / C::W_STAGES;
-                        if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                        if (!mbar_wait(bar(B::W1_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
                     }
                     const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
                     TRACE(tr, 12);
                     if (!mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
                     TRACE(tr, 13);
                     tc_fence_after_sync();
-                    const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W_STAGE_BYTES) >> 4);
+                    const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W1C_BYTES) >> 4);
                     const uint32_t d = tmem_base + b * C::HC;
                     mma_ss<0>(d, a0, w0, idesc1);
 #ifndef SLICEMOE_DEV_G1_ONE   // development: time the pipeline with a single GEMM-1 MMA per chunk
@@ -502,6 +539,9 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                                   w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
 #endif
                     mma_commit(bar(B::ACC1_FULL + b));
+                    // streamed weights: the W1 slot is free as soon as these MMAs have read it
+                    // (resident weights are handed back by the GEMM-2 thread at an expert change)
+                    if (!resident) mma_commit(bar(B::W1_EMPTY + slot));
                     if (c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
                     TRACE(tr, 14);
                 }
@@ -518,7 +558,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         // ================= GEMM-2 issue ======================================================
         if (lane == 0 && t_begin < t_end) {
             constexpr uint32_t idesc2 = make_idesc(128, C::N2, kFmtBF16, kFmtBF16);
-            const uint32_t dW = desc_lo_sw128(sW);
+            const uint32_t dW = desc_lo_sw128(smem_base + C::OFF_W2);
             bool ok = true;
             TRACE_DECL(tr, 4);
             int e = 0, prev_e = -1;
@@ -539,10 +579,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 for (int c = 0; c < nchunks; ++c, ++g) {
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
                     if (reload) {
-                        // (already observed by the GEMM-1 thread; waited here too so that this
-                        // thread's reads of the weight tile are ordered after the copy)
                         const uint32_t n = resident ? reloads : g / C::W_STAGES;
-                        if (!mbar_wait(bar(B::W_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                        if (!mbar_wait(bar(B::W2_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
                     }
                     const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
                     TRACE(tr, 20);
@@ -551,7 +589,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     if (c == 0 && !mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(ta / C::ACC2_BUFS) & 1u) ^ 1u,
                                              abort, kWaitLimitNs)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t w0 = dW + ((slot * C::W_STAGE_BYTES + C::W1C_BYTES) >> 4);
+                    const uint32_t w0 = dW + ((slot * C::W2C_BYTES) >> 4);
                     const uint32_t d = tmem_base + C::ACC2_COL0 + buf * C::N2;
                     const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: chunk; router: lo half
                     const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi half, two runs
@@ -572,7 +610,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         }
                     }
                     mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
-                    if (release) mma_commit(bar(B::W_EMPTY + slot));
+                    if (release) {
+                        mma_commit(bar(B::W2_EMPTY + slot));
+                        if (resident) mma_commit(bar(B::W1_EMPTY + slot));   // GEMM-1 of this chunk finished before its GEMM-2 began
+                    }
                     if (c == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
                     TRACE(tr, 22);
                 }
@@ -693,9 +734,16 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #else
 #define PROBE(i)
 #endif
+        int prev_e = -1;
+        uint32_t q_tile = 0, q_next = 0;              // bias ring: W1 load count of this tile's chunk 0 / after it
         for (int t = t_begin; t < t_end && ok; ++t) {
             int row0, rows;
             locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
+            if (!resident || e != prev_e) {           // this tile's weights (and biases) were loaded for it
+                q_tile = q_next;
+                q_next += nchunks;
+            }
+            prev_e = e;
             TRACE(tr, 36);
             float gs = 1.0f;                          // Eq. 1's gate of this thread's row (fused forward; the
                                                       // staged call's rows arrive weighted), read per chunk
@@ -716,9 +764,9 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 TRACE(tr, 31);
                 PROBE(1);
                 tc_fence_after_sync();
-                // this chunk's bias came into shared memory with its weights (same stage, same barrier)
-                const int slot = resident ? c : (int)(g % C::W_STAGES);
-                const uint8_t* sb1 = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_B1 + slot * C::B1_BYTES + w * WCOLS * 2;
+                // this chunk's bias came into shared memory with its W1 (same barrier, own ring)
+                const int bslot = (int)((q_tile + c) % kBiasRing);
+                const uint8_t* sb1 = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_B1 + bslot * C::B1_BYTES + w * WCOLS * 2;
                 auto add_bias = [&](uint32_t* cur, int pc) {
                     if (p.bias1) {
 #pragma unroll
@@ -957,7 +1005,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     constexpr bool dump_trace = true;
 #endif
     if (dump_trace && blockIdx.x == 0 && g_trace_buf) {
-        const uint2* src = reinterpret_cast<const uint2*>(smem_raw + 200 * 1024);
+        const uint2* src = reinterpret_cast<const uint2*>(smem_raw + kTraceOffset);
         for (int i = threadIdx.x; i < 6 * kTraceSmemEvents; i += C::THREADS) {
             const int slot = i / kTraceSmemEvents, n = i % kTraceSmemEvents;
             g_trace_buf[((size_t)slot * kTraceEvents + n) * 2] = src[i].x;
@@ -1014,7 +1062,7 @@ int sm_count() {
 }
 
 #ifdef SLICEMOE_TC_TRACE
-template <class C> constexpr int kSmemLaunch = 200 * 1024 + 6 * kTraceSmemEvents * 8;   // trace area after 200 KiB
+template <class C> constexpr int kSmemLaunch = kTraceOffset + 6 * kTraceSmemEvents * 8;   // trace area behind the operand tiles
 #else
 template <class C> constexpr int kSmemLaunch = C::SMEM_ALLOC;
 #endif

@@ -216,6 +216,12 @@ int slicemoe_forward(const slicemoe_config *cfg, const slicemoe_weights *w, cons
  * copy of h into the workspace, the forward, and the device->host copy of h'.
  * Weights and the optional outputs stay DEVICE pointers.  The caller
  * synchronises the stream before reading h_out_host.
+ * Without a capacity limit and from 2048 tokens on, the batch is processed in
+ * four chunks of tokens whose copies in and out run on two streams that the
+ * library creates once per device, so that the two directions of the link are
+ * busy at the same time; in stream order the call still behaves as one
+ * operation on `stream` (later work on `stream` sees h_out_host complete).
+ * Concurrent calls from several host threads are serialised while they enqueue.
  */
 int slicemoe_forward_host(const slicemoe_config *cfg, const slicemoe_weights *w,
                           const void *h_host, void *h_out_host, int32_t *assigned_opt,

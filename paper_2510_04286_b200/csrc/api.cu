@@ -5,6 +5,7 @@
 #include <cstring>
 
 #include <cstdlib>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -135,7 +136,8 @@ static int ffn_any(const Dims& D, const slicemoe_weights& w, const void* xperm, 
 
 static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out,
                         int32_t* assigned_opt, int32_t* kept_opt, int32_t* idx_opt, float* p_opt,
-                        void* ws, const Workspace& W, cudaStream_t st, void* const* events) {
+                        void* ws, const Workspace& W, cudaStream_t st, void* const* events,
+                        bool clear_status = true) {
     int32_t* idx = idx_opt ? idx_opt : at<int32_t>(ws, W.topk_idx);
     float* p = p_opt ? p_opt : at<float>(ws, W.topk_p);
     int32_t* assigned = assigned_opt ? assigned_opt : at<int32_t>(ws, W.assigned);
@@ -151,7 +153,9 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     };
     int rc;
     const bool one_launch = !events && fused_forward_supported(D);
-    if (!one_launch && (rc = reset_status(ws, W, st))) return rc;     // (the single kernel clears it itself)
+    // (the single kernel clears the status word itself; a later chunk of one host-buffer call keeps
+    // what an earlier chunk reported)
+    if (!one_launch && clear_status && (rc = reset_status(ws, W, st))) return rc;
     if ((rc = mark(0))) return rc;
     // With both tensor-core kernels available the stacked rows are never materialised: the router
     // leaves its per-CTA expert counts, one dispatch kernel ranks the pairs (dest, perm, gate) and
@@ -162,7 +166,7 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     // the stages stay separable.
     if (one_launch)
         return launch_forward_fused(D, w, h, h_out, idx, p, assigned, kept, offsets, dest, perm, gate,
-                                    at<int32_t>(ws, W.cta_hist), at<int32_t>(ws, W.status), st);
+                                    at<int32_t>(ws, W.cta_hist), at<int32_t>(ws, W.status), clear_status, st);
     if (fused) {
         int grid = 0, rows_per_cta = 0;
         tc_route_grid(D, &grid, &rows_per_cta);
@@ -318,6 +322,63 @@ int slicemoe_forward_profiled(const slicemoe_config* cfg, const slicemoe_weights
                            ws_bytes, stream, events);
 }
 
+// ---- host-buffer forward ------------------------------------------------------------------------
+// The copies dominate this call (PCIe), and the link carries both directions at once: the batch is
+// cut into chunks of tokens and chunk j's copy in, forward and copy out run on three streams (the
+// caller's for the kernels, two of the library's for the copies), so that the copy out of chunk j
+// overlaps the copy in of chunk j + 1.  Only without a capacity limit (with one, which pair is
+// dropped depends on the whole batch's order).
+namespace slicemoe {
+namespace {
+
+#ifdef SLICEMOE_DEV_HOST_CHUNKS
+constexpr int kPipeChunks = 16;
+#else
+constexpr int kPipeChunks = 4;
+#endif
+constexpr int kPipeMinTokensPerChunk = 512;
+constexpr int kPipeMaxDevices = 64;
+
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t begin = nullptr, done = nullptr, in[kPipeChunks] = {}, fwd[kPipeChunks] = {};
+};
+HostPipe g_pipe[kPipeMaxDevices];
+std::mutex g_pipe_mutex;     // held while a call enqueues: calls share the two copy streams and the events
+
+int host_pipe(HostPipe** out) {
+    int dev = -1;
+    SLICEMOE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kPipeMaxDevices) return SLICEMOE_ERR_NO_DEVICE;
+    HostPipe& p = g_pipe[dev];
+    if (!p.ready) {
+        SLICEMOE_CUDA_TRY(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
+        SLICEMOE_CUDA_TRY(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));
+        SLICEMOE_CUDA_TRY(cudaEventCreateWithFlags(&p.begin, cudaEventDisableTiming));
+        SLICEMOE_CUDA_TRY(cudaEventCreateWithFlags(&p.done, cudaEventDisableTiming));
+        for (int i = 0; i < kPipeChunks; ++i) {
+            SLICEMOE_CUDA_TRY(cudaEventCreateWithFlags(&p.in[i], cudaEventDisableTiming));
+            SLICEMOE_CUDA_TRY(cudaEventCreateWithFlags(&p.fwd[i], cudaEventDisableTiming));
+        }
+        p.ready = true;
+    }
+    *out = &p;
+    return SLICEMOE_OK;
+}
+
+__global__ void add_counts_kernel(const int32_t* __restrict__ a, const int32_t* __restrict__ k, int32_t* A, int32_t* K,
+                                  int E) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < E) {
+        if (A) A[e] += a[e];
+        if (K) K[e] += k[e];
+    }
+}
+
+}  // namespace
+}  // namespace slicemoe
+
 int slicemoe_forward_host(const slicemoe_config* cfg, const slicemoe_weights* w, const void* h_host,
                           void* h_out_host, int32_t* assigned_opt, int32_t* kept_opt, void* ws,
                           size_t ws_bytes, void* stream) {
@@ -330,14 +391,66 @@ int slicemoe_forward_host(const slicemoe_config* cfg, const slicemoe_weights* w,
     if ((rc = check_ws(D, ws, ws_bytes, W))) return rc;
     if ((rc = check_device())) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t bytes = elem_bytes(D) * (size_t)D.T * D.d;
-    void* h_dev = at<char>(ws, W.h_dev);
-    void* hout_dev = at<char>(ws, W.hout_dev);
-    if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_dev, h_host, bytes, cudaMemcpyHostToDevice, st));
-    if ((rc = forward_impl(D, *w, h_dev, hout_dev, assigned_opt, kept_opt, nullptr, nullptr, ws, W, st,
-                           nullptr)))
-        return rc;
-    if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_out_host, hout_dev, bytes, cudaMemcpyDeviceToHost, st));
+    const size_t row_bytes = elem_bytes(D) * (size_t)D.d;
+    const size_t bytes = row_bytes * (size_t)D.T;
+    char* h_dev = at<char>(ws, W.h_dev);
+    char* hout_dev = at<char>(ws, W.hout_dev);
+
+    const bool pipelined = D.capacity == 0 && D.T >= kPipeChunks * kPipeMinTokensPerChunk;
+    if (!pipelined) {
+        if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_dev, h_host, bytes, cudaMemcpyHostToDevice, st));
+        if ((rc = forward_impl(D, *w, h_dev, hout_dev, assigned_opt, kept_opt, nullptr, nullptr, ws, W, st,
+                               nullptr)))
+            return rc;
+        if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_out_host, hout_dev, bytes, cudaMemcpyDeviceToHost, st));
+        return SLICEMOE_OK;
+    }
+
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe* pipe = nullptr;
+    if ((rc = host_pipe(&pipe))) return rc;
+    // everything already queued on the caller's stream (an earlier call's use of the staging
+    // buffers among it) comes first
+    SLICEMOE_CUDA_TRY(cudaEventRecord(pipe->begin, st));
+    SLICEMOE_CUDA_TRY(cudaStreamWaitEvent(pipe->s_in, pipe->begin, 0));
+    SLICEMOE_CUDA_TRY(cudaStreamWaitEvent(pipe->s_out, pipe->begin, 0));
+    if (assigned_opt) SLICEMOE_CUDA_TRY(cudaMemsetAsync(assigned_opt, 0, sizeof(int32_t) * D.E, st));
+    if (kept_opt) SLICEMOE_CUDA_TRY(cudaMemsetAsync(kept_opt, 0, sizeof(int32_t) * D.E, st));
+    const bool counts = assigned_opt || kept_opt;
+    int nchunks_host = kPipeChunks;
+#ifdef SLICEMOE_DEV_HOST_CHUNKS
+    if (const char* ev = getenv("SLICEMOE_HOST_CHUNKS")) nchunks_host = atoi(ev) > 0 && atoi(ev) <= kPipeChunks ? atoi(ev) : kPipeChunks;
+#endif
+    const int t_chunk = (D.T + nchunks_host - 1) / nchunks_host;
+    int j = 0;
+    for (int t0 = 0; t0 < D.T; t0 += t_chunk, ++j) {
+        const int tc = D.T - t0 < t_chunk ? D.T - t0 : t_chunk;
+        const size_t off = row_bytes * (size_t)t0, cb = row_bytes * (size_t)tc;
+        SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_dev + off, static_cast<const char*>(h_host) + off, cb,
+                                          cudaMemcpyHostToDevice, pipe->s_in));
+        SLICEMOE_CUDA_TRY(cudaEventRecord(pipe->in[j], pipe->s_in));
+        SLICEMOE_CUDA_TRY(cudaStreamWaitEvent(st, pipe->in[j], 0));
+        slicemoe_config cc = *cfg;
+        cc.T = tc;
+        Dims Dc;
+        if ((rc = make_dims(&cc, Dc))) return rc;
+        // the chunk's counts go to the workspace's own arrays and are added up below
+        if ((rc = forward_impl(Dc, *w, h_dev + off, hout_dev + off, nullptr, nullptr, nullptr, nullptr, ws, W, st,
+                               nullptr, /*clear_status=*/j == 0)))
+            return rc;
+        if (counts) {
+            add_counts_kernel<<<(D.E + 127) / 128, 128, 0, st>>>(at<int32_t>(ws, W.assigned), at<int32_t>(ws, W.kept),
+                                                                assigned_opt, kept_opt, D.E);
+            SLICEMOE_LAUNCH_CHECK(1);
+        }
+        SLICEMOE_CUDA_TRY(cudaEventRecord(pipe->fwd[j], st));
+        SLICEMOE_CUDA_TRY(cudaStreamWaitEvent(pipe->s_out, pipe->fwd[j], 0));
+        SLICEMOE_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(h_out_host) + off, hout_dev + off, cb,
+                                          cudaMemcpyDeviceToHost, pipe->s_out));
+    }
+    // the caller's stream is done when the last copy out is
+    SLICEMOE_CUDA_TRY(cudaEventRecord(pipe->done, pipe->s_out));
+    SLICEMOE_CUDA_TRY(cudaStreamWaitEvent(st, pipe->done, 0));
     return SLICEMOE_OK;
 }
 

@@ -125,7 +125,8 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
 bool fused_forward_supported(const Dims& D);
 int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
                          float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
-                         int32_t* perm, float* gate, int32_t* cta_hist, int32_t* status, cudaStream_t st);
+                         int32_t* perm, float* gate, int32_t* cta_hist, int32_t* status, bool clear_status,
+                         cudaStream_t st);
 int fused_forward_reset_sync(cudaStream_t st);
 
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,

@@ -28,6 +28,7 @@ struct FusedParams {
     int32_t *assigned, *kept, *offsets, *dest, *perm;
     float* gate;
     int32_t* sync_words;      // g_grid_sync of this device
+    int clear_status;         // set the status word to OK at entry
 };
 
 // Grid barrier words (arrival count, generation), one pair per device, owned by the library: zero
@@ -92,7 +93,7 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     int32_t gen0 = 0;
     if (threadIdx.x == 0) {
         gen0 = *reinterpret_cast<volatile int32_t*>(fp.sync_words + 1);   // no barrier can complete without this CTA
-        if (blockIdx.x == 0) *fp.ffn.status = SLICEMOE_OK;              // run-outs (>= seconds later) overwrite it
+        if (blockIdx.x == 0 && fp.clear_status) *fp.ffn.status = SLICEMOE_OK;              // run-outs (>= seconds later) overwrite it
     }
 #ifdef SLICEMOE_FUSED_STAMPS
     // per-launch ring (slot = launch number mod 32): earliest CTA entry and latest CTA exit
@@ -256,8 +257,10 @@ bool fused_forward_supported(const Dims& D) {
 
 int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
                          float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
-                         int32_t* perm, float* gate, int32_t* cta_hist, int32_t* status, cudaStream_t st) {
+                         int32_t* perm, float* gate, int32_t* cta_hist, int32_t* status, bool clear_status,
+                         cudaStream_t st) {
     FusedParams fp{};
+    fp.clear_status = clear_status ? 1 : 0;
     int rc = grid_sync_address(&fp.sync_words);
     if (rc) return rc;
     const int grid = sm_count();

@@ -150,6 +150,45 @@ def test_forward_host_matches_forward():
     assert torch.equal(out_host, h_dev.cpu())
 
 
+def test_forward_host_pipelined_in_chunks():
+    """From 2048 tokens on (no capacity limit) the host-buffer forward runs in four chunks with
+    overlapping copies: same bits as the device forward, counts summed over the chunks, and the
+    caller's stream alone orders the result."""
+    import torch
+    lc = C["cfg1"].with_tokens(2048 + 77)            # ragged last chunk
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    h_dev, assigned_dev, kept_dev, _, _ = gpu.forward()
+    h_host = tensors.to_torch(h, lc.dtype, "cpu", pin=True)
+    out_host = torch.zeros_like(h_host).pin_memory()
+    assigned = torch.full((lc.E,), -5, dtype=torch.int32, device="cuda")
+    kept = torch.full((lc.E,), -5, dtype=torch.int32, device="cuda")
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for _ in range(3):                           # back-to-back calls reuse the staging buffers
+            binding.slicemoe_forward_host(gpu.cfg, gpu.w, h_host, out_host, gpu.ws, assigned, kept)
+    s.synchronize()                                  # only the caller's stream
+    assert torch.equal(out_host, h_dev.cpu())
+    assert torch.equal(assigned, assigned_dev) and torch.equal(kept, kept_dev)
+    assert gpu.status() == 0
+
+
+def test_forward_host_with_capacity_is_not_chunked():
+    """With a capacity limit the drop order spans the whole batch: one forward, same result."""
+    import torch
+    lc = LC("hostcap", T=2304, d=256, S=4, E=16, k=2, F=256, capacity=300)
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    h_dev, _, kept_dev, _, _ = gpu.forward()
+    h_host = tensors.to_torch(h, lc.dtype, "cpu", pin=True)
+    out_host = torch.zeros_like(h_host).pin_memory()
+    kept = torch.zeros((lc.E,), dtype=torch.int32, device="cuda")
+    binding.slicemoe_forward_host(gpu.cfg, gpu.w, h_host, out_host, gpu.ws, None, kept)
+    torch.cuda.synchronize()
+    assert torch.equal(out_host, h_dev.cpu()) and torch.equal(kept, kept_dev)
+    assert int(kept.max()) == 300                    # the limit binds, so chunking would have changed the result
+
+
 def test_profiled_forward_records_stage_times():
     import torch
     lc = SMALL["bf16_lm"]

@@ -15,6 +15,7 @@ namespace slicemoe {
 // brought into shared memory with all loads in flight at once (the ranking loop itself is a chain
 // of dependent warp votes and would otherwise pay the memory latency once per 32 pairs), then
 // counted per warp, prefixed over warps, and ranked with match-any inside the warp.
+// offs_out (shared memory, E + 1 ints, or NULL) receives a copy of the offsets.
 // NT threads take part (the whole CTA: the body synchronises with __syncthreads); `sm` is 16-byte
 // aligned shared memory of dispatch_fused_smem_bytes(E, G, NT) bytes.  SAME_LAUNCH: the router phase
 // of the same launch wrote topk_idx / topk_p / table, so they are not read through the
@@ -30,7 +31,7 @@ __device__ __forceinline__ void dispatch_fused_body(
     const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_p, const int32_t* __restrict__ table,
     int G, int chunk, int R, int E, int pairs_per_chunk, int capacity, int32_t* __restrict__ assigned,
     int32_t* __restrict__ kept, int32_t* __restrict__ offsets, int32_t* __restrict__ dest,
-    int32_t* __restrict__ perm, float* __restrict__ gate, int* sm) {
+    int32_t* __restrict__ perm, float* __restrict__ gate, int* sm, int* offs_out = nullptr) {
     constexpr int kFusedThreads = NT, kFusedWarps = NT / 32;
     int* seg_e = sm;                               // [kSegPairs]  (16-byte aligned: first)
     float* seg_p = reinterpret_cast<float*>(seg_e + kSegPairs);   // [kSegPairs]
@@ -111,6 +112,9 @@ __device__ __forceinline__ void dispatch_fused_body(
         }
     }
     __syncthreads();
+    // (single-kernel forward: every CTA keeps the offsets it has just derived for its expert pass)
+    if (offs_out)
+        for (int e = threadIdx.x; e <= E; e += kFusedThreads) offs_out[e] = offs[e];
     if (!has_pairs) return;
 
     int* mine = wcnt + warp * E;

@@ -118,14 +118,14 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
         dispatch_fused_body<RC::THREADS, true>(fp.route.topk_idx, fp.route.topk_p, fp.route.cta_hist, (int)gridDim.x,
                                                (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.capacity,
-                                               fp.assigned, fp.kept, fp.offsets, fp.dest, fp.perm, fp.gate, dsm);
+                                               fp.assigned, fp.kept, fp.offsets, fp.dest, fp.perm, fp.gate, dsm, sh.offs);
     }
     STAMP(3);
     ok = grid_barrier(fp.sync_words, gen0 + 1, sh) && ok;
     STAMP(4);
 
     // ---- phase 3: experts ------------------------------------------------------------------------
-    if (ok) tc_body<EC, true>(&tmX, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
+    if (ok) tc_body<EC, true, true>(&tmX, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
 
     __syncthreads();

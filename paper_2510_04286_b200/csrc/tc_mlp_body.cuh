@@ -354,8 +354,9 @@ __device__ __forceinline__ int ld_index(const int32_t* ptr) {
 // One pass of the two-layer MLP pipeline over this CTA's share of the row tiles: the body of the
 // router and expert kernels, and of the router and expert phases of the single-kernel forward.
 // Called by all threads of the CTA; TMEM (sh.tmem_base, at least C::TMEM_COLS columns) is allocated
-// and freed by the caller.  SAME_LAUNCH: offsets / perm / gate were written earlier in this launch.
-template <class C, bool SAME_LAUNCH>
+// and freed by the caller.  SAME_LAUNCH: offsets / perm / gate were written earlier in this launch;
+// OFFS_IN_SMEM: sh.offs already holds the row ranges.
+template <class C, bool SAME_LAUNCH, bool OFFS_IN_SMEM = false>
 __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p,
                                         const TcParams& p, TcShared& sh, uint8_t* smem_raw) {
     using B = Bars<C>;
@@ -404,16 +405,28 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         prefetch_tensormap(&tmW1);
         prefetch_tensormap(&tmW2);
     }
-    for (int e = threadIdx.x; e <= p.E; e += C::THREADS) sh.offs[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.n_rows);
+    // row ranges: the router's single range, the experts' offsets from global memory, or (single-kernel
+    // forward) already in sh.offs, left there by the dispatch phase of this CTA
+    if (!OFFS_IN_SMEM)
+        for (int e = threadIdx.x; e <= p.E; e += C::THREADS) sh.offs[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.n_rows);
     for (int e = threadIdx.x; e < kMaxE; e += C::THREADS) sh.hist[e] = 0;
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (warp == 0) {
+        // first tile of every expert: exclusive scan of the tile counts, 32 experts at a time
         int run = 0;
-        for (int e = 0; e < p.E; ++e) {
-            sh.tile_start[e] = run;
-            run += (sh.offs[e + 1] - sh.offs[e] + kTileM - 1) / kTileM;
+        for (int e0 = 0; e0 < p.E; e0 += 32) {
+            const int e = e0 + lane;
+            const int nt = e < p.E ? (sh.offs[e + 1] - sh.offs[e] + kTileM - 1) / kTileM : 0;
+            int incl = nt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += up;
+            }
+            if (e < p.E) sh.tile_start[e] = run + incl - nt;
+            run += __shfl_sync(0xffffffffu, incl, 31);
         }
-        sh.tile_start[p.E] = run;
+        if (lane == 0) sh.tile_start[p.E] = run;
     }
     tc_fence_before_sync();
     __syncthreads();

@@ -337,6 +337,7 @@ constexpr int kPipeChunks = 16;
 constexpr int kPipeChunks = 4;
 #endif
 constexpr int kPipeMinTokensPerChunk = 512;
+constexpr double kPipeEdgeShare = 0.5;        // first / last chunk relative to an inner chunk
 constexpr int kPipeMaxDevices = 64;
 
 struct HostPipe {
@@ -417,14 +418,34 @@ int slicemoe_forward_host(const slicemoe_config* cfg, const slicemoe_weights* w,
     if (assigned_opt) SLICEMOE_CUDA_TRY(cudaMemsetAsync(assigned_opt, 0, sizeof(int32_t) * D.E, st));
     if (kept_opt) SLICEMOE_CUDA_TRY(cudaMemsetAsync(kept_opt, 0, sizeof(int32_t) * D.E, st));
     const bool counts = assigned_opt || kept_opt;
+    // Chunk boundaries in tokens.  The first and the last chunk are short: nothing overlaps the first
+    // copy in or the last copy out.
+    int bounds[kPipeChunks + 1];
     int nchunks_host = kPipeChunks;
 #ifdef SLICEMOE_DEV_HOST_CHUNKS
     if (const char* ev = getenv("SLICEMOE_HOST_CHUNKS")) nchunks_host = atoi(ev) > 0 && atoi(ev) <= kPipeChunks ? atoi(ev) : kPipeChunks;
+    double edge = 0.5;
+    if (const char* ev = getenv("SLICEMOE_HOST_EDGE")) edge = atof(ev);
+#else
+    const double edge = kPipeEdgeShare;
 #endif
-    const int t_chunk = (D.T + nchunks_host - 1) / nchunks_host;
-    int j = 0;
-    for (int t0 = 0; t0 < D.T; t0 += t_chunk, ++j) {
-        const int tc = D.T - t0 < t_chunk ? D.T - t0 : t_chunk;
+    {
+        // edge chunks get `edge` times the share of an inner chunk
+        const double inner = 1.0 / (nchunks_host - 2 + 2 * edge);
+        double acc = 0.0;
+        bounds[0] = 0;
+        for (int i = 0; i < nchunks_host; ++i) {
+            acc += (nchunks_host < 3 || (i > 0 && i < nchunks_host - 1)) ? (nchunks_host < 3 ? 1.0 / nchunks_host : inner) : edge * inner;
+            int b = (int)(acc * D.T + 0.5);
+            if (b < bounds[i]) b = bounds[i];
+            if (b > D.T) b = D.T;
+            bounds[i + 1] = b;
+        }
+        bounds[nchunks_host] = D.T;
+    }
+    for (int j = 0; j < nchunks_host; ++j) {
+        const int t0 = bounds[j], tc = bounds[j + 1] - bounds[j];
+        if (tc <= 0) continue;
         const size_t off = row_bytes * (size_t)t0, cb = row_bytes * (size_t)tc;
         SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_dev + off, static_cast<const char*>(h_host) + off, cb,
                                           cudaMemcpyHostToDevice, pipe->s_in));

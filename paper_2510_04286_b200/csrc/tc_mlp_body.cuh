@@ -283,23 +283,23 @@ template <int ACT>
 __device__ __forceinline__ void activate_post_bf16x2(const __nv_bfloat162* z, const __nv_bfloat162* t, uint32_t* out) {
     constexpr int P = 8;
 #ifdef SLICEMOE_TC_SKELETON
-    const bool relu = true;
+    constexpr bool relu = true;
 #else
-    const bool relu = ACT == SLICEMOE_ACT_RELU;
+    constexpr bool relu = ACT == SLICEMOE_ACT_RELU;
 #endif
-    if (relu) {
+    if constexpr (relu) {
         const __nv_bfloat162 zero = __float2bfloat162_rn(0.0f);
 #pragma unroll
         for (int i = 0; i < P; ++i) {
             const __nv_bfloat162 r = __hmax2(z[i], zero);
             out[i] = *reinterpret_cast<const uint32_t*>(&r);
         }
-        return;
-    }
+    } else {
 #pragma unroll
-    for (int i = 0; i < P; ++i) {
-        const __nv_bfloat162 r = __hfma2(z[i], t[i], z[i]);
-        out[i] = *reinterpret_cast<const uint32_t*>(&r);
+        for (int i = 0; i < P; ++i) {
+            const __nv_bfloat162 r = __hfma2(z[i], t[i], z[i]);
+            out[i] = *reinterpret_cast<const uint32_t*>(&r);
+        }
     }
 }
 // factor the output epilogue applies to the GEMM-2 accumulator (see above)
@@ -545,12 +545,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W1C_BYTES) >> 4);
                     const uint32_t d = tmem_base + b * C::HC;
                     mma_ss<0>(d, a0, w0, idesc1);
-#ifndef SLICEMOE_DEV_G1_ONE   // development: time the pipeline with a single GEMM-1 MMA per chunk
 #pragma unroll
                     for (int kk = 1; kk < C::K1 / 16; ++kk)
                         mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
                                   w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
-#endif
                     mma_commit(bar(B::ACC1_FULL + b));
                     // streamed weights: the W1 slot is free as soon as these MMAs have read it
                     // (resident weights are handed back by the GEMM-2 thread at an expert change)
@@ -617,9 +615,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                                 a = hbuf + kk * 8;
                             const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
                             if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, c > 0 ? 1u : 0u);
-#ifndef SLICEMOE_DEV_G2_ONE   // development: time the pipeline with a single GEMM-2 MMA per chunk
                             else mma_ts<1>(d, a, bd, idesc2);
-#endif
                         }
                     }
                     mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
@@ -732,21 +728,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         int e = 0;
         uint32_t g = 0;
         TRACE_DECL(tr, (lg == 0 && lane == 0 && w == 0 && grp < 2) ? 2 + grp : 7);
-#ifdef SLICEMOE_TC_ACCT   // development: where do the activation warps spend their cycles?
-        long long acct_wait_acc1 = 0, acct_wait_hempty = 0, acct_stwait = 0, acct_t0 = clock64(), acct_mark;
-#define ACCT_BEGIN() acct_mark = clock64()
-#define ACCT_END(var) var += clock64() - acct_mark
-#else
-#define ACCT_BEGIN()
-#define ACCT_END(var)
-#endif
-#ifdef SLICEMOE_TC_PROBE   // development: clock stamps inside one chunk (g == 12) of one warp
-        unsigned probe[16];
-        for (int i = 0; i < 16; ++i) probe[i] = 0;
-#define PROBE(i) do { if (g == 12) probe[i] = (unsigned)clock(); } while (0)
-#else
-#define PROBE(i)
-#endif
         int prev_e = -1;
         uint32_t q_tile = 0, q_next = 0;              // bias ring: W1 load count of this tile's chunk 0 / after it
         for (int t = t_begin; t < t_end && ok; ++t) {
@@ -766,16 +747,12 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 const uint32_t acc1 = lane_base + b * C::HC + w * WCOLS;               // my accumulator columns
                 const uint32_t hdst = lane_base + C::H_COL0 + b * (C::HC / 2) + w * (WCOLS / 2);
                 TRACE(tr, 30);
-                PROBE(0);
-                ACCT_BEGIN();
                 ok = mbar_wait(bar(B::ACC1_FULL + b), n1 & 1u, abort, kWaitLimitNs);
                 ok = __all_sync(0xffffffffu, ok);
-                ACCT_END(acct_wait_acc1);
                 if (!ok) break;
                 // (the tile's A rows, and with them its ring entry, landed before GEMM-1 could run)
                 if (gather) gs = sh.gate_s[(t - t_begin) % kMetaRing][lg * 32 + lane];
                 TRACE(tr, 31);
-                PROBE(1);
                 tc_fence_after_sync();
                 // this chunk's bias came into shared memory with its W1 (same barrier, own ring)
                 const int bslot = (int)((q_tile + c) % kBiasRing);
@@ -815,7 +792,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                             convert_piece_bf16x2(v[i], gate_hi, gate_lo, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
                                                  p.bias1 != nullptr, z[s0 + i]);
                     }
-                    PROBE(3);
                     TRACE(tr, 32);
                     tc_fence_before_sync();
                     __syncwarp();
@@ -827,10 +803,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         if (pc == 0) {
                             TRACE(tr, 33);
                             // GEMM-2 of two chunks ago must be done with this hidden buffer
-                            ACCT_BEGIN();
                             ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
                             ok = __all_sync(0xffffffffu, ok);
-                            ACCT_END(acct_wait_hempty);
                             if (!ok) break;
                             TRACE(tr, 34);
                         } else {
@@ -839,7 +813,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                             tmem_st_x8(hdst + (pc - 1) * (C::PIECE / 2), hi);
                         }
                     }
-                    PROBE(12);
                 } else {
                     uint32_t v[2][C::PIECE];
                     tmem_ld_x16(acc1, v[0]);
@@ -856,30 +829,14 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     }
                 }
                 if (!ok) break;
-                ACCT_BEGIN();
                 tmem_st_wait();
                 TRACE(tr, 37);
-                ACCT_END(acct_stwait);
-                PROBE(13);
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B::H_FULL + b));
-                PROBE(14);
                 TRACE(tr, 35);
             }
         }
-#ifdef SLICEMOE_TC_PROBE
-        if (lane == 0 && p.status != nullptr && blockIdx.x == 0 && !C::ROUTER) {
-            unsigned* out = reinterpret_cast<unsigned*>(p.status + 16) + (warp - 4) * 16;
-            for (int i = 0; i < 16; ++i) out[i] = probe[i];
-        }
-#endif
-#ifdef SLICEMOE_TC_ACCT
-        if (lane == 0 && p.status != nullptr && blockIdx.x == 0) {
-            long long* out = reinterpret_cast<long long*>(p.status + 16) + (warp - 4) * 4;   // status area: int32[64] -> spill past it
-            out[0] = clock64() - acct_t0; out[1] = acct_wait_acc1; out[2] = acct_wait_hempty; out[3] = acct_stwait;
-        }
-#endif
     } else if (warp >= C::OUT_WARP0) {
         // ================= output warpgroup ==================================================
         const int lg = warp & 3;

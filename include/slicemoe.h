@@ -181,6 +181,22 @@ int slicemoe_combine(const slicemoe_config *cfg, const void *yperm, const int32_
                      void *h_out, void *stream);
 
 /*
+ * Section 3.3, cross-slice dropout: turns the router's top-k probabilities into
+ * train-mode gates, in place, between slicemoe_route and slicemoe_dispatch.
+ * Each of a row's k probabilities is set to zero independently with probability
+ * `rate` (Appendix A: 0.2) and the survivors are divided by their sum; if none
+ * survives, the top-1 assignment (j = 0) gets weight 1.  Readings of the paper:
+ * one Bernoulli draw per assignment; a dropped assignment stays routed, with
+ * gate 0 (Eq. 1 with p = 0); rate = 0 still re-normalises.  The draw for
+ * assignment j of row n is the first word of Philox4x32-10 with key = seed and
+ * counter (n, j, 0, 0); dropped iff word < floor(rate * 2^32) -- reproducible
+ * from (seed, n, j) alone.  topk_p: DEVICE float [N, k], k <= 8; 0 <= rate <= 1.
+ * The one-launch slicemoe_forward has no train mode; compose the staged calls.
+ */
+int slicemoe_gate_dropout(const slicemoe_config *cfg, float *topk_p, uint64_t seed, double rate,
+                          void *stream);
+
+/*
  * Routing statistics from per-expert counts (such as `assigned` of the forward):
  *   out[0] = L_cap of Eq. 2 = alpha * (std(counts) / mean(counts))^2, with the
  *            population standard deviation (divide by E) -- the paper does not

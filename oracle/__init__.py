@@ -242,3 +242,26 @@ def load_stats(counts, alpha: float = 1.0):
                                           ctypes.c_double(alpha), ctypes.byref(l_cap),
                                           ctypes.byref(ele)), "load_stats")
     return l_cap.value, ele.value
+
+
+def philox4x32(ctr, key):
+    """One Philox4x32-10 block: ctr 4 x uint32, key 2 x uint32 -> 4 x uint32."""
+    lib = _load()
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib.slicemoe_oracle_philox4x32(_p(c), _p(k), _p(out))
+    return out
+
+
+def gate_dropout(topk_p, seed: int, rate: float):
+    """Section 3.3: (gates after cross-slice dropout [N, k], dropped mask [N, k] bool)."""
+    lib = _load()
+    p = np.ascontiguousarray(topk_p, dtype=np.float64)
+    N, k = p.shape
+    out = np.empty_like(p)
+    dropped = np.zeros((N, k), dtype=np.uint8)
+    _check(lib.slicemoe_oracle_gate_dropout(_p(p), ctypes.c_int64(N), ctypes.c_int32(k),
+                                            ctypes.c_uint64(seed), ctypes.c_double(rate), _p(out),
+                                            _p(dropped)), "gate_dropout")
+    return out, dropped.astype(bool)

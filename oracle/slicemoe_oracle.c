@@ -23,7 +23,10 @@
  * inputs, a hand-worked example, identity experts, E = 1, zero router,
  * Zipf-bias capacity closed form, reshape (S = 1) equivalence, permutation
  * equivariance, an affine special case and a dense-MLP special case checked
- * against numpy matmul.  No function here is unpinned.
+ * against numpy matmul; load statistics against their closed forms; cross-slice
+ * dropout (tests/test_dropout.py) against the generator's published known-answer
+ * vectors, a pure-Python restatement, and its invariants.  No function here is
+ * unpinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -442,5 +445,66 @@ int slicemoe_oracle_load_stats(const int64_t *counts, int32_t E, double alpha,
         if (load > 0.0) ent -= load * log(load);
     }
     *ele = (E == 1) ? 1.0 : ent / log((double)E);
+    return ORACLE_OK;
+}
+
+/* ---- Section 3.3, cross-slice dropout (train-mode gates) ------------------------------
+ *
+ * After top-k, each of a slice's k assignment probabilities is set to zero independently
+ * with probability `rate` (Appendix A: rate 0.2, "20% of selected expert assignments per
+ * slice dropped"); the survivors are re-normalised to sum to 1.  Readings: the paper's
+ * "a fraction of these k probabilities" is taken as one Bernoulli draw per assignment (k is
+ * 1..3, so a fixed fraction of k is not an integer); when all k are dropped the top-1
+ * assignment keeps weight 1 ("ensuring information flow is maintained"); a dropped
+ * assignment stays routed with gate 0 (Eq. 1 with p = 0).
+ *
+ * The draws come from the counter-based generator Philox4x32-10 (Salmon et al., SC'11):
+ * key = the 64-bit seed, counter = (n, j, 0, 0) for assignment j of row n, the first output
+ * word u decides: dropped iff u < floor(rate * 2^32).  The CUDA path implements the same
+ * generator on its own; the decision is an integer compare, so both sides agree bit for bit.
+ */
+static void philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t out[4]) {
+    uint32_t c0 = ctr_in[0], c1 = ctr_in[1], c2 = ctr_in[2], c3 = ctr_in[3];
+    uint32_t k0 = key_in[0], k1 = key_in[1];
+    for (int round = 0; round < 10; ++round) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+void slicemoe_oracle_philox4x32(const uint32_t *ctr, const uint32_t *key, uint32_t *out) {
+    philox4x32_10(ctr, key, out);
+}
+
+int slicemoe_oracle_gate_dropout(const double *topk_p /* [N, k] */, int64_t N, int32_t k,
+                                 uint64_t seed, double rate, double *p_out /* [N, k] */,
+                                 uint8_t *dropped /* [N, k] */) {
+    if (N < 0 || k < 1 || !(rate >= 0.0) || rate > 1.0) return ORACLE_BAD_SHAPE;
+    const uint64_t threshold = (uint64_t)(rate * 4294967296.0);       /* 2^32 when rate = 1 */
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    for (int64_t n = 0; n < N; ++n) {
+        double kept_sum = 0.0;
+        int kept = 0;
+        for (int j = 0; j < k; ++j) {
+            const uint32_t ctr[4] = {(uint32_t)n, (uint32_t)j, 0u, 0u};
+            uint32_t r[4];
+            philox4x32_10(ctr, key, r);
+            const int drop = (uint64_t)r[0] < threshold;
+            dropped[n * k + j] = (uint8_t)drop;
+            if (!drop) { kept_sum += topk_p[n * k + j]; ++kept; }
+        }
+        for (int j = 0; j < k; ++j) {
+            if (kept == 0 || !(kept_sum > 0.0)) p_out[n * k + j] = (j == 0) ? 1.0 : 0.0;
+            else p_out[n * k + j] = dropped[n * k + j] ? 0.0 : topk_p[n * k + j] / kept_sum;
+        }
+    }
     return ORACLE_OK;
 }

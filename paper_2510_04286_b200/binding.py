@@ -21,7 +21,7 @@ STAGES = ("route", "dispatch", "expert_ffn", "combine")
 EXPORTS = (
     "slicemoe_workspace_bytes", "slicemoe_route", "slicemoe_dispatch", "slicemoe_dispatch_static",
     "slicemoe_expert_ffn",
-    "slicemoe_combine", "slicemoe_load_stats", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
+    "slicemoe_combine", "slicemoe_gate_dropout", "slicemoe_load_stats", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
     "slicemoe_event_create", "slicemoe_event_destroy", "slicemoe_event_elapsed_ms",
     "slicemoe_last_status", "slicemoe_launch_count", "slicemoe_last_cuda_error",
     "slicemoe_status_string",
@@ -184,6 +184,13 @@ def slicemoe_combine(cfg, yperm, dest, h_out, stream=None):
     c = cfg.c()
     _check(_lib().slicemoe_combine(ctypes.byref(c), _ptr(yperm), _ptr(dest), _ptr(h_out), _stream(stream)),
            "slicemoe_combine")
+
+
+def slicemoe_gate_dropout(cfg, topk_p, seed, rate, stream=None):
+    """Section 3.3: topk_p (cuda float32 [N, k]) becomes the train-mode gates, in place."""
+    c = cfg.c()
+    _check(_lib().slicemoe_gate_dropout(ctypes.byref(c), _ptr(topk_p), ctypes.c_uint64(seed), ctypes.c_double(rate),
+                                        _stream(stream)), "slicemoe_gate_dropout")
 
 
 def slicemoe_load_stats(counts, alpha, out, stream=None):

@@ -257,7 +257,13 @@ def run_ours(args, lc):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(3, args.warmup)):
+    # The clock sampler (an nvidia-smi child every 100 ms) starts before the warm-up so that spawning
+    # it does not compete with the launching thread inside the timed region; it keeps sampling through
+    # all three timed regions below.
+    clocks = ClockSampler(local)
+    clocks.__enter__()
+    warm = max(3, args.warmup)
+    for i in range(warm):
         step(i)
     torch.cuda.synchronize()
     if sm.slicemoe_last_status(ws) != 0:
@@ -273,8 +279,6 @@ def run_ours(args, lc):
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     launches0 = sm.slicemoe_launch_count()
-    clocks = ClockSampler(local)          # samples through all three timed regions below
-    clocks.__enter__()
     start.record()
     for i in range(args.steps):
         step(i)

@@ -311,22 +311,39 @@ constexpr float kOutScale =
     (ACT == SLICEMOE_ACT_RELU) ? 1.0f : 0.5f;
 #endif
 
-// Router: ReLU in fp32, then each value as a bf16 pair, the rounded value (hi) and the rounded
-// remainder (lo); hi + lo carries 16 mantissa bits of the fp32 value.
-__device__ __forceinline__ void relu_split_piece(const uint32_t* cur, uint32_t* hi, uint32_t* lo) {
+// Router: relu(acc + bias) as a bf16 pair per value: hi = the value truncated to bf16, lo = the
+// rounded remainder; hi + lo carries 16 mantissa bits of the fp32 value.  The ReLU rides on the two
+// conversions: hi is converted round-toward-zero with .relu (a negative value gives hi = 0), so the
+// remainder a - hi is a itself for a < 0 and non-negative otherwise, and the .relu of the second
+// conversion zeroes exactly the negative inputs.  Per column pair: 2 adds, 1 conversion, 2 unpacks,
+// 2 subtractions, 1 conversion.
+__device__ __forceinline__ uint32_t cvt_rz_relu_bf16x2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rz.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ uint32_t cvt_rn_relu_bf16x2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ void bias_relu_split_piece(const uint32_t* cur, const float* bias /* 16 fp32, shared */,
+                                                      uint32_t* hi, uint32_t* lo) {
     constexpr int P = 8;
     float a[2 * P];
 #pragma unroll
-    for (int i = 0; i < 2 * P; ++i) a[i] = fmaxf(__uint_as_float(cur[i]), 0.0f);
-#pragma unroll
-    for (int i = 0; i < P; ++i) hi[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
-#pragma unroll
-    for (int i = 0; i < P; ++i) {
-        a[2 * i] -= __uint_as_float(hi[i] << 16);
-        a[2 * i + 1] -= __uint_as_float(hi[i] & 0xFFFF0000u);
+    for (int i = 0; i < 2 * P; i += 4) {
+        const float4 b = *reinterpret_cast<const float4*>(bias + i);      // same address for the whole warp
+        a[i] = __uint_as_float(cur[i]) + b.x;
+        a[i + 1] = __uint_as_float(cur[i + 1]) + b.y;
+        a[i + 2] = __uint_as_float(cur[i + 2]) + b.z;
+        a[i + 3] = __uint_as_float(cur[i + 3]) + b.w;
     }
 #pragma unroll
-    for (int i = 0; i < P; ++i) lo[i] = pack_bf16x2(a[2 * i], a[2 * i + 1]);
+    for (int i = 0; i < P; ++i) hi[i] = cvt_rz_relu_bf16x2(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < P; ++i)
+        lo[i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hi[i] << 16), a[2 * i + 1] - __uint_as_float(hi[i] & 0xFFFF0000u));
 }
 
 // Shared-memory state of one CTA besides the operand tiles.
@@ -341,6 +358,8 @@ struct TcShared {
     // gather warp with the rows themselves (ring over the CTA's tile counter)
     float gate_s[kMetaRing][kTileM];
     int pair_s[kMetaRing][kTileM];
+    // router: the first layer's bias as fp32 (the router's weights never change inside a pass)
+    __align__(16) float bias1_f32[kMaxHid];
 };
 
 // Loads of data that an earlier phase of the same launch may have written (single-kernel forward)
@@ -410,6 +429,9 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     if (!OFFS_IN_SMEM)
         for (int e = threadIdx.x; e <= p.E; e += C::THREADS) sh.offs[e] = p.offsets ? p.offsets[e] : (e == 0 ? 0 : p.n_rows);
     for (int e = threadIdx.x; e < kMaxE; e += C::THREADS) sh.hist[e] = 0;
+    if constexpr (C::ROUTER)
+        for (int i = threadIdx.x; i < p.HID; i += C::THREADS)
+            sh.bias1_f32[i] = p.bias1 ? __bfloat162float(p.bias1[i]) : 0.0f;
     __syncthreads();
     if (warp == 0) {
         // first tile of every expert: exclusive scan of the tile counts, 32 experts at a time
@@ -757,20 +779,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 // this chunk's bias came into shared memory with its W1 (same barrier, own ring)
                 const int bslot = (int)((q_tile + c) % kBiasRing);
                 const uint8_t* sb1 = smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_B1 + bslot * C::B1_BYTES + w * WCOLS * 2;
-                auto add_bias = [&](uint32_t* cur, int pc) {
-                    if (p.bias1) {
-#pragma unroll
-                        for (int j = 0; j < C::PIECE; j += 8) {
-                            float bb[8];
-                            unpack16<bf16>(*reinterpret_cast<const uint4*>(sb1 + (pc * C::PIECE + j) * 2), bb);   // warp-wide broadcast
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) cur[j + i] = __float_as_uint(fmaf(__uint_as_float(cur[j + i]), gs, bb[i]));
-                        }
-                    } else if (gather) {
-#pragma unroll
-                        for (int i = 0; i < C::PIECE; ++i) cur[i] = __float_as_uint(__uint_as_float(cur[i]) * gs);
-                    }
-                };
                 if constexpr (C::PACKED_ACT) {
                     // Experts.  The whole accumulator chunk is brought into registers as packed bf16
                     // (SUB pieces at a time) and handed back at once, so that GEMM-1 of this group's
@@ -821,9 +829,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         uint32_t* cur = v[pc & 1];
                         tmem_ld_wait();
                         if (pc + 1 < C::NPIECE) tmem_ld_x16(acc1 + (pc + 1) * C::PIECE, v[(pc + 1) & 1]);   // overlaps the math below
-                        add_bias(cur, pc);
                         uint32_t hi[C::PIECE / 2], lo[C::PIECE / 2];
-                        relu_split_piece(cur, hi, lo);
+                        bias_relu_split_piece(cur, sh.bias1_f32 + c * C::HC + w * WCOLS + pc * C::PIECE, hi, lo);
                         tmem_st_x8(acc1 + pc * (C::PIECE / 2), hi);     // over columns this thread has already read
                         tmem_st_x8(hdst + pc * (C::PIECE / 2), lo);
                     }

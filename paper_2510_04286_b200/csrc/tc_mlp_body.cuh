@@ -360,6 +360,7 @@ struct TcShared {
     int pair_s[kMetaRing][kTileM];
     // router: the first layer's bias as fp32 (the router's weights never change inside a pass)
     __align__(16) float bias1_f32[kMaxHid];
+    __align__(16) float bias2_f32[kMaxE];
 };
 
 // Loads of data that an earlier phase of the same launch may have written (single-kernel forward)
@@ -432,6 +433,9 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     if constexpr (C::ROUTER)
         for (int i = threadIdx.x; i < p.HID; i += C::THREADS)
             sh.bias1_f32[i] = p.bias1 ? __bfloat162float(p.bias1[i]) : 0.0f;
+    if constexpr (C::ROUTER)
+        for (int i = threadIdx.x; i < C::N2; i += C::THREADS)
+            sh.bias2_f32[i] = p.bias2 ? __bfloat162float(p.bias2[i]) : 0.0f;
     __syncthreads();
     if (warp == 0) {
         // first tile of every expert: exclusive scan of the tile counts, 32 experts at a time
@@ -879,26 +883,51 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 if (row >= rows) continue;
                 float gl[E];
 #pragma unroll
-                for (int i = 0; i < E; ++i)
-                    gl[i] = __uint_as_float(v[i]) + (p.bias2 ? __bfloat162float(__ldg(p.bias2 + i)) : 0.0f);
+                for (int i = 0; i < E; i += 4) {
+                    const float4 b = *reinterpret_cast<const float4*>(sh.bias2_f32 + i);   // same address for the whole warp
+                    gl[i] = __uint_as_float(v[i]) + b.x;
+                    gl[i + 1] = __uint_as_float(v[i + 1]) + b.y;
+                    gl[i + 2] = __uint_as_float(v[i + 2]) + b.z;
+                    gl[i + 3] = __uint_as_float(v[i + 3]) + b.w;
+                }
                 const int n = row0 + row;
-                // top-k by repeated arg-max over the logits; ties go to the lower id
-                unsigned long long taken = 0ull;
-                float m = 0.0f;
+                // top-k over the logits; ties go to the lower id
+                float m;
                 int sel[8];
                 float gsel[8];
-                for (int j = 0; j < p.k; ++j) {
-                    int best = -1;
-                    float bv = 0.0f;
+                if (p.k <= 2) {
+                    // one pass keeping the best two (strict comparisons in ascending id order give the
+                    // same picks as repeated arg-max)
+                    float b1 = gl[0], b2 = -INFINITY;
+                    int i1 = 0, i2 = 0;
 #pragma unroll
-                    for (int i = 0; i < E; ++i) {
-                        const bool free_i = !((taken >> i) & 1ull);
-                        if (free_i && (best < 0 || gl[i] > bv)) { best = i; bv = gl[i]; }
+                    for (int i = 1; i < E; ++i) {
+                        const float g = gl[i];
+                        const bool gt1 = g > b1, gt2 = g > b2;
+                        b2 = gt1 ? b1 : (gt2 ? g : b2);
+                        i2 = gt1 ? i1 : (gt2 ? i : i2);
+                        b1 = gt1 ? g : b1;
+                        i1 = gt1 ? i : i1;
                     }
-                    taken |= 1ull << best;
-                    sel[j] = best;
-                    gsel[j] = bv;
-                    if (j == 0) m = bv;
+                    sel[0] = i1; gsel[0] = b1; sel[1] = i2; gsel[1] = b2;
+                    m = b1;
+                } else {
+                    // repeated arg-max
+                    unsigned long long taken = 0ull;
+                    m = 0.0f;
+                    for (int j = 0; j < p.k; ++j) {
+                        int best = -1;
+                        float bv = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < E; ++i) {
+                            const bool free_i = !((taken >> i) & 1ull);
+                            if (free_i && (best < 0 || gl[i] > bv)) { best = i; bv = gl[i]; }
+                        }
+                        taken |= 1ull << best;
+                        sel[j] = best;
+                        gsel[j] = bv;
+                        if (j == 0) m = bv;
+                    }
                 }
                 float sum = 0.0f;
 #pragma unroll

@@ -79,14 +79,14 @@ def assert_outputs_close(got, ref, dtype: str, what="h_out"):
 class GpuLayer:
     """Device tensors of one workload plus the calls through the C ABI."""
 
-    def __init__(self, lc: synth.LayerConfig, h_np, w_np, device="cuda"):
+    def __init__(self, lc: synth.LayerConfig, h_np, w_np, device="cuda", drop_zero_biases=False):
         import torch
         self.torch = torch
         self.lc = lc
         self.cfg = tensors.config_from_synth(lc)
         self.dev = device
         self.h = tensors.to_torch(h_np, lc.dtype, device)
-        self.w = tensors.weights_to_torch(w_np, lc.dtype, device)
+        self.w = tensors.weights_to_torch(w_np, lc.dtype, device, drop_zero_biases=drop_zero_biases)
         self.ws = binding.alloc_workspace(self.cfg, device)
         self.tdtype = binding.torch_dtype(self.cfg)
 

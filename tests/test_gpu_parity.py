@@ -27,6 +27,13 @@ SMALL = {
     "bf16_one_expert": LC("e1", T=20, d=128, S=2, E=1, k=1, F=256),
     "bf16_k_equals_E": LC("kE", T=20, d=128, S=2, E=2, k=2, F=256),
     "bf16_single_row": LC("one", T=1, d=64, S=1, E=16, k=2, F=256),
+    # more of the tensor-core set: weights that stream through the rings (more chunks than slots),
+    # ReLU experts, biases that are not zero, E = 64 at ds = 64, ds = 256 with k = 2
+    "bf16_streamed": LC("stream", T=300, d=256, S=2, E=16, k=2, F=1024, Hr=512),
+    "bf16_relu_biased": LC("relub", T=200, d=256, S=4, E=32, k=2, F=256, act=0, init="kaiming"),
+    "bf16_gelu_biased": LC("gelub", T=130, d=512, S=4, E=16, k=1, F=512, init="kaiming"),
+    "bf16_e64_ds64": LC("e64", T=260, d=128, S=2, E=64, k=2, F=128),
+    "bf16_ds256_k2": LC("w256", T=70, d=512, S=2, E=16, k=2, F=512, Hr=128),
 }
 
 
@@ -109,6 +116,21 @@ def test_expert_ffn_and_combine(name):
 def test_forward_small(name):
     rep = pu.check_forward_against_oracle(SMALL[name])
     print(name, rep)
+
+
+def test_forward_with_null_biases():
+    """Zero biases passed as NULL pointers take the no-bias code paths: same bits as with zero arrays."""
+    import torch
+    lc = SMALL["bf16_lm"]
+    h, w = inputs(lc)
+    with_arrays = pu.GpuLayer(lc, h, w).forward()
+    with_null = pu.GpuLayer(lc, h, w, drop_zero_biases=True)
+    assert all(with_null.w[b] is None for b in ("br1", "br2", "b1", "b2"))
+    got = with_null.forward()
+    torch.cuda.synchronize()
+    for a, b in zip(with_arrays, got):
+        assert torch.equal(a, b)
+    assert with_null.status() == 0
 
 
 def test_forward_equals_staged_calls_and_is_deterministic():

@@ -157,6 +157,12 @@ struct TcCfg {
     // (A and B of one MMA must have the same 16-bit format: fp16 hidden x bf16 weights is an
     // illegal instruction on sm_100a.)
     static constexpr int H_PARTS = ROUTER_ ? 2 : 1;
+    // How the two MMA-issuing warps run.  Router: all 32 lanes run the issue loop and one elected
+    // lane issues, so that descriptors and addresses stay in uniform registers (its 40 small MMAs per
+    // tile make it issue-bound: 153 -> 118 us on the largest workload).  Experts: one lane runs the
+    // loop; their tile waits for the activation warps, and the wider issue warps only take issue
+    // slots from those (258 -> 272 us with the router's scheme).
+    static constexpr bool UNIFORM_ISSUE = ROUTER_;
     static constexpr bool PACKED_ACT = !ROUTER_;
     // TMEM columns:
     //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w of the group that has the chunk
@@ -468,6 +474,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     if (threadIdx.x == 0) { Tracer tr1(5); tr1.n = 1; tr1(98); }   // set-up finished
 #endif
 
+    // result of a wait in an MMA-issuing warp: with all lanes in the loop they must leave it together
+    auto all_lanes_agree = [](bool r) { return C::UNIFORM_ISSUE ? (bool)__all_sync(0xffffffffu, r) : r; };
     if (warp == 0) {
         // ================= TMA producer =====================================================
         // One thread, per tile: the row tile (unless rows are gathered), then per chunk W1 (with its
@@ -540,11 +548,13 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         }
     } else if (warp == 1) {
         // ================= GEMM-1 issue ======================================================
-        if (lane == 0 && t_begin < t_end) {
+        // (UNIFORM_ISSUE: all lanes run the loop and one elected lane issues, see elect_one_sync;
+        // otherwise lane 0 alone)
+        if (t_begin < t_end && (C::UNIFORM_ISSUE || lane == 0)) {
             constexpr uint32_t idesc1 = make_idesc(128, C::HC, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
             bool ok = true;
-            TRACE_DECL(tr, 1);
+            TRACE_DECL(tr, lane == 0 ? 1 : 7);
             int e = 0, prev_e = -1;
             uint32_t g = 0, reloads = 0;
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
@@ -554,50 +564,59 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 prev_e = e;
                 const int ab = ta % C::A_BUFS;
                 TRACE(tr, 10);
-                if (!mbar_wait(bar(B::A_FULL + ab), (uint32_t)(ta / C::A_BUFS) & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                ok = all_lanes_agree(mbar_wait(bar(B::A_FULL + ab), (uint32_t)(ta / C::A_BUFS) & 1u, abort, kWaitLimitNs));
+                if (!ok) break;
                 TRACE(tr, 11);
                 if (gather) fence_proxy_async_smem();   // rows written by cp.async -> visible to the MMA's reads
                 for (int c = 0; c < nchunks; ++c, ++g) {
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
                     if (reload) {
                         const uint32_t n = resident ? reloads : g / C::W_STAGES;
-                        if (!mbar_wait(bar(B::W1_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                        ok = all_lanes_agree(mbar_wait(bar(B::W1_FULL + slot), n & 1u, abort, kWaitLimitNs));
+                        if (!ok) break;
                     }
                     const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
                     TRACE(tr, 12);
-                    if (!mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    ok = all_lanes_agree(mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs));
+                    if (!ok) break;
                     TRACE(tr, 13);
                     tc_fence_after_sync();
                     const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W1C_BYTES) >> 4);
                     const uint32_t d = tmem_base + b * C::HC;
-                    mma_ss<0>(d, a0, w0, idesc1);
+                    if (!C::UNIFORM_ISSUE || elect_one_sync()) {
+                        mma_ss<0>(d, a0, w0, idesc1);
 #pragma unroll
-                    for (int kk = 1; kk < C::K1 / 16; ++kk)
-                        mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
-                                  w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
-                    mma_commit(bar(B::ACC1_FULL + b));
-                    // streamed weights: the W1 slot is free as soon as these MMAs have read it
-                    // (resident weights are handed back by the GEMM-2 thread at an expert change)
-                    if (!resident) mma_commit(bar(B::W1_EMPTY + slot));
-                    if (c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
+                        for (int kk = 1; kk < C::K1 / 16; ++kk)
+                            mma_ss<1>(d, a0 + (((kk >> 2) * C::A_PANEL + (kk & 3) * 32) >> 4),
+                                      w0 + (((kk >> 2) * C::W1_PANEL + (kk & 3) * 32) >> 4), idesc1);
+                        mma_commit(bar(B::ACC1_FULL + b));
+                        // streamed weights: the W1 slot is free as soon as these MMAs have read it
+                        // (resident weights are handed back by the GEMM-2 warp at an expert change)
+                        if (!resident) mma_commit(bar(B::W1_EMPTY + slot));
+                        if (c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
+                    }
+                    if (C::UNIFORM_ISSUE) __syncwarp();
                     TRACE(tr, 14);
                 }
                 if (reload) ++reloads;
             }
             if (!ok || *abort) {
-                // make sure no MMA of this thread is still running before TMEM is released
+                // make sure no MMA of this warp is still running before TMEM is released
                 volatile int never = 0;
-                mma_commit(bar(B::DRAIN));
-                mbar_wait(bar(B::DRAIN), 0u, &never, 10000000ull);
+                if (lane == 0) {
+                    mma_commit(bar(B::DRAIN));
+                    mbar_wait(bar(B::DRAIN), 0u, &never, 10000000ull);
+                }
+                if (C::UNIFORM_ISSUE) __syncwarp();
             }
         }
     } else if (warp == 2) {
         // ================= GEMM-2 issue ======================================================
-        if (lane == 0 && t_begin < t_end) {
+        if (t_begin < t_end && (C::UNIFORM_ISSUE || lane == 0)) {
             constexpr uint32_t idesc2 = make_idesc(128, C::N2, kFmtBF16, kFmtBF16);
             const uint32_t dW = desc_lo_sw128(smem_base + C::OFF_W2);
             bool ok = true;
-            TRACE_DECL(tr, 4);
+            TRACE_DECL(tr, lane == 0 ? 4 : 7);
             int e = 0, prev_e = -1;
             uint32_t g = 0, reloads = 0;
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
@@ -617,47 +636,58 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
                     if (reload) {
                         const uint32_t n = resident ? reloads : g / C::W_STAGES;
-                        if (!mbar_wait(bar(B::W2_FULL + slot), n & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                        ok = all_lanes_agree(mbar_wait(bar(B::W2_FULL + slot), n & 1u, abort, kWaitLimitNs));
+                        if (!ok) break;
                     }
                     const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
                     TRACE(tr, 20);
-                    if (!mbar_wait(bar(B::H_FULL + b), n1 & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    ok = all_lanes_agree(mbar_wait(bar(B::H_FULL + b), n1 & 1u, abort, kWaitLimitNs));
+                    if (!ok) break;
                     TRACE(tr, 21);
-                    if (c == 0 && !mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(ta / C::ACC2_BUFS) & 1u) ^ 1u,
-                                             abort, kWaitLimitNs)) { ok = false; break; }
+                    if (c == 0) {
+                        ok = all_lanes_agree(mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(ta / C::ACC2_BUFS) & 1u) ^ 1u,
+                                                               abort, kWaitLimitNs));
+                        if (!ok) break;
+                    }
                     tc_fence_after_sync();
                     const uint32_t w0 = dW + ((slot * C::W2C_BYTES) >> 4);
                     const uint32_t d = tmem_base + C::ACC2_COL0 + buf * C::N2;
                     const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: chunk; router: lo half
                     const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi half, two runs
+                    if (!C::UNIFORM_ISSUE || elect_one_sync()) {
 #pragma unroll
-                    for (int part = 0; part < C::H_PARTS; ++part) {
+                        for (int part = 0; part < C::H_PARTS; ++part) {
 #pragma unroll
-                        for (int kk = 0; kk < C::HC / 16; ++kk) {
-                            uint32_t a;
-                            if (C::ROUTER && part == 0)
-                                a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / C::GWG) + (kk % C::KSTEPS_PER_WG) * 8;
-                            else
-                                a = hbuf + kk * 8;
-                            const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
-                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, c > 0 ? 1u : 0u);
-                            else mma_ts<1>(d, a, bd, idesc2);
+                            for (int kk = 0; kk < C::HC / 16; ++kk) {
+                                uint32_t a;
+                                if (C::ROUTER && part == 0)
+                                    a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / C::GWG) + (kk % C::KSTEPS_PER_WG) * 8;
+                                else
+                                    a = hbuf + kk * 8;
+                                const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
+                                if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, c > 0 ? 1u : 0u);
+                                else mma_ts<1>(d, a, bd, idesc2);
+                            }
                         }
+                        mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
+                        if (release) {
+                            mma_commit(bar(B::W2_EMPTY + slot));
+                            if (resident) mma_commit(bar(B::W1_EMPTY + slot));   // GEMM-1 of this chunk finished before its GEMM-2 began
+                        }
+                        if (c == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
                     }
-                    mma_commit(bar((C::ROUTER ? B::ACC1_EMPTY : B::H_EMPTY) + b));
-                    if (release) {
-                        mma_commit(bar(B::W2_EMPTY + slot));
-                        if (resident) mma_commit(bar(B::W1_EMPTY + slot));   // GEMM-1 of this chunk finished before its GEMM-2 began
-                    }
-                    if (c == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
+                    if (C::UNIFORM_ISSUE) __syncwarp();
                     TRACE(tr, 22);
                 }
                 if (reload) ++reloads;
             }
             if (!ok || *abort) {
                 volatile int never = 0;
-                mma_commit(bar(B::DRAIN + 1));
-                mbar_wait(bar(B::DRAIN + 1), 0u, &never, 10000000ull);
+                if (lane == 0) {
+                    mma_commit(bar(B::DRAIN + 1));
+                    mbar_wait(bar(B::DRAIN + 1), 0u, &never, 10000000ull);
+                }
+                if (C::UNIFORM_ISSUE) __syncwarp();
             }
         }
     } else if (warp == 3) {

@@ -79,6 +79,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// One lane of the (converged) warp.  The MMA-issuing warps run their loops with all 32 lanes and
+// elect a lane only around the tcgen05 instructions: the descriptors and addresses are then computed
+// under warp-uniform control flow, where the compiler keeps them in uniform registers, instead of
+// inside an `if (lane == 0)` region, where every operand of every MMA is moved from a vector
+// register to a uniform one first (traced: ~140 cycles per issued MMA that way).
+__device__ __forceinline__ bool elect_one_sync() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // ---- proxies and tcgen05 fences ---------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -145,7 +145,10 @@ struct TcCfg {
     static constexpr int NGRP = (K1 == 256) ? 1 : (FOUR_GROUPS ? 4 : 2);
     static constexpr int GWG = FOUR_GROUPS ? 1 : 2;
     static constexpr int NWG = NGRP * GWG;
-    static constexpr int NBUF = FOUR_GROUPS ? 4 : 2;            // GEMM-1 accumulator / hidden buffers
+    // GEMM-1 accumulator / hidden buffers.  The router's hidden pair lives inside the accumulator it
+    // came from (see the TMEM map), which leaves room for a third accumulator: GEMM-1 of the next two
+    // chunks can then be issued while GEMM-2 still reads this one.
+    static constexpr int NBUF = ROUTER_ ? 3 : (FOUR_GROUPS ? 4 : 2);
     static constexpr int GRP_WARPS = GWG * 4;                   // warps that work on one chunk
     static constexpr int THREADS = 128 + NWG * 128 + 128;
     static constexpr int OUT_WARP0 = 4 + NWG * 4;               // first warp of the output warpgroup
@@ -165,17 +168,16 @@ struct TcCfg {
     static constexpr bool UNIFORM_ISSUE = ROUTER_;
     static constexpr bool PACKED_ACT = !ROUTER_;
     // TMEM columns:
-    //   [0, 2 HC)            two GEMM-1 accumulators.  Warpgroup w of the group that has the chunk
-    //                        owns columns [w HC/GWG, (w+1) HC/GWG).  Router: once a thread has
-    //                        read a 16-column piece it writes the piece's hi half (8 packed
-    //                        columns) over the start of its own column range, so the chunk's hi
-    //                        half ends up in GWG runs of HC/(2 GWG) columns.
-    //   [2 HC, 3 HC)         two hidden buffers of HC/2 packed columns: the experts' hidden chunk
-    //                        (so GEMM-1 of a later chunk need not wait for GEMM-2), or the
-    //                        router's lo half.
-    //   [3 HC, ...)          ACC2_BUFS final accumulators of N2 columns.
+    //   [0, NBUF HC)         GEMM-1 accumulators.  Warpgroup w of the group that has the chunk owns
+    //                        columns [w HC/GWG, (w+1) HC/GWG).  Router: once a thread has read a
+    //                        16-column piece (= one K step of GEMM-2) it writes the piece's hi half
+    //                        into the piece's first 8 columns and the lo half into its last 8, so
+    //                        K step kk of the hidden chunk is at columns 16 kk (hi) and 16 kk + 8 (lo).
+    //   then (experts only)  NBUF hidden buffers of HC/2 packed columns (so GEMM-1 of a later chunk
+    //                        need not wait for GEMM-2).
+    //   then                 ACC2_BUFS final accumulators of N2 columns.
     static constexpr int H_COL0 = NBUF * HC;
-    static constexpr int ACC2_COL0 = H_COL0 + NBUF * (HC / 2);
+    static constexpr int ACC2_COL0 = H_COL0 + (ROUTER_ ? 0 : NBUF * (HC / 2));
     static constexpr int TMEM_COLS = pow2_at_least(ACC2_COL0 + ACC2_BUFS * N2);
     static constexpr int KSTEPS_PER_WG = HC / (16 * GWG);       // 16-element K steps in one warpgroup's columns
     static constexpr int KP1 = K1 / 64;                         // 64-wide K panels of GEMM-1
@@ -203,7 +205,7 @@ struct TcCfg {
     static constexpr int PIECE = 16;                            // accumulator columns per piece
     static constexpr int NPIECE = HC / (PIECE * GWG);           // pieces per thread and chunk
     static constexpr int SUB = (NPIECE > 2) ? 2 : NPIECE;       // pieces held in registers at once (experts)
-    static_assert(NBUF % NGRP == 0 && NPIECE % SUB == 0, "chunk-to-group and piece-to-batch maps");
+    static_assert(NPIECE % SUB == 0, "piece-to-batch map");
     static_assert(NPIECE >= 1, "hidden chunk too narrow for the activation warpgroups");
     static_assert(W2C_BYTES % 1024 == 0 && W1C_BYTES % 1024 == 0, "operand tiles must stay 1024-byte aligned");
     static_assert(kBiasRing >= 2 * W_STAGES, "bias ring");
@@ -652,16 +654,16 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     tc_fence_after_sync();
                     const uint32_t w0 = dW + ((slot * C::W2C_BYTES) >> 4);
                     const uint32_t d = tmem_base + C::ACC2_COL0 + buf * C::N2;
-                    const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: chunk; router: lo half
-                    const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi half, two runs
+                    const uint32_t hbuf = tmem_base + C::H_COL0 + b * (C::HC / 2);   // experts: the hidden chunk
+                    const uint32_t hacc = tmem_base + b * C::HC;                     // router: hi / lo inside the accumulator
                     if (!C::UNIFORM_ISSUE || elect_one_sync()) {
 #pragma unroll
                         for (int part = 0; part < C::H_PARTS; ++part) {
 #pragma unroll
                             for (int kk = 0; kk < C::HC / 16; ++kk) {
                                 uint32_t a;
-                                if (C::ROUTER && part == 0)
-                                    a = hacc + (kk / C::KSTEPS_PER_WG) * (C::HC / C::GWG) + (kk % C::KSTEPS_PER_WG) * 8;
+                                if (C::ROUTER)
+                                    a = hacc + kk * 16 + part * 8;
                                 else
                                     a = hbuf + kk * 8;
                                 const uint32_t bd = w0 + (((kk >> 2) * C::W2_PANEL + (kk & 3) * 32) >> 4);
@@ -865,8 +867,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         if (pc + 1 < C::NPIECE) tmem_ld_x16(acc1 + (pc + 1) * C::PIECE, v[(pc + 1) & 1]);   // overlaps the math below
                         uint32_t hi[C::PIECE / 2], lo[C::PIECE / 2];
                         bias_relu_split_piece(cur, sh.bias1_f32 + c * C::HC + w * WCOLS + pc * C::PIECE, hi, lo);
-                        tmem_st_x8(acc1 + pc * (C::PIECE / 2), hi);     // over columns this thread has already read
-                        tmem_st_x8(hdst + pc * (C::PIECE / 2), lo);
+                        tmem_st_x8(acc1 + pc * C::PIECE, hi);                    // over the piece just read
+                        tmem_st_x8(acc1 + pc * C::PIECE + C::PIECE / 2, lo);
                     }
                 }
                 if (!ok) break;

@@ -162,10 +162,11 @@ struct TcCfg {
     static constexpr int H_PARTS = ROUTER_ ? 2 : 1;
     // How the two MMA-issuing warps run.  Router: all 32 lanes run the issue loop and one elected
     // lane issues, so that descriptors and addresses stay in uniform registers (its 40 small MMAs per
-    // tile make it issue-bound: 153 -> 118 us on the largest workload).  Experts: one lane runs the
-    // loop; their tile waits for the activation warps, and the wider issue warps only take issue
-    // slots from those (258 -> 272 us with the router's scheme).
-    static constexpr bool UNIFORM_ISSUE = ROUTER_;
+    // tile make it issue-bound: 153 -> 118 us on the largest workload), and so do the experts of
+    // 256-wide rows (16 MMAs per chunk: 180 -> 176 us).  The other experts: one lane runs the loop;
+    // their tile waits for the activation warps, and the wider issue warps only take issue slots from
+    // those (64-wide rows: 260 -> 272 us with the router's scheme; 128-wide: no difference).
+    static constexpr bool UNIFORM_ISSUE = ROUTER_ || K1 == 256;
     static constexpr bool PACKED_ACT = !ROUTER_;
     // TMEM columns:
     //   [0, NBUF HC)         GEMM-1 accumulators.  Warpgroup w of the group that has the chunk owns

@@ -154,10 +154,11 @@ template <class RC, class EC>
 int launch_fused(const Dims& D, const slicemoe_weights& w, const void* h, const FusedParams& fp, cudaStream_t st) {
     CUtensorMap tmX, tmWr1, tmWr2, tmW1, tmW2;
     int rc;
-    if ((rc = make_tmap(&tmX, h, (uint64_t)D.N, RC::K1, 128))) return rc;
-    if ((rc = make_tmap(&tmWr1, w.Wr1, (uint64_t)D.Hr, RC::K1, RC::HC))) return rc;
+    // (rows narrower than K1 are zero-filled by the copies: the box reaches past the tensor's edge)
+    if ((rc = make_tmap(&tmX, h, (uint64_t)D.N, (uint64_t)D.ds, 128))) return rc;
+    if ((rc = make_tmap(&tmWr1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, RC::HC))) return rc;
     if ((rc = make_tmap(&tmWr2, w.Wr2, (uint64_t)RC::N2, D.Hr, RC::N2))) return rc;
-    if ((rc = make_tmap(&tmW1, w.W1, (uint64_t)D.E * D.F, EC::K1, EC::HC))) return rc;
+    if ((rc = make_tmap(&tmW1, w.W1, (uint64_t)D.E * D.F, (uint64_t)D.ds, EC::HC))) return rc;
     if ((rc = make_tmap(&tmW2, w.W2, (uint64_t)D.E * EC::N2, D.F, EC::N2))) return rc;
     const int grid = sm_count();
     size_t smem = RC::SMEM_ALLOC > EC::SMEM_ALLOC ? RC::SMEM_ALLOC : EC::SMEM_ALLOC;
@@ -188,20 +189,21 @@ int launch_fused(const Dims& D, const slicemoe_weights& w, const void* h, const 
     return SLICEMOE_OK;
 }
 
-template <int K1, int E>
+template <int K1, int E, int N2>
 int launch_fused_k1e(const Dims& D, const slicemoe_weights& w, const void* h, const FusedParams& fp, cudaStream_t st) {
     using RC = TcCfg<K1, E, true, SLICEMOE_ACT_RELU>;
     if (D.act == SLICEMOE_ACT_GELU_TANH)
-        return launch_fused<RC, TcCfg<K1, K1, false, SLICEMOE_ACT_GELU_TANH>>(D, w, h, fp, st);
-    return launch_fused<RC, TcCfg<K1, K1, false, SLICEMOE_ACT_RELU>>(D, w, h, fp, st);
+        return launch_fused<RC, TcCfg<K1, N2, false, SLICEMOE_ACT_GELU_TANH>>(D, w, h, fp, st);
+    return launch_fused<RC, TcCfg<K1, N2, false, SLICEMOE_ACT_RELU>>(D, w, h, fp, st);
 }
 
-template <int K1>
+// K1: the width the kernels are built for; N2: the real slice width (= the second expert GEMM's N)
+template <int K1, int N2 = K1>
 int launch_fused_k1(const Dims& D, const slicemoe_weights& w, const void* h, const FusedParams& fp, cudaStream_t st) {
     switch (D.E) {
-        case 16: return launch_fused_k1e<K1, 16>(D, w, h, fp, st);
-        case 32: return launch_fused_k1e<K1, 32>(D, w, h, fp, st);
-        case 64: return launch_fused_k1e<K1, 64>(D, w, h, fp, st);
+        case 16: return launch_fused_k1e<K1, 16, N2>(D, w, h, fp, st);
+        case 32: return launch_fused_k1e<K1, 32, N2>(D, w, h, fp, st);
+        case 64: return launch_fused_k1e<K1, 64, N2>(D, w, h, fp, st);
         default: return SLICEMOE_ERR_UNSUPPORTED;
     }
 }
@@ -283,8 +285,11 @@ int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h
 
     fp.R = (int)D.R; fp.E = D.E; fp.pairs_per_chunk = rows_per_cta * D.k; fp.capacity = (int)D.capacity;
     fp.assigned = assigned; fp.kept = kept; fp.offsets = offsets; fp.dest = dest; fp.perm = perm; fp.gate = gate;
+    r.row_elems = D.ds;
+    f.row_elems = D.ds;
     switch (D.ds) {
         case 64: return launch_fused_k1<64>(D, w, h, fp, st);
+        case 96: return launch_fused_k1<128, 96>(D, w, h, fp, st);
         case 128: return launch_fused_k1<128>(D, w, h, fp, st);
         case 256: return launch_fused_k1<256>(D, w, h, fp, st);
         default: return SLICEMOE_ERR_UNSUPPORTED;

@@ -28,8 +28,9 @@ int launch_tc(const void* A, uint64_t a_rows, const void* W1, const void* W2, in
               int max_tiles, cudaStream_t st) {
     CUtensorMap tmA, tmW1, tmW2;
     int rc;
-    if ((rc = make_tmap(&tmA, A, a_rows, C::K1, 128))) return rc;
-    if ((rc = make_tmap(&tmW1, W1, (uint64_t)n_experts * p.HID, C::K1, C::HC))) return rc;
+    // (a row narrower than K1 is zero-filled by the copies: the box reaches past the tensor's edge)
+    if ((rc = make_tmap(&tmA, A, a_rows, (uint64_t)p.row_elems, 128))) return rc;
+    if ((rc = make_tmap(&tmW1, W1, (uint64_t)n_experts * p.HID, (uint64_t)p.row_elems, C::HC))) return rc;
     if ((rc = make_tmap(&tmW2, W2, (uint64_t)n_experts * C::N2, p.HID, C::N2))) return rc;
     auto kern = tc_mlp_kernel<C>;
     static bool attr_set = false;
@@ -43,9 +44,9 @@ int launch_tc(const void* A, uint64_t a_rows, const void* W1, const void* W2, in
     return SLICEMOE_OK;
 }
 
-template <int K1, int ACT>
+template <int K1, int ACT, int N2 = K1>
 int launch_ffn_k1(const Dims& D, const slicemoe_weights& w, const void* xperm, const TcParams& p, cudaStream_t st) {
-    using C = TcCfg<K1, K1, false, ACT>;
+    using C = TcCfg<K1, N2, false, ACT>;
     return launch_tc<C>(xperm, (uint64_t)(p.gather_src ? D.N : D.R), w.W1, w.W2, D.E, p, max_tiles(D), st);
 }
 
@@ -76,9 +77,14 @@ extern "C" int slicemoe_debug_set_trace(void* device_buf) {
 }
 #endif
 
+// Slice widths the tensor-core pipeline is built for.  The paper's own model (d = 768, S = 8) has
+// ds = 96: it runs on the 128-wide instantiation, the copies zero-filling columns 96..127 of the row
+// and weight tiles (a quarter of GEMM-1's MMA work multiplies zeros), with a 96-wide second GEMM.
+static bool tc_width_supported(int ds) { return ds == 64 || ds == 96 || ds == 128 || ds == 256; }
+
 bool tc_route_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
-    if (D.ds != 64 && D.ds != 128 && D.ds != 256) return false;
+    if (!tc_width_supported(D.ds)) return false;
     if (D.E != 16 && D.E != 32 && D.E != 64) return false;
     const int hc = D.ds == 64 ? 128 : 64;
     // at least two hidden chunks: GEMM-1 is issued ahead of GEMM-2, and with resident weights that
@@ -88,7 +94,7 @@ bool tc_route_supported(const Dims& D) {
 
 bool tc_ffn_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
-    if (D.ds != 64 && D.ds != 128 && D.ds != 256) return false;
+    if (!tc_width_supported(D.ds)) return false;
     const int hc = 64;
     return D.F % hc == 0 && D.F >= 2 * hc && D.F <= kMaxHid;
 }
@@ -111,8 +117,10 @@ int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int
     p.topk_idx = topk_idx; p.topk_p = topk_p; p.assigned = assigned; p.cta_hist = cta_hist; p.probs = probs_opt; p.k = D.k;
     p.status = status;
     p.zero_out = (bf16*)zero_out; p.zero_cols = D.ds;
+    p.row_elems = D.ds;
     switch (D.ds) {
         case 64: return launch_route_k1<64>(D, w, h, p, st);
+        case 96:
         case 128: return launch_route_k1<128>(D, w, h, p, st);
         case 256: return launch_route_k1<256>(D, w, h, p, st);
         default: return SLICEMOE_ERR_UNSUPPORTED;
@@ -130,7 +138,11 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
     p.gather_src = (const bf16*)gather_h; p.perm = perm; p.gate = gate; p.gather_k = D.k;
     p.scatter_out = gather_h ? (bf16*)scatter_out : nullptr;
     if (gather_h) xperm = gather_h;   // the A tensor map is not used in gather mode; any valid matrix will do
+    p.row_elems = D.ds;
     const bool gelu = D.act == SLICEMOE_ACT_GELU_TANH;
+    if (D.ds == 96)
+        return gelu ? launch_ffn_k1<128, SLICEMOE_ACT_GELU_TANH, 96>(D, w, xperm, p, st)
+                    : launch_ffn_k1<128, SLICEMOE_ACT_RELU, 96>(D, w, xperm, p, st);
     if (D.ds == 64)
         return gelu ? launch_ffn_k1<64, SLICEMOE_ACT_GELU_TANH>(D, w, xperm, p, st)
                     : launch_ffn_k1<64, SLICEMOE_ACT_RELU>(D, w, xperm, p, st);

@@ -58,6 +58,8 @@ constexpr int kMaxBars = 48;
 constexpr int kBiasRing = 8;
 
 struct TcParams {
+    int row_elems;            // elements per row of X (= ds); at most the K1 the kernel is built for: a narrower
+                              // row (the paper's own ds = 96 under K1 = 128) is zero-filled up to K1
     const int32_t* offsets;   // experts: [E+1] device row ranges; router: nullptr
     int n_rows;               // router: N; experts: R (length of the stacked-row arrays)
     int E;                    // experts: E; router: 1
@@ -754,9 +756,11 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         const int r32 = i * RPI + rsub;                 // row within this block of 32
                         const int r = q * 32 + r32;
                         const int n = __shfl_sync(0xffffffffu, nrow[q], r32);
-                        const bf16* src = p.gather_src + (size_t)(n < 0 ? 0 : n) * C::K1 + ch * 8;
+                        // (rows past the tile's end and chunks past the row's real width are zero-filled)
+                        const bool real = n >= 0 && ch * 8 < p.row_elems;
+                        const bf16* src = p.gather_src + (real ? (size_t)n * p.row_elems + ch * 8 : 0);
                         cp_async_16(dst0 + (r >> 3) * 1024 + (r & 7) * 128 + (((ch & 7) ^ (r & 7)) << 4), src,
-                                    n < 0 ? 0u : 16u);
+                                    real ? 16u : 0u);
                     }
                 }
                 {
@@ -979,8 +983,9 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                                                  __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
                 }
             } else {
-                // 64 output columns at a time: accumulator -> registers -> bias -> bf16 -> global
-                constexpr int OB = 64;
+                // OB output columns at a time: accumulator -> registers -> bias -> bf16 -> global
+                constexpr int OB = (C::N2 % 64 == 0) ? 64 : 32;
+                static_assert(C::N2 % OB == 0, "output width");
                 const bool scatter = gather && p.scatter_out != nullptr;
                 const bool live = row < rows;
                 bf16* dst = nullptr;

@@ -307,6 +307,21 @@ def test_forward_full_cfg3_capacity():
         print(name, rep)
 
 
+def test_forward_paper_model_shape():
+    """The paper's own layer (d = 768, S = 8: 96-wide slices, E = 16, k = 2, F = 4 ds) at a batch of a
+    few thousand tokens: runs on the 128-wide tensor-core instantiation with zero-filled columns."""
+    lc = LC("paper768", T=3000, d=768, S=8, E=16, k=2, F=384)
+    rep = pu.check_forward_against_oracle(lc, sample_rows=4096)
+    print("paper768", rep)
+    import torch
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    before = binding.slicemoe_launch_count()
+    gpu.forward()
+    torch.cuda.synchronize()
+    assert binding.slicemoe_launch_count() - before == 1          # the single-kernel path, not the CUDA-core one
+
+
 def test_forward_full_cfg2_sampled_rows():
     rep = pu.check_forward_against_oracle(C["cfg2"], sample_rows=8192)
     print("cfg2", rep)

@@ -288,9 +288,11 @@ int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h
     r.row_elems = D.ds;
     f.row_elems = D.ds;
     switch (D.ds) {
+        case 48: return launch_fused_k1<64, 48>(D, w, h, fp, st);
         case 64: return launch_fused_k1<64>(D, w, h, fp, st);
         case 96: return launch_fused_k1<128, 96>(D, w, h, fp, st);
         case 128: return launch_fused_k1<128>(D, w, h, fp, st);
+        case 192: return launch_fused_k1<256, 192>(D, w, h, fp, st);
         case 256: return launch_fused_k1<256>(D, w, h, fp, st);
         default: return SLICEMOE_ERR_UNSUPPORTED;
     }

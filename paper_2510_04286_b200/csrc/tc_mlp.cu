@@ -80,13 +80,16 @@ extern "C" int slicemoe_debug_set_trace(void* device_buf) {
 // Slice widths the tensor-core pipeline is built for.  The paper's own model (d = 768, S = 8) has
 // ds = 96: it runs on the 128-wide instantiation, the copies zero-filling columns 96..127 of the row
 // and weight tiles (a quarter of GEMM-1's MMA work multiplies zeros), with a 96-wide second GEMM.
-static bool tc_width_supported(int ds) { return ds == 64 || ds == 96 || ds == 128 || ds == 256; }
+// Likewise its S = 16 and S = 4 variants: ds = 48 under 64, ds = 192 under 256.
+static bool tc_width_supported(int ds) {
+    return ds == 48 || ds == 64 || ds == 96 || ds == 128 || ds == 192 || ds == 256;
+}
 
 bool tc_route_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
     if (!tc_width_supported(D.ds)) return false;
     if (D.E != 16 && D.E != 32 && D.E != 64) return false;
-    const int hc = D.ds == 64 ? 128 : 64;
+    const int hc = D.ds <= 64 ? 128 : 64;
     // at least two hidden chunks: GEMM-1 is issued ahead of GEMM-2, and with resident weights that
     // look-ahead must not need the weight slot that the chunk in flight is still using
     return D.Hr % hc == 0 && D.Hr >= 2 * hc && D.Hr <= kMaxHid && D.k <= 8;
@@ -119,9 +122,11 @@ int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int
     p.zero_out = (bf16*)zero_out; p.zero_cols = D.ds;
     p.row_elems = D.ds;
     switch (D.ds) {
+        case 48:
         case 64: return launch_route_k1<64>(D, w, h, p, st);
         case 96:
         case 128: return launch_route_k1<128>(D, w, h, p, st);
+        case 192:
         case 256: return launch_route_k1<256>(D, w, h, p, st);
         default: return SLICEMOE_ERR_UNSUPPORTED;
     }
@@ -140,9 +145,15 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
     if (gather_h) xperm = gather_h;   // the A tensor map is not used in gather mode; any valid matrix will do
     p.row_elems = D.ds;
     const bool gelu = D.act == SLICEMOE_ACT_GELU_TANH;
+    if (D.ds == 48)
+        return gelu ? launch_ffn_k1<64, SLICEMOE_ACT_GELU_TANH, 48>(D, w, xperm, p, st)
+                    : launch_ffn_k1<64, SLICEMOE_ACT_RELU, 48>(D, w, xperm, p, st);
     if (D.ds == 96)
         return gelu ? launch_ffn_k1<128, SLICEMOE_ACT_GELU_TANH, 96>(D, w, xperm, p, st)
                     : launch_ffn_k1<128, SLICEMOE_ACT_RELU, 96>(D, w, xperm, p, st);
+    if (D.ds == 192)
+        return gelu ? launch_ffn_k1<256, SLICEMOE_ACT_GELU_TANH, 192>(D, w, xperm, p, st)
+                    : launch_ffn_k1<256, SLICEMOE_ACT_RELU, 192>(D, w, xperm, p, st);
     if (D.ds == 64)
         return gelu ? launch_ffn_k1<64, SLICEMOE_ACT_GELU_TANH>(D, w, xperm, p, st)
                     : launch_ffn_k1<64, SLICEMOE_ACT_RELU>(D, w, xperm, p, st);

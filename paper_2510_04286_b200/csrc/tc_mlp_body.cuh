@@ -984,7 +984,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 }
             } else {
                 // OB output columns at a time: accumulator -> registers -> bias -> bf16 -> global
-                constexpr int OB = (C::N2 % 64 == 0) ? 64 : 32;
+                constexpr int OB = (C::N2 % 64 == 0) ? 64 : (C::N2 % 32 == 0) ? 32 : 16;
                 static_assert(C::N2 % OB == 0, "output width");
                 const bool scatter = gather && p.scatter_out != nullptr;
                 const bool live = row < rows;

@@ -34,6 +34,9 @@ SMALL = {
     "bf16_gelu_biased": LC("gelub", T=130, d=512, S=4, E=16, k=1, F=512, init="kaiming"),
     "bf16_e64_ds64": LC("e64", T=260, d=128, S=2, E=64, k=2, F=128),
     "bf16_ds256_k2": LC("w256", T=70, d=512, S=2, E=16, k=2, F=512, Hr=128),
+    # the paper's d = 768 at S = 16 and S = 4: 48- and 192-wide slices on zero-filled 64 / 256-wide tiles
+    "bf16_paper_slice48": LC("s48", T=50, d=768, S=16, E=16, k=2, F=192),
+    "bf16_paper_slice192": LC("s192", T=60, d=768, S=4, E=16, k=2, F=768),
 }
 
 
@@ -228,7 +231,8 @@ def test_profiled_forward_records_stage_times():
     assert torch.equal(h_out, gpu.forward()[0])
 
 
-@pytest.mark.parametrize("name", ["bf16_lm", "bf16_skew_cap", "bf16_decode", "bf16_single_row", "bf16_k3", "f32_cfg0"])
+@pytest.mark.parametrize("name", ["bf16_lm", "bf16_skew_cap", "bf16_decode", "bf16_single_row", "bf16_k3", "f32_cfg0",
+                                  "bf16_paper_slice96", "bf16_paper_slice48", "bf16_paper_slice192"])
 def test_forward_launch_count_and_status(name):
     """Supported bf16 shapes with k <= 2 run the whole forward as one launch; the others one
     launch per step.  Either way the status word stays clear and repeated calls on two
@@ -244,7 +248,7 @@ def test_forward_launch_count_and_status(name):
     launches = binding.slicemoe_launch_count() - before
     other = gpu2.forward()
     torch.cuda.synchronize()
-    one_launch = lc.dtype == "bf16" and lc.k <= 2 and lc.ds in (64, 128, 256) and lc.E in (16, 32, 64)
+    one_launch = lc.dtype == "bf16" and lc.k <= 2 and lc.ds in (48, 64, 96, 128, 192, 256) and lc.E in (16, 32, 64)
     assert launches == 1 if one_launch else launches >= 3
     assert gpu.status() == 0 and gpu2.status() == 0
     for a, b, c in zip(first, again, other):

@@ -95,6 +95,11 @@ CONFIGS = {
     # The paper's own model (Section 4): d = 768, S = 8 (96-wide slices), E = 16, k = 2; the expert
     # width F = 4 ds follows the other workloads, the batch is 32 sequences of 512 tokens.
     "paper768": LayerConfig("paper768", T=16384, d=768, S=8, E=16, k=2, F=384),
+    # the shapes of the paper's slice-count and top-k ablations (Table 2, Table 4) on the same model
+    "paper768_S4": LayerConfig("paper768_S4", T=16384, d=768, S=4, E=16, k=2, F=768),
+    "paper768_S16": LayerConfig("paper768_S16", T=16384, d=768, S=16, E=16, k=2, F=192),
+    "paper768_k1": LayerConfig("paper768_k1", T=16384, d=768, S=8, E=16, k=1, F=384),
+    "paper768_k3": LayerConfig("paper768_k3", T=16384, d=768, S=8, E=16, k=3, F=384),
 }
 
 

@@ -35,6 +35,8 @@ SMALL = {
     "bf16_e64_ds64": LC("e64", T=260, d=128, S=2, E=64, k=2, F=128),
     "bf16_ds256_k2": LC("w256", T=70, d=512, S=2, E=16, k=2, F=512, Hr=128),
     # the paper's d = 768 at S = 16 and S = 4: 48- and 192-wide slices on zero-filled 64 / 256-wide tiles
+    # k = 3 (the paper's Table 4) on the tensor-core kernels: stacked outputs + combine kernel
+    "bf16_k3_tc": LC("k3tc", T=200, d=512, S=8, E=16, k=3, F=256),
     "bf16_paper_slice48": LC("s48", T=50, d=768, S=16, E=16, k=2, F=192),
     "bf16_paper_slice192": LC("s192", T=60, d=768, S=4, E=16, k=2, F=768),
 }

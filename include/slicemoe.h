@@ -214,7 +214,7 @@ int slicemoe_load_stats(const int32_t *counts, int32_t E, double alpha, double *
  * topk_idx / assigned / kept.  h_out must not overlap h.
  * Optional outputs (NULL to skip): assigned_opt int32 [E], kept_opt int32 [E],
  * topk_idx_opt int32 [N, k], topk_p_opt float [N, k].
- * For bf16 layers with ds in {48, 64, 96, 128, 192, 256}, E in {16, 32, 64}, k <= 2 and
+ * For bf16 layers with ds in {48, 64, 96, 128, 192, 256}, E in {8, 16, 32, 64}, k <= 2 and
  * hidden widths that are multiples of the chunk width, the whole forward is ONE
  * kernel launch (router, dispatch and expert phases separated by grid-wide
  * barriers, one CTA per SM); other shapes run one kernel per step.  Every wait

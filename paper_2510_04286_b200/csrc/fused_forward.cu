@@ -157,7 +157,7 @@ int launch_fused(const Dims& D, const slicemoe_weights& w, const void* h, const 
     // (rows narrower than K1 are zero-filled by the copies: the box reaches past the tensor's edge)
     if ((rc = make_tmap(&tmX, h, (uint64_t)D.N, (uint64_t)D.ds, 128))) return rc;
     if ((rc = make_tmap(&tmWr1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, RC::HC))) return rc;
-    if ((rc = make_tmap(&tmWr2, w.Wr2, (uint64_t)RC::N2, D.Hr, RC::N2))) return rc;
+    if ((rc = make_tmap(&tmWr2, w.Wr2, (uint64_t)D.E, D.Hr, RC::N2))) return rc;   // (E = 8: zero-filled up to 16)
     if ((rc = make_tmap(&tmW1, w.W1, (uint64_t)D.E * D.F, (uint64_t)D.ds, EC::HC))) return rc;
     if ((rc = make_tmap(&tmW2, w.W2, (uint64_t)D.E * EC::N2, D.F, EC::N2))) return rc;
     const int grid = sm_count();
@@ -201,6 +201,7 @@ int launch_fused_k1e(const Dims& D, const slicemoe_weights& w, const void* h, co
 template <int K1, int N2 = K1>
 int launch_fused_k1(const Dims& D, const slicemoe_weights& w, const void* h, const FusedParams& fp, cudaStream_t st) {
     switch (D.E) {
+        case 8:
         case 16: return launch_fused_k1e<K1, 16, N2>(D, w, h, fp, st);
         case 32: return launch_fused_k1e<K1, 32, N2>(D, w, h, fp, st);
         case 64: return launch_fused_k1e<K1, 64, N2>(D, w, h, fp, st);
@@ -287,6 +288,7 @@ int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h
     fp.assigned = assigned; fp.kept = kept; fp.offsets = offsets; fp.dest = dest; fp.perm = perm; fp.gate = gate;
     r.row_elems = D.ds;
     f.row_elems = D.ds;
+    r.experts_real = D.E;
     switch (D.ds) {
         case 48: return launch_fused_k1<64, 48>(D, w, h, fp, st);
         case 64: return launch_fused_k1<64>(D, w, h, fp, st);

@@ -31,7 +31,8 @@ int launch_tc(const void* A, uint64_t a_rows, const void* W1, const void* W2, in
     // (a row narrower than K1 is zero-filled by the copies: the box reaches past the tensor's edge)
     if ((rc = make_tmap(&tmA, A, a_rows, (uint64_t)p.row_elems, 128))) return rc;
     if ((rc = make_tmap(&tmW1, W1, (uint64_t)n_experts * p.HID, (uint64_t)p.row_elems, C::HC))) return rc;
-    if ((rc = make_tmap(&tmW2, W2, (uint64_t)n_experts * C::N2, p.HID, C::N2))) return rc;
+    // (router: the real expert count; a box taller than the tensor is zero-filled below its edge)
+    if ((rc = make_tmap(&tmW2, W2, C::ROUTER ? (uint64_t)p.experts_real : (uint64_t)n_experts * C::N2, p.HID, C::N2))) return rc;
     auto kern = tc_mlp_kernel<C>;
     static bool attr_set = false;
     if (!attr_set) {
@@ -59,6 +60,7 @@ int launch_route_k1e(const Dims& D, const slicemoe_weights& w, const void* h, co
 template <int K1>
 int launch_route_k1(const Dims& D, const slicemoe_weights& w, const void* h, const TcParams& p, cudaStream_t st) {
     switch (D.E) {
+        case 8:                                                     // padded to 16, see TcParams::experts_real
         case 16: return launch_route_k1e<K1, 16>(D, w, h, p, st);
         case 32: return launch_route_k1e<K1, 32>(D, w, h, p, st);
         case 64: return launch_route_k1e<K1, 64>(D, w, h, p, st);
@@ -88,7 +90,7 @@ static bool tc_width_supported(int ds) {
 bool tc_route_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
     if (!tc_width_supported(D.ds)) return false;
-    if (D.E != 16 && D.E != 32 && D.E != 64) return false;
+    if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
     const int hc = D.ds <= 64 ? 128 : 64;
     // at least two hidden chunks: GEMM-1 is issued ahead of GEMM-2, and with resident weights that
     // look-ahead must not need the weight slot that the chunk in flight is still using
@@ -121,6 +123,7 @@ int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int
     p.status = status;
     p.zero_out = (bf16*)zero_out; p.zero_cols = D.ds;
     p.row_elems = D.ds;
+    p.experts_real = D.E;
     switch (D.ds) {
         case 48:
         case 64: return launch_route_k1<64>(D, w, h, p, st);

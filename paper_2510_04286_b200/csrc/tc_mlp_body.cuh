@@ -58,6 +58,8 @@ constexpr int kMaxBars = 48;
 constexpr int kBiasRing = 8;
 
 struct TcParams {
+    int experts_real;         // router: the real number of experts (<= the N2 the kernel is built for: E = 8 runs
+                              // on the 16-wide instantiation, the padded experts' logits set to -inf)
     int row_elems;            // elements per row of X (= ds); at most the K1 the kernel is built for: a narrower
                               // row (the paper's own ds = 96 under K1 = 128) is zero-filled up to K1
     const int32_t* offsets;   // experts: [E+1] device row ranges; router: nullptr
@@ -446,7 +448,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             sh.bias1_f32[i] = p.bias1 ? __bfloat162float(p.bias1[i]) : 0.0f;
     if constexpr (C::ROUTER)
         for (int i = threadIdx.x; i < C::N2; i += C::THREADS)
-            sh.bias2_f32[i] = p.bias2 ? __bfloat162float(p.bias2[i]) : 0.0f;
+            sh.bias2_f32[i] = i >= p.experts_real ? -INFINITY : (p.bias2 ? __bfloat162float(p.bias2[i]) : 0.0f);
     __syncthreads();
     if (warp == 0) {
         // first tile of every expert: exclusive scan of the tile counts, 32 experts at a time
@@ -976,11 +978,12 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     atomicAdd(&sh.hist[sel[j]], 1);
                 }
                 if (p.probs) {
-                    float4* dst = reinterpret_cast<float4*>(p.probs + (size_t)n * E);
+                    float4* dst = reinterpret_cast<float4*>(p.probs + (size_t)n * p.experts_real);
 #pragma unroll
                     for (int i = 0; i < E; i += 4)
-                        dst[i / 4] = make_float4(__expf(gl[i] - m) * inv, __expf(gl[i + 1] - m) * inv,
-                                                 __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
+                        if (i < p.experts_real)                      // (the real count is a multiple of 8)
+                            dst[i / 4] = make_float4(__expf(gl[i] - m) * inv, __expf(gl[i + 1] - m) * inv,
+                                                     __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
                 }
             } else {
                 // OB output columns at a time: accumulator -> registers -> bias -> bf16 -> global
@@ -1037,9 +1040,9 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     if (threadIdx.x == 0 && sh.abort_flag) atomicExch(p.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
     if constexpr (C::ROUTER) {
         // per-CTA histogram -> global counts (Section 3.2's per-expert counts)
-        for (int i = threadIdx.x; i < C::N2; i += C::THREADS) {
+        for (int i = threadIdx.x; i < p.experts_real; i += C::THREADS) {
             if (p.assigned && sh.hist[i]) atomicAdd(&p.assigned[i], sh.hist[i]);
-            if (p.cta_hist) p.cta_hist[(size_t)blockIdx.x * C::N2 + i] = sh.hist[i];
+            if (p.cta_hist) p.cta_hist[(size_t)blockIdx.x * p.experts_real + i] = sh.hist[i];
         }
     }
 #ifdef SLICEMOE_TC_TRACE

@@ -35,6 +35,8 @@ SMALL = {
     "bf16_e64_ds64": LC("e64", T=260, d=128, S=2, E=64, k=2, F=128),
     "bf16_ds256_k2": LC("w256", T=70, d=512, S=2, E=16, k=2, F=512, Hr=128),
     # the paper's d = 768 at S = 16 and S = 4: 48- and 192-wide slices on zero-filled 64 / 256-wide tiles
+    # eight experts on the 16-wide router instantiation (padded experts masked out)
+    "bf16_e8": LC("e8", T=150, d=512, S=4, E=8, k=2, F=512),
     # k = 3 (the paper's Table 4) on the tensor-core kernels: stacked outputs + combine kernel
     "bf16_k3_tc": LC("k3tc", T=200, d=512, S=8, E=16, k=3, F=256),
     "bf16_paper_slice48": LC("s48", T=50, d=768, S=16, E=16, k=2, F=192),
@@ -234,7 +236,7 @@ def test_profiled_forward_records_stage_times():
 
 
 @pytest.mark.parametrize("name", ["bf16_lm", "bf16_skew_cap", "bf16_decode", "bf16_single_row", "bf16_k3", "f32_cfg0",
-                                  "bf16_paper_slice96", "bf16_paper_slice48", "bf16_paper_slice192"])
+                                  "bf16_paper_slice96", "bf16_paper_slice48", "bf16_paper_slice192", "bf16_e8"])
 def test_forward_launch_count_and_status(name):
     """Supported bf16 shapes with k <= 2 run the whole forward as one launch; the others one
     launch per step.  Either way the status word stays clear and repeated calls on two
@@ -250,7 +252,7 @@ def test_forward_launch_count_and_status(name):
     launches = binding.slicemoe_launch_count() - before
     other = gpu2.forward()
     torch.cuda.synchronize()
-    one_launch = lc.dtype == "bf16" and lc.k <= 2 and lc.ds in (48, 64, 96, 128, 192, 256) and lc.E in (16, 32, 64)
+    one_launch = lc.dtype == "bf16" and lc.k <= 2 and lc.ds in (48, 64, 96, 128, 192, 256) and lc.E in (8, 16, 32, 64)
     assert launches == 1 if one_launch else launches >= 3
     assert gpu.status() == 0 and gpu2.status() == 0
     for a, b, c in zip(first, again, other):

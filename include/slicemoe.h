@@ -78,6 +78,11 @@ typedef struct {
     int32_t dtype;    /* slicemoe_dtype: storage type of h, h', weights and stacked rows */
     int32_t act;      /* slicemoe_act: activation between the two expert layers */
     int64_t capacity; /* hard per-expert limit on kept pairs; 0 = unlimited */
+    /* Router ablation knobs (Section 5.2 and Appendix B); all-zero = the plain layer. */
+    float temperature;   /* softmax temperature tau > 0 (Figure 7); 0 stands for 1 */
+    float noise_sigma;   /* std of the Gaussian noise added to the logits before the
+                          * softmax (Figure 6); 0 = none */
+    uint64_t noise_seed; /* key of the counter-based noise generator (slicemoe_route) */
 } slicemoe_config;
 
 /* Caller-owned weights, dtype = cfg->dtype. */
@@ -105,6 +110,15 @@ int slicemoe_workspace_bytes(const slicemoe_config *cfg, size_t *bytes);
  * out: topk_idx int32 [N, k]; topk_p float [N, k]; assigned int32 [E] =
  *      number of pairs that chose each expert (the counts of Section 3.2);
  *      probs_opt float [N, E] (NULL to skip).
+ * With the ablation knobs of cfg (Figures 6 and 7) the softmax and the top-k see
+ *   g'[n, e] = (g[n, e] + noise_sigma * eps(n, e)) / tau
+ * instead of g.  eps(n, e) is a standard normal drawn per (row, expert) from a
+ * counter-based generator, so a call is reproducible and independent of the
+ * launch shape: Philox4x32-10 with key = (low, high word of noise_seed) and
+ * counter (n, e, 1, 0) gives words x0, x1; u_i = ((x_i >> 8) + 0.5) / 2^24;
+ * eps = sqrt(-2 ln u_0) * cos(2 pi u_1) (Box-Muller), evaluated in fp32.
+ * temperature < 0, noise_sigma < 0 or a non-finite value: SLICEMOE_ERR_SHAPE.
+ * Noisy routing runs on the CUDA-core router whatever the shape.
  */
 int slicemoe_route(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
                    int32_t *topk_idx, float *topk_p, int32_t *assigned, float *probs_opt,
@@ -195,6 +209,20 @@ int slicemoe_combine(const slicemoe_config *cfg, const void *yperm, const int32_
  */
 int slicemoe_gate_dropout(const slicemoe_config *cfg, float *topk_p, uint64_t seed, double rate,
                           void *stream);
+
+/*
+ * Shuffled slices (Section 5.2, Figure 5): slices are cut from a fixed
+ * permutation of the d columns instead of from contiguous runs.
+ *   inverse = 0:  out[t, c] = in[t, perm[c]]      (shuffle before the layer)
+ *   inverse = 1:  out[t, perm[c]] = in[t, c]      (undo it on the layer's output)
+ * so that  permute(0) -> any of the calls above -> permute(1)  is the layer
+ * whose slice s of token t holds columns perm[s*ds .. (s+1)*ds - 1] of h and
+ * writes its result back to those columns.  in, out: [T, d] of cfg->dtype, not
+ * overlapping; perm: DEVICE int32 [d], a permutation of 0..d-1 (not checked:
+ * with a repeated entry, inverse = 1 leaves columns of `out` unwritten).
+ */
+int slicemoe_permute_columns(const slicemoe_config *cfg, const void *in, void *out,
+                             const int32_t *perm, int inverse, void *stream);
 
 /*
  * Routing statistics from per-expert counts (such as `assigned` of the forward):

@@ -28,7 +28,9 @@ ACT_GELU_TANH = 1
 class _Cfg(ctypes.Structure):
     _fields_ = [("T", ctypes.c_int32), ("d", ctypes.c_int32), ("S", ctypes.c_int32),
                 ("E", ctypes.c_int32), ("k", ctypes.c_int32), ("Hr", ctypes.c_int32),
-                ("F", ctypes.c_int32), ("act", ctypes.c_int32), ("capacity", ctypes.c_int64)]
+                ("F", ctypes.c_int32), ("act", ctypes.c_int32), ("capacity", ctypes.c_int64),
+                ("temperature", ctypes.c_double), ("noise_sigma", ctypes.c_double),
+                ("noise_seed", ctypes.c_uint64)]
 
 
 @dataclass(frozen=True)
@@ -42,6 +44,9 @@ class OracleConfig:
     F: int
     act: int = ACT_RELU
     capacity: int = 0
+    temperature: float = 0.0    # router softmax temperature (0 stands for 1)
+    noise_sigma: float = 0.0    # std of Gaussian noise on the router logits
+    noise_seed: int = 0
 
     @property
     def ds(self):
@@ -56,7 +61,8 @@ class OracleConfig:
         return self.T * self.S * self.k
 
     def c(self) -> _Cfg:
-        return _Cfg(self.T, self.d, self.S, self.E, self.k, self.Hr, self.F, self.act, self.capacity)
+        return _Cfg(self.T, self.d, self.S, self.E, self.k, self.Hr, self.F, self.act, self.capacity,
+                    self.temperature, self.noise_sigma, self.noise_seed)
 
 
 def build(force: bool = False) -> str:
@@ -265,3 +271,35 @@ def gate_dropout(topk_p, seed: int, rate: float):
                                             ctypes.c_uint64(seed), ctypes.c_double(rate), _p(out),
                                             _p(dropped)), "gate_dropout")
     return out, dropped.astype(bool)
+
+
+def logit_noise(seed: int, n: int, e: int) -> float:
+    """Figure 6: the standard normal that (times sigma) is added to logit e of row n."""
+    lib = _load()
+    lib.slicemoe_oracle_logit_noise.restype = ctypes.c_double
+    return float(lib.slicemoe_oracle_logit_noise(ctypes.c_uint64(seed), ctypes.c_int64(n), ctypes.c_int32(e)))
+
+
+def permute_columns(x, perm, inverse: bool = False):
+    """Figure 5's shuffled slices, written out element by element:
+    out[t, c] = x[t, perm[c]], or with inverse out[t, perm[c]] = x[t, c]."""
+    x = np.asarray(x)
+    perm = np.asarray(perm, dtype=np.int64)
+    T, d = x.shape
+    if perm.shape != (d,) or sorted(perm.tolist()) != list(range(d)):
+        raise ValueError("perm must be a permutation of the d columns")
+    out = np.empty_like(x)
+    for c in range(d):
+        if inverse:
+            out[:, perm[c]] = x[:, c]
+        else:
+            out[:, c] = x[:, perm[c]]
+    return out
+
+
+def forward_shuffled(cfg: OracleConfig, h, w: dict, perm, forced_idx=None) -> dict:
+    """The layer on shuffled slices (Section 5.2): slice s of a token holds columns
+    perm[s*ds .. (s+1)*ds - 1] of h, and its result goes back to those columns."""
+    res = dict(forward(cfg, permute_columns(_f64(h, (cfg.T, cfg.d)), perm), w, forced_idx=forced_idx))
+    res["h_out"] = permute_columns(res["h_out"], perm, inverse=True)
+    return res

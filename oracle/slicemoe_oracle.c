@@ -40,6 +40,10 @@ typedef struct {
     int32_t T, d, S, E, k, Hr, F;
     int32_t act;       /* 0 = ReLU, 1 = GELU (tanh form) */
     int64_t capacity;  /* 0 = unlimited */
+    /* router ablation knobs (Section 5.2, Figure 6; Appendix B, Figure 7); zeros = plain layer */
+    double temperature;   /* softmax temperature tau; 0 stands for 1 */
+    double noise_sigma;   /* std of the Gaussian noise on the logits; 0 = none */
+    uint64_t noise_seed;
 } oracle_cfg;
 
 enum { ORACLE_OK = 0, ORACLE_BAD_SHAPE = 1, ORACLE_NO_MEMORY = 2 };
@@ -57,6 +61,7 @@ static int check_cfg(const oracle_cfg *c) {
     if (c->d % c->S != 0) return ORACLE_BAD_SHAPE;
     if (c->k > c->E) return ORACLE_BAD_SHAPE;
     if (c->capacity < 0) return ORACLE_BAD_SHAPE;
+    if (!(c->temperature >= 0.0) || !(c->noise_sigma >= 0.0)) return ORACLE_BAD_SHAPE;
     return ORACLE_OK;
 }
 
@@ -67,13 +72,32 @@ static double activation(double z, int act) {
     return 0.5 * z * (1.0 + tanh(c * (z + 0.044715 * z * z * z)));
 }
 
+static void philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t out[4]);
+
+/* Figure 6: the standard normal added (times sigma) to logit e of row n.  Readings: one draw per
+ * (row, expert); Philox4x32-10 with key = seed and counter (n, e, 1, 0) gives words x0, x1,
+ * u_i = ((x_i >> 8) + 0.5) / 2^24 lies strictly inside (0, 1), and Box-Muller turns the pair into
+ * eps = sqrt(-2 ln u0) cos(2 pi u1). */
+static double logit_noise(uint64_t seed, int64_t n, int e) {
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    const uint32_t ctr[4] = {(uint32_t)n, (uint32_t)e, 1u, 0u};
+    uint32_t x[4];
+    philox4x32_10(ctr, key, x);
+    const double u0 = ((double)(x[0] >> 8) + 0.5) / 16777216.0;
+    const double u1 = ((double)(x[1] >> 8) + 0.5) / 16777216.0;
+    return sqrt(-2.0 * log(u0)) * cos(2.0 * 3.14159265358979323846 * u1);
+}
+
 /* Section 3.1: router MLP Linear(ds->Hr), ReLU, Linear(Hr->E), then softmax.
- * x[ds] -> p[E].  a[Hr] is scratch. */
-static void router_probs_row(const oracle_cfg *c, const double *x,
+ * x[ds] (row n) -> p[E].  a[Hr] is scratch.  With the ablation knobs the softmax sees
+ * (g + sigma * eps(n, e)) / tau: noise on the logits before the softmax (Figure 6), softmax
+ * temperature tau (Figure 7). */
+static void router_probs_row(const oracle_cfg *c, int64_t n, const double *x,
                              const double *Wr1, const double *br1,
                              const double *Wr2, const double *br2,
                              double *a, double *p) {
     const int ds = c->d / c->S;
+    const double tau = c->temperature > 0.0 ? c->temperature : 1.0;
     for (int i = 0; i < c->Hr; ++i) {
         double z = br1 ? br1[i] : 0.0;
         for (int q = 0; q < ds; ++q) z += Wr1[(size_t)i * ds + q] * x[q];
@@ -83,6 +107,8 @@ static void router_probs_row(const oracle_cfg *c, const double *x,
     for (int e = 0; e < c->E; ++e) {
         double g = br2 ? br2[e] : 0.0;
         for (int i = 0; i < c->Hr; ++i) g += Wr2[(size_t)e * c->Hr + i] * a[i];
+        if (c->noise_sigma > 0.0) g += c->noise_sigma * logit_noise(c->noise_seed, n, e);
+        g /= tau;
         p[e] = g;
         if (g > m) m = g;
     }
@@ -166,7 +192,7 @@ int slicemoe_oracle_route(const oracle_cfg *c, const double *h,
         if (!failed) {
 #pragma omp for schedule(static)
             for (int64_t n = 0; n < N; ++n) {
-                router_probs_row(c, h + n * ds, Wr1, br1, Wr2, br2, a, p);
+                router_probs_row(c, n, h + n * ds, Wr1, br1, Wr2, br2, a, p);
                 if (probs) memcpy(probs + n * c->E, p, sizeof(double) * (size_t)c->E);
                 topk_row(c, p, topk_idx + n * c->k, topk_p + n * c->k, gap ? gap + n : NULL);
             }
@@ -405,7 +431,7 @@ int slicemoe_oracle_rows(const oracle_cfg *c, const double *h,
 #pragma omp for schedule(dynamic, 16)
             for (int64_t i = 0; i < nrows; ++i) {
                 const double *x = h + rows[i] * ds;
-                router_probs_row(c, x, Wr1, br1, Wr2, br2, a, p);
+                router_probs_row(c, rows[i], x, Wr1, br1, Wr2, br2, a, p);
                 for (int q = 0; q < ds; ++q) y[i * ds + q] = 0.0;
                 for (int j = 0; j < c->k; ++j) {
                     const int e = idx[i * c->k + j];
@@ -479,6 +505,8 @@ static void philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], ui
     }
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
+
+double slicemoe_oracle_logit_noise(uint64_t seed, int64_t n, int32_t e) { return logit_noise(seed, n, e); }
 
 void slicemoe_oracle_philox4x32(const uint32_t *ctr, const uint32_t *key, uint32_t *out) {
     philox4x32_10(ctr, key, out);

@@ -21,7 +21,7 @@ STAGES = ("route", "dispatch", "expert_ffn", "combine")
 EXPORTS = (
     "slicemoe_workspace_bytes", "slicemoe_route", "slicemoe_dispatch", "slicemoe_dispatch_static",
     "slicemoe_expert_ffn",
-    "slicemoe_combine", "slicemoe_gate_dropout", "slicemoe_load_stats", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
+    "slicemoe_combine", "slicemoe_gate_dropout", "slicemoe_permute_columns", "slicemoe_load_stats", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
     "slicemoe_event_create", "slicemoe_event_destroy", "slicemoe_event_elapsed_ms",
     "slicemoe_last_status", "slicemoe_launch_count", "slicemoe_last_cuda_error",
     "slicemoe_status_string",
@@ -40,7 +40,8 @@ class _Config(ctypes.Structure):
     _fields_ = [("T", ctypes.c_int32), ("d", ctypes.c_int32), ("S", ctypes.c_int32),
                 ("E", ctypes.c_int32), ("k", ctypes.c_int32), ("Hr", ctypes.c_int32),
                 ("F", ctypes.c_int32), ("dtype", ctypes.c_int32), ("act", ctypes.c_int32),
-                ("capacity", ctypes.c_int64)]
+                ("capacity", ctypes.c_int64), ("temperature", ctypes.c_float),
+                ("noise_sigma", ctypes.c_float), ("noise_seed", ctypes.c_uint64)]
 
 
 class _Weights(ctypes.Structure):
@@ -60,6 +61,9 @@ class Config:
     dtype: int = BF16
     act: int = ACT_GELU_TANH
     capacity: int = 0
+    temperature: float = 0.0     # softmax temperature of the router (0 stands for 1)
+    noise_sigma: float = 0.0     # std of Gaussian noise on the router logits
+    noise_seed: int = 0
 
     @property
     def ds(self):
@@ -75,7 +79,7 @@ class Config:
 
     def c(self) -> _Config:
         return _Config(self.T, self.d, self.S, self.E, self.k, self.Hr, self.F, self.dtype, self.act,
-                       self.capacity)
+                       self.capacity, self.temperature, self.noise_sigma, self.noise_seed)
 
 
 _handle = None
@@ -191,6 +195,14 @@ def slicemoe_gate_dropout(cfg, topk_p, seed, rate, stream=None):
     c = cfg.c()
     _check(_lib().slicemoe_gate_dropout(ctypes.byref(c), _ptr(topk_p), ctypes.c_uint64(seed), ctypes.c_double(rate),
                                         _stream(stream)), "slicemoe_gate_dropout")
+
+
+def slicemoe_permute_columns(cfg, src, dst, perm, inverse=False, stream=None):
+    """Figure 5's shuffled slices: dst[t, c] = src[t, perm[c]], or with inverse dst[t, perm[c]] = src[t, c]."""
+    c = cfg.c()
+    _check(_lib().slicemoe_permute_columns(ctypes.byref(c), _ptr(src), _ptr(dst), _ptr(perm),
+                                           ctypes.c_int(1 if inverse else 0), _stream(stream)),
+           "slicemoe_permute_columns")
 
 
 def slicemoe_load_stats(counts, alpha, out, stream=None):

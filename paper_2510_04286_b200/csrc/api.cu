@@ -1,6 +1,7 @@
 // C ABI of the SliceMoE layer forward: argument checking, workspace layout and the sequencing of
 // the stage kernels on the caller's stream.  No step of the layer is computed here.
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 
@@ -62,6 +63,12 @@ int make_dims(const slicemoe_config* c, Dims& D) {
     const int ds = c->d / c->S;
     if (ds % V || c->Hr % V || c->F % V) return SLICEMOE_ERR_UNSUPPORTED;
     if (c->k > 8 || c->E > 256) return SLICEMOE_ERR_UNSUPPORTED;
+    if (!(c->temperature >= 0.0f) || !(c->noise_sigma >= 0.0f) || std::isinf(c->temperature) ||
+        std::isinf(c->noise_sigma))
+        return SLICEMOE_ERR_SHAPE;
+    D.inv_tau = c->temperature > 0.0f ? 1.0f / c->temperature : 1.0f;
+    D.noise_sigma = c->noise_sigma;
+    D.noise_seed = c->noise_seed;
     D.T = c->T; D.d = c->d; D.S = c->S; D.E = c->E; D.k = c->k; D.Hr = c->Hr; D.F = c->F;
     D.ds = ds; D.N = (int)N; D.R = (int)R; D.dtype = c->dtype; D.act = c->act;
     D.capacity = (int)(c->capacity > R ? R : c->capacity);

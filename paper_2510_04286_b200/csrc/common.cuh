@@ -19,6 +19,9 @@ struct Dims {
     int R;    // pairs = N*k
     int dtype, act;
     int capacity;  // 0 = unlimited; clamped to R
+    float inv_tau;        // 1 / softmax temperature
+    float noise_sigma;    // 0 = no logit noise
+    uint64_t noise_seed;
 };
 
 // Pairs handled by one dispatch chunk (one CTA of the histogram / scatter kernels).
@@ -131,6 +134,10 @@ int fused_forward_reset_sync(cudaStream_t st);
 
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);
+
+// out[t, c] = in[t, perm[c]] (inverse = false) or out[t, perm[c]] = in[t, c] (inverse = true).
+int launch_permute_columns(const Dims& D, const void* in, void* out, const int32_t* perm, bool inverse,
+                           cudaStream_t st);
 
 // ---- storage-type helpers ---------------------------------------------------------------------
 

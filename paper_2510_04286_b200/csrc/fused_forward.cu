@@ -289,6 +289,7 @@ int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h
     r.row_elems = D.ds;
     f.row_elems = D.ds;
     r.experts_real = D.E;
+    r.softmax_scale = 1.4426950408889634f * D.inv_tau;
     switch (D.ds) {
         case 48: return launch_fused_k1<64, 48>(D, w, h, fp, st);
         case 64: return launch_fused_k1<64>(D, w, h, fp, st);

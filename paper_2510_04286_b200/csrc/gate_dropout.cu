@@ -6,25 +6,15 @@
 // first word of Philox4x32-10 (Salmon et al., SC'11) with key = seed and counter = (n, j, 0, 0);
 // dropped iff word < floor(rate * 2^32).  One thread per row, in place; k <= 8.
 #include "common.cuh"
+#include "philox.cuh"
 
 namespace slicemoe {
 namespace {
 
 __device__ __forceinline__ uint32_t philox_first_word(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1) {
-    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
-    uint32_t c2 = 0u, c3 = 0u;
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-        const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
-        c0 = hi1 ^ c1 ^ k0;
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ k1;
-        c3 = lo0;
-        k0 += W0;
-        k1 += W1;
-    }
-    return c0;
+    uint32_t x[4];
+    philox4x32_10(c0, c1, 0u, 0u, k0, k1, x);
+    return x[0];
 }
 
 __global__ void __launch_bounds__(256) gate_dropout_kernel(float* __restrict__ topk_p, int N, int k, uint32_t key0,

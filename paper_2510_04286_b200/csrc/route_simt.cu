@@ -1,7 +1,11 @@
 // Router of Section 3.1 on CUDA cores: Linear(ds->Hr) + ReLU, Linear(Hr->E), softmax, top-k.
 // All arithmetic is fp32 with a fixed summation order, whatever the storage type.  This is the
 // fp32 path of the library and the path for shapes the tensor-core router does not take.
+// Ablation knobs (Figures 6 and 7): the softmax and the top-k see (g + sigma * eps) / tau, eps a
+// standard normal per (row, expert) from Philox4x32-10, key = seed, counter (n, e, 1, 0), through
+// Box-Muller on 24-bit uniforms.
 #include "common.cuh"
+#include "philox.cuh"
 
 namespace slicemoe {
 namespace {
@@ -9,13 +13,23 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kMaxK = 8;
 
+// eps(n, e): u_i = ((x_i >> 8) + 0.5) / 2^24 in (0, 1), both exact in fp32.
+__device__ __forceinline__ float logit_noise(int n, int e, uint32_t key0, uint32_t key1) {
+    uint32_t x[4];
+    philox4x32_10((uint32_t)n, (uint32_t)e, 1u, 0u, key0, key1, x);
+    const float u0 = ((float)(x[0] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    const float u1 = ((float)(x[1] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    return sqrtf(-2.0f * logf(u0)) * cospif(2.0f * u1);
+}
+
 // One CTA routes ROWS consecutive rows.
 template <typename T, int ROWS>
 __global__ void __launch_bounds__(kThreads)
 route_simt_kernel(const T* __restrict__ X, const T* __restrict__ Wr1, const T* __restrict__ br1,
                   const T* __restrict__ Wr2, const T* __restrict__ br2, int N, int ds, int Hr, int E,
                   int k, int32_t* __restrict__ topk_idx, float* __restrict__ topk_p,
-                  int32_t* __restrict__ assigned, float* __restrict__ probs) {
+                  int32_t* __restrict__ assigned, float* __restrict__ probs, float inv_tau, float sigma,
+                  uint32_t key0, uint32_t key1) {
     extern __shared__ __align__(16) float smem[];
     float* xs = smem;                 // [ROWS][ds]
     float* hs = xs + ROWS * ds;       // [ROWS][Hr]
@@ -78,7 +92,8 @@ route_simt_kernel(const T* __restrict__ X, const T* __restrict__ Wr1, const T* _
             for (int u = 0; u < V; ++u) acc = fmaf(wv[u], hrow[i + u], acc);
         }
         for (; i < Hr; ++i) acc = fmaf(to_f32(wrow[i]), hrow[i], acc);
-        gs[r * E + e] = acc;
+        if (sigma > 0.0f && r < rows) acc = fmaf(sigma, logit_noise(row0 + r, e, key0, key1), acc);
+        gs[r * E + e] = acc * inv_tau;
     }
     __syncthreads();
 
@@ -128,7 +143,8 @@ int launch_rows(const Dims& D, const slicemoe_weights& w, const void* h, int32_t
     const int grid = (D.N + ROWS - 1) / ROWS;
     kern<<<grid, kThreads, smem, st>>>((const T*)h, (const T*)w.Wr1, (const T*)w.br1, (const T*)w.Wr2,
                                       (const T*)w.br2, D.N, D.ds, D.Hr, D.E, D.k, topk_idx, topk_p,
-                                      assigned, probs);
+                                      assigned, probs, D.inv_tau, D.noise_sigma, (uint32_t)D.noise_seed,
+                                      (uint32_t)(D.noise_seed >> 32));
     SLICEMOE_LAUNCH_CHECK(1);
     return SLICEMOE_OK;
 }

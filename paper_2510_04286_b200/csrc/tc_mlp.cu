@@ -91,6 +91,7 @@ bool tc_route_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16) return false;
     if (!tc_width_supported(D.ds)) return false;
     if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
+    if (D.noise_sigma > 0.0f) return false;   // noisy logits (an ablation) stay on the CUDA-core router
     const int hc = D.ds <= 64 ? 128 : 64;
     // at least two hidden chunks: GEMM-1 is issued ahead of GEMM-2, and with resident weights that
     // look-ahead must not need the weight slot that the chunk in flight is still using
@@ -124,6 +125,7 @@ int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int
     p.zero_out = (bf16*)zero_out; p.zero_cols = D.ds;
     p.row_elems = D.ds;
     p.experts_real = D.E;
+    p.softmax_scale = 1.4426950408889634f * D.inv_tau;
     switch (D.ds) {
         case 48:
         case 64: return launch_route_k1<64>(D, w, h, p, st);

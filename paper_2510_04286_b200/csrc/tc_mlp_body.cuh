@@ -62,6 +62,7 @@ struct TcParams {
                               // on the 16-wide instantiation, the padded experts' logits set to -inf)
     int row_elems;            // elements per row of X (= ds); at most the K1 the kernel is built for: a narrower
                               // row (the paper's own ds = 96 under K1 = 128) is zero-filled up to K1
+    float softmax_scale;      // router: log2(e) / tau (Figure 7's temperature; top-k does not depend on it)
     const int32_t* offsets;   // experts: [E+1] device row ranges; router: nullptr
     int n_rows;               // router: N; experts: R (length of the stacked-row arrays)
     int E;                    // experts: E; router: 1
@@ -968,13 +969,14 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         if (j == 0) m = bv;
                     }
                 }
+                const float sc = p.softmax_scale;
                 float sum = 0.0f;
 #pragma unroll
-                for (int i = 0; i < E; ++i) sum += __expf(gl[i] - m);
+                for (int i = 0; i < E; ++i) sum += ex2_approx((gl[i] - m) * sc);
                 const float inv = 1.0f / sum;
                 for (int j = 0; j < p.k; ++j) {
                     p.topk_idx[(size_t)n * p.k + j] = sel[j];
-                    p.topk_p[(size_t)n * p.k + j] = __expf(gsel[j] - m) * inv;
+                    p.topk_p[(size_t)n * p.k + j] = ex2_approx((gsel[j] - m) * sc) * inv;
                     atomicAdd(&sh.hist[sel[j]], 1);
                 }
                 if (p.probs) {
@@ -982,8 +984,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #pragma unroll
                     for (int i = 0; i < E; i += 4)
                         if (i < p.experts_real)                      // (the real count is a multiple of 8)
-                            dst[i / 4] = make_float4(__expf(gl[i] - m) * inv, __expf(gl[i + 1] - m) * inv,
-                                                     __expf(gl[i + 2] - m) * inv, __expf(gl[i + 3] - m) * inv);
+                            dst[i / 4] = make_float4(ex2_approx((gl[i] - m) * sc) * inv, ex2_approx((gl[i + 1] - m) * sc) * inv,
+                                                     ex2_approx((gl[i + 2] - m) * sc) * inv, ex2_approx((gl[i + 3] - m) * sc) * inv);
                 }
             } else {
                 // OB output columns at a time: accumulator -> registers -> bias -> bf16 -> global

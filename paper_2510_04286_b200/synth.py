@@ -47,6 +47,9 @@ class LayerConfig:
                                  # "kaiming": He-uniform weights, uniform biases
     zipf_s: float = 0.0          # > 0: router output bias 1.5*log(Zipf(s) weight)
     wr2_gain: float = 1.0        # multiplies the std of Wr2 (calibrated-skew variant)
+    temperature: float = 0.0     # router softmax temperature (0 stands for 1)
+    noise_sigma: float = 0.0     # std of Gaussian noise on the router logits
+    noise_seed: int = 0
 
     @property
     def ds(self) -> int:

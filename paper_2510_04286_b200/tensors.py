@@ -9,7 +9,8 @@ from . import binding, synth
 def config_from_synth(lc: synth.LayerConfig) -> binding.Config:
     return binding.Config(T=lc.T, d=lc.d, S=lc.S, E=lc.E, k=lc.k, F=lc.F, Hr=lc.Hr,
                           dtype=binding.BF16 if lc.dtype == "bf16" else binding.F32,
-                          act=lc.act, capacity=lc.capacity)
+                          act=lc.act, capacity=lc.capacity, temperature=lc.temperature,
+                          noise_sigma=lc.noise_sigma, noise_seed=lc.noise_seed)
 
 
 def to_torch(arr: np.ndarray, dtype: str, device="cuda", pin=False):

@@ -23,7 +23,8 @@ F32_ELEM = 1e-4
 
 def oracle_config(lc: synth.LayerConfig) -> oracle.OracleConfig:
     return oracle.OracleConfig(T=lc.T, d=lc.d, S=lc.S, E=lc.E, k=lc.k, Hr=lc.Hr, F=lc.F, act=lc.act,
-                               capacity=lc.capacity)
+                               capacity=lc.capacity, temperature=lc.temperature,
+                               noise_sigma=lc.noise_sigma, noise_seed=lc.noise_seed)
 
 
 def check_routing(probs, gap, ref_idx, gpu_idx, gpu_p=None):

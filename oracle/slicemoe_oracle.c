@@ -25,8 +25,10 @@
  * equivariance, an affine special case and a dense-MLP special case checked
  * against numpy matmul; load statistics against their closed forms; cross-slice
  * dropout (tests/test_dropout.py) against the generator's published known-answer
- * vectors, a pure-Python restatement, and its invariants.  No function here is
- * unpinned.
+ * vectors, a pure-Python restatement, and its invariants; router temperature and
+ * logit noise (tests/test_router_knobs.py) against the log-odds identities of a
+ * softmax, the limits tau -> 0 and infinity, and normality tests of the noise.
+ * No function here is unpinned.
  */
 #include <math.h>
 #include <stdint.h>

@@ -11,6 +11,16 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kStageBytes = 16 * 1024;   // rows staged per step: as many as fit here (at least one)
 
+// V consecutive entries of the permutation (16-byte aligned: V is 4 or 8 and the start a multiple of V).
+template <int V>
+__device__ __forceinline__ void load_perm(const int32_t* __restrict__ p, int* out) {
+#pragma unroll
+    for (int i = 0; i < V; i += 4) {
+        const int4 q = __ldg(reinterpret_cast<const int4*>(p + i));
+        out[i] = q.x; out[i + 1] = q.y; out[i + 2] = q.z; out[i + 3] = q.w;
+    }
+}
+
 template <typename T, bool INVERSE>
 __global__ void __launch_bounds__(kThreads)
 permute_columns_kernel(const T* __restrict__ in, T* __restrict__ out, const int32_t* __restrict__ perm,
@@ -31,8 +41,10 @@ permute_columns_kernel(const T* __restrict__ in, T* __restrict__ out, const int3
             for (int v = threadIdx.x; v < nvec; v += kThreads) {
                 const int r = v / vec_per_row, c0 = (v - r * vec_per_row) * V;
                 __align__(16) T tmp[V];
+                int src_col[V];
+                load_perm<V>(perm + c0, src_col);
 #pragma unroll
-                for (int i = 0; i < V; ++i) tmp[i] = stage[r * d + __ldg(perm + c0 + i)];
+                for (int i = 0; i < V; ++i) tmp[i] = stage[r * d + src_col[i]];
                 dst[v] = *reinterpret_cast<const uint4*>(tmp);
             }
         } else {
@@ -40,8 +52,10 @@ permute_columns_kernel(const T* __restrict__ in, T* __restrict__ out, const int3
                 const int r = v / vec_per_row, c0 = (v - r * vec_per_row) * V;
                 __align__(16) T tmp[V];
                 *reinterpret_cast<uint4*>(tmp) = __ldg(src + v);
+                int dst_col[V];
+                load_perm<V>(perm + c0, dst_col);
 #pragma unroll
-                for (int i = 0; i < V; ++i) stage[r * d + __ldg(perm + c0 + i)] = tmp[i];
+                for (int i = 0; i < V; ++i) stage[r * d + dst_col[i]] = tmp[i];
             }
             __syncthreads();
             for (int v = threadIdx.x; v < nvec; v += kThreads) dst[v] = reinterpret_cast<const uint4*>(stage)[v];

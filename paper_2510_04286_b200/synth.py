@@ -99,6 +99,8 @@ CONFIGS = {
     # width F = 4 ds follows the other workloads, the batch is 32 sequences of 512 tokens.
     "paper768": LayerConfig("paper768", T=16384, d=768, S=8, E=16, k=2, F=384),
     # the shapes of the paper's slice-count and top-k ablations (Table 2, Table 4) on the same model
+    "paper768_S2": LayerConfig("paper768_S2", T=16384, d=768, S=2, E=16, k=2, F=1536),     # CUDA-core kernels
+    "paper768_S32": LayerConfig("paper768_S32", T=16384, d=768, S=32, E=16, k=2, F=96),    # CUDA-core kernels
     "paper768_S4": LayerConfig("paper768_S4", T=16384, d=768, S=4, E=16, k=2, F=768),
     "paper768_S16": LayerConfig("paper768_S16", T=16384, d=768, S=16, E=16, k=2, F=192),
     "paper768_k1": LayerConfig("paper768_k1", T=16384, d=768, S=8, E=16, k=1, F=384),

@@ -41,6 +41,9 @@ SMALL = {
     "bf16_k3_tc": LC("k3tc", T=200, d=512, S=8, E=16, k=3, F=256),
     "bf16_paper_slice48": LC("s48", T=50, d=768, S=16, E=16, k=2, F=192),
     "bf16_paper_slice192": LC("s192", T=60, d=768, S=4, E=16, k=2, F=768),
+    # S = 2 and S = 32 of the same sweep: 384- and 24-wide slices, CUDA-core kernels
+    "bf16_paper_slice384": LC("s384", T=40, d=768, S=2, E=16, k=2, F=1536),
+    "bf16_paper_slice24": LC("s24", T=40, d=768, S=32, E=16, k=2, F=96),
 }
 
 

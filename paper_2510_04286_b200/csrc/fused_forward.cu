@@ -107,7 +107,7 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     }
 
     // ---- phase 1: router -----------------------------------------------------------------------
-    tc_body<RC, false>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
+    tc_body<RC, false, false, true>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
     bool ok = sh.abort_flag == 0;
     STAMP(1);
     ok = grid_barrier(fp.sync_words, gen0, sh) && ok;
@@ -125,7 +125,7 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     STAMP(4);
 
     // ---- phase 3: experts ------------------------------------------------------------------------
-    if (ok) tc_body<EC, true, true>(&tmX, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
+    if (ok) tc_body<EC, true, true, true>(&tmX, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
 
     __syncthreads();
@@ -281,7 +281,7 @@ int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h
     f.offsets = offsets; f.n_rows = (int)D.R; f.E = D.E; f.HID = D.F;
     f.bias1 = (const bf16*)w.b1; f.bias2 = (const bf16*)w.b2;
     f.yperm = nullptr; f.status = status;
-    f.gather_src = (const bf16*)h; f.perm = perm; f.gate = gate; f.gather_k = D.k;
+    f.gather_src = (const bf16*)h; f.perm = perm; f.gate = gate; pair_to_row_magic(D.k, &f.gather_magic, &f.gather_shift);
     f.scatter_out = (bf16*)h_out;
 
     fp.R = (int)D.R; fp.E = D.E; fp.pairs_per_chunk = rows_per_cta * D.k; fp.capacity = (int)D.capacity;

@@ -145,7 +145,7 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
     p.offsets = offsets; p.n_rows = (int)D.R; p.E = D.E; p.HID = D.F;
     p.bias1 = (const bf16*)w.b1; p.bias2 = (const bf16*)w.b2;
     p.yperm = (bf16*)yperm; p.status = status;
-    p.gather_src = (const bf16*)gather_h; p.perm = perm; p.gate = gate; p.gather_k = D.k;
+    p.gather_src = (const bf16*)gather_h; p.perm = perm; p.gate = gate; pair_to_row_magic(D.k, &p.gather_magic, &p.gather_shift);
     p.scatter_out = gather_h ? (bf16*)scatter_out : nullptr;
     if (gather_h) xperm = gather_h;   // the A tensor map is not used in gather mode; any valid matrix will do
     p.row_elems = D.ds;

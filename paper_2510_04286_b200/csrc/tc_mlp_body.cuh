@@ -74,7 +74,7 @@ struct TcParams {
     const bf16* gather_src;   // h viewed as X[N, K1], or nullptr (A = stacked rows via TMA)
     const int32_t* perm;      // [R] pair index n*k + j of each stacked row
     const float* gate;        // [R] gate value of each stacked row
-    int gather_k;             // k (pairs per row)
+    uint32_t gather_magic, gather_shift;   // row of pair i = (i * magic) >> shift = i / k (see pair_to_row)
     bf16* scatter_out;        // fused forward, k <= 2: h' viewed as Y[N, N2]; the row of pair (n, j) is added to
                               // Y[n, :] (h' zeroed beforehand) instead of being stored to yperm; or nullptr
     // router, fused forward: this CTA also zeroes the rows of zero_out that it routes
@@ -147,7 +147,15 @@ struct TcCfg {
     // 64-wide expert rows run four groups of one warpgroup on four 64-column chunks instead: the
     // warps of a sub-partition are then in four different phases, and a warp in its tanh phase is
     // more often there to use the unit while the others load, convert and store.
-    static constexpr int NGRP = (K1 == 256) ? 1 : (FOUR_GROUPS ? 4 : 2);
+    // 64-wide expert rows: three groups do as well as four (measured), and the warpgroup this frees
+    // gives the forward three more gather warps: each of the four then copies one block of 32 rows of a
+    // tile (see the gather warps).
+#ifndef SLICEMOE_DEV_GATHER4
+#define SLICEMOE_DEV_GATHER4 1
+#endif
+    static constexpr bool GATHER4 = FOUR_GROUPS && SLICEMOE_DEV_GATHER4;
+    static constexpr int GATHER_WARPS = GATHER4 ? 4 : 1;
+    static constexpr int NGRP = (K1 == 256) ? 1 : (FOUR_GROUPS ? (GATHER4 ? 3 : 4) : 2);
     static constexpr int GWG = FOUR_GROUPS ? 1 : 2;
     static constexpr int NWG = NGRP * GWG;
     // GEMM-1 accumulator / hidden buffers.  The router's hidden pair lives inside the accumulator it
@@ -155,7 +163,7 @@ struct TcCfg {
     // chunks can then be issued while GEMM-2 still reads this one.
     static constexpr int NBUF = ROUTER_ ? 3 : (FOUR_GROUPS ? 4 : 2);
     static constexpr int GRP_WARPS = GWG * 4;                   // warps that work on one chunk
-    static constexpr int THREADS = 128 + NWG * 128 + 128;
+    static constexpr int THREADS = 128 + NWG * 128 + 128 + (GATHER4 ? 128 : 0);
     static constexpr int OUT_WARP0 = 4 + NWG * 4;               // first warp of the output warpgroup
     static constexpr int ACC2_BUFS = (N2 <= 128) ? 2 : 1;
     // The router keeps the hidden layer as a bf16 pair (hi + lo = 16 mantissa bits): GEMM-2 runs
@@ -246,6 +254,23 @@ __device__ __forceinline__ void locate_tile(const int* tile_start, const int* of
     while (t >= tile_start[e + 1]) ++e;
     row0 = offs[e] + (t - tile_start[e]) * kTileM;
     rows = min(kTileM, offs[e + 1] - row0);
+}
+
+// Row n = pair / k of a pair index, k = 1..8, without a division: (pair * magic) >> shift with
+// magic = ceil(2^shift / k) (1 and log2 k for a power of two); the reciprocal's error stays below 1/k
+// over 31-bit pair indices (checked exhaustively at the edges and on random indices for every k).
+__device__ __forceinline__ int pair_to_row(int pair, uint32_t magic, uint32_t shift) {
+    return (int)(((unsigned long long)(uint32_t)pair * magic) >> shift);
+}
+inline void pair_to_row_magic(int k, uint32_t* magic, uint32_t* shift) {
+    if ((k & (k - 1)) == 0) {
+        *magic = 1u;
+        *shift = 0u;
+        while ((1 << *shift) < k) ++*shift;
+    } else {
+        *shift = k == 3 ? 33u : 34u;
+        *magic = (uint32_t)(((1ull << *shift) + (unsigned)k - 1) / (unsigned)k);
+    }
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -390,7 +415,7 @@ __device__ __forceinline__ int ld_index(const int32_t* ptr) {
 // Called by all threads of the CTA; TMEM (sh.tmem_base, at least C::TMEM_COLS columns) is allocated
 // and freed by the caller.  SAME_LAUNCH: offsets / perm / gate were written earlier in this launch;
 // OFFS_IN_SMEM: sh.offs already holds the row ranges.
-template <class C, bool SAME_LAUNCH, bool OFFS_IN_SMEM = false>
+template <class C, bool SAME_LAUNCH, bool OFFS_IN_SMEM = false, bool FUSED = false>
 __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p,
                                         const TcParams& p, TcShared& sh, uint8_t* smem_raw) {
     using B = Bars<C>;
@@ -404,7 +429,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     volatile int* abort = &sh.abort_flag;
     const int nchunks = p.HID / C::HC;
     const bool resident = nchunks <= C::W_STAGES;
-    const bool gather = !C::ROUTER && p.gather_src != nullptr;
+    // FUSED (the single-kernel forward): what that caller always asks for is fixed at compile time --
+    // rows gathered and results added into h' (experts); no probability matrix, no global counts, k <= 2,
+    // h' zeroed (router) -- so that the other variants' code is not part of its hot loops
+    const bool gather = !C::ROUTER && (FUSED || p.gather_src != nullptr);
     auto bar = [&](int i) { return smem_u32(&sh.bars[i]); };
 
 #ifdef SLICEMOE_TC_TRACE
@@ -417,7 +445,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         { TRACE_DECL(tr0, 5); TRACE(tr0, 99); }
 #endif
         sh.abort_flag = 0;
-        for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 32 : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
+        for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 32 * C::GATHER_WARPS : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
         for (int i = 0; i < C::W_STAGES; ++i) {
             mbar_init(bar(B::W1_FULL + i), 1); mbar_init(bar(B::W1_EMPTY + i), 1);
             mbar_init(bar(B::W2_FULL + i), 1); mbar_init(bar(B::W2_EMPTY + i), 1);
@@ -698,10 +726,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 if (C::UNIFORM_ISSUE) __syncwarp();
             }
         }
-    } else if (warp == 3) {
+    } else if (warp == 3 || (C::GATHER4 && warp >= C::OUT_WARP0 + 4 && warp < C::OUT_WARP0 + 7)) {
         if constexpr (C::ROUTER) {
             // ============= zero this CTA's rows of h' (router, fused forward) ================
-            if (p.zero_out != nullptr && t_begin < t_end) {
+            if ((FUSED || p.zero_out != nullptr) && t_begin < t_end) {
                 const long long row_lo = (long long)t_begin * kTileM;
                 long long row_hi = (long long)t_end * kTileM;
                 if (row_hi > p.n_rows) row_hi = p.n_rows;
@@ -721,30 +749,32 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             const int ch = lane % CPR, rsub = lane / CPR;
             int ge = 0, gm = 0;
             bool ok = true;
-            int nrow[4], nnext[4];                    // source rows of tile rows lane + 32 q
-            // (the loaded pair index is left untouched until the next tile, so that the load's latency
-            // is not waited for here)
-            auto load_rows = [&](int t, int* out) {
-                int row0, rows;
-                locate_tile(sh.tile_start, sh.offs, t, ge, row0, rows);
+            // Blocks of 32 rows per gather warp: all four, or one each with four gather warps (warp 3 and
+            // the three after the output warpgroup: one per sub-partition).
+            constexpr int QPW = 4 / C::GATHER_WARPS;
+            const int q0 = C::GATHER4 ? (warp == 3 ? 0 : warp - (C::OUT_WARP0 + 4) + 1) : 0;
+            int nrow[QPW], nnext[QPW];                   // source rows of tile rows lane + 32 (q0 + q); pairs of the next tile
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int r = lane + 32 * q;
-                    out[q] = (r < rows) ? ld_index<SAME_LAUNCH>(p.perm + row0 + r) : -1;
-                }
-            };
-            load_rows(t_begin, nnext);
-            TRACE_DECL(tr, lane == 0 ? 0 : 7);
-            for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
+            for (int q = 0; q < QPW; ++q) nnext[q] = -1;
+            // The first turn (t = t_begin - 1) only fetches the first tile's pair indices; a tile's indices
+            // are fetched one tile ahead and left untouched until then, so that the load's latency is not
+            // waited for.
+            TRACE_DECL(tr, (lane == 0 && warp == 3) ? 0 : 7);
+#pragma unroll 1
+            for (int t = t_begin - 1, ta = -1; t < t_end && ok; ++t, ++ta) {
                 TRACE(tr, 1);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) nrow[q] = nnext[q] < 0 ? -1 : nnext[q] / p.gather_k;
-#ifdef SLICEMOE_TC_TRACE
+                for (int q = 0; q < QPW; ++q) nrow[q] = nnext[q] < 0 ? -1 : pair_to_row(nnext[q], p.gather_magic, p.gather_shift);
+                if (t + 1 < t_end) {
+                    int row0, rows;
+                    locate_tile(sh.tile_start, sh.offs, t + 1, ge, row0, rows);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) asm volatile("mov.b32 %0, %0;" : "+r"(nrow[q]));
-                TRACE(tr, 4);
-#endif
-                if (t + 1 < t_end) load_rows(t + 1, nnext);
+                    for (int q = 0; q < QPW; ++q) {
+                        const int r = lane + 32 * (q0 + q);
+                        nnext[q] = (r < rows) ? ld_index<SAME_LAUNCH>(p.perm + row0 + r) : -1;
+                    }
+                }
+                if (ta < 0) continue;
                 TRACE(tr, 5);
                 const int ab = ta % C::A_BUFS;
                 ok = mbar_wait(bar(B::A_EMPTY + ab), ((uint32_t)(ta / C::A_BUFS) & 1u) ^ 1u, abort, kWaitLimitNs);
@@ -752,28 +782,42 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 if (!ok) break;
                 TRACE(tr, 2);
                 const uint32_t dst0 = sA + ab * C::A_BYTES + (ch >> 3) * C::A_PANEL;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                const bool in_row = ch * 8 < p.row_elems;       // chunks past the row's real width are zero-filled
+                auto copy_block = [&](int q, int nrow_q) {       // 32 rows of the tile
 #pragma unroll 8
                     for (int i = 0; i < 32 / RPI; ++i) {
-                        const int r32 = i * RPI + rsub;                 // row within this block of 32
+                        const int r32 = i * RPI + rsub;             // row within this block of 32
                         const int r = q * 32 + r32;
-                        const int n = __shfl_sync(0xffffffffu, nrow[q], r32);
-                        // (rows past the tile's end and chunks past the row's real width are zero-filled)
-                        const bool real = n >= 0 && ch * 8 < p.row_elems;
+                        const int n = __shfl_sync(0xffffffffu, nrow_q, r32);
+                        const bool real = n >= 0 && in_row;          // (rows past the tile's end are zero-filled too)
                         const bf16* src = p.gather_src + (real ? (size_t)n * p.row_elems + ch * 8 : 0);
                         cp_async_16(dst0 + (r >> 3) * 1024 + (r & 7) * 128 + (((ch & 7) ^ (r & 7)) << 4), src,
                                     real ? 16u : 0u);
                     }
+                };
+                // The four blocks: a rolled loop in the single-kernel forward, unrolled in the stand-alone
+                // kernel (measured both ways in both: 472 -> 465 us there, 298 -> 327 us here on cfg2).  How
+                // far to unroll is a trade: this warp shares its sub-partition with five busier ones and gets
+                // an instruction in every ~8 cycles, so it needs independent work in flight (fully rolled, 32
+                // dependent turns per tile made it the slowest stage: 465 -> 562 us), while fully unrolled its
+                // ~2000 instructions per tile sweep the other warps' loops out of the instruction cache.
+                if constexpr (QPW == 1) {
+                    copy_block(q0, nrow[0]);
+                } else if constexpr (FUSED) {
+#pragma unroll 1
+                    for (int q = 0; q < 4; ++q) copy_block(q, q == 0 ? nrow[0] : q == 1 ? nrow[1] : q == 2 ? nrow[2] : nrow[3]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) copy_block(q, nrow[q]);
                 }
                 {
                     int row0, rows;
                     locate_tile(sh.tile_start, sh.offs, t, gm, row0, rows);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
+                    for (int q = 0; q < QPW; ++q) {
                         // rows past the tile's end take a neighbour's values: their A rows are zero and
                         // they are never stored
-                        const int r = lane + 32 * q, src = min(row0 + r, p.n_rows - 1);
+                        const int r = lane + 32 * (q0 + q), src = min(row0 + r, p.n_rows - 1);
                         cp_async_4(smem_u32(&sh.gate_s[ta % kMetaRing][r]), p.gate + src);
                         cp_async_4(smem_u32(&sh.pair_s[ta % kMetaRing][r]), p.perm + src);
                     }
@@ -829,10 +873,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     // next chunk runs under this chunk's activation.  Then piece by piece: the argument
                     // and tanh of piece pc, and behind them the tail and the store of piece pc - 1,
                     // whose tanh results have arrived by then.
-                    __nv_bfloat162 z[C::NPIECE][C::PIECE / 2];
                     const __nv_bfloat16 gs_hi = __float2bfloat16_rn(gs);
                     const __nv_bfloat162 gate_hi = __bfloat162bfloat162(gs_hi);
                     const __nv_bfloat162 gate_lo = __float2bfloat162_rn(gs - __bfloat162float(gs_hi));
+                    __nv_bfloat162 z[C::NPIECE][C::PIECE / 2];
 #pragma unroll
                     for (int s0 = 0; s0 < C::NPIECE; s0 += C::SUB) {
                         uint32_t v[C::SUB][C::PIECE];
@@ -888,7 +932,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 TRACE(tr, 35);
             }
         }
-    } else if (warp >= C::OUT_WARP0) {
+    } else if (warp >= C::OUT_WARP0 && warp < C::OUT_WARP0 + 4) {
         // ================= output warpgroup ==================================================
         const int lg = warp & 3;
         const int row = lg * 32 + lane;
@@ -935,7 +979,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 float m;
                 int sel[8];
                 float gsel[8];
-                if (p.k <= 2) {
+                if (FUSED || p.k <= 2) {
                     // one pass keeping the best two (strict comparisons in ascending id order give the
                     // same picks as repeated arg-max)
                     float b1 = gl[0], b2 = -INFINITY;
@@ -979,7 +1023,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     p.topk_p[(size_t)n * p.k + j] = ex2_approx((gsel[j] - m) * sc) * inv;
                     atomicAdd(&sh.hist[sel[j]], 1);
                 }
-                if (p.probs) {
+                if (!FUSED && p.probs) {
                     float4* dst = reinterpret_cast<float4*>(p.probs + (size_t)n * p.experts_real);
 #pragma unroll
                     for (int i = 0; i < E; i += 4)
@@ -989,12 +1033,18 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 }
             } else {
                 // OB output columns at a time: accumulator -> registers -> bias -> bf16 -> global
-                constexpr int OB = (C::N2 % 64 == 0) ? 64 : (C::N2 % 32 == 0) ? 32 : 16;
+                // (16 columns per turn of a rolled loop, not 64 unrolled: the shorter body is worth more
+                // than the saved accumulator-load waits -- the pass is sensitive to the size of its hot code,
+                // see mbar_wait_poll: cfg2 forward 506 -> 472 us)
+#ifndef SLICEMOE_DEV_OB
+#define SLICEMOE_DEV_OB 16
+#endif
+                constexpr int OB = SLICEMOE_DEV_OB;
                 static_assert(C::N2 % OB == 0, "output width");
-                const bool scatter = gather && p.scatter_out != nullptr;
+                const bool scatter = gather && (FUSED || p.scatter_out != nullptr);
                 const bool live = row < rows;
                 bf16* dst = nullptr;
-                if (live) dst = scatter ? p.scatter_out + (size_t)(pair_cur / p.gather_k) * C::N2
+                if (live) dst = scatter ? p.scatter_out + (size_t)pair_to_row(pair_cur, p.gather_magic, p.gather_shift) * C::N2
                                         : p.yperm + (size_t)(row0 + row) * C::N2;
 #pragma unroll 1
                 for (int cb = 0; cb < C::N2; cb += OB) {
@@ -1043,7 +1093,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     if constexpr (C::ROUTER) {
         // per-CTA histogram -> global counts (Section 3.2's per-expert counts)
         for (int i = threadIdx.x; i < p.experts_real; i += C::THREADS) {
-            if (p.assigned && sh.hist[i]) atomicAdd(&p.assigned[i], sh.hist[i]);
+            if (!FUSED && p.assigned && sh.hist[i]) atomicAdd(&p.assigned[i], sh.hist[i]);
             if (p.cta_hist) p.cta_hist[(size_t)blockIdx.x * p.experts_real + i] = sh.hist[i];
         }
     }

@@ -63,9 +63,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait: gives up after `limit_ns` or as soon as another thread raised *abort.
 // Returns false on give-up (and raises *abort itself when its own limit ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort,
-                                          uint64_t limit_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
+// The polling loop is one out-of-line function for all call sites: a third of all executed
+// instructions are such polls, and with a copy of the loop at each of the ~25 waits of the pipeline the
+// warps of an SM kept missing in the instruction cache (ncu: 93 % hit rate in the SM's instruction
+// cache, the next level's instruction port at 72 % of its peak).
+#ifndef SLICEMOE_DEV_INLINE_WAIT
+static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int* abort, uint64_t limit_ns) {
+#else
+__device__ __forceinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int* abort, uint64_t limit_ns) {
+#endif
     const uint64_t t0 = globaltimer_ns();
     for (;;) {
 #pragma unroll 1
@@ -77,6 +83,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort,
+                                          uint64_t limit_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_poll(bar, parity, abort, limit_ns);
 }
 
 // One lane of the (converged) warp.  The MMA-issuing warps run their loops with all 32 lanes and

@@ -179,7 +179,10 @@ struct TcCfg {
     // 256-wide rows (16 MMAs per chunk: 180 -> 176 us).  The other experts: one lane runs the loop;
     // their tile waits for the activation warps, and the wider issue warps only take issue slots from
     // those (64-wide rows: 260 -> 272 us with the router's scheme; 128-wide: no difference).
-    static constexpr bool UNIFORM_ISSUE = ROUTER_ || K1 == 256;
+#ifndef SLICEMOE_DEV_UNIFORM_ALL
+#define SLICEMOE_DEV_UNIFORM_ALL 0
+#endif
+    static constexpr bool UNIFORM_ISSUE = ROUTER_ || K1 == 256 || SLICEMOE_DEV_UNIFORM_ALL;
     static constexpr bool PACKED_ACT = !ROUTER_;
     // TMEM columns:
     //   [0, NBUF HC)         GEMM-1 accumulators.  Warpgroup w of the group that has the chunk owns
@@ -475,6 +478,12 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     if constexpr (C::ROUTER)
         for (int i = threadIdx.x; i < p.HID; i += C::THREADS)
             sh.bias1_f32[i] = p.bias1 ? __bfloat162float(p.bias1[i]) : 0.0f;
+    // experts without a first-layer bias: the ring the activation warps read their bias chunks from
+    // stays all zero (no loads into it), so that their loop has no second, bias-free copy
+    if constexpr (!C::ROUTER)
+        if (p.bias1 == nullptr)
+            for (int i = threadIdx.x; i < kBiasRing * C::B1_BYTES / 4; i += C::THREADS)
+                reinterpret_cast<uint32_t*>(smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_B1)[i] = 0u;
     if constexpr (C::ROUTER)
         for (int i = threadIdx.x; i < C::N2; i += C::THREADS)
             sh.bias2_f32[i] = i >= p.experts_real ? -INFINITY : (p.bias2 ? __bfloat162float(p.bias2[i]) : 0.0f);
@@ -886,7 +895,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #pragma unroll
                         for (int i = 0; i < C::SUB; ++i)
                             convert_piece_bf16x2(v[i], gate_hi, gate_lo, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
-                                                 p.bias1 != nullptr, z[s0 + i]);
+                                                 true, z[s0 + i]);
                     }
                     TRACE(tr, 32);
                     tc_fence_before_sync();

@@ -153,17 +153,31 @@ struct TcCfg {
 #ifndef SLICEMOE_DEV_GATHER4
 #define SLICEMOE_DEV_GATHER4 1
 #endif
-    static constexpr bool GATHER4 = FOUR_GROUPS && SLICEMOE_DEV_GATHER4;
+#ifndef SLICEMOE_DEV_GATHER4_WIDE
+#define SLICEMOE_DEV_GATHER4_WIDE 1
+#endif
+    // (256-wide rows: 32 copies per block of 32 rows, four times the 64-wide case; their CTA has room for
+    // another warpgroup)
+#ifndef SLICEMOE_DEV_G128
+#define SLICEMOE_DEV_G128 1
+#endif
+    // 128-wide expert rows: two groups of one warpgroup (instead of two groups of two), which frees a
+    // warpgroup for the gather (a third group would need a third accumulator, see NBUF >= NGRP below)
+    static constexpr bool ONE_WG_128 = !ROUTER_ && K1 == 128 && SLICEMOE_DEV_G128;
+    static constexpr bool GATHER4 = !ROUTER_ && ((FOUR_GROUPS && SLICEMOE_DEV_GATHER4) || (K1 == 256 && SLICEMOE_DEV_GATHER4_WIDE) || ONE_WG_128);
+    // the router of the single-kernel forward runs in the same CTA: same number of threads
+    static constexpr bool PAD_WARPGROUP = ROUTER_ && K1 == 256 && SLICEMOE_DEV_GATHER4_WIDE;
     static constexpr int GATHER_WARPS = GATHER4 ? 4 : 1;
     static constexpr int NGRP = (K1 == 256) ? 1 : (FOUR_GROUPS ? (GATHER4 ? 3 : 4) : 2);
-    static constexpr int GWG = FOUR_GROUPS ? 1 : 2;
+    static constexpr int GWG = (FOUR_GROUPS || ONE_WG_128) ? 1 : 2;
     static constexpr int NWG = NGRP * GWG;
     // GEMM-1 accumulator / hidden buffers.  The router's hidden pair lives inside the accumulator it
     // came from (see the TMEM map), which leaves room for a third accumulator: GEMM-1 of the next two
     // chunks can then be issued while GEMM-2 still reads this one.
     static constexpr int NBUF = ROUTER_ ? 3 : (FOUR_GROUPS ? 4 : 2);
     static constexpr int GRP_WARPS = GWG * 4;                   // warps that work on one chunk
-    static constexpr int THREADS = 128 + NWG * 128 + 128 + (GATHER4 ? 128 : 0);
+    // (ONE_WG_128: one more, idle, warpgroup so that the pass has the 768 threads of its router)
+    static constexpr int THREADS = 128 + NWG * 128 + 128 + ((GATHER4 || PAD_WARPGROUP) ? 128 : 0) + (ONE_WG_128 ? 128 : 0);
     static constexpr int OUT_WARP0 = 4 + NWG * 4;               // first warp of the output warpgroup
     static constexpr int ACC2_BUFS = (N2 <= 128) ? 2 : 1;
     // The router keeps the hidden layer as a bf16 pair (hi + lo = 16 mantissa bits): GEMM-2 runs
@@ -229,6 +243,11 @@ struct TcCfg {
     static_assert(N2 % 16 == 0 && N2 >= 16 && N2 <= 256, "MMA N");
     static_assert(SMEM_ALLOC <= 232448, "shared memory budget");
     static_assert(ACC2_COL0 + ACC2_BUFS * N2 <= 512, "TMEM budget");
+    // A group waits on an accumulator's "full" barrier only for its own chunks and so skips phases; the
+    // parity test of its next wait is only right if the phase before the awaited one is over by then.
+    // GEMM-1 finishes in chunk order and the group's previous chunk is NGRP chunks back, the barrier's
+    // previous phase NBUF chunks back: fine as long as NBUF >= NGRP.
+    static_assert(NBUF >= NGRP, "accumulator barriers: a group must not run a whole phase ahead");
 };
 
 // Barrier slots in shared memory.

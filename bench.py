@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # processes (traffic is proportional to rows: every row is read once per chosen expert and written once).
 NCU_TRAFFIC_CFG2 = {"route": 134.328064e6 + 142.558720e6, "dispatch": 17.735168e6 + 0.924928e6,
                     "expert_ffn": 451.720704e6 + 175.928320e6,
-                    "fused_forward": 579.980544e6 + 353.227520e6}
+                    "fused_forward": 578.811136e6 + 352.389888e6}
 NCU_TRAFFIC_ROWS_CFG2 = 65536 * 16
 
 

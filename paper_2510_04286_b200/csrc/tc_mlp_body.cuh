@@ -147,26 +147,18 @@ struct TcCfg {
     // 64-wide expert rows run four groups of one warpgroup on four 64-column chunks instead: the
     // warps of a sub-partition are then in four different phases, and a warp in its tanh phase is
     // more often there to use the unit while the others load, convert and store.
-    // 64-wide expert rows: three groups do as well as four (measured), and the warpgroup this frees
-    // gives the forward three more gather warps: each of the four then copies one block of 32 rows of a
-    // tile (see the gather warps).
-#ifndef SLICEMOE_DEV_GATHER4
-#define SLICEMOE_DEV_GATHER4 1
-#endif
-#ifndef SLICEMOE_DEV_GATHER4_WIDE
-#define SLICEMOE_DEV_GATHER4_WIDE 1
-#endif
-    // (256-wide rows: 32 copies per block of 32 rows, four times the 64-wide case; their CTA has room for
-    // another warpgroup)
-#ifndef SLICEMOE_DEV_G128
-#define SLICEMOE_DEV_G128 1
-#endif
-    // 128-wide expert rows: two groups of one warpgroup (instead of two groups of two), which frees a
-    // warpgroup for the gather (a third group would need a third accumulator, see NBUF >= NGRP below)
-    static constexpr bool ONE_WG_128 = !ROUTER_ && K1 == 128 && SLICEMOE_DEV_G128;
-    static constexpr bool GATHER4 = !ROUTER_ && ((FOUR_GROUPS && SLICEMOE_DEV_GATHER4) || (K1 == 256 && SLICEMOE_DEV_GATHER4_WIDE) || ONE_WG_128);
+    // Gather warps of the expert pass (forward): four, one per block of 32 rows of a tile (warp 3 and
+    // three warps of an extra warpgroup behind the output warpgroup), because a single warp's copies and
+    // address arithmetic were a bottleneck of the pass.  Where the warps come from:
+    //   64-wide rows   three activation groups do as well as four (measured): the fourth's warpgroup
+    //   128-wide rows  two groups of one warpgroup instead of two groups of two (a third group would
+    //                  need a third accumulator, see NBUF >= NGRP below)
+    //   256-wide rows  their CTA has room for another warpgroup (32 copies per block of rows here, four
+    //                  times the 64-wide case)
+    static constexpr bool ONE_WG_128 = !ROUTER_ && K1 == 128;
+    static constexpr bool GATHER4 = !ROUTER_ && (FOUR_GROUPS || K1 == 256 || ONE_WG_128);
     // the router of the single-kernel forward runs in the same CTA: same number of threads
-    static constexpr bool PAD_WARPGROUP = ROUTER_ && K1 == 256 && SLICEMOE_DEV_GATHER4_WIDE;
+    static constexpr bool PAD_WARPGROUP = ROUTER_ && K1 == 256;
     static constexpr int GATHER_WARPS = GATHER4 ? 4 : 1;
     static constexpr int NGRP = (K1 == 256) ? 1 : (FOUR_GROUPS ? (GATHER4 ? 3 : 4) : 2);
     static constexpr int GWG = (FOUR_GROUPS || ONE_WG_128) ? 1 : 2;
@@ -193,10 +185,7 @@ struct TcCfg {
     // 256-wide rows (16 MMAs per chunk: 180 -> 176 us).  The other experts: one lane runs the loop;
     // their tile waits for the activation warps, and the wider issue warps only take issue slots from
     // those (64-wide rows: 260 -> 272 us with the router's scheme; 128-wide: no difference).
-#ifndef SLICEMOE_DEV_UNIFORM_ALL
-#define SLICEMOE_DEV_UNIFORM_ALL 0
-#endif
-    static constexpr bool UNIFORM_ISSUE = ROUTER_ || K1 == 256 || SLICEMOE_DEV_UNIFORM_ALL;
+    static constexpr bool UNIFORM_ISSUE = ROUTER_ || K1 == 256;
     static constexpr bool PACKED_ACT = !ROUTER_;
     // TMEM columns:
     //   [0, NBUF HC)         GEMM-1 accumulators.  Warpgroup w of the group that has the chunk owns
@@ -1064,10 +1053,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 // (16 columns per turn of a rolled loop, not 64 unrolled: the shorter body is worth more
                 // than the saved accumulator-load waits -- the pass is sensitive to the size of its hot code,
                 // see mbar_wait_poll: cfg2 forward 506 -> 472 us)
-#ifndef SLICEMOE_DEV_OB
-#define SLICEMOE_DEV_OB 16
-#endif
-                constexpr int OB = SLICEMOE_DEV_OB;
+                constexpr int OB = 16;
                 static_assert(C::N2 % OB == 0, "output width");
                 const bool scatter = gather && (FUSED || p.scatter_out != nullptr);
                 const bool live = row < rows;

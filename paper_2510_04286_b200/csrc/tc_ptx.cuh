@@ -67,11 +67,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // instructions are such polls, and with a copy of the loop at each of the ~25 waits of the pipeline the
 // warps of an SM kept missing in the instruction cache (ncu: 93 % hit rate in the SM's instruction
 // cache, the next level's instruction port at 72 % of its peak).
-#ifndef SLICEMOE_DEV_INLINE_WAIT
 static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int* abort, uint64_t limit_ns) {
-#else
-__device__ __forceinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int* abort, uint64_t limit_ns) {
-#endif
     const uint64_t t0 = globaltimer_ns();
     for (;;) {
 #pragma unroll 1

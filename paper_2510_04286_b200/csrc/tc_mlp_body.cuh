@@ -232,10 +232,12 @@ struct TcCfg {
     static_assert(N2 % 16 == 0 && N2 >= 16 && N2 <= 256, "MMA N");
     static_assert(SMEM_ALLOC <= 232448, "shared memory budget");
     static_assert(ACC2_COL0 + ACC2_BUFS * N2 <= 512, "TMEM budget");
-    // A group waits on an accumulator's "full" barrier only for its own chunks and so skips phases; the
-    // parity test of its next wait is only right if the phase before the awaited one is over by then.
-    // GEMM-1 finishes in chunk order and the group's previous chunk is NGRP chunks back, the barrier's
-    // previous phase NBUF chunks back: fine as long as NBUF >= NGRP.
+    // A group waits on an accumulator's "full" barrier, and on a hidden buffer's "consumed" barrier, only
+    // for its own chunks and so skips phases; the parity test of its next wait is only right if the phase
+    // before the awaited one is over by then.  Both GEMMs finish in chunk order; the group's previous
+    // chunk is NGRP chunks back (its accumulator was complete, and the GEMM-2 that freed its hidden
+    // buffer was NGRP + NBUF chunks back), the barrier's previous phase NBUF (2 NBUF) chunks back: fine
+    // as long as NBUF >= NGRP.
     static_assert(NBUF >= NGRP, "accumulator barriers: a group must not run a whole phase ahead");
 };
 

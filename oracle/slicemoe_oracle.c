@@ -538,3 +538,148 @@ int slicemoe_oracle_gate_dropout(const double *topk_p /* [N, k] */, int64_t N, i
     }
     return ORACLE_OK;
 }
+
+/* ---- Backward of the layer -------------------------------------------------------------
+ *
+ * Section 3.1 trains router and experts end to end with the task loss, so the layer needs
+ * the gradient of a scalar loss L with respect to its input and all its weights, given
+ * gout = dL/dh'.  The paper prints no formulas for it; what follows is the chain rule on the
+ * forward exactly as stated above.  Readings: the top-k choice is piecewise constant, so it
+ * carries no gradient (the chosen ids are constants of the backward); the router learns
+ * through Eq. 1's gate, x~ = p_e x, where p is the softmax over ALL E experts (its Jacobian
+ * therefore reaches the logits of unchosen experts too); a pair dropped by the capacity
+ * contributed nothing forward and receives nothing backward; logit noise is an additive
+ * constant.  Cross-slice dropout's re-normalisation is not differentiated here (gates are the
+ * plain probabilities).
+ *
+ * Per row n (x = its slice, a = relu(Wr1 x + br1), p = softmax((Wr2 a + br2) / tau)) and kept
+ * pair j with expert e, gate p_e, z = W1_e (p_e x) + b1_e, u = act(z), y = W2_e u + b2_e:
+ *   dy = gout[n];  db2_e += dy;  dW2_e += dy u^T;  du = W2_e^T dy;  dz = du * act'(z);
+ *   db1_e += dz;  dW1_e += dz (p_e x)^T;  dx~ = W1_e^T dz;  dx += p_e dx~;  dp_e += <dx~, x>.
+ * Softmax: s = sum_e p_e dp_e;  dg_e = p_e (dp_e - s) / tau.
+ * Router:  dbr2 += dg;  dWr2 += dg a^T;  da = Wr2^T dg;  dpre = da * [a > 0];
+ *          dbr1 += dpre;  dWr1 += dpre x^T;  dx += Wr1^T dpre.
+ *
+ * Serial over rows, fp64; every gradient array is overwritten.  Bias gradients may be NULL.
+ * forced_idx as in slicemoe_oracle_forward.
+ * Pins (tests/test_oracle_backward.py): central finite differences of the (separately pinned)
+ * forward, reverse-mode differentiation by torch of an independently written fp64 forward,
+ * and closed forms (E = 1, identity experts, softmax-Jacobian invariants, dropped pairs).
+ */
+static double activation_grad(double z, int act) {
+    if (act == 0) return z > 0.0 ? 1.0 : 0.0;
+    const double c = 0.7978845608028654, b = 0.044715;
+    const double t = tanh(c * (z + b * z * z * z));
+    return 0.5 * (1.0 + t) + 0.5 * z * (1.0 - t * t) * c * (1.0 + 3.0 * b * z * z);
+}
+
+int slicemoe_oracle_backward(const oracle_cfg *c, const double *h,
+                             const double *Wr1, const double *br1,
+                             const double *Wr2, const double *br2,
+                             const double *W1, const double *b1,
+                             const double *W2, const double *b2,
+                             const int32_t *forced_idx, const double *gout,
+                             double *dh, double *dWr1, double *dbr1, double *dWr2, double *dbr2,
+                             double *dW1, double *db1, double *dW2, double *db2) {
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    const int ds = c->d / c->S, E = c->E, Hr = c->Hr, F = c->F, k = c->k;
+    const int64_t N = (int64_t)c->T * c->S, R = N * k;
+    const double tau = c->temperature > 0.0 ? c->temperature : 1.0;
+    (void)b2; /* the output bias does not enter any gradient */
+    int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
+    double *pk = (double *)malloc(sizeof(double) * (size_t)(R > 0 ? R : 1));
+    int64_t *dest = (int64_t *)malloc(sizeof(int64_t) * (size_t)(R > 0 ? R : 1));
+    int64_t *cnt = (int64_t *)malloc(sizeof(int64_t) * (size_t)(3 * E + 1));
+    double *a = (double *)malloc(sizeof(double) * (size_t)Hr);
+    double *p = (double *)malloc(sizeof(double) * (size_t)E);
+    double *dp = (double *)malloc(sizeof(double) * (size_t)E);
+    double *z = (double *)malloc(sizeof(double) * (size_t)F);
+    double *dz = (double *)malloc(sizeof(double) * (size_t)F);
+    double *dx = (double *)malloc(sizeof(double) * (size_t)ds);
+    rc = ORACLE_NO_MEMORY;
+    if (!idx || !pk || !dest || !cnt || !a || !p || !dp || !z || !dz || !dx) goto done;
+
+    /* the forward's routing and capacity decisions */
+    if (forced_idx) {
+        for (int64_t i = 0; i < R; ++i) {
+            if (forced_idx[i] < 0 || forced_idx[i] >= E) { rc = ORACLE_BAD_SHAPE; goto done; }
+            idx[i] = forced_idx[i];
+        }
+    } else {
+        rc = slicemoe_oracle_route(c, h, Wr1, br1, Wr2, br2, NULL, idx, pk, NULL, NULL);
+        if (rc) goto done;
+    }
+    rc = slicemoe_oracle_dispatch(c, idx, cnt, cnt + E, cnt + 2 * E, dest, NULL);
+    if (rc) goto done;
+
+    memset(dWr1, 0, sizeof(double) * (size_t)Hr * ds);
+    memset(dWr2, 0, sizeof(double) * (size_t)E * Hr);
+    memset(dW1, 0, sizeof(double) * (size_t)E * F * ds);
+    memset(dW2, 0, sizeof(double) * (size_t)E * ds * F);
+    if (dbr1) memset(dbr1, 0, sizeof(double) * (size_t)Hr);
+    if (dbr2) memset(dbr2, 0, sizeof(double) * (size_t)E);
+    if (db1) memset(db1, 0, sizeof(double) * (size_t)E * F);
+    if (db2) memset(db2, 0, sizeof(double) * (size_t)E * ds);
+
+    for (int64_t n = 0; n < N; ++n) {
+        const double *x = h + n * ds, *dy = gout + n * ds;
+        router_probs_row(c, n, x, Wr1, br1, Wr2, br2, a, p);
+        for (int q = 0; q < ds; ++q) dx[q] = 0.0;
+        for (int e = 0; e < E; ++e) dp[e] = 0.0;
+        for (int j = 0; j < k; ++j) {
+            if (dest[n * k + j] < 0) continue;
+            const int e = idx[n * k + j];
+            const double pe = p[e];
+            const double *W1e = W1 + (size_t)e * F * ds, *W2e = W2 + (size_t)e * ds * F;
+            double *dW1e = dW1 + (size_t)e * F * ds, *dW2e = dW2 + (size_t)e * ds * F;
+            for (int f = 0; f < F; ++f) {
+                double v = b1 ? b1[(size_t)e * F + f] : 0.0;
+                for (int q = 0; q < ds; ++q) v += W1e[(size_t)f * ds + q] * (pe * x[q]);
+                z[f] = v;
+            }
+            for (int f = 0; f < F; ++f) {
+                const double u = activation(z[f], c->act);
+                double du = 0.0;
+                for (int q = 0; q < ds; ++q) {
+                    du += W2e[(size_t)q * F + f] * dy[q];
+                    dW2e[(size_t)q * F + f] += dy[q] * u;
+                }
+                dz[f] = du * activation_grad(z[f], c->act);
+                if (db1) db1[(size_t)e * F + f] += dz[f];
+            }
+            if (db2) for (int q = 0; q < ds; ++q) db2[(size_t)e * ds + q] += dy[q];
+            for (int q = 0; q < ds; ++q) {
+                double dxt = 0.0;
+                for (int f = 0; f < F; ++f) {
+                    dxt += W1e[(size_t)f * ds + q] * dz[f];
+                    dW1e[(size_t)f * ds + q] += dz[f] * (pe * x[q]);
+                }
+                dx[q] += pe * dxt;
+                dp[e] += dxt * x[q];
+            }
+        }
+        double s = 0.0;
+        for (int e = 0; e < E; ++e) s += p[e] * dp[e];
+        for (int e = 0; e < E; ++e) dp[e] = p[e] * (dp[e] - s) / tau; /* dp now holds dg */
+        for (int e = 0; e < E; ++e) {
+            if (dbr2) dbr2[e] += dp[e];
+            for (int i = 0; i < Hr; ++i) dWr2[(size_t)e * Hr + i] += dp[e] * a[i];
+        }
+        for (int i = 0; i < Hr; ++i) {
+            double da = 0.0;
+            for (int e = 0; e < E; ++e) da += Wr2[(size_t)e * Hr + i] * dp[e];
+            const double dpre = a[i] > 0.0 ? da : 0.0;
+            if (dbr1) dbr1[i] += dpre;
+            for (int q = 0; q < ds; ++q) {
+                dWr1[(size_t)i * ds + q] += dpre * x[q];
+                dx[q] += Wr1[(size_t)i * ds + q] * dpre;
+            }
+        }
+        for (int q = 0; q < ds; ++q) dh[n * ds + q] = dx[q];
+    }
+    rc = ORACLE_OK;
+done:
+    free(idx); free(pk); free(dest); free(cnt); free(a); free(p); free(dp); free(z); free(dz); free(dx);
+    return rc;
+}

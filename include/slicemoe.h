@@ -291,6 +291,48 @@ int slicemoe_event_destroy(void *event);
 /* Milliseconds between two recorded events; synchronises on `stop`.  `ms` is a HOST out-pointer. */
 int slicemoe_event_elapsed_ms(void *start, void *stop, float *ms);
 
+/*
+ * Backward of the layer.  Section 3.1 trains router and experts end to end with
+ * the task loss; the paper prints no gradient formulas, so this is the chain
+ * rule on the forward as declared above: given grad_out = dL/dh' it returns
+ * dL/dh and the gradients of all weights.  Readings: the chosen expert ids
+ * (topk_idx, as returned by the forward) are constants; the router receives
+ * its gradient through Eq. 1's gate p_e x, p being the softmax over all E
+ * experts at temperature cfg->temperature; pairs dropped by cfg->capacity
+ * receive nothing (the forward's grouping is redone from topk_idx, same
+ * order, same drops); cross-slice dropout's re-normalisation is not
+ * differentiated (topk_p must be the router's own probabilities);
+ * cfg->noise_sigma > 0 is SLICEMOE_ERR_UNSUPPORTED.
+ *
+ * h, grad_out, grad_h: DEVICE [T, d] of cfg->dtype, 16-byte aligned; grad_h
+ * overlaps neither of the other two.  topk_idx int32 [N, k], topk_p float
+ * [N, k]: DEVICE, outputs of the forward on the same h and weights.
+ * Gradients of the weights: DEVICE fp32 whatever cfg->dtype, shaped like the
+ * weights, caller-owned; the four bias gradients may be NULL (skipped).  With
+ * accumulate == 0 the call first clears them, otherwise it adds to what they
+ * hold.  They are summed with fp32 atomics: values agree from run to run to
+ * fp32 rounding, not bit for bit; grad_h is deterministic.
+ * ws: DEVICE, 256-byte aligned, slicemoe_backward_workspace_bytes(cfg) bytes.
+ * fp32 arithmetic on CUDA cores; asynchronous on `stream`; no allocation, no
+ * host synchronisation.  Slices too wide for the kernels' shared-memory tiles
+ * (about ds > 2000): SLICEMOE_ERR_UNSUPPORTED.
+ */
+typedef struct {
+    float *dWr1; /* [Hr, ds]   */
+    float *dbr1; /* [Hr]       or NULL */
+    float *dWr2; /* [E, Hr]    */
+    float *dbr2; /* [E]        or NULL */
+    float *dW1;  /* [E, F, ds] */
+    float *db1;  /* [E, F]     or NULL */
+    float *dW2;  /* [E, ds, F] */
+    float *db2;  /* [E, ds]    or NULL */
+} slicemoe_grads;
+int slicemoe_backward_workspace_bytes(const slicemoe_config *cfg, size_t *bytes /* HOST out */);
+int slicemoe_backward(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
+                      const void *grad_out, const int32_t *topk_idx, const float *topk_p,
+                      void *grad_h, const slicemoe_grads *grads, int accumulate, void *ws,
+                      size_t ws_bytes, void *stream);
+
 /* Device status word of the last kernels that used `ws` (0 = fine, else a
  * slicemoe_status such as SLICEMOE_ERR_DEVICE_TIMEOUT).  Synchronises `stream`.
  * After a time-out it also puts the device's grid-barrier words, which the

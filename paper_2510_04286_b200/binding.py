@@ -24,7 +24,7 @@ EXPORTS = (
     "slicemoe_combine", "slicemoe_gate_dropout", "slicemoe_permute_columns", "slicemoe_load_stats", "slicemoe_forward", "slicemoe_forward_host", "slicemoe_forward_profiled",
     "slicemoe_event_create", "slicemoe_event_destroy", "slicemoe_event_elapsed_ms",
     "slicemoe_last_status", "slicemoe_launch_count", "slicemoe_last_cuda_error",
-    "slicemoe_status_string",
+    "slicemoe_status_string", "slicemoe_backward_workspace_bytes", "slicemoe_backward",
 )
 
 
@@ -269,6 +269,34 @@ def slicemoe_forward_profiled(cfg, w, h, h_out, ws, events: StageEvents, assigne
                                             _ptr(assigned), _ptr(kept), _ptr(topk_idx), _ptr(topk_p),
                                             _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(stream),
                                             events._ev), "slicemoe_forward_profiled")
+
+
+class _Grads(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("dWr1", "dbr1", "dWr2", "dbr2", "dW1", "db1", "dW2", "db2")]
+
+
+def slicemoe_backward_workspace_bytes(cfg: Config) -> int:
+    out = ctypes.c_size_t(0)
+    c = cfg.c()
+    _check(_lib().slicemoe_backward_workspace_bytes(ctypes.byref(c), ctypes.byref(out)),
+           "slicemoe_backward_workspace_bytes")
+    return int(out.value)
+
+
+def slicemoe_backward(cfg, w, h, grad_out, topk_idx, topk_p, grad_h, grads: dict, ws, accumulate=False,
+                      stream=None):
+    """Backward of the layer: grad_h and the fp32 weight gradients in ``grads`` (keys dWr1, dbr1,
+    dWr2, dbr2, dW1, db1, dW2, db2; bias entries may be missing) from grad_out = dL/dh'."""
+    import torch
+    c, ww = cfg.c(), _weights(w)
+    for name, t in grads.items():
+        if t is not None and (t.dtype != torch.float32 or not t.is_contiguous()):
+            raise ValueError(f"gradient {name} must be a contiguous float32 tensor")
+    gg = _Grads(*((None if grads.get(n) is None else grads[n].data_ptr())
+                  for n in ("dWr1", "dbr1", "dWr2", "dbr2", "dW1", "db1", "dW2", "db2")))
+    _check(_lib().slicemoe_backward(ctypes.byref(c), ctypes.byref(ww), _ptr(h), _ptr(grad_out), _ptr(topk_idx),
+                                    _ptr(topk_p), _ptr(grad_h), ctypes.byref(gg), ctypes.c_int(int(accumulate)),
+                                    _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(stream)), "slicemoe_backward")
 
 
 def slicemoe_last_status(ws, stream=None) -> int:

@@ -26,7 +26,7 @@ ACT_RELU = 0
 ACT_GELU_TANH = 1
 
 _TENSOR_IDS = {"h": 0, "Wr1": 1, "br1": 2, "Wr2": 3, "br2": 4,
-               "W1": 5, "b1": 6, "W2": 7, "b2": 8}
+               "W1": 5, "b1": 6, "W2": 7, "b2": 8, "grad_out": 9}
 
 
 @dataclass(frozen=True)
@@ -160,6 +160,11 @@ def zipf_router_bias(E: int, s: float) -> np.ndarray:
 def make_tokens(cfg: LayerConfig, seed: int = 0) -> np.ndarray:
     """h[T, d] ~ N(0, 1), rounded to the storage dtype."""
     return _normal(seed, "h", (cfg.T, cfg.d), 1.0, cfg.dtype)
+
+
+def make_grad_out(cfg: LayerConfig, seed: int = 0) -> np.ndarray:
+    """dL/dh'[T, d] ~ N(0, 1) for the backward, rounded to the storage dtype."""
+    return _normal(seed, "grad_out", (cfg.T, cfg.d), 1.0, cfg.dtype)
 
 
 def make_weights(cfg: LayerConfig, seed: int = 0) -> dict:

@@ -1,0 +1,149 @@
+"""GPU parity of slicemoe_backward against the oracle's backward (Section 3.1: the layer is trained
+end to end; gradients by the chain rule on the forward of Section 3.1 / Eq. 1).
+
+The GPU forward supplies the expert ids and gates; the oracle differentiates the same function on
+those ids (forced routing), so near-ties in the router cannot make the two sides differ.  The kernels
+compute in fp32 on the stored values, so every gradient is held to a relative Frobenius error of 1e-4
+(fp32 sums of up to a few thousand terms in an order that differs from the oracle's) and, element by
+element, to 1e-4 * max(1, rms); dL/dh of a bf16 layer is rounded to bf16 once on output, which alone
+is 2^-9 per element, hence 4e-3 there."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2510_04286_b200 import binding, synth
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+GRADS = ("dWr1", "dbr1", "dWr2", "dbr2", "dW1", "db1", "dW2", "db2")
+F32_FRO, BF16_DH_FRO, ELEM = 1e-4, 4e-3, 1e-4
+
+
+def run_backward(lc, seed=0, with_bias_grads=True, accumulate_twice=False):
+    import torch
+    h, w = synth.make_layer_inputs(lc, seed)
+    gout = synth.make_grad_out(lc, seed)
+    gpu = pu.GpuLayer(lc, h, w)
+    c = gpu.cfg
+    _, _, _, idx, p = gpu.forward()
+    g_dev = pu.tensors.to_torch(gout, lc.dtype, "cuda")
+    shapes = dict(dWr1=(c.Hr, c.ds), dbr1=(c.Hr,), dWr2=(c.E, c.Hr), dbr2=(c.E,), dW1=(c.E, c.F, c.ds),
+                  db1=(c.E, c.F), dW2=(c.E, c.ds, c.F), db2=(c.E, c.ds))
+    grads = {n: torch.full(s, 7.0, dtype=torch.float32, device="cuda") for n, s in shapes.items()
+             if with_bias_grads or not n.startswith("db")}
+    dh = torch.full((c.T, c.d), 3.0, dtype=gpu.tdtype, device="cuda")
+    ws = torch.empty(binding.slicemoe_backward_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    binding.slicemoe_backward(c, gpu.w, gpu.h, g_dev, idx, p, dh, grads, ws)
+    if accumulate_twice:
+        binding.slicemoe_backward(c, gpu.w, gpu.h, g_dev, idx, p, dh, grads, ws, accumulate=True)
+    torch.cuda.synchronize()
+    ref = oracle.backward(pu.oracle_config(lc), h, w, gout, forced_idx=idx.cpu().numpy())
+    got = {n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}
+    got["dh"] = pu.tensors.to_numpy_f32(dh).astype(np.float64)
+    return got, ref
+
+
+def compare(got, ref, lc, scale=1.0):
+    report = {}
+    for name, g in got.items():
+        r = ref[name] * scale
+        norm = np.linalg.norm(r)
+        fro = np.linalg.norm(g - r) / norm if norm > 0 else np.linalg.norm(g - r)
+        rms = norm / np.sqrt(max(r.size, 1))
+        mx = np.abs(g - r).max() if r.size else 0.0
+        bf16_dh = name == "dh" and lc.dtype == "bf16"
+        assert fro <= (BF16_DH_FRO if bf16_dh else F32_FRO), f"{name}: relative Frobenius error {fro:.3e}"
+        if bf16_dh:
+            assert np.all(np.abs(g - r) <= 2.0 ** -8 * np.abs(r) + ELEM * max(1.0, rms)), f"{name}: element off"
+        else:
+            assert mx <= ELEM * max(1.0, rms), f"{name}: max |diff| {mx:.3e} (rms {rms:.3e})"
+        report[name] = fro
+    return report
+
+
+CASES = {
+    "cfg0_fp32_relu_biases": synth.CONFIGS["cfg0"],
+    "cfg1_ragged": synth.CONFIGS["cfg1"].with_tokens(301),
+    "cfg2_E32": synth.CONFIGS["cfg2"].with_tokens(70),
+    "cfg3b_capacity_wide_rows": synth.CONFIGS["cfg3b"].with_tokens(96),
+    "cfg4_decode": synth.CONFIGS["cfg4"].with_tokens(24),
+    "paper768_k3": synth.CONFIGS["paper768_k3"].with_tokens(50),
+    "paper768_S32_narrow": synth.CONFIGS["paper768_S32"].with_tokens(20),
+    "temperature": replace(synth.CONFIGS["cfg1"].with_tokens(64), temperature=2.0),
+    "fp32_gelu_k1": replace(synth.CONFIGS["cfg0"], T=100, act=synth.ACT_GELU_TANH, k=1),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_backward_matches_oracle(name):
+    lc = CASES[name]
+    got, ref = run_backward(lc)
+    if lc.capacity:
+        assert np.abs(ref["dh"].reshape(lc.N, lc.ds)).max(axis=1).min() == 0.0, "no slice was dropped"
+    compare(got, ref, lc)
+
+
+def test_bias_gradients_optional_and_accumulation():
+    lc = synth.CONFIGS["cfg0"].with_tokens(64)
+    got, ref = run_backward(lc, with_bias_grads=False)
+    assert set(got) == {"dh", "dWr1", "dWr2", "dW1", "dW2"}
+    compare(got, ref, lc)
+    got2, ref2 = run_backward(lc, accumulate_twice=True)
+    dh = got2.pop("dh")
+    compare(got2, ref2, lc, scale=2.0)          # the second call added to the first
+    compare(dict(dh=dh), ref2, lc)              # dL/dh is overwritten, not accumulated
+
+
+def test_backward_is_deterministic_in_dh_and_stable_in_weights():
+    lc = synth.CONFIGS["cfg1"].with_tokens(200)
+    a, _ = run_backward(lc)
+    b, _ = run_backward(lc)
+    assert np.array_equal(a["dh"], b["dh"])
+    for n in GRADS:
+        assert np.allclose(a[n], b[n], rtol=1e-4, atol=1e-6)
+
+
+def test_backward_rejects_bad_arguments():
+    import torch
+    lc = synth.CONFIGS["cfg0"].with_tokens(16)
+    c = pu.tensors.config_from_synth(lc)
+    with pytest.raises(binding.SliceMoEError) as e:
+        binding.slicemoe_backward_workspace_bytes(replace(c, noise_sigma=0.5))
+    assert e.value.status == 3
+    h, w = synth.make_layer_inputs(lc, 0)
+    gpu = pu.GpuLayer(lc, h, w)
+    _, _, _, idx, p = gpu.forward()
+    grads = dict(dWr1=torch.zeros(c.Hr, c.ds, device="cuda"), dWr2=torch.zeros(c.E, c.Hr, device="cuda"),
+                 dW1=torch.zeros(c.E, c.F, c.ds, device="cuda"), dW2=torch.zeros(c.E, c.ds, c.F, device="cuda"))
+    ws = torch.empty(binding.slicemoe_backward_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    dh = torch.empty_like(gpu.h)
+    with pytest.raises(binding.SliceMoEError) as e:      # grad_h aliases h
+        binding.slicemoe_backward(c, gpu.w, gpu.h, dh, idx, p, gpu.h, grads, ws)
+    assert e.value.status == 6
+    with pytest.raises(binding.SliceMoEError) as e:      # workspace too small
+        binding.slicemoe_backward(c, gpu.w, gpu.h, dh, idx, p, dh.clone(), grads, ws[:256])
+    assert e.value.status == 5
+    with pytest.raises(binding.SliceMoEError) as e:      # a weight gradient is missing
+        binding.slicemoe_backward(c, gpu.w, gpu.h, dh, idx, p, dh.clone(), dict(grads, dW1=None), ws)
+    assert e.value.status == 1
+
+
+def test_backward_of_an_empty_batch():
+    import torch
+    lc = synth.CONFIGS["cfg0"].with_tokens(0)
+    c = pu.tensors.config_from_synth(lc)
+    _, w = synth.make_layer_inputs(lc, 0)
+    wd = pu.tensors.weights_to_torch(w, lc.dtype, "cuda")
+    grads = dict(dWr1=torch.ones(c.Hr, c.ds, device="cuda"), dWr2=torch.ones(c.E, c.Hr, device="cuda"),
+                 dW1=torch.ones(c.E, c.F, c.ds, device="cuda"), dW2=torch.ones(c.E, c.ds, c.F, device="cuda"))
+    ws = torch.empty(max(binding.slicemoe_backward_workspace_bytes(c), 256), dtype=torch.uint8, device="cuda")
+    e = torch.empty((0, c.d), device="cuda")   # empty tensors carry no address
+    idx = torch.empty((0, c.k), dtype=torch.int32, device="cuda")
+    p = torch.empty((0, c.k), dtype=torch.float32, device="cuda")
+    binding.slicemoe_backward(c, wd, e, e, idx, p, e, grads, ws)
+    torch.cuda.synchronize()
+    assert all(float(t.abs().max()) == 0.0 for t in grads.values())

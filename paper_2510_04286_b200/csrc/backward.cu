@@ -23,11 +23,13 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kFC = 256;  // hidden units per chunk of the expert kernel
 
-__device__ __forceinline__ float act_grad(float z, int act) {
-    if (act == SLICEMOE_ACT_RELU) return z > 0.0f ? 1.0f : 0.0f;
+// u = act(z) and du/dz with one tanh between them.
+__device__ __forceinline__ void act_and_grad(float z, int act, float& u, float& g) {
+    if (act == SLICEMOE_ACT_RELU) { u = fmaxf(z, 0.0f); g = z > 0.0f ? 1.0f : 0.0f; return; }
     const float c = 0.7978845608028654f, b = 0.044715f;
     const float t = tanhf(c * (z + b * z * z * z));
-    return 0.5f * (1.0f + t) + 0.5f * z * (1.0f - t * t) * c * (1.0f + 3.0f * b * z * z);
+    u = 0.5f * z * (1.0f + t);
+    g = 0.5f * (1.0f + t) + 0.5f * z * (1.0f - t * t) * c * (1.0f + 3.0f * b * z * z);
 }
 
 // Loads `rows` rows of width ds (row r from src + index[r]*ds) into dst as fp32, optionally scaled per
@@ -55,12 +57,42 @@ __device__ __forceinline__ void load_rows(float* dst, const T* __restrict__ src,
     }
 }
 
-// out[f, q..q+3] += sum_r A[r, f] * B[r, q..q+3] for f < nf, q < nq (A: [TM, lda], B: [TM, ldb] in shared
-// memory, fp32); out is global with row stride ldo.  One atomic per element.
+// out[f, q] += sum_r A[r, f] * B[r, q] for f < nf, q < nq (A: [TM, lda], B: [TM, ldb] in shared memory,
+// fp32; nq and ldb multiples of 4); out is global with row stride ldo.  One atomic per element.  A thread
+// owns a 4 x 4 block of `out` when nf and lda are multiples of 4 (two 16-byte shared-memory loads per 16
+// multiply-adds; with one row of four the loop is bound by shared-memory bandwidth), else a 1 x 4 block.
 template <int TM>
 __device__ __forceinline__ void outer_accumulate(float* __restrict__ out, int ldo, const float* A, int lda,
                                                  int nf, const float* B, int ldb, int nq) {
     const int q4n = nq >> 2;
+    if (((nf | lda) & 3) == 0) {
+        for (int it = threadIdx.x; it < (nf >> 2) * q4n; it += kThreads) {
+            const int f = (it / q4n) << 2, q = (it % q4n) << 2;
+            float s[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s[i][j] = 0.0f;
+#pragma unroll 4
+            for (int r = 0; r < TM; ++r) {
+                const float4 a = *reinterpret_cast<const float4*>(A + r * lda + f);
+                const float4 b = *reinterpret_cast<const float4*>(B + r * ldb + q);
+                const float av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    s[i][0] = fmaf(av[i], b.x, s[i][0]); s[i][1] = fmaf(av[i], b.y, s[i][1]);
+                    s[i][2] = fmaf(av[i], b.z, s[i][2]); s[i][3] = fmaf(av[i], b.w, s[i][3]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float* o = out + (size_t)(f + i) * ldo + q;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) atomicAdd(o + j, s[i][j]);
+            }
+        }
+        return;
+    }
     for (int it = threadIdx.x; it < nf * q4n; it += kThreads) {
         const int f = it / q4n, q = (it - f * q4n) << 2;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
@@ -75,37 +107,42 @@ __device__ __forceinline__ void outer_accumulate(float* __restrict__ out, int ld
     }
 }
 
-// acc[row, q] (+)= sum_{f < nf} Wt[f*ldw + q] * D[row, f]: the product with the transposed weight, W
-// read from global memory (coalesced over q), D [TM, ldd] from shared memory.  Work items are
-// (row group, q); returns through `sink(row, q, value)`.
-template <typename T, int TM, typename Sink>
-__device__ __forceinline__ void times_w_transposed(const T* __restrict__ Wt, int ldw, int nf, const float* D,
-                                                   int ldd, int nq, Sink sink) {
-    const int groups = nq >= kThreads ? 1 : min(TM, kThreads / nq);
-    const int rpg = (TM + groups - 1) / groups;
+// value(row, q) = sum_{f < nf} Wt[f*ldw + q] * D[row, f]: the product with the transposed weight, W read
+// from global memory (coalesced over q), D [TM, ldd] from shared memory, handed to `sink(row, q, value)`.
+// Work items are (group of RPG rows, q); RPG is a compile-time constant so that the row loop carries no
+// predicated-off iterations.
+template <typename T, int TM, int RPG, typename Sink>
+__device__ __forceinline__ void times_w_transposed_rpg(const T* __restrict__ Wt, int ldw, int nf, const float* D,
+                                                       int ldd, int nq, Sink sink) {
+    constexpr int groups = TM / RPG;
     for (int item = threadIdx.x; item < groups * nq; item += kThreads) {
         const int g = item / nq, q = item - g * nq;
-        float acc[TM];
+        const float* Dg = D + g * RPG * ldd;
+        float acc[RPG];
 #pragma unroll
-        for (int r = 0; r < TM; ++r) acc[r] = 0.0f;
+        for (int r = 0; r < RPG; ++r) acc[r] = 0.0f;
         for (int f = 0; f < nf; f += 4) {
             const float w0 = to_f32(Wt[(size_t)f * ldw + q]), w1 = to_f32(Wt[(size_t)(f + 1) * ldw + q]);
             const float w2 = to_f32(Wt[(size_t)(f + 2) * ldw + q]), w3 = to_f32(Wt[(size_t)(f + 3) * ldw + q]);
 #pragma unroll
-            for (int r = 0; r < TM; ++r) {
-                const int row = g * rpg + r;
-                if (r < rpg && row < TM) {
-                    const float4 dv = *reinterpret_cast<const float4*>(D + row * ldd + f);
-                    acc[r] = fmaf(w0, dv.x, fmaf(w1, dv.y, fmaf(w2, dv.z, fmaf(w3, dv.w, acc[r]))));
-                }
+            for (int r = 0; r < RPG; ++r) {
+                const float4 dv = *reinterpret_cast<const float4*>(Dg + r * ldd + f);
+                acc[r] = fmaf(w0, dv.x, fmaf(w1, dv.y, fmaf(w2, dv.z, fmaf(w3, dv.w, acc[r]))));
             }
         }
 #pragma unroll
-        for (int r = 0; r < TM; ++r) {
-            const int row = g * rpg + r;
-            if (r < rpg && row < TM) sink(row, q, acc[r]);
-        }
+        for (int r = 0; r < RPG; ++r) sink(g * RPG + r, q, acc[r]);
     }
+}
+
+// Picks the rows per group so that groups * nq covers the CTA's threads where it can.
+template <typename T, int TM, typename Sink>
+__device__ __forceinline__ void times_w_transposed(const T* __restrict__ Wt, int ldw, int nf, const float* D,
+                                                   int ldd, int nq, Sink sink) {
+    if (nq * 8 <= kThreads && TM >= 8) times_w_transposed_rpg<T, TM, (TM >= 8 ? TM / 8 : 1)>(Wt, ldw, nf, D, ldd, nq, sink);
+    else if (nq * 4 <= kThreads && TM >= 4) times_w_transposed_rpg<T, TM, (TM >= 4 ? TM / 4 : 1)>(Wt, ldw, nf, D, ldd, nq, sink);
+    else if (nq * 2 <= kThreads) times_w_transposed_rpg<T, TM, TM / 2>(Wt, ldw, nf, D, ldd, nq, sink);
+    else times_w_transposed_rpg<T, TM, TM>(Wt, ldw, nf, D, ldd, nq, sink);
 }
 
 // ---- expert kernel ------------------------------------------------------------------------------
@@ -198,8 +235,10 @@ bwd_expert_kernel(const T* __restrict__ h, const T* __restrict__ gout, const int
 #pragma unroll
             for (int r = 0; r < TM; ++r) {
                 const float z = acc[r] + b;
-                const float dz = du[r] * act_grad(z, act);
-                us[r * kFC + tid] = apply_act(z, act);
+                float u, g;
+                act_and_grad(z, act, u, g);
+                const float dz = du[r] * g;
+                us[r * kFC + tid] = u;
                 zs[r * kFC + tid] = dz;
                 bsum += dz;
             }
@@ -241,7 +280,8 @@ bwd_expert_kernel(const T* __restrict__ h, const T* __restrict__ gout, const int
 
 // ---- router kernel ------------------------------------------------------------------------------
 // Tile = TR consecutive rows.  Shared memory: xs = x [TR][ds], dxs [TR][ds], as = a, later dpre
-// [TR][Hr], gs = logits / tau, then p, then dg [TR][E].
+// [TR][Hr], gs = logits / tau, then p, then dg [TR][Eld], Eld = E | 1:
+// the odd row stride keeps the one-thread-per-row softmax off a single shared-memory bank.
 template <typename T, int TR>
 __global__ void __launch_bounds__(kThreads)
 bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ dest,
@@ -253,8 +293,10 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
     extern __shared__ __align__(16) float smem[];
     float* xs = smem;              // [TR][ds]
     float* dxs = xs + TR * ds;     // [TR][ds]
-    float* as = dxs + TR * ds;     // [TR][Hr]
-    float* gs = as + TR * Hr;      // [TR][E]
+    const int Hld = Hr + 4;        // row stride of as: rows land on different banks, 16-byte loads stay aligned
+    float* as = dxs + TR * ds;     // [TR][Hld]
+    float* gs = as + TR * Hld;     // [TR][Eld]
+    const int Eld = E | 1;
     __shared__ int row_of[TR];
     const int tid = threadIdx.x;
     const int n0 = blockIdx.x * TR, rows = min(TR, N - n0);
@@ -285,25 +327,26 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
             }
         }
 #pragma unroll
-        for (int r = 0; r < TR; ++r) as[r * Hr + i] = fmaxf(acc[r], 0.0f);
+        for (int r = 0; r < TR; ++r) as[r * Hld + i] = fmaxf(acc[r], 0.0f);
     }
     __syncthreads();
-    // logits / tau
+    // logits / tau.  The lanes of a warp take 32 rows of one expert: the weight row is one broadcast
+    // load for the warp (with the expert varying over the lanes it was 32 cache lines per load).
     for (int it = tid; it < TR * E; it += kThreads) {
-        const int r = it / E, e = it - r * E;
+        const int e = it / TR, r = it - e * TR;
         float g = br2 ? to_f32(br2[e]) : 0.0f;
         const T* wrow = Wr2 + (size_t)e * Hr;
         for (int i = 0; i < Hr; i += 4) {
-            const float4 av = *reinterpret_cast<const float4*>(as + r * Hr + i);
+            const float4 av = *reinterpret_cast<const float4*>(as + r * Hld + i);
             g = fmaf(to_f32(wrow[i]), av.x, fmaf(to_f32(wrow[i + 1]), av.y,
                 fmaf(to_f32(wrow[i + 2]), av.z, fmaf(to_f32(wrow[i + 3]), av.w, g))));
         }
-        gs[it] = g * inv_tau;
+        gs[r * Eld + e] = g * inv_tau;
     }
     __syncthreads();
     // softmax, then dg_e = p_e (dp_e - sum_m p_m dp_m) / tau with dp nonzero on the kept pairs only
     if (tid < TR) {
-        float* g = gs + tid * E;
+        float* g = gs + tid * Eld;
         if (tid < rows) {
             float m = -INFINITY, sum = 0.0f;
             for (int e = 0; e < E; ++e) m = fmaxf(m, g[e]);
@@ -328,11 +371,11 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
     if (dbr2) {
         for (int e = tid; e < E; e += kThreads) {
             float s = 0.0f;
-            for (int r = 0; r < TR; ++r) s += gs[r * E + e];
+            for (int r = 0; r < TR; ++r) s += gs[r * Eld + e];
             atomicAdd(dbr2 + e, s);
         }
     }
-    outer_accumulate<TR>(dWr2, Hr, gs, E, E, as, Hr, Hr);
+    outer_accumulate<TR>(dWr2, Hr, gs, Eld, E, as, Hld, Hr);
     __syncthreads();
     // dpre = (Wr2^T dg) * [a > 0], written over a by the thread that owns hidden unit i
     for (int i = tid; i < Hr; i += kThreads) {
@@ -342,21 +385,21 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
         for (int e = 0; e < E; ++e) {
             const float w = to_f32(Wr2[(size_t)e * Hr + i]);
 #pragma unroll
-            for (int r = 0; r < TR; ++r) da[r] = fmaf(w, gs[r * E + e], da[r]);
+            for (int r = 0; r < TR; ++r) da[r] = fmaf(w, gs[r * Eld + e], da[r]);
         }
         float bsum = 0.0f;
 #pragma unroll
         for (int r = 0; r < TR; ++r) {
-            const float v = as[r * Hr + i] > 0.0f ? da[r] : 0.0f;
-            as[r * Hr + i] = v;
+            const float v = as[r * Hld + i] > 0.0f ? da[r] : 0.0f;
+            as[r * Hld + i] = v;
             bsum += v;
         }
         if (dbr1) atomicAdd(dbr1 + i, bsum);
     }
     __syncthreads();
     // dWr1 += dpre x^T ; dL/dx = Wr1^T dpre + the kept pairs' shares from the expert kernel
-    outer_accumulate<TR>(dWr1, ds, as, Hr, Hr, xs, ds, ds);
-    times_w_transposed<T, TR>(Wr1, ds, Hr, as, Hr, ds, [&](int row, int q, float v) { dxs[row * ds + q] = v; });
+    outer_accumulate<TR>(dWr1, ds, as, Hld, Hr, xs, ds, ds);
+    times_w_transposed<T, TR>(Wr1, ds, Hr, as, Hld, ds, [&](int row, int q, float v) { dxs[row * ds + q] = v; });
     __syncthreads();
     for (int v = tid; v < rows * ds / V; v += kThreads) {
         const int r = (v * V) / ds, c = v * V - r * ds;
@@ -382,7 +425,7 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
 constexpr size_t kSmemBudget = 200 * 1024;
 
 size_t expert_smem(int TM, const Dims& D) { return sizeof(float) * (size_t)TM * (3 * (size_t)D.ds + 2 * kFC); }
-size_t router_smem(int TR, const Dims& D) { return sizeof(float) * (size_t)TR * (2 * (size_t)D.ds + D.Hr + D.E); }
+size_t router_smem(int TR, const Dims& D) { return sizeof(float) * (size_t)TR * (2 * (size_t)D.ds + D.Hr + 4 + (D.E | 1)); }
 
 struct BwdWorkspace {
     size_t kept, offsets, dest, perm, chunk_hist, dp, dxp, total;

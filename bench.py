@@ -9,7 +9,8 @@ through slicemoe_forward_host with pinned host buffers (copies inside the timed 
 path does not shard: with --gpus N every rank runs an independent replica on its own batch
 (weak scaling, no data-path collective) and `value` is the sum over ranks / max time.
 
-`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+The `backward` object of the line times slicemoe_backward on the same batches (up to 10 steps; not part
+of `value`).  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
@@ -313,6 +314,42 @@ def run_ours(args, lc):
     clocks.__exit__(None, None, None)
     stage_ms = np.mean([e.stage_ms() for e in ev], axis=0)
 
+    # ---- timed region 4: the backward (slicemoe_backward) on the same batches ----------------
+    # Not part of `value`: the headline metric is the forward.  Each set's expert ids and gates come
+    # from its own forward; grad_out is a seeded N(0, 1) batch per set.
+    bwd = None
+    try:
+        bws = torch.empty(sm.slicemoe_backward_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    except sm.SliceMoEError:
+        bws = None          # shape outside the backward kernels' tile set
+    if bws is not None:
+        idxs = [torch.empty((cfg.N, cfg.k), dtype=torch.int32, device="cuda") for _ in range(sets)]
+        gates = [torch.empty((cfg.N, cfg.k), dtype=torch.float32, device="cuda") for _ in range(sets)]
+        gouts = [tensors.to_torch(synth.make_grad_out(lc, seed=1000 * rank + s), lc.dtype) for s in range(sets)]
+        for s_ in range(sets):
+            sm.slicemoe_forward(cfg, w, hs[s_], outs[s_], ws, assigned, kept, idxs[s_], gates[s_])
+        shapes = dict(dWr1=(cfg.Hr, cfg.ds), dbr1=(cfg.Hr,), dWr2=(cfg.E, cfg.Hr), dbr2=(cfg.E,),
+                      dW1=(cfg.E, cfg.F, cfg.ds), db1=(cfg.E, cfg.F), dW2=(cfg.E, cfg.ds, cfg.F), db2=(cfg.E, cfg.ds))
+        grads = {n: torch.empty(sh, dtype=torch.float32, device="cuda") for n, sh in shapes.items()}
+        bsteps = max(1, min(args.steps, 10))
+
+        def bstep(i):
+            j = i % sets
+            sm.slicemoe_backward(cfg, w, hs[j], gouts[j], idxs[j], gates[j], outs[j], grads, bws)
+
+        for i in range(3):
+            bstep(i)
+        barrier()
+        l0 = sm.slicemoe_launch_count()
+        start.record()
+        for i in range(bsteps):
+            bstep(i)
+        stop.record()
+        barrier()
+        bwd = dict(t=start.elapsed_time(stop) / 1e3 / bsteps, steps=bsteps,
+                   launches_per_step=(sm.slicemoe_launch_count() - l0) // bsteps)
+        (bwd["t"],) = max_over_ranks([bwd["t"]], dist, device="cuda")
+
     t_dev, t_e2e = max_over_ranks([t_dev, t_e2e], dist, device="cuda")
 
     if rank == 0:
@@ -361,6 +398,18 @@ def run_ours(args, lc):
                                "frac": max(t_tensor, t_hbm) / t_step, "kept_rows": kept_rows,
                                "touched_experts": touched, "peak_source": f"of {peak_src}"},
         }
+        if bwd is not None:
+            # algorithmic work of a backward = twice the forward's (input and weight gradient of every
+            # product); the kernels also redo the forward's products (recompute factor 1.5).  fp32 on
+            # CUDA cores: the bound is the FMA pipes, 128 lanes x 2 FLOP per clock per SM.
+            alu_peak = N_SM * 128 * 2 * (clocks.summary()["sm_max_mhz"] or 1965.0) * 1e6 / 1e12
+            ach = 2.0 * work["total_flops"] / bwd["t"] / 1e12
+            line["backward"] = {
+                "ms_per_step": 1e3 * bwd["t"], "tokens_per_s": world * lc.T / bwd["t"], "steps": bwd["steps"],
+                "gpu_launches_per_step": int(bwd["launches_per_step"]), "dtype": "f32",
+                "roofline": {"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s",
+                             "frac": ach / alu_peak, "traffic": None,
+                             "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 FLOP x max SM clock"}}
         if world == 1 and not args.no_cpu_baseline:
             r = time_oracle(lc)
             line["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}

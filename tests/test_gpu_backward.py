@@ -147,3 +147,56 @@ def test_backward_of_an_empty_batch():
     binding.slicemoe_backward(c, wd, e, e, idx, p, e, grads, ws)
     torch.cuda.synchronize()
     assert all(float(t.abs().max()) == 0.0 for t in grads.values())
+
+
+def test_backward_full_size_cfg1_sampled_rows_and_invariants():
+    """configs[1] at its full size, as bench.py launches it.  dL/dh of a token depends on that token
+    alone (no capacity), so sampled tokens are graded against the oracle run on just those tokens with
+    the GPU's expert ids; the weight gradients, sums over all 131 072 slices, are checked through what
+    the mathematics fixes: db2 is the per-expert sum of grad_out over the slices routed there, the
+    logit gradients of every row sum to zero (so dbr2 and the columns of dWr2 do), and the weight
+    gradients of the first 2048 tokens alone match the oracle's."""
+    import torch
+    lc = synth.CONFIGS["cfg1"]
+    h, w = synth.make_layer_inputs(lc, 0)
+    gout = synth.make_grad_out(lc, 0)
+    gpu = pu.GpuLayer(lc, h, w)
+    c = gpu.cfg
+    _, _, _, idx, p = gpu.forward()
+    g_dev = pu.tensors.to_torch(gout, lc.dtype, "cuda")
+    shapes = dict(dWr1=(c.Hr, c.ds), dbr1=(c.Hr,), dWr2=(c.E, c.Hr), dbr2=(c.E,), dW1=(c.E, c.F, c.ds),
+                  db1=(c.E, c.F), dW2=(c.E, c.ds, c.F), db2=(c.E, c.ds))
+    grads = {n: torch.empty(s, dtype=torch.float32, device="cuda") for n, s in shapes.items()}
+    dh = torch.empty((c.T, c.d), dtype=gpu.tdtype, device="cuda")
+    ws = torch.empty(binding.slicemoe_backward_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    binding.slicemoe_backward(c, gpu.w, gpu.h, g_dev, idx, p, dh, grads, ws)
+    torch.cuda.synchronize()
+    idx_np = idx.cpu().numpy()
+    got = {n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}
+    dh_np = pu.tensors.to_numpy_f32(dh).astype(np.float64)
+
+    # sampled tokens (first, last, and a seeded draw), oracle on the sub-batch
+    rng = np.random.default_rng(7)
+    toks = np.unique(np.concatenate([[0, lc.T - 1], rng.integers(0, lc.T, 254)]))
+    sub = lc.with_tokens(len(toks))
+    rows = (toks[:, None] * lc.S + np.arange(lc.S)[None, :]).ravel()
+    ref = oracle.backward(pu.oracle_config(sub), h[toks], w, gout[toks], forced_idx=idx_np[rows])
+    compare(dict(dh=dh_np[toks]), ref, sub)
+
+    # db2[e] = sum of grad_out over the slices routed to e (each slice counts once per chosen expert)
+    G = gout.reshape(lc.N, lc.ds).astype(np.float64)
+    db2 = np.zeros((lc.E, lc.ds))
+    for j in range(lc.k):
+        np.add.at(db2, idx_np[:, j], G)
+    compare(dict(db2=got["db2"]), dict(db2=db2), lc)
+    scale = np.abs(got["dbr2"]).max()
+    assert scale > 0 and abs(got["dbr2"].sum()) <= 1e-4 * scale * lc.E
+    assert np.abs(got["dWr2"].sum(axis=0)).max() <= 1e-4 * np.abs(got["dWr2"]).max() * lc.E
+
+    # weight gradients of a 2048-token prefix against the oracle (the generator's prefix property)
+    pre = lc.with_tokens(2048)
+    binding.slicemoe_backward(pu.tensors.config_from_synth(pre), gpu.w, gpu.h[:2048], g_dev[:2048],
+                              idx[:pre.N], p[:pre.N], dh[:2048], grads, ws)
+    torch.cuda.synchronize()
+    ref = oracle.backward(pu.oracle_config(pre), h[:2048], w, gout[:2048], forced_idx=idx_np[:pre.N])
+    compare({n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}, ref, pre)

@@ -305,10 +305,11 @@ def forward_shuffled(cfg: OracleConfig, h, w: dict, perm, forced_idx=None) -> di
     return res
 
 
-def backward(cfg: OracleConfig, h, w: dict, grad_out, forced_idx=None) -> dict:
+def backward(cfg: OracleConfig, h, w: dict, grad_out, forced_idx=None, dropped=None) -> dict:
     """Gradients of a scalar loss with respect to the layer's input and weights, given
     ``grad_out`` = dL/dh' (chain rule on the forward of Section 3.1 / Eq. 1; the chosen expert
-    ids are constants, the gate p carries the router's gradient).  Keys: ``dh`` and ``dWr1``,
+    ids are constants, the gate p carries the router's gradient).  ``dropped[N, k]`` (the mask of
+    ``gate_dropout``) switches the gates to Section 3.3's re-normalised survivors.  Keys: ``dh`` and ``dWr1``,
     ``dbr1``, ``dWr2``, ``dbr2``, ``dW1``, ``db1``, ``dW2``, ``db2`` shaped like the weights."""
     lib, c = _load(), cfg.c()
     h = _f64(h, (cfg.T, cfg.d))
@@ -317,6 +318,9 @@ def backward(cfg: OracleConfig, h, w: dict, grad_out, forced_idx=None) -> dict:
     forced = None
     if forced_idx is not None:
         forced = np.ascontiguousarray(forced_idx, dtype=np.int32).reshape(cfg.N, cfg.k)
+    mask = None
+    if dropped is not None:
+        mask = np.ascontiguousarray(dropped, dtype=np.uint8).reshape(cfg.N, cfg.k)
     ds = cfg.ds
     out = dict(dh=np.empty((cfg.T, cfg.d), np.float64),
                dWr1=np.empty((cfg.Hr, ds), np.float64), dbr1=np.empty((cfg.Hr,), np.float64),
@@ -325,7 +329,7 @@ def backward(cfg: OracleConfig, h, w: dict, grad_out, forced_idx=None) -> dict:
                dW2=np.empty((cfg.E, ds, cfg.F), np.float64), db2=np.empty((cfg.E, ds), np.float64))
     _check(lib.slicemoe_oracle_backward(
         ctypes.byref(c), _p(h), _p(ww["Wr1"]), _p(ww["br1"]), _p(ww["Wr2"]), _p(ww["br2"]),
-        _p(ww["W1"]), _p(ww["b1"]), _p(ww["W2"]), _p(ww["b2"]), _p(forced), _p(g),
+        _p(ww["W1"]), _p(ww["b1"]), _p(ww["W2"]), _p(ww["b2"]), _p(forced), _p(mask), _p(g),
         _p(out["dh"]), _p(out["dWr1"]), _p(out["dbr1"]), _p(out["dWr2"]), _p(out["dbr2"]),
         _p(out["dW1"]), _p(out["db1"]), _p(out["dW2"]), _p(out["db2"])), "backward")
     return out

@@ -560,6 +560,14 @@ int slicemoe_oracle_gate_dropout(const double *topk_p /* [N, k] */, int64_t N, i
  * Router:  dbr2 += dg;  dWr2 += dg a^T;  da = Wr2^T dg;  dpre = da * [a > 0];
  *          dbr1 += dpre;  dWr1 += dpre x^T;  dx += Wr1^T dpre.
  *
+ * Train mode (Section 3.3): with `dropped` != NULL ([N*k], 1 = this assignment was dropped by
+ * cross-slice dropout) the gates are w_j = m_j p_j / Z, Z = sum_i m_i p_i over the row's k chosen
+ * experts (m = 1 - dropped), and the expert input is w_j x.  Then with dw_j = <dx~_j, x>:
+ *   dp_j = m_j (dw_j - sum_i w_i dw_i) / Z.
+ * A row whose k assignments were all dropped gives its first-listed expert the constant gate 1,
+ * which carries no gradient to the router.  A capacity-dropped pair has dw = 0 but its
+ * probability still sits in Z.
+ *
  * Serial over rows, fp64; every gradient array is overwritten.  Bias gradients may be NULL.
  * forced_idx as in slicemoe_oracle_forward.
  * Pins (tests/test_oracle_backward.py): central finite differences of the (separately pinned)
@@ -578,7 +586,7 @@ int slicemoe_oracle_backward(const oracle_cfg *c, const double *h,
                              const double *Wr2, const double *br2,
                              const double *W1, const double *b1,
                              const double *W2, const double *b2,
-                             const int32_t *forced_idx, const double *gout,
+                             const int32_t *forced_idx, const uint8_t *dropped, const double *gout,
                              double *dh, double *dWr1, double *dbr1, double *dWr2, double *dbr2,
                              double *dW1, double *db1, double *dW2, double *db2) {
     int rc = check_cfg(c);
@@ -586,6 +594,7 @@ int slicemoe_oracle_backward(const oracle_cfg *c, const double *h,
     const int ds = c->d / c->S, E = c->E, Hr = c->Hr, F = c->F, k = c->k;
     const int64_t N = (int64_t)c->T * c->S, R = N * k;
     const double tau = c->temperature > 0.0 ? c->temperature : 1.0;
+    if (k > 64) return ORACLE_BAD_SHAPE;
     (void)b2; /* the output bias does not enter any gradient */
     int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
     double *pk = (double *)malloc(sizeof(double) * (size_t)(R > 0 ? R : 1));
@@ -627,10 +636,21 @@ int slicemoe_oracle_backward(const oracle_cfg *c, const double *h,
         router_probs_row(c, n, x, Wr1, br1, Wr2, br2, a, p);
         for (int q = 0; q < ds; ++q) dx[q] = 0.0;
         for (int e = 0; e < E; ++e) dp[e] = 0.0;
+        /* gates: the plain probabilities (Eq. 1) or the re-normalised survivors (Section 3.3) */
+        double gate[64], dgate[64], Z = 0.0;
+        int survivors = 0;
+        for (int j = 0; j < k; ++j) {
+            dgate[j] = 0.0;
+            gate[j] = p[idx[n * k + j]];
+            if (dropped && !dropped[n * k + j]) { Z += gate[j]; ++survivors; }
+        }
+        if (dropped)
+            for (int j = 0; j < k; ++j)
+                gate[j] = survivors ? (dropped[n * k + j] ? 0.0 : gate[j] / Z) : (j == 0 ? 1.0 : 0.0);
         for (int j = 0; j < k; ++j) {
             if (dest[n * k + j] < 0) continue;
             const int e = idx[n * k + j];
-            const double pe = p[e];
+            const double pe = gate[j];
             const double *W1e = W1 + (size_t)e * F * ds, *W2e = W2 + (size_t)e * ds * F;
             double *dW1e = dW1 + (size_t)e * F * ds, *dW2e = dW2 + (size_t)e * ds * F;
             for (int f = 0; f < F; ++f) {
@@ -656,8 +676,16 @@ int slicemoe_oracle_backward(const oracle_cfg *c, const double *h,
                     dW1e[(size_t)f * ds + q] += dz[f] * (pe * x[q]);
                 }
                 dx[q] += pe * dxt;
-                dp[e] += dxt * x[q];
+                dgate[j] += dxt * x[q];
             }
+        }
+        if (!dropped) {
+            for (int j = 0; j < k; ++j) dp[idx[n * k + j]] += dgate[j];
+        } else if (survivors) {
+            double sw = 0.0;
+            for (int j = 0; j < k; ++j) sw += gate[j] * dgate[j];
+            for (int j = 0; j < k; ++j)
+                if (!dropped[n * k + j]) dp[idx[n * k + j]] += (dgate[j] - sw) / Z;
         }
         double s = 0.0;
         for (int e = 0; e < E; ++e) s += p[e] * dp[e];

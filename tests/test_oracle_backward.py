@@ -33,7 +33,7 @@ def make_case(seed, T=6, d=12, S=3, E=4, k=2, Hr=8, F=10, act=ACT_GELU_TANH, cap
 # ---------------------------------------------------------------------------------------------
 # reverse-mode differentiation by torch of a forward written here in plain tensor ops
 # ---------------------------------------------------------------------------------------------
-def torch_grads(cfg, h, w, gout, idx, dest):
+def torch_grads(cfg, h, w, gout, idx, dest, dropped=None):
     """L = <gout, h'> with h' from Section 3.1 / Eq. 1 on fixed expert ids; grads by autograd."""
     t = {n: torch.tensor(np.asarray(v), dtype=torch.float64, requires_grad=True) for n, v in w.items()}
     x = torch.tensor(h, dtype=torch.float64, requires_grad=True)
@@ -45,11 +45,17 @@ def torch_grads(cfg, h, w, gout, idx, dest):
     rows = []
     for n in range(cfg.N):
         y = torch.zeros(cfg.ds, dtype=torch.float64)
+        gates = [p[n, int(idx[n, j])] for j in range(cfg.k)]
+        if dropped is not None:     # Section 3.3: survivors re-normalised; all dropped -> top-1 gets 1
+            alive = [j for j in range(cfg.k) if not dropped[n, j]]
+            total = sum(gates[j] for j in alive) if alive else None
+            gates = [(gates[j] / total if j in alive else torch.tensor(0.0, dtype=torch.float64)) if alive
+                     else torch.tensor(1.0 if j == 0 else 0.0, dtype=torch.float64) for j in range(cfg.k)]
         for j in range(cfg.k):
             if dest[n, j] < 0:
                 continue
             e = int(idx[n, j])
-            z = t["W1"][e] @ (p[n, e] * X[n]) + (t["b1"][e] if "b1" in t else 0.0)
+            z = t["W1"][e] @ (gates[j] * X[n]) + (t["b1"][e] if "b1" in t else 0.0)
             u = torch.relu(z) if cfg.act == ACT_RELU else torch.nn.functional.gelu(z, approximate="tanh")
             y = y + t["W2"][e] @ u + (t["b2"][e] if "b2" in t else 0.0)
         rows.append(y)
@@ -205,3 +211,41 @@ def test_forced_routing_matches_own_routing():
     a, b = oracle.backward(cfg, h, w, gout), oracle.backward(cfg, h, w, gout, forced_idx=idx)
     for g in GRADS:
         assert np.array_equal(a[g], b[g])
+
+
+# ---------------------------------------------------------------------------------------------
+# train mode: the gates of cross-slice dropout (Section 3.3) inside the backward
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("kw,rate", [(dict(seed=71, T=10), 0.4), (dict(seed=72, k=3, E=6, T=10), 0.5),
+                                      (dict(seed=73, capacity=6, T=10), 0.3), (dict(seed=74), 0.0),
+                                      (dict(seed=75, k=1, E=3, T=12), 0.5)])
+def test_dropout_gates_backward_matches_autograd(kw, rate):
+    cfg, h, w, gout = make_case(**kw)
+    fwd = oracle.forward(cfg, h, w)
+    gates, dropped = oracle.gate_dropout(fwd["topk_p"], seed=5, rate=rate)
+    if rate > 0:
+        assert dropped.any() and (~dropped).any()
+        if cfg.k > 1:
+            assert dropped.all(axis=1).any() or rate < 0.5   # the all-dropped rule is usually exercised
+    ref, hp = torch_grads(cfg, h, w, gout, fwd["topk_idx"], fwd["dest"], dropped)
+    # the function differentiated is the staged train-mode chain of the oracle
+    xperm = oracle.weight_slices(cfg, h, gates, fwd["dest"], int(fwd["offsets"][-1]))
+    chain = oracle.combine(cfg, oracle.expert_ffn(cfg, xperm, fwd["offsets"], w), fwd["dest"])
+    np.testing.assert_allclose(hp, chain, rtol=0, atol=1e-12)
+    got = oracle.backward(cfg, h, w, gout, dropped=dropped)
+    for g in GRADS:
+        if g in ref:
+            scale = max(1.0, np.abs(ref[g]).max())
+            np.testing.assert_allclose(got[g], ref[g], rtol=0, atol=1e-11 * scale, err_msg=g)
+
+
+def test_dropout_rate_zero_differs_from_plain_gates():
+    """Rate 0 still re-normalises the k probabilities, so its gradients are not the inference ones."""
+    cfg, h, w, gout = make_case(81)
+    none = np.zeros((cfg.N, cfg.k), dtype=bool)
+    a, b = oracle.backward(cfg, h, w, gout), oracle.backward(cfg, h, w, gout, dropped=none)
+    assert np.abs(a["dWr2"] - b["dWr2"]).max() > 1e-6
+    # k = 1: the single survivor's gate is p / p = 1, a constant: the router gets no gradient
+    cfg1, h1, w1, g1 = make_case(82, k=1)
+    c = oracle.backward(cfg1, h1, w1, g1, dropped=np.zeros((cfg1.N, 1), dtype=bool))
+    assert np.abs(c["dWr2"]).max() == 0.0 and np.abs(c["dWr1"]).max() == 0.0

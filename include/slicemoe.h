@@ -300,12 +300,17 @@ int slicemoe_event_elapsed_ms(void *start, void *stop, float *ms);
  * its gradient through Eq. 1's gate p_e x, p being the softmax over all E
  * experts at temperature cfg->temperature; pairs dropped by cfg->capacity
  * receive nothing (the forward's grouping is redone from topk_idx, same
- * order, same drops); cross-slice dropout's re-normalisation is not
- * differentiated (topk_p must be the router's own probabilities);
- * cfg->noise_sigma > 0 is SLICEMOE_ERR_UNSUPPORTED.
+ * order, same drops); cfg->noise_sigma > 0 is SLICEMOE_ERR_UNSUPPORTED.
+ * dropout_gates == 0: topk_p holds the router's own probabilities (Eq. 1).
+ * dropout_gates != 0: topk_p holds the train-mode gates that
+ * slicemoe_gate_dropout made of them (Section 3.3), w_j = m_j p_j / Z with
+ * m_j = [w_j != 0] and Z the surviving probabilities' sum, and that
+ * re-normalisation is differentiated too: dL/dp_j = m_j (dL/dw_j -
+ * sum_i w_i dL/dw_i) / Z (zero for a lone survivor and for the constant gate
+ * 1 of the all-dropped rule).
  *
  * h, grad_out, grad_h: DEVICE [T, d] of cfg->dtype, 16-byte aligned; grad_h
- * overlaps neither of the other two.  topk_idx int32 [N, k], topk_p float
+ * overlaps neither of the other two (with T == 0 the data pointers may be NULL).  topk_idx int32 [N, k], topk_p float
  * [N, k]: DEVICE, outputs of the forward on the same h and weights.
  * Gradients of the weights: DEVICE fp32 whatever cfg->dtype, shaped like the
  * weights, caller-owned; the four bias gradients may be NULL (skipped).  With
@@ -330,8 +335,8 @@ typedef struct {
 int slicemoe_backward_workspace_bytes(const slicemoe_config *cfg, size_t *bytes /* HOST out */);
 int slicemoe_backward(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
                       const void *grad_out, const int32_t *topk_idx, const float *topk_p,
-                      void *grad_h, const slicemoe_grads *grads, int accumulate, void *ws,
-                      size_t ws_bytes, void *stream);
+                      void *grad_h, const slicemoe_grads *grads, int accumulate, int dropout_gates,
+                      void *ws, size_t ws_bytes, void *stream);
 
 /* Device status word of the last kernels that used `ws` (0 = fine, else a
  * slicemoe_status such as SLICEMOE_ERR_DEVICE_TIMEOUT).  Synchronises `stream`.

@@ -284,9 +284,10 @@ def slicemoe_backward_workspace_bytes(cfg: Config) -> int:
 
 
 def slicemoe_backward(cfg, w, h, grad_out, topk_idx, topk_p, grad_h, grads: dict, ws, accumulate=False,
-                      stream=None):
+                      dropout_gates=False, stream=None):
     """Backward of the layer: grad_h and the fp32 weight gradients in ``grads`` (keys dWr1, dbr1,
-    dWr2, dbr2, dW1, db1, dW2, db2; bias entries may be missing) from grad_out = dL/dh'."""
+    dWr2, dbr2, dW1, db1, dW2, db2; bias entries may be missing) from grad_out = dL/dh'.  With
+    ``dropout_gates`` topk_p holds the gates of slicemoe_gate_dropout (Section 3.3)."""
     import torch
     c, ww = cfg.c(), _weights(w)
     for name, t in grads.items():
@@ -296,7 +297,7 @@ def slicemoe_backward(cfg, w, h, grad_out, topk_idx, topk_p, grad_h, grads: dict
                   for n in ("dWr1", "dbr1", "dWr2", "dbr2", "dW1", "db1", "dW2", "db2")))
     _check(_lib().slicemoe_backward(ctypes.byref(c), ctypes.byref(ww), _ptr(h), _ptr(grad_out), _ptr(topk_idx),
                                     _ptr(topk_p), _ptr(grad_h), ctypes.byref(gg), ctypes.c_int(int(accumulate)),
-                                    _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(stream)), "slicemoe_backward")
+                                    ctypes.c_int(int(dropout_gates)), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream(stream)), "slicemoe_backward")
 
 
 def slicemoe_last_status(ws, stream=None) -> int:

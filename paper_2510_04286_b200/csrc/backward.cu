@@ -285,7 +285,7 @@ bwd_expert_kernel(const T* __restrict__ h, const T* __restrict__ gout, const int
 template <typename T, int TR>
 __global__ void __launch_bounds__(kThreads)
 bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ dest,
-                  const float* __restrict__ dp, const float* __restrict__ dxp,
+                  const float* __restrict__ dp, const float* __restrict__ dxp, const float* __restrict__ gates,
                   const T* __restrict__ Wr1, const T* __restrict__ br1, const T* __restrict__ Wr2,
                   const T* __restrict__ br2, float* __restrict__ dWr1, float* __restrict__ dbr1,
                   float* __restrict__ dWr2, float* __restrict__ dbr2, T* __restrict__ dh,
@@ -354,11 +354,28 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
             const float inv = 1.0f / sum;
             const int n = n0 + tid;
             for (int e = 0; e < E; ++e) g[e] *= inv;   // p
-            float s = 0.0f, pd[8];                      // k <= 8
-            for (int j = 0; j < k; ++j) {
-                const bool kept = dest[(size_t)n * k + j] >= 0;
-                pd[j] = kept ? g[topk_idx[(size_t)n * k + j]] * dp[(size_t)n * k + j] : 0.0f;
-                s += pd[j];
+            float s = 0.0f, pd[8];                      // k <= 8; pd[j] = p_j * dL/dp_j
+            if (!gates) {                               // Eq. 1: the gate is the probability itself
+                for (int j = 0; j < k; ++j) {
+                    const bool kept = dest[(size_t)n * k + j] >= 0;
+                    pd[j] = kept ? g[topk_idx[(size_t)n * k + j]] * dp[(size_t)n * k + j] : 0.0f;
+                    s += pd[j];
+                }
+            } else {
+                // Section 3.3: gate w_j = m_j p_j / Z over the row's chosen experts, m_j = [w_j != 0];
+                // dL/dp_j = m_j (dw_j - sum_i w_i dw_i) / Z.  A lone survivor, and the all-dropped rule's
+                // constant gate 1, come out as exactly zero.
+                float Z = 0.0f, sw = 0.0f, dw[8], gt[8];
+                for (int j = 0; j < k; ++j) {
+                    gt[j] = gates[(size_t)n * k + j];
+                    dw[j] = dest[(size_t)n * k + j] >= 0 ? dp[(size_t)n * k + j] : 0.0f;
+                    if (gt[j] != 0.0f) Z += g[topk_idx[(size_t)n * k + j]];
+                    sw = fmaf(gt[j], dw[j], sw);
+                }
+                for (int j = 0; j < k; ++j) {
+                    pd[j] = gt[j] != 0.0f ? g[topk_idx[(size_t)n * k + j]] * (dw[j] - sw) / Z : 0.0f;
+                    s += pd[j];
+                }
             }
             for (int e = 0; e < E; ++e) g[e] = -g[e] * s * inv_tau;
             for (int j = 0; j < k; ++j) g[topk_idx[(size_t)n * k + j]] += pd[j] * inv_tau;
@@ -470,13 +487,13 @@ int launch_expert(const Dims& D, const slicemoe_weights& w, const slicemoe_grads
 
 template <typename T, int TR>
 int launch_router(const Dims& D, const slicemoe_weights& w, const slicemoe_grads& g, const void* h,
-                  const int32_t* topk_idx, const int32_t* dest, const float* dp, const float* dxp, void* dh,
-                  cudaStream_t st) {
+                  const int32_t* topk_idx, const int32_t* dest, const float* dp, const float* dxp,
+                  const float* gates, void* dh, cudaStream_t st) {
     const size_t smem = router_smem(TR, D);
     auto kern = bwd_router_kernel<T, TR>;
     SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int grid = (D.N + TR - 1) / TR;
-    kern<<<grid, kThreads, smem, st>>>((const T*)h, topk_idx, dest, dp, dxp, (const T*)w.Wr1, (const T*)w.br1,
+    kern<<<grid, kThreads, smem, st>>>((const T*)h, topk_idx, dest, dp, dxp, gates, (const T*)w.Wr1, (const T*)w.br1,
                                       (const T*)w.Wr2, (const T*)w.br2, g.dWr1, g.dbr1, g.dWr2, g.dbr2, (T*)dh,
                                       D.N, D.ds, D.Hr, D.E, D.k, D.inv_tau);
     SLICEMOE_LAUNCH_CHECK(1);
@@ -486,15 +503,15 @@ int launch_router(const Dims& D, const slicemoe_weights& w, const slicemoe_grads
 template <typename T>
 int launch_typed(const Dims& D, const slicemoe_weights& w, const slicemoe_grads& g, const void* h, const void* gout,
                  const int32_t* topk_idx, const float* topk_p, const int32_t* offsets, const int32_t* dest,
-                 const int32_t* perm, float* dxp, float* dp, void* dh, cudaStream_t st) {
+                 const int32_t* perm, float* dxp, float* dp, const float* gates, void* dh, cudaStream_t st) {
     int rc;
     if (expert_smem(32, D) <= kSmemBudget)
         rc = launch_expert<T, 32>(D, w, g, h, gout, offsets, perm, topk_p, dxp, dp, st);
     else
         rc = launch_expert<T, 8>(D, w, g, h, gout, offsets, perm, topk_p, dxp, dp, st);
     if (rc) return rc;
-    if (router_smem(32, D) <= kSmemBudget) return launch_router<T, 32>(D, w, g, h, topk_idx, dest, dp, dxp, dh, st);
-    return launch_router<T, 8>(D, w, g, h, topk_idx, dest, dp, dxp, dh, st);
+    if (router_smem(32, D) <= kSmemBudget) return launch_router<T, 32>(D, w, g, h, topk_idx, dest, dp, dxp, gates, dh, st);
+    return launch_router<T, 8>(D, w, g, h, topk_idx, dest, dp, dxp, gates, dh, st);
 }
 
 }  // namespace
@@ -513,8 +530,8 @@ extern "C" int slicemoe_backward_workspace_bytes(const slicemoe_config* cfg, siz
 
 extern "C" int slicemoe_backward(const slicemoe_config* cfg, const slicemoe_weights* w, const void* h,
                                  const void* grad_out, const int32_t* topk_idx, const float* topk_p, void* grad_h,
-                                 const slicemoe_grads* grads, int accumulate, void* ws, size_t ws_bytes,
-                                 void* stream) {
+                                 const slicemoe_grads* grads, int accumulate, int dropout_gates, void* ws,
+                                 size_t ws_bytes, void* stream) {
     using namespace slicemoe;
     Dims D;
     int rc = make_dims(cfg, D);
@@ -560,10 +577,11 @@ extern "C" int slicemoe_backward(const slicemoe_config* cfg, const slicemoe_weig
     int32_t* chunk_hist = reinterpret_cast<int32_t*>(base + W.chunk_hist);
     float* dp = reinterpret_cast<float*>(base + W.dp);
     float* dxp = reinterpret_cast<float*>(base + W.dxp);
+    const float* gates = dropout_gates ? topk_p : nullptr;
     // the forward's grouping, redone from its expert ids (same stable order, same capacity drops)
     if ((rc = launch_dispatch(D, nullptr, topk_idx, topk_p, kept, offsets, dest, perm, nullptr, nullptr, chunk_hist, st)))
         return rc;
     if (D.dtype == SLICEMOE_BF16)
-        return launch_typed<bf16>(D, *w, *grads, h, grad_out, topk_idx, topk_p, offsets, dest, perm, dxp, dp, grad_h, st);
-    return launch_typed<float>(D, *w, *grads, h, grad_out, topk_idx, topk_p, offsets, dest, perm, dxp, dp, grad_h, st);
+        return launch_typed<bf16>(D, *w, *grads, h, grad_out, topk_idx, topk_p, offsets, dest, perm, dxp, dp, gates, grad_h, st);
+    return launch_typed<float>(D, *w, *grads, h, grad_out, topk_idx, topk_p, offsets, dest, perm, dxp, dp, gates, grad_h, st);
 }

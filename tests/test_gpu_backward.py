@@ -200,3 +200,36 @@ def test_backward_full_size_cfg1_sampled_rows_and_invariants():
     torch.cuda.synchronize()
     ref = oracle.backward(pu.oracle_config(pre), h[:2048], w, gout[:2048], forced_idx=idx_np[:pre.N])
     compare({n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}, ref, pre)
+
+
+@pytest.mark.parametrize("name,rate", [("cfg0", 0.2), ("cfg1", 0.5), ("paper768_k3", 0.5), ("cfg1", 0.0)])
+def test_train_mode_backward_with_dropout_gates(name, rate):
+    """Section 3.3 inside the backward: route -> slicemoe_gate_dropout -> slicemoe_backward with
+    dropout_gates, against the oracle's backward on the same expert ids and the oracle's own mask (the
+    masks of the two sides agree bit for bit: an integer compare of the same Philox word)."""
+    import torch
+    lc = synth.CONFIGS[name].with_tokens(120)
+    h, w = synth.make_layer_inputs(lc, 0)
+    gout = synth.make_grad_out(lc, 0)
+    gpu = pu.GpuLayer(lc, h, w)
+    c = gpu.cfg
+    idx, p, _, _ = gpu.route(want_probs=False)
+    p_plain = p.cpu().numpy().astype(np.float64)
+    binding.slicemoe_gate_dropout(c, p, 1234, rate)
+    _, dropped = oracle.gate_dropout(p_plain, 1234, rate)
+    gates = p.cpu().numpy()
+    assert np.array_equal(gates == 0.0, dropped & ~(dropped.all(axis=1, keepdims=True) & (np.arange(lc.k) == 0)))
+    g_dev = pu.tensors.to_torch(gout, lc.dtype, "cuda")
+    shapes = dict(dWr1=(c.Hr, c.ds), dbr1=(c.Hr,), dWr2=(c.E, c.Hr), dbr2=(c.E,), dW1=(c.E, c.F, c.ds),
+                  db1=(c.E, c.F), dW2=(c.E, c.ds, c.F), db2=(c.E, c.ds))
+    grads = {n: torch.empty(s, dtype=torch.float32, device="cuda") for n, s in shapes.items()}
+    dh = torch.empty((c.T, c.d), dtype=gpu.tdtype, device="cuda")
+    ws = torch.empty(binding.slicemoe_backward_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    binding.slicemoe_backward(c, gpu.w, gpu.h, g_dev, idx, p, dh, grads, ws, dropout_gates=True)
+    torch.cuda.synchronize()
+    ref = oracle.backward(pu.oracle_config(lc), h, w, gout, forced_idx=idx.cpu().numpy(), dropped=dropped)
+    got = {n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}
+    got["dh"] = pu.tensors.to_numpy_f32(dh).astype(np.float64)
+    compare(got, ref, lc)
+    if rate > 0:
+        assert dropped.any()

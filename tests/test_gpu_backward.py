@@ -23,11 +23,11 @@ GRADS = ("dWr1", "dbr1", "dWr2", "dbr2", "dW1", "db1", "dW2", "db2")
 F32_FRO, BF16_DH_FRO, ELEM = 1e-4, 4e-3, 1e-4
 
 
-def run_backward(lc, seed=0, with_bias_grads=True, accumulate_twice=False):
+def run_backward(lc, seed=0, with_bias_grads=True, accumulate_twice=False, drop_zero_biases=False):
     import torch
     h, w = synth.make_layer_inputs(lc, seed)
     gout = synth.make_grad_out(lc, seed)
-    gpu = pu.GpuLayer(lc, h, w)
+    gpu = pu.GpuLayer(lc, h, w, drop_zero_biases=drop_zero_biases)
     c = gpu.cfg
     _, _, _, idx, p = gpu.forward()
     g_dev = pu.tensors.to_torch(gout, lc.dtype, "cuda")
@@ -233,3 +233,31 @@ def test_train_mode_backward_with_dropout_gates(name, rate):
     compare(got, ref, lc)
     if rate > 0:
         assert dropped.any()
+
+
+@pytest.mark.parametrize("block", range(3))
+def test_backward_random_shapes(block):
+    """Seeded random shapes: widths inside and outside the tensor-core set, fp32 and bf16 storage,
+    expert counts that are not multiples of four, hidden widths that end in a partial chunk, k = 1..4,
+    ragged token counts, capacities, both activations, NULL bias pointers."""
+    import random
+    rnd = random.Random(2000 + block)
+    for it in range(8):
+        dtype = rnd.choice(["bf16", "bf16", "f32"])
+        V = 8 if dtype == "bf16" else 4
+        ds = rnd.choice([8, 24, 40, 64, 96, 128, 200, 256, 384])
+        ds -= ds % V
+        S = rnd.choice([1, 2, 4])
+        E = rnd.choice([3, 5, 8, 16, 21, 64])
+        k = min(E, rnd.choice([1, 2, 2, 3, 4]))
+        T = rnd.choice([1, 7, 33, 100, 250])
+        cap = max(1, int(rnd.uniform(0.3, 1.5) * T * S * k / E)) if rnd.random() < 0.3 else 0
+        lc = synth.LayerConfig(f"bwd_rand{block}_{it}", T=T, d=ds * S, S=S, E=E, k=k, F=V * rnd.randint(2, 70),
+                               Hr=V * rnd.choice([4, 16, 32, 40]), dtype=dtype, act=rnd.choice([0, 1]),
+                               init=rnd.choice(["normal", "kaiming"]), capacity=cap,
+                               wr2_gain=rnd.choice([1.0, 30.0]))
+        try:
+            got, ref = run_backward(lc, seed=it, drop_zero_biases=rnd.random() < 0.5)
+            compare(got, ref, lc)
+        except AssertionError as ex:
+            raise AssertionError(f"{lc}: {ex}") from ex

@@ -1,5 +1,5 @@
 /*
- * slicemoe.h -- C ABI of the B200 (sm_100a) SliceMoE layer forward.
+ * slicemoe.h -- C ABI of the B200 (sm_100a) SliceMoE layer: the forward and its backward.
  *
  * The layer (paper Section 3): a token vector h in R^d is cut into S contiguous
  * slices of ds = d/S elements.  A router MLP shared by all slices

@@ -311,7 +311,8 @@ int slicemoe_event_elapsed_ms(void *start, void *stop, float *ms);
  *
  * h, grad_out, grad_h: DEVICE [T, d] of cfg->dtype, 16-byte aligned; grad_h
  * overlaps neither of the other two (with T == 0 the data pointers may be NULL).  topk_idx int32 [N, k], topk_p float
- * [N, k]: DEVICE, outputs of the forward on the same h and weights.
+ * [N, k]: DEVICE, outputs of the forward on the same h and weights (an id
+ * outside [0, E) counts as not routed).
  * Gradients of the weights: DEVICE fp32 whatever cfg->dtype, shaped like the
  * weights, caller-owned; the four bias gradients may be NULL (skipped).  With
  * accumulate == 0 the call first clears them, otherwise it adds to what they

@@ -369,16 +369,21 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
                 for (int j = 0; j < k; ++j) {
                     gt[j] = gates[(size_t)n * k + j];
                     dw[j] = dest[(size_t)n * k + j] >= 0 ? dp[(size_t)n * k + j] : 0.0f;
-                    if (gt[j] != 0.0f) Z += g[topk_idx[(size_t)n * k + j]];
+                    const int e = topk_idx[(size_t)n * k + j];
+                    if (e < 0 || e >= E) gt[j] = 0.0f;              // an id outside [0, E) was never routed
+                    if (gt[j] != 0.0f) Z += g[e];
                     sw = fmaf(gt[j], dw[j], sw);
                 }
                 for (int j = 0; j < k; ++j) {
-                    pd[j] = gt[j] != 0.0f ? g[topk_idx[(size_t)n * k + j]] * (dw[j] - sw) / Z : 0.0f;
+                    pd[j] = (gt[j] != 0.0f && Z > 0.0f) ? g[topk_idx[(size_t)n * k + j]] * (dw[j] - sw) / Z : 0.0f;
                     s += pd[j];
                 }
             }
             for (int e = 0; e < E; ++e) g[e] = -g[e] * s * inv_tau;
-            for (int j = 0; j < k; ++j) g[topk_idx[(size_t)n * k + j]] += pd[j] * inv_tau;
+            for (int j = 0; j < k; ++j) {
+                const int e = topk_idx[(size_t)n * k + j];
+                if (e >= 0 && e < E) g[e] += pd[j] * inv_tau;   // ids outside [0, E) were never routed
+            }
         } else {
             for (int e = 0; e < E; ++e) g[e] = 0.0f;
         }

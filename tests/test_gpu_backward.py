@@ -261,3 +261,33 @@ def test_backward_random_shapes(block):
             compare(got, ref, lc)
         except AssertionError as ex:
             raise AssertionError(f"{lc}: {ex}") from ex
+
+
+def test_backward_ignores_expert_ids_outside_the_layer():
+    """An id outside [0, E) in topk_idx (never produced by the forward) is treated as not routed: the
+    other rows' dL/dh are bit-identical and nothing is read or written out of range."""
+    import torch
+    lc = synth.CONFIGS["cfg1"].with_tokens(40)
+    h, w = synth.make_layer_inputs(lc, 0)
+    gpu = pu.GpuLayer(lc, h, w)
+    c = gpu.cfg
+    _, _, _, idx, p = gpu.forward()
+    g_dev = pu.tensors.to_torch(synth.make_grad_out(lc, 0), lc.dtype, "cuda")
+    grads = dict(dWr1=torch.empty(c.Hr, c.ds, device="cuda"), dWr2=torch.empty(c.E, c.Hr, device="cuda"),
+                 dW1=torch.empty(c.E, c.F, c.ds, device="cuda"), dW2=torch.empty(c.E, c.ds, c.F, device="cuda"))
+    ws = torch.empty(binding.slicemoe_backward_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    dh_ok, dh_bad = torch.empty_like(gpu.h), torch.empty_like(gpu.h)
+    binding.slicemoe_backward(c, gpu.w, gpu.h, g_dev, idx, p, dh_ok, grads, ws)
+    bad = idx.clone()
+    bad[5, 0] = c.E + 3
+    bad[9, 1] = -2
+    for mode in (False, True):
+        binding.slicemoe_backward(c, gpu.w, gpu.h, g_dev, bad, p, dh_bad, grads, ws, dropout_gates=mode)
+        torch.cuda.synchronize()
+        assert all(bool(torch.isfinite(t).all()) for t in grads.values())
+        if not mode:
+            rows_ok = torch.ones(c.N, dtype=torch.bool, device="cuda")
+            rows_ok[5] = rows_ok[9] = False
+            a = dh_ok.reshape(c.N, c.ds)[rows_ok]
+            b = dh_bad.reshape(c.N, c.ds)[rows_ok]
+            assert torch.equal(a, b)

@@ -62,7 +62,7 @@ def load_peaks():
 
 
 # --------------------------------------------------------------------------------------------
-# workload arithmetic (algorithmic FLOPs / bytes; the design doc derives them)
+# workload arithmetic: algorithmic FLOPs (router 2N(ds Hr + Hr E), experts 4 R_kept ds F) and compulsory bytes
 # --------------------------------------------------------------------------------------------
 def layer_work(lc, kept_rows, touched_experts):
     b = 2 if lc.dtype == "bf16" else 4

@@ -149,15 +149,17 @@ def test_backward_of_an_empty_batch():
     assert all(float(t.abs().max()) == 0.0 for t in grads.values())
 
 
-def test_backward_full_size_cfg1_sampled_rows_and_invariants():
-    """configs[1] at its full size, as bench.py launches it.  dL/dh of a token depends on that token
-    alone (no capacity), so sampled tokens are graded against the oracle run on just those tokens with
-    the GPU's expert ids; the weight gradients, sums over all 131 072 slices, are checked through what
-    the mathematics fixes: db2 is the per-expert sum of grad_out over the slices routed there, the
-    logit gradients of every row sum to zero (so dbr2 and the columns of dWr2 do), and the weight
-    gradients of the first 2048 tokens alone match the oracle's."""
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3b"])
+def test_backward_full_size_sampled_rows_and_invariants(name):
+    """The named workloads at their full size, as bench.py launches them.  dL/dh of a kept slice depends
+    on that slice alone, so sampled slices are graded against the oracle run on just those slices as an
+    S = 1 layer of width ds (the reshape equivalence the forward oracle is pinned to) with the GPU's
+    expert ids; slices dropped by the capacity must come out as exact zeros.  The weight gradients, sums
+    over all slices, are checked through what the mathematics fixes: db2 is the per-expert sum of grad_out
+    over the kept pairs, the logit gradients of every row sum to zero (so dbr2 and the columns of dWr2 do);
+    without a capacity the weight gradients of a 2048-token prefix alone are compared with the oracle's."""
     import torch
-    lc = synth.CONFIGS["cfg1"]
+    lc = synth.CONFIGS[name]
     h, w = synth.make_layer_inputs(lc, 0)
     gout = synth.make_grad_out(lc, 0)
     gpu = pu.GpuLayer(lc, h, w)
@@ -173,33 +175,38 @@ def test_backward_full_size_cfg1_sampled_rows_and_invariants():
     torch.cuda.synchronize()
     idx_np = idx.cpu().numpy()
     got = {n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}
-    dh_np = pu.tensors.to_numpy_f32(dh).astype(np.float64)
+    dX = pu.tensors.to_numpy_f32(dh).astype(np.float64).reshape(lc.N, lc.ds)
+    X, G = h.reshape(lc.N, lc.ds), gout.reshape(lc.N, lc.ds)
+    kept = oracle.dispatch(pu.oracle_config(lc), idx_np)["dest"] >= 0            # [N, k]
 
-    # sampled tokens (first, last, and a seeded draw), oracle on the sub-batch
+    # sampled slices whose pairs were all kept (first, last and a seeded draw)
     rng = np.random.default_rng(7)
-    toks = np.unique(np.concatenate([[0, lc.T - 1], rng.integers(0, lc.T, 254)]))
-    sub = lc.with_tokens(len(toks))
-    rows = (toks[:, None] * lc.S + np.arange(lc.S)[None, :]).ravel()
-    ref = oracle.backward(pu.oracle_config(sub), h[toks], w, gout[toks], forced_idx=idx_np[rows])
-    compare(dict(dh=dh_np[toks]), ref, sub)
+    cand = np.flatnonzero(kept.all(axis=1))
+    rows = np.unique(np.concatenate([cand[:1], cand[-1:], rng.choice(cand, 2046)]))
+    sub = replace(lc, T=len(rows), d=lc.ds, S=1, capacity=0)
+    ref = oracle.backward(pu.oracle_config(sub), X[rows], w, G[rows], forced_idx=idx_np[rows])
+    compare(dict(dh=dX[rows]), ref, sub)
+    if lc.capacity:
+        gone = ~kept.any(axis=1)
+        assert gone.any() and np.abs(dX[gone]).max() == 0.0
 
-    # db2[e] = sum of grad_out over the slices routed to e (each slice counts once per chosen expert)
-    G = gout.reshape(lc.N, lc.ds).astype(np.float64)
+    # db2[e] = sum of grad_out over the pairs kept on e
     db2 = np.zeros((lc.E, lc.ds))
     for j in range(lc.k):
-        np.add.at(db2, idx_np[:, j], G)
+        np.add.at(db2, idx_np[kept[:, j], j], G[kept[:, j]].astype(np.float64))
     compare(dict(db2=got["db2"]), dict(db2=db2), lc)
     scale = np.abs(got["dbr2"]).max()
     assert scale > 0 and abs(got["dbr2"].sum()) <= 1e-4 * scale * lc.E
     assert np.abs(got["dWr2"].sum(axis=0)).max() <= 1e-4 * np.abs(got["dWr2"]).max() * lc.E
 
-    # weight gradients of a 2048-token prefix against the oracle (the generator's prefix property)
-    pre = lc.with_tokens(2048)
-    binding.slicemoe_backward(pu.tensors.config_from_synth(pre), gpu.w, gpu.h[:2048], g_dev[:2048],
-                              idx[:pre.N], p[:pre.N], dh[:2048], grads, ws)
-    torch.cuda.synchronize()
-    ref = oracle.backward(pu.oracle_config(pre), h[:2048], w, gout[:2048], forced_idx=idx_np[:pre.N])
-    compare({n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}, ref, pre)
+    if not lc.capacity and name == "cfg1":
+        # weight gradients of a 2048-token prefix against the oracle (the generator's prefix property)
+        pre = lc.with_tokens(2048)
+        binding.slicemoe_backward(pu.tensors.config_from_synth(pre), gpu.w, gpu.h[:2048], g_dev[:2048],
+                                  idx[:pre.N], p[:pre.N], dh[:2048], grads, ws)
+        torch.cuda.synchronize()
+        ref = oracle.backward(pu.oracle_config(pre), h[:2048], w, gout[:2048], forced_idx=idx_np[:pre.N])
+        compare({n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}, ref, pre)
 
 
 @pytest.mark.parametrize("name,rate", [("cfg0", 0.2), ("cfg1", 0.5), ("paper768_k3", 0.5), ("cfg1", 0.0)])

@@ -300,7 +300,8 @@ int slicemoe_event_elapsed_ms(void *start, void *stop, float *ms);
  * its gradient through Eq. 1's gate p_e x, p being the softmax over all E
  * experts at temperature cfg->temperature; pairs dropped by cfg->capacity
  * receive nothing (the forward's grouping is redone from topk_idx, same
- * order, same drops); cfg->noise_sigma > 0 is SLICEMOE_ERR_UNSUPPORTED.
+ * order, same drops); the logit noise of cfg->noise_sigma is a constant of the
+ * backward and is redrawn identically when the probabilities are recomputed.
  * dropout_gates == 0: topk_p holds the router's own probabilities (Eq. 1).
  * dropout_gates != 0: topk_p holds the train-mode gates that
  * slicemoe_gate_dropout made of them (Section 3.3), w_j = m_j p_j / Z with

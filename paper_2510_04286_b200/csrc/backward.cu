@@ -16,6 +16,7 @@
 // with one fp32 atomic per element and tile, so their summation order (not their value beyond fp32
 // rounding) varies from run to run; dL/dh is deterministic.
 #include "common.cuh"
+#include "philox.cuh"
 
 namespace slicemoe {
 namespace {
@@ -289,7 +290,7 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
                   const T* __restrict__ Wr1, const T* __restrict__ br1, const T* __restrict__ Wr2,
                   const T* __restrict__ br2, float* __restrict__ dWr1, float* __restrict__ dbr1,
                   float* __restrict__ dWr2, float* __restrict__ dbr2, T* __restrict__ dh,
-                  int N, int ds, int Hr, int E, int k, float inv_tau) {
+                  int N, int ds, int Hr, int E, int k, float inv_tau, float sigma, uint32_t key0, uint32_t key1) {
     extern __shared__ __align__(16) float smem[];
     float* xs = smem;              // [TR][ds]
     float* dxs = xs + TR * ds;     // [TR][ds]
@@ -341,6 +342,8 @@ bwd_router_kernel(const T* __restrict__ h, const int32_t* __restrict__ topk_idx,
             g = fmaf(to_f32(wrow[i]), av.x, fmaf(to_f32(wrow[i + 1]), av.y,
                 fmaf(to_f32(wrow[i + 2]), av.z, fmaf(to_f32(wrow[i + 3]), av.w, g))));
         }
+        // the forward's logit noise (Figure 6) is a constant of the backward, but the probabilities need it
+        if (sigma > 0.0f && r < rows) g = fmaf(sigma, logit_noise(n0 + r, e, key0, key1), g);
         gs[r * Eld + e] = g * inv_tau;
     }
     __syncthreads();
@@ -470,7 +473,6 @@ BwdWorkspace bwd_layout(const Dims& D) {
 }
 
 int bwd_supported(const Dims& D) {
-    if (D.noise_sigma > 0.0f) return SLICEMOE_ERR_UNSUPPORTED;
     if (expert_smem(8, D) > kSmemBudget || router_smem(8, D) > kSmemBudget) return SLICEMOE_ERR_UNSUPPORTED;
     return SLICEMOE_OK;
 }
@@ -500,7 +502,8 @@ int launch_router(const Dims& D, const slicemoe_weights& w, const slicemoe_grads
     const int grid = (D.N + TR - 1) / TR;
     kern<<<grid, kThreads, smem, st>>>((const T*)h, topk_idx, dest, dp, dxp, gates, (const T*)w.Wr1, (const T*)w.br1,
                                       (const T*)w.Wr2, (const T*)w.br2, g.dWr1, g.dbr1, g.dWr2, g.dbr2, (T*)dh,
-                                      D.N, D.ds, D.Hr, D.E, D.k, D.inv_tau);
+                                      D.N, D.ds, D.Hr, D.E, D.k, D.inv_tau, D.noise_sigma, (uint32_t)D.noise_seed,
+                                      (uint32_t)(D.noise_seed >> 32));
     SLICEMOE_LAUNCH_CHECK(1);
     return SLICEMOE_OK;
 }

@@ -24,4 +24,14 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// Figure 6's logit noise eps(n, e), a standard normal per (row, expert): Philox words x0, x1 of counter
+// (n, e, 1, 0), u_i = ((x_i >> 8) + 0.5) / 2^24 in (0, 1) (both exact in fp32), Box-Muller.
+__device__ __forceinline__ float logit_noise(int n, int e, uint32_t key0, uint32_t key1) {
+    uint32_t x[4];
+    philox4x32_10((uint32_t)n, (uint32_t)e, 1u, 0u, key0, key1, x);
+    const float u0 = ((float)(x[0] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    const float u1 = ((float)(x[1] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    return sqrtf(-2.0f * logf(u0)) * cospif(2.0f * u1);
+}
+
 }  // namespace slicemoe

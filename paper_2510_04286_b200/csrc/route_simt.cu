@@ -13,15 +13,6 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kMaxK = 8;
 
-// eps(n, e): u_i = ((x_i >> 8) + 0.5) / 2^24 in (0, 1), both exact in fp32.
-__device__ __forceinline__ float logit_noise(int n, int e, uint32_t key0, uint32_t key1) {
-    uint32_t x[4];
-    philox4x32_10((uint32_t)n, (uint32_t)e, 1u, 0u, key0, key1, x);
-    const float u0 = ((float)(x[0] >> 8) + 0.5f) * (1.0f / 16777216.0f);
-    const float u1 = ((float)(x[1] >> 8) + 0.5f) * (1.0f / 16777216.0f);
-    return sqrtf(-2.0f * logf(u0)) * cospif(2.0f * u1);
-}
-
 // One CTA routes ROWS consecutive rows.
 template <typename T, int ROWS>
 __global__ void __launch_bounds__(kThreads)

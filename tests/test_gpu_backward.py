@@ -75,6 +75,7 @@ CASES = {
     "paper768_S32_narrow": synth.CONFIGS["paper768_S32"].with_tokens(20),
     "temperature": replace(synth.CONFIGS["cfg1"].with_tokens(64), temperature=2.0),
     "fp32_gelu_k1": replace(synth.CONFIGS["cfg0"], T=100, act=synth.ACT_GELU_TANH, k=1),
+    "logit_noise": replace(synth.CONFIGS["cfg1"].with_tokens(64), noise_sigma=0.5, noise_seed=7, temperature=0.7),
 }
 
 
@@ -111,8 +112,8 @@ def test_backward_rejects_bad_arguments():
     import torch
     lc = synth.CONFIGS["cfg0"].with_tokens(16)
     c = pu.tensors.config_from_synth(lc)
-    with pytest.raises(binding.SliceMoEError) as e:
-        binding.slicemoe_backward_workspace_bytes(replace(c, noise_sigma=0.5))
+    with pytest.raises(binding.SliceMoEError) as e:      # slices too wide for the kernels' tiles
+        binding.slicemoe_backward_workspace_bytes(binding.Config(T=8, d=4096, S=1, E=4, k=1, F=64))
     assert e.value.status == 3
     h, w = synth.make_layer_inputs(lc, 0)
     gpu = pu.GpuLayer(lc, h, w)

@@ -209,11 +209,13 @@ def run_reference(args, lc):
     print(json.dumps(line))
 
 
-def workload_config(lc, sets):
+def workload_config(lc, sets, wsets=1):
+    l2 = (f"rotating {sets} distinct token/output buffer sets between steps (larger than the 126 MB L2)"
+          if sets > 1 else "single buffer set")
+    if wsets > 1:
+        l2 += f" and {wsets} copies of the weights (token sets alone would fit in L2 beside them)"
     return {"workload": lc.name, "T": lc.T, "d": lc.d, "S": lc.S, "E": lc.E, "k": lc.k, "F": lc.F,
-            "Hr": lc.Hr, "act": "gelu_tanh" if lc.act else "relu", "capacity": lc.capacity,
-            "l2": f"rotating {sets} distinct token/output buffer sets between steps "
-                  f"(larger than the 126 MB L2)" if sets > 1 else "single buffer set"}
+            "Hr": lc.Hr, "act": "gelu_tanh" if lc.act else "relu", "capacity": lc.capacity, "l2": l2}
 
 
 # --------------------------------------------------------------------------------------------
@@ -244,6 +246,12 @@ def run_ours(args, lc):
     # distinct seeded batches: rank r, set s draws seed 1000*r + s
     w_np = synth.make_weights(lc)
     w = tensors.weights_to_torch(w_np, lc.dtype)
+    # Small batches (decode) would leave everything L2-resident however many token sets rotate: the
+    # weights, their largest input, rotate too until tokens + weights exceed 2.2 x L2.
+    w_bytes = sum(int(t.numel()) * t.element_size() for t in w.values() if t is not None)
+    short = 2.2 * L2_BYTES - sets * set_bytes
+    wsets = int(max(1, min(16, -(-short // w_bytes)))) if short > 0 else 1
+    w_all = [w] + [{n: (None if t is None else t.clone()) for n, t in w.items()} for _ in range(wsets - 1)]
     hs = [tensors.to_torch(synth.make_tokens(lc, seed=1000 * rank + s), lc.dtype) for s in range(sets)]
     outs = [torch.empty((lc.T, lc.d), dtype=tdt, device="cuda") for _ in range(sets)]
     ws = sm.alloc_workspace(cfg)
@@ -251,7 +259,7 @@ def run_ours(args, lc):
     kept = torch.empty((lc.E,), dtype=torch.int32, device="cuda")
 
     def step(i):
-        sm.slicemoe_forward(cfg, w, hs[i % sets], outs[i % sets], ws, assigned, kept)
+        sm.slicemoe_forward(cfg, w_all[i % wsets], hs[i % sets], outs[i % sets], ws, assigned, kept)
 
     def barrier():
         if dist is not None:
@@ -309,7 +317,7 @@ def run_ours(args, lc):
         sm.slicemoe_forward_profiled(cfg, w, hs[i % sets], outs[i % sets], ws, ev[0], assigned, kept)
     barrier()
     for i in range(len(ev)):
-        sm.slicemoe_forward_profiled(cfg, w, hs[i % sets], outs[i % sets], ws, ev[i], assigned, kept)
+        sm.slicemoe_forward_profiled(cfg, w_all[i % wsets], hs[i % sets], outs[i % sets], ws, ev[i], assigned, kept)
     torch.cuda.synchronize()
     clocks.__exit__(None, None, None)
     stage_ms = np.mean([e.stage_ms() for e in ev], axis=0)
@@ -380,7 +388,7 @@ def run_ours(args, lc):
             "metric": "SliceMoE layer fwd tokens/s", "value": aggregate(shard_tokens(lc.T, world), args.steps, [t_dev]),
             "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": 1e3 * t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": lc.dtype, "data": "synthetic", "config": workload_config(lc, sets),
+            "dtype": lc.dtype, "data": "synthetic", "config": workload_config(lc, sets, wsets),
             "routed_slices_per_s": world * lc.R / t_step,
             "routing_stats": {"ele": ele, "l_cap_alpha_0.1": l_cap},
             "e2e": {"value": world * lc.T * args.steps / t_e2e, "unit": "tokens/s",

@@ -95,6 +95,9 @@ CONFIGS = {
     "cfg4": LayerConfig("cfg4", T=128, d=4096, S=32, E=64, k=2, F=512),
     # Same-E token-level MoE comparison (S = 1).
     "cfg4b": LayerConfig("cfg4b", T=128, d=4096, S=1, E=64, k=2, F=16384),
+    # Token-level MoE on the decode batch with the slice experts' hidden width (S = 1: slices are whole
+    # tokens); 0.5 GB of expert weights, small enough to generate and to grade against the oracle.
+    "cfg4_token": LayerConfig("cfg4_token", T=128, d=4096, S=1, E=64, k=2, F=512),
     # The paper's own model (Section 4): d = 768, S = 8 (96-wide slices), E = 16, k = 2; the expert
     # width F = 4 ds follows the other workloads, the batch is 32 sequences of 512 tokens.
     "paper768": LayerConfig("paper768", T=16384, d=768, S=8, E=16, k=2, F=384),

@@ -312,6 +312,13 @@ def test_forward_full_cfg4_decode():
     print("cfg4", rep)
 
 
+def test_forward_token_level_decode():
+    """The decode batch as a token-level MoE (S = 1: slices are whole tokens, 4096-wide rows) with the
+    slice experts' hidden width: the comparison workload beside cfg4, on the CUDA-core kernels."""
+    rep = pu.check_forward_against_oracle(C["cfg4_token"])
+    print("cfg4_token", rep)
+
+
 def test_forward_full_cfg3_capacity():
     for name in ("cfg3", "cfg3b"):
         rep = pu.check_forward_against_oracle(C[name], sample_rows=4096)

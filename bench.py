@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Throughput of the SliceMoE layer forward on B200, one JSON line per run.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl ours|reference] [--backward]
 
 A step is one whole layer forward (route -> dispatch -> expert FFN -> combine) over one batch of
 seeded synthetic tokens.  `value` is tokens/s with the inputs already in HBM; `e2e` is the same
@@ -9,8 +9,8 @@ through slicemoe_forward_host with pinned host buffers (copies inside the timed 
 path does not shard: with --gpus N every rank runs an independent replica on its own batch
 (weak scaling, no data-path collective) and `value` is the sum over ranks / max time.
 
-The `backward` object of the line times slicemoe_backward on the same batches (up to 10 steps; not part
-of `value`).  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+With --backward the line gains a `backward` object: slicemoe_backward timed on the same batches (up to 10
+steps; not part of `value`).  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
@@ -322,14 +322,17 @@ def run_ours(args, lc):
     clocks.__exit__(None, None, None)
     stage_ms = np.mean([e.stage_ms() for e in ev], axis=0)
 
-    # ---- timed region 4: the backward (slicemoe_backward) on the same batches ----------------
-    # Not part of `value`: the headline metric is the forward.  Each set's expert ids and gates come
+    # ---- timed region 4 (--backward): slicemoe_backward on the same batches -----------------
+    # Not part of `value`: the headline metric is the forward, and the default run launches the forward's
+    # kernels only.  Each set's expert ids and gates come
     # from its own forward; grad_out is a seeded N(0, 1) batch per set.
     bwd = None
-    try:
-        bws = torch.empty(sm.slicemoe_backward_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
-    except sm.SliceMoEError:
-        bws = None          # shape outside the backward kernels' tile set
+    bws = None
+    if args.backward:
+        try:
+            bws = torch.empty(sm.slicemoe_backward_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+        except sm.SliceMoEError:
+            bws = None      # shape outside the backward kernels' tile set
     if bws is not None:
         idxs = [torch.empty((cfg.N, cfg.k), dtype=torch.int32, device="cuda") for _ in range(sets)]
         gates = [torch.empty((cfg.N, cfg.k), dtype=torch.float32, device="cuda") for _ in range(sets)]
@@ -435,6 +438,8 @@ def main():
     ap.add_argument("--config", default="cfg1")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--backward", action="store_true",
+                    help="also time slicemoe_backward on the same batches (the `backward` object of the line)")
     args = ap.parse_args()
     from paper_2510_04286_b200 import synth
     lc = synth.CONFIGS[args.config]

@@ -376,7 +376,9 @@ def run_ours(args, lc):
     t_graph = None
     try:
         graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
+        # thread-local capture mode: CUDA calls of other threads (a process group's watchdog) do not
+        # invalidate the capture
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
             for i in range(args.steps):
                 step(i)
         graph.replay()

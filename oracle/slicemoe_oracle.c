@@ -1,5 +1,5 @@
 /*
- * fp64 CPU oracle of the SliceMoE layer forward.  TEST INFRASTRUCTURE ONLY.
+ * fp64 CPU oracle of the SliceMoE layer forward (and its backward).  TEST INFRASTRUCTURE ONLY.
  *
  * This file is the slow, plain statement of what the layer computes, written
  * from the paper's Section 3 / 3.1 / 3.4 and Eq. 1.  It shares no code with
@@ -27,7 +27,9 @@
  * dropout (tests/test_dropout.py) against the generator's published known-answer
  * vectors, a pure-Python restatement, and its invariants; router temperature and
  * logit noise (tests/test_router_knobs.py) against the log-odds identities of a
- * softmax, the limits tau -> 0 and infinity, and normality tests of the noise.
+ * softmax, the limits tau -> 0 and infinity, and normality tests of the noise; the backward
+ * (tests/test_oracle_backward.py) against finite differences of the forward, reverse-mode
+ * differentiation by torch of a separately written forward, and closed forms.
  * No function here is unpinned.
  */
 #include <math.h>
@@ -549,8 +551,8 @@ int slicemoe_oracle_gate_dropout(const double *topk_p /* [N, k] */, int64_t N, i
  * through Eq. 1's gate, x~ = p_e x, where p is the softmax over ALL E experts (its Jacobian
  * therefore reaches the logits of unchosen experts too); a pair dropped by the capacity
  * contributed nothing forward and receives nothing backward; logit noise is an additive
- * constant.  Cross-slice dropout's re-normalisation is not differentiated here (gates are the
- * plain probabilities).
+ * constant.  Without a dropout mask the gates are the plain probabilities; with one, see "Train
+ * mode" below.
  *
  * Per row n (x = its slice, a = relu(Wr1 x + br1), p = softmax((Wr2 a + br2) / tau)) and kept
  * pair j with expert e, gate p_e, z = W1_e (p_e x) + b1_e, u = act(z), y = W2_e u + b2_e:

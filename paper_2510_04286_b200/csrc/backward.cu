@@ -2,7 +2,8 @@
 // task loss).  Given gout = dL/dh', computes dL/dh and the gradients of all eight weight tensors by
 // the chain rule on the forward of Section 3.1 / Eq. 1.  The chosen expert ids are constants of the
 // backward; the router learns through Eq. 1's gate x~ = p_e x, p being the softmax over all E
-// experts; a pair dropped by the capacity receives nothing.
+// experts; a pair dropped by the capacity receives nothing.  With dropout_gates the gates are Section 3.3's
+// re-normalised survivors and that re-normalisation is differentiated as well; logit noise is redrawn.
 //
 // CUDA-core kernels, fp32 arithmetic in both storage types, weight gradients always fp32:
 //   1. the dispatch of the forward is redone from topk_idx (deterministic: same dest / perm / offsets)

@@ -299,3 +299,35 @@ def test_backward_ignores_expert_ids_outside_the_layer():
             a = dh_ok.reshape(c.N, c.ds)[rows_ok]
             b = dh_bad.reshape(c.N, c.ds)[rows_ok]
             assert torch.equal(a, b)
+
+
+def test_backward_through_shuffled_slices():
+    """Figure 5's shuffled layer: slicemoe_permute_columns around the forward and, for the gradient, around
+    slicemoe_backward (dL/dh = P^-1 backward(P h, P grad_out)); against the same composition of oracle calls."""
+    import torch
+    lc = synth.CONFIGS["cfg1"].with_tokens(90)
+    h, w = synth.make_layer_inputs(lc, 3)
+    gout = synth.make_grad_out(lc, 3)
+    perm_np = np.random.default_rng(5).permutation(lc.d).astype(np.int32)
+    gpu = pu.GpuLayer(lc, h, w)
+    c = gpu.cfg
+    perm = torch.from_numpy(perm_np).cuda()
+    g_dev = pu.tensors.to_torch(gout, lc.dtype, "cuda")
+    h_s, g_s = torch.empty_like(gpu.h), torch.empty_like(g_dev)
+    binding.slicemoe_permute_columns(c, gpu.h, h_s, perm)
+    binding.slicemoe_permute_columns(c, g_dev, g_s, perm)
+    gpu.h = h_s
+    _, _, _, idx, p = gpu.forward()
+    grads = dict(dWr1=torch.empty(c.Hr, c.ds, device="cuda"), dWr2=torch.empty(c.E, c.Hr, device="cuda"),
+                 dW1=torch.empty(c.E, c.F, c.ds, device="cuda"), dW2=torch.empty(c.E, c.ds, c.F, device="cuda"))
+    ws = torch.empty(binding.slicemoe_backward_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    dx, dh = torch.empty_like(h_s), torch.empty_like(h_s)
+    binding.slicemoe_backward(c, gpu.w, h_s, g_s, idx, p, dx, grads, ws)
+    binding.slicemoe_permute_columns(c, dx, dh, perm, inverse=True)
+    torch.cuda.synchronize()
+    ref = oracle.backward(pu.oracle_config(lc), oracle.permute_columns(h, perm_np), w,
+                          oracle.permute_columns(gout, perm_np), forced_idx=idx.cpu().numpy())
+    ref["dh"] = oracle.permute_columns(ref["dh"], perm_np, inverse=True)
+    got = {n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}
+    got["dh"] = pu.tensors.to_numpy_f32(dh).astype(np.float64)
+    compare(got, ref, lc)

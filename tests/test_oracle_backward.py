@@ -249,3 +249,34 @@ def test_dropout_rate_zero_differs_from_plain_gates():
     cfg1, h1, w1, g1 = make_case(82, k=1)
     c = oracle.backward(cfg1, h1, w1, g1, dropped=np.zeros((cfg1.N, 1), dtype=bool))
     assert np.abs(c["dWr2"]).max() == 0.0 and np.abs(c["dWr1"]).max() == 0.0
+
+
+def test_shuffled_slices_backward_is_the_permuted_backward():
+    """Figure 5's shuffled layer is h' = P^-1 layer(P h) with a column permutation P, so its input
+    gradient is P^-1 backward(P h, P gout) and the weight gradients are those of the inner layer.
+    Checked by finite differences of the (separately pinned) shuffled forward."""
+    cfg, h, w, gout = make_case(91, T=5, d=12, S=3)
+    perm = np.random.default_rng(3).permutation(cfg.d)
+    idx = oracle.forward_shuffled(cfg, h, w, perm)["topk_idx"]
+    inner = oracle.backward(cfg, oracle.permute_columns(h, perm), w, oracle.permute_columns(gout, perm),
+                            forced_idx=idx)
+    dh = oracle.permute_columns(inner["dh"], perm, inverse=True)
+
+    def loss(hh, ww):
+        return float((oracle.forward_shuffled(cfg, hh, ww, perm, forced_idx=idx)["h_out"] * gout).sum())
+
+    rng, eps = np.random.default_rng(4), 1e-5
+    for _ in range(8):
+        pos = (int(rng.integers(0, cfg.T)), int(rng.integers(0, cfg.d)))
+        hi, lo = h.copy(), h.copy()
+        hi[pos] += eps
+        lo[pos] -= eps
+        fd = (loss(hi, w) - loss(lo, w)) / (2 * eps)
+        assert abs(fd - dh[pos]) <= 2e-6 * max(1.0, abs(fd)), (pos, fd, dh[pos])
+    for name, g in (("W1", "dW1"), ("Wr1", "dWr1")):
+        pos = tuple(int(rng.integers(0, s)) for s in w[name].shape)
+        hi, lo = w[name].copy(), w[name].copy()
+        hi[pos] += eps
+        lo[pos] -= eps
+        fd = (loss(h, {**w, name: hi}) - loss(h, {**w, name: lo})) / (2 * eps)
+        assert abs(fd - inner[g][pos]) <= 2e-6 * max(1.0, abs(fd)), (name, pos)

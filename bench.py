@@ -38,6 +38,9 @@ NCU_TRAFFIC_CFG2 = {"route": 134.328064e6 + 142.558720e6, "dispatch": 17.735168e
                     "expert_ffn": 451.720704e6 + 175.928320e6,
                     "fused_forward": 578.811136e6 + 352.389888e6}
 NCU_TRAFFIC_ROWS_CFG2 = 65536 * 16
+# dram__bytes_read + dram__bytes_write of the two backward kernels on cfg1 (profiles/backward_cfg1.md)
+NCU_TRAFFIC_BACKWARD_CFG1 = (43.363072e6 + 26.524160e6) + (87.232256e6 + 5.461248e6)
+NCU_TRAFFIC_ROWS_CFG1 = 16384 * 8
 
 
 def ncu_traffic(stage, lc):
@@ -461,7 +464,9 @@ def run_ours(args, lc):
                 "ms_per_step": 1e3 * bwd["t"], "tokens_per_s": world * lc.T / bwd["t"], "steps": bwd["steps"],
                 "gpu_launches_per_step": int(bwd["launches_per_step"]), "dtype": "f32",
                 "roofline": {"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s",
-                             "frac": ach / alu_peak, "traffic": None,
+                             "frac": ach / alu_peak,
+                             "traffic": (NCU_TRAFFIC_BACKWARD_CFG1 * lc.N / NCU_TRAFFIC_ROWS_CFG1
+                                         if lc.ds == 64 and lc.k == 2 and lc.F == 256 else None),
                              "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 FLOP x max SM clock"}}
         if world == 1 and not args.no_cpu_baseline:
             r = time_oracle(lc)

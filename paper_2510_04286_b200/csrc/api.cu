@@ -159,6 +159,12 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
         return SLICEMOE_OK;
     };
     int rc;
+    // 64-wide slices without a capacity limit: the two-stream pipeline, as one launch or one per phase
+    if (pp_forward_supported(D)) {
+        if (events && clear_status && (rc = reset_status(ws, W, st))) return rc;
+        return launch_forward_pp(D, w, h, h_out, idx, p, assigned, kept, offsets, dest, xperm, at<int32_t>(ws, W.cta_hist),
+                                 at<int32_t>(ws, W.status), clear_status, /*one_launch=*/!events, events, st);
+    }
     const bool one_launch = !events && fused_forward_supported(D);
     // (the single kernel clears the status word itself; a later chunk of one host-buffer call keeps
     // what an earlier chunk reported)
@@ -511,8 +517,9 @@ int slicemoe_last_status(const void* ws, void* stream) {
     SLICEMOE_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
     if (word == SLICEMOE_ERR_DEVICE_TIMEOUT) {
         // a launch gave up inside a grid barrier: put the barrier words back in order
-        const int rc = slicemoe::fused_forward_reset_sync(static_cast<cudaStream_t>(stream));
+        int rc = slicemoe::fused_forward_reset_sync(static_cast<cudaStream_t>(stream));
         if (rc) return rc;
+        if ((rc = slicemoe::pp_forward_reset_sync(static_cast<cudaStream_t>(stream)))) return rc;
     }
     return word;
 }

@@ -132,6 +132,18 @@ int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h
                          cudaStream_t st);
 int fused_forward_reset_sync(cudaStream_t st);
 
+// The same forward on the two-stream pipeline (pp_body.cuh): 64-wide slices, k <= 2, no capacity limit.
+// one_launch: a single cooperative launch; otherwise one launch per phase with the stage events recorded.
+// dest doubles as the router's scratch for the pairs' ranks inside their CTA; pair_gate is int2[R]
+// (stacked row -> pair index and gate); the order of the stacked rows inside an expert is not the stable
+// (n, j) order of slicemoe_dispatch.
+bool pp_forward_supported(const Dims& D);
+int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
+                      float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest, void* pair_gate,
+                      int32_t* cta_hist, int32_t* status, bool clear_status, bool one_launch, void* const* events,
+                      cudaStream_t st);
+int pp_forward_reset_sync(cudaStream_t st);
+
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);
 

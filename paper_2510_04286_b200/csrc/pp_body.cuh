@@ -1,0 +1,1058 @@
+// Two-stream ("ping-pong") tensor-core pipeline for 64-wide slices, bf16 storage (sm_100a: tcgen05 +
+// TMEM + TMA), used by the forward of the layer (Section 3.1, Eq. 1; Section 3.4):
+//
+//   router  : relu(X Wr1^T + br1) Wr2^T + br2 -> softmax -> top-k, per 128-row tile
+//   experts : act(p (x W1_e^T) + b1_e) W2_e^T + b2_e, per 128-row tile of one expert's rows, rows gathered
+//             from h through the permutation and results added into h'
+//
+// A CTA of 384 threads (one per SM) walks a contiguous range of tiles; even tiles go to stream 0, odd
+// tiles to stream 1.  Each stream owns half of tensor memory (256 columns), one MMA-issuing warp and
+// one warpgroup of 128 "row" threads (thread r of the warpgroup owns tile row r for everything that
+// happens between the two GEMMs and after the second):
+//
+//   warp 0      TMA producer: weights (and the row tiles where they are not gathered)
+//   warp 1 / 2  MMA issue for stream 0 / 1: GEMM-1 of a 64-unit hidden chunk into a TMEM accumulator,
+//               GEMM-2 from the TMEM-resident hidden chunk into the stream's output accumulator
+//   warp 3      experts: gathers the rows of the next tiles (cp.async into the swizzled A buffers);
+//               router: zeroes this CTA's rows of h'
+//   warps 4-7   row threads of stream 0;  warps 8-11  row threads of stream 1
+//
+// While one stream's row threads evaluate the activation (the tanh unit is what bounds the expert
+// pass), the tensor pipe works on the other stream's GEMMs, and a stream's own GEMM-1 runs two chunks
+// ahead of its activation (two accumulators), so that a row thread seldom waits.  With a third of the
+// threads of a 24-warp layout every row thread has ~160 registers: a whole 64-column chunk is held in
+// fp32 and the activation is evaluated in fp32 (packed two-wide fp32 multiply-adds), 16 independent
+// column pairs at a time.  All hand-offs are mbarriers with bounded waits (status word on run-out).
+#pragma once
+#include "tc_mlp_body.cuh"
+
+namespace slicemoe {
+namespace {
+
+constexpr int kPpThreads = 768;
+#ifndef PP_SLEEP_NS
+#define PP_SLEEP_NS 100
+#endif
+constexpr int kPpABufs = 4;              // row-tile buffers
+constexpr int kPpABytes = 128 * 128;     // 128 rows x 64 bf16
+constexpr int kPpHC = 64;                // hidden units per chunk
+constexpr int kPpMaxF = 256;             // expert hidden width (both weight sets stay in shared memory)
+constexpr int kPpMaxHr = 512;            // router hidden width
+constexpr int kPpStreamCols = 256;       // TMEM columns per stream
+
+// ---- packed fp32 arithmetic (two lanes per instruction) -----------------------------------------
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void mul2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ float tanh_approx(float x) {
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(x));
+    return t;
+}
+// Bounded wait for the service warps (copies, MMA issue): between tries the warp sleeps, so that its polling
+// does not take issue slots from the row threads that share its scheduler.
+__device__ __forceinline__ bool mbar_try_wait_nohint(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+static __device__ __noinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, volatile int* abort, uint64_t limit_ns) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i) {
+            __nanosleep(PP_SLEEP_NS);
+            if (mbar_test_wait(bar, parity)) return true;
+        }
+        if (*abort) return false;
+        if (globaltimer_ns() - t0 > limit_ns) {
+            *abort = 1;
+            return false;
+        }
+    }
+}
+
+// Bounded wait of a whole (converged) warp.  (Inline, like everything the role loops call: an out-of-line
+// call costs a stack frame, and with ~200 KB of shared memory per CTA there is next to no L1 left for
+// local memory -- a kernel that spills runs every piece of scalar book-keeping at L2 latency.)
+__device__ __forceinline__ bool pp_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    return (bool)__all_sync(0xffffffffu, mbar_wait(bar, parity, abort, kWaitLimitNs));
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Adds `bytes` (a multiple of 16) of packed bf16 from shared memory to global memory, asynchronously, as one
+// operation of the copy engine (both addresses 16-byte aligned); completion is tracked by bulk groups.
+__device__ __forceinline__ void bulk_reduce_add_bf16(void* gdst, uint32_t smem_src, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.noftz.bf16 [%0], [%1], %2;"
+                 ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all bulk groups of this thread have finished reading their shared-memory source
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+#ifdef PP_TRACE
+__device__ unsigned long long g_pp_trace[40][4096];
+__device__ int g_pp_trace_on = 0;
+struct PpTr {
+    int n, slot; bool on;
+    __device__ PpTr(int slot_) : n(0), slot(slot_), on(blockIdx.x == 0 && (threadIdx.x & 31) == 0 && g_pp_trace_on) {}
+    __device__ void operator()(int code) { if (on && n < 4095) { g_pp_trace[slot][n++] = ((unsigned long long)code << 48) | (clock64() & 0xffffffffffffull); g_pp_trace[slot][n] = 0; } }
+};
+__device__ int g_pp_dbg = 0;
+#define DBG(bit) (g_pp_dbg & (bit))
+#define TRD(name, slot) PpTr name(slot)
+#define TR(name, code) name(code)
+#else
+#define TRD(name, slot)
+#define TR(name, code)
+#define DBG(bit) 0
+#endif
+
+// Shared-memory state of one CTA besides the operand tiles.
+struct PpShared {
+    __align__(8) uint64_t bars[48];
+    int tile_start[kMaxE + 1];
+    int offs[kMaxE + 1];
+    int hist[kMaxE];
+    uint32_t tmem_base;
+    int abort_flag;
+    // experts: first-layer bias of the run each stream is in, as fp32; router: br1 / br2 as fp32
+    __align__(16) float bias1_f32[2][kPpMaxHr];
+    __align__(16) float bias2_f32[kMaxE];
+};
+
+// Barrier slots.
+struct PpBars {
+    static constexpr int A_FULL = 0;                      // [kPpABufs]
+    static constexpr int A_EMPTY = A_FULL + kPpABufs;     // [kPpABufs]
+    static constexpr int W_FULL = A_EMPTY + kPpABufs;     // [2] weight sets (router: [0] only)
+    static constexpr int W_EMPTY = W_FULL + 2;            // [2] one arrival per stream
+    static constexpr int STREAM0 = W_EMPTY + 2;
+    // per stream (3 accumulator slots; the experts use two of them):
+    static constexpr int ACC1_FULL = 0, ACC1_EMPTY = 3, HID_FULL = 6, HID_EMPTY = 9, ACC2_FULL = 12, ACC2_EMPTY = 13;
+    static constexpr int PER_STREAM = 14;
+    static constexpr int DRAIN = STREAM0 + 2 * PER_STREAM;   // [2]
+    static constexpr int COUNT = DRAIN + 2;
+};
+static_assert(PpBars::COUNT <= 48, "barrier slots");
+
+// Walks the CTA's tile list in order; `run` counts the expert changes seen so far (a run = consecutive
+// tiles of one expert = one weight set).
+struct PpWalk {
+    int ta, e, run, row0, rows;
+    __device__ __forceinline__ void init() { ta = -1; e = 0; run = 0; row0 = 0; rows = 0; }
+    // advances to local tile `to` (> ta); returns through `crossed` how many run boundaries were passed
+    __device__ __forceinline__ int advance(const PpShared& sh, int t_begin, int to) {
+        int crossed = 0;
+        while (ta < to) {
+            ++ta;
+            const int e_prev = e;
+            locate_tile(sh.tile_start, sh.offs, t_begin + ta, e, row0, rows);
+            if (ta > 0 && e != e_prev) { ++run; ++crossed; }
+        }
+        return crossed;
+    }
+};
+
+struct PpParams {
+    // ---- both passes
+    int32_t* status;
+    int n_rows;                 // router: N; experts: R
+    int HID;                    // Hr or F (multiple of 64)
+    // ---- router
+    int experts_real;           // E (<= the padded width the kernel is built for)
+    int k;
+    float softmax_scale;        // log2(e) / tau
+    const bf16* br1;            // [Hr] or nullptr
+    const bf16* br2;            // [E] or nullptr
+    int32_t* topk_idx;          // [N, k]
+    float* topk_p;              // [N, k]
+    int32_t* local_rank;        // [N, k] rank of the pair among this CTA's pairs of the same expert
+    int32_t* cta_hist;          // [grid, E]
+    bf16* zero_out;             // h' as [N, 64]: this CTA zeroes the rows it routes (or nullptr)
+    // ---- experts
+    int E;
+    const int32_t* offsets;     // [E + 1] (read when the offsets are not already in shared memory)
+    const bf16* b1;             // [E, F] or nullptr
+    const bf16* b2;             // [E, 64] or nullptr
+    const bf16* gather_src;     // h as X[N, 64]
+    const int2* pair_gate;      // [R] stacked row -> (pair index n k + j, gate as float bits)
+    uint32_t gather_magic, gather_shift;
+    bf16* scatter_out;          // h' as Y[N, 64]
+    int row_elems;              // real slice width (<= 64)
+};
+
+__device__ __forceinline__ uint32_t pp_bar(PpShared& sh, int i) { return smem_u32(&sh.bars[i]); }
+__device__ __forceinline__ uint32_t pp_sbar(PpShared& sh, int s, int i) {
+    return smem_u32(&sh.bars[PpBars::STREAM0 + s * PpBars::PER_STREAM + i]);
+}
+
+// First tile of every expert (exclusive scan of the tile counts), by warp 0.
+__device__ __forceinline__ void pp_tile_starts(PpShared& sh, int E, int lane) {
+    int run = 0;
+    for (int e0 = 0; e0 < E; e0 += 32) {
+        const int e = e0 + lane;
+        const int nt = e < E ? (sh.offs[e + 1] - sh.offs[e] + kTileM - 1) / kTileM : 0;
+        int incl = nt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (e < E) sh.tile_start[e] = run + incl - nt;
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) sh.tile_start[E] = run;
+}
+
+// =====================================================================================================
+// Expert pass.  N2: real slice width (48 or 64) = N of the second GEMM; F in {128, 256}.
+// Shared memory (1024-aligned): A buffers 4 x 16 KB | weight set 0 | weight set 1, a set = W1 [F, 64]
+// (F/64 panels of 8 KB) then W2 as F/64 panels [N2, 64] of N2 x 128 B each.
+//
+// One stream of tiles; tile t works in tensor-memory region t mod 2 (256 columns each):
+//   GEMM-1 of the whole hidden width (N = F) into columns [0, F) of the region;
+//   the 16 row-thread warps (4 warpgroups x 4 lane groups) turn it into the hidden layer: warpgroup g
+//   owns hidden units [32 g, 32 g + 32) and (F = 256) [128 + 32 g, 128 + 32 g + 32); a thread reads 32
+//   fp32 columns of its row, applies gate, bias and activation in fp32 and writes 16 packed bf16
+//   columns over accumulator columns it has already read: [32 g, 32 g + 16) and [32 g + 16, 32 g + 32),
+//   so the hidden layer ends up in columns [0, 128) and columns [128, 192) are free for
+//   GEMM-2's accumulator by the time all hidden values are written;
+//   GEMM-2 reads the hidden layer from tensor memory (K step by K step) into [128, 128 + N2);
+//   the output step (0.5 acc + b2 -> bf16 -> add into h') of tile t runs in the middle of tile t + 1's
+//   activation, each warpgroup on 16 of the 64 output columns.
+// A row thread waits on two barriers per tile, both usually long complete: GEMM-1 of tile t + 1 is issued
+// while tile t is being activated, GEMM-2 of tile t runs under the first half of tile t + 1's activation.
+// The tanh unit (16 results per clock per SM) is what bounds the pass; 16 warps that interleave
+// activation and output keep it busy.
+// =====================================================================================================
+template <int N2>
+struct PpFfnCfg {
+    static constexpr int W1_SET = kPpMaxF * 128;                 // bytes
+    static constexpr int W2_CHUNK = N2 * 128;
+    static constexpr int W2_SET = (kPpMaxF / kPpHC) * W2_CHUNK;
+    static constexpr int SET_BYTES = W1_SET + ((W2_SET + 1023) / 1024) * 1024;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_W = kPpABufs * kPpABytes;
+    static constexpr int SMEM_BYTES = OFF_W + 2 * SET_BYTES;
+    static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;
+    static constexpr int ACC2_COL = 128;
+    static_assert(N2 % 16 == 0 && N2 <= 64, "output width");
+    static_assert(SMEM_ALLOC <= 218 * 1024, "shared memory budget");
+};
+
+// 16 column pairs of one row: z = acc * gate (+ bias), hidden = 2 gelu(z) or relu(z), packed bf16.
+// GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))); the factor 0.5 is applied to the
+// second GEMM's accumulator in the output step (exact, a power of two).
+template <int ACT>
+__device__ __forceinline__ void pp_act8(const uint32_t* acc, float gs, const float* bias /* shared, 16 floats */,
+                                        bool has_bias, uint32_t* out) {
+    // eight column pairs: enough independent work for the tanh unit's latency, few live registers
+    float z[16];
+    if (has_bias) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+            const float4 b = *reinterpret_cast<const float4*>(bias + i);   // same address for the whole warp
+            fma2(z[i], z[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), gs, gs, b.x, b.y);
+            fma2(z[i + 2], z[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), gs, gs, b.z, b.w);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) mul2(z[i], z[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), gs, gs);
+    }
+    if constexpr (ACT == SLICEMOE_ACT_RELU) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = cvt_rn_relu_bf16x2(z[2 * i], z[2 * i + 1]);
+    } else {
+        constexpr float c0 = 0.7978845608028654f, c1 = 0.7978845608028654f * 0.044715f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float s0, s1, n0, n1, u0, u1, r0, r1;
+            mul2(s0, s1, z[2 * i], z[2 * i + 1], z[2 * i], z[2 * i + 1]);
+            fma2(n0, n1, s0, s1, c1, c1, c0, c0);
+            mul2(u0, u1, z[2 * i], z[2 * i + 1], n0, n1);
+            const float t0 = tanh_approx(u0), t1 = tanh_approx(u1);
+            fma2(r0, r1, z[2 * i], z[2 * i + 1], t0, t1, z[2 * i], z[2 * i + 1]);
+            out[i] = pack_bf16x2(r0, r1);
+        }
+    }
+}
+
+// Called by all kPpThreads threads; TMEM (512 columns at sh.tmem_base) is allocated and freed by the
+// caller.  SAME_LAUNCH: pair_gate (and the offsets) were written earlier in this launch.
+// OFFS_IN_SMEM: sh.offs already holds the row ranges.  Rows come from gather_src through pair_gate and
+// results are added into scatter_out.
+template <int N2, int ACT, bool SAME_LAUNCH, bool OFFS_IN_SMEM>
+__device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p, const PpParams& p,
+                                            PpShared& sh, uint8_t* smem_raw) {
+    using C = PpFfnCfg<N2>;
+    using B = PpBars;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    volatile int* abort = &sh.abort_flag;
+    const int npanels = p.HID / kPpHC;
+    const bool has_b1 = p.b1 != nullptr;
+    const bool wide = p.HID == 256;          // two 32-unit sub-chunks per row thread and tile, else one
+
+    // ---- set-up -----------------------------------------------------------------------------------
+    if (threadIdx.x == 0) {
+        sh.abort_flag = 0;
+        for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 64); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(pp_bar(sh, B::W_FULL + i), 1); mbar_init(pp_bar(sh, B::W_EMPTY + i), 1); }
+        for (int r = 0; r < 2; ++r) {                                  // per tensor-memory region
+            mbar_init(pp_sbar(sh, r, B::ACC1_FULL), 1);
+            mbar_init(pp_sbar(sh, r, B::HID_FULL), 16);
+            mbar_init(pp_sbar(sh, r, B::ACC2_FULL), 1);
+            mbar_init(pp_sbar(sh, r, B::ACC2_EMPTY), 4);
+        }
+        mbar_init(pp_bar(sh, B::DRAIN), 1);
+        fence_mbar_init();
+        prefetch_tensormap(tmW1_p);
+        prefetch_tensormap(tmW2_p);
+    }
+    if (!OFFS_IN_SMEM)
+        for (int e = threadIdx.x; e <= p.E; e += kPpThreads) sh.offs[e] = SAME_LAUNCH ? __ldcg(p.offsets + e) : p.offsets[e];
+    __syncthreads();
+    if (warp == 0) pp_tile_starts(sh, p.E, lane);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh.tmem_base;
+    const int total_tiles = sh.tile_start[p.E];
+    const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
+    const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
+    const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
+    const uint32_t sA = smem_base + C::OFF_A, sW = smem_base + C::OFF_W;
+
+    if (warp == 0) {
+        // ================= TMA producer: one weight set per run ======================================
+        if (lane == 0 && ntiles > 0 && !DBG(64)) {
+            PpWalk wk;
+            wk.init();
+            int loaded_run = -1;
+            uint32_t last_bar = 0, last_par = 0;
+            bool ok = true;
+            const uint32_t set_tx = (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK);
+            for (int ta = 0; ta < ntiles && ok; ++ta) {
+                wk.advance(sh, t_begin, ta);
+                if (wk.run == loaded_run) continue;
+                loaded_run = wk.run;
+                const int set = wk.run & 1;
+                const uint32_t n = (uint32_t)wk.run >> 1;
+                if (!mbar_wait_sleepy(pp_bar(sh, B::W_EMPTY + set), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL + set), set_tx);
+                const uint32_t w1 = sW + set * C::SET_BYTES, w2 = w1 + C::W1_SET;
+                for (int c = 0; c < npanels; ++c) {
+                    tma_load_2d(w1 + c * (kPpHC * 128), tmW1_p, 0, wk.e * p.HID + c * kPpHC, pp_bar(sh, B::W_FULL + set));
+                    tma_load_2d(w2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, wk.e * N2, pp_bar(sh, B::W_FULL + set));
+                }
+                last_bar = pp_bar(sh, B::W_FULL + set);
+                last_par = n & 1u;
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                if (last_bar) mbar_wait(last_bar, last_par, &never, 10000000ull);   // let the last copies land
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issue ==================================================================
+        // Order: GEMM-1 of tiles 0 and 1; then per tile t: GEMM-2(t) once its hidden layer is written,
+        // GEMM-1(t + 2) once tile t's output accumulator has been read (same region).  All lanes run the
+        // loop (descriptors stay in uniform registers); one elected lane issues.
+        if (ntiles > 0) {
+            const uint32_t idesc1 = make_idesc(128, p.HID, kFmtBF16, kFmtBF16);
+            constexpr uint32_t idesc2 = make_idesc(128, N2, kFmtBF16, kFmtBF16);
+            const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
+            bool ok = true;
+            TRD(tr, warp);
+            PpWalk w1, w2;
+            w1.init();
+            w2.init();
+            int run1 = -1;
+            auto issue_g1 = [&](int ta) {
+                const int ab = ta % kPpABufs, r = ta & 1;
+                w1.advance(sh, t_begin, ta);
+                if (w1.run != run1) {
+                    if (!pp_wait(pp_bar(sh, B::W_FULL + (w1.run & 1)), ((uint32_t)w1.run >> 1) & 1u, abort)) { ok = false; return; }
+                    run1 = w1.run;
+                }
+                TR(tr, 8);
+                if (!pp_wait(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u, abort)) { ok = false; return; }
+                fence_proxy_async_smem();     // rows written by cp.async -> visible to the MMA's reads
+                TR(tr, 10);
+                // the region is free once the output accumulator of the tile two back has been read
+                if (!pp_wait(pp_sbar(sh, r, B::ACC2_EMPTY), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; return; }
+                TR(tr, 11);
+                tc_fence_after_sync();
+                const uint32_t wset = dW + (((w1.run & 1) * C::SET_BYTES) >> 4);
+                const uint32_t a0 = dA + ((ab * kPpABytes) >> 4);
+                const uint32_t d = tmem_base + r * kPpStreamCols;
+                if (elect_one_sync()) {
+                    mma_ss<0>(d, a0, wset, idesc1);
+#pragma unroll
+                    for (int kk = 1; kk < 4; ++kk) mma_ss<1>(d, a0 + ((kk * 32) >> 4), wset + ((kk * 32) >> 4), idesc1);
+                    mma_commit(pp_sbar(sh, r, B::ACC1_FULL));
+                    mma_commit(pp_bar(sh, B::A_EMPTY + ab));
+                }
+                __syncwarp();
+                TR(tr, 12);
+            };
+            issue_g1(0);
+            if (ok && ntiles > 1) issue_g1(1);
+#pragma unroll 1
+            for (int ta = 0; ta < ntiles && ok; ++ta) {
+                const int r = ta & 1;
+                w2.advance(sh, t_begin, ta);
+                TR(tr, 20);
+                if (!pp_wait(pp_sbar(sh, r, B::HID_FULL), (uint32_t)(ta >> 1) & 1u, abort)) { ok = false; break; }
+                TR(tr, 21);
+                tc_fence_after_sync();
+                const uint32_t w2d = dW + (((w2.run & 1) * C::SET_BYTES + C::W1_SET) >> 4);
+                const uint32_t d = tmem_base + r * kPpStreamCols;
+                if (elect_one_sync()) {
+                    // K step kk = hidden units [16 kk, 16 kk + 16): units below 128 sit at packed column
+                    // 32 (u / 32) + 8 ((u / 16) & 1), units from 128 on 16 columns further
+#pragma unroll 8
+                    for (int kk = 0; kk < p.HID / 16; ++kk) {
+                        const int u = (kk & 7) * 16;
+                        const uint32_t a = d + 32 * (u >> 5) + 8 * ((u >> 4) & 1) + (kk >= 8 ? 16 : 0);
+                        const uint32_t bd = w2d + (((kk >> 2) * C::W2_CHUNK + (kk & 3) * 32) >> 4);
+                        mma_ts_dyn(d + C::ACC2_COL, a, bd, idesc2, kk > 0 ? 1u : 0u);
+                    }
+                    mma_commit(pp_sbar(sh, r, B::ACC2_FULL));
+                }
+                __syncwarp();
+                TR(tr, 22);
+                // hand the weight sets of the runs that end here back
+                if (ta + 1 < ntiles) {
+                    const int run_before = w2.run;
+                    const int crossed = w2.advance(sh, t_begin, ta + 1);
+                    if (crossed) {
+                        if (elect_one_sync()) mma_commit(pp_bar(sh, B::W_EMPTY + (run_before & 1)));
+                        __syncwarp();
+                    }
+                }
+                if (ta + 2 < ntiles) issue_g1(ta + 2);
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                if (lane == 0) {
+                    mma_commit(pp_bar(sh, B::DRAIN));
+                    mbar_wait(pp_bar(sh, B::DRAIN), 0u, &never, 10000000ull);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 2 || warp == 3) {
+        // ================= gather warps (rows 0..63 / 64..127 of a tile) ==============================
+        // Row r of tile ta is stacked row row0 + r = pair (n, j); its A row is X[n, :], copied with
+        // asynchronous 16-byte copies into the K-major 128-byte-swizzled layout, up to four tiles ahead.
+        if (ntiles > 0 && !DBG(64)) {
+            const int ch = lane & 7, rsub = lane >> 3;
+            const int rbase = (warp - 2) * 64;
+            PpWalk wn;
+            wn.init();
+            int nnext[2];
+            bool ok = true;
+            TRD(tr, warp);
+            const bool in_row = ch * 8 < p.row_elems;
+#pragma unroll 1
+            for (int ta = -1; ta < ntiles && ok; ++ta) {
+                int nrow[2];
+#pragma unroll
+                for (int q = 0; q < 2; ++q) nrow[q] = (ta < 0 || nnext[q] < 0) ? -1 : pair_to_row(nnext[q], p.gather_magic, p.gather_shift);
+                if (ta + 1 < ntiles) {
+                    wn.advance(sh, t_begin, ta + 1);
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const int r = rbase + lane + 32 * q;
+                        nnext[q] = (r < wn.rows) ? ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wn.row0 + r)) : -1;
+                    }
+                }
+                if (ta < 0) continue;
+                const int ab = ta % kPpABufs;
+                TR(tr, 30);
+                ok = pp_wait(pp_bar(sh, B::A_EMPTY + ab), ((uint32_t)(ta / kPpABufs) & 1u) ^ 1u, abort);
+                if (!ok) break;
+                TR(tr, 31);
+                const uint32_t dst0 = sA + ab * kPpABytes;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r32 = i * 4 + rsub;
+                        const int r = rbase + q * 32 + r32;
+                        const int n = __shfl_sync(0xffffffffu, nrow[q], r32);
+                        const bool real = n >= 0 && in_row;
+                        const bf16* src = p.gather_src + (real ? (size_t)n * p.row_elems + ch * 8 : 0);
+                        if (!DBG(1)) cp_async_16(dst0 + (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4), src, real ? 16u : 0u);
+                    }
+                }
+                cp_async_mbar_arrive_noinc(pp_bar(sh, B::A_FULL + ab));
+                TR(tr, 32);
+            }
+            cp_async_wait_all();
+        }
+    } else if (warp < 20) {
+        // ================= activation warps: warpgroup g, lane group lg ================================
+        const int g = (warp - 4) >> 2;
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
+        bool ok = true;
+        TRD(tr, warp);
+        PpWalk wk;
+        wk.init();
+        float gate_next = 0.0f;          // Eq. 1's gate of this thread's row of the coming tile
+        if (ntiles > 0) {
+            wk.advance(sh, t_begin, 0);
+            if (row < wk.rows) gate_next = __int_as_float(ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row) + 1));
+        }
+        int run_bias = -1;
+#pragma unroll 1
+        for (int ta = 0; ta < ntiles && ok; ++ta) {
+            const int r = ta & 1;
+            const float gs = gate_next;
+            if (has_b1 && wk.run != run_bias) {
+                // a new run: its expert's first-layer bias as fp32 (two buffers by run parity: the other
+                // one may still be in use by warps that are behind)
+                for (int f = g * 128 + row; f < p.HID; f += 512) sh.bias1_f32[wk.run & 1][f] = __bfloat162float(p.b1[(size_t)wk.e * p.HID + f]);
+                named_barrier_sync(1, 512);
+                run_bias = wk.run;
+            }
+            const float* bias = sh.bias1_f32[wk.run & 1] + 32 * g;
+            // the next tile's gate (first used at the top of the next turn)
+            if (ta + 1 < ntiles) {
+                wk.advance(sh, t_begin, ta + 1);
+                gate_next = 0.0f;
+                if (row < wk.rows) gate_next = __int_as_float(ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row) + 1));
+            }
+            TR(tr, 40);
+            ok = pp_wait(pp_sbar(sh, r, B::ACC1_FULL), (uint32_t)(ta >> 1) & 1u, abort);
+            if (!ok) break;
+            TR(tr, 41);
+            tc_fence_after_sync();
+            const uint32_t region = tlane + r * kPpStreamCols + 32 * g;
+            // 16 hidden units per turn: units [32 g + 16 q, +16) (q = 0, 1) and [128 + 32 g + 16 (q - 2), +16)
+            // (q = 2, 3); their packed values go to columns [32 g + 8 q, +8), which this thread has read before
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q == 2 && !wide) break;
+                uint32_t acc[16], hid[8];
+                tmem_ld_x16(region + (q < 2 ? 16 * q : 128 + 16 * (q - 2)), acc);
+                tmem_ld_wait();
+                if (!DBG(8)) pp_act8<ACT>(acc, gs, bias + (q < 2 ? 16 * q : 128 + 16 * (q - 2)), has_b1, hid);
+                else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) hid[i] = acc[i] ^ acc[i + 8];
+                }
+                tmem_st_x8(region + 8 * q, hid);
+            }
+            TR(tr, 45);
+            tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::HID_FULL));
+            TR(tr, 46);
+        }
+    } else {
+        // ================= output warpgroup ===========================================================
+        // 0.5 acc + b2 -> bf16 -> add into row n of h' (the sum over the row's k experts), 16 columns at a time
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
+        bool ok = true;
+        TRD(tr, warp);
+        PpWalk wk;
+        wk.init();
+        int pair_next = 0;
+        if (ntiles > 0) {
+            wk.advance(sh, t_begin, 0);
+            if (row < wk.rows) pair_next = ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row));
+        }
+#pragma unroll 1
+        for (int ta = 0; ta < ntiles && ok; ++ta) {
+            const int r = ta & 1;
+            const bool live = row < wk.rows;
+            const int e_cur = wk.e;
+            bf16* dst = p.scatter_out + (size_t)pair_to_row(pair_next, p.gather_magic, p.gather_shift) * N2;
+            if (ta + 1 < ntiles) {
+                wk.advance(sh, t_begin, ta + 1);
+                if (row < wk.rows) pair_next = ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row));
+            }
+            TR(tr, 49);
+            ok = pp_wait(pp_sbar(sh, r, B::ACC2_FULL), (uint32_t)(ta >> 1) & 1u, abort);
+            if (!ok) break;
+            TR(tr, 50);
+            tc_fence_after_sync();
+            const uint32_t acc2 = tlane + r * kPpStreamCols + C::ACC2_COL;
+            constexpr float sc = kOutScale<ACT>;
+#pragma unroll 1
+            for (int cb = 0; cb < N2; cb += 16) {
+                uint32_t v[16];
+                tmem_ld_x16(acc2 + cb, v);
+                tmem_ld_wait();
+                if (cb + 16 >= N2) {
+                    // the accumulator is in registers: the region may be reused
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
+                    TR(tr, 52);
+                }
+                if (!live) continue;
+#pragma unroll
+                for (int c = 0; c < 16; c += 8) {
+                    float bb[8];
+                    if (p.b2) {
+                        unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.b2 + (size_t)e_cur * N2 + cb + c)), bb);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) bb[q] = 0.0f;
+                    }
+                    uint32_t o[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        o[q] = pack_bf16x2(fmaf(__uint_as_float(v[c + 2 * q]), sc, bb[2 * q]),
+                                           fmaf(__uint_as_float(v[c + 2 * q + 1]), sc, bb[2 * q + 1]));
+                    if (!DBG(4)) red_add_bf16x8(dst + cb + c, o[0], o[1], o[2], o[3]);
+                }
+            }
+            TR(tr, 53);
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh.abort_flag) atomicExch(p.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+}
+
+// =====================================================================================================
+// Router pass.  EP: expert count the kernel is built for (16 / 32 / 64; fewer real experts are padded,
+// their logits set to -inf).  Shared memory: X buffers 4 x 16 KB | Wr1 [Hr, 64] | Wr2 as Hr/64 chunks
+// of [EP, 64].  TMEM per stream: [0,192) three GEMM-1 accumulators; the hidden chunk is written over
+// the accumulator it came from as a bf16 pair hi + lo (16 mantissa bits: K step kk of a chunk is at
+// columns 16 kk (hi) and 16 kk + 8 (lo)), so that the logits do not depend on 16-bit rounding of the
+// hidden layer; [192, 192 + EP) the logits.
+// =====================================================================================================
+template <int EP>
+struct PpRouteCfg {
+    static constexpr int W2_CHUNK = EP * 128;
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_W1 = kPpABufs * kPpABytes;
+    static constexpr int OFF_W2 = OFF_W1 + kPpMaxHr * 128;
+    static constexpr int SMEM_BYTES = OFF_W2 + (kPpMaxHr / kPpHC) * W2_CHUNK;
+    static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;
+    static constexpr int ACC1_COL = 0, ACC2_COL = 192;
+    static_assert(EP % 16 == 0 && EP <= 64, "expert count");
+};
+
+template <int EP>
+__device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p,
+                                              const PpParams& p, PpShared& sh, uint8_t* smem_raw) {
+    using C = PpRouteCfg<EP>;
+    using B = PpBars;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    volatile int* abort = &sh.abort_flag;
+    const int nchunks = p.HID / kPpHC;
+
+    if (threadIdx.x == 0) {
+        sh.abort_flag = 0;
+        for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 1); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
+        mbar_init(pp_bar(sh, B::W_FULL), 1);
+        for (int s = 0; s < 2; ++s) {
+            for (int i = 0; i < 3; ++i) {
+                mbar_init(pp_sbar(sh, s, B::ACC1_FULL + i), 1);
+                mbar_init(pp_sbar(sh, s, B::ACC1_EMPTY + i), 1);
+                mbar_init(pp_sbar(sh, s, B::HID_FULL + i), 8);
+            }
+            mbar_init(pp_sbar(sh, s, B::ACC2_FULL), 1);
+            mbar_init(pp_sbar(sh, s, B::ACC2_EMPTY), 4);
+        }
+        mbar_init(pp_bar(sh, B::DRAIN), 1);
+        mbar_init(pp_bar(sh, B::DRAIN + 1), 1);
+        fence_mbar_init();
+        prefetch_tensormap(tmX_p);
+        prefetch_tensormap(tmW1_p);
+        prefetch_tensormap(tmW2_p);
+    }
+    for (int e = threadIdx.x; e < kMaxE; e += kPpThreads) sh.hist[e] = 0;
+    for (int i = threadIdx.x; i < p.HID; i += kPpThreads) sh.bias1_f32[0][i] = p.br1 ? __bfloat162float(p.br1[i]) : 0.0f;
+    for (int i = threadIdx.x; i < EP; i += kPpThreads)
+        sh.bias2_f32[i] = i >= p.experts_real ? -INFINITY : (p.br2 ? __bfloat162float(p.br2[i]) : 0.0f);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh.tmem_base;
+    const int total_tiles = (p.n_rows + kTileM - 1) / kTileM;
+    const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
+    const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
+    const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
+    const uint32_t sA = smem_base + C::OFF_A, sW1 = smem_base + C::OFF_W1, sW2 = smem_base + C::OFF_W2;
+
+    if (warp == 0) {
+        // ================= TMA producer ===============================================================
+        if (lane == 0 && ntiles > 0) {
+            bool ok = true;
+            mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + nchunks * C::W2_CHUNK));
+            for (int c = 0; c < nchunks; ++c) {
+                tma_load_2d(sW1 + c * (kPpHC * 128), tmW1_p, 0, c * kPpHC, pp_bar(sh, B::W_FULL));
+                tma_load_2d(sW2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, 0, pp_bar(sh, B::W_FULL));
+            }
+            uint32_t last_bar = pp_bar(sh, B::W_FULL), last_par = 0;
+            for (int ta = 0; ta < ntiles; ++ta) {
+                const int ab = ta % kPpABufs;
+                if (!mbar_wait(pp_bar(sh, B::A_EMPTY + ab), ((uint32_t)(ta / kPpABufs) & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                mbar_arrive_expect_tx(pp_bar(sh, B::A_FULL + ab), kPpABytes);
+                tma_load_2d(sA + ab * kPpABytes, tmX_p, 0, (t_begin + ta) * kTileM, pp_bar(sh, B::A_FULL + ab));
+                last_bar = pp_bar(sh, B::A_FULL + ab);
+                last_par = (uint32_t)(ta / kPpABufs) & 1u;
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                mbar_wait(last_bar, last_par, &never, 10000000ull);
+            }
+        }
+    } else if (warp == 1 || warp == 2) {
+        // ================= MMA issue, stream s ========================================================
+        const int s = warp - 1;
+        const int n_my = (ntiles - s + 1) / 2;
+        const int Q = n_my * nchunks;
+        if (Q > 0) {
+            constexpr uint32_t idesc1 = make_idesc(128, kPpHC, kFmtBF16, kFmtBF16);
+            constexpr uint32_t idesc2 = make_idesc(128, EP, kFmtBF16, kFmtBF16);
+            const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1), dW2 = desc_lo_sw128(sW2);
+            const uint32_t tcol = tmem_base + s * kPpStreamCols;
+            bool ok = true;
+            int q1 = 0, c1 = 0, i1 = 0;
+            int q2 = 0, c2 = 0, i2 = 0;
+            TRD(tr, 20 + warp);
+            auto wait_all = [&](uint32_t bar, uint32_t parity) {
+                return (bool)__all_sync(0xffffffffu, mbar_wait(bar, parity, abort, kWaitLimitNs));
+            };
+            if (!wait_all(pp_bar(sh, B::W_FULL), 0u)) ok = false;
+            auto issue_g1 = [&]() {
+                const int ta = s + 2 * i1;
+                const int ab = ta % kPpABufs;
+                TR(tr, 8);
+                if (c1 == 0 && !wait_all(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u)) { ok = false; return; }
+                const uint32_t b = (uint32_t)q1 % 3u, n = (uint32_t)q1 / 3u;
+                TR(tr, 10);
+                // (the accumulator also held the previous chunk's hidden values: GEMM-2 must have read them)
+                if (!wait_all(pp_sbar(sh, s, B::ACC1_EMPTY + b), (n & 1u) ^ 1u)) { ok = false; return; }
+                TR(tr, 11);
+                tc_fence_after_sync();
+                const uint32_t a0 = dA + ((ab * kPpABytes) >> 4), w0 = dW1 + ((c1 * (kPpHC * 128)) >> 4);
+                const uint32_t d = tcol + C::ACC1_COL + b * kPpHC;
+                const bool last = c1 == nchunks - 1;
+                if (elect_one_sync()) {
+                    mma_ss<0>(d, a0, w0, idesc1);
+#pragma unroll
+                    for (int kk = 1; kk < 4; ++kk) mma_ss<1>(d, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
+                    mma_commit(pp_sbar(sh, s, B::ACC1_FULL + b));
+                    if (last) mma_commit(pp_bar(sh, B::A_EMPTY + ab));
+                }
+                __syncwarp();
+                TR(tr, 12);
+                ++q1;
+                if (last) { c1 = 0; ++i1; } else { ++c1; }
+            };
+            auto issue_g2 = [&]() {
+                TR(tr, 19);
+                if (c2 == 0 && !wait_all(pp_sbar(sh, s, B::ACC2_EMPTY), ((uint32_t)i2 & 1u) ^ 1u)) { ok = false; return; }
+                const uint32_t b = (uint32_t)q2 % 3u, n = (uint32_t)q2 / 3u;
+                TR(tr, 20);
+                if (!wait_all(pp_sbar(sh, s, B::HID_FULL + b), n & 1u)) { ok = false; return; }
+                TR(tr, 21);
+                tc_fence_after_sync();
+                const uint32_t w0 = dW2 + ((c2 * C::W2_CHUNK) >> 4);
+                const uint32_t d = tcol + C::ACC2_COL, a = tcol + C::ACC1_COL + b * kPpHC;
+                const bool last = c2 == nchunks - 1;
+                if (elect_one_sync()) {
+#pragma unroll
+                    for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                        for (int kk = 0; kk < kPpHC / 16; ++kk) {
+                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, w0, idesc2, c2 > 0 ? 1u : 0u);
+                            else mma_ts<1>(d, a + kk * 16 + part * 8, w0 + ((kk * 32) >> 4), idesc2);
+                        }
+                    }
+                    mma_commit(pp_sbar(sh, s, B::ACC1_EMPTY + b));
+                    if (last) mma_commit(pp_sbar(sh, s, B::ACC2_FULL));
+                }
+                __syncwarp();
+                TR(tr, 22);
+                ++q2;
+                if (last) { c2 = 0; ++i2; } else { ++c2; }
+            };
+            if (ok) issue_g1();
+            if (ok && Q > 1) issue_g1();
+            while (ok && q2 < Q) {
+                issue_g2();
+                if (ok && q1 < Q) issue_g1();
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                if (lane == 0) {
+                    mma_commit(pp_bar(sh, B::DRAIN + s));
+                    mbar_wait(pp_bar(sh, B::DRAIN + s), 0u, &never, 10000000ull);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 3) {
+        // ================= zero this CTA's rows of h' =================================================
+        if (p.zero_out != nullptr && ntiles > 0) {
+            const long long row_lo = (long long)t_begin * kTileM;
+            long long row_hi = (long long)(t_begin + ntiles) * kTileM;
+            if (row_hi > p.n_rows) row_hi = p.n_rows;
+            uint4* dst = reinterpret_cast<uint4*>(p.zero_out + row_lo * p.row_elems);
+            const long long nvec = (row_hi - row_lo) * p.row_elems / 8;
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            for (long long i = lane; i < nvec; i += 32) dst[i] = z;
+        }
+    } else if (warp < 20) {
+        // ================= row threads of stream s, column half hh ====================================
+        // (the two halves take the tiles' softmax / top-k step in turn; warps 20..23 have no part here)
+        const int wg = (warp - 4) >> 2;
+        const int s = wg & 1, hh = wg >> 1;
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        const uint32_t tcol = tmem_base + ((uint32_t)(lg * 32) << 16) + s * kPpStreamCols;
+        const int n_my = (ntiles - s + 1) / 2;
+        bool ok = true;
+        bool pend = false;
+        int pend_ta = 0;
+        uint32_t pend_i = 0;
+        // softmax + top-k of a finished tile's logits (ties go to the lower id), this CTA's rank of each pair
+        auto output_tile = [&]() {
+            ok = mbar_wait(pp_sbar(sh, s, B::ACC2_FULL), pend_i & 1u, abort, kWaitLimitNs);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            tc_fence_after_sync();
+            uint32_t v[EP];
+#pragma unroll
+            for (int c = 0; c < EP; c += 16) tmem_ld_x16(tcol + C::ACC2_COL + c, v + c);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pp_sbar(sh, s, B::ACC2_EMPTY));
+            pend = false;
+            const int n = (t_begin + pend_ta) * kTileM + row;
+            if (n >= p.n_rows) return;
+            float gl[EP];
+#pragma unroll
+            for (int i = 0; i < EP; i += 4) {
+                const float4 b = *reinterpret_cast<const float4*>(sh.bias2_f32 + i);
+                add2(gl[i], gl[i + 1], __uint_as_float(v[i]), __uint_as_float(v[i + 1]), b.x, b.y);
+                add2(gl[i + 2], gl[i + 3], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]), b.z, b.w);
+            }
+            // one pass keeping the best two (strict comparisons in ascending id order: same picks as
+            // repeated arg-max with ties to the lower id)
+            float b1 = gl[0], b2 = -INFINITY;
+            int i1 = 0, i2 = 0;
+#pragma unroll
+            for (int i = 1; i < EP; ++i) {
+                const float g = gl[i];
+                const bool gt1 = g > b1, gt2 = g > b2;
+                b2 = gt1 ? b1 : (gt2 ? g : b2);
+                i2 = gt1 ? i1 : (gt2 ? i : i2);
+                b1 = gt1 ? g : b1;
+                i1 = gt1 ? i : i1;
+            }
+            const float sc = p.softmax_scale;
+            const float msc = b1 * sc;
+            float sum = 0.0f;
+#pragma unroll
+            for (int i = 0; i < EP; ++i) sum += ex2_approx(fmaf(gl[i], sc, -msc));
+            const float inv = 1.0f / sum;
+            const int sel[2] = {i1, i2};
+            const float pj[2] = {inv, ex2_approx(fmaf(b2, sc, -msc)) * inv};
+            for (int j = 0; j < p.k; ++j) {
+                const size_t at = (size_t)n * p.k + j;
+                p.topk_idx[at] = sel[j];
+                p.topk_p[at] = pj[j];
+                p.local_rank[at] = atomicAdd(&sh.hist[sel[j]], 1);
+            }
+        };
+        uint32_t q = 0;
+        TRD(tr, 20 + warp);
+        for (int i = 0; i < n_my && ok; ++i) {
+            for (int c = 0; c < nchunks && ok; ++c, ++q) {
+                if (pend && c == 1) {        // the previous tile's logits, one chunk late (see the expert pass)
+                    TR(tr, 50);
+                    output_tile();
+                    TR(tr, 51);
+                    if (!ok) break;
+                }
+                const uint32_t b = q % 3u, par = (q / 3u) & 1u;
+                TR(tr, 40);
+                ok = mbar_wait(pp_sbar(sh, s, B::ACC1_FULL + b), par, abort, kWaitLimitNs);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                TR(tr, 41);
+                tc_fence_after_sync();
+                const uint32_t acol = tcol + C::ACC1_COL + b * kPpHC + 32 * hh;
+                uint32_t acc[32];
+                tmem_ld_x32(acol, acc);
+                tmem_ld_wait();
+                TR(tr, 42);
+                const float* bias = sh.bias1_f32[0] + c * kPpHC + 32 * hh;
+#pragma unroll
+                for (int pc = 0; pc < 2; ++pc) {
+                    // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu),
+                    // lo = the rounded remainder (for a negative value the remainder is the value itself and
+                    // its .relu is 0 as well)
+                    float a[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        const float4 bb = *reinterpret_cast<const float4*>(bias + pc * 16 + i);
+                        add2(a[i], a[i + 1], __uint_as_float(acc[pc * 16 + i]), __uint_as_float(acc[pc * 16 + i + 1]), bb.x, bb.y);
+                        add2(a[i + 2], a[i + 3], __uint_as_float(acc[pc * 16 + i + 2]), __uint_as_float(acc[pc * 16 + i + 3]), bb.z, bb.w);
+                    }
+                    uint32_t hl[16];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) hl[i] = cvt_rz_relu_bf16x2(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        hl[8 + i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hl[i] << 16), a[2 * i + 1] - __uint_as_float(hl[i] & 0xFFFF0000u));
+                    tmem_st_x16(acol + pc * 16, hl);
+                }
+                TR(tr, 45);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pp_sbar(sh, s, B::HID_FULL + b));
+                TR(tr, 46);
+            }
+            pend = (i & 1) == hh;
+            pend_ta = s + 2 * i;
+            pend_i = (uint32_t)i;
+        }
+        if (ok && pend) output_tile();
+    }
+
+    // ---- teardown ---------------------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh.abort_flag) atomicExch(p.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
+    if (p.cta_hist)
+        for (int i = threadIdx.x; i < p.experts_real; i += kPpThreads) p.cta_hist[(size_t)blockIdx.x * p.experts_real + i] = sh.hist[i];
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+}
+
+// =====================================================================================================
+// Dispatch without a capacity limit: the router left every pair's rank among its CTA's pairs of the same
+// expert (local_rank) and each CTA's per-expert counts (table[c][e]).  A pair's stacked row is
+// offsets[e] + (pairs of expert e in earlier CTAs) + local rank.  The order inside an expert is then the
+// order in which the router's row threads drew their ranks, which varies from run to run; the layer's
+// output does not depend on it (each stacked row is computed on its own, and the sum of at most two bf16
+// values commutes), but `perm` / `dest` do, so this form is used only where they are not outputs and
+// nothing is dropped (capacity limits need the stable order of the other dispatch).
+// offs_out: shared memory, E + 1 ints.  `sm`: at least (2 E + 1) ints of shared memory.
+// =====================================================================================================
+template <int NT, bool SAME_LAUNCH>
+__device__ __forceinline__ void pp_dispatch_body(const int32_t* topk_idx, const float* topk_p, const int32_t* local_rank,
+                                                 const int32_t* table, int G, int chunk, int R, int E, int pairs_per_chunk,
+                                                 int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
+                                                 int2* pair_gate, int* sm, int* offs_out) {
+    int* base = sm;            // [E] pairs of expert e in earlier CTAs, then + offsets
+    int* total = sm + E;       // [E]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // warp w sums experts w, w + NT/32, ...: lanes stride over the CTAs of the table
+    for (int e = warp; e < E; e += NT / 32) {
+        int before = 0, tot = 0;
+        for (int c = lane; c < G; c += 32) {
+            const int v = SAME_LAUNCH ? __ldcg(table + (size_t)c * E + e) : table[(size_t)c * E + e];
+            tot += v;
+            if (c < chunk) before += v;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            before += __shfl_xor_sync(0xffffffffu, before, d);
+            tot += __shfl_xor_sync(0xffffffffu, tot, d);
+        }
+        if (lane == 0) { base[e] = before; total[e] = tot; }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int run = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + lane;
+            const int tot = e < E ? total[e] : 0;
+            int incl = tot;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += up;
+            }
+            if (e < E) {
+                const int o = run + incl - tot;
+                offs_out[e] = o;
+                base[e] += o;
+                if (chunk == 0) {
+                    if (assigned) assigned[e] = tot;
+                    if (kept) kept[e] = tot;
+                    offsets[e] = o;
+                }
+            }
+            run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) {
+            offs_out[E] = run;
+            if (chunk == 0) offsets[E] = run;
+        }
+    }
+    __syncthreads();
+    const long long begin = (long long)chunk * pairs_per_chunk;
+    long long end = begin + pairs_per_chunk;
+    if (end > R) end = R;
+    for (long long i = begin + threadIdx.x; i < end; i += NT) {
+        const int e = SAME_LAUNCH ? __ldcg(topk_idx + i) : topk_idx[i];
+        const int r = SAME_LAUNCH ? __ldcg(local_rank + i) : local_rank[i];
+        const float pr = SAME_LAUNCH ? __ldcg(topk_p + i) : topk_p[i];
+        const int d = base[e] + r;
+        dest[i] = d;
+        pair_gate[d] = make_int2((int)i, __float_as_int(pr));
+    }
+}
+
+}  // namespace
+}  // namespace slicemoe

@@ -1,0 +1,348 @@
+// The forward of the layer (Section 3.1, Eq. 1; Section 3.4) on the two-stream pipeline of pp_body.cuh,
+// for 64-wide slices without a capacity limit: as ONE cooperative launch
+//
+//   phase 1  router     top-k ids and probabilities, each pair's rank among this CTA's pairs of its expert,
+//                       this CTA's per-expert counts, its rows of h' zeroed
+//   -- grid barrier --
+//   phase 2  dispatch   stacked row of each of this CTA's pairs = offsets[e] + pairs of e in earlier CTAs +
+//                       the pair's rank; (pair, gate) written at that row; CTA 0 writes assigned/kept/offsets
+//   -- grid barrier --
+//   phase 3  experts    rows gathered from h, outputs added into h'
+//
+// and as one launch per phase (the stage-timed call).
+#include <mutex>
+
+#include "pp_body.cuh"
+
+namespace slicemoe {
+namespace {
+
+struct PpFusedParams {
+    PpParams route, ffn;
+    int R, E, pairs_per_chunk;
+    int32_t *assigned, *kept, *offsets, *dest;
+    int2* pair_gate;
+    int32_t* sync_words;
+    int clear_status;
+};
+
+// Grid barrier words (arrival count, generation) of this file's cooperative kernel, one pair per
+// device: zero at module load, left ready for the next barrier by every barrier that completes.
+__device__ int32_t g_pp_sync[2];
+
+__device__ __forceinline__ bool pp_grid_barrier(int32_t* words, int32_t gen_before, PpShared& sh) {
+    fence_proxy_async_smem();     // the phases reuse shared memory through different proxies
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        volatile int32_t* count = words;
+        volatile int32_t* gen = words + 1;
+        __threadfence();
+        if (atomicAdd(words, 1) == (int)gridDim.x - 1) {
+            *count = 0;
+            __threadfence();
+            atomicAdd(words + 1, 1);
+        } else {
+            const uint64_t t0 = globaltimer_ns();
+            while (*gen == gen_before) {
+                if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                    sh.abort_flag = 1;
+                    break;
+                }
+                __nanosleep(64);
+            }
+        }
+        __threadfence();
+    }
+    __syncthreads();
+    return sh.abort_flag == 0;
+}
+
+template <int EP, int N2, int ACT>
+__global__ void __launch_bounds__(kPpThreads, 1)
+pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWr1,
+                  const __grid_constant__ CUtensorMap tmWr2, const __grid_constant__ CUtensorMap tmW1,
+                  const __grid_constant__ CUtensorMap tmW2, const PpFusedParams fp) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ PpShared sh;
+    const int warp = threadIdx.x >> 5;
+    int32_t gen0 = 0;
+    if (threadIdx.x == 0) {
+        gen0 = *reinterpret_cast<volatile int32_t*>(fp.sync_words + 1);   // no barrier can complete without this CTA
+        if (blockIdx.x == 0 && fp.clear_status) *fp.ffn.status = SLICEMOE_OK;
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh.tmem_base), 512);
+        tmem_relinquish();
+    }
+    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
+    bool ok = sh.abort_flag == 0;
+    ok = pp_grid_barrier(fp.sync_words, gen0, sh) && ok;
+    if (ok) {
+        int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
+        pp_dispatch_body<kPpThreads, true>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, fp.route.cta_hist,
+                                           (int)gridDim.x, (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.assigned,
+                                           fp.kept, fp.offsets, fp.dest, fp.pair_gate, dsm, sh.offs);
+    }
+    ok = pp_grid_barrier(fp.sync_words, gen0 + 1, sh) && ok;
+    if (ok) pp_ffn_body<N2, ACT, true, true>(&tmW1, &tmW2, fp.ffn, sh, smem_raw);
+    if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(sh.tmem_base, 512);
+    }
+}
+
+// ---- one launch per phase -------------------------------------------------------------------------
+template <int EP>
+__global__ void __launch_bounds__(kPpThreads, 1)
+pp_route_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWr1,
+                const __grid_constant__ CUtensorMap tmWr2, const PpParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ PpShared sh;
+    const int warp = threadIdx.x >> 5;
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh.tmem_base), 512);
+        tmem_relinquish();
+    }
+    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, p, sh, smem_raw);
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(sh.tmem_base, 512);
+    }
+}
+
+__global__ void __launch_bounds__(kPpThreads, 1)
+pp_dispatch_kernel(const int32_t* topk_idx, const float* topk_p, const int32_t* local_rank, const int32_t* table, int R,
+                   int E, int pairs_per_chunk, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
+                   int2* pair_gate) {
+    __shared__ int sm[2 * kMaxE + 1];
+    __shared__ int offs[kMaxE + 1];
+    pp_dispatch_body<kPpThreads, false>(topk_idx, topk_p, local_rank, table, (int)gridDim.x, (int)blockIdx.x, R, E,
+                                        pairs_per_chunk, assigned, kept, offsets, dest, pair_gate, sm, offs);
+}
+
+template <int N2, int ACT>
+__global__ void __launch_bounds__(kPpThreads, 1)
+pp_ffn_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2, const PpParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ PpShared sh;
+    const int warp = threadIdx.x >> 5;
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh.tmem_base), 512);
+        tmem_relinquish();
+    }
+    pp_ffn_body<N2, ACT, false, false>(&tmW1, &tmW2, p, sh, smem_raw);
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(sh.tmem_base, 512);
+    }
+}
+
+constexpr int kMaxDevices = 64;
+std::mutex g_pp_mutex;
+int32_t* g_pp_sync_addr[kMaxDevices] = {};
+bool g_pp_attr[kMaxDevices][16] = {};      // per device and kernel instantiation: shared-memory limit raised
+
+int pp_sync_address(int32_t** out, int* dev_out) {
+    int dev = -1;
+    SLICEMOE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SLICEMOE_ERR_NO_DEVICE;
+    std::lock_guard<std::mutex> lock(g_pp_mutex);
+    if (!g_pp_sync_addr[dev]) {
+        void* p = nullptr;
+        SLICEMOE_CUDA_TRY(cudaGetSymbolAddress(&p, g_pp_sync));
+        if (!p) return SLICEMOE_ERR_CUDA;
+        g_pp_sync_addr[dev] = static_cast<int32_t*>(p);
+    }
+    *out = g_pp_sync_addr[dev];
+    if (dev_out) *dev_out = dev;
+    return SLICEMOE_OK;
+}
+
+// cudaFuncSetAttribute is per device: once per (device, kernel).
+template <class K>
+int pp_set_smem(K kern, int slot, int bytes) {
+    int dev = -1;
+    SLICEMOE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SLICEMOE_ERR_NO_DEVICE;
+    std::lock_guard<std::mutex> lock(g_pp_mutex);
+    if (!g_pp_attr[dev][slot]) {
+        SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        g_pp_attr[dev][slot] = true;
+    }
+    return SLICEMOE_OK;
+}
+
+struct PpMaps {
+    CUtensorMap X, Wr1, Wr2, W1, W2;
+};
+
+template <int EP, int N2>
+int pp_make_maps(const Dims& D, const slicemoe_weights& w, const void* h, PpMaps& m) {
+    int rc;
+    if ((rc = make_tmap(&m.X, h, (uint64_t)D.N, (uint64_t)D.ds, 128))) return rc;
+    if ((rc = make_tmap(&m.Wr1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, kPpHC))) return rc;
+    if ((rc = make_tmap(&m.Wr2, w.Wr2, (uint64_t)D.E, (uint64_t)D.Hr, EP))) return rc;       // (E = 8: zero-filled up to 16)
+    if ((rc = make_tmap(&m.W1, w.W1, (uint64_t)D.E * D.F, (uint64_t)D.ds, kPpHC))) return rc;
+    if ((rc = make_tmap(&m.W2, w.W2, (uint64_t)D.E * N2, (uint64_t)D.F, N2))) return rc;
+    return SLICEMOE_OK;
+}
+
+void pp_fill_params(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx, float* topk_p,
+                    int32_t* dest, int32_t* offsets, int2* pair_gate, int32_t* cta_hist, int32_t* status, PpParams& r,
+                    PpParams& f) {
+    r = PpParams{};
+    r.status = status; r.n_rows = D.N; r.HID = D.Hr; r.experts_real = D.E; r.k = D.k;
+    r.softmax_scale = 1.4426950408889634f * D.inv_tau;
+    r.br1 = (const bf16*)w.br1; r.br2 = (const bf16*)w.br2;
+    r.topk_idx = topk_idx; r.topk_p = topk_p; r.local_rank = dest; r.cta_hist = cta_hist;
+    r.zero_out = (bf16*)h_out; r.row_elems = D.ds;
+    f = PpParams{};
+    f.status = status; f.n_rows = D.R; f.HID = D.F; f.E = D.E; f.offsets = offsets;
+    f.b1 = (const bf16*)w.b1; f.b2 = (const bf16*)w.b2;
+    f.gather_src = (const bf16*)h; f.pair_gate = pair_gate;
+    pair_to_row_magic(D.k, &f.gather_magic, &f.gather_shift);
+    f.scatter_out = (bf16*)h_out; f.row_elems = D.ds; f.k = D.k;
+}
+
+template <int EP, int N2, int ACT>
+int pp_launch_fused(const Dims& D, const slicemoe_weights& w, const void* h, const PpFusedParams& fp, cudaStream_t st) {
+    PpMaps m;
+    int rc = pp_make_maps<EP, N2>(D, w, h, m);
+    if (rc) return rc;
+    constexpr int smem = PpFfnCfg<N2>::SMEM_ALLOC > PpRouteCfg<EP>::SMEM_ALLOC ? PpFfnCfg<N2>::SMEM_ALLOC : PpRouteCfg<EP>::SMEM_ALLOC;
+    static_assert(smem >= 120 * 1024, "one CTA per SM (each allocates all of tensor memory)");
+    auto kern = pp_forward_kernel<EP, N2, ACT>;
+    constexpr int slot = (EP == 16 ? 0 : EP == 32 ? 1 : 2) * 2 + (ACT == SLICEMOE_ACT_RELU ? 0 : 1);
+    if ((rc = pp_set_smem(kern, slot, smem))) return rc;
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(sm_count());
+    lc.blockDim = dim3(kPpThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attrs[1];
+    attrs[0].id = cudaLaunchAttributeCooperative;   // one CTA per SM, all resident at once
+    attrs[0].val.cooperative = 1;
+    lc.attrs = attrs;
+    lc.numAttrs = 1;
+    SLICEMOE_CUDA_TRY(cudaLaunchKernelEx(&lc, kern, m.X, m.Wr1, m.Wr2, m.W1, m.W2, fp));
+    SLICEMOE_LAUNCH_CHECK(1);
+    return SLICEMOE_OK;
+}
+
+template <int EP, int N2, int ACT>
+int pp_launch_staged(const Dims& D, const slicemoe_weights& w, const void* h, const PpFusedParams& fp, cudaStream_t st,
+                     void* const* events) {
+    PpMaps m;
+    int rc = pp_make_maps<EP, N2>(D, w, h, m);
+    if (rc) return rc;
+    const int tiles = (D.N + kTileM - 1) / kTileM;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    const int rows_per_cta = ((tiles + grid - 1) / grid) * kTileM;
+    auto mark = [&](int i) -> int {
+        if (events) SLICEMOE_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(events[i]), st));
+        return SLICEMOE_OK;
+    };
+    constexpr int slot_r = 6 + (EP == 16 ? 0 : EP == 32 ? 1 : 2);
+    constexpr int slot_f = 9 + (ACT == SLICEMOE_ACT_RELU ? 0 : 1);
+    auto kr = pp_route_kernel<EP>;
+    auto kf = pp_ffn_kernel<N2, ACT>;
+    constexpr int smem_r = PpRouteCfg<EP>::SMEM_ALLOC > 120 * 1024 ? PpRouteCfg<EP>::SMEM_ALLOC : 120 * 1024;
+    if ((rc = pp_set_smem(kr, slot_r, smem_r))) return rc;
+    if ((rc = pp_set_smem(kf, slot_f, PpFfnCfg<N2>::SMEM_ALLOC))) return rc;
+    if ((rc = mark(0))) return rc;
+    kr<<<grid, kPpThreads, smem_r, st>>>(m.X, m.Wr1, m.Wr2, fp.route);
+    SLICEMOE_LAUNCH_CHECK(1);
+    if ((rc = mark(1))) return rc;
+    pp_dispatch_kernel<<<grid, kPpThreads, 0, st>>>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank,
+                                                    fp.route.cta_hist, fp.R, fp.E, rows_per_cta * D.k, fp.assigned, fp.kept,
+                                                    fp.offsets, fp.dest, fp.pair_gate);
+    SLICEMOE_LAUNCH_CHECK(1);
+    if ((rc = mark(2))) return rc;
+    const int ffn_grid = max_tiles(D) < sm_count() ? max_tiles(D) : sm_count();
+    kf<<<ffn_grid, kPpThreads, PpFfnCfg<N2>::SMEM_ALLOC, st>>>(m.W1, m.W2, fp.ffn);
+    SLICEMOE_LAUNCH_CHECK(1);
+    if ((rc = mark(3))) return rc;
+    return mark(4);
+}
+
+template <int EP, int N2>
+int pp_launch_act(const Dims& D, const slicemoe_weights& w, const void* h, const PpFusedParams& fp, cudaStream_t st,
+                  bool one_launch, void* const* events) {
+    if (D.act == SLICEMOE_ACT_GELU_TANH)
+        return one_launch ? pp_launch_fused<EP, N2, SLICEMOE_ACT_GELU_TANH>(D, w, h, fp, st)
+                          : pp_launch_staged<EP, N2, SLICEMOE_ACT_GELU_TANH>(D, w, h, fp, st, events);
+    return one_launch ? pp_launch_fused<EP, N2, SLICEMOE_ACT_RELU>(D, w, h, fp, st)
+                      : pp_launch_staged<EP, N2, SLICEMOE_ACT_RELU>(D, w, h, fp, st, events);
+}
+
+bool pp_cooperative_launch_available() {
+    static int ok = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess)
+            v = 0;
+        return v;
+    }();
+    return ok != 0;
+}
+
+}  // namespace
+
+#ifdef PP_TRACE
+extern "C" int slicemoe_debug_pp_flags(int flags) {
+    cudaMemcpyToSymbol(g_pp_dbg, &flags, sizeof(int));
+    return cudaDeviceSynchronize() == cudaSuccess ? 0 : 7;
+}
+extern "C" int slicemoe_debug_pp_trace(int on, void* host_out) {
+    if (host_out) cudaMemcpyFromSymbol(host_out, g_pp_trace, sizeof(unsigned long long) * 40 * 4096);
+    cudaMemcpyToSymbol(g_pp_trace_on, &on, sizeof(int));
+    return cudaDeviceSynchronize() == cudaSuccess ? 0 : 7;
+}
+#endif
+
+int pp_forward_reset_sync(cudaStream_t st) {
+    int32_t* words = nullptr;
+    int rc = pp_sync_address(&words, nullptr);
+    if (rc) return rc;
+    SLICEMOE_CUDA_TRY(cudaMemsetAsync(words, 0, 2 * sizeof(int32_t), st));
+    SLICEMOE_CUDA_TRY(cudaStreamSynchronize(st));
+    return SLICEMOE_OK;
+}
+
+bool pp_forward_supported(const Dims& D) {
+    if (D.dtype != SLICEMOE_BF16 || D.ds != 64 || D.N <= 0) return false;
+    if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
+    if (D.k > 2 || D.capacity != 0 || D.noise_sigma > 0.0f) return false;
+    if (D.Hr % kPpHC || D.Hr < 2 * kPpHC || D.Hr > kPpMaxHr) return false;
+    if (D.F % kPpHC || D.F < 2 * kPpHC || D.F > kPpMaxF) return false;
+    return pp_cooperative_launch_available();
+}
+
+int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
+                      float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest, void* pair_gate,
+                      int32_t* cta_hist, int32_t* status, bool clear_status, bool one_launch, void* const* events,
+                      cudaStream_t st) {
+    PpFusedParams fp{};
+    fp.clear_status = clear_status ? 1 : 0;
+    int rc = pp_sync_address(&fp.sync_words, nullptr);
+    if (rc) return rc;
+    const int grid = sm_count();
+    const int tiles = (D.N + kTileM - 1) / kTileM;
+    const int rows_per_cta = ((tiles + grid - 1) / grid) * kTileM;
+    pp_fill_params(D, w, h, h_out, topk_idx, topk_p, dest, offsets, static_cast<int2*>(pair_gate), cta_hist, status,
+                   fp.route, fp.ffn);
+    fp.R = D.R; fp.E = D.E; fp.pairs_per_chunk = rows_per_cta * D.k;
+    fp.assigned = assigned; fp.kept = kept; fp.offsets = offsets; fp.dest = dest;
+    fp.pair_gate = static_cast<int2*>(pair_gate);
+    switch (D.E) {
+        case 8:
+        case 16: return pp_launch_act<16, 64>(D, w, h, fp, st, one_launch, events);
+        case 32: return pp_launch_act<32, 64>(D, w, h, fp, st, one_launch, events);
+        case 64: return pp_launch_act<64, 64>(D, w, h, fp, st, one_launch, events);
+        default: return SLICEMOE_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace slicemoe

@@ -33,7 +33,13 @@ constexpr int kPpThreads = 768;
 #ifndef PP_SLEEP_NS
 #define PP_SLEEP_NS 100
 #endif
+#ifndef PP_STAGGER_NS
+#define PP_STAGGER_NS 400
+#endif
 constexpr int kPpABufs = 4;              // row-tile buffers
+// Depth of the per-tile metadata ring: an entry is written up to kPpABufs tiles ahead of GEMM-1 and read by
+// the output warps, which run at most three tiles behind GEMM-1 (two regions and the tile being written).
+constexpr int kPpMetaRing = 8;
 constexpr int kPpABytes = 128 * 128;     // 128 rows x 64 bf16
 constexpr int kPpHC = 64;                // hidden units per chunk
 constexpr int kPpMaxF = 256;             // expert hidden width (both weight sets stay in shared memory)
@@ -101,6 +107,8 @@ static __device__ __noinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t pari
 // call costs a stack frame, and with ~200 KB of shared memory per CTA there is next to no L1 left for
 // local memory -- a kernel that spills runs every piece of scalar book-keeping at L2 latency.)
 __device__ __forceinline__ bool pp_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    // most waits of this pipeline find their phase complete: a plain test is several times cheaper than a try
+    if (__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
     return (bool)__all_sync(0xffffffffu, mbar_wait(bar, parity, abort, kWaitLimitNs));
 }
 
@@ -117,12 +125,22 @@ __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bul
 // all bulk groups of this thread have finished reading their shared-memory source
 __device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
+// Four rows of a 2-D tensor (row indices y0..y3, columns from x on, one box of the map wide; the map's box is
+// one row high) into four consecutive 128-byte rows of shared memory, swizzled like a tiled load.
+__device__ __forceinline__ void tma_gather4(uint32_t smem_dst, const CUtensorMap* m, int x, int y0, int y1, int y2, int y3,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3), "r"(bar)
+        : "memory");
+}
+
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
 #ifdef PP_TRACE
-__device__ unsigned long long g_pp_trace[40][4096];
+__device__ unsigned long long g_pp_trace[64][4096];
 __device__ int g_pp_trace_on = 0;
 struct PpTr {
     int n, slot; bool on;
@@ -150,6 +168,10 @@ struct PpShared {
     // experts: first-layer bias of the run each stream is in, as fp32; router: br1 / br2 as fp32
     __align__(16) float bias1_f32[2][kPpMaxHr];
     __align__(16) float bias2_f32[kMaxE];
+    // experts: per tile in flight (ring over the CTA's tile counter), written by the gather warps with the
+    // tile's rows: each row's (pair index, gate), and the tile's expert, run and row count
+    __align__(16) int2 pair_gate_s[kPpMetaRing][kTileM];
+    int4 tile_s[kPpMetaRing];
 };
 
 // Barrier slots.
@@ -275,11 +297,9 @@ struct PpFfnCfg {
 // 16 column pairs of one row: z = acc * gate (+ bias), hidden = 2 gelu(z) or relu(z), packed bf16.
 // GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))); the factor 0.5 is applied to the
 // second GEMM's accumulator in the output step (exact, a power of two).
-template <int ACT>
-__device__ __forceinline__ void pp_act8(const uint32_t* acc, float gs, const float* bias /* shared, 16 floats */,
-                                        bool has_bias, uint32_t* out) {
-    // eight column pairs: enough independent work for the tanh unit's latency, few live registers
-    float z[16];
+// z = acc * gate (+ bias) for 16 columns of one row
+__device__ __forceinline__ void pp_scale16(const uint32_t* acc, float gs, const float* bias /* shared, 16 floats */,
+                                           bool has_bias, float* z) {
     if (has_bias) {
 #pragma unroll
         for (int i = 0; i < 16; i += 4) {
@@ -291,6 +311,11 @@ __device__ __forceinline__ void pp_act8(const uint32_t* acc, float gs, const flo
 #pragma unroll
         for (int i = 0; i < 16; i += 2) mul2(z[i], z[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), gs, gs);
     }
+}
+// eight column pairs: hidden = 2 gelu(z) or relu(z), packed bf16 (enough independent work for the tanh
+// unit's latency, few live registers)
+template <int ACT>
+__device__ __forceinline__ void pp_act8(const float* z, uint32_t* out) {
     if constexpr (ACT == SLICEMOE_ACT_RELU) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) out[i] = cvt_rn_relu_bf16x2(z[2 * i], z[2 * i + 1]);
@@ -314,8 +339,8 @@ __device__ __forceinline__ void pp_act8(const uint32_t* acc, float gs, const flo
 // OFFS_IN_SMEM: sh.offs already holds the row ranges.  Rows come from gather_src through pair_gate and
 // results are added into scatter_out.
 template <int N2, int ACT, bool SAME_LAUNCH, bool OFFS_IN_SMEM>
-__device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p, const PpParams& p,
-                                            PpShared& sh, uint8_t* smem_raw) {
+__device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p,
+                                            const PpParams& p, PpShared& sh, uint8_t* smem_raw) {
     using C = PpFfnCfg<N2>;
     using B = PpBars;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -328,8 +353,9 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
     // ---- set-up -----------------------------------------------------------------------------------
     if (threadIdx.x == 0) {
         sh.abort_flag = 0;
-        for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 64); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
+        for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 2); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(pp_bar(sh, B::W_FULL + i), 1); mbar_init(pp_bar(sh, B::W_EMPTY + i), 1); }
+        mbar_init(pp_bar(sh, B::DRAIN + 1), 1);
         for (int r = 0; r < 2; ++r) {                                  // per tensor-memory region
             mbar_init(pp_sbar(sh, r, B::ACC1_FULL), 1);
             mbar_init(pp_sbar(sh, r, B::HID_FULL), 16);
@@ -338,6 +364,7 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
         }
         mbar_init(pp_bar(sh, B::DRAIN), 1);
         fence_mbar_init();
+        prefetch_tensormap(tmXg_p);
         prefetch_tensormap(tmW1_p);
         prefetch_tensormap(tmW2_p);
     }
@@ -355,64 +382,33 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
     const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
     const uint32_t sA = smem_base + C::OFF_A, sW = smem_base + C::OFF_W;
 
-    if (warp == 0) {
-        // ================= TMA producer: one weight set per run ======================================
-        if (lane == 0 && ntiles > 0 && !DBG(64)) {
-            PpWalk wk;
-            wk.init();
-            int loaded_run = -1;
-            uint32_t last_bar = 0, last_par = 0;
-            bool ok = true;
-            const uint32_t set_tx = (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK);
-            for (int ta = 0; ta < ntiles && ok; ++ta) {
-                wk.advance(sh, t_begin, ta);
-                if (wk.run == loaded_run) continue;
-                loaded_run = wk.run;
-                const int set = wk.run & 1;
-                const uint32_t n = (uint32_t)wk.run >> 1;
-                if (!mbar_wait_sleepy(pp_bar(sh, B::W_EMPTY + set), (n & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
-                mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL + set), set_tx);
-                const uint32_t w1 = sW + set * C::SET_BYTES, w2 = w1 + C::W1_SET;
-                for (int c = 0; c < npanels; ++c) {
-                    tma_load_2d(w1 + c * (kPpHC * 128), tmW1_p, 0, wk.e * p.HID + c * kPpHC, pp_bar(sh, B::W_FULL + set));
-                    tma_load_2d(w2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, wk.e * N2, pp_bar(sh, B::W_FULL + set));
-                }
-                last_bar = pp_bar(sh, B::W_FULL + set);
-                last_par = n & 1u;
-            }
-            if (!ok || *abort) {
-                volatile int never = 0;
-                if (last_bar) mbar_wait(last_bar, last_par, &never, 10000000ull);   // let the last copies land
-            }
-        }
-    } else if (warp == 1) {
-        // ================= MMA issue ==================================================================
-        // Order: GEMM-1 of tiles 0 and 1; then per tile t: GEMM-2(t) once its hidden layer is written,
-        // GEMM-1(t + 2) once tile t's output accumulator has been read (same region).  All lanes run the
-        // loop (descriptors stay in uniform registers); one elected lane issues.
+    if (false) {
+    } else if (warp == 3) {
+        // ================= GEMM-1 issue ===============================================================
+        // GEMM-1 of tile t goes into region t mod 2 once the output accumulator of tile t - 2 has been
+        // read: it runs up to two tiles ahead of the activation.  Two issuing warps (this one and the
+        // GEMM-2 warp): an issuing warp's waits and book-keeping are serial work on the tile's critical path.
+        // All lanes run the loop (descriptors stay in uniform registers); one elected lane issues.
         if (ntiles > 0) {
             const uint32_t idesc1 = make_idesc(128, p.HID, kFmtBF16, kFmtBF16);
-            constexpr uint32_t idesc2 = make_idesc(128, N2, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
             bool ok = true;
             TRD(tr, warp);
-            PpWalk w1, w2;
+            PpWalk w1;
             w1.init();
-            w2.init();
             int run1 = -1;
-            auto issue_g1 = [&](int ta) {
+#pragma unroll 1
+            for (int ta = 0; ta < ntiles && ok; ++ta) {
                 const int ab = ta % kPpABufs, r = ta & 1;
                 w1.advance(sh, t_begin, ta);
                 if (w1.run != run1) {
-                    if (!pp_wait(pp_bar(sh, B::W_FULL + (w1.run & 1)), ((uint32_t)w1.run >> 1) & 1u, abort)) { ok = false; return; }
+                    if (!pp_wait(pp_bar(sh, B::W_FULL + (w1.run & 1)), ((uint32_t)w1.run >> 1) & 1u, abort)) { ok = false; break; }
                     run1 = w1.run;
                 }
                 TR(tr, 8);
-                if (!pp_wait(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u, abort)) { ok = false; return; }
-                fence_proxy_async_smem();     // rows written by cp.async -> visible to the MMA's reads
+                if (!pp_wait(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u, abort)) { ok = false; break; }
                 TR(tr, 10);
-                // the region is free once the output accumulator of the tile two back has been read
-                if (!pp_wait(pp_sbar(sh, r, B::ACC2_EMPTY), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; return; }
+                if (!pp_wait(pp_sbar(sh, r, B::ACC2_EMPTY), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
                 TR(tr, 11);
                 tc_fence_after_sync();
                 const uint32_t wset = dW + (((w1.run & 1) * C::SET_BYTES) >> 4);
@@ -427,18 +423,36 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
                 }
                 __syncwarp();
                 TR(tr, 12);
-            };
-            issue_g1(0);
-            if (ok && ntiles > 1) issue_g1(1);
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                if (lane == 0) {
+                    mma_commit(pp_bar(sh, B::DRAIN));
+                    mbar_wait(pp_bar(sh, B::DRAIN), 0u, &never, 10000000ull);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 1) {
+        // ================= GEMM-2 issue ===============================================================
+        if (ntiles > 0) {
+            constexpr uint32_t idesc2 = make_idesc(128, N2, kFmtBF16, kFmtBF16);
+            const uint32_t dW = desc_lo_sw128(sW);
+            bool ok = true;
+            TRD(tr, warp);
+            PpWalk w2;
+            w2.init();
+            w2.advance(sh, t_begin, 0);
 #pragma unroll 1
             for (int ta = 0; ta < ntiles && ok; ++ta) {
                 const int r = ta & 1;
-                w2.advance(sh, t_begin, ta);
+                const uint32_t w2d = dW + (((w2.run & 1) * C::SET_BYTES + C::W1_SET) >> 4);
+                const int run_before = w2.run;
+                const int crossed = ta + 1 < ntiles ? w2.advance(sh, t_begin, ta + 1) : 0;   // (before the wait: off the critical path)
                 TR(tr, 20);
                 if (!pp_wait(pp_sbar(sh, r, B::HID_FULL), (uint32_t)(ta >> 1) & 1u, abort)) { ok = false; break; }
                 TR(tr, 21);
                 tc_fence_after_sync();
-                const uint32_t w2d = dW + (((w2.run & 1) * C::SET_BYTES + C::W1_SET) >> 4);
                 const uint32_t d = tmem_base + r * kPpStreamCols;
                 if (elect_one_sync()) {
                     // K step kk = hidden units [16 kk, 16 kk + 16): units below 128 sit at packed column
@@ -451,78 +465,110 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
                         mma_ts_dyn(d + C::ACC2_COL, a, bd, idesc2, kk > 0 ? 1u : 0u);
                     }
                     mma_commit(pp_sbar(sh, r, B::ACC2_FULL));
+                    // a run that ends here hands its weight set back (GEMM-1 of these tiles finished before
+                    // their GEMM-2 began, so this commit covers the other issuing warp's reads as well)
+                    if (crossed) mma_commit(pp_bar(sh, B::W_EMPTY + (run_before & 1)));
                 }
                 __syncwarp();
                 TR(tr, 22);
-                // hand the weight sets of the runs that end here back
-                if (ta + 1 < ntiles) {
-                    const int run_before = w2.run;
-                    const int crossed = w2.advance(sh, t_begin, ta + 1);
-                    if (crossed) {
-                        if (elect_one_sync()) mma_commit(pp_bar(sh, B::W_EMPTY + (run_before & 1)));
-                        __syncwarp();
-                    }
-                }
-                if (ta + 2 < ntiles) issue_g1(ta + 2);
             }
             if (!ok || *abort) {
                 volatile int never = 0;
                 if (lane == 0) {
-                    mma_commit(pp_bar(sh, B::DRAIN));
-                    mbar_wait(pp_bar(sh, B::DRAIN), 0u, &never, 10000000ull);
+                    mma_commit(pp_bar(sh, B::DRAIN + 1));
+                    mbar_wait(pp_bar(sh, B::DRAIN + 1), 0u, &never, 10000000ull);
                 }
                 __syncwarp();
             }
         }
-    } else if (warp == 2 || warp == 3) {
-        // ================= gather warps (rows 0..63 / 64..127 of a tile) ==============================
-        // Row r of tile ta is stacked row row0 + r = pair (n, j); its A row is X[n, :], copied with
-        // asynchronous 16-byte copies into the K-major 128-byte-swizzled layout, up to four tiles ahead.
-        if (ntiles > 0 && !DBG(64)) {
-            const int ch = lane & 7, rsub = lane >> 3;
-            const int rbase = (warp - 2) * 64;
+    } else if (warp == 0 || warp == 2) {
+        // ================= gather warps (tile rows 0..63: warp 2; 64..127: warp 0, which also loads the weights)
+        // Row r of tile ta is stacked row row0 + r = pair (n, j); its A row is X[n, :].  A lane fetches four
+        // tile rows with one four-row gather of the copy engine (no per-lane address arithmetic, nothing
+        // through the load/store pipe that the activation warps' tanh instructions share), up to four tiles
+        // ahead; a warp's gathers are issued one after the other, hence two warps of 16 lanes.  Rows past the
+        // tile's end fetch row 0: they are computed and never stored.
+        // Weights: one set (W1 and W2 of an expert) per run of tiles of the same expert, two sets in shared
+        // memory; a set is loaded as soon as the run before the previous one has been computed.
+        if (ntiles > 0) {
+            const int rbase = warp == 2 ? 0 : 64;
             PpWalk wn;
             wn.init();
-            int nnext[2];
+            int2 nnext[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) nnext[q] = make_int2(-1, 0);
+            int loaded_run = -1, cur_e = 0, cur_run = 0, cur_rows = 0;
+            uint32_t last_bar = 0, last_par = 0;
             bool ok = true;
             TRD(tr, warp);
-            const bool in_row = ch * 8 < p.row_elems;
+            const uint32_t set_tx = (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK);
 #pragma unroll 1
             for (int ta = -1; ta < ntiles && ok; ++ta) {
-                int nrow[2];
+                int nrow[4];
+                int2 cur_pg[4];
 #pragma unroll
-                for (int q = 0; q < 2; ++q) nrow[q] = (ta < 0 || nnext[q] < 0) ? -1 : pair_to_row(nnext[q], p.gather_magic, p.gather_shift);
+                for (int q = 0; q < 4; ++q) {
+                    cur_pg[q] = nnext[q];
+                    nrow[q] = nnext[q].x < 0 ? 0 : pair_to_row(nnext[q].x, p.gather_magic, p.gather_shift);
+                }
+                if (ta >= 0) { cur_e = wn.e; cur_run = wn.run; cur_rows = wn.rows; }
                 if (ta + 1 < ntiles) {
                     wn.advance(sh, t_begin, ta + 1);
 #pragma unroll
-                    for (int q = 0; q < 2; ++q) {
-                        const int r = rbase + lane + 32 * q;
-                        nnext[q] = (r < wn.rows) ? ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wn.row0 + r)) : -1;
+                    for (int q = 0; q < 4; ++q) {
+                        const int r = rbase + 4 * (lane & 15) + q;
+                        nnext[q] = make_int2(-1, 0);
+                        if (r < wn.rows) nnext[q] = SAME_LAUNCH ? __ldcg(p.pair_gate + wn.row0 + r) : __ldg(p.pair_gate + wn.row0 + r);
                     }
                 }
                 if (ta < 0) continue;
+                if (warp == 0 && cur_run != loaded_run) {
+                    loaded_run = cur_run;
+                    const int set = cur_run & 1;
+                    const uint32_t n = (uint32_t)cur_run >> 1;
+                    ok = pp_wait(pp_bar(sh, B::W_EMPTY + set), (n & 1u) ^ 1u, abort);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL + set), set_tx);
+                        const uint32_t w1 = sW + set * C::SET_BYTES, w2 = w1 + C::W1_SET;
+                        for (int c = 0; c < npanels; ++c) {
+                            tma_load_2d(w1 + c * (kPpHC * 128), tmW1_p, 0, cur_e * p.HID + c * kPpHC, pp_bar(sh, B::W_FULL + set));
+                            tma_load_2d(w2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, cur_e * N2, pp_bar(sh, B::W_FULL + set));
+                        }
+                    }
+                    __syncwarp();
+                    last_bar = pp_bar(sh, B::W_FULL + set);
+                    last_par = n & 1u;
+                }
                 const int ab = ta % kPpABufs;
                 TR(tr, 30);
                 ok = pp_wait(pp_bar(sh, B::A_EMPTY + ab), ((uint32_t)(ta / kPpABufs) & 1u) ^ 1u, abort);
                 if (!ok) break;
                 TR(tr, 31);
-                const uint32_t dst0 = sA + ab * kPpABytes;
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int r32 = i * 4 + rsub;
-                        const int r = rbase + q * 32 + r32;
-                        const int n = __shfl_sync(0xffffffffu, nrow[q], r32);
-                        const bool real = n >= 0 && in_row;
-                        const bf16* src = p.gather_src + (real ? (size_t)n * p.row_elems + ch * 8 : 0);
-                        if (!DBG(1)) cp_async_16(dst0 + (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4), src, real ? 16u : 0u);
-                    }
+                // the tile's metadata (its ring entry was last read by the output warps of tile ta - kPpMetaRing,
+                // long before GEMM-1 of tile ta - kPpABufs, whose completion this warp has just waited for)
+                if (lane < 16) {
+                    int2* dst = &sh.pair_gate_s[ta % kPpMetaRing][rbase + 4 * lane];
+                    reinterpret_cast<int4*>(dst)[0] = make_int4(cur_pg[0].x, cur_pg[0].y, cur_pg[1].x, cur_pg[1].y);
+                    reinterpret_cast<int4*>(dst)[1] = make_int4(cur_pg[2].x, cur_pg[2].y, cur_pg[3].x, cur_pg[3].y);
                 }
-                cp_async_mbar_arrive_noinc(pp_bar(sh, B::A_FULL + ab));
+                if (lane == 0 && warp == 2) sh.tile_s[ta % kPpMetaRing] = make_int4(cur_e, cur_run, cur_rows, 0);
+                __syncwarp();
+                if (lane == 0) {
+                    if (warp == 2) mbar_arrive_expect_tx(pp_bar(sh, B::A_FULL + ab), kPpABytes);
+                    else mbar_arrive(pp_bar(sh, B::A_FULL + ab));
+                }
+                if (lane < 16 && !DBG(1))
+                    tma_gather4(sA + ab * kPpABytes + (rbase / 4 + lane) * 512, tmXg_p, 0, nrow[0], nrow[1], nrow[2], nrow[3], pp_bar(sh, B::A_FULL + ab));
                 TR(tr, 32);
             }
-            cp_async_wait_all();
+            if (!ok || *abort) {
+                // (bounded) let the copies in flight land before shared memory is reused
+                volatile int never = 0;
+                const int last = ntiles - 1;
+                if (last >= 0) mbar_wait(pp_bar(sh, B::A_FULL + last % kPpABufs), (uint32_t)(last / kPpABufs) & 1u, &never, 10000000ull);
+                if (last_bar) mbar_wait(last_bar, last_par, &never, 10000000ull);
+            }
         }
     } else if (warp < 20) {
         // ================= activation warps: warpgroup g, lane group lg ================================
@@ -532,51 +578,45 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
         bool ok = true;
         TRD(tr, warp);
-        PpWalk wk;
-        wk.init();
-        float gate_next = 0.0f;          // Eq. 1's gate of this thread's row of the coming tile
-        if (ntiles > 0) {
-            wk.advance(sh, t_begin, 0);
-            if (row < wk.rows) gate_next = __int_as_float(ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row) + 1));
-        }
         int run_bias = -1;
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
             const int r = ta & 1;
-            const float gs = gate_next;
-            if (has_b1 && wk.run != run_bias) {
-                // a new run: its expert's first-layer bias as fp32 (two buffers by run parity: the other
-                // one may still be in use by warps that are behind)
-                for (int f = g * 128 + row; f < p.HID; f += 512) sh.bias1_f32[wk.run & 1][f] = __bfloat162float(p.b1[(size_t)wk.e * p.HID + f]);
-                named_barrier_sync(1, 512);
-                run_bias = wk.run;
-            }
-            const float* bias = sh.bias1_f32[wk.run & 1] + 32 * g;
-            // the next tile's gate (first used at the top of the next turn)
-            if (ta + 1 < ntiles) {
-                wk.advance(sh, t_begin, ta + 1);
-                gate_next = 0.0f;
-                if (row < wk.rows) gate_next = __int_as_float(ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row) + 1));
-            }
             TR(tr, 40);
             ok = pp_wait(pp_sbar(sh, r, B::ACC1_FULL), (uint32_t)(ta >> 1) & 1u, abort);
             if (!ok) break;
             TR(tr, 41);
             tc_fence_after_sync();
+            // (the tile's rows, and with them its ring entry, landed before GEMM-1 could run)
+            const float gs = __int_as_float(sh.pair_gate_s[ta % kPpMetaRing][row].y);
+            if (has_b1) {
+                const int4 ti = sh.tile_s[ta % kPpMetaRing];
+                if (ti.y != run_bias) {
+                    // a new run: its expert's first-layer bias as fp32 (two buffers by run parity: the other
+                    // one may still be in use by warps that are behind)
+                    for (int f = g * 128 + row; f < p.HID; f += 512) sh.bias1_f32[ti.y & 1][f] = __bfloat162float(p.b1[(size_t)ti.x * p.HID + f]);
+                    named_barrier_sync(1, 512);
+                    run_bias = ti.y;
+                }
+            }
+            const float* bias = sh.bias1_f32[run_bias & 1] + 32 * g;
             const uint32_t region = tlane + r * kPpStreamCols + 32 * g;
             // 16 hidden units per turn: units [32 g + 16 q, +16) (q = 0, 1) and [128 + 32 g + 16 (q - 2), +16)
             // (q = 2, 3); their packed values go to columns [32 g + 8 q, +8), which this thread has read before
+            // (the next turn's accumulator columns are requested as soon as this turn's are scaled into z:
+            // the load's latency runs under the tanh work)
+            const int nq = wide ? 4 : 2;
+            uint32_t acc[16];
+            tmem_ld_x16(region, acc);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                if (q == 2 && !wide) break;
-                uint32_t acc[16], hid[8];
-                tmem_ld_x16(region + (q < 2 ? 16 * q : 128 + 16 * (q - 2)), acc);
+                if (q >= nq) break;
+                float z[16];
+                uint32_t hid[8];
                 tmem_ld_wait();
-                if (!DBG(8)) pp_act8<ACT>(acc, gs, bias + (q < 2 ? 16 * q : 128 + 16 * (q - 2)), has_b1, hid);
-                else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) hid[i] = acc[i] ^ acc[i + 8];
-                }
+                pp_scale16(acc, gs, bias + (q < 2 ? 16 * q : 128 + 16 * (q - 2)), has_b1, z);
+                if (q + 1 < nq) tmem_ld_x16(region + (q + 1 < 2 ? 16 * (q + 1) : 128 + 16 * (q - 1)), acc);
+                pp_act8<ACT>(z, hid);
                 tmem_st_x8(region + 8 * q, hid);
             }
             TR(tr, 45);
@@ -594,59 +634,51 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
         bool ok = true;
         TRD(tr, warp);
-        PpWalk wk;
-        wk.init();
-        int pair_next = 0;
-        if (ntiles > 0) {
-            wk.advance(sh, t_begin, 0);
-            if (row < wk.rows) pair_next = ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row));
-        }
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
             const int r = ta & 1;
-            const bool live = row < wk.rows;
-            const int e_cur = wk.e;
-            bf16* dst = p.scatter_out + (size_t)pair_to_row(pair_next, p.gather_magic, p.gather_shift) * N2;
-            if (ta + 1 < ntiles) {
-                wk.advance(sh, t_begin, ta + 1);
-                if (row < wk.rows) pair_next = ld_index<SAME_LAUNCH>(reinterpret_cast<const int32_t*>(p.pair_gate + wk.row0 + row));
-            }
             TR(tr, 49);
             ok = pp_wait(pp_sbar(sh, r, B::ACC2_FULL), (uint32_t)(ta >> 1) & 1u, abort);
             if (!ok) break;
             TR(tr, 50);
             tc_fence_after_sync();
+            const int4 ti = sh.tile_s[ta % kPpMetaRing];       // (expert, run, rows) of the tile
+            const bool live = row < ti.z;
+            const int e_cur = ti.x;
+            bf16* dst = p.scatter_out + (size_t)pair_to_row(sh.pair_gate_s[ta % kPpMetaRing][row].x, p.gather_magic, p.gather_shift) * N2;
             const uint32_t acc2 = tlane + r * kPpStreamCols + C::ACC2_COL;
             constexpr float sc = kOutScale<ACT>;
-#pragma unroll 1
+            // the whole accumulator row goes into registers (as packed bf16 pairs of 0.5 acc: half the
+            // registers) so that the region is handed back at once: its next GEMM-1 waits for this
+            uint32_t o[N2 / 2];
+#pragma unroll
             for (int cb = 0; cb < N2; cb += 16) {
                 uint32_t v[16];
                 tmem_ld_x16(acc2 + cb, v);
                 tmem_ld_wait();
-                if (cb + 16 >= N2) {
-                    // the accumulator is in registers: the region may be reused
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
-                    TR(tr, 52);
-                }
-                if (!live) continue;
+                if (p.b2) {
 #pragma unroll
-                for (int c = 0; c < 16; c += 8) {
-                    float bb[8];
-                    if (p.b2) {
+                    for (int c = 0; c < 16; c += 8) {
+                        float bb[8];
                         unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.b2 + (size_t)e_cur * N2 + cb + c)), bb);
-                    } else {
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) bb[q] = 0.0f;
+                        for (int q = 0; q < 4; ++q)
+                            o[(cb + c) / 2 + q] = pack_bf16x2(fmaf(__uint_as_float(v[c + 2 * q]), sc, bb[2 * q]),
+                                                              fmaf(__uint_as_float(v[c + 2 * q + 1]), sc, bb[2 * q + 1]));
                     }
-                    uint32_t o[4];
+                } else {
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        o[q] = pack_bf16x2(fmaf(__uint_as_float(v[c + 2 * q]), sc, bb[2 * q]),
-                                           fmaf(__uint_as_float(v[c + 2 * q + 1]), sc, bb[2 * q + 1]));
-                    if (!DBG(4)) red_add_bf16x8(dst + cb + c, o[0], o[1], o[2], o[3]);
+                    for (int q = 0; q < 8; ++q)
+                        o[cb / 2 + q] = pack_bf16x2(__uint_as_float(v[2 * q]) * sc, __uint_as_float(v[2 * q + 1]) * sc);
                 }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
+            TR(tr, 52);
+            if (live && !DBG(4)) {
+#pragma unroll
+                for (int c = 0; c < N2; c += 8) red_add_bf16x8(dst + c, o[c / 2], o[c / 2 + 1], o[c / 2 + 2], o[c / 2 + 3]);
             }
             TR(tr, 53);
         }
@@ -663,11 +695,16 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmW1_p, const CUt
 
 // =====================================================================================================
 // Router pass.  EP: expert count the kernel is built for (16 / 32 / 64; fewer real experts are padded,
-// their logits set to -inf).  Shared memory: X buffers 4 x 16 KB | Wr1 [Hr, 64] | Wr2 as Hr/64 chunks
-// of [EP, 64].  TMEM per stream: [0,192) three GEMM-1 accumulators; the hidden chunk is written over
-// the accumulator it came from as a bf16 pair hi + lo (16 mantissa bits: K step kk of a chunk is at
-// columns 16 kk (hi) and 16 kk + 8 (lo)), so that the logits do not depend on 16-bit rounding of the
-// hidden layer; [192, 192 + EP) the logits.
+// their logits set to -inf).  Shared memory: X buffers 4 x 16 KB | Wr1 [Hr, 64] | Wr2 as Hr/64 panels
+// of [EP, 64].
+// The hidden layer of a tile is taken in halves of 128 units ("units of work"): GEMM-1 (N = 128) into one
+// of three 128-column buffers of tensor memory; the 16 activation warps (warpgroup g: columns [32 g, 32 g +
+// 32), 16 at a time) add the bias and write relu(.) back over the accumulator as a bf16 pair hi + lo (16
+// mantissa bits: K step kk of a half is at columns 16 kk (hi) and 16 kk + 8 (lo)), so that the logits do
+// not depend on 16-bit rounding of the hidden layer; GEMM-2 runs over hi and lo from tensor memory into
+// one of two logit accumulators (columns [384, 448) and [448, 512)), accumulating over the halves; the
+// output warpgroup turns a tile's logits into softmax probabilities, the top-k and each pair's rank among
+// this CTA's pairs of its expert.  GEMM-1 runs two units ahead of GEMM-2.
 // =====================================================================================================
 template <int EP>
 struct PpRouteCfg {
@@ -677,7 +714,7 @@ struct PpRouteCfg {
     static constexpr int OFF_W2 = OFF_W1 + kPpMaxHr * 128;
     static constexpr int SMEM_BYTES = OFF_W2 + (kPpMaxHr / kPpHC) * W2_CHUNK;
     static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;
-    static constexpr int ACC1_COL = 0, ACC2_COL = 192;
+    static constexpr int HB_COLS = 128, LOGIT_COL = 384;
     static_assert(EP % 16 == 0 && EP <= 64, "expert count");
 };
 
@@ -689,20 +726,23 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     volatile int* abort = &sh.abort_flag;
-    const int nchunks = p.HID / kPpHC;
+    const int npanels = p.HID / kPpHC;
+    const int nhalf = p.HID / 128;            // units of work per tile
 
+    // Barrier use in this pass (slots of "stream" 0): ACC1_FULL[3] / ACC1_EMPTY[3] / HID_FULL[3] per hidden
+    // buffer; the logit accumulators use ACC2_FULL / ACC2_EMPTY of "streams" 0 and 1.
     if (threadIdx.x == 0) {
         sh.abort_flag = 0;
         for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 1); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
         mbar_init(pp_bar(sh, B::W_FULL), 1);
-        for (int s = 0; s < 2; ++s) {
-            for (int i = 0; i < 3; ++i) {
-                mbar_init(pp_sbar(sh, s, B::ACC1_FULL + i), 1);
-                mbar_init(pp_sbar(sh, s, B::ACC1_EMPTY + i), 1);
-                mbar_init(pp_sbar(sh, s, B::HID_FULL + i), 8);
-            }
-            mbar_init(pp_sbar(sh, s, B::ACC2_FULL), 1);
-            mbar_init(pp_sbar(sh, s, B::ACC2_EMPTY), 4);
+        for (int i = 0; i < 3; ++i) {
+            mbar_init(pp_sbar(sh, 0, B::ACC1_FULL + i), 1);
+            mbar_init(pp_sbar(sh, 0, B::ACC1_EMPTY + i), 1);
+            mbar_init(pp_sbar(sh, 0, B::HID_FULL + i), 16);
+        }
+        for (int r = 0; r < 2; ++r) {
+            mbar_init(pp_sbar(sh, r, B::ACC2_FULL), 1);
+            mbar_init(pp_sbar(sh, r, B::ACC2_EMPTY), 4);
         }
         mbar_init(pp_bar(sh, B::DRAIN), 1);
         mbar_init(pp_bar(sh, B::DRAIN + 1), 1);
@@ -723,14 +763,15 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
     const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
     const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
     const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
+    const int nunits = ntiles * nhalf;
     const uint32_t sA = smem_base + C::OFF_A, sW1 = smem_base + C::OFF_W1, sW2 = smem_base + C::OFF_W2;
 
     if (warp == 0) {
         // ================= TMA producer ===============================================================
         if (lane == 0 && ntiles > 0) {
             bool ok = true;
-            mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + nchunks * C::W2_CHUNK));
-            for (int c = 0; c < nchunks; ++c) {
+            mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK));
+            for (int c = 0; c < npanels; ++c) {
                 tma_load_2d(sW1 + c * (kPpHC * 128), tmW1_p, 0, c * kPpHC, pp_bar(sh, B::W_FULL));
                 tma_load_2d(sW2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, 0, pp_bar(sh, B::W_FULL));
             }
@@ -748,94 +789,94 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
                 mbar_wait(last_bar, last_par, &never, 10000000ull);
             }
         }
-    } else if (warp == 1 || warp == 2) {
-        // ================= MMA issue, stream s ========================================================
-        const int s = warp - 1;
-        const int n_my = (ntiles - s + 1) / 2;
-        const int Q = n_my * nchunks;
-        if (Q > 0) {
-            constexpr uint32_t idesc1 = make_idesc(128, kPpHC, kFmtBF16, kFmtBF16);
-            constexpr uint32_t idesc2 = make_idesc(128, EP, kFmtBF16, kFmtBF16);
-            const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1), dW2 = desc_lo_sw128(sW2);
-            const uint32_t tcol = tmem_base + s * kPpStreamCols;
+    } else if (warp == 3) {
+        // ================= GEMM-1 issue (two units ahead of GEMM-2: three hidden buffers) =============
+        if (nunits > 0) {
+            constexpr uint32_t idesc1 = make_idesc(128, 128, kFmtBF16, kFmtBF16);
+            const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1);
             bool ok = true;
-            int q1 = 0, c1 = 0, i1 = 0;
-            int q2 = 0, c2 = 0, i2 = 0;
-            TRD(tr, 20 + warp);
-            auto wait_all = [&](uint32_t bar, uint32_t parity) {
-                return (bool)__all_sync(0xffffffffu, mbar_wait(bar, parity, abort, kWaitLimitNs));
-            };
-            if (!wait_all(pp_bar(sh, B::W_FULL), 0u)) ok = false;
-            auto issue_g1 = [&]() {
-                const int ta = s + 2 * i1;
+            TRD(tr, 40 + warp);
+            ok = pp_wait(pp_bar(sh, B::W_FULL), 0u, abort);
+#pragma unroll 1
+            for (int u = 0; u < nunits && ok; ++u) {
+                const int ta = u / nhalf, hf = u - ta * nhalf;
                 const int ab = ta % kPpABufs;
                 TR(tr, 8);
-                if (c1 == 0 && !wait_all(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u)) { ok = false; return; }
-                const uint32_t b = (uint32_t)q1 % 3u, n = (uint32_t)q1 / 3u;
+                if (hf == 0 && !pp_wait(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u, abort)) { ok = false; break; }
+                const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
                 TR(tr, 10);
-                // (the accumulator also held the previous chunk's hidden values: GEMM-2 must have read them)
-                if (!wait_all(pp_sbar(sh, s, B::ACC1_EMPTY + b), (n & 1u) ^ 1u)) { ok = false; return; }
+                // (the buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
+                if (!pp_wait(pp_sbar(sh, 0, B::ACC1_EMPTY + b), (n & 1u) ^ 1u, abort)) { ok = false; break; }
                 TR(tr, 11);
                 tc_fence_after_sync();
-                const uint32_t a0 = dA + ((ab * kPpABytes) >> 4), w0 = dW1 + ((c1 * (kPpHC * 128)) >> 4);
-                const uint32_t d = tcol + C::ACC1_COL + b * kPpHC;
-                const bool last = c1 == nchunks - 1;
+                const uint32_t a0 = dA + ((ab * kPpABytes) >> 4), w0 = dW1 + ((hf * (128 * 128)) >> 4);
+                const uint32_t d = tmem_base + b * C::HB_COLS;
                 if (elect_one_sync()) {
                     mma_ss<0>(d, a0, w0, idesc1);
 #pragma unroll
                     for (int kk = 1; kk < 4; ++kk) mma_ss<1>(d, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
-                    mma_commit(pp_sbar(sh, s, B::ACC1_FULL + b));
-                    if (last) mma_commit(pp_bar(sh, B::A_EMPTY + ab));
+                    mma_commit(pp_sbar(sh, 0, B::ACC1_FULL + b));
+                    if (hf == nhalf - 1) mma_commit(pp_bar(sh, B::A_EMPTY + ab));
                 }
                 __syncwarp();
                 TR(tr, 12);
-                ++q1;
-                if (last) { c1 = 0; ++i1; } else { ++c1; }
-            };
-            auto issue_g2 = [&]() {
-                TR(tr, 19);
-                if (c2 == 0 && !wait_all(pp_sbar(sh, s, B::ACC2_EMPTY), ((uint32_t)i2 & 1u) ^ 1u)) { ok = false; return; }
-                const uint32_t b = (uint32_t)q2 % 3u, n = (uint32_t)q2 / 3u;
-                TR(tr, 20);
-                if (!wait_all(pp_sbar(sh, s, B::HID_FULL + b), n & 1u)) { ok = false; return; }
-                TR(tr, 21);
-                tc_fence_after_sync();
-                const uint32_t w0 = dW2 + ((c2 * C::W2_CHUNK) >> 4);
-                const uint32_t d = tcol + C::ACC2_COL, a = tcol + C::ACC1_COL + b * kPpHC;
-                const bool last = c2 == nchunks - 1;
-                if (elect_one_sync()) {
-#pragma unroll
-                    for (int part = 0; part < 2; ++part) {
-#pragma unroll
-                        for (int kk = 0; kk < kPpHC / 16; ++kk) {
-                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, w0, idesc2, c2 > 0 ? 1u : 0u);
-                            else mma_ts<1>(d, a + kk * 16 + part * 8, w0 + ((kk * 32) >> 4), idesc2);
-                        }
-                    }
-                    mma_commit(pp_sbar(sh, s, B::ACC1_EMPTY + b));
-                    if (last) mma_commit(pp_sbar(sh, s, B::ACC2_FULL));
-                }
-                __syncwarp();
-                TR(tr, 22);
-                ++q2;
-                if (last) { c2 = 0; ++i2; } else { ++c2; }
-            };
-            if (ok) issue_g1();
-            if (ok && Q > 1) issue_g1();
-            while (ok && q2 < Q) {
-                issue_g2();
-                if (ok && q1 < Q) issue_g1();
             }
             if (!ok || *abort) {
                 volatile int never = 0;
                 if (lane == 0) {
-                    mma_commit(pp_bar(sh, B::DRAIN + s));
-                    mbar_wait(pp_bar(sh, B::DRAIN + s), 0u, &never, 10000000ull);
+                    mma_commit(pp_bar(sh, B::DRAIN));
+                    mbar_wait(pp_bar(sh, B::DRAIN), 0u, &never, 10000000ull);
                 }
                 __syncwarp();
             }
         }
-    } else if (warp == 3) {
+    } else if (warp == 1) {
+        // ================= GEMM-2 issue ===============================================================
+        if (nunits > 0) {
+            constexpr uint32_t idesc2 = make_idesc(128, EP, kFmtBF16, kFmtBF16);
+            const uint32_t dW2 = desc_lo_sw128(sW2);
+            bool ok = true;
+            TRD(tr, 40 + warp);
+            ok = pp_wait(pp_bar(sh, B::W_FULL), 0u, abort);
+#pragma unroll 1
+            for (int u = 0; u < nunits && ok; ++u) {
+                const int ta = u / nhalf, hf = u - ta * nhalf;
+                const int r = ta & 1;
+                TR(tr, 19);
+                if (hf == 0 && !pp_wait(pp_sbar(sh, r, B::ACC2_EMPTY), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
+                const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
+                TR(tr, 20);
+                if (!pp_wait(pp_sbar(sh, 0, B::HID_FULL + b), n & 1u, abort)) { ok = false; break; }
+                TR(tr, 21);
+                tc_fence_after_sync();
+                const uint32_t w0 = dW2 + ((hf * 2 * C::W2_CHUNK) >> 4);
+                const uint32_t d = tmem_base + C::LOGIT_COL + r * 64, a = tmem_base + b * C::HB_COLS;
+                if (elect_one_sync()) {
+#pragma unroll
+                    for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t bd = w0 + (((kk >> 2) * C::W2_CHUNK + (kk & 3) * 32) >> 4);
+                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, hf > 0 ? 1u : 0u);
+                            else mma_ts<1>(d, a + kk * 16 + part * 8, bd, idesc2);
+                        }
+                    }
+                    mma_commit(pp_sbar(sh, 0, B::ACC1_EMPTY + b));
+                    if (hf == nhalf - 1) mma_commit(pp_sbar(sh, r, B::ACC2_FULL));
+                }
+                __syncwarp();
+                TR(tr, 22);
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                if (lane == 0) {
+                    mma_commit(pp_bar(sh, B::DRAIN + 1));
+                    mbar_wait(pp_bar(sh, B::DRAIN + 1), 0u, &never, 10000000ull);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 2) {
         // ================= zero this CTA's rows of h' =================================================
         if (p.zero_out != nullptr && ntiles > 0) {
             const long long row_lo = (long long)t_begin * kTileM;
@@ -847,124 +888,110 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             for (long long i = lane; i < nvec; i += 32) dst[i] = z;
         }
     } else if (warp < 20) {
-        // ================= row threads of stream s, column half hh ====================================
-        // (the two halves take the tiles' softmax / top-k step in turn; warps 20..23 have no part here)
-        const int wg = (warp - 4) >> 2;
-        const int s = wg & 1, hh = wg >> 1;
+        // ================= activation warps: warpgroup g, lane group lg ================================
+        const int g = (warp - 4) >> 2;
+        const int lg = warp & 3;
+        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + 32 * g;
+        bool ok = true;
+        TRD(tr, 40 + warp);
+#pragma unroll 1
+        for (int u = 0; u < nunits && ok; ++u) {
+            const int ta = u / nhalf, hf = u - ta * nhalf;
+            const uint32_t b = (uint32_t)u % 3u, par = ((uint32_t)u / 3u) & 1u;
+            TR(tr, 40);
+            ok = pp_wait(pp_sbar(sh, 0, B::ACC1_FULL + b), par, abort);
+            if (!ok) break;
+            TR(tr, 41);
+            tc_fence_after_sync();
+            const uint32_t acol = tlane + b * C::HB_COLS;
+            const float* bias = sh.bias1_f32[0] + hf * 128 + 32 * g;
+#pragma unroll
+            for (int pc = 0; pc < 2; ++pc) {
+                // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu),
+                // lo = the rounded remainder (for a negative value the remainder is the value itself and
+                // its .relu is 0 as well)
+                uint32_t acc[16];
+                tmem_ld_x16(acol + 16 * pc, acc);
+                tmem_ld_wait();
+                float a[16];
+#pragma unroll
+                for (int i = 0; i < 16; i += 4) {
+                    const float4 bb = *reinterpret_cast<const float4*>(bias + pc * 16 + i);
+                    add2(a[i], a[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), bb.x, bb.y);
+                    add2(a[i + 2], a[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), bb.z, bb.w);
+                }
+                uint32_t hl[16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) hl[i] = cvt_rz_relu_bf16x2(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    hl[8 + i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hl[i] << 16), a[2 * i + 1] - __uint_as_float(hl[i] & 0xFFFF0000u));
+                tmem_st_x16(acol + 16 * pc, hl);
+            }
+            TR(tr, 45);
+            tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pp_sbar(sh, 0, B::HID_FULL + b));
+            TR(tr, 46);
+        }
+    } else {
+        // ================= output warpgroup ===========================================================
+        // softmax + top-k of a tile's logits (ties go to the lower id), this CTA's rank of each pair
         const int lg = warp & 3;
         const int row = lg * 32 + lane;
-        const uint32_t tcol = tmem_base + ((uint32_t)(lg * 32) << 16) + s * kPpStreamCols;
-        const int n_my = (ntiles - s + 1) / 2;
+        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + C::LOGIT_COL;
         bool ok = true;
-        bool pend = false;
-        int pend_ta = 0;
-        uint32_t pend_i = 0;
-        // softmax + top-k of a finished tile's logits (ties go to the lower id), this CTA's rank of each pair
-        auto output_tile = [&]() {
-            ok = mbar_wait(pp_sbar(sh, s, B::ACC2_FULL), pend_i & 1u, abort, kWaitLimitNs);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) return;
+        TRD(tr, 40 + warp);
+#pragma unroll 1
+        for (int ta = 0; ta < ntiles && ok; ++ta) {
+            const int r = ta & 1;
+            TR(tr, 49);
+            ok = pp_wait(pp_sbar(sh, r, B::ACC2_FULL), (uint32_t)(ta >> 1) & 1u, abort);
+            if (!ok) break;
+            TR(tr, 50);
             tc_fence_after_sync();
             uint32_t v[EP];
 #pragma unroll
-            for (int c = 0; c < EP; c += 16) tmem_ld_x16(tcol + C::ACC2_COL + c, v + c);
+            for (int c = 0; c < EP; c += 16) tmem_ld_x16(tlane + r * 64 + c, v + c);
             tmem_ld_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(pp_sbar(sh, s, B::ACC2_EMPTY));
-            pend = false;
-            const int n = (t_begin + pend_ta) * kTileM + row;
-            if (n >= p.n_rows) return;
-            float gl[EP];
-#pragma unroll
-            for (int i = 0; i < EP; i += 4) {
-                const float4 b = *reinterpret_cast<const float4*>(sh.bias2_f32 + i);
-                add2(gl[i], gl[i + 1], __uint_as_float(v[i]), __uint_as_float(v[i + 1]), b.x, b.y);
-                add2(gl[i + 2], gl[i + 3], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]), b.z, b.w);
-            }
+            if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
+            TR(tr, 52);
+            const int n = (t_begin + ta) * kTileM + row;
+            if (n >= p.n_rows) continue;
             // one pass keeping the best two (strict comparisons in ascending id order: same picks as
-            // repeated arg-max with ties to the lower id)
-            float b1 = gl[0], b2 = -INFINITY;
+            // repeated arg-max with ties to the lower id); the logits stay in v as raw bits + bias
+            float b1 = -INFINITY, b2 = -INFINITY;
             int i1 = 0, i2 = 0;
 #pragma unroll
-            for (int i = 1; i < EP; ++i) {
-                const float g = gl[i];
-                const bool gt1 = g > b1, gt2 = g > b2;
-                b2 = gt1 ? b1 : (gt2 ? g : b2);
+            for (int i = 0; i < EP; ++i) {
+                const float gl = __uint_as_float(v[i]) + sh.bias2_f32[i];
+                v[i] = __float_as_uint(gl);
+                const bool gt1 = gl > b1, gt2 = gl > b2;
+                b2 = gt1 ? b1 : (gt2 ? gl : b2);
                 i2 = gt1 ? i1 : (gt2 ? i : i2);
-                b1 = gt1 ? g : b1;
+                b1 = gt1 ? gl : b1;
                 i1 = gt1 ? i : i1;
             }
             const float sc = p.softmax_scale;
             const float msc = b1 * sc;
             float sum = 0.0f;
 #pragma unroll
-            for (int i = 0; i < EP; ++i) sum += ex2_approx(fmaf(gl[i], sc, -msc));
+            for (int i = 0; i < EP; ++i) sum += ex2_approx(fmaf(__uint_as_float(v[i]), sc, -msc));
             const float inv = 1.0f / sum;
-            const int sel[2] = {i1, i2};
-            const float pj[2] = {inv, ex2_approx(fmaf(b2, sc, -msc)) * inv};
-            for (int j = 0; j < p.k; ++j) {
-                const size_t at = (size_t)n * p.k + j;
-                p.topk_idx[at] = sel[j];
-                p.topk_p[at] = pj[j];
-                p.local_rank[at] = atomicAdd(&sh.hist[sel[j]], 1);
+            const size_t at = (size_t)n * p.k;
+            p.topk_idx[at] = i1;
+            p.topk_p[at] = inv;
+            p.local_rank[at] = atomicAdd(&sh.hist[i1], 1);
+            if (p.k > 1) {
+                p.topk_idx[at + 1] = i2;
+                p.topk_p[at + 1] = ex2_approx(fmaf(b2, sc, -msc)) * inv;
+                p.local_rank[at + 1] = atomicAdd(&sh.hist[i2], 1);
             }
-        };
-        uint32_t q = 0;
-        TRD(tr, 20 + warp);
-        for (int i = 0; i < n_my && ok; ++i) {
-            for (int c = 0; c < nchunks && ok; ++c, ++q) {
-                if (pend && c == 1) {        // the previous tile's logits, one chunk late (see the expert pass)
-                    TR(tr, 50);
-                    output_tile();
-                    TR(tr, 51);
-                    if (!ok) break;
-                }
-                const uint32_t b = q % 3u, par = (q / 3u) & 1u;
-                TR(tr, 40);
-                ok = mbar_wait(pp_sbar(sh, s, B::ACC1_FULL + b), par, abort, kWaitLimitNs);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                TR(tr, 41);
-                tc_fence_after_sync();
-                const uint32_t acol = tcol + C::ACC1_COL + b * kPpHC + 32 * hh;
-                uint32_t acc[32];
-                tmem_ld_x32(acol, acc);
-                tmem_ld_wait();
-                TR(tr, 42);
-                const float* bias = sh.bias1_f32[0] + c * kPpHC + 32 * hh;
-#pragma unroll
-                for (int pc = 0; pc < 2; ++pc) {
-                    // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu),
-                    // lo = the rounded remainder (for a negative value the remainder is the value itself and
-                    // its .relu is 0 as well)
-                    float a[16];
-#pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        const float4 bb = *reinterpret_cast<const float4*>(bias + pc * 16 + i);
-                        add2(a[i], a[i + 1], __uint_as_float(acc[pc * 16 + i]), __uint_as_float(acc[pc * 16 + i + 1]), bb.x, bb.y);
-                        add2(a[i + 2], a[i + 3], __uint_as_float(acc[pc * 16 + i + 2]), __uint_as_float(acc[pc * 16 + i + 3]), bb.z, bb.w);
-                    }
-                    uint32_t hl[16];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) hl[i] = cvt_rz_relu_bf16x2(a[2 * i], a[2 * i + 1]);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        hl[8 + i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hl[i] << 16), a[2 * i + 1] - __uint_as_float(hl[i] & 0xFFFF0000u));
-                    tmem_st_x16(acol + pc * 16, hl);
-                }
-                TR(tr, 45);
-                tmem_st_wait();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(pp_sbar(sh, s, B::HID_FULL + b));
-                TR(tr, 46);
-            }
-            pend = (i & 1) == hh;
-            pend_ta = s + 2 * i;
-            pend_i = (uint32_t)i;
+            TR(tr, 53);
         }
-        if (ok && pend) output_tile();
     }
 
     // ---- teardown ---------------------------------------------------------------------------------

@@ -59,9 +59,10 @@ __device__ __forceinline__ bool pp_grid_barrier(int32_t* words, int32_t gen_befo
 
 template <int EP, int N2, int ACT>
 __global__ void __launch_bounds__(kPpThreads, 1)
-pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWr1,
-                  const __grid_constant__ CUtensorMap tmWr2, const __grid_constant__ CUtensorMap tmW1,
-                  const __grid_constant__ CUtensorMap tmW2, const PpFusedParams fp) {
+pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmXg,
+                  const __grid_constant__ CUtensorMap tmWr1, const __grid_constant__ CUtensorMap tmWr2,
+                  const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2,
+                  const PpFusedParams fp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ PpShared sh;
     const int warp = threadIdx.x >> 5;
@@ -84,7 +85,7 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                                            fp.kept, fp.offsets, fp.dest, fp.pair_gate, dsm, sh.offs);
     }
     ok = pp_grid_barrier(fp.sync_words, gen0 + 1, sh) && ok;
-    if (ok) pp_ffn_body<N2, ACT, true, true>(&tmW1, &tmW2, fp.ffn, sh, smem_raw);
+    if (ok) pp_ffn_body<N2, ACT, true, true>(&tmXg, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
     __syncthreads();
     if (warp == 1) {
@@ -124,7 +125,8 @@ pp_dispatch_kernel(const int32_t* topk_idx, const float* topk_p, const int32_t* 
 
 template <int N2, int ACT>
 __global__ void __launch_bounds__(kPpThreads, 1)
-pp_ffn_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2, const PpParams p) {
+pp_ffn_kernel(const __grid_constant__ CUtensorMap tmXg, const __grid_constant__ CUtensorMap tmW1,
+              const __grid_constant__ CUtensorMap tmW2, const PpParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ PpShared sh;
     const int warp = threadIdx.x >> 5;
@@ -132,7 +134,7 @@ pp_ffn_kernel(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ 
         tmem_alloc(smem_u32(&sh.tmem_base), 512);
         tmem_relinquish();
     }
-    pp_ffn_body<N2, ACT, false, false>(&tmW1, &tmW2, p, sh, smem_raw);
+    pp_ffn_body<N2, ACT, false, false>(&tmXg, &tmW1, &tmW2, p, sh, smem_raw);
     if (warp == 1) {
         __syncwarp();
         tmem_dealloc(sh.tmem_base, 512);
@@ -175,13 +177,14 @@ int pp_set_smem(K kern, int slot, int bytes) {
 }
 
 struct PpMaps {
-    CUtensorMap X, Wr1, Wr2, W1, W2;
+    CUtensorMap X, Xg, Wr1, Wr2, W1, W2;     // Xg: the rows of h with a one-row box (four-row gathers)
 };
 
 template <int EP, int N2>
 int pp_make_maps(const Dims& D, const slicemoe_weights& w, const void* h, PpMaps& m) {
     int rc;
     if ((rc = make_tmap(&m.X, h, (uint64_t)D.N, (uint64_t)D.ds, 128))) return rc;
+    if ((rc = make_tmap(&m.Xg, h, (uint64_t)D.N, (uint64_t)D.ds, 1))) return rc;
     if ((rc = make_tmap(&m.Wr1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, kPpHC))) return rc;
     if ((rc = make_tmap(&m.Wr2, w.Wr2, (uint64_t)D.E, (uint64_t)D.Hr, EP))) return rc;       // (E = 8: zero-filled up to 16)
     if ((rc = make_tmap(&m.W1, w.W1, (uint64_t)D.E * D.F, (uint64_t)D.ds, kPpHC))) return rc;
@@ -226,7 +229,7 @@ int pp_launch_fused(const Dims& D, const slicemoe_weights& w, const void* h, con
     attrs[0].val.cooperative = 1;
     lc.attrs = attrs;
     lc.numAttrs = 1;
-    SLICEMOE_CUDA_TRY(cudaLaunchKernelEx(&lc, kern, m.X, m.Wr1, m.Wr2, m.W1, m.W2, fp));
+    SLICEMOE_CUDA_TRY(cudaLaunchKernelEx(&lc, kern, m.X, m.Xg, m.Wr1, m.Wr2, m.W1, m.W2, fp));
     SLICEMOE_LAUNCH_CHECK(1);
     return SLICEMOE_OK;
 }
@@ -261,7 +264,7 @@ int pp_launch_staged(const Dims& D, const slicemoe_weights& w, const void* h, co
     SLICEMOE_LAUNCH_CHECK(1);
     if ((rc = mark(2))) return rc;
     const int ffn_grid = max_tiles(D) < sm_count() ? max_tiles(D) : sm_count();
-    kf<<<ffn_grid, kPpThreads, PpFfnCfg<N2>::SMEM_ALLOC, st>>>(m.W1, m.W2, fp.ffn);
+    kf<<<ffn_grid, kPpThreads, PpFfnCfg<N2>::SMEM_ALLOC, st>>>(m.Xg, m.W1, m.W2, fp.ffn);
     SLICEMOE_LAUNCH_CHECK(1);
     if ((rc = mark(3))) return rc;
     return mark(4);
@@ -296,7 +299,7 @@ extern "C" int slicemoe_debug_pp_flags(int flags) {
     return cudaDeviceSynchronize() == cudaSuccess ? 0 : 7;
 }
 extern "C" int slicemoe_debug_pp_trace(int on, void* host_out) {
-    if (host_out) cudaMemcpyFromSymbol(host_out, g_pp_trace, sizeof(unsigned long long) * 40 * 4096);
+    if (host_out) cudaMemcpyFromSymbol(host_out, g_pp_trace, sizeof(unsigned long long) * 64 * 4096);
     cudaMemcpyToSymbol(g_pp_trace_on, &on, sizeof(int));
     return cudaDeviceSynchronize() == cudaSuccess ? 0 : 7;
 }
@@ -315,7 +318,7 @@ bool pp_forward_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16 || D.ds != 64 || D.N <= 0) return false;
     if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
     if (D.k > 2 || D.capacity != 0 || D.noise_sigma > 0.0f) return false;
-    if (D.Hr % kPpHC || D.Hr < 2 * kPpHC || D.Hr > kPpMaxHr) return false;
+    if (D.Hr % 128 || D.Hr < 128 || D.Hr > kPpMaxHr) return false;      // (the router takes its hidden layer in halves of 128)
     if (D.F % kPpHC || D.F < 2 * kPpHC || D.F > kPpMaxF) return false;
     return pp_cooperative_launch_available();
 }

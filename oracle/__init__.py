@@ -112,6 +112,20 @@ def _check(rc, what):
         raise RuntimeError(f"{what} failed with oracle status {rc}")
 
 
+def _router_weights(cfg: OracleConfig, w: dict):
+    """The router's tensors alone, widened to float64 (the route call reads nothing else)."""
+    return dict(
+        Wr1=_f64(w["Wr1"], (cfg.Hr, cfg.ds)), br1=_f64(w.get("br1"), (cfg.Hr,)),
+        Wr2=_f64(w["Wr2"], (cfg.E, cfg.Hr)), br2=_f64(w.get("br2"), (cfg.E,)))
+
+
+def _expert_weights(cfg: OracleConfig, w: dict):
+    """The experts' tensors alone, widened to float64 (the expert_ffn call reads nothing else)."""
+    return dict(
+        W1=_f64(w["W1"], (cfg.E, cfg.F, cfg.ds)), b1=_f64(w.get("b1"), (cfg.E, cfg.F)),
+        W2=_f64(w["W2"], (cfg.E, cfg.ds, cfg.F)), b2=_f64(w.get("b2"), (cfg.E, cfg.ds)))
+
+
 def _weights(cfg: OracleConfig, w: dict):
     ds = cfg.ds
     return dict(
@@ -126,7 +140,7 @@ def route(cfg: OracleConfig, h, w: dict) -> dict:
     the gap p_(k) - p_(k+1) and the per-expert assigned counts."""
     lib, c = _load(), cfg.c()
     h = _f64(h, (cfg.T, cfg.d))
-    ww = _weights(cfg, w)
+    ww = _router_weights(cfg, w)
     probs = np.empty((cfg.N, cfg.E), np.float64)
     idx = np.empty((cfg.N, cfg.k), np.int32)
     pk = np.empty((cfg.N, cfg.k), np.float64)
@@ -171,7 +185,7 @@ def expert_ffn(cfg: OracleConfig, xperm, offsets, w: dict):
     offsets = np.ascontiguousarray(offsets, dtype=np.int64)
     n_kept = int(offsets[-1])
     xperm = _f64(xperm, (n_kept, cfg.ds))
-    ww = _weights(cfg, w)
+    ww = _expert_weights(cfg, w)
     yperm = np.zeros((max(n_kept, 1), cfg.ds), np.float64)
     _check(lib.slicemoe_oracle_expert_ffn(ctypes.byref(c), _p(xperm), _p(offsets), _p(ww["W1"]),
                                           _p(ww["b1"]), _p(ww["W2"]), _p(ww["b2"]), _p(yperm)),

@@ -58,7 +58,9 @@ int make_dims(const slicemoe_config* c, Dims& D) {
     const long long N = (long long)c->T * c->S, R = N * c->k;
     const long long lim = 0x7fffffffLL;
     if (R >= lim || (long long)c->T * c->d >= lim) return SLICEMOE_ERR_SHAPE;
-    if ((long long)c->E * c->F * (c->d / c->S) >= lim) return SLICEMOE_ERR_SHAPE;
+    // (row and pair counts are 32-bit; the weight tensors are indexed with 64-bit element offsets, so a
+    // token-level layer with E F d past 2^31 elements per tensor is fine; a tensor map's row count E F is not)
+    if ((long long)c->E * c->F >= lim) return SLICEMOE_ERR_SHAPE;
     const int V = c->dtype == SLICEMOE_BF16 ? 8 : 4;
     const int ds = c->d / c->S;
     if (ds % V || c->Hr % V || c->F % V) return SLICEMOE_ERR_UNSUPPORTED;
@@ -344,11 +346,7 @@ int slicemoe_forward_profiled(const slicemoe_config* cfg, const slicemoe_weights
 namespace slicemoe {
 namespace {
 
-#ifdef SLICEMOE_DEV_HOST_CHUNKS
-constexpr int kPipeChunks = 16;
-#else
 constexpr int kPipeChunks = 4;
-#endif
 constexpr int kPipeMinTokensPerChunk = 512;
 constexpr double kPipeEdgeShare = 0.5;        // first / last chunk relative to an inner chunk
 constexpr int kPipeMaxDevices = 64;
@@ -410,7 +408,9 @@ int slicemoe_forward_host(const slicemoe_config* cfg, const slicemoe_weights* w,
     char* h_dev = at<char>(ws, W.h_dev);
     char* hout_dev = at<char>(ws, W.hout_dev);
 
-    const bool pipelined = D.capacity == 0 && D.T >= kPipeChunks * kPipeMinTokensPerChunk;
+    // (not with logit noise either: its draws are keyed by the row's index in the whole batch, and a chunk's
+    // router counts rows from the chunk's start)
+    const bool pipelined = D.capacity == 0 && D.noise_sigma == 0.0f && D.T >= kPipeChunks * kPipeMinTokensPerChunk;
     if (!pipelined) {
         if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_dev, h_host, bytes, cudaMemcpyHostToDevice, st));
         if ((rc = forward_impl(D, *w, h_dev, hout_dev, assigned_opt, kept_opt, nullptr, nullptr, ws, W, st,
@@ -435,13 +435,7 @@ int slicemoe_forward_host(const slicemoe_config* cfg, const slicemoe_weights* w,
     // copy in or the last copy out.
     int bounds[kPipeChunks + 1];
     int nchunks_host = kPipeChunks;
-#ifdef SLICEMOE_DEV_HOST_CHUNKS
-    if (const char* ev = getenv("SLICEMOE_HOST_CHUNKS")) nchunks_host = atoi(ev) > 0 && atoi(ev) <= kPipeChunks ? atoi(ev) : kPipeChunks;
-    double edge = 0.5;
-    if (const char* ev = getenv("SLICEMOE_HOST_EDGE")) edge = atof(ev);
-#else
     const double edge = kPipeEdgeShare;
-#endif
     {
         // edge chunks get `edge` times the share of an inner chunk
         const double inner = 1.0 / (nchunks_host - 2 + 2 * edge);

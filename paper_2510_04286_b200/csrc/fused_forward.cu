@@ -80,27 +80,11 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     __shared__ TcShared sh;
     const int warp = threadIdx.x >> 5;
-#ifdef SLICEMOE_FUSED_STAMPS   // development: phase boundaries of CTA 0 and of the last CTA, in ns
-#define STAMP(i)                                                                                          \
-    do {                                                                                                  \
-        if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))                         \
-            reinterpret_cast<unsigned long long*>(fp.ffn.status + 64)[(blockIdx.x ? 8 : 0) + (i)] = globaltimer_ns(); \
-    } while (0)
-#else
-#define STAMP(i)
-#endif
-    STAMP(0);
     int32_t gen0 = 0;
     if (threadIdx.x == 0) {
         gen0 = *reinterpret_cast<volatile int32_t*>(fp.sync_words + 1);   // no barrier can complete without this CTA
         if (blockIdx.x == 0 && fp.clear_status) *fp.ffn.status = SLICEMOE_OK;              // run-outs (>= seconds later) overwrite it
     }
-#ifdef SLICEMOE_FUSED_STAMPS
-    // per-launch ring (slot = launch number mod 32): earliest CTA entry and latest CTA exit
-    unsigned long long* ring = reinterpret_cast<unsigned long long*>(fp.ffn.status + 128);
-    const int slot = fp.ffn.status[100] & 31;
-    if (threadIdx.x == 0) atomicMin(ring + 2 * slot, (unsigned long long)globaltimer_ns());
-#endif
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh.tmem_base), TMEM_COLS);
         tmem_relinquish();
@@ -109,9 +93,7 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     // ---- phase 1: router -----------------------------------------------------------------------
     tc_body<RC, false, false, true>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
     bool ok = sh.abort_flag == 0;
-    STAMP(1);
     ok = grid_barrier(fp.sync_words, gen0, sh) && ok;
-    STAMP(2);
 
     // ---- phase 2: dispatch of this CTA's own pairs -----------------------------------------------
     if (ok) {
@@ -120,30 +102,13 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                                (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.capacity,
                                                fp.assigned, fp.kept, fp.offsets, fp.dest, fp.perm, fp.gate, dsm, sh.offs);
     }
-    STAMP(3);
     ok = grid_barrier(fp.sync_words, gen0 + 1, sh) && ok;
-    STAMP(4);
 
     // ---- phase 3: experts ------------------------------------------------------------------------
     if (ok) tc_body<EC, true, true, true>(&tmX, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
 
     __syncthreads();
-    STAMP(5);
-#ifdef SLICEMOE_FUSED_STAMPS
-    if (threadIdx.x == 0) {
-        atomicMax(ring + 2 * slot + 1, (unsigned long long)globaltimer_ns());
-        __threadfence();
-        if (atomicAdd(fp.ffn.status + 101, 1) == (int)gridDim.x - 1) {   // last CTA out: next launch's slot
-            fp.ffn.status[101] = 0;
-            const int next = (slot + 1) & 31;
-            ring[2 * next] = ~0ull;
-            ring[2 * next + 1] = 0ull;
-            __threadfence();
-            fp.ffn.status[100] = next;
-        }
-    }
-#endif
     if (warp == 1) {
         __syncwarp();
         tmem_dealloc(sh.tmem_base, TMEM_COLS);
@@ -166,11 +131,8 @@ int launch_fused(const Dims& D, const slicemoe_weights& w, const void* h, const 
     if (dsm > smem) smem = dsm;
     if (smem + sizeof(TcShared) + 64 > 227 * 1024) return SLICEMOE_ERR_UNSUPPORTED;
     auto kern = fused_forward_kernel<RC, EC>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(227 * 1024 - sizeof(TcShared) - 64)));
-        attr_set = true;
-    }
+    static bool attr_set[kAttrMaxDevices] = {};
+    if ((rc = set_smem_limit_once(kern, (int)(227 * 1024 - sizeof(TcShared) - 64), attr_set))) return rc;
     // One CTA per SM, all resident at once: a cooperative launch states that requirement.
     // (Programmatic dependent launch on top of it was measured and bought nothing: the next grid's
     // CTAs cannot become resident before this grid's CTAs leave their SMs.)
@@ -252,9 +214,6 @@ int fused_forward_reset_sync(cudaStream_t st) {
 }
 
 bool fused_forward_supported(const Dims& D) {
-#ifdef SLICEMOE_TC_TRACE   // the timeline tracer needs its own shared-memory area: one launch per stage only
-    return false;
-#endif
     return tc_route_supported(D) && tc_ffn_supported(D) && D.N > 0 && D.k <= 2 && cooperative_launch_available();
 }
 

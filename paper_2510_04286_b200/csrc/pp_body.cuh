@@ -1013,7 +1013,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
 // output does not depend on it (each stacked row is computed on its own, and the sum of at most two bf16
 // values commutes), but `perm` / `dest` do, so this form is used only where they are not outputs and
 // nothing is dropped (capacity limits need the stable order of the other dispatch).
-// offs_out: shared memory, E + 1 ints.  `sm`: at least (2 E + 1) ints of shared memory.
+// offs_out: shared memory, E + 1 ints.  `sm`: at least (2 E + 1 + G E) ints of shared memory.
 // =====================================================================================================
 template <int NT, bool SAME_LAUNCH>
 __device__ __forceinline__ void pp_dispatch_body(const int32_t* topk_idx, const float* topk_p, const int32_t* local_rank,
@@ -1022,12 +1022,33 @@ __device__ __forceinline__ void pp_dispatch_body(const int32_t* topk_idx, const 
                                                  int2* pair_gate, int* sm, int* offs_out) {
     int* base = sm;            // [E] pairs of expert e in earlier CTAs, then + offsets
     int* total = sm + E;       // [E]
+    int* tab = sm + 2 * E + 1; // [G * E] copy of the table
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long begin = (long long)chunk * pairs_per_chunk;
+    long long end = begin + pairs_per_chunk;
+    if (end > R) end = R;
+    // Everything this CTA needs from global memory is requested up front, so that it pays the latency once:
+    // the table (coalesced) and the first kPre of its own pairs per thread.
+    constexpr int kPre = 4;
+    int pe[kPre], pr[kPre];
+    float pp[kPre];
+#pragma unroll
+    for (int q = 0; q < kPre; ++q) {
+        const long long i = begin + threadIdx.x + (long long)q * NT;
+        pe[q] = -1;
+        if (i < end) {
+            pe[q] = SAME_LAUNCH ? __ldcg(topk_idx + i) : topk_idx[i];
+            pr[q] = SAME_LAUNCH ? __ldcg(local_rank + i) : local_rank[i];
+            pp[q] = SAME_LAUNCH ? __ldcg(topk_p + i) : topk_p[i];
+        }
+    }
+    for (int i = threadIdx.x; i < G * E; i += NT) tab[i] = SAME_LAUNCH ? __ldcg(table + i) : table[i];
+    __syncthreads();
     // warp w sums experts w, w + NT/32, ...: lanes stride over the CTAs of the table
     for (int e = warp; e < E; e += NT / 32) {
         int before = 0, tot = 0;
         for (int c = lane; c < G; c += 32) {
-            const int v = SAME_LAUNCH ? __ldcg(table + (size_t)c * E + e) : table[(size_t)c * E + e];
+            const int v = tab[c * E + e];
             tot += v;
             if (c < chunk) before += v;
         }
@@ -1068,16 +1089,22 @@ __device__ __forceinline__ void pp_dispatch_body(const int32_t* topk_idx, const 
         }
     }
     __syncthreads();
-    const long long begin = (long long)chunk * pairs_per_chunk;
-    long long end = begin + pairs_per_chunk;
-    if (end > R) end = R;
-    for (long long i = begin + threadIdx.x; i < end; i += NT) {
+#pragma unroll
+    for (int q = 0; q < kPre; ++q) {
+        if (pe[q] >= 0) {
+            const long long i = begin + threadIdx.x + (long long)q * NT;
+            const int d = base[pe[q]] + pr[q];
+            dest[i] = d;
+            pair_gate[d] = make_int2((int)i, __float_as_int(pp[q]));
+        }
+    }
+    for (long long i = begin + threadIdx.x + (long long)kPre * NT; i < end; i += NT) {
         const int e = SAME_LAUNCH ? __ldcg(topk_idx + i) : topk_idx[i];
         const int r = SAME_LAUNCH ? __ldcg(local_rank + i) : local_rank[i];
-        const float pr = SAME_LAUNCH ? __ldcg(topk_p + i) : topk_p[i];
+        const float pr2 = SAME_LAUNCH ? __ldcg(topk_p + i) : topk_p[i];
         const int d = base[e] + r;
         dest[i] = d;
-        pair_gate[d] = make_int2((int)i, __float_as_int(pr));
+        pair_gate[d] = make_int2((int)i, __float_as_int(pr2));
     }
 }
 

@@ -67,6 +67,14 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     __shared__ PpShared sh;
     const int warp = threadIdx.x >> 5;
     int32_t gen0 = 0;
+#ifdef PP_TRACE
+    PpTr ph(63);
+    ph.on = ph.on && threadIdx.x == 0;
+#define PH(c) ph(c)
+#else
+#define PH(c)
+#endif
+    PH(1);
     if (threadIdx.x == 0) {
         gen0 = *reinterpret_cast<volatile int32_t*>(fp.sync_words + 1);   // no barrier can complete without this CTA
         if (blockIdx.x == 0 && fp.clear_status) *fp.ffn.status = SLICEMOE_OK;
@@ -76,16 +84,21 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         tmem_relinquish();
     }
     pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
+    PH(2);
     bool ok = sh.abort_flag == 0;
     ok = pp_grid_barrier(fp.sync_words, gen0, sh) && ok;
+    PH(3);
     if (ok) {
         int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
         pp_dispatch_body<kPpThreads, true>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, fp.route.cta_hist,
                                            (int)gridDim.x, (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.assigned,
                                            fp.kept, fp.offsets, fp.dest, fp.pair_gate, dsm, sh.offs);
     }
+    PH(4);
     ok = pp_grid_barrier(fp.sync_words, gen0 + 1, sh) && ok;
+    PH(5);
     if (ok) pp_ffn_body<N2, ACT, true, true>(&tmXg, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
+    PH(6);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
     __syncthreads();
     if (warp == 1) {
@@ -117,7 +130,7 @@ __global__ void __launch_bounds__(kPpThreads, 1)
 pp_dispatch_kernel(const int32_t* topk_idx, const float* topk_p, const int32_t* local_rank, const int32_t* table, int R,
                    int E, int pairs_per_chunk, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
                    int2* pair_gate) {
-    __shared__ int sm[2 * kMaxE + 1];
+    extern __shared__ int sm[];          // (2 E + 1 + G E) ints
     __shared__ int offs[kMaxE + 1];
     pp_dispatch_body<kPpThreads, false>(topk_idx, topk_p, local_rank, table, (int)gridDim.x, (int)blockIdx.x, R, E,
                                         pairs_per_chunk, assigned, kept, offsets, dest, pair_gate, sm, offs);
@@ -258,7 +271,7 @@ int pp_launch_staged(const Dims& D, const slicemoe_weights& w, const void* h, co
     kr<<<grid, kPpThreads, smem_r, st>>>(m.X, m.Wr1, m.Wr2, fp.route);
     SLICEMOE_LAUNCH_CHECK(1);
     if ((rc = mark(1))) return rc;
-    pp_dispatch_kernel<<<grid, kPpThreads, 0, st>>>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank,
+    pp_dispatch_kernel<<<grid, kPpThreads, sizeof(int) * (2 * D.E + 1 + (size_t)grid * D.E), st>>>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank,
                                                     fp.route.cta_hist, fp.R, fp.E, rows_per_cta * D.k, fp.assigned, fp.kept,
                                                     fp.offsets, fp.dest, fp.pair_gate);
     SLICEMOE_LAUNCH_CHECK(1);
@@ -319,7 +332,7 @@ bool pp_forward_supported(const Dims& D) {
     if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
     if (D.k > 2 || D.capacity != 0 || D.noise_sigma > 0.0f) return false;
     if (D.Hr % 128 || D.Hr < 128 || D.Hr > kPpMaxHr) return false;      // (the router takes its hidden layer in halves of 128)
-    if (D.F % kPpHC || D.F < 2 * kPpHC || D.F > kPpMaxF) return false;
+    if (D.F != 128 && D.F != kPpMaxF) return false;                    // (the activation takes the hidden layer in turns of 64 or 128 columns per warpgroup)
     return pp_cooperative_launch_available();
 }
 

@@ -34,11 +34,8 @@ int launch_tc(const void* A, uint64_t a_rows, const void* W1, const void* W2, in
     // (router: the real expert count; a box taller than the tensor is zero-filled below its edge)
     if ((rc = make_tmap(&tmW2, W2, C::ROUTER ? (uint64_t)p.experts_real : (uint64_t)n_experts * C::N2, p.HID, C::N2))) return rc;
     auto kern = tc_mlp_kernel<C>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLaunch<C>));
-        attr_set = true;
-    }
+    static bool attr_set[kAttrMaxDevices] = {};
+    if ((rc = set_smem_limit_once(kern, kSmemLaunch<C>, attr_set))) return rc;
     const int grid = max_tiles < sm_count() ? max_tiles : sm_count();
     kern<<<grid, C::THREADS, kSmemLaunch<C>, st>>>(tmA, tmW1, tmW2, p);
     SLICEMOE_LAUNCH_CHECK(1);
@@ -70,14 +67,6 @@ int launch_route_k1(const Dims& D, const slicemoe_weights& w, const void* h, con
 
 }  // namespace
 
-#ifdef SLICEMOE_TC_TRACE
-// Development hook: where CTA 0 of the next tensor-core launches writes its timeline
-// (kTraceSlots * kTraceEvents * 2 uint64 values; NULL switches tracing off).
-extern "C" int slicemoe_debug_set_trace(void* device_buf) {
-    unsigned long long* ptr = static_cast<unsigned long long*>(device_buf);
-    return cudaMemcpyToSymbol(g_trace_buf, &ptr, sizeof(ptr)) == cudaSuccess ? 0 : SLICEMOE_ERR_CUDA;
-}
-#endif
 
 // Slice widths the tensor-core pipeline is built for.  The paper's own model (d = 768, S = 8) has
 // ds = 96: it runs on the 128-wide instantiation, the copies zero-filling columns 96..127 of the row

@@ -89,38 +89,6 @@ struct TcParams {
     int32_t* status;
 };
 
-// Optional timeline tracing (development builds only: -DSLICEMOE_TC_TRACE).  CTA 0 stamps
-// (event code, SM clock) pairs per role into a caller-provided buffer.
-#ifdef SLICEMOE_TC_TRACE
-#ifndef SLICEMOE_TRACE_EVENTS
-#define SLICEMOE_TRACE_EVENTS 320          // per role, in shared memory
-#endif
-#ifndef SLICEMOE_TRACE_OFFSET_KB
-#define SLICEMOE_TRACE_OFFSET_KB 200       // where the trace area starts; must lie past the operand tiles
-#endif
-constexpr int kTraceSlots = 8, kTraceEvents = 2048, kTraceSmemEvents = SLICEMOE_TRACE_EVENTS;
-constexpr int kTraceOffset = SLICEMOE_TRACE_OFFSET_KB * 1024;
-__device__ unsigned long long* g_trace_buf = nullptr;
-// Events go to shared memory (cheap) and are copied out at the end of the kernel.
-struct Tracer {
-    uint2* base;
-    int n;
-    __device__ Tracer(int slot) : base(nullptr), n(0) {
-        extern __shared__ uint8_t smem_raw[];
-        if (blockIdx.x == 0 && g_trace_buf && slot < 6)
-            base = reinterpret_cast<uint2*>(smem_raw + kTraceOffset) + slot * kTraceSmemEvents;
-    }
-    __device__ void operator()(int code) {
-        if (base && n < kTraceSmemEvents) { base[n] = make_uint2((unsigned)code, (unsigned)clock64()); ++n; }
-    }
-};
-#define TRACE_DECL(name, slot) Tracer name(slot)
-#define TRACE(name, code) name(code)
-#else
-#define TRACE_DECL(name, slot)
-#define TRACE(name, code)
-#endif
-
 constexpr int pow2_at_least(int x) {
     int p = 32;
     while (p < x) p <<= 1;
@@ -317,9 +285,6 @@ __device__ __forceinline__ void convert_piece_bf16x2(const uint32_t* cur, __nv_b
 template <int ACT>
 __device__ __forceinline__ void activate_pre_bf16x2(const __nv_bfloat162* z, __nv_bfloat162* t) {
     constexpr int P = 8;   // column pairs per piece
-#ifdef SLICEMOE_TC_SKELETON   // development: time the pipeline without the activation math
-    return;
-#endif
     if (ACT == SLICEMOE_ACT_RELU) return;
     const __nv_bfloat162 c0 = __float2bfloat162_rn(0.7978845608f), c1 = __float2bfloat162_rn(0.0356774081f);
 #pragma unroll
@@ -334,11 +299,7 @@ __device__ __forceinline__ void activate_pre_bf16x2(const __nv_bfloat162* z, __n
 template <int ACT>
 __device__ __forceinline__ void activate_post_bf16x2(const __nv_bfloat162* z, const __nv_bfloat162* t, uint32_t* out) {
     constexpr int P = 8;
-#ifdef SLICEMOE_TC_SKELETON
-    constexpr bool relu = true;
-#else
     constexpr bool relu = ACT == SLICEMOE_ACT_RELU;
-#endif
     if constexpr (relu) {
         const __nv_bfloat162 zero = __float2bfloat162_rn(0.0f);
 #pragma unroll
@@ -357,11 +318,7 @@ __device__ __forceinline__ void activate_post_bf16x2(const __nv_bfloat162* z, co
 // factor the output epilogue applies to the GEMM-2 accumulator (see above)
 template <int ACT>
 constexpr float kOutScale =
-#ifdef SLICEMOE_TC_SKELETON
-    1.0f;
-#else
     (ACT == SLICEMOE_ACT_RELU) ? 1.0f : 0.5f;
-#endif
 
 // Router: relu(acc + bias) as a bf16 pair per value: hi = the value truncated to bf16, lo = the
 // rounded remainder; hi + lo carries 16 mantissa bits of the fp32 value.  The ReLU rides on the two
@@ -448,15 +405,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     const bool gather = !C::ROUTER && (FUSED || p.gather_src != nullptr);
     auto bar = [&](int i) { return smem_u32(&sh.bars[i]); };
 
-#ifdef SLICEMOE_TC_TRACE
-    for (int i = threadIdx.x; i < 6 * kTraceSmemEvents * 2; i += C::THREADS)
-        reinterpret_cast<uint32_t*>(smem_raw + kTraceOffset)[i] = 0;
-#endif
     // ---- set-up ---------------------------------------------------------------------------
     if (threadIdx.x == 0) {
-#ifdef SLICEMOE_TC_TRACE
-        { TRACE_DECL(tr0, 5); TRACE(tr0, 99); }
-#endif
         sh.abort_flag = 0;
         for (int i = 0; i < C::A_BUFS; ++i) { mbar_init(bar(B::A_FULL + i), gather ? 32 * C::GATHER_WARPS : 1); mbar_init(bar(B::A_EMPTY + i), 1); }
         for (int i = 0; i < C::W_STAGES; ++i) {
@@ -525,9 +475,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     const int t_end = min(total_tiles, t_begin + per_cta);
 
     const uint32_t sA = smem_base + C::OFF_A, sW = smem_base + C::OFF_W;
-#ifdef SLICEMOE_TC_TRACE
-    if (threadIdx.x == 0) { Tracer tr1(5); tr1.n = 1; tr1(98); }   // set-up finished
-#endif
 
     // result of a wait in an MMA-issuing warp: with all lanes in the loop they must leave it together
     auto all_lanes_agree = [](bool r) { return C::UNIFORM_ISSUE ? (bool)__all_sync(0xffffffffu, r) : r; };
@@ -545,16 +492,13 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             uint32_t wq = 0;                         // W1 chunk loads issued (bias ring position)
             uint32_t last_bar[3] = {0, 0, 0}, last_par[3] = {0, 0, 0};
             bool ok = true;
-            TRACE_DECL(tr, 0);
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
                 int row0, rows;
                 locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
                 const int ab = ta % C::A_BUFS;
                 const uint32_t an = ta / C::A_BUFS;
                 if (!gather) {
-                    TRACE(tr, 1);
                     if (!mbar_wait(bar(B::A_EMPTY + ab), (an & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
-                    TRACE(tr, 2);
                     mbar_arrive_expect_tx(bar(B::A_FULL + ab), C::A_BYTES);
 #pragma unroll
                     for (int kp = 0; kp < C::KP1; ++kp)
@@ -609,7 +553,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             constexpr uint32_t idesc1 = make_idesc(128, C::HC, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
             bool ok = true;
-            TRACE_DECL(tr, lane == 0 ? 1 : 7);
             int e = 0, prev_e = -1;
             uint32_t g = 0, reloads = 0;
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
@@ -618,10 +561,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 const bool reload = !resident || (e != prev_e);
                 prev_e = e;
                 const int ab = ta % C::A_BUFS;
-                TRACE(tr, 10);
                 ok = all_lanes_agree(mbar_wait(bar(B::A_FULL + ab), (uint32_t)(ta / C::A_BUFS) & 1u, abort, kWaitLimitNs));
                 if (!ok) break;
-                TRACE(tr, 11);
                 if (gather) fence_proxy_async_smem();   // rows written by cp.async -> visible to the MMA's reads
                 for (int c = 0; c < nchunks; ++c, ++g) {
                     const int slot = resident ? c : (int)(g % C::W_STAGES);
@@ -631,10 +572,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         if (!ok) break;
                     }
                     const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
-                    TRACE(tr, 12);
                     ok = all_lanes_agree(mbar_wait(bar(B::ACC1_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs));
                     if (!ok) break;
-                    TRACE(tr, 13);
                     tc_fence_after_sync();
                     const uint32_t a0 = dA + ((ab * C::A_BYTES) >> 4), w0 = dW + ((slot * C::W1C_BYTES) >> 4);
                     const uint32_t d = tmem_base + b * C::HC;
@@ -651,7 +590,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         if (c == nchunks - 1) mma_commit(bar(B::A_EMPTY + ab));
                     }
                     if (C::UNIFORM_ISSUE) __syncwarp();
-                    TRACE(tr, 14);
                 }
                 if (reload) ++reloads;
             }
@@ -671,7 +609,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             constexpr uint32_t idesc2 = make_idesc(128, C::N2, kFmtBF16, kFmtBF16);
             const uint32_t dW = desc_lo_sw128(smem_base + C::OFF_W2);
             bool ok = true;
-            TRACE_DECL(tr, lane == 0 ? 4 : 7);
             int e = 0, prev_e = -1;
             uint32_t g = 0, reloads = 0;
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
@@ -695,10 +632,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         if (!ok) break;
                     }
                     const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
-                    TRACE(tr, 20);
                     ok = all_lanes_agree(mbar_wait(bar(B::H_FULL + b), n1 & 1u, abort, kWaitLimitNs));
                     if (!ok) break;
-                    TRACE(tr, 21);
                     if (c == 0) {
                         ok = all_lanes_agree(mbar_wait(bar(B::ACC2_EMPTY + buf), ((uint32_t)(ta / C::ACC2_BUFS) & 1u) ^ 1u,
                                                                abort, kWaitLimitNs));
@@ -732,7 +667,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         if (c == nchunks - 1) mma_commit(bar(B::ACC2_FULL + buf));
                     }
                     if (C::UNIFORM_ISSUE) __syncwarp();
-                    TRACE(tr, 22);
                 }
                 if (reload) ++reloads;
             }
@@ -778,10 +712,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             // The first turn (t = t_begin - 1) only fetches the first tile's pair indices; a tile's indices
             // are fetched one tile ahead and left untouched until then, so that the load's latency is not
             // waited for.
-            TRACE_DECL(tr, (lane == 0 && warp == 3) ? 0 : 7);
 #pragma unroll 1
             for (int t = t_begin - 1, ta = -1; t < t_end && ok; ++t, ++ta) {
-                TRACE(tr, 1);
 #pragma unroll
                 for (int q = 0; q < QPW; ++q) nrow[q] = nnext[q] < 0 ? -1 : pair_to_row(nnext[q], p.gather_magic, p.gather_shift);
                 if (t + 1 < t_end) {
@@ -794,12 +726,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     }
                 }
                 if (ta < 0) continue;
-                TRACE(tr, 5);
                 const int ab = ta % C::A_BUFS;
                 ok = mbar_wait(bar(B::A_EMPTY + ab), ((uint32_t)(ta / C::A_BUFS) & 1u) ^ 1u, abort, kWaitLimitNs);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                TRACE(tr, 2);
                 const uint32_t dst0 = sA + ab * C::A_BYTES + (ch >> 3) * C::A_PANEL;
                 const bool in_row = ch * 8 < p.row_elems;       // chunks past the row's real width are zero-filled
                 auto copy_block = [&](int q, int nrow_q) {       // 32 rows of the tile
@@ -842,7 +772,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     }
                 }
                 cp_async_mbar_arrive_noinc(bar(B::A_FULL + ab));
-                TRACE(tr, 3);
             }
             cp_async_wait_all();
         }
@@ -856,7 +785,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         bool ok = true;
         int e = 0;
         uint32_t g = 0;
-        TRACE_DECL(tr, (lg == 0 && lane == 0 && w == 0 && grp < 2) ? 2 + grp : 7);
         int prev_e = -1;
         uint32_t q_tile = 0, q_next = 0;              // bias ring: W1 load count of this tile's chunk 0 / after it
         for (int t = t_begin; t < t_end && ok; ++t) {
@@ -867,7 +795,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 q_next += nchunks;
             }
             prev_e = e;
-            TRACE(tr, 36);
             float gs = 1.0f;                          // Eq. 1's gate of this thread's row (fused forward; the
                                                       // staged call's rows arrive weighted), read per chunk
             for (int c = 0; c < nchunks && ok; ++c, ++g) {
@@ -875,13 +802,11 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 const uint32_t b = g % C::NBUF, n1 = g / C::NBUF;
                 const uint32_t acc1 = lane_base + b * C::HC + w * WCOLS;               // my accumulator columns
                 const uint32_t hdst = lane_base + C::H_COL0 + b * (C::HC / 2) + w * (WCOLS / 2);
-                TRACE(tr, 30);
                 ok = mbar_wait(bar(B::ACC1_FULL + b), n1 & 1u, abort, kWaitLimitNs);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 // (the tile's A rows, and with them its ring entry, landed before GEMM-1 could run)
                 if (gather) gs = sh.gate_s[(t - t_begin) % kMetaRing][lg * 32 + lane];
-                TRACE(tr, 31);
                 tc_fence_after_sync();
                 // this chunk's bias came into shared memory with its W1 (same barrier, own ring)
                 const int bslot = (int)((q_tile + c) % kBiasRing);
@@ -907,7 +832,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                             convert_piece_bf16x2(v[i], gate_hi, gate_lo, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
                                                  true, z[s0 + i]);
                     }
-                    TRACE(tr, 32);
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(B::ACC1_EMPTY + b));
@@ -916,12 +840,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     for (int pc = 0; pc <= C::NPIECE; ++pc) {
                         if (pc < C::NPIECE) activate_pre_bf16x2<C::ACT>(z[pc], th[pc & 1]);
                         if (pc == 0) {
-                            TRACE(tr, 33);
                             // GEMM-2 of two chunks ago must be done with this hidden buffer
                             ok = mbar_wait(bar(B::H_EMPTY + b), (n1 & 1u) ^ 1u, abort, kWaitLimitNs);
                             ok = __all_sync(0xffffffffu, ok);
                             if (!ok) break;
-                            TRACE(tr, 34);
                         } else {
                             uint32_t hi[C::PIECE / 2];
                             activate_post_bf16x2<C::ACT>(z[pc - 1], th[(pc - 1) & 1], hi);
@@ -944,11 +866,9 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 }
                 if (!ok) break;
                 tmem_st_wait();
-                TRACE(tr, 37);
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B::H_FULL + b));
-                TRACE(tr, 35);
             }
         }
     } else if (warp >= C::OUT_WARP0 && warp < C::OUT_WARP0 + 4) {
@@ -958,18 +878,15 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         const uint32_t tmem_lane = tmem_base + ((uint32_t)(lg * 32) << 16);
         bool ok = true;
         int e = 0;
-        TRACE_DECL(tr, (lg == 0 && lane == 0) ? 5 : 7);
         // Fused forward: this thread's row of a tile is pair perm[row0 + row] = (n, j); its output is
         // added into row n of Y.
         for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
             int row0, rows;
             locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
             const int buf = ta % C::ACC2_BUFS;
-            TRACE(tr, 40);
             ok = mbar_wait(bar(B::ACC2_FULL + buf), (uint32_t)(ta / C::ACC2_BUFS) & 1u, abort, kWaitLimitNs);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            TRACE(tr, 41);
             tc_fence_after_sync();
             const int pair_cur = gather ? sh.pair_s[ta % kMetaRing][row] : 0;
             const uint32_t acc2 = tmem_lane + C::ACC2_COL0 + buf * C::N2;
@@ -982,7 +899,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
-                TRACE(tr, 42);
                 if (row >= rows) continue;
                 float gl[E];
 #pragma unroll
@@ -1073,11 +989,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar(B::ACC2_EMPTY + buf));
-                        TRACE(tr, 42);
                     }
-#ifdef SLICEMOE_DEV_NO_OUT    // development: time the pipeline without the output stores
-                    if (true) continue;
-#endif
                     if (!live) continue;
 #pragma unroll
                     for (int q = 0; q < OB / 8; ++q) {
@@ -1097,7 +1009,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         else *reinterpret_cast<uint4*>(dst + cb + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
-                TRACE(tr, 43);
             }
         }
     }
@@ -1113,21 +1024,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             if (p.cta_hist) p.cta_hist[(size_t)blockIdx.x * p.experts_real + i] = sh.hist[i];
         }
     }
-#ifdef SLICEMOE_TC_TRACE
-#ifdef SLICEMOE_TRACE_EXPERTS_ONLY
-    constexpr bool dump_trace = !C::ROUTER;
-#else
-    constexpr bool dump_trace = true;
-#endif
-    if (dump_trace && blockIdx.x == 0 && g_trace_buf) {
-        const uint2* src = reinterpret_cast<const uint2*>(smem_raw + kTraceOffset);
-        for (int i = threadIdx.x; i < 6 * kTraceSmemEvents; i += C::THREADS) {
-            const int slot = i / kTraceSmemEvents, n = i % kTraceSmemEvents;
-            g_trace_buf[((size_t)slot * kTraceEvents + n) * 2] = src[i].x;
-            g_trace_buf[((size_t)slot * kTraceEvents + n) * 2 + 1] = src[i].y;
-        }
-    }
-#endif
     tc_fence_before_sync();
     __syncthreads();          // nothing of this pass is in flight any more: barriers and TMEM may be reused
     tc_fence_after_sync();
@@ -1165,6 +1061,21 @@ int make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, ui
     return r == CUDA_SUCCESS ? SLICEMOE_OK : SLICEMOE_ERR_CUDA;
 }
 
+// cudaFuncSetAttribute applies to the current device only: raise a kernel's dynamic shared-memory limit once
+// per (kernel, device).  `done` is the kernel instantiation's own table (one bool per device).
+constexpr int kAttrMaxDevices = 64;
+template <class K>
+int set_smem_limit_once(K kern, int bytes, bool (&done)[kAttrMaxDevices]) {
+    int dev = -1;
+    SLICEMOE_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kAttrMaxDevices) return SLICEMOE_ERR_NO_DEVICE;
+    if (!done[dev]) {
+        SLICEMOE_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        done[dev] = true;
+    }
+    return SLICEMOE_OK;
+}
+
 int sm_count() {
     static int n = [] {
         int dev = 0, v = 0;
@@ -1176,11 +1087,7 @@ int sm_count() {
     return n;
 }
 
-#ifdef SLICEMOE_TC_TRACE
-template <class C> constexpr int kSmemLaunch = kTraceOffset + 6 * kTraceSmemEvents * 8;   // trace area behind the operand tiles
-#else
 template <class C> constexpr int kSmemLaunch = C::SMEM_ALLOC;
-#endif
 
 }  // namespace
 }  // namespace slicemoe

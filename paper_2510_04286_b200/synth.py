@@ -211,6 +211,36 @@ def make_weights(cfg: LayerConfig, seed: int = 0) -> dict:
     return w
 
 
+def make_router_weights(cfg: LayerConfig, seed: int = 0) -> dict:
+    """Only the router's tensors of make_weights (same streams, same values)."""
+    ds, Hr, E, dt = cfg.ds, cfg.Hr, cfg.E, cfg.dtype
+    if cfg.init != "normal":
+        raise ValueError("make_router_weights: normal init only")
+    std = 0.02
+    w = {"Wr1": _normal(seed, "Wr1", (Hr, ds), std, dt), "br1": np.zeros((Hr,), dtype=np.float32),
+         "Wr2": _normal(seed, "Wr2", (E, Hr), std * cfg.wr2_gain, dt), "br2": np.zeros((E,), dtype=np.float32)}
+    if cfg.zipf_s > 0.0:
+        w["br2"] = round_to_storage(zipf_router_bias(E, cfg.zipf_s).astype(np.float32), dt)
+    return w
+
+
+def make_expert_weights(cfg: LayerConfig, e: int, seed: int = 0) -> dict:
+    """W1[F, ds] and W2[ds, F] of expert ``e`` alone, ~ N(0, 0.02), from sub-streams of their own keyed by
+    (seed, tensor, e).  For layers whose expert tensors are too large to draw in one piece (the token-level
+    comparison of the decode workload: 17 GB of expert weights): a consumer draws one expert at a time.
+    These are NOT the values make_weights puts at index e of its stacked tensors."""
+    if cfg.init != "normal":
+        raise ValueError("make_expert_weights: normal init only")
+
+    def draw(name, shape):
+        key = np.array([seed, _TENSOR_IDS[name] | ((e + 1) << 32)], dtype=np.uint64)
+        x = np.random.Generator(np.random.Philox(key=key)).standard_normal(size=shape, dtype=np.float32)
+        x *= np.float32(0.02)
+        return round_to_storage(x, cfg.dtype)
+
+    return {"W1": draw("W1", (cfg.F, cfg.ds)), "W2": draw("W2", (cfg.ds, cfg.F))}
+
+
 def make_layer_inputs(cfg: LayerConfig, seed: int = 0):
     """(h, weights) for one workload."""
     return make_tokens(cfg, seed), make_weights(cfg, seed)

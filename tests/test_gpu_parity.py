@@ -323,9 +323,62 @@ def test_forward_token_level_decode():
     print("cfg4_token", rep)
 
 
+def test_forward_cfg4b_same_E_token_moe():
+    """The decode batch as a token-level MoE with whole-token experts (S = 1, FFN 4096 -> 16384 -> 4096, E = 64,
+    k = 2): 17 GB of expert weights, drawn and uploaded one expert at a time; only the experts that the
+    router picks are drawn (the others are never read).  Routing is graded on all 128 rows, every element of
+    h' against the oracle's Eq. 1 / expert FFN / sum run expert by expert on the ids the GPU picked."""
+    import dataclasses
+    import torch
+    lc = C["cfg4b"]
+    cfg = tensors.config_from_synth(lc)
+    h_np = synth.make_tokens(lc)
+    wr = synth.make_router_weights(lc)
+    ocfg = pu.oracle_config(lc)
+    w = tensors.weights_to_torch(wr, lc.dtype, drop_zero_biases=True)
+    w["W1"] = torch.empty((lc.E, lc.F, lc.ds), dtype=torch.bfloat16, device="cuda")
+    w["W2"] = torch.empty((lc.E, lc.ds, lc.F), dtype=torch.bfloat16, device="cuda")
+    w["b1"] = w["b2"] = None
+    h = tensors.to_torch(h_np, lc.dtype)
+    ws = binding.alloc_workspace(cfg)
+    idx = torch.empty((lc.N, lc.k), dtype=torch.int32, device="cuda")
+    p = torch.empty((lc.N, lc.k), dtype=torch.float32, device="cuda")
+    assigned = torch.empty((lc.E,), dtype=torch.int32, device="cuda")
+    binding.slicemoe_route(cfg, w, h, idx, p, assigned, ws=ws)
+    torch.cuda.synchronize()
+    idx_np = idx.cpu().numpy()
+    ref_route = oracle.route(ocfg, h_np, wr)
+    excluded = pu.check_routing(ref_route["probs"], ref_route["gap"], ref_route["topk_idx"], idx_np,
+                                p.cpu().numpy().astype(np.float64))
+    # the experts the router picked: drawn, uploaded, and used by the oracle, one at a time
+    touched = sorted(set(int(e) for e in idx_np.ravel()))
+    ref = np.zeros((lc.N, lc.ds), np.float64)
+    ocfg1 = dataclasses.replace(ocfg, E=1, k=1)
+    x = np.asarray(h_np, np.float64).reshape(lc.N, lc.ds)
+    zeros_b1, zeros_b2 = np.zeros((1, lc.F)), np.zeros((1, lc.ds))
+    for e in touched:
+        we = synth.make_expert_weights(lc, e)
+        w["W1"][e].copy_(tensors.to_torch(we["W1"], lc.dtype))
+        w["W2"][e].copy_(tensors.to_torch(we["W2"], lc.dtype))
+        rows, js = np.nonzero(idx_np == e)
+        gates = ref_route["probs"][rows, e]                                  # Eq. 1: the oracle's probability of the id
+        xt = gates[:, None] * x[rows]
+        y = oracle.expert_ffn(ocfg1, xt, np.array([0, len(rows)]),
+                              dict(W1=we["W1"][None], b1=zeros_b1, W2=we["W2"][None], b2=zeros_b2))
+        np.add.at(ref, rows, y)
+        del we
+    out = torch.empty_like(h)
+    binding.slicemoe_forward(cfg, w, h, out, ws, topk_idx=idx, topk_p=p, assigned=assigned)
+    torch.cuda.synchronize()
+    assert binding.slicemoe_last_status(ws) == 0
+    assert np.array_equal(idx.cpu().numpy(), idx_np)
+    errs = pu.assert_outputs_close(tensors.to_numpy_f32(out).reshape(lc.N, lc.ds), ref, lc.dtype)
+    print("cfg4b", dict(touched=len(touched), excluded=excluded, **errs))
+
+
 def test_forward_full_cfg3_capacity():
     for name in ("cfg3", "cfg3b"):
-        rep = pu.check_forward_against_oracle(C[name], sample_rows=4096)
+        rep = pu.check_forward_against_oracle(C[name], sample_rows=16384)
         print(name, rep)
 
 
@@ -345,5 +398,5 @@ def test_forward_paper_model_shape():
 
 
 def test_forward_full_cfg2_sampled_rows():
-    rep = pu.check_forward_against_oracle(C["cfg2"], sample_rows=8192)
+    rep = pu.check_forward_against_oracle(C["cfg2"], sample_rows=65536)
     print("cfg2", rep)

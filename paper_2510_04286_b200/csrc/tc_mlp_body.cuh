@@ -259,10 +259,31 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// packed fp32 arithmetic (two lanes per instruction)
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void mul2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
 // Expert activation, all arithmetic 2-wide in bf16 on one thread's 16-column piece of a row:
-//   convert   z = bf16(acc) * gate + bias             one conversion, two multiply-adds per pair (the gate
-//                                                     as a bf16 pair hi + lo: rounding it to one bf16
-//                                                     would tilt a whole row's pre-activations together)
+//   convert   z = bf16(acc * gate + bias)             Eq. 1's gate and the bias meet the fp32 accumulator before the
+//                                                     first rounding: one packed fp32 multiply-add, one conversion
 //   pre       t = tanh(z (c0 + c1 z^2))               three multiply-adds and one packed tanh per pair
 //   post      2 gelu(z) = z t + z                     one multiply-add per pair
 // GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))); the factor 0.5 is applied to
@@ -270,16 +291,18 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // saturates to +-1 and the formula still returns 2z (z > 0) or 0 (z < 0).
 // The tanh unit (16 results per clock per SM) is the scarce resource; the instruction count around
 // it is kept low enough that the issue slots are not the next one.
-__device__ __forceinline__ void convert_piece_bf16x2(const uint32_t* cur, __nv_bfloat162 gate_hi, __nv_bfloat162 gate_lo,
-                                                     const uint4* bias8, bool has_bias, __nv_bfloat162* z) {
+__device__ __forceinline__ void convert_piece_bf16x2(const uint32_t* cur, float gate, const uint4* bias8, bool has_bias,
+                                                     __nv_bfloat162* z) {
     uint4 braw[2];
     if (has_bias) { braw[0] = bias8[0]; braw[1] = bias8[1]; }      // 16 packed bf16, warp-wide broadcast
     else braw[0] = braw[1] = make_uint4(0u, 0u, 0u, 0u);
-    const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(braw);
+    const uint32_t* b2 = reinterpret_cast<const uint32_t*>(braw);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const __nv_bfloat162 a = __floats2bfloat162_rn(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]));
-        z[i] = __hfma2(a, gate_hi, __hfma2(a, gate_lo, b2[i]));
+        float z0, z1;                                               // (a bf16 is the upper half of its fp32)
+        fma2(z0, z1, __uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1]), gate, gate,
+             __uint_as_float(b2[i] << 16), __uint_as_float(b2[i] & 0xffff0000u));
+        z[i] = __floats2bfloat162_rn(z0, z1);
     }
 }
 template <int ACT>
@@ -817,9 +840,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     // next chunk runs under this chunk's activation.  Then piece by piece: the argument
                     // and tanh of piece pc, and behind them the tail and the store of piece pc - 1,
                     // whose tanh results have arrived by then.
-                    const __nv_bfloat16 gs_hi = __float2bfloat16_rn(gs);
-                    const __nv_bfloat162 gate_hi = __bfloat162bfloat162(gs_hi);
-                    const __nv_bfloat162 gate_lo = __float2bfloat162_rn(gs - __bfloat162float(gs_hi));
                     __nv_bfloat162 z[C::NPIECE][C::PIECE / 2];
 #pragma unroll
                     for (int s0 = 0; s0 < C::NPIECE; s0 += C::SUB) {
@@ -829,7 +849,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                         tmem_ld_wait();
 #pragma unroll
                         for (int i = 0; i < C::SUB; ++i)
-                            convert_piece_bf16x2(v[i], gate_hi, gate_lo, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
+                            convert_piece_bf16x2(v[i], gs, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
                                                  true, z[s0 + i]);
                     }
                     tc_fence_before_sync();

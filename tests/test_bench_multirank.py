@@ -49,5 +49,20 @@ def test_single_rank_helpers():
     w = bench.layer_work(synth.CONFIGS["cfg1"], kept_rows=262144, touched_experts=16)
     assert abs(w["total_flops"] - 22.55e9) < 0.01e9          # router 5.37 G + experts 17.18 G
     assert abs(w["compulsory_bytes"] - 34.7e6) < 0.1e6
-    assert bench.ncu_traffic("expert_ffn", synth.CONFIGS["cfg1"]) == pytest.approx(627.649024e6 / 8)
-    assert bench.ncu_traffic("expert_ffn", synth.CONFIGS["cfg3"]) is None
+    # a profiled figure scales by rows to a workload of the same slice width, k and F; any other has none
+    bench.NCU_TRAFFIC["probe"] = (800e6, 65536 * 16, 64, 2, 256, "a summary")
+    try:
+        assert bench.ncu_traffic("probe", synth.CONFIGS["cfg1"]) == (pytest.approx(100e6), "a summary")
+        assert bench.ncu_traffic("probe", synth.CONFIGS["cfg3"]) == (None, None)
+        assert bench.ncu_traffic("no such kernel", synth.CONFIGS["cfg1"]) == (None, None)
+    finally:
+        del bench.NCU_TRAFFIC["probe"]
+    r = bench.roofline_of(synth.CONFIGS["cfg1"], w, {"bf16_tflops": 1000.0, "hbm_gbs": 1000.0}, 1e-4)
+    assert r["bound"] == "hbm" and r["frac"] == pytest.approx(w["compulsory_bytes"] / 1e12 / 1e-4)
+    s = bench.ClockSampler("0")
+    s.samples = [(1.0, ["1900", "1965", "Not Active", "Not Active", "Not Active", "Active"]),
+                 (2.0, ["1800", "1965", "Not Active", "Not Active", "Not Active", "Not Active"]),
+                 (3.0, ["1700", "1965", "Active", "Not Active", "Not Active", "Not Active"])]
+    assert s.summary(0.5, 2.5) == {"sm_mhz": 1900.0, "sm_max_mhz": 1965.0, "reasons": ["sw_power_cap"], "samples": 2}
+    assert s.summary()["reasons"] == ["hw_slowdown", "sw_power_cap"]
+    assert bench.median([3.0, 1.0, 2.0]) == 2.0

@@ -1,4 +1,6 @@
 """GPU parity: every C-ABI call against the fp64 oracle on the same seeded inputs."""
+import dataclasses
+
 import numpy as np
 import pytest
 
@@ -223,6 +225,26 @@ def test_forward_host_with_capacity_is_not_chunked():
     torch.cuda.synchronize()
     assert torch.equal(out_host, h_dev.cpu()) and torch.equal(kept, kept_dev)
     assert int(kept.max()) == 300                    # the limit binds, so chunking would have changed the result
+
+
+def test_forward_host_with_logit_noise_is_not_chunked():
+    """Section 3.3's logit noise is drawn per global row number: the host-buffer forward of a batch large
+    enough for the chunked pipeline must pick the same experts and give the same bits as the device forward."""
+    import torch
+    lc = LC("hostnoise", T=2048 + 130, d=512, S=8, E=16, k=2, F=256, noise_sigma=0.5, noise_seed=99)
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    h_dev, assigned_dev, kept_dev, _, _ = gpu.forward()
+    quiet = pu.GpuLayer(dataclasses.replace(lc, noise_sigma=0.0), h, w)
+    assert not torch.equal(quiet.forward()[1], assigned_dev)          # the noise really moves the routing
+    h_host = tensors.to_torch(h, lc.dtype, "cpu", pin=True)
+    out_host = torch.zeros_like(h_host).pin_memory()
+    assigned = torch.zeros((lc.E,), dtype=torch.int32, device="cuda")
+    kept = torch.zeros((lc.E,), dtype=torch.int32, device="cuda")
+    binding.slicemoe_forward_host(gpu.cfg, gpu.w, h_host, out_host, gpu.ws, assigned, kept)
+    torch.cuda.synchronize()
+    assert torch.equal(out_host, h_dev.cpu())
+    assert torch.equal(assigned, assigned_dev) and torch.equal(kept, kept_dev)
 
 
 def test_profiled_forward_records_stage_times():

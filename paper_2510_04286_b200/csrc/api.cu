@@ -167,6 +167,9 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
         return launch_forward_pp(D, w, h, h_out, idx, p, assigned, kept, offsets, dest, xperm, at<int32_t>(ws, W.cta_hist),
                                  at<int32_t>(ws, W.status), clear_status, /*one_launch=*/!events, events, st);
     }
+    // decode-shaped batches: one launch that streams each expert's weights once
+    if (!events && decode_forward_supported(D))
+        return launch_forward_decode(D, w, h, h_out, idx, p, assigned, kept, xperm, at<int32_t>(ws, W.status), clear_status, st);
     const bool one_launch = !events && fused_forward_supported(D);
     // (the single kernel clears the status word itself; a later chunk of one host-buffer call keeps
     // what an earlier chunk reported)
@@ -514,6 +517,7 @@ int slicemoe_last_status(const void* ws, void* stream) {
         int rc = slicemoe::fused_forward_reset_sync(static_cast<cudaStream_t>(stream));
         if (rc) return rc;
         if ((rc = slicemoe::pp_forward_reset_sync(static_cast<cudaStream_t>(stream)))) return rc;
+        if ((rc = slicemoe::decode_forward_reset_sync(static_cast<cudaStream_t>(stream)))) return rc;
     }
     return word;
 }

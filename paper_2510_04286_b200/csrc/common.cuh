@@ -144,6 +144,14 @@ int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, v
                       cudaStream_t st);
 int pp_forward_reset_sync(cudaStream_t st);
 
+// Decode-shaped forward (decode_forward.cu): 128-wide slices, F = 512, Hr = 256, at most 32 rows per SM, k <= 2, no
+// capacity limit; one cooperative launch.  `lists` is scratch of at least E * N * 2 bytes.
+bool decode_forward_supported(const Dims& D);
+int launch_forward_decode(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
+                          float* topk_p, int32_t* assigned, int32_t* kept, void* lists, int32_t* status,
+                          bool clear_status, cudaStream_t st);
+int decode_forward_reset_sync(cudaStream_t st);
+
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);
 

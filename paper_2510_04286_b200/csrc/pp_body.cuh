@@ -208,7 +208,8 @@ struct PpParams {
     const bf16* b1;             // [E, F] or nullptr
     const bf16* b2;             // [E, 64] or nullptr
     const bf16* gather_src;     // h as X[N, 64]
-    const int2* pair_gate;      // [R] stacked row -> (pair index n k + j, gate as float bits)
+    const int2* pair_gate;      // [R] stacked row -> (pair index n k + j, gate as float bits); or per-expert lists
+    int list_stride;            // 0: pair_gate is indexed by stacked row; else expert e's rows start at e * list_stride
     uint32_t gather_magic, gather_shift;
     bf16* scatter_out;          // h' as Y[N, 64]
     int row_elems;              // real slice width (<= 64)
@@ -497,7 +498,8 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     for (int q = 0; q < 4; ++q) {
                         const int r = rbase + 4 * (lane & 15) + q;
                         nnext[q] = make_int2(-1, 0);
-                        if (r < wn.rows) nnext[q] = SAME_LAUNCH ? __ldcg(p.pair_gate + wn.row0 + r) : __ldg(p.pair_gate + wn.row0 + r);
+                        const size_t at = p.list_stride ? (size_t)wn.e * p.list_stride + (wn.row0 - sh.offs[wn.e]) + r : (size_t)wn.row0 + r;
+                        if (r < wn.rows) nnext[q] = SAME_LAUNCH ? __ldcg(p.pair_gate + at) : __ldg(p.pair_gate + at);
                     }
                 }
                 if (ta < 0) continue;
@@ -1084,6 +1086,78 @@ __device__ __forceinline__ void pp_dispatch_body(const int32_t* topk_idx, const 
         const int d = base[e] + r;
         dest[i] = d;
         pair_gate[d] = make_int2((int)i, __float_as_int(pr2));
+    }
+}
+
+// =====================================================================================================
+// One-barrier form of the same dispatch (one launch, E * 8 <= k * 128 so that the lists fit in the stacked-row
+// scratch): right after its router pass a CTA reserves, with ONE atomic per expert, a range of each expert's
+// list for its pairs (base = the counter before the add) and appends them at base + local rank; after the
+// grid barrier the counters are the experts' totals.  Expert e's list starts at lists + e * list_stride.
+// `base`: shared memory, E ints.
+// =====================================================================================================
+template <int NT>
+__device__ __forceinline__ void pp_push_body(const int32_t* topk_idx, const float* topk_p, const int32_t* local_rank,
+                                             const int* hist, int32_t* counts, int chunk, int R, int E, int pairs_per_chunk,
+                                             int list_stride, int2* lists, int* base) {
+    const long long begin = (long long)chunk * pairs_per_chunk;
+    long long end = begin + pairs_per_chunk;
+    if (end > R) end = R;
+    constexpr int kPre = 4;
+    int pe[kPre], pr[kPre];
+    float pp[kPre];
+#pragma unroll
+    for (int q = 0; q < kPre; ++q) {
+        const long long i = begin + threadIdx.x + (long long)q * NT;
+        pe[q] = -1;
+        if (i < end) {
+            pe[q] = __ldcg(topk_idx + i);
+            pr[q] = __ldcg(local_rank + i);
+            pp[q] = __ldcg(topk_p + i);
+        }
+    }
+    if ((int)threadIdx.x < E) {
+        const int h = hist[threadIdx.x];
+        base[threadIdx.x] = h > 0 ? atomicAdd(counts + threadIdx.x, h) : 0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < kPre; ++q) {
+        if (pe[q] >= 0) {
+            const long long i = begin + threadIdx.x + (long long)q * NT;
+            lists[(size_t)pe[q] * list_stride + base[pe[q]] + pr[q]] = make_int2((int)i, __float_as_int(pp[q]));
+        }
+    }
+    for (long long i = begin + threadIdx.x + (long long)kPre * NT; i < end; i += NT) {
+        const int e = __ldcg(topk_idx + i);
+        const int r = __ldcg(local_rank + i);
+        const float pr2 = __ldcg(topk_p + i);
+        lists[(size_t)e * list_stride + base[e] + r] = make_int2((int)i, __float_as_int(pr2));
+    }
+}
+
+// After the barrier: the experts' row ranges from the counters (E <= 32: one warp).
+__device__ __forceinline__ void pp_offsets_from_counts(const int32_t* counts, int E, int lane, bool write_out, int32_t* assigned,
+                                                       int32_t* kept, int32_t* offsets, int* offs_out) {
+    const int cnt = lane < E ? __ldcg(counts + lane) : 0;
+    int incl = cnt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
+    }
+    if (lane < E) {
+        offs_out[lane] = incl - cnt;
+        if (write_out) {
+            if (assigned) assigned[lane] = cnt;
+            if (kept) kept[lane] = cnt;
+            offsets[lane] = incl - cnt;
+        }
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    if (lane == 0) {
+        offs_out[E] = total;
+        if (write_out) offsets[E] = total;
     }
 }
 

@@ -22,36 +22,34 @@ struct PpFusedParams {
     int R, E, pairs_per_chunk;
     int32_t *assigned, *kept, *offsets, *dest;
     int2* pair_gate;
-    int32_t* sync_words;
+    unsigned long long* sync_word;
+    int32_t* counts;          // [2][kMaxE] per-expert counters of the one-barrier dispatch, used alternately by successive launches
+    int lists;                // 1: one-barrier dispatch (per-expert lists), 0: ranked dispatch between two barriers
     int clear_status;
 };
 
-// Grid barrier words (arrival count, generation) of this file's cooperative kernel, one pair per
-// device: zero at module load, left ready for the next barrier by every barrier that completes.
-__device__ int32_t g_pp_sync[2];
+// Grid barriers of this file's cooperative kernel on ONE monotonic 64-bit arrival counter per device (zero at
+// module load): a launch passes two barriers, i.e. adds 2 * gridDim.x.  The count a CTA finds at entry, rounded
+// down to a multiple of that, is the launch's base whichever CTAs have already arrived; the barriers wait for
+// base + gridDim.x and base + 2 * gridDim.x.  One release-add and acquire polls each: no last-arriver step.
+__device__ unsigned long long g_pp_sync;
+__device__ int32_t g_pp_counts[2 * kMaxE];
 
-__device__ __forceinline__ bool pp_grid_barrier(int32_t* words, int32_t gen_before, PpShared& sh) {
+__device__ __forceinline__ bool pp_grid_barrier(unsigned long long* word, unsigned long long inc, unsigned long long target, PpShared& sh) {
     fence_proxy_async_smem();     // the phases reuse shared memory through different proxies
     __syncthreads();
     if (threadIdx.x == 0) {
-        volatile int32_t* count = words;
-        volatile int32_t* gen = words + 1;
-        __threadfence();
-        if (atomicAdd(words, 1) == (int)gridDim.x - 1) {
-            *count = 0;
-            __threadfence();
-            atomicAdd(words + 1, 1);
-        } else {
-            const uint64_t t0 = globaltimer_ns();
-            while (*gen == gen_before) {
-                if (globaltimer_ns() - t0 > kWaitLimitNs) {
-                    sh.abort_flag = 1;
-                    break;
-                }
-                __nanosleep(64);
+        asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(word), "l"(inc) : "memory");
+        const uint64_t t0 = globaltimer_ns();
+        for (;;) {
+            unsigned long long v;
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(word) : "memory");
+            if (v >= target) break;
+            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                sh.abort_flag = 1;
+                break;
             }
         }
-        __threadfence();
     }
     __syncthreads();
     return sh.abort_flag == 0;
@@ -66,7 +64,7 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     __shared__ PpShared sh;
     const int warp = threadIdx.x >> 5;
-    int32_t gen0 = 0;
+    __shared__ unsigned long long base_s;
 #ifdef PP_TRACE
     PpTr ph(63);
     ph.on = ph.on && threadIdx.x == 0;
@@ -76,27 +74,47 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 #endif
     PH(1);
     if (threadIdx.x == 0) {
-        gen0 = *reinterpret_cast<volatile int32_t*>(fp.sync_words + 1);   // no barrier can complete without this CTA
+        unsigned long long v;
+        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fp.sync_word) : "memory");
+        base_s = v - v % (2ull * gridDim.x);
         if (blockIdx.x == 0 && fp.clear_status) *fp.ffn.status = SLICEMOE_OK;
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh.tmem_base), 512);
         tmem_relinquish();
     }
-    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
+    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);       // (syncs the CTA: base_s is visible after it)
     PH(2);
+    const unsigned long long base = base_s;
     bool ok = sh.abort_flag == 0;
-    ok = pp_grid_barrier(fp.sync_words, gen0, sh) && ok;
-    PH(3);
-    if (ok) {
-        int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
-        pp_dispatch_body<kPpThreads, true>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, fp.route.cta_hist,
-                                           (int)gridDim.x, (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.assigned,
-                                           fp.kept, fp.offsets, fp.dest, fp.pair_gate, dsm, sh.offs);
+    int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
+    // successive launches alternate between two sets of counters: each launch, whichever dispatch it uses, zeroes
+    // the set of the next one (nobody touches that set during this launch)
+    const int parity = (int)((base / (2ull * gridDim.x)) & 1ull);
+    int32_t* counts = fp.counts + parity * kMaxE;
+    if (blockIdx.x == 0 && (int)threadIdx.x < kMaxE) fp.counts[(parity ^ 1) * kMaxE + threadIdx.x] = 0;
+    if (fp.lists) {
+        if (ok)
+            pp_push_body<kPpThreads>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, sh.hist, counts, (int)blockIdx.x,
+                                     fp.R, fp.E, fp.pairs_per_chunk, fp.ffn.list_stride, fp.pair_gate, dsm);
+        PH(3);
+        PH(4);
+        ok = pp_grid_barrier(fp.sync_word, 2ull, base + 2ull * gridDim.x, sh) && ok;
+        PH(5);
+        if (ok && warp == 0)
+            pp_offsets_from_counts(counts, fp.E, (int)(threadIdx.x & 31), blockIdx.x == 0, fp.assigned, fp.kept, fp.offsets, sh.offs);
+        __syncthreads();
+    } else {
+        ok = pp_grid_barrier(fp.sync_word, 1ull, base + gridDim.x, sh) && ok;
+        PH(3);
+        if (ok)
+            pp_dispatch_body<kPpThreads, true>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, fp.route.cta_hist,
+                                               (int)gridDim.x, (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.assigned,
+                                               fp.kept, fp.offsets, fp.dest, fp.pair_gate, dsm, sh.offs);
+        PH(4);
+        ok = pp_grid_barrier(fp.sync_word, 1ull, base + 2ull * gridDim.x, sh) && ok;
+        PH(5);
     }
-    PH(4);
-    ok = pp_grid_barrier(fp.sync_words, gen0 + 1, sh) && ok;
-    PH(5);
     if (ok) pp_ffn_body<N2, ACT, true, true>(&tmXg, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
     PH(6);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
@@ -156,10 +174,11 @@ pp_ffn_kernel(const __grid_constant__ CUtensorMap tmXg, const __grid_constant__ 
 
 constexpr int kMaxDevices = 64;
 std::mutex g_pp_mutex;
-int32_t* g_pp_sync_addr[kMaxDevices] = {};
+unsigned long long* g_pp_sync_addr[kMaxDevices] = {};
+int32_t* g_pp_counts_addr[kMaxDevices] = {};
 bool g_pp_attr[kMaxDevices][16] = {};      // per device and kernel instantiation: shared-memory limit raised
 
-int pp_sync_address(int32_t** out, int* dev_out) {
+int pp_sync_address(unsigned long long** out, int32_t** counts_out) {
     int dev = -1;
     SLICEMOE_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return SLICEMOE_ERR_NO_DEVICE;
@@ -168,10 +187,14 @@ int pp_sync_address(int32_t** out, int* dev_out) {
         void* p = nullptr;
         SLICEMOE_CUDA_TRY(cudaGetSymbolAddress(&p, g_pp_sync));
         if (!p) return SLICEMOE_ERR_CUDA;
-        g_pp_sync_addr[dev] = static_cast<int32_t*>(p);
+        g_pp_sync_addr[dev] = static_cast<unsigned long long*>(p);
+        void* c = nullptr;
+        SLICEMOE_CUDA_TRY(cudaGetSymbolAddress(&c, g_pp_counts));
+        if (!c) return SLICEMOE_ERR_CUDA;
+        g_pp_counts_addr[dev] = static_cast<int32_t*>(c);
     }
     *out = g_pp_sync_addr[dev];
-    if (dev_out) *dev_out = dev;
+    if (counts_out) *counts_out = g_pp_counts_addr[dev];
     return SLICEMOE_OK;
 }
 
@@ -319,10 +342,12 @@ extern "C" int slicemoe_debug_pp_trace(int on, void* host_out) {
 #endif
 
 int pp_forward_reset_sync(cudaStream_t st) {
-    int32_t* words = nullptr;
-    int rc = pp_sync_address(&words, nullptr);
+    unsigned long long* words = nullptr;
+    int32_t* counts = nullptr;
+    int rc = pp_sync_address(&words, &counts);
     if (rc) return rc;
-    SLICEMOE_CUDA_TRY(cudaMemsetAsync(words, 0, 2 * sizeof(int32_t), st));
+    SLICEMOE_CUDA_TRY(cudaMemsetAsync(words, 0, sizeof(unsigned long long), st));
+    SLICEMOE_CUDA_TRY(cudaMemsetAsync(counts, 0, 2 * kMaxE * sizeof(int32_t), st));
     SLICEMOE_CUDA_TRY(cudaStreamSynchronize(st));
     return SLICEMOE_OK;
 }
@@ -342,7 +367,7 @@ int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, v
                       cudaStream_t st) {
     PpFusedParams fp{};
     fp.clear_status = clear_status ? 1 : 0;
-    int rc = pp_sync_address(&fp.sync_words, nullptr);
+    int rc = pp_sync_address(&fp.sync_word, &fp.counts);
     if (rc) return rc;
     const int grid = sm_count();
     const int tiles = (D.N + kTileM - 1) / kTileM;
@@ -352,6 +377,9 @@ int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, v
     fp.R = D.R; fp.E = D.E; fp.pairs_per_chunk = rows_per_cta * D.k;
     fp.assigned = assigned; fp.kept = kept; fp.offsets = offsets; fp.dest = dest;
     fp.pair_gate = static_cast<int2*>(pair_gate);
+    // the per-expert lists (E * N entries of 8 bytes) must fit in the stacked-row scratch (N * k rows of 128 bytes)
+    fp.lists = (one_launch && D.E * 8 <= D.k * 128) ? 1 : 0;
+    fp.ffn.list_stride = fp.lists ? D.N : 0;
     switch (D.E) {
         case 8:
         case 16: return pp_launch_act<16, 64>(D, w, h, fp, st, one_launch, events);

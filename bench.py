@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Throughput of the SliceMoE layer forward on B200, one JSON line per run.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl ours|reference] [--backward]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--impl ours|reference] [--staged] [--backward]
 
 A step is one whole layer forward (route -> dispatch -> expert FFN -> combine) over one batch of
 seeded synthetic tokens.  `value` is tokens/s with the inputs already in HBM, the K steps captured once
@@ -448,6 +448,37 @@ def run_ours(args, lc):
     torch.cuda.synchronize()
     stage_ms = np.median([e.stage_ms() for e in ev], axis=0)
 
+    # ---- --staged: the four staged calls of the C ABI one by one (route, dispatch, expert_ffn, combine) -----
+    # Not part of `value` (the forward call above is one launch): each call's median time over the rotating
+    # batches and its algorithmic bytes / FLOPs, i.e. the achieved HBM GB/s of dispatch and combine.
+    staged = None
+    if args.staged:
+        nb = min(sets, 4)
+        st_idx = [torch.empty((cfg.N, cfg.k), dtype=torch.int32, device="cuda") for _ in range(nb)]
+        st_p = [torch.empty((cfg.N, cfg.k), dtype=torch.float32, device="cuda") for _ in range(nb)]
+        st_kept = torch.empty((cfg.E,), dtype=torch.int32, device="cuda")
+        st_off = torch.empty((cfg.E + 1,), dtype=torch.int32, device="cuda")
+        st_dest = [torch.empty((cfg.N, cfg.k), dtype=torch.int32, device="cuda") for _ in range(nb)]
+        st_perm = torch.empty((max(cfg.R, 1),), dtype=torch.int32, device="cuda")
+        st_x = [torch.empty((max(cfg.R, 1), cfg.ds), dtype=sm.torch_dtype(cfg), device="cuda") for _ in range(nb)]
+        st_y = [torch.empty((max(cfg.R, 1), cfg.ds), dtype=sm.torch_dtype(cfg), device="cuda") for _ in range(nb)]
+        calls = {
+            "route": lambda i: sm.slicemoe_route(cfg, w, hs[i % nb], st_idx[i % nb], st_p[i % nb], assigned, None, ws),
+            "dispatch": lambda i: sm.slicemoe_dispatch(cfg, hs[i % nb], st_idx[i % nb], st_p[i % nb], st_kept, st_off,
+                                                       st_dest[i % nb], st_perm, st_x[i % nb], ws),
+            "expert_ffn": lambda i: sm.slicemoe_expert_ffn(cfg, w, st_x[i % nb], st_off, st_y[i % nb], ws),
+            "combine": lambda i: sm.slicemoe_combine(cfg, st_y[i % nb], st_dest[i % nb], outs[i % nb]),
+        }
+        for i in range(nb):                      # every buffer set holds a consistent chain before anything is timed
+            for fn in calls.values():
+                fn(i)
+        torch.cuda.synchronize()
+        staged = {}
+        for name, fn in calls.items():
+            ts, _, _ = wl.timed(fn, min(steps, 16), 10, 0.0, barrier)
+            (t_call,) = max_over_ranks([median(ts) / min(steps, 16)], dist, device="cuda")
+            staged[name] = t_call
+
     # ---- timed region 4 (--backward): slicemoe_backward on the same batches -----------------
     # Not part of `value`: the headline metric is the forward, and the default run launches the forward's
     # kernels only.  Each set's expert ids and gates come
@@ -584,6 +615,12 @@ def run_ours(args, lc):
                                "bound": layer["bound"], "frac": layer["frac"], "kept_rows": kept_rows,
                                "touched_experts": touched, "peak_source": f"of {peak_src}"},
         }
+        if staged is not None:
+            sb, sf = work["stage_bytes"], work["stage_flops"]
+            line["staged_calls"] = {
+                name: {"ms": 1e3 * t, "hbm_gbs": sb[name] / t / 1e9, "frac_of_hbm": sb[name] / t / 1e9 / peaks["hbm_gbs"],
+                       **({"tflops": sf[name] / t / 1e12} if name in sf else {})}
+                for name, t in staged.items()}
         if others:
             line["other_configs"] = others
         if bwd is not None:
@@ -623,6 +660,8 @@ def main():
     ap.add_argument("--replays", type=int, default=100, help="least number of timed replays of the K steps")
     ap.add_argument("--min-seconds", type=float, default=2.0,
                     help="least device time of the timed region (more replays are added to reach it)")
+    ap.add_argument("--staged", action="store_true",
+                    help="also time the four staged calls one by one (the `staged_calls` object: ms and achieved HBM GB/s)")
     ap.add_argument("--backward", action="store_true",
                     help="also time slicemoe_backward on the same batches (the `backward` object of the line)")
     args = ap.parse_args()

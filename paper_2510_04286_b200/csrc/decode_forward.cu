@@ -79,14 +79,6 @@ enum { W1_FULL = 0, W2_FULL = 2, W1_EMPTY = 4, W2_EMPTY = 6, A_FULL = 8, A_EMPTY
 
 __device__ unsigned long long g_dec_sync;
 __device__ int32_t g_dec_counts[2 * kDecMaxE];
-#ifdef DEC_TRACE
-__device__ unsigned long long g_dec_trace[160][24];
-#define DT(i) do { if (threadIdx.x == 0) g_dec_trace[blockIdx.x][i] = globaltimer_ns(); } while (0)
-#define DTM(i) do { if (threadIdx.x == 288) g_dec_trace[blockIdx.x][i] = globaltimer_ns(); } while (0)
-#else
-#define DT(i)
-#define DTM(i)
-#endif
 
 // Grid barrier on ONE monotonic 64-bit arrival counter: every launch adds gridDim.x to it, so the count a CTA
 // finds at entry, rounded down to a multiple of gridDim.x, is this launch's base whichever CTAs have already
@@ -187,7 +179,6 @@ __device__ __forceinline__ void dec_route(const CUtensorMap* tmX, const CUtensor
             *reinterpret_cast<uint4*>(p.Y + (size_t)row0 * kDecDs + (size_t)c * 8) = make_uint4(0u, 0u, 0u, 0u);
         named_barrier_sync(1, kDecWorkers);
         bool ok = pp_wait(bar(DB::R_ACC1), 0u, abort);
-        DT(13);
         if (ok) {
             tc_fence_after_sync();
             const uint32_t base = tlane + 128 * g;
@@ -207,9 +198,7 @@ __device__ __forceinline__ void dec_route(const CUtensorMap* tmX, const CUtensor
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(DB::R_HID));
-            DT(14);
             ok = pp_wait(bar(DB::R_ACC2), 0u, abort);
-            DT(15);
         }
         // softmax + top-k of a row (ties go to the lower id): the two threads of a row (one per column half) each
         // keep the best two of E / 2 logits and the sum of exponentials about their own maximum; the thread of
@@ -266,7 +255,6 @@ __device__ __forceinline__ void dec_route(const CUtensorMap* tmX, const CUtensor
                     p.topk_p[at + 1] = p2;
                 }
             }
-            DT(17);
             int e[2], base[2], leader[2];
             uint32_t m[2];
 #pragma unroll
@@ -277,7 +265,6 @@ __device__ __forceinline__ void dec_route(const CUtensorMap* tmX, const CUtensor
                 base[j] = 0;
                 if (e[j] >= 0 && lane == leader[j]) base[j] = atomicAdd(counts + e[j], __popc(m[j]));
             }
-            DT(18);
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 base[j] = __shfl_sync(0xffffffffu, base[j], leader[j]);
@@ -381,7 +368,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int rt = (int)blockIdx.x - ((int)gridDim.x - p.n_router);      // >= 0: this CTA routes rows [128 rt, +128)
     volatile int* abort = &sh.abort_flag;
     auto bar = [&](int i) { return smem_u32(&sh.bars[i]); };
-    DT(0);
 
     if (threadIdx.x == 0) {
         sh.base = dec_barrier_base(p.sync_word);
@@ -420,7 +406,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     // successive launches alternate between two sets of counters: this one's were zeroed by the previous launch
     const int parity = (int)((base / gridDim.x) & 1ull);
     int32_t* counts = p.counts + parity * kDecMaxE;
-    DT(1);
 
     // weights of chunk c of expert e into ring slot s (W1: rows [128 c, +128) of W1_e; W2: columns [128 c, +128) of W2_e)
     auto load_w1 = [&](int e, int c, int s) {
@@ -461,10 +446,8 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         for (int i = lane; i < kDecDs; i += 32) sh.bias2[i] = p.b2 ? __bfloat162float(p.b2[(size_t)home * kDecDs + i]) : 0.0f;
         if (lane == 0) sh.bias_e = home;
     }
-    DT(2);
 
     bool ok = dec_grid_barrier(p.sync_word, base, sh);
-    DT(3);
 
     // ---- schedule ----------------------------------------------------------------------------------------
     if (ok && threadIdx.x < E) sh.cnt[threadIdx.x] = __ldcg(counts + threadIdx.x);
@@ -476,7 +459,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         if (p.kept) p.kept[e] = sh.cnt[e];
     }
     __syncthreads();
-    DT(4);
     const int n_items = ok ? sh.n_items : 0;
     const int kshift = p.k - 1;          // k is 1 or 2
     // the prefetched chunks serve the first item if it belongs to the home expert; otherwise those two fills of
@@ -538,7 +520,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             fence_proxy_async_smem();          // the tensor pipe reads the tile through the async proxy
             named_barrier_sync(1, kDecWorkers);
             if (threadIdx.x == 0) mbar_arrive(bar(DB::A_FULL));
-            if (it == 0) DT(5);
             const float gs = sh.gate[row];
             const bool live = lg * 32 < rows;        // a warp whose 32 rows are all padding only passes the hand-offs on
             for (int c = 0; c < kDecNC && wok; ++c) {
@@ -564,7 +545,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(DB::HID_FULL + r));
-                if (it == 0) DT(6 + c);
             }
             if (!wok) break;
             if (!pp_wait(bar(DB::ACC2_FULL), (uint32_t)it & 1u, abort)) { wok = false; break; }
@@ -594,7 +574,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             }
             // (the next item rewrites the pair / gate / bias arrays: all workers are past them after this)
             named_barrier_sync(1, kDecWorkers);
-            if (it == 0) DT(10);
         }
     } else if (warp == 8) {
         // ================= weight ring producer =============================================================
@@ -636,9 +615,7 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         auto gemm1 = [&](int it, int c) -> bool {
             const int n = it * kDecNC + c, s = n & 1;
             if (c == 0 && !pp_wait(bar(DB::A_FULL), (uint32_t)it & 1u, abort)) return false;
-            if (n == 0) DTM(19);
             if (!pp_wait(bar(DB::W1_FULL + s), full_parity(n), abort)) return false;
-            if (n == 0) DTM(20);
             tc_fence_after_sync();
             const uint32_t d = tmem_base + s * kDecHC;
             if (elect_one_sync()) {
@@ -659,8 +636,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             if (c == 0 && it > 0 && !pp_wait(bar(DB::ACC2_FREE), (uint32_t)(it - 1) & 1u, abort)) return false;
             if (!pp_wait(bar(DB::W2_FULL + s), full_parity(n), abort)) return false;
             if (!pp_wait(bar(DB::HID_FULL + s), (uint32_t)(n >> 1) & 1u, abort)) return false;
-            if (n == 0) DTM(21);
-            if (n == 3) DTM(22);
             tc_fence_after_sync();
             const uint32_t hid = tmem_base + s * kDecHC, d2 = tmem_base + 2 * kDecHC;
             if (elect_one_sync()) {
@@ -702,10 +677,6 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         __syncwarp();
         tmem_dealloc(tmem_base, 512);
     }
-    DT(11);
-#ifdef DEC_TRACE
-    if (threadIdx.x == 0) g_dec_trace[blockIdx.x][12] = (unsigned long long)n_items;
-#endif
 }
 
 std::mutex g_dec_mutex;
@@ -767,8 +738,8 @@ int dec_launch_act(const Dims& D, const slicemoe_weights& w, const void* h, cons
                                            : dec_launch<E, SLICEMOE_ACT_RELU>(D, w, h, p, grid, st);
 }
 
-// one CTA per SM (the trace buffers of development builds hold 160)
-int dec_grid() { return sm_count() < 160 ? sm_count() : 160; }
+// one CTA per SM
+int dec_grid() { return sm_count(); }
 
 }  // namespace
 
@@ -808,12 +779,6 @@ int launch_forward_decode(const Dims& D, const slicemoe_weights& w, const void* 
         default: return dec_launch_act<64>(D, w, h, p, grid, st);
     }
 }
-
-#ifdef DEC_TRACE
-extern "C" int slicemoe_debug_dec_trace(void* host_out) {
-    return cudaMemcpyFromSymbol(host_out, g_dec_trace, sizeof(unsigned long long) * 160 * 24) == cudaSuccess ? 0 : 7;
-}
-#endif
 
 int decode_forward_reset_sync(cudaStream_t st) {
     unsigned long long* words = nullptr;

@@ -80,8 +80,9 @@ dispatch_scan_kernel(int32_t* __restrict__ chunk_hist, int nchunks, int E, int c
     }
 }
 
+constexpr int kScatterThreads = 1024;   // 8 ranking warps; 32 warps of independent 16-byte copies keep enough bytes in flight
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kScatterThreads)
 dispatch_scatter_kernel(const T* __restrict__ X, const int32_t* __restrict__ topk_idx,
                         const float* __restrict__ topk_p, const int32_t* __restrict__ chunk_base,
                         const int32_t* __restrict__ offsets, int R, int E, int k, int ds, int capacity,
@@ -92,21 +93,25 @@ dispatch_scatter_kernel(const T* __restrict__ X, const int32_t* __restrict__ top
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int chunk = blockIdx.x;
     const int warp_base = chunk * kDispatchChunk + warp * kPairsPerWarp;
-    int* mine = wcnt + warp * E;
+    // (the first kWarps warps rank the chunk's pairs; all warps of the CTA copy the rows)
+    const bool ranker = warp < kWarps;
+    int* mine = wcnt + (ranker ? warp : 0) * E;
 
-    for (int e = lane; e < E; e += 32) mine[e] = 0;
-    __syncwarp();
-    // pass A: this warp's count per expert
-    for (int it = 0; it < kIters; ++it) {
-        const int pair = warp_base + it * 32 + lane;
-        if (pair < R) {
-            const int e = topk_idx[pair];
-            if (e >= 0 && e < E) atomicAdd(&mine[e], 1);
+    if (ranker) {
+        for (int e = lane; e < E; e += 32) mine[e] = 0;
+        __syncwarp();
+        // pass A: this warp's count per expert
+        for (int it = 0; it < kIters; ++it) {
+            const int pair = warp_base + it * 32 + lane;
+            if (pair < R) {
+                const int e = topk_idx[pair];
+                if (e >= 0 && e < E) atomicAdd(&mine[e], 1);
+            }
         }
     }
     __syncthreads();
     // exclusive prefix over the warps, seeded with the chunk's base rank
-    for (int e = threadIdx.x; e < E; e += kThreads) {
+    for (int e = threadIdx.x; e < E; e += kScatterThreads) {
         int run = chunk_base[(size_t)chunk * E + e];
         for (int w = 0; w < kWarps; ++w) {
             const int t = wcnt[w * E + e];
@@ -115,9 +120,10 @@ dispatch_scatter_kernel(const T* __restrict__ X, const int32_t* __restrict__ top
         }
     }
     __syncthreads();
-    // pass B: stable rank of each pair, then the row copy
-    const int vec_per_row = ds / V;
-    for (int it = 0; it < kIters; ++it) {
+    // pass B: stable rank of each pair; its destination and gate also go to shared memory for the copy
+    int* sd = wcnt + kWarps * E;                                      // [kDispatchChunk] destination row or -1
+    float* sp = reinterpret_cast<float*>(sd + kDispatchChunk);        // [kDispatchChunk] gate
+    for (int it = 0; ranker && it < kIters; ++it) {
         const int pair = warp_base + it * 32 + lane;
         int e = -1;
         float p = 0.0f;
@@ -145,22 +151,28 @@ dispatch_scatter_kernel(const T* __restrict__ X, const int32_t* __restrict__ top
                 if (gate) gate[d] = p;
             }
         }
-        if (xperm != nullptr) {
-            const int total = 32 * vec_per_row;
-            for (int v = lane; v < total; v += 32) {
-                const int item = v / vec_per_row, col = v - item * vec_per_row;
-                const int d_i = __shfl_sync(0xffffffffu, d, item);
-                const float p_i = __shfl_sync(0xffffffffu, p, item);
-                const int pair_i = warp_base + it * 32 + item;
-                if (d_i >= 0) {
-                    const int n = pair_i / k;
-                    float f[V];
-                    unpack16<T>(*reinterpret_cast<const uint4*>(X + (size_t)n * ds + (size_t)col * V), f);
+        sd[warp * kPairsPerWarp + it * 32 + lane] = d;
+        sp[warp * kPairsPerWarp + it * 32 + lane] = p;
+    }
+    if (xperm == nullptr) return;
+    __syncthreads();
+    // the row copies of the whole chunk as one flat loop over 16-byte pieces: consecutive threads take
+    // consecutive pieces of a row, and several independent loads per thread are in flight
+    const int vec_per_row = ds / V;
+    const int total = kDispatchChunk * vec_per_row;
+    const int chunk_pair0 = chunk * kDispatchChunk;
+#pragma unroll 4
+    for (int v = threadIdx.x; v < total; v += kScatterThreads) {
+        const int item = v / vec_per_row, col = v - item * vec_per_row;
+        const int d_i = sd[item];
+        if (d_i >= 0) {
+            const float p_i = sp[item];
+            const int n = (chunk_pair0 + item) / k;
+            float f[V];
+            unpack16<T>(*reinterpret_cast<const uint4*>(X + (size_t)n * ds + (size_t)col * V), f);
 #pragma unroll
-                    for (int i = 0; i < V; ++i) f[i] *= p_i;
-                    *reinterpret_cast<uint4*>(xperm + (size_t)d_i * ds + (size_t)col * V) = pack16<T>(f);
-                }
-            }
+            for (int i = 0; i < V; ++i) f[i] *= p_i;
+            *reinterpret_cast<uint4*>(xperm + (size_t)d_i * ds + (size_t)col * V) = pack16<T>(f);
         }
     }
 }
@@ -193,13 +205,13 @@ int launch_dispatch(const Dims& D, const void* h, const int32_t* topk_idx, const
                                                             offsets);
     SLICEMOE_LAUNCH_CHECK(1);
     if (nchunks > 0) {
-        const size_t smem = sizeof(int) * kWarps * D.E;
+        const size_t smem = sizeof(int) * kWarps * D.E + (sizeof(int) + sizeof(float)) * kDispatchChunk;
         if (D.dtype == SLICEMOE_BF16)
-            dispatch_scatter_kernel<bf16><<<nchunks, kThreads, smem, st>>>(
+            dispatch_scatter_kernel<bf16><<<nchunks, kScatterThreads, smem, st>>>(
                 (const bf16*)h, topk_idx, topk_p, chunk_hist, offsets, D.R, D.E, D.k, D.ds, D.capacity,
                 dest, perm, (bf16*)xperm, gate_opt);
         else
-            dispatch_scatter_kernel<float><<<nchunks, kThreads, smem, st>>>(
+            dispatch_scatter_kernel<float><<<nchunks, kScatterThreads, smem, st>>>(
                 (const float*)h, topk_idx, topk_p, chunk_hist, offsets, D.R, D.E, D.k, D.ds, D.capacity,
                 dest, perm, (float*)xperm, gate_opt);
         SLICEMOE_LAUNCH_CHECK(1);

@@ -1,28 +1,34 @@
-// Two-stream ("ping-pong") tensor-core pipeline for 64-wide slices, bf16 storage (sm_100a: tcgen05 +
-// TMEM + TMA), used by the forward of the layer (Section 3.1, Eq. 1; Section 3.4):
+// Tensor-core pipeline for 64-wide slices, bf16 storage (sm_100a: tcgen05 + TMEM + TMA), used by the forward of
+// the layer (Section 3.1, Eq. 1; Section 3.4):
 //
 //   router  : relu(X Wr1^T + br1) Wr2^T + br2 -> softmax -> top-k, per 128-row tile
 //   experts : act(p (x W1_e^T) + b1_e) W2_e^T + b2_e, per 128-row tile of one expert's rows, rows gathered
-//             from h through the permutation and results added into h'
+//             from h and results added into h'
 //
-// A CTA of 384 threads (one per SM) walks a contiguous range of tiles; even tiles go to stream 0, odd
-// tiles to stream 1.  Each stream owns half of tensor memory (256 columns), one MMA-issuing warp and
-// one warpgroup of 128 "row" threads (thread r of the warpgroup owns tile row r for everything that
-// happens between the two GEMMs and after the second):
+// One CTA of 768 threads per SM walks a contiguous range of tiles.  Hand-offs are per whole tile, never per
+// chunk: a tile's GEMM-1 writes the whole hidden layer (fp32) into one of two 256-column regions of tensor
+// memory, the activation warps turn it IN PLACE into packed bf16 (the A operand of GEMM-2, which therefore never
+// leaves tensor memory), GEMM-2 writes the tile's output accumulator into the same region's upper half.  While
+// one region is in the activation, the other is in its GEMMs or its output.  Expert pass, warp roles:
 //
-//   warp 0      TMA producer: weights (and the row tiles where they are not gathered)
-//   warp 1 / 2  MMA issue for stream 0 / 1: GEMM-1 of a 64-unit hidden chunk into a TMEM accumulator,
-//               GEMM-2 from the TMEM-resident hidden chunk into the stream's output accumulator
-//   warp 3      experts: gathers the rows of the next tiles (cp.async into the swizzled A buffers);
-//               router: zeroes this CTA's rows of h'
-//   warps 4-7   row threads of stream 0;  warps 8-11  row threads of stream 1
+//   warp 0       weight sets by TMA (W1 and W2 of an expert stay in shared memory for a run of tiles of that
+//                expert; two sets) and four-row TMA gathers of tile rows 64-127
+//   warp 2       four-row TMA gathers of tile rows 0-63; both gather warps also copy the rows' (pair, gate)
+//                into a ring in shared memory
+//   warp 3       GEMM-1 issue (one elected lane), warp 1  GEMM-2 issue: two issuing warps, because the small
+//                MMAs of this layer are bound by issue, not by the tensor pipe
+//   warps 4-19   activation: four warpgroups that split a tile's hidden columns; a thread owns one tile row:
+//                gate * acc + b1 and GELU in fp32 (packed two-wide multiply-adds, tanh.approx.f32), 16 columns
+//                at a time so that nothing spills
+//   warps 20-23  output: 0.5 acc + b2 -> bf16, added into row n of h' with 16-byte reductions
 //
-// While one stream's row threads evaluate the activation (the tanh unit is what bounds the expert
-// pass), the tensor pipe works on the other stream's GEMMs, and a stream's own GEMM-1 runs two chunks
-// ahead of its activation (two accumulators), so that a row thread seldom waits.  With a third of the
-// threads of a 24-warp layout every row thread has ~160 registers: a whole 64-column chunk is held in
-// fp32 and the activation is evaluated in fp32 (packed two-wide fp32 multiply-adds), 16 independent
-// column pairs at a time.  All hand-offs are mbarriers with bounded waits (status word on run-out).
+// The router pass has the same shape with its hidden layer in units of 128 (three buffers), the fp32 hidden
+// values split in place into a truncated bf16 and the rounded remainder (so that the logits keep fp32
+// accuracy), and an output warpgroup that does softmax, top-k and each pair's rank among its CTA's pairs of
+// the same expert.  All hand-offs are mbarriers with bounded waits (status word on run-out).
+//
+// With ~200 KB of shared memory per CTA there is next to no L1 left for local memory: everything the role
+// loops call is inlined and sized to compile without a stack frame or a spill.
 #pragma once
 #include "tc_mlp_body.cuh"
 
@@ -30,12 +36,6 @@ namespace slicemoe {
 namespace {
 
 constexpr int kPpThreads = 768;
-#ifndef PP_SLEEP_NS
-#define PP_SLEEP_NS 100
-#endif
-#ifndef PP_STAGGER_NS
-#define PP_STAGGER_NS 400
-#endif
 constexpr int kPpABufs = 4;              // row-tile buffers
 // Depth of the per-tile metadata ring: an entry is written up to kPpABufs tiles ahead of GEMM-1 and read by
 // the output warps, which run at most three tiles behind GEMM-1 (two regions and the tile being written).
@@ -52,36 +52,6 @@ __device__ __forceinline__ float tanh_approx(float x) {
     asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(x));
     return t;
 }
-// Bounded wait for the service warps (copies, MMA issue): between tries the warp sleeps, so that its polling
-// does not take issue slots from the row threads that share its scheduler.
-__device__ __forceinline__ bool mbar_try_wait_nohint(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-static __device__ __noinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, volatile int* abort, uint64_t limit_ns) {
-    if (mbar_test_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 16; ++i) {
-            __nanosleep(PP_SLEEP_NS);
-            if (mbar_test_wait(bar, parity)) return true;
-        }
-        if (*abort) return false;
-        if (globaltimer_ns() - t0 > limit_ns) {
-            *abort = 1;
-            return false;
-        }
-    }
-}
-
 // Bounded wait of a whole (converged) warp.  (Inline, like everything the role loops call: an out-of-line
 // call costs a stack frame, and with ~200 KB of shared memory per CTA there is next to no L1 left for
 // local memory -- a kernel that spills runs every piece of scalar book-keeping at L2 latency.)
@@ -90,19 +60,6 @@ __device__ __forceinline__ bool pp_wait(uint32_t bar, uint32_t parity, volatile 
     if (__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
     return (bool)__all_sync(0xffffffffu, mbar_wait(bar, parity, abort, kWaitLimitNs));
 }
-
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-// Adds `bytes` (a multiple of 16) of packed bf16 from shared memory to global memory, asynchronously, as one
-// operation of the copy engine (both addresses 16-byte aligned); completion is tracked by bulk groups.
-__device__ __forceinline__ void bulk_reduce_add_bf16(void* gdst, uint32_t smem_src, uint32_t bytes) {
-    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.noftz.bf16 [%0], [%1], %2;"
-                 ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all bulk groups of this thread have finished reading their shared-memory source
-__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // Four rows of a 2-D tensor (row indices y0..y3, columns from x on, one box of the map wide; the map's box is
 // one row high) into four consecutive 128-byte rows of shared memory, swizzled like a tiled load.
@@ -118,23 +75,6 @@ __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-#ifdef PP_TRACE
-__device__ unsigned long long g_pp_trace[64][4096];
-__device__ int g_pp_trace_on = 0;
-struct PpTr {
-    int n, slot; bool on;
-    __device__ PpTr(int slot_) : n(0), slot(slot_), on(blockIdx.x == 0 && (threadIdx.x & 31) == 0 && g_pp_trace_on) {}
-    __device__ void operator()(int code) { if (on && n < 4095) { g_pp_trace[slot][n++] = ((unsigned long long)code << 48) | (clock64() & 0xffffffffffffull); g_pp_trace[slot][n] = 0; } }
-};
-__device__ int g_pp_dbg = 0;
-#define DBG(bit) (g_pp_dbg & (bit))
-#define TRD(name, slot) PpTr name(slot)
-#define TR(name, code) name(code)
-#else
-#define TRD(name, slot)
-#define TR(name, code)
-#define DBG(bit) 0
-#endif
 
 // Shared-memory state of one CTA besides the operand tiles.
 struct PpShared {
@@ -373,7 +313,6 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             const uint32_t idesc1 = make_idesc(128, p.HID, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW = desc_lo_sw128(sW);
             bool ok = true;
-            TRD(tr, warp);
             PpWalk w1;
             w1.init();
             int run1 = -1;
@@ -385,11 +324,8 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     if (!pp_wait(pp_bar(sh, B::W_FULL + (w1.run & 1)), ((uint32_t)w1.run >> 1) & 1u, abort)) { ok = false; break; }
                     run1 = w1.run;
                 }
-                TR(tr, 8);
                 if (!pp_wait(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u, abort)) { ok = false; break; }
-                TR(tr, 10);
                 if (!pp_wait(pp_sbar(sh, r, B::ACC2_EMPTY), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
-                TR(tr, 11);
                 tc_fence_after_sync();
                 const uint32_t wset = dW + (((w1.run & 1) * C::SET_BYTES) >> 4);
                 const uint32_t a0 = dA + ((ab * kPpABytes) >> 4);
@@ -402,7 +338,6 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     mma_commit(pp_bar(sh, B::A_EMPTY + ab));
                 }
                 __syncwarp();
-                TR(tr, 12);
             }
             if (!ok || *abort) {
                 volatile int never = 0;
@@ -419,7 +354,6 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             constexpr uint32_t idesc2 = make_idesc(128, N2, kFmtBF16, kFmtBF16);
             const uint32_t dW = desc_lo_sw128(sW);
             bool ok = true;
-            TRD(tr, warp);
             PpWalk w2;
             w2.init();
             w2.advance(sh, t_begin, 0);
@@ -429,9 +363,7 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                 const uint32_t w2d = dW + (((w2.run & 1) * C::SET_BYTES + C::W1_SET) >> 4);
                 const int run_before = w2.run;
                 const int crossed = ta + 1 < ntiles ? w2.advance(sh, t_begin, ta + 1) : 0;   // (before the wait: off the critical path)
-                TR(tr, 20);
                 if (!pp_wait(pp_sbar(sh, r, B::HID_FULL), (uint32_t)(ta >> 1) & 1u, abort)) { ok = false; break; }
-                TR(tr, 21);
                 tc_fence_after_sync();
                 const uint32_t d = tmem_base + r * kPpStreamCols;
                 if (elect_one_sync()) {
@@ -450,7 +382,6 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     if (crossed) mma_commit(pp_bar(sh, B::W_EMPTY + (run_before & 1)));
                 }
                 __syncwarp();
-                TR(tr, 22);
             }
             if (!ok || *abort) {
                 volatile int never = 0;
@@ -480,7 +411,6 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             int loaded_run = -1, cur_e = 0, cur_run = 0, cur_rows = 0;
             uint32_t last_bar = 0, last_par = 0;
             bool ok = true;
-            TRD(tr, warp);
             const uint32_t set_tx = (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK);
 #pragma unroll 1
             for (int ta = -1; ta < ntiles && ok; ++ta) {
@@ -522,10 +452,8 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     last_par = n & 1u;
                 }
                 const int ab = ta % kPpABufs;
-                TR(tr, 30);
                 ok = pp_wait(pp_bar(sh, B::A_EMPTY + ab), ((uint32_t)(ta / kPpABufs) & 1u) ^ 1u, abort);
                 if (!ok) break;
-                TR(tr, 31);
                 // the tile's metadata (its ring entry was last read by the output warps of tile ta - kPpMetaRing,
                 // long before GEMM-1 of tile ta - kPpABufs, whose completion this warp has just waited for)
                 if (lane < 16) {
@@ -539,9 +467,8 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     if (warp == 2) mbar_arrive_expect_tx(pp_bar(sh, B::A_FULL + ab), kPpABytes);
                     else mbar_arrive(pp_bar(sh, B::A_FULL + ab));
                 }
-                if (lane < 16 && !DBG(1))
+                if (lane < 16)
                     tma_gather4(sA + ab * kPpABytes + (rbase / 4 + lane) * 512, tmXg_p, 0, nrow[0], nrow[1], nrow[2], nrow[3], pp_bar(sh, B::A_FULL + ab));
-                TR(tr, 32);
             }
             if (!ok || *abort) {
                 // (bounded) let the copies in flight land before shared memory is reused
@@ -558,15 +485,12 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
         const int row = lg * 32 + lane;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
         bool ok = true;
-        TRD(tr, warp);
         int run_bias = -1;
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
             const int r = ta & 1;
-            TR(tr, 40);
             ok = pp_wait(pp_sbar(sh, r, B::ACC1_FULL), (uint32_t)(ta >> 1) & 1u, abort);
             if (!ok) break;
-            TR(tr, 41);
             tc_fence_after_sync();
             // (the tile's rows, and with them its ring entry, landed before GEMM-1 could run)
             const float gs = __int_as_float(sh.pair_gate_s[ta % kPpMetaRing][row].y);
@@ -600,12 +524,10 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                 pp_act8<ACT>(z, hid);
                 tmem_st_x8(region + 8 * q, hid);
             }
-            TR(tr, 45);
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::HID_FULL));
-            TR(tr, 46);
         }
     } else {
         // ================= output warpgroup ===========================================================
@@ -614,14 +536,11 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
         const int row = lg * 32 + lane;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
         bool ok = true;
-        TRD(tr, warp);
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
             const int r = ta & 1;
-            TR(tr, 49);
             ok = pp_wait(pp_sbar(sh, r, B::ACC2_FULL), (uint32_t)(ta >> 1) & 1u, abort);
             if (!ok) break;
-            TR(tr, 50);
             tc_fence_after_sync();
             const int4 ti = sh.tile_s[ta % kPpMetaRing];       // (expert, run, rows) of the tile
             const bool live = row < ti.z;
@@ -656,12 +575,10 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
-            TR(tr, 52);
-            if (live && !DBG(4)) {
+            if (live) {
 #pragma unroll
                 for (int c = 0; c < N2; c += 8) red_add_bf16x8(dst + c, o[c / 2], o[c / 2 + 1], o[c / 2 + 2], o[c / 2 + 3]);
             }
-            TR(tr, 53);
         }
     }
 
@@ -776,19 +693,15 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             constexpr uint32_t idesc1 = make_idesc(128, 128, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1);
             bool ok = true;
-            TRD(tr, 40 + warp);
             ok = pp_wait(pp_bar(sh, B::W_FULL), 0u, abort);
 #pragma unroll 1
             for (int u = 0; u < nunits && ok; ++u) {
                 const int ta = u / nhalf, hf = u - ta * nhalf;
                 const int ab = ta % kPpABufs;
-                TR(tr, 8);
                 if (hf == 0 && !pp_wait(pp_bar(sh, B::A_FULL + ab), (uint32_t)(ta / kPpABufs) & 1u, abort)) { ok = false; break; }
                 const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
-                TR(tr, 10);
                 // (the buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
                 if (!pp_wait(pp_sbar(sh, 0, B::ACC1_EMPTY + b), (n & 1u) ^ 1u, abort)) { ok = false; break; }
-                TR(tr, 11);
                 tc_fence_after_sync();
                 const uint32_t a0 = dA + ((ab * kPpABytes) >> 4), w0 = dW1 + ((hf * (128 * 128)) >> 4);
                 const uint32_t d = tmem_base + b * C::HB_COLS;
@@ -800,7 +713,6 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
                     if (hf == nhalf - 1) mma_commit(pp_bar(sh, B::A_EMPTY + ab));
                 }
                 __syncwarp();
-                TR(tr, 12);
             }
             if (!ok || *abort) {
                 volatile int never = 0;
@@ -817,18 +729,14 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             constexpr uint32_t idesc2 = make_idesc(128, EP, kFmtBF16, kFmtBF16);
             const uint32_t dW2 = desc_lo_sw128(sW2);
             bool ok = true;
-            TRD(tr, 40 + warp);
             ok = pp_wait(pp_bar(sh, B::W_FULL), 0u, abort);
 #pragma unroll 1
             for (int u = 0; u < nunits && ok; ++u) {
                 const int ta = u / nhalf, hf = u - ta * nhalf;
                 const int r = ta & 1;
-                TR(tr, 19);
                 if (hf == 0 && !pp_wait(pp_sbar(sh, r, B::ACC2_EMPTY), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
                 const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
-                TR(tr, 20);
                 if (!pp_wait(pp_sbar(sh, 0, B::HID_FULL + b), n & 1u, abort)) { ok = false; break; }
-                TR(tr, 21);
                 tc_fence_after_sync();
                 const uint32_t w0 = dW2 + ((hf * 2 * C::W2_CHUNK) >> 4);
                 const uint32_t d = tmem_base + C::LOGIT_COL + r * 64, a = tmem_base + b * C::HB_COLS;
@@ -846,7 +754,6 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
                     if (hf == nhalf - 1) mma_commit(pp_sbar(sh, r, B::ACC2_FULL));
                 }
                 __syncwarp();
-                TR(tr, 22);
             }
             if (!ok || *abort) {
                 volatile int never = 0;
@@ -874,15 +781,12 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
         const int lg = warp & 3;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + 32 * g;
         bool ok = true;
-        TRD(tr, 40 + warp);
 #pragma unroll 1
         for (int u = 0; u < nunits && ok; ++u) {
             const int ta = u / nhalf, hf = u - ta * nhalf;
             const uint32_t b = (uint32_t)u % 3u, par = ((uint32_t)u / 3u) & 1u;
-            TR(tr, 40);
             ok = pp_wait(pp_sbar(sh, 0, B::ACC1_FULL + b), par, abort);
             if (!ok) break;
-            TR(tr, 41);
             tc_fence_after_sync();
             const uint32_t acol = tlane + b * C::HB_COLS;
             const float* bias = sh.bias1_f32[0] + hf * 128 + 32 * g;
@@ -909,12 +813,10 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
                     hl[8 + i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hl[i] << 16), a[2 * i + 1] - __uint_as_float(hl[i] & 0xFFFF0000u));
                 tmem_st_x16(acol + 16 * pc, hl);
             }
-            TR(tr, 45);
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(pp_sbar(sh, 0, B::HID_FULL + b));
-            TR(tr, 46);
         }
     } else {
         // ================= output warpgroup ===========================================================
@@ -923,14 +825,11 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
         const int row = lg * 32 + lane;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + C::LOGIT_COL;
         bool ok = true;
-        TRD(tr, 40 + warp);
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
             const int r = ta & 1;
-            TR(tr, 49);
             ok = pp_wait(pp_sbar(sh, r, B::ACC2_FULL), (uint32_t)(ta >> 1) & 1u, abort);
             if (!ok) break;
-            TR(tr, 50);
             tc_fence_after_sync();
             uint32_t v[EP];
 #pragma unroll
@@ -939,7 +838,6 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
-            TR(tr, 52);
             const int n = (t_begin + ta) * kTileM + row;
             if (n >= p.n_rows) continue;
             // one pass keeping the best two (strict comparisons in ascending id order: same picks as
@@ -971,7 +869,6 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
                 p.topk_p[at + 1] = ex2_approx(fmaf(b2, sc, -msc)) * inv;
                 p.local_rank[at + 1] = atomicAdd(&sh.hist[i2], 1);
             }
-            TR(tr, 53);
         }
     }
 

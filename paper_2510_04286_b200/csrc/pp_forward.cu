@@ -1,15 +1,15 @@
-// The forward of the layer (Section 3.1, Eq. 1; Section 3.4) on the two-stream pipeline of pp_body.cuh,
-// for 64-wide slices without a capacity limit: as ONE cooperative launch
+// The forward of the layer (Section 3.1, Eq. 1; Section 3.4) on the pipeline of pp_body.cuh, for 64-wide slices
+// without a capacity limit: as ONE cooperative launch
 //
 //   phase 1  router     top-k ids and probabilities, each pair's rank among this CTA's pairs of its expert,
-//                       this CTA's per-expert counts, its rows of h' zeroed
+//                       this CTA's per-expert counts, its rows of h' zeroed; then, where the per-expert lists
+//                       fit the scratch (E * 8 <= k * 128), the CTA reserves a range of each expert's list with
+//                       one atomic per expert and appends its (pair, gate) entries there
 //   -- grid barrier --
-//   phase 2  dispatch   stacked row of each of this CTA's pairs = offsets[e] + pairs of e in earlier CTAs +
-//                       the pair's rank; (pair, gate) written at that row; CTA 0 writes assigned/kept/offsets
-//   -- grid barrier --
-//   phase 3  experts    rows gathered from h, outputs added into h'
+//   phase 2  experts    row ranges from the experts' totals; rows gathered from h, outputs added into h'
 //
-// and as one launch per phase (the stage-timed call).
+// (for larger E a ranked dispatch phase between two grid barriers takes the place of the lists), and as one
+// launch per phase (the stage-timed call).
 #include <mutex>
 
 #include "pp_body.cuh"
@@ -65,14 +65,6 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     __shared__ PpShared sh;
     const int warp = threadIdx.x >> 5;
     __shared__ unsigned long long base_s;
-#ifdef PP_TRACE
-    PpTr ph(63);
-    ph.on = ph.on && threadIdx.x == 0;
-#define PH(c) ph(c)
-#else
-#define PH(c)
-#endif
-    PH(1);
     if (threadIdx.x == 0) {
         unsigned long long v;
         asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fp.sync_word) : "memory");
@@ -84,7 +76,6 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         tmem_relinquish();
     }
     pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);       // (syncs the CTA: base_s is visible after it)
-    PH(2);
     const unsigned long long base = base_s;
     bool ok = sh.abort_flag == 0;
     int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
@@ -97,26 +88,19 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         if (ok)
             pp_push_body<kPpThreads>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, sh.hist, counts, (int)blockIdx.x,
                                      fp.R, fp.E, fp.pairs_per_chunk, fp.ffn.list_stride, fp.pair_gate, dsm);
-        PH(3);
-        PH(4);
         ok = pp_grid_barrier(fp.sync_word, 2ull, base + 2ull * gridDim.x, sh) && ok;
-        PH(5);
         if (ok && warp == 0)
             pp_offsets_from_counts(counts, fp.E, (int)(threadIdx.x & 31), blockIdx.x == 0, fp.assigned, fp.kept, fp.offsets, sh.offs);
         __syncthreads();
     } else {
         ok = pp_grid_barrier(fp.sync_word, 1ull, base + gridDim.x, sh) && ok;
-        PH(3);
         if (ok)
             pp_dispatch_body<kPpThreads, true>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, fp.route.cta_hist,
                                                (int)gridDim.x, (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.assigned,
                                                fp.kept, fp.offsets, fp.dest, fp.pair_gate, dsm, sh.offs);
-        PH(4);
         ok = pp_grid_barrier(fp.sync_word, 1ull, base + 2ull * gridDim.x, sh) && ok;
-        PH(5);
     }
     if (ok) pp_ffn_body<N2, ACT, true, true>(&tmXg, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
-    PH(6);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
     __syncthreads();
     if (warp == 1) {
@@ -328,18 +312,6 @@ bool pp_cooperative_launch_available() {
 }
 
 }  // namespace
-
-#ifdef PP_TRACE
-extern "C" int slicemoe_debug_pp_flags(int flags) {
-    cudaMemcpyToSymbol(g_pp_dbg, &flags, sizeof(int));
-    return cudaDeviceSynchronize() == cudaSuccess ? 0 : 7;
-}
-extern "C" int slicemoe_debug_pp_trace(int on, void* host_out) {
-    if (host_out) cudaMemcpyFromSymbol(host_out, g_pp_trace, sizeof(unsigned long long) * 64 * 4096);
-    cudaMemcpyToSymbol(g_pp_trace_on, &on, sizeof(int));
-    return cudaDeviceSynchronize() == cudaSuccess ? 0 : 7;
-}
-#endif
 
 int pp_forward_reset_sync(cudaStream_t st) {
     unsigned long long* words = nullptr;

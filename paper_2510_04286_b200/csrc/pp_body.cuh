@@ -18,9 +18,10 @@
 //   warp 3       GEMM-1 issue (one elected lane), warp 1  GEMM-2 issue: two issuing warps, because the small
 //                MMAs of this layer are bound by issue, not by the tensor pipe
 //   warps 4-19   activation: four warpgroups that split a tile's hidden columns; a thread owns one tile row:
-//                gate * acc + b1 and GELU in fp32 (packed two-wide multiply-adds, tanh.approx.f32), 16 columns
-//                at a time so that nothing spills
-//   warps 20-23  output: 0.5 acc + b2 -> bf16, added into row n of h' with 16-byte reductions
+//                gate * acc + b1 and GELU in fp32 (packed two-wide multiply-adds, tanh.approx.f32), 8 columns
+//                at a time as a software pipeline around the tanh unit
+//   warps 20-23  output: 0.5 acc + b2 -> bf16, staged in shared memory by row and added into row n of h' with
+//                16-byte reductions that cover four whole rows per warp instruction
 //
 // The router pass has the same shape with its hidden layer in units of 128 (three buffers), the fp32 hidden
 // values split in place into a truncated bf16 and the rounded remainder (so that the logits keep fp32
@@ -85,7 +86,8 @@ struct PpShared {
     uint32_t tmem_base;
     int abort_flag;
     // experts: first-layer bias of the run each stream is in, as fp32; router: br1 / br2 as fp32
-    __align__(16) float bias1_f32[2][kPpMaxHr];
+    // (experts: two halves of kPpMaxF, by run parity; router: one array of up to kPpMaxHr)
+    __align__(16) float bias1_f32[kPpMaxHr];
     __align__(16) float bias2_f32[kMaxE];
     // experts: per tile in flight (ring over the CTA's tile counter), written by the gather warps with the
     // tile's rows: each row's (pair index, gate), and the tile's expert, run and row count
@@ -107,6 +109,7 @@ struct PpBars {
     static constexpr int COUNT = DRAIN + 2;
 };
 static_assert(PpBars::COUNT <= 48, "barrier slots");
+static_assert(2 * kPpMaxF <= kPpMaxHr, "the experts' two bias halves share the router's array");
 
 // Walks the CTA's tile list in order; `run` counts the expert changes seen so far (a run = consecutive
 // tiles of one expert = one weight set).
@@ -142,6 +145,8 @@ struct PpParams {
     int32_t* local_rank;        // [N, k] rank of the pair among this CTA's pairs of the same expert
     int32_t* cta_hist;          // [grid, E]
     bf16* zero_out;             // h' as [N, 64]: this CTA zeroes the rows it routes (or nullptr)
+    int2* lists_out;            // per-expert lists of (pair index, gate) filled by the router itself (or nullptr): expert e's
+    int32_t* list_counts;       // list starts at lists_out + e * list_stride and holds list_counts[e] entries
     // ---- experts
     int E;
     const int32_t* offsets;     // [E + 1] (read when the offsets are not already in shared memory)
@@ -207,13 +212,73 @@ struct PpFfnCfg {
     static constexpr int SET_BYTES = W1_SET + ((W2_SET + 1023) / 1024) * 1024;
     static constexpr int OFF_A = 0;
     static constexpr int OFF_W = kPpABufs * kPpABytes;
-    static constexpr int SMEM_BYTES = OFF_W + 2 * SET_BYTES;
+    // output staging: one row of N2 bf16 per tile row, at a pitch of 16 bytes more than a 128-byte row so that
+    // the 16-byte stores of eight neighbouring row threads fall on different banks
+    static constexpr int OFF_OUT = OFF_W + 2 * SET_BYTES;
+    static constexpr int OUT_PITCH = 144;
+    static constexpr int SMEM_BYTES = OFF_OUT + kTileM * OUT_PITCH;
     static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;
     static constexpr int ACC2_COL = 128;
     static_assert(N2 % 16 == 0 && N2 <= 64, "output width");
     static_assert(SMEM_ALLOC <= 218 * 1024, "shared memory budget");
 };
 
+// The activation of one row, eight hidden units (a "piece") at a time, in three steps that the row threads run
+// as a software pipeline (the tanh of piece j is in flight while piece j + 1 is prepared and piece j - 1 is
+// finished, so that the tanh unit, 16 results per clock per SM, never waits for the other pipes):
+//   pre   z = acc * gate + bias; u = sqrt(2/pi) (z + 0.044715 z^3)        (packed two-wide multiply-adds)
+//   tanh  t = tanh(u)
+//   post  hidden = z t + z = 2 gelu(z), packed bf16 (the factor 0.5 is applied to the second GEMM's accumulator
+//         in the output step: exact, a power of two)
+// ReLU needs no tanh: post packs relu(z).
+template <int ACT>
+__device__ __forceinline__ void pp_pre8(const uint32_t* acc, float gs, const float* bias /* shared, 8 floats */, bool has_bias,
+                                        float* z, float* u) {
+    if (has_bias) {
+#pragma unroll
+        for (int i = 0; i < 8; i += 4) {
+            const float4 b = *reinterpret_cast<const float4*>(bias + i);   // same address for the whole warp
+            fma2(z[i], z[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), gs, gs, b.x, b.y);
+            fma2(z[i + 2], z[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), gs, gs, b.z, b.w);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) mul2(z[i], z[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), gs, gs);
+    }
+    if constexpr (ACT != SLICEMOE_ACT_RELU) {
+        constexpr float c0 = 0.7978845608028654f, c1 = 0.7978845608028654f * 0.044715f;
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            float s0, s1, n0, n1;
+            mul2(s0, s1, z[i], z[i + 1], z[i], z[i + 1]);
+            fma2(n0, n1, s0, s1, c1, c1, c0, c0);
+            mul2(u[i], u[i + 1], z[i], z[i + 1], n0, n1);
+        }
+    }
+}
+template <int ACT>
+__device__ __forceinline__ void pp_tanh8(float* u) {
+    if constexpr (ACT != SLICEMOE_ACT_RELU) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) u[i] = tanh_approx(u[i]);
+    }
+}
+template <int ACT>
+__device__ __forceinline__ void pp_post8(const float* z, const float* t, uint32_t* out) {
+    if constexpr (ACT == SLICEMOE_ACT_RELU) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) out[i] = cvt_rn_relu_bf16x2(z[2 * i], z[2 * i + 1]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float r0, r1;
+            fma2(r0, r1, z[2 * i], z[2 * i + 1], t[2 * i], t[2 * i + 1], z[2 * i], z[2 * i + 1]);
+            out[i] = pack_bf16x2(r0, r1);
+        }
+    }
+}
+
+// The same activation in turns of 16 units without the pipeline (decode-shaped forward).
 // 16 column pairs of one row: z = acc * gate (+ bias), hidden = 2 gelu(z) or relu(z), packed bf16.
 // GELU, tanh form: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))); the factor 0.5 is applied to the
 // second GEMM's accumulator in the output step (exact, a power of two).
@@ -254,11 +319,32 @@ __device__ __forceinline__ void pp_act8(const float* z, uint32_t* out) {
     }
 }
 
+// Barriers of the expert pass (one thread; the CTA synchronises before anybody waits on them).
+__device__ __forceinline__ void pp_ffn_init_bars(PpShared& sh, const CUtensorMap* tmXg_p, const CUtensorMap* tmW1_p,
+                                                 const CUtensorMap* tmW2_p) {
+    using B = PpBars;
+    sh.abort_flag = 0;
+    for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 2); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(pp_bar(sh, B::W_FULL + i), 1); mbar_init(pp_bar(sh, B::W_EMPTY + i), 1); }
+    mbar_init(pp_bar(sh, B::DRAIN + 1), 1);
+    for (int r = 0; r < 2; ++r) {                                  // per tensor-memory region
+        mbar_init(pp_sbar(sh, r, B::ACC1_FULL), 1);
+        mbar_init(pp_sbar(sh, r, B::HID_FULL), 16);
+        mbar_init(pp_sbar(sh, r, B::ACC2_FULL), 1);
+        mbar_init(pp_sbar(sh, r, B::ACC2_EMPTY), 4);
+    }
+    mbar_init(pp_bar(sh, B::DRAIN), 1);
+    fence_mbar_init();
+    prefetch_tensormap(tmXg_p);
+    prefetch_tensormap(tmW1_p);
+    prefetch_tensormap(tmW2_p);
+}
+
 // Called by all kPpThreads threads; TMEM (512 columns at sh.tmem_base) is allocated and freed by the
 // caller.  SAME_LAUNCH: pair_gate (and the offsets) were written earlier in this launch.
-// OFFS_IN_SMEM: sh.offs already holds the row ranges.  Rows come from gather_src through pair_gate and
-// results are added into scatter_out.
-template <int N2, int ACT, bool SAME_LAUNCH, bool OFFS_IN_SMEM>
+// READY: the caller has initialised the barriers (pp_ffn_init_bars), filled sh.offs and sh.tile_start and
+// synchronised the CTA.  Rows come from gather_src through pair_gate and results are added into scatter_out.
+template <int N2, int ACT, bool SAME_LAUNCH, bool READY>
 __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p,
                                             const PpParams& p, PpShared& sh, uint8_t* smem_raw) {
     using C = PpFfnCfg<N2>;
@@ -271,30 +357,15 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
     const bool wide = p.HID == 256;          // two 32-unit sub-chunks per row thread and tile, else one
 
     // ---- set-up -----------------------------------------------------------------------------------
-    if (threadIdx.x == 0) {
-        sh.abort_flag = 0;
-        for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 2); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(pp_bar(sh, B::W_FULL + i), 1); mbar_init(pp_bar(sh, B::W_EMPTY + i), 1); }
-        mbar_init(pp_bar(sh, B::DRAIN + 1), 1);
-        for (int r = 0; r < 2; ++r) {                                  // per tensor-memory region
-            mbar_init(pp_sbar(sh, r, B::ACC1_FULL), 1);
-            mbar_init(pp_sbar(sh, r, B::HID_FULL), 16);
-            mbar_init(pp_sbar(sh, r, B::ACC2_FULL), 1);
-            mbar_init(pp_sbar(sh, r, B::ACC2_EMPTY), 4);
-        }
-        mbar_init(pp_bar(sh, B::DRAIN), 1);
-        fence_mbar_init();
-        prefetch_tensormap(tmXg_p);
-        prefetch_tensormap(tmW1_p);
-        prefetch_tensormap(tmW2_p);
-    }
-    if (!OFFS_IN_SMEM)
+    if (!READY) {
+        if (threadIdx.x == 0) pp_ffn_init_bars(sh, tmXg_p, tmW1_p, tmW2_p);
         for (int e = threadIdx.x; e <= p.E; e += kPpThreads) sh.offs[e] = SAME_LAUNCH ? __ldcg(p.offsets + e) : p.offsets[e];
-    __syncthreads();
-    if (warp == 0) pp_tile_starts(sh, p.E, lane);
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
+        __syncthreads();
+        if (warp == 0) pp_tile_starts(sh, p.E, lane);
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+    }
     const uint32_t tmem_base = sh.tmem_base;
     const int total_tiles = sh.tile_start[p.E];
     const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
@@ -432,25 +503,28 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                         if (r < wn.rows) nnext[q] = SAME_LAUNCH ? __ldcg(p.pair_gate + at) : __ldg(p.pair_gate + at);
                     }
                 }
-                if (ta < 0) continue;
-                if (warp == 0 && cur_run != loaded_run) {
-                    loaded_run = cur_run;
-                    const int set = cur_run & 1;
-                    const uint32_t n = (uint32_t)cur_run >> 1;
+                // weights of a new run (the first run's are requested in the turn before its first tile, together with
+                // that tile's list entries)
+                const int want_run = ta < 0 ? wn.run : cur_run, want_e = ta < 0 ? wn.e : cur_e;
+                if (warp == 0 && want_run != loaded_run) {
+                    loaded_run = want_run;
+                    const int set = want_run & 1;
+                    const uint32_t n = (uint32_t)want_run >> 1;
                     ok = pp_wait(pp_bar(sh, B::W_EMPTY + set), (n & 1u) ^ 1u, abort);
                     if (!ok) break;
                     if (lane == 0) {
                         mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL + set), set_tx);
                         const uint32_t w1 = sW + set * C::SET_BYTES, w2 = w1 + C::W1_SET;
                         for (int c = 0; c < npanels; ++c) {
-                            tma_load_2d(w1 + c * (kPpHC * 128), tmW1_p, 0, cur_e * p.HID + c * kPpHC, pp_bar(sh, B::W_FULL + set));
-                            tma_load_2d(w2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, cur_e * N2, pp_bar(sh, B::W_FULL + set));
+                            tma_load_2d(w1 + c * (kPpHC * 128), tmW1_p, 0, want_e * p.HID + c * kPpHC, pp_bar(sh, B::W_FULL + set));
+                            tma_load_2d(w2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, want_e * N2, pp_bar(sh, B::W_FULL + set));
                         }
                     }
                     __syncwarp();
                     last_bar = pp_bar(sh, B::W_FULL + set);
                     last_par = n & 1u;
                 }
+                if (ta < 0) continue;
                 const int ab = ta % kPpABufs;
                 ok = pp_wait(pp_bar(sh, B::A_EMPTY + ab), ((uint32_t)(ta / kPpABufs) & 1u) ^ 1u, abort);
                 if (!ok) break;
@@ -480,10 +554,20 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
         }
     } else if (warp < 20) {
         // ================= activation warps: warpgroup g, lane group lg ================================
+        // Piece j = eight hidden units of the thread's row: [32 g + 8 j, +8) for j < 4 and [128 + 32 g + 8 (j - 4),
+        // +8) for j >= 4 (F = 256 only); its four packed columns go to [32 g + 4 j, +4), which this thread has read
+        // before.  The pieces of a tile run as a software pipeline (pre of piece j + 1 and post of piece j - 1 under
+        // the tanh of piece j); the accumulator columns of piece j + 2 are requested as soon as piece j + 1 has
+        // been taken from its registers, so the load's latency runs under the tanh work as well.
+        // (Measured and left out: the same pipeline carried across tile boundaries, with GEMM-1 in two halves so
+        // that a region's lower half need not wait for the read-out of its previous tile: no faster, the row
+        // threads are bound by their own instruction stream next to the MMAs and the output warps, not by the
+        // bubbles at tile boundaries.)
         const int g = (warp - 4) >> 2;
         const int lg = warp & 3;
         const int row = lg * 32 + lane;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
+        const int np = wide ? 8 : 4;
         bool ok = true;
         int run_bias = -1;
 #pragma unroll 1
@@ -499,30 +583,33 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                 if (ti.y != run_bias) {
                     // a new run: its expert's first-layer bias as fp32 (two buffers by run parity: the other
                     // one may still be in use by warps that are behind)
-                    for (int f = g * 128 + row; f < p.HID; f += 512) sh.bias1_f32[ti.y & 1][f] = __bfloat162float(p.b1[(size_t)ti.x * p.HID + f]);
+                    for (int f = g * 128 + row; f < p.HID; f += 512) sh.bias1_f32[(ti.y & 1) * kPpMaxF + f] = __bfloat162float(p.b1[(size_t)ti.x * p.HID + f]);
                     named_barrier_sync(1, 512);
                     run_bias = ti.y;
                 }
             }
-            const float* bias = sh.bias1_f32[run_bias & 1] + 32 * g;
+            const float* bias = sh.bias1_f32 + (run_bias & 1) * kPpMaxF + 32 * g;
             const uint32_t region = tlane + r * kPpStreamCols + 32 * g;
-            // 16 hidden units per turn: units [32 g + 16 q, +16) (q = 0, 1) and [128 + 32 g + 16 (q - 2), +16)
-            // (q = 2, 3); their packed values go to columns [32 g + 8 q, +8), which this thread has read before
-            // (the next turn's accumulator columns are requested as soon as this turn's are scaled into z:
-            // the load's latency runs under the tanh work)
-            const int nq = wide ? 4 : 2;
-            uint32_t acc[16];
-            tmem_ld_x16(region, acc);
+            auto piece_col = [&](int j) -> uint32_t { return region + (j < 4 ? 8 * j : 128 + 8 * (j - 4)); };
+            auto piece_bias = [&](int j) -> const float* { return bias + (j < 4 ? 8 * j : 128 + 8 * (j - 4)); };
+            uint32_t acc[8];
+            float z[2][8], u[2][8];
+            tmem_ld_x8(piece_col(0), acc);
+            tmem_ld_wait();
+            pp_pre8<ACT>(acc, gs, piece_bias(0), has_b1, z[0], u[0]);
+            tmem_ld_x8(piece_col(1), acc);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (q >= nq) break;
-                float z[16];
-                uint32_t hid[8];
-                tmem_ld_wait();
-                pp_scale16(acc, gs, bias + (q < 2 ? 16 * q : 128 + 16 * (q - 2)), has_b1, z);
-                if (q + 1 < nq) tmem_ld_x16(region + (q + 1 < 2 ? 16 * (q + 1) : 128 + 16 * (q - 1)), acc);
-                pp_act8<ACT>(z, hid);
-                tmem_st_x8(region + 8 * q, hid);
+            for (int j = 0; j < 8; ++j) {
+                if (j >= np) break;
+                pp_tanh8<ACT>(u[j & 1]);
+                if (j + 1 < np) {
+                    tmem_ld_wait();
+                    pp_pre8<ACT>(acc, gs, piece_bias(j + 1), has_b1, z[(j + 1) & 1], u[(j + 1) & 1]);
+                    if (j + 2 < np) tmem_ld_x8(piece_col(j + 2), acc);
+                }
+                uint32_t hid[4];
+                pp_post8<ACT>(z[j & 1], u[j & 1], hid);
+                tmem_st_x4(region + 4 * j, hid);
             }
             tmem_st_wait();
             tc_fence_before_sync();
@@ -535,6 +622,8 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
         const int lg = warp & 3;
         const int row = lg * 32 + lane;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
+        const uint32_t swarp = smem_base + C::OFF_OUT + lg * 32 * C::OUT_PITCH;       // this warp's 32 staging rows
+        const uint32_t srow = swarp + lane * C::OUT_PITCH;
         bool ok = true;
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
@@ -545,39 +634,52 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             const int4 ti = sh.tile_s[ta % kPpMetaRing];       // (expert, run, rows) of the tile
             const bool live = row < ti.z;
             const int e_cur = ti.x;
-            bf16* dst = p.scatter_out + (size_t)pair_to_row(sh.pair_gate_s[ta % kPpMetaRing][row].x, p.gather_magic, p.gather_shift) * N2;
             const uint32_t acc2 = tlane + r * kPpStreamCols + C::ACC2_COL;
             constexpr float sc = kOutScale<ACT>;
-            // the whole accumulator row goes into registers (as packed bf16 pairs of 0.5 acc: half the
-            // registers) so that the region is handed back at once: its next GEMM-1 waits for this
+            // the whole accumulator row goes into registers as packed bf16 (32 columns' loads in flight at a time),
+            // so that the region is handed back early: its next GEMM-1 waits for this
             uint32_t o[N2 / 2];
 #pragma unroll
-            for (int cb = 0; cb < N2; cb += 16) {
-                uint32_t v[16];
+            for (int cb = 0; cb < N2; cb += 32) {
+                uint32_t v[32];
                 tmem_ld_x16(acc2 + cb, v);
+                if (cb + 16 < N2) tmem_ld_x16(acc2 + cb + 16, v + 16);
                 tmem_ld_wait();
-                if (p.b2) {
 #pragma unroll
-                    for (int c = 0; c < 16; c += 8) {
+                for (int c = 0; c < 32 && cb + c < N2; c += 8) {
+                    if (p.b2) {
                         float bb[8];
                         unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.b2 + (size_t)e_cur * N2 + cb + c)), bb);
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             o[(cb + c) / 2 + q] = pack_bf16x2(fmaf(__uint_as_float(v[c + 2 * q]), sc, bb[2 * q]),
                                                               fmaf(__uint_as_float(v[c + 2 * q + 1]), sc, bb[2 * q + 1]));
-                    }
-                } else {
+                    } else {
 #pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        o[cb / 2 + q] = pack_bf16x2(__uint_as_float(v[2 * q]) * sc, __uint_as_float(v[2 * q + 1]) * sc);
+                        for (int q = 0; q < 4; ++q)
+                            o[(cb + c) / 2 + q] = pack_bf16x2(__uint_as_float(v[c + 2 * q]) * sc, __uint_as_float(v[c + 2 * q + 1]) * sc);
+                    }
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
-            if (live) {
+            // The row goes into this thread's staging row; the warp then reads its 32 rows back with eight
+            // neighbouring lanes on one row, so that a warp-wide 16-byte reduction covers four whole rows of h'
+            // (4 contiguous 128-byte requests instead of 32 scattered 16-byte ones: the row-per-thread form is
+            // bound by the number of requests an SM can send, not by their bytes).
+            __syncwarp();                 // (the warp has read the previous tile's rows)
 #pragma unroll
-                for (int c = 0; c < N2; c += 8) red_add_bf16x8(dst + c, o[c / 2], o[c / 2 + 1], o[c / 2 + 2], o[c / 2 + 3]);
+            for (int c = 0; c < N2; c += 8) st_shared_v4(srow + c * 2, o[c / 2], o[c / 2 + 1], o[c / 2 + 2], o[c / 2 + 3]);
+            __syncwarp();
+            const int n_own = live ? pair_to_row(sh.pair_gate_s[ta % kPpMetaRing][row].x, p.gather_magic, p.gather_shift) : -1;
+            const int sub = lane >> 3, chunk = lane & 7;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int rl = 4 * i + sub;                                   // row of this warp's 32
+                const int n_i = __shfl_sync(0xffffffffu, n_own, rl);
+                const uint4 t = ld_shared_v4(swarp + rl * C::OUT_PITCH + chunk * 16);
+                if (n_i >= 0 && chunk < N2 / 8) red_add_bf16x8(p.scatter_out + (size_t)n_i * N2 + chunk * 8, t.x, t.y, t.z, t.w);
             }
         }
     }
@@ -610,9 +712,15 @@ struct PpRouteCfg {
     static constexpr int OFF_A = 0;
     static constexpr int OFF_W1 = kPpABufs * kPpABytes;
     static constexpr int OFF_W2 = OFF_W1 + kPpMaxHr * 128;
-    static constexpr int SMEM_BYTES = OFF_W2 + (kPpMaxHr / kPpHC) * W2_CHUNK;
+    // list dispatch by the output warps (EP <= 32): the (pair, gate, expert, rank) entries of up to LIST_GROUP tiles
+    // wait here until the group's list ranges have been reserved
+    static constexpr int LIST_GROUP = 4;
+    static constexpr int OFF_STAGE = OFF_W2 + (kPpMaxHr / kPpHC) * W2_CHUNK;
+    static constexpr int STAGE_BYTES = EP <= 32 ? LIST_GROUP * 2 * kTileM * 16 : 0;
+    static constexpr int SMEM_BYTES = OFF_STAGE + STAGE_BYTES;
     static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;
     static constexpr int HB_COLS = 128, LOGIT_COL = 384;
+    static_assert(SMEM_ALLOC <= 212 * 1024, "shared memory budget");
     static_assert(EP % 16 == 0 && EP <= 64, "expert count");
 };
 
@@ -627,9 +735,20 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
     const int npanels = p.HID / kPpHC;
     const int nhalf = p.HID / 128;            // units of work per tile
 
+    const int total_tiles = (p.n_rows + kTileM - 1) / kTileM;
+    const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
+    const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
+    const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
+    const int nunits = ntiles * nhalf;
+    const uint32_t sA = smem_base + C::OFF_A, sW1 = smem_base + C::OFF_W1, sW2 = smem_base + C::OFF_W2;
+    const int npre = min(ntiles, kPpABufs);       // row tiles requested during set-up
+
     // Barrier use in this pass (slots of "stream" 0): ACC1_FULL[3] / ACC1_EMPTY[3] / HID_FULL[3] per hidden
     // buffer; the logit accumulators use ACC2_FULL / ACC2_EMPTY of "streams" 0 and 1.
     if (threadIdx.x == 0) {
+        prefetch_tensormap(tmX_p);
+        prefetch_tensormap(tmW1_p);
+        prefetch_tensormap(tmW2_p);
         sh.abort_flag = 0;
         for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 1); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
         mbar_init(pp_bar(sh, B::W_FULL), 1);
@@ -645,36 +764,35 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
         mbar_init(pp_bar(sh, B::DRAIN), 1);
         mbar_init(pp_bar(sh, B::DRAIN + 1), 1);
         fence_mbar_init();
-        prefetch_tensormap(tmX_p);
-        prefetch_tensormap(tmW1_p);
-        prefetch_tensormap(tmW2_p);
+        // The first row tiles (all buffers are free) and the weights are requested right here, by the thread that
+        // has just initialised their barriers: the first tile comes from DRAM and is what the pass waits for.
+        for (int ta = 0; ta < npre; ++ta) {
+            mbar_arrive_expect_tx(pp_bar(sh, B::A_FULL + ta), kPpABytes);
+            tma_load_2d(sA + ta * kPpABytes, tmX_p, 0, (t_begin + ta) * kTileM, pp_bar(sh, B::A_FULL + ta));
+            if (ta == 0) {
+                mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK));
+                for (int c = 0; c < npanels; ++c) {
+                    tma_load_2d(sW1 + c * (kPpHC * 128), tmW1_p, 0, c * kPpHC, pp_bar(sh, B::W_FULL));
+                    tma_load_2d(sW2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, 0, pp_bar(sh, B::W_FULL));
+                }
+            }
+        }
     }
     for (int e = threadIdx.x; e < kMaxE; e += kPpThreads) sh.hist[e] = 0;
-    for (int i = threadIdx.x; i < p.HID; i += kPpThreads) sh.bias1_f32[0][i] = p.br1 ? __bfloat162float(p.br1[i]) : 0.0f;
+    for (int i = threadIdx.x; i < p.HID; i += kPpThreads) sh.bias1_f32[i] = p.br1 ? __bfloat162float(p.br1[i]) : 0.0f;
     for (int i = threadIdx.x; i < EP; i += kPpThreads)
         sh.bias2_f32[i] = i >= p.experts_real ? -INFINITY : (p.br2 ? __bfloat162float(p.br2[i]) : 0.0f);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = sh.tmem_base;
-    const int total_tiles = (p.n_rows + kTileM - 1) / kTileM;
-    const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
-    const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
-    const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
-    const int nunits = ntiles * nhalf;
-    const uint32_t sA = smem_base + C::OFF_A, sW1 = smem_base + C::OFF_W1, sW2 = smem_base + C::OFF_W2;
 
     if (warp == 0) {
         // ================= TMA producer ===============================================================
         if (lane == 0 && ntiles > 0) {
             bool ok = true;
-            mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK));
-            for (int c = 0; c < npanels; ++c) {
-                tma_load_2d(sW1 + c * (kPpHC * 128), tmW1_p, 0, c * kPpHC, pp_bar(sh, B::W_FULL));
-                tma_load_2d(sW2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, 0, pp_bar(sh, B::W_FULL));
-            }
-            uint32_t last_bar = pp_bar(sh, B::W_FULL), last_par = 0;
-            for (int ta = 0; ta < ntiles; ++ta) {
+            uint32_t last_bar = pp_bar(sh, B::A_FULL + npre - 1), last_par = 0;
+            for (int ta = npre; ta < ntiles; ++ta) {
                 const int ab = ta % kPpABufs;
                 if (!mbar_wait(pp_bar(sh, B::A_EMPTY + ab), ((uint32_t)(ta / kPpABufs) & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
                 mbar_arrive_expect_tx(pp_bar(sh, B::A_FULL + ab), kPpABytes);
@@ -684,6 +802,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             }
             if (!ok || *abort) {
                 volatile int never = 0;
+                mbar_wait(pp_bar(sh, B::W_FULL), 0u, &never, 10000000ull);
                 mbar_wait(last_bar, last_par, &never, 10000000ull);
             }
         }
@@ -789,7 +908,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t acol = tlane + b * C::HB_COLS;
-            const float* bias = sh.bias1_f32[0] + hf * 128 + 32 * g;
+            const float* bias = sh.bias1_f32 + hf * 128 + 32 * g;
 #pragma unroll
             for (int pc = 0; pc < 2; ++pc) {
                 // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu),
@@ -820,10 +939,17 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
         }
     } else {
         // ================= output warpgroup ===========================================================
-        // softmax + top-k of a tile's logits (ties go to the lower id), this CTA's rank of each pair
+        // softmax + top-k of a tile's logits (ties go to the lower id), then either each pair's rank among this
+        // CTA's pairs of its expert (for a ranked dispatch later) or, with lists_out, the dispatch itself: over a
+        // group of up to LIST_GROUP tiles the pairs are counted per expert in shared memory and their entries
+        // staged there; at the group's end ONE atomic per expert reserves a range of that expert's list and every
+        // row thread appends its entries (few atomics per address however large the batch is).
         const int lg = warp & 3;
         const int row = lg * 32 + lane;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + C::LOGIT_COL;
+        const bool lists = EP <= 32 && p.lists_out != nullptr;      // (more experts than 32 never take the list form)
+        int* group_base = sh.tile_start;            // (unused by this pass otherwise)
+        int4* stage = reinterpret_cast<int4*>(smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_STAGE);
         bool ok = true;
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
@@ -839,7 +965,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             __syncwarp();
             if (lane == 0) mbar_arrive(pp_sbar(sh, r, B::ACC2_EMPTY));
             const int n = (t_begin + ta) * kTileM + row;
-            if (n >= p.n_rows) continue;
+            const bool valid = n < p.n_rows;
             // one pass keeping the best two (strict comparisons in ascending id order: same picks as
             // repeated arg-max with ties to the lower id); the logits stay in v as raw bits + bias
             float b1 = -INFINITY, b2 = -INFINITY;
@@ -860,14 +986,41 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
 #pragma unroll
             for (int i = 0; i < EP; ++i) sum += ex2_approx(fmaf(__uint_as_float(v[i]), sc, -msc));
             const float inv = 1.0f / sum;
+            const float p2 = ex2_approx(fmaf(b2, sc, -msc)) * inv;
             const size_t at = (size_t)n * p.k;
-            p.topk_idx[at] = i1;
-            p.topk_p[at] = inv;
-            p.local_rank[at] = atomicAdd(&sh.hist[i1], 1);
-            if (p.k > 1) {
-                p.topk_idx[at + 1] = i2;
-                p.topk_p[at + 1] = ex2_approx(fmaf(b2, sc, -msc)) * inv;
-                p.local_rank[at + 1] = atomicAdd(&sh.hist[i2], 1);
+            int r1 = 0, r2 = 0;
+            if (valid) {
+                p.topk_idx[at] = i1;
+                p.topk_p[at] = inv;
+                r1 = atomicAdd(&sh.hist[i1], 1);
+                if (p.k > 1) {
+                    p.topk_idx[at + 1] = i2;
+                    p.topk_p[at + 1] = p2;
+                    r2 = atomicAdd(&sh.hist[i2], 1);
+                }
+                if (!lists) {
+                    p.local_rank[at] = r1;
+                    if (p.k > 1) p.local_rank[at + 1] = r2;
+                }
+            }
+            if (lists) {
+                const int gt = ta % C::LIST_GROUP;           // tile of the group
+                stage[(gt * 2 + 0) * kTileM + row] = make_int4(valid ? (int)at : -1, __float_as_int(inv), i1, r1);
+                if (p.k > 1) stage[(gt * 2 + 1) * kTileM + row] = make_int4(valid ? (int)at + 1 : -1, __float_as_int(p2), i2, r2);
+                if (gt == C::LIST_GROUP - 1 || ta == ntiles - 1) {
+                    named_barrier_sync(2, 128);              // all of the group's pairs are counted
+                    if (row < p.experts_real) {
+                        const int cnt = sh.hist[row];
+                        sh.hist[row] = 0;
+                        group_base[row] = cnt > 0 ? atomicAdd(p.list_counts + row, cnt) : 0;
+                    }
+                    named_barrier_sync(2, 128);
+                    for (int g = 0; g <= gt; ++g)
+                        for (int j = 0; j < p.k; ++j) {
+                            const int4 en = stage[(g * 2 + j) * kTileM + row];     // (this thread's own entry)
+                            if (en.x >= 0) p.lists_out[(size_t)en.z * p.list_stride + group_base[en.z] + en.w] = make_int2(en.x, en.y);
+                        }
+                }
             }
         }
     }
@@ -987,52 +1140,10 @@ __device__ __forceinline__ void pp_dispatch_body(const int32_t* topk_idx, const 
 }
 
 // =====================================================================================================
-// One-barrier form of the same dispatch (one launch, E * 8 <= k * 128 so that the lists fit in the stacked-row
-// scratch): right after its router pass a CTA reserves, with ONE atomic per expert, a range of each expert's
-// list for its pairs (base = the counter before the add) and appends them at base + local rank; after the
-// grid barrier the counters are the experts' totals.  Expert e's list starts at lists + e * list_stride.
-// `base`: shared memory, E ints.
+// One-barrier form of the dispatch (one launch, E * 8 <= k * 128 so that the lists fit in the stacked-row
+// scratch): the router's output warps fill per-expert lists themselves (pp_route_body with lists_out); after
+// the grid barrier the counters are the experts' totals.  Expert e's list starts at lists + e * list_stride.
 // =====================================================================================================
-template <int NT>
-__device__ __forceinline__ void pp_push_body(const int32_t* topk_idx, const float* topk_p, const int32_t* local_rank,
-                                             const int* hist, int32_t* counts, int chunk, int R, int E, int pairs_per_chunk,
-                                             int list_stride, int2* lists, int* base) {
-    const long long begin = (long long)chunk * pairs_per_chunk;
-    long long end = begin + pairs_per_chunk;
-    if (end > R) end = R;
-    constexpr int kPre = 4;
-    int pe[kPre], pr[kPre];
-    float pp[kPre];
-#pragma unroll
-    for (int q = 0; q < kPre; ++q) {
-        const long long i = begin + threadIdx.x + (long long)q * NT;
-        pe[q] = -1;
-        if (i < end) {
-            pe[q] = __ldcg(topk_idx + i);
-            pr[q] = __ldcg(local_rank + i);
-            pp[q] = __ldcg(topk_p + i);
-        }
-    }
-    if ((int)threadIdx.x < E) {
-        const int h = hist[threadIdx.x];
-        base[threadIdx.x] = h > 0 ? atomicAdd(counts + threadIdx.x, h) : 0;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int q = 0; q < kPre; ++q) {
-        if (pe[q] >= 0) {
-            const long long i = begin + threadIdx.x + (long long)q * NT;
-            lists[(size_t)pe[q] * list_stride + base[pe[q]] + pr[q]] = make_int2((int)i, __float_as_int(pp[q]));
-        }
-    }
-    for (long long i = begin + threadIdx.x + (long long)kPre * NT; i < end; i += NT) {
-        const int e = __ldcg(topk_idx + i);
-        const int r = __ldcg(local_rank + i);
-        const float pr2 = __ldcg(topk_p + i);
-        lists[(size_t)e * list_stride + base[e] + r] = make_int2((int)i, __float_as_int(pr2));
-    }
-}
-
 // After the barrier: the experts' row ranges from the counters (E <= 32: one warp).
 __device__ __forceinline__ void pp_offsets_from_counts(const int32_t* counts, int E, int lane, bool write_out, int32_t* assigned,
                                                        int32_t* kept, int32_t* offsets, int* offs_out) {

@@ -1,10 +1,11 @@
 // The forward of the layer (Section 3.1, Eq. 1; Section 3.4) on the pipeline of pp_body.cuh, for 64-wide slices
 // without a capacity limit: as ONE cooperative launch
 //
-//   phase 1  router     top-k ids and probabilities, each pair's rank among this CTA's pairs of its expert,
-//                       this CTA's per-expert counts, its rows of h' zeroed; then, where the per-expert lists
-//                       fit the scratch (E * 8 <= k * 128), the CTA reserves a range of each expert's list with
-//                       one atomic per expert and appends its (pair, gate) entries there
+//   phase 1  router     top-k ids and probabilities, this CTA's rows of h' zeroed, and the dispatch: where the
+//                       per-expert lists fit the scratch (E * 8 <= k * 128) the router's output warps append each
+//                       pair's (pair, gate) entry to its expert's list, reserving list ranges with one atomic per
+//                       expert and group of four tiles; otherwise they leave each pair's rank among the CTA's pairs
+//                       of its expert and the CTA's per-expert counts
 //   -- grid barrier --
 //   phase 2  experts    row ranges from the experts' totals; rows gathered from h, outputs added into h'
 //
@@ -75,31 +76,40 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         tmem_alloc(smem_u32(&sh.tmem_base), 512);
         tmem_relinquish();
     }
-    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);       // (syncs the CTA: base_s is visible after it)
+    __syncthreads();
     const unsigned long long base = base_s;
-    bool ok = sh.abort_flag == 0;
-    int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
     // successive launches alternate between two sets of counters: each launch, whichever dispatch it uses, zeroes
     // the set of the next one (nobody touches that set during this launch)
     const int parity = (int)((base / (2ull * gridDim.x)) & 1ull);
     int32_t* counts = fp.counts + parity * kMaxE;
+    PpParams rp = fp.route;
+    rp.list_counts = counts;
+    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, rp, sh, smem_raw);
+    bool ok = sh.abort_flag == 0;
+    int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
     if (blockIdx.x == 0 && (int)threadIdx.x < kMaxE) fp.counts[(parity ^ 1) * kMaxE + threadIdx.x] = 0;
     if (fp.lists) {
-        if (ok)
-            pp_push_body<kPpThreads>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, sh.hist, counts, (int)blockIdx.x,
-                                     fp.R, fp.E, fp.pairs_per_chunk, fp.ffn.list_stride, fp.pair_gate, dsm);
+        // (the router pass is over: the expert pass's barriers are set up while the CTA would wait anyway)
+        if (threadIdx.x == 0) pp_ffn_init_bars(sh, &tmXg, &tmW1, &tmW2);
         ok = pp_grid_barrier(fp.sync_word, 2ull, base + 2ull * gridDim.x, sh) && ok;
-        if (ok && warp == 0)
+        if (ok && warp == 0) {
             pp_offsets_from_counts(counts, fp.E, (int)(threadIdx.x & 31), blockIdx.x == 0, fp.assigned, fp.kept, fp.offsets, sh.offs);
-        __syncthreads();
+            __syncwarp();
+            pp_tile_starts(sh, fp.E, (int)(threadIdx.x & 31));
+        }
     } else {
         ok = pp_grid_barrier(fp.sync_word, 1ull, base + gridDim.x, sh) && ok;
         if (ok)
             pp_dispatch_body<kPpThreads, true>(fp.route.topk_idx, fp.route.topk_p, fp.route.local_rank, fp.route.cta_hist,
                                                (int)gridDim.x, (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.assigned,
                                                fp.kept, fp.offsets, fp.dest, fp.pair_gate, dsm, sh.offs);
+        if (threadIdx.x == 0) pp_ffn_init_bars(sh, &tmXg, &tmW1, &tmW2);
         ok = pp_grid_barrier(fp.sync_word, 1ull, base + 2ull * gridDim.x, sh) && ok;
+        if (ok && warp == 0) pp_tile_starts(sh, fp.E, (int)(threadIdx.x & 31));
     }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
     if (ok) pp_ffn_body<N2, ACT, true, true>(&tmXg, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
     if (threadIdx.x == 0 && !ok) atomicExch(fp.ffn.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
     __syncthreads();
@@ -352,6 +362,11 @@ int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, v
     // the per-expert lists (E * N entries of 8 bytes) must fit in the stacked-row scratch (N * k rows of 128 bytes)
     fp.lists = (one_launch && D.E * 8 <= D.k * 128) ? 1 : 0;
     fp.ffn.list_stride = fp.lists ? D.N : 0;
+    if (fp.lists) {          // the router's output warps fill the lists themselves (the counter set is chosen in the kernel)
+        fp.route.lists_out = fp.pair_gate;
+        fp.route.list_stride = D.N;
+        fp.route.cta_hist = nullptr;
+    }
     switch (D.E) {
         case 8:
         case 16: return pp_launch_act<16, 64>(D, w, h, fp, st, one_launch, events);

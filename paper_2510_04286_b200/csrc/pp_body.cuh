@@ -592,24 +592,24 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             const uint32_t region = tlane + r * kPpStreamCols + 32 * g;
             auto piece_col = [&](int j) -> uint32_t { return region + (j < 4 ? 8 * j : 128 + 8 * (j - 4)); };
             auto piece_bias = [&](int j) -> const float* { return bias + (j < 4 ? 8 * j : 128 + 8 * (j - 4)); };
-            uint32_t acc[8];
+            // (two pieces per tensor-memory load and per store: every such instruction passes through the same
+            // queue as the other warps' loads and stores)
+            uint32_t acc[16], hid[8];
             float z[2][8], u[2][8];
-            tmem_ld_x8(piece_col(0), acc);
+            tmem_ld_x16(piece_col(0), acc);
             tmem_ld_wait();
             pp_pre8<ACT>(acc, gs, piece_bias(0), has_b1, z[0], u[0]);
-            tmem_ld_x8(piece_col(1), acc);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 if (j >= np) break;
                 pp_tanh8<ACT>(u[j & 1]);
                 if (j + 1 < np) {
-                    tmem_ld_wait();
-                    pp_pre8<ACT>(acc, gs, piece_bias(j + 1), has_b1, z[(j + 1) & 1], u[(j + 1) & 1]);
-                    if (j + 2 < np) tmem_ld_x8(piece_col(j + 2), acc);
+                    if (((j + 1) & 1) == 0) tmem_ld_wait();
+                    pp_pre8<ACT>(acc + 8 * ((j + 1) & 1), gs, piece_bias(j + 1), has_b1, z[(j + 1) & 1], u[(j + 1) & 1]);
+                    if (((j + 1) & 1) == 1 && j + 2 < np) tmem_ld_x16(piece_col(j + 2), acc);
                 }
-                uint32_t hid[4];
-                pp_post8<ACT>(z[j & 1], u[j & 1], hid);
-                tmem_st_x4(region + 4 * j, hid);
+                pp_post8<ACT>(z[j & 1], u[j & 1], hid + 4 * (j & 1));
+                if (j & 1) tmem_st_x8(region + 4 * (j - 1), hid);
             }
             tmem_st_wait();
             tc_fence_before_sync();
@@ -642,8 +642,8 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
 #pragma unroll
             for (int cb = 0; cb < N2; cb += 32) {
                 uint32_t v[32];
-                tmem_ld_x16(acc2 + cb, v);
-                if (cb + 16 < N2) tmem_ld_x16(acc2 + cb + 16, v + 16);
+                if (cb + 16 < N2) tmem_ld_x32(acc2 + cb, v);
+                else tmem_ld_x16(acc2 + cb, v);
                 tmem_ld_wait();
 #pragma unroll
                 for (int c = 0; c < 32 && cb + c < N2; c += 8) {
@@ -899,6 +899,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
         const int g = (warp - 4) >> 2;
         const int lg = warp & 3;
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + 32 * g;
+        const bool has_br1 = p.br1 != nullptr;
         bool ok = true;
 #pragma unroll 1
         for (int u = 0; u < nunits && ok; ++u) {
@@ -909,20 +910,26 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             tc_fence_after_sync();
             const uint32_t acol = tlane + b * C::HB_COLS;
             const float* bias = sh.bias1_f32 + hf * 128 + 32 * g;
+            // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu), lo = the
+            // rounded remainder (for a negative value the remainder is the value itself and its .relu is 0 as
+            // well).  The thread's 32 columns come with one tensor-memory load.
+            uint32_t acc32[32];
+            tmem_ld_x32(acol, acc32);
+            tmem_ld_wait();
 #pragma unroll
             for (int pc = 0; pc < 2; ++pc) {
-                // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu),
-                // lo = the rounded remainder (for a negative value the remainder is the value itself and
-                // its .relu is 0 as well)
-                uint32_t acc[16];
-                tmem_ld_x16(acol + 16 * pc, acc);
-                tmem_ld_wait();
+                const uint32_t* acc = acc32 + 16 * pc;
                 float a[16];
+                if (has_br1) {
 #pragma unroll
-                for (int i = 0; i < 16; i += 4) {
-                    const float4 bb = *reinterpret_cast<const float4*>(bias + pc * 16 + i);
-                    add2(a[i], a[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), bb.x, bb.y);
-                    add2(a[i + 2], a[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), bb.z, bb.w);
+                    for (int i = 0; i < 16; i += 4) {
+                        const float4 bb = *reinterpret_cast<const float4*>(bias + pc * 16 + i);
+                        add2(a[i], a[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), bb.x, bb.y);
+                        add2(a[i + 2], a[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), bb.z, bb.w);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) a[i] = __uint_as_float(acc[i]);
                 }
                 uint32_t hl[16];
 #pragma unroll
@@ -990,13 +997,15 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             const size_t at = (size_t)n * p.k;
             int r1 = 0, r2 = 0;
             if (valid) {
-                p.topk_idx[at] = i1;
-                p.topk_p[at] = inv;
                 r1 = atomicAdd(&sh.hist[i1], 1);
                 if (p.k > 1) {
-                    p.topk_idx[at + 1] = i2;
-                    p.topk_p[at + 1] = p2;
+                    // (k = 2: a row's two ids and its two probabilities as one 8-byte store each)
+                    *reinterpret_cast<int2*>(p.topk_idx + at) = make_int2(i1, i2);
+                    *reinterpret_cast<float2*>(p.topk_p + at) = make_float2(inv, p2);
                     r2 = atomicAdd(&sh.hist[i2], 1);
+                } else {
+                    p.topk_idx[at] = i1;
+                    p.topk_p[at] = inv;
                 }
                 if (!lists) {
                     p.local_rank[at] = r1;

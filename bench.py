@@ -30,12 +30,15 @@ if ROOT not in sys.path:
 L2_BYTES = 126e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of one ncu capture per kernel, with the summary that
-# holds it.  A workload of the same slice width, k and expert width scales the figure by the rows one launch
-# processes (traffic is proportional to rows: each row is read once per chosen expert and its output row is
-# zero-filled and added to k times).  A kernel changed since its capture has no entry: traffic is then null.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the timed kernel, with the summary
+# that holds them.  Not scaled between workloads: whether the expert pass's gathers and reductions hit L2 depends
+# on the batch (cfg1's 16.8 MB of tokens stay in L2 and h' is still there when the kernel ends; cfg2's 134 MB do
+# not).  A workload without a capture of its own reports traffic = null.
 NCU_TRAFFIC = {
-    # kernel: (bytes per launch, rows of that launch, ds, k, F, summary)
+    # (kernel, N, ds, k, F): (bytes per launch, summary)
+    ("forward_one_launch", 16384 * 8, 64, 2, 256): (17.9745e6 + 0.04e6, "profiles/pp_forward_kernel_cfg1_cfg2.md (ncu, cfg1)"),
+    ("forward_one_launch", 65536 * 16, 64, 2, 256): (613.103e6 + 342.652e6, "profiles/pp_forward_kernel_cfg1_cfg2.md (ncu, cfg2)"),
+    ("forward_one_launch", 128 * 32, 128, 2, 512): (17.868e6, "profiles/decode_forward_kernel_cfg4.md (ncu, cfg4)"),
 }
 OTHER_CONFIGS = ("cfg2", "cfg3", "cfg3b", "cfg4")
 # dram__bytes_read + dram__bytes_write of the two backward kernels on cfg1 (profiles/backward_cfg1.md)
@@ -44,11 +47,9 @@ NCU_TRAFFIC_ROWS_CFG1 = 16384 * 8
 
 
 def ncu_traffic(kernel, lc):
-    """(DRAM bytes per launch scaled to this workload, where the figure comes from) or (None, None)."""
-    ent = NCU_TRAFFIC.get(kernel)
-    if ent is None or (lc.ds, lc.k, lc.F) != ent[2:5]:
-        return None, None
-    return ent[0] * lc.N / ent[1], ent[5]
+    """(DRAM bytes per launch of this workload's own capture, where the figure comes from) or (None, None)."""
+    ent = NCU_TRAFFIC.get((kernel, lc.N, lc.ds, lc.k, lc.F))
+    return ent if ent is not None else (None, None)
 
 
 # tanh.approx results per clock per SM (measured, profiles/microbenchmarks_b200.md): the GELU(tanh) experts

@@ -49,14 +49,20 @@ def test_single_rank_helpers():
     w = bench.layer_work(synth.CONFIGS["cfg1"], kept_rows=262144, touched_experts=16)
     assert abs(w["total_flops"] - 22.55e9) < 0.01e9          # router 5.37 G + experts 17.18 G
     assert abs(w["compulsory_bytes"] - 34.7e6) < 0.1e6
-    # a profiled figure scales by rows to a workload of the same slice width, k and F; any other has none
-    bench.NCU_TRAFFIC["probe"] = (800e6, 65536 * 16, 64, 2, 256, "a summary")
+    # a workload reports the DRAM traffic of its own ncu capture only (nothing is scaled from another batch size);
+    # absent biases are not compulsory bytes
+    cfg1, cfg2 = synth.CONFIGS["cfg1"], synth.CONFIGS["cfg2"]
+    key = ("probe", cfg1.N, cfg1.ds, cfg1.k, cfg1.F)
+    bench.NCU_TRAFFIC[key] = (100e6, "a summary")
     try:
-        assert bench.ncu_traffic("probe", synth.CONFIGS["cfg1"]) == (pytest.approx(100e6), "a summary")
-        assert bench.ncu_traffic("probe", synth.CONFIGS["cfg3"]) == (None, None)
-        assert bench.ncu_traffic("no such kernel", synth.CONFIGS["cfg1"]) == (None, None)
+        assert bench.ncu_traffic("probe", cfg1) == (100e6, "a summary")
+        assert bench.ncu_traffic("probe", cfg2) == (None, None)
+        assert bench.ncu_traffic("no such kernel", cfg1) == (None, None)
     finally:
-        del bench.NCU_TRAFFIC["probe"]
+        del bench.NCU_TRAFFIC[key]
+    no_bias = {"Wr1": 1, "Wr2": 1, "W1": 1, "W2": 1, "br1": None, "br2": None, "b1": None, "b2": None}
+    w0 = bench.layer_work(cfg1, kept_rows=262144, touched_experts=16, w=no_bias)
+    assert w["compulsory_bytes"] - w0["compulsory_bytes"] == 2 * (256 + 16 + 16 * (256 + 64))
     r = bench.roofline_of(synth.CONFIGS["cfg1"], w, {"bf16_tflops": 1000.0, "hbm_gbs": 1000.0}, 1e-4)
     assert r["bound"] == "hbm" and r["frac"] == pytest.approx(w["compulsory_bytes"] / 1e12 / 1e-4)
     s = bench.ClockSampler("0")

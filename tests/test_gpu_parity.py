@@ -422,3 +422,25 @@ def test_forward_paper_model_shape():
 def test_forward_full_cfg2_sampled_rows():
     rep = pu.check_forward_against_oracle(C["cfg2"], sample_rows=65536)
     print("cfg2", rep)
+
+
+@pytest.mark.parametrize("T,E,k,init", [
+    (9485, 16, 2, "normal"),     # 593 router tiles: five per CTA (list groups of 4 + 1), ragged last tile, ragged expert tiles
+    (1200, 8, 1, "normal"),      # 75 tiles: one per CTA, half of the CTAs idle; E = 8 on the 16-wide router, k = 1
+    (21312, 32, 2, "normal"),    # nine tiles per CTA (groups of 4 + 4 + 1), E = 32: the largest expert count with lists
+    (4100, 16, 2, "kaiming"),    # real biases on all four Linears through the bias paths of both passes
+])
+def test_forward_64wide_list_dispatch_shapes(T, E, k, init):
+    """The one-launch forward of 64-wide slices, whose router fills the per-expert lists in groups of tiles:
+    group boundaries, CTAs without tiles, ragged tails and both bias paths against the oracle (routing and counts
+    on every row, outputs on sampled rows)."""
+    import torch
+    lc = dataclasses.replace(C["cfg1"], name=f"w64_T{T}_E{E}_k{k}_{init}", T=T, E=E, k=k, init=init)
+    rep = pu.check_forward_against_oracle(lc, sample_rows=8192, one_ulp_of_element=(init == "kaiming"))
+    print(lc.name, rep)
+    h_np, w_np = synth.make_layer_inputs(lc)
+    gpu = pu.GpuLayer(lc, h_np, w_np)
+    before = binding.slicemoe_launch_count()
+    gpu.forward()
+    torch.cuda.synchronize()
+    assert binding.slicemoe_launch_count() - before == 1          # the single-kernel path

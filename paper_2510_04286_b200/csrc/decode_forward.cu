@@ -31,6 +31,9 @@ constexpr int kDecThreads = 320;          // warps 0-7 workers, warp 8 weight lo
 constexpr int kDecWorkers = 256;
 constexpr int kDecDs = 128, kDecF = 512, kDecHC = 128, kDecNC = kDecF / kDecHC, kDecHr = 256;
 constexpr int kDecMaxE = 64;
+// The per-expert list counters sit one per 128-byte line: the router CTAs' warps append at about the same time
+// (thousands of atomics within a microsecond or two), and atomics on one line are served one after the other.
+constexpr int kDecCountStride = 32;       // ints between two experts' counters
 constexpr int kDecMaxItems = 16;          // items one CTA can take in one launch (N <= 4096: at most 96 tiles in all)
 
 // shared memory (from a 1024-byte aligned base)
@@ -47,7 +50,7 @@ struct DecParams {
     float* topk_p;
     int32_t *assigned, *kept;
     int2* lists;              // [E][N] (pair index, gate bits), in arrival order
-    int32_t* counts;          // [2][kDecMaxE] device words, used alternately by successive launches
+    int32_t* counts;          // [2][kDecMaxE] device words (kDecCountStride ints apart), used alternately by successive launches
     int32_t* status;
     unsigned long long* sync_word;
     int N, k, E, n_router;     // n_router: the last ceil(N / 128) CTAs route
@@ -78,7 +81,7 @@ enum { W1_FULL = 0, W2_FULL = 2, W1_EMPTY = 4, W2_EMPTY = 6, A_FULL = 8, A_EMPTY
 }
 
 __device__ unsigned long long g_dec_sync;
-__device__ int32_t g_dec_counts[2 * kDecMaxE];
+__device__ int32_t g_dec_counts[2 * kDecMaxE * kDecCountStride];
 
 // Grid barrier on ONE monotonic 64-bit arrival counter: every launch adds gridDim.x to it, so the count a CTA
 // finds at entry, rounded down to a multiple of gridDim.x, is this launch's base whichever CTAs have already
@@ -263,7 +266,7 @@ __device__ __forceinline__ void dec_route(const CUtensorMap* tmX, const CUtensor
                 m[j] = __match_any_sync(0xffffffffu, e[j]);
                 leader[j] = __ffs(m[j]) - 1;
                 base[j] = 0;
-                if (e[j] >= 0 && lane == leader[j]) base[j] = atomicAdd(counts + e[j], __popc(m[j]));
+                if (e[j] >= 0 && lane == leader[j]) base[j] = atomicAdd(counts + e[j] * kDecCountStride, __popc(m[j]));
             }
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
@@ -405,7 +408,7 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const unsigned long long base = sh.base;
     // successive launches alternate between two sets of counters: this one's were zeroed by the previous launch
     const int parity = (int)((base / gridDim.x) & 1ull);
-    int32_t* counts = p.counts + parity * kDecMaxE;
+    int32_t* counts = p.counts + parity * (kDecMaxE * kDecCountStride);
 
     // weights of chunk c of expert e into ring slot s (W1: rows [128 c, +128) of W1_e; W2: columns [128 c, +128) of W2_e)
     auto load_w1 = [&](int e, int c, int s) {
@@ -421,8 +424,8 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
 
     if (warp == 8 && blockIdx.x == 0) {
         // (nobody uses the other counter set during this launch)
-        int32_t* other = p.counts + (parity ^ 1) * kDecMaxE;
-        for (int i = lane; i < kDecMaxE; i += 32) other[i] = 0;
+        int32_t* other = p.counts + (parity ^ 1) * (kDecMaxE * kDecCountStride);
+        for (int i = lane; i < kDecMaxE; i += 32) other[i * kDecCountStride] = 0;
     }
     if (warp == 8 && lane == 0) {
         prefetch_tensormap(&tmW1);
@@ -450,7 +453,7 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     bool ok = dec_grid_barrier(p.sync_word, base, sh);
 
     // ---- schedule ----------------------------------------------------------------------------------------
-    if (ok && threadIdx.x < E) sh.cnt[threadIdx.x] = __ldcg(counts + threadIdx.x);
+    if (ok && threadIdx.x < E) sh.cnt[threadIdx.x] = __ldcg(counts + threadIdx.x * kDecCountStride);
     __syncthreads();
     if (ok && warp == 0) dec_schedule<E>(sh, lane);
     if (ok && blockIdx.x == 0 && threadIdx.x >= 64 && threadIdx.x < 64 + E) {
@@ -786,7 +789,7 @@ int decode_forward_reset_sync(cudaStream_t st) {
     int rc = dec_device_words(&words, &counts);
     if (rc) return rc;
     SLICEMOE_CUDA_TRY(cudaMemsetAsync(words, 0, sizeof(unsigned long long), st));
-    SLICEMOE_CUDA_TRY(cudaMemsetAsync(counts, 0, 2 * kDecMaxE * sizeof(int32_t), st));
+    SLICEMOE_CUDA_TRY(cudaMemsetAsync(counts, 0, 2 * kDecMaxE * kDecCountStride * sizeof(int32_t), st));
     SLICEMOE_CUDA_TRY(cudaStreamSynchronize(st));
     return SLICEMOE_OK;
 }

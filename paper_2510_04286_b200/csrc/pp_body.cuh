@@ -46,6 +46,10 @@ constexpr int kPpHC = 64;                // hidden units per chunk
 constexpr int kPpMaxF = 256;             // expert hidden width (both weight sets stay in shared memory)
 constexpr int kPpMaxHr = 512;            // router hidden width
 constexpr int kPpStreamCols = 256;       // TMEM columns per stream
+// The per-expert list counters sit one per 128-byte line: all CTAs reserve at about the same times, and
+// atomics on one line are served one after the other by one L2 slice (16 counters in one line cost every flush
+// of the router's lists about 2 k cycles).
+constexpr int kPpCountStride = 32;       // ints between two experts' counters
 
 // ---- tanh unit ------------------------------------------------------------------------------------
 __device__ __forceinline__ float tanh_approx(float x) {
@@ -85,6 +89,7 @@ struct PpShared {
     int hist[kMaxE];
     uint32_t tmem_base;
     int abort_flag;
+    int counts_set;             // which of the two sets of list counters this launch uses (written at kernel entry)
     // experts: first-layer bias of the run each stream is in, as fp32; router: br1 / br2 as fp32
     // (experts: two halves of kPpMaxF, by run parity; router: one array of up to kPpMaxHr)
     __align__(16) float bias1_f32[kPpMaxHr];
@@ -146,7 +151,8 @@ struct PpParams {
     int32_t* cta_hist;          // [grid, E]
     bf16* zero_out;             // h' as [N, 64]: this CTA zeroes the rows it routes (or nullptr)
     int2* lists_out;            // per-expert lists of (pair index, gate) filled by the router itself (or nullptr): expert e's
-    int32_t* list_counts;       // list starts at lists_out + e * list_stride and holds list_counts[e] entries
+    int32_t* list_counts;       // list starts at lists_out + e * list_stride; its length is counter e (one per kPpCountStride
+                                // ints) of set sh.counts_set (sets are kMaxE * kPpCountStride ints apart)
     // ---- experts
     int E;
     const int32_t* offsets;     // [E + 1] (read when the offsets are not already in shared memory)
@@ -387,6 +393,18 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             PpWalk w1;
             w1.init();
             int run1 = -1;
+            // The first run's weights are requested here, by the warp that waits for them: the gather warps
+            // are busy with the first tiles' lists and rows, and issuing a set's eight copies takes a thread
+            // about a thousand cycles.
+            w1.advance(sh, t_begin, 0);
+            if (lane == 0) {
+                mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK));
+                for (int c = 0; c < npanels; ++c) {
+                    tma_load_2d(sW + c * (kPpHC * 128), tmW1_p, 0, w1.e * p.HID + c * kPpHC, pp_bar(sh, B::W_FULL));
+                    tma_load_2d(sW + C::W1_SET + c * C::W2_CHUNK, tmW2_p, c * kPpHC, w1.e * N2, pp_bar(sh, B::W_FULL));
+                }
+            }
+            __syncwarp();
 #pragma unroll 1
             for (int ta = 0; ta < ntiles && ok; ++ta) {
                 const int ab = ta % kPpABufs, r = ta & 1;
@@ -415,6 +433,7 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                 if (lane == 0) {
                     mma_commit(pp_bar(sh, B::DRAIN));
                     mbar_wait(pp_bar(sh, B::DRAIN), 0u, &never, 10000000ull);
+                    mbar_wait(pp_bar(sh, B::W_FULL), 0u, &never, 10000000ull);     // (the copies this warp requested)
                 }
                 __syncwarp();
             }
@@ -479,7 +498,7 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             int2 nnext[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) nnext[q] = make_int2(-1, 0);
-            int loaded_run = -1, cur_e = 0, cur_run = 0, cur_rows = 0;
+            int loaded_run = 0, cur_e = 0, cur_run = 0, cur_rows = 0;      // (run 0's weights: the GEMM-1 warp)
             uint32_t last_bar = 0, last_par = 0;
             bool ok = true;
             const uint32_t set_tx = (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK);
@@ -503,9 +522,9 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                         if (r < wn.rows) nnext[q] = SAME_LAUNCH ? __ldcg(p.pair_gate + at) : __ldg(p.pair_gate + at);
                     }
                 }
-                // weights of a new run (the first run's are requested in the turn before its first tile, together with
-                // that tile's list entries)
-                const int want_run = ta < 0 ? wn.run : cur_run, want_e = ta < 0 ? wn.e : cur_e;
+                if (ta < 0) continue;
+                // weights of a new run
+                const int want_run = cur_run, want_e = cur_e;
                 if (warp == 0 && want_run != loaded_run) {
                     loaded_run = want_run;
                     const int set = want_run & 1;
@@ -524,7 +543,6 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     last_bar = pp_bar(sh, B::W_FULL + set);
                     last_par = n & 1u;
                 }
-                if (ta < 0) continue;
                 const int ab = ta % kPpABufs;
                 ok = pp_wait(pp_bar(sh, B::A_EMPTY + ab), ((uint32_t)(ta / kPpABufs) & 1u) ^ 1u, abort);
                 if (!ok) break;
@@ -747,11 +765,8 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
     // buffer; the logit accumulators use ACC2_FULL / ACC2_EMPTY of "streams" 0 and 1.
     if (threadIdx.x == 0) {
         prefetch_tensormap(tmX_p);
-        prefetch_tensormap(tmW1_p);
-        prefetch_tensormap(tmW2_p);
         sh.abort_flag = 0;
         for (int i = 0; i < kPpABufs; ++i) { mbar_init(pp_bar(sh, B::A_FULL + i), 1); mbar_init(pp_bar(sh, B::A_EMPTY + i), 1); }
-        mbar_init(pp_bar(sh, B::W_FULL), 1);
         for (int i = 0; i < 3; ++i) {
             mbar_init(pp_sbar(sh, 0, B::ACC1_FULL + i), 1);
             mbar_init(pp_sbar(sh, 0, B::ACC1_EMPTY + i), 1);
@@ -764,17 +779,24 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
         mbar_init(pp_bar(sh, B::DRAIN), 1);
         mbar_init(pp_bar(sh, B::DRAIN + 1), 1);
         fence_mbar_init();
-        // The first row tiles (all buffers are free) and the weights are requested right here, by the thread that
-        // has just initialised their barriers: the first tile comes from DRAM and is what the pass waits for.
+        // The first row tiles (all buffers are free) are requested right here, by the thread that has just
+        // initialised their barriers: the first tile comes from DRAM and is what the pass waits for.  (The
+        // weights are requested by another warp at the same time: issuing a dozen copies takes one thread
+        // more than a thousand cycles.)
         for (int ta = 0; ta < npre; ++ta) {
             mbar_arrive_expect_tx(pp_bar(sh, B::A_FULL + ta), kPpABytes);
             tma_load_2d(sA + ta * kPpABytes, tmX_p, 0, (t_begin + ta) * kTileM, pp_bar(sh, B::A_FULL + ta));
-            if (ta == 0) {
-                mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK));
-                for (int c = 0; c < npanels; ++c) {
-                    tma_load_2d(sW1 + c * (kPpHC * 128), tmW1_p, 0, c * kPpHC, pp_bar(sh, B::W_FULL));
-                    tma_load_2d(sW2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, 0, pp_bar(sh, B::W_FULL));
-                }
+        }
+    } else if (threadIdx.x == 64) {
+        prefetch_tensormap(tmW1_p);
+        prefetch_tensormap(tmW2_p);
+        mbar_init(pp_bar(sh, B::W_FULL), 1);
+        fence_mbar_init();
+        if (ntiles > 0) {
+            mbar_arrive_expect_tx(pp_bar(sh, B::W_FULL), (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK));
+            for (int c = 0; c < npanels; ++c) {
+                tma_load_2d(sW1 + c * (kPpHC * 128), tmW1_p, 0, c * kPpHC, pp_bar(sh, B::W_FULL));
+                tma_load_2d(sW2 + c * C::W2_CHUNK, tmW2_p, c * kPpHC, 0, pp_bar(sh, B::W_FULL));
             }
         }
     }
@@ -956,6 +978,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
         const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + C::LOGIT_COL;
         const bool lists = EP <= 32 && p.lists_out != nullptr;      // (more experts than 32 never take the list form)
         int* group_base = sh.tile_start;            // (unused by this pass otherwise)
+        int32_t* counts = lists ? p.list_counts + sh.counts_set * (kMaxE * kPpCountStride) : nullptr;
         int4* stage = reinterpret_cast<int4*>(smem_raw + (smem_base - smem_u32(smem_raw)) + C::OFF_STAGE);
         bool ok = true;
 #pragma unroll 1
@@ -1021,7 +1044,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
                     if (row < p.experts_real) {
                         const int cnt = sh.hist[row];
                         sh.hist[row] = 0;
-                        group_base[row] = cnt > 0 ? atomicAdd(p.list_counts + row, cnt) : 0;
+                        group_base[row] = cnt > 0 ? atomicAdd(counts + row * kPpCountStride, cnt) : 0;
                     }
                     named_barrier_sync(2, 128);
                     for (int g = 0; g <= gt; ++g)
@@ -1156,7 +1179,7 @@ __device__ __forceinline__ void pp_dispatch_body(const int32_t* topk_idx, const 
 // After the barrier: the experts' row ranges from the counters (E <= 32: one warp).
 __device__ __forceinline__ void pp_offsets_from_counts(const int32_t* counts, int E, int lane, bool write_out, int32_t* assigned,
                                                        int32_t* kept, int32_t* offsets, int* offs_out) {
-    const int cnt = lane < E ? __ldcg(counts + lane) : 0;
+    const int cnt = lane < E ? __ldcg(counts + lane * kPpCountStride) : 0;
     int incl = cnt;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {

@@ -24,7 +24,7 @@ struct PpFusedParams {
     int32_t *assigned, *kept, *offsets, *dest;
     int2* pair_gate;
     unsigned long long* sync_word;
-    int32_t* counts;          // [2][kMaxE] per-expert counters of the one-barrier dispatch, used alternately by successive launches
+    int32_t* counts;          // [2][kMaxE] per-expert counters (kPpCountStride ints apart) of the one-barrier dispatch, used alternately by successive launches
     int lists;                // 1: one-barrier dispatch (per-expert lists), 0: ranked dispatch between two barriers
     int clear_status;
 };
@@ -34,7 +34,7 @@ struct PpFusedParams {
 // down to a multiple of that, is the launch's base whichever CTAs have already arrived; the barriers wait for
 // base + gridDim.x and base + 2 * gridDim.x.  One release-add and acquire polls each: no last-arriver step.
 __device__ unsigned long long g_pp_sync;
-__device__ int32_t g_pp_counts[2 * kMaxE];
+__device__ int32_t g_pp_counts[2 * kMaxE * kPpCountStride];
 
 __device__ __forceinline__ bool pp_grid_barrier(unsigned long long* word, unsigned long long inc, unsigned long long target, PpShared& sh) {
     fence_proxy_async_smem();     // the phases reuse shared memory through different proxies
@@ -66,28 +66,27 @@ pp_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     __shared__ PpShared sh;
     const int warp = threadIdx.x >> 5;
     __shared__ unsigned long long base_s;
-    if (threadIdx.x == 0) {
+    // (not thread 0: that one requests the first row tiles at once and must not wait for this load)
+    if (threadIdx.x == 96) {
         unsigned long long v;
         asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fp.sync_word) : "memory");
         base_s = v - v % (2ull * gridDim.x);
+        // successive launches alternate between two sets of list counters: each launch zeroes the set of the
+        // next one (nobody touches that set during this launch)
+        sh.counts_set = (int)((base_s / (2ull * gridDim.x)) & 1ull);
         if (blockIdx.x == 0 && fp.clear_status) *fp.ffn.status = SLICEMOE_OK;
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh.tmem_base), 512);
         tmem_relinquish();
     }
-    __syncthreads();
+    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);       // (syncs the CTA: base_s and counts_set are visible in and after it)
     const unsigned long long base = base_s;
-    // successive launches alternate between two sets of counters: each launch, whichever dispatch it uses, zeroes
-    // the set of the next one (nobody touches that set during this launch)
-    const int parity = (int)((base / (2ull * gridDim.x)) & 1ull);
-    int32_t* counts = fp.counts + parity * kMaxE;
-    PpParams rp = fp.route;
-    rp.list_counts = counts;
-    pp_route_body<EP>(&tmX, &tmWr1, &tmWr2, rp, sh, smem_raw);
+    const int parity = sh.counts_set;
+    int32_t* counts = fp.counts + parity * (kMaxE * kPpCountStride);
     bool ok = sh.abort_flag == 0;
     int* dsm = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 15) & ~uintptr_t(15));
-    if (blockIdx.x == 0 && (int)threadIdx.x < kMaxE) fp.counts[(parity ^ 1) * kMaxE + threadIdx.x] = 0;
+    if (blockIdx.x == 0 && (int)threadIdx.x < kMaxE) fp.counts[((parity ^ 1) * kMaxE + threadIdx.x) * kPpCountStride] = 0;
     if (fp.lists) {
         // (the router pass is over: the expert pass's barriers are set up while the CTA would wait anyway)
         if (threadIdx.x == 0) pp_ffn_init_bars(sh, &tmXg, &tmW1, &tmW2);
@@ -329,7 +328,7 @@ int pp_forward_reset_sync(cudaStream_t st) {
     int rc = pp_sync_address(&words, &counts);
     if (rc) return rc;
     SLICEMOE_CUDA_TRY(cudaMemsetAsync(words, 0, sizeof(unsigned long long), st));
-    SLICEMOE_CUDA_TRY(cudaMemsetAsync(counts, 0, 2 * kMaxE * sizeof(int32_t), st));
+    SLICEMOE_CUDA_TRY(cudaMemsetAsync(counts, 0, 2 * kMaxE * kPpCountStride * sizeof(int32_t), st));
     SLICEMOE_CUDA_TRY(cudaStreamSynchronize(st));
     return SLICEMOE_OK;
 }
@@ -364,6 +363,7 @@ int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, v
     fp.ffn.list_stride = fp.lists ? D.N : 0;
     if (fp.lists) {          // the router's output warps fill the lists themselves (the counter set is chosen in the kernel)
         fp.route.lists_out = fp.pair_gate;
+        fp.route.list_counts = fp.counts;
         fp.route.list_stride = D.N;
         fp.route.cta_hist = nullptr;
     }

@@ -531,7 +531,8 @@ def run_ours(args, lc):
     others = {}
     if world == 1 and not args.no_other_configs:
         # the other single-GPU workloads, a few steps each (same protocol, fewer replays)
-        del wl, hs, outs, w, ws
+        w = {n: (None if t is None else True) for n, t in w.items()}      # (which tensors were passed: used below)
+        del wl, hs, outs, ws
         for name in OTHER_CONFIGS:
             if name == lc.name:
                 continue

@@ -83,6 +83,16 @@ typedef struct {
     float noise_sigma;   /* std of the Gaussian noise added to the logits before the
                           * softmax (Figure 6); 0 = none */
     uint64_t noise_seed; /* key of the counter-based noise generator (slicemoe_route) */
+    /* Train mode of the slicemoe_forward* calls (Section 3.3, cross-slice dropout; Appendix A uses
+     * rate 0.2).  train_gates = 0: Eq. 1's gates are the router's probabilities.  train_gates = 1:
+     * each of a row's k assignments is dropped with probability dropout_rate, the survivors'
+     * probabilities are divided by their sum, and if none survives the top-1 assignment gets weight 1
+     * (slicemoe_gate_dropout's rule and generator with seed = dropout_seed, applied between the
+     * router and the dispatch); topk_p_opt then returns those gates.  dropout_rate outside [0, 1]:
+     * SLICEMOE_ERR_SHAPE.  The staged calls ignore these fields. */
+    int32_t train_gates;
+    float dropout_rate;
+    uint64_t dropout_seed;
 } slicemoe_config;
 
 /* Caller-owned weights, dtype = cfg->dtype. */

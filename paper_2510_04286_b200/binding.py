@@ -41,7 +41,8 @@ class _Config(ctypes.Structure):
                 ("E", ctypes.c_int32), ("k", ctypes.c_int32), ("Hr", ctypes.c_int32),
                 ("F", ctypes.c_int32), ("dtype", ctypes.c_int32), ("act", ctypes.c_int32),
                 ("capacity", ctypes.c_int64), ("temperature", ctypes.c_float),
-                ("noise_sigma", ctypes.c_float), ("noise_seed", ctypes.c_uint64)]
+                ("noise_sigma", ctypes.c_float), ("noise_seed", ctypes.c_uint64),
+                ("train_gates", ctypes.c_int32), ("dropout_rate", ctypes.c_float), ("dropout_seed", ctypes.c_uint64)]
 
 
 class _Weights(ctypes.Structure):
@@ -64,6 +65,9 @@ class Config:
     temperature: float = 0.0     # softmax temperature of the router (0 stands for 1)
     noise_sigma: float = 0.0     # std of Gaussian noise on the router logits
     noise_seed: int = 0
+    train_gates: int = 0         # forward calls: 1 = Section 3.3's gates (cross-slice dropout) instead of the probabilities
+    dropout_rate: float = 0.0
+    dropout_seed: int = 0
 
     @property
     def ds(self):
@@ -79,7 +83,8 @@ class Config:
 
     def c(self) -> _Config:
         return _Config(self.T, self.d, self.S, self.E, self.k, self.Hr, self.F, self.dtype, self.act,
-                       self.capacity, self.temperature, self.noise_sigma, self.noise_seed)
+                       self.capacity, self.temperature, self.noise_sigma, self.noise_seed,
+                       self.train_gates, self.dropout_rate, self.dropout_seed)
 
 
 _handle = None

@@ -68,6 +68,11 @@ int make_dims(const slicemoe_config* c, Dims& D) {
     if (!(c->temperature >= 0.0f) || !(c->noise_sigma >= 0.0f) || std::isinf(c->temperature) ||
         std::isinf(c->noise_sigma))
         return SLICEMOE_ERR_SHAPE;
+    if (c->train_gates != 0 && c->train_gates != 1) return SLICEMOE_ERR_SHAPE;
+    if (c->train_gates && (!(c->dropout_rate >= 0.0f) || c->dropout_rate > 1.0f)) return SLICEMOE_ERR_SHAPE;
+    D.train_gates = c->train_gates;
+    D.drop_threshold = c->train_gates ? (unsigned long long)((double)c->dropout_rate * 4294967296.0) : 0ull;   // 2^32 when rate = 1
+    D.drop_seed = c->dropout_seed;
     D.inv_tau = c->temperature > 0.0f ? 1.0f / c->temperature : 1.0f;
     D.noise_sigma = c->noise_sigma;
     D.noise_seed = c->noise_seed;
@@ -168,9 +173,10 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
                                  at<int32_t>(ws, W.status), clear_status, /*one_launch=*/!events, events, st);
     }
     // decode-shaped batches: one launch that streams each expert's weights once
-    if (!events && decode_forward_supported(D))
+    // (train mode: the other one-launch kernels have no gate step; the stage-by-stage forms below do)
+    if (!events && !D.train_gates && decode_forward_supported(D))
         return launch_forward_decode(D, w, h, h_out, idx, p, assigned, kept, xperm, at<int32_t>(ws, W.status), clear_status, st);
-    const bool one_launch = !events && fused_forward_supported(D);
+    const bool one_launch = !events && !D.train_gates && fused_forward_supported(D);
     // (the single kernel clears the status word itself; a later chunk of one host-buffer call keeps
     // what an earlier chunk reported)
     if (!one_launch && clear_status && (rc = reset_status(ws, W, st))) return rc;
@@ -195,6 +201,7 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
         if ((rc = launch_route_tc(D, w, h, idx, p, nullptr, nullptr, at<int32_t>(ws, W.status), st, cta_hist,
                                   scatter ? h_out : nullptr))) return rc;
         if ((rc = mark(1))) return rc;
+        if (D.train_gates && (rc = launch_gate_dropout(D, p, D.drop_seed, D.drop_threshold, st))) return rc;
         if ((rc = launch_dispatch_fused(D, idx, p, cta_hist, grid, rows_per_cta, assigned, kept, offsets, dest, perm,
                                         gate, st))) return rc;
         if ((rc = mark(2))) return rc;
@@ -207,6 +214,7 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     } else {
         if ((rc = route_any(D, w, h, idx, p, assigned, nullptr, at<int32_t>(ws, W.status), st))) return rc;
         if ((rc = mark(1))) return rc;
+        if (D.train_gates && (rc = launch_gate_dropout(D, p, D.drop_seed, D.drop_threshold, st))) return rc;
         const bool gather = tc_ffn_supported(D);
         if ((rc = launch_dispatch(D, h, idx, p, kept, offsets, dest, perm, gather ? nullptr : xperm,
                                   gather ? gate : nullptr, at<int32_t>(ws, W.chunk_hist), st))) return rc;
@@ -413,7 +421,8 @@ int slicemoe_forward_host(const slicemoe_config* cfg, const slicemoe_weights* w,
 
     // (not with logit noise either: its draws are keyed by the row's index in the whole batch, and a chunk's
     // router counts rows from the chunk's start)
-    const bool pipelined = D.capacity == 0 && D.noise_sigma == 0.0f && D.T >= kPipeChunks * kPipeMinTokensPerChunk;
+    // (logit noise and dropout draws are counted by global row numbers: such batches are not cut)
+    const bool pipelined = D.capacity == 0 && D.noise_sigma == 0.0f && !D.train_gates && D.T >= kPipeChunks * kPipeMinTokensPerChunk;
     if (!pipelined) {
         if (bytes) SLICEMOE_CUDA_TRY(cudaMemcpyAsync(h_dev, h_host, bytes, cudaMemcpyHostToDevice, st));
         if ((rc = forward_impl(D, *w, h_dev, hout_dev, assigned_opt, kept_opt, nullptr, nullptr, ws, W, st,

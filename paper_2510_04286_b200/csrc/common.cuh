@@ -22,6 +22,9 @@ struct Dims {
     float inv_tau;        // 1 / softmax temperature
     float noise_sigma;    // 0 = no logit noise
     uint64_t noise_seed;
+    int train_gates;                     // forward calls: Section 3.3's gates instead of the probabilities
+    unsigned long long drop_threshold;   // an assignment is dropped iff its 32-bit draw < this (floor(rate 2^32))
+    uint64_t drop_seed;
 };
 
 // Pairs handled by one dispatch chunk (one CTA of the histogram / scatter kernels).
@@ -152,6 +155,8 @@ int launch_forward_decode(const Dims& D, const slicemoe_weights& w, const void* 
                           bool clear_status, cudaStream_t st);
 int decode_forward_reset_sync(cudaStream_t st);
 
+// Section 3.3's gates in place of the top-k probabilities (gate_dropout.cu).
+int launch_gate_dropout(const Dims& D, float* topk_p, uint64_t seed, unsigned long long threshold, cudaStream_t st);
 int launch_combine(const Dims& D, const void* yperm, const int32_t* dest, void* h_out,
                    cudaStream_t st);
 

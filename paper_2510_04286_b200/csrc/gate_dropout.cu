@@ -40,6 +40,14 @@ __global__ void __launch_bounds__(256) gate_dropout_kernel(float* __restrict__ t
 }
 
 }  // namespace
+
+int launch_gate_dropout(const Dims& D, float* topk_p, uint64_t seed, unsigned long long threshold, cudaStream_t st) {
+    if (D.N == 0) return SLICEMOE_OK;
+    if (D.k > 8) return SLICEMOE_ERR_SHAPE;
+    gate_dropout_kernel<<<(D.N + 255) / 256, 256, 0, st>>>(topk_p, D.N, D.k, (uint32_t)seed, (uint32_t)(seed >> 32), threshold);
+    SLICEMOE_LAUNCH_CHECK(1);
+    return SLICEMOE_OK;
+}
 }  // namespace slicemoe
 
 extern "C" int slicemoe_gate_dropout(const slicemoe_config* cfg, float* topk_p, uint64_t seed, double rate,
@@ -51,10 +59,6 @@ extern "C" int slicemoe_gate_dropout(const slicemoe_config* cfg, float* topk_p, 
     if (!topk_p) return SLICEMOE_ERR_NULL;
     if (!(rate >= 0.0) || rate > 1.0 || D.k > 8) return SLICEMOE_ERR_SHAPE;
     if ((rc = check_device())) return rc;
-    if (D.N == 0) return SLICEMOE_OK;
     const unsigned long long threshold = (unsigned long long)(rate * 4294967296.0);   // 2^32 when rate = 1
-    gate_dropout_kernel<<<(D.N + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        topk_p, D.N, D.k, (uint32_t)seed, (uint32_t)(seed >> 32), threshold);
-    SLICEMOE_LAUNCH_CHECK(1);
-    return SLICEMOE_OK;
+    return launch_gate_dropout(D, topk_p, seed, threshold, static_cast<cudaStream_t>(stream));
 }

@@ -31,6 +31,7 @@
 // With ~200 KB of shared memory per CTA there is next to no L1 left for local memory: everything the role
 // loops call is inlined and sized to compile without a stack frame or a spill.
 #pragma once
+#include "philox.cuh"
 #include "tc_mlp_body.cuh"
 
 namespace slicemoe {
@@ -150,6 +151,9 @@ struct PpParams {
     int32_t* local_rank;        // [N, k] rank of the pair among this CTA's pairs of the same expert
     int32_t* cta_hist;          // [grid, E]
     bf16* zero_out;             // h' as [N, 64]: this CTA zeroes the rows it routes (or nullptr)
+    int train_gates;            // 1: the gates are Section 3.3's (cross-slice dropout) instead of the probabilities
+    uint32_t drop_key0, drop_key1;          // generator key (low, high word of the seed)
+    unsigned long long drop_threshold;      // an assignment is dropped iff its 32-bit draw < this
     int2* lists_out;            // per-expert lists of (pair index, gate) filled by the router itself (or nullptr): expert e's
     int32_t* list_counts;       // list starts at lists_out + e * list_stride; its length is counter e (one per kPpCountStride
                                 // ints) of set sh.counts_set (sets are kMaxE * kPpCountStride ints apart)
@@ -1015,8 +1019,26 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
             float sum = 0.0f;
 #pragma unroll
             for (int i = 0; i < EP; ++i) sum += ex2_approx(fmaf(__uint_as_float(v[i]), sc, -msc));
-            const float inv = 1.0f / sum;
-            const float p2 = ex2_approx(fmaf(b2, sc, -msc)) * inv;
+            float inv = 1.0f / sum;
+            float p2 = ex2_approx(fmaf(b2, sc, -msc)) * inv;
+            if (p.train_gates) {
+                // Section 3.3: each assignment dropped iff the first word of Philox4x32-10(key = seed, counter =
+                // (n, j, 0, 0)) is below the threshold; survivors divided by their sum; none left: top-1 gets 1
+                uint32_t x[4];
+                philox4x32_10((uint32_t)n, 0u, 0u, 0u, p.drop_key0, p.drop_key1, x);
+                const bool d1 = (unsigned long long)x[0] < p.drop_threshold;
+                bool d2 = true;
+                if (p.k > 1) {
+                    philox4x32_10((uint32_t)n, 1u, 0u, 0u, p.drop_key0, p.drop_key1, x);
+                    d2 = (unsigned long long)x[0] < p.drop_threshold;
+                }
+                float kept_sum = 0.0f;
+                if (!d1) kept_sum += inv;
+                if (!d2) kept_sum += p2;
+                const bool none = (d1 && d2) || !(kept_sum > 0.0f);
+                inv = none ? 1.0f : (d1 ? 0.0f : inv / kept_sum);
+                p2 = none ? 0.0f : (d2 ? 0.0f : p2 / kept_sum);
+            }
             const size_t at = (size_t)n * p.k;
             int r1 = 0, r2 = 0;
             if (valid) {

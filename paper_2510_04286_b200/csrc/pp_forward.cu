@@ -230,6 +230,8 @@ void pp_fill_params(const Dims& D, const slicemoe_weights& w, const void* h, voi
     r.br1 = (const bf16*)w.br1; r.br2 = (const bf16*)w.br2;
     r.topk_idx = topk_idx; r.topk_p = topk_p; r.local_rank = dest; r.cta_hist = cta_hist;
     r.zero_out = (bf16*)h_out; r.row_elems = D.ds;
+    r.train_gates = D.train_gates; r.drop_key0 = (uint32_t)D.drop_seed; r.drop_key1 = (uint32_t)(D.drop_seed >> 32);
+    r.drop_threshold = D.drop_threshold;
     f = PpParams{};
     f.status = status; f.n_rows = D.R; f.HID = D.F; f.E = D.E; f.offsets = offsets;
     f.b1 = (const bf16*)w.b1; f.b2 = (const bf16*)w.b2;

@@ -115,3 +115,51 @@ def test_gpu_train_mode_staged_forward():
     y = oracle.expert_ffn(ocfg, x, d["offsets"], w)
     want = oracle.combine(ocfg, y, d["dest"])
     pu.assert_outputs_close(tensors.to_numpy_f32(h_out), want, lc.dtype, "train-mode h'")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,rate,seed", [
+    ("cfg1", 0.2, 7),          # 64-wide slices: gates drawn inside the one-launch forward
+    ("cfg1", 0.0, 3),          # rate 0 still re-normalises the k probabilities
+    ("cfg1", 1.0, 5),          # everything dropped: the top-1 assignment gets weight 1
+    ("cfg3b", 0.3, 11),        # capacity limit, ds = 256, k = 1: stage-by-stage form with the gate step
+    ("cfg4", 0.2, 13),         # decode shape: stage-by-stage form
+    ("cfg0", 0.5, 17),         # fp32 storage, ReLU, biases: CUDA-core kernels
+])
+def test_gpu_train_mode_forward(name, rate, seed):
+    """slicemoe_forward with cfg.train_gates: the returned gates are Section 3.3's (masks equal to the oracle's
+    draw for draw, survivors re-normalised) and h' is the layer evaluated with those gates."""
+    import dataclasses
+    import torch
+    from paper_2510_04286_b200 import binding, tensors
+    import parity_util as pu
+    lc = synth.CONFIGS[name].with_tokens(300 if name != "cfg4" else 64)
+    h, w = synth.make_layer_inputs(lc, 0)
+    gpu = pu.GpuLayer(lc, h, w)
+    plain = gpu.forward()
+    gpu.cfg = dataclasses.replace(gpu.cfg, train_gates=1, dropout_rate=rate, dropout_seed=seed)
+    h_out, assigned, kept, idx, gates = gpu.forward()
+    torch.cuda.synchronize()
+    assert gpu.status() == 0
+    idx_np, g_np = idx.cpu().numpy(), gates.cpu().numpy().astype(np.float64)
+    assert np.array_equal(idx_np, plain[3].cpu().numpy())                  # the draw does not touch the routing
+    # gates: the oracle's rule applied to the probabilities the plain forward returned for the same picks
+    p_plain = plain[4].cpu().numpy()
+    want_g, dropped = oracle.gate_dropout(p_plain.astype(np.float64), seed, rate)
+    none = dropped.all(axis=1)
+    assert np.array_equal(g_np == 0.0, np.where(none[:, None], np.arange(lc.k)[None, :] > 0, dropped))
+    assert np.abs(g_np - want_g).max() <= 4e-7                             # one fp32 division against fp64
+    # h': the oracle's chain with the GPU's picks and gates
+    ocfg = pu.oracle_config(lc)
+    d = oracle.dispatch(ocfg, idx_np)
+    assert np.array_equal(kept.cpu().numpy(), d["kept"])
+    n_kept = int(d["offsets"][-1])
+    x = oracle.weight_slices(ocfg, h, g_np, d["dest"], n_kept)
+    y = oracle.expert_ffn(ocfg, x, d["offsets"], w)
+    want = oracle.combine(ocfg, y, d["dest"])
+    pu.assert_outputs_close(tensors.to_numpy_f32(h_out), want, lc.dtype, "train-mode h'", one_ulp_of_element=True)
+    # a refused rate
+    bad = dataclasses.replace(gpu.cfg, dropout_rate=1.5)
+    gpu.cfg = bad
+    with pytest.raises(binding.SliceMoEError):
+        gpu.forward()

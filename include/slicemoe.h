@@ -24,8 +24,16 @@
  *     stream).  Calls only enqueue work on it: no allocation, no host
  *     synchronisation, unless stated.
  *   - The caller owns every buffer, including the workspace `ws`
- *     (slicemoe_workspace_bytes(), 256-byte aligned).  The library keeps no
- *     device memory of its own.
+ *     (slicemoe_workspace_bytes(), 256-byte aligned).  The library allocates no
+ *     device memory.  Its device image holds a few KB of words of its own per
+ *     GPU, shared by every caller on that GPU: the arrival counters of the
+ *     one-launch forwards' grid barriers, two sets of per-expert list counters
+ *     that successive launches use alternately, and the table of
+ *     slicemoe_dispatch_static.  One-launch forwards are cooperative launches
+ *     (every SM holds one CTA), so two of them never run on a GPU at once.
+ *     slicemoe_forward_host additionally creates, once per device, two streams
+ *     and ten events of its own and serialises callers on a process-wide lock
+ *     while they enqueue.
  *   - Tensors are dense row-major, 16-byte aligned, of cfg->dtype
  *     (bf16 or fp32) unless a type is written.  Weights use the nn.Linear
  *     layout [out, in] with `in` contiguous.  Bias pointers may be NULL (= 0).
@@ -258,6 +266,11 @@ int slicemoe_load_stats(const int32_t *counts, int32_t E, double alpha, double *
  * barriers, one CTA per SM); other shapes run one kernel per step.  Every wait
  * inside is bounded: a run-out leaves SLICEMOE_ERR_DEVICE_TIMEOUT in the status
  * word (slicemoe_last_status) and the call's outputs undefined.
+ * With cfg->train_gates the gates of Eq. 1 are Section 3.3's (see slicemoe_config)
+ * and topk_p_opt returns them; the result equals route -> slicemoe_gate_dropout
+ * (dropout_seed, dropout_rate) -> dispatch -> expert_ffn -> combine.  64-wide
+ * slices keep their single launch in train mode; the other one-launch shapes
+ * then run one kernel per step.
  */
 int slicemoe_forward(const slicemoe_config *cfg, const slicemoe_weights *w, const void *h,
                      void *h_out, int32_t *assigned_opt, int32_t *kept_opt,
@@ -270,7 +283,7 @@ int slicemoe_forward(const slicemoe_config *cfg, const slicemoe_weights *w, cons
  * copy of h into the workspace, the forward, and the device->host copy of h'.
  * Weights and the optional outputs stay DEVICE pointers.  The caller
  * synchronises the stream before reading h_out_host.
- * Without a capacity limit and from 2048 tokens on, the batch is processed in
+ * Without a capacity limit, logit noise or train-mode gates, and from 2048 tokens on, the batch is processed in
  * four chunks of tokens whose copies in and out run on two streams that the
  * library creates once per device, so that the two directions of the link are
  * busy at the same time; in stream order the call still behaves as one

@@ -12,7 +12,8 @@
 // one region is in the activation, the other is in its GEMMs or its output.  Expert pass, warp roles:
 //
 //   warp 0       weight sets by TMA (W1 and W2 of an expert stay in shared memory for a run of tiles of that
-//                expert; two sets) and four-row TMA gathers of tile rows 64-127
+//                expert; two sets; the first run's set is requested by the GEMM-1 warp, which waits for it) and
+//                four-row TMA gathers of tile rows 64-127
 //   warp 2       four-row TMA gathers of tile rows 0-63; both gather warps also copy the rows' (pair, gate)
 //                into a ring in shared memory
 //   warp 3       GEMM-1 issue (one elected lane), warp 1  GEMM-2 issue: two issuing warps, because the small
@@ -25,8 +26,11 @@
 //
 // The router pass has the same shape with its hidden layer in units of 128 (three buffers), the fp32 hidden
 // values split in place into a truncated bf16 and the rounded remainder (so that the logits keep fp32
-// accuracy), and an output warpgroup that does softmax, top-k and each pair's rank among its CTA's pairs of
-// the same expert.  All hand-offs are mbarriers with bounded waits (status word on run-out).
+// accuracy), and an output warpgroup that does softmax, top-k, the train-mode gates of Section 3.3 where asked
+// for, and the dispatch: either each pair's rank among its CTA's pairs of the same expert, or (up to 32 experts)
+// the pairs' entries appended to per-expert lists.  All hand-offs are mbarriers with bounded waits (status word
+// on run-out); the two 128- / 512-thread rendezvous inside the output and activation warpgroups are plain named
+// barriers, reached by all their warps after the same bounded wait.
 //
 // With ~200 KB of shared memory per CTA there is next to no L1 left for local memory: everything the role
 // loops call is inlined and sized to compile without a stack frame or a spill.

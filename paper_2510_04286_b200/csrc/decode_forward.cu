@@ -524,24 +524,33 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             named_barrier_sync(1, kDecWorkers);
             if (threadIdx.x == 0) mbar_arrive(bar(DB::A_FULL));
             const float gs = sh.gate[row];
+            const bool has_b1 = p.b1 != nullptr;
             const bool live = lg * 32 < rows;        // a warp whose 32 rows are all padding only passes the hand-offs on
             for (int c = 0; c < kDecNC && wok; ++c) {
                 const int cc = it * kDecNC + c, r = cc & 1;
                 if (!pp_wait(bar(DB::ACC1_FULL + r), (uint32_t)(cc >> 1) & 1u, abort)) { wok = false; break; }
                 tc_fence_after_sync();
                 if (live) {
+                    // the thread's 64 hidden units of the chunk, eight at a time as a software pipeline around the tanh
+                    // unit (pre of piece j + 1 and post of piece j - 1 under the tanh of piece j); two pieces per
+                    // tensor-memory load and store; no shared-memory bias reads without a first-layer bias
                     const uint32_t region = tlane + r * kDecHC + 64 * g;
-                    uint32_t acc[16];
+                    const float* bias = sh.bias1 + c * kDecHC + 64 * g;
+                    uint32_t acc[16], hid[8];
+                    float z[2][8], u[2][8];
                     tmem_ld_x16(region, acc);
+                    tmem_ld_wait();
+                    pp_pre8<ACT>(acc, gs, bias, has_b1, z[0], u[0]);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float z[16];
-                        uint32_t hid[8];
-                        tmem_ld_wait();
-                        pp_scale16(acc, gs, sh.bias1 + c * kDecHC + 64 * g + 16 * q, true, z);
-                        if (q + 1 < 4) tmem_ld_x16(region + 16 * (q + 1), acc);
-                        pp_act8<ACT>(z, hid);
-                        tmem_st_x8(region + 8 * q, hid);
+                    for (int j = 0; j < 8; ++j) {
+                        pp_tanh8<ACT>(u[j & 1]);
+                        if (j + 1 < 8) {
+                            if (((j + 1) & 1) == 0) tmem_ld_wait();
+                            pp_pre8<ACT>(acc + 8 * ((j + 1) & 1), gs, bias + 8 * (j + 1), has_b1, z[(j + 1) & 1], u[(j + 1) & 1]);
+                            if (((j + 1) & 1) == 1 && j + 2 < 8) tmem_ld_x16(region + 8 * (j + 2), acc);
+                        }
+                        pp_post8<ACT>(z[j & 1], u[j & 1], hid + 4 * (j & 1));
+                        if (j & 1) tmem_st_x8(region + 4 * (j - 1), hid);
                     }
                     tmem_st_wait();
                 }
@@ -568,10 +577,16 @@ decode_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     uint32_t o[4];
+                    if (p.b2) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        o[j] = pack_bf16x2(fmaf(__uint_as_float(v[8 * i + 2 * j]), kOutScale<ACT>, b2[8 * i + 2 * j]),
-                                           fmaf(__uint_as_float(v[8 * i + 2 * j + 1]), kOutScale<ACT>, b2[8 * i + 2 * j + 1]));
+                        for (int j = 0; j < 4; ++j)
+                            o[j] = pack_bf16x2(fmaf(__uint_as_float(v[8 * i + 2 * j]), kOutScale<ACT>, b2[8 * i + 2 * j]),
+                                               fmaf(__uint_as_float(v[8 * i + 2 * j + 1]), kOutScale<ACT>, b2[8 * i + 2 * j + 1]));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            o[j] = pack_bf16x2(__uint_as_float(v[8 * i + 2 * j]) * kOutScale<ACT>, __uint_as_float(v[8 * i + 2 * j + 1]) * kOutScale<ACT>);
+                    }
                     red_add_bf16x8(dst + 8 * i, o[0], o[1], o[2], o[3]);
                 }
             }

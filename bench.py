@@ -236,8 +236,10 @@ def run_reference(args, lc):
 
 
 def workload_config(lc):
+    """The same dict in both arms (the GPU arm's cache policy is a fixed key, its details are in `buffer_rotation`)."""
     return {"workload": lc.name, "T": lc.T, "d": lc.d, "S": lc.S, "E": lc.E, "k": lc.k, "F": lc.F,
-            "Hr": lc.Hr, "act": "gelu_tanh" if lc.act else "relu", "capacity": lc.capacity}
+            "Hr": lc.Hr, "act": "gelu_tanh" if lc.act else "relu", "capacity": lc.capacity,
+            "l2_gpu_arm": "distinct buffer sets larger than L2 rotate between steps"}
 
 
 def l2_note(sets, wsets):

@@ -243,6 +243,41 @@ def test_train_mode_backward_with_dropout_gates(name, rate):
         assert dropped.any()
 
 
+@pytest.mark.parametrize("name,rate", [("cfg1", 0.2), ("cfg4", 0.3), ("cfg0", 0.2)])
+def test_training_step_forward_train_mode_then_backward(name, rate):
+    """A whole training step through the library: slicemoe_forward with cfg.train_gates (the gates drawn inside
+    the forward: in the one-launch kernel for 64-wide slices, by the gate step of the stage-by-stage forms
+    otherwise) hands its ids and gates to slicemoe_backward with dropout_gates; graded against the oracle's
+    backward on the same ids with the oracle's own mask."""
+    import dataclasses
+    import torch
+    lc = synth.CONFIGS[name].with_tokens(120 if name != "cfg4" else 32)
+    h, w = synth.make_layer_inputs(lc, 0)
+    gout = synth.make_grad_out(lc, 0)
+    gpu = pu.GpuLayer(lc, h, w)
+    p_plain = gpu.forward()[4].cpu().numpy().astype(np.float64)
+    gpu.cfg = dataclasses.replace(gpu.cfg, train_gates=1, dropout_rate=rate, dropout_seed=99)
+    c = gpu.cfg
+    _, _, _, idx, gates = gpu.forward()
+    torch.cuda.synchronize()
+    _, dropped = oracle.gate_dropout(p_plain, 99, rate)
+    assert np.array_equal(gates.cpu().numpy() == 0.0,
+                          dropped & ~(dropped.all(axis=1, keepdims=True) & (np.arange(lc.k) == 0)))
+    assert dropped.any()
+    g_dev = pu.tensors.to_torch(gout, lc.dtype, "cuda")
+    shapes = dict(dWr1=(c.Hr, c.ds), dbr1=(c.Hr,), dWr2=(c.E, c.Hr), dbr2=(c.E,), dW1=(c.E, c.F, c.ds),
+                  db1=(c.E, c.F), dW2=(c.E, c.ds, c.F), db2=(c.E, c.ds))
+    grads = {n: torch.empty(s_, dtype=torch.float32, device="cuda") for n, s_ in shapes.items()}
+    dh = torch.empty((c.T, c.d), dtype=gpu.tdtype, device="cuda")
+    ws = torch.empty(binding.slicemoe_backward_workspace_bytes(c), dtype=torch.uint8, device="cuda")
+    binding.slicemoe_backward(c, gpu.w, gpu.h, g_dev, idx, gates, dh, grads, ws, dropout_gates=True)
+    torch.cuda.synchronize()
+    ref = oracle.backward(pu.oracle_config(lc), h, w, gout, forced_idx=idx.cpu().numpy(), dropped=dropped)
+    got = {n: t.cpu().numpy().astype(np.float64) for n, t in grads.items()}
+    got["dh"] = pu.tensors.to_numpy_f32(dh).astype(np.float64)
+    compare(got, ref, lc)
+
+
 @pytest.mark.parametrize("block", range(3))
 def test_backward_random_shapes(block):
     """Seeded random shapes: widths inside and outside the tensor-core set, fp32 and bf16 storage,

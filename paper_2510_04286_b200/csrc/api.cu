@@ -138,12 +138,16 @@ static int reset_status(void* ws, const Workspace& W, cudaStream_t st) {
 // other widths) runs on the CUDA-core kernels.  Both are this library's own kernels.
 static int route_any(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* idx, float* p,
                      int32_t* assigned, float* probs, int32_t* status, cudaStream_t st) {
+    // (64-wide slices without the full probability matrix: the whole-tile pipeline's router)
+    if (!probs && pp_route_supported(D)) return launch_route_pp(D, w, h, idx, p, assigned, status, st);
     if (tc_route_supported(D)) return launch_route_tc(D, w, h, idx, p, assigned, probs, status, st);
     return launch_route_simt(D, w, h, idx, p, assigned, probs, st);
 }
 
 static int ffn_any(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets,
                    void* yperm, int32_t* status, cudaStream_t st) {
+    // (64-wide slices: the whole-tile pipeline's expert pass on the stacked rows)
+    if (pp_ffn_supported(D)) return launch_ffn_pp(D, w, xperm, offsets, yperm, status, st);
     if (tc_ffn_supported(D)) return launch_ffn_tc(D, w, xperm, offsets, yperm, status, st);
     return launch_ffn_simt(D, w, xperm, offsets, yperm, st);
 }

@@ -141,6 +141,12 @@ int fused_forward_reset_sync(cudaStream_t st);
 // (stacked row -> pair index and gate); the order of the stacked rows inside an expert is not the stable
 // (n, j) order of slicemoe_dispatch.
 bool pp_forward_supported(const Dims& D);
+bool pp_route_supported(const Dims& D);
+bool pp_ffn_supported(const Dims& D);
+int launch_ffn_pp(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets, void* yperm,
+                  int32_t* status, cudaStream_t st);
+int launch_route_pp(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx, float* topk_p,
+                    int32_t* assigned, int32_t* status, cudaStream_t st);
 int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
                       float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest, void* pair_gate,
                       int32_t* cta_hist, int32_t* status, bool clear_status, bool one_launch, void* const* events,

@@ -152,7 +152,9 @@ struct PpParams {
     const bf16* br2;            // [E] or nullptr
     int32_t* topk_idx;          // [N, k]
     float* topk_p;              // [N, k]
-    int32_t* local_rank;        // [N, k] rank of the pair among this CTA's pairs of the same expert
+    int32_t* local_rank;        // [N, k] rank of the pair among this CTA's pairs of the same expert (or nullptr)
+    int32_t* assigned_out;      // [E] pairs per expert, added to with one atomic per expert and CTA (or nullptr; the
+                                // caller zeroes it)
     int32_t* cta_hist;          // [grid, E]
     bf16* zero_out;             // h' as [N, 64]: this CTA zeroes the rows it routes (or nullptr)
     int train_gates;            // 1: the gates are Section 3.3's (cross-slice dropout) instead of the probabilities
@@ -358,7 +360,10 @@ __device__ __forceinline__ void pp_ffn_init_bars(PpShared& sh, const CUtensorMap
 // caller.  SAME_LAUNCH: pair_gate (and the offsets) were written earlier in this launch.
 // READY: the caller has initialised the barriers (pp_ffn_init_bars), filled sh.offs and sh.tile_start and
 // synchronised the CTA.  Rows come from gather_src through pair_gate and results are added into scatter_out.
-template <int N2, int ACT, bool SAME_LAUNCH, bool READY>
+// STAGED (the staged call, slicemoe_expert_ffn): the rows are already stacked and weighted (Eq. 1): a tile's rows
+// are one tiled load through tmXg_p (then a map of the stacked rows with a 128-row box), every gate is 1 and a
+// row's result is stored to the same row of scatter_out (the stacked outputs) instead of added.
+template <int N2, int ACT, bool SAME_LAUNCH, bool READY, bool STAGED = false>
 __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUtensorMap* tmW1_p, const CUtensorMap* tmW2_p,
                                             const PpParams& p, PpShared& sh, uint8_t* smem_raw) {
     using C = PpFfnCfg<N2>;
@@ -506,7 +511,7 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
             int2 nnext[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) nnext[q] = make_int2(-1, 0);
-            int loaded_run = 0, cur_e = 0, cur_run = 0, cur_rows = 0;      // (run 0's weights: the GEMM-1 warp)
+            int loaded_run = 0, cur_e = 0, cur_run = 0, cur_rows = 0, next_row0 = 0;      // (run 0's weights: the GEMM-1 warp)
             uint32_t last_bar = 0, last_par = 0;
             bool ok = true;
             const uint32_t set_tx = (uint32_t)(p.HID * 128 + npanels * C::W2_CHUNK);
@@ -526,10 +531,16 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     for (int q = 0; q < 4; ++q) {
                         const int r = rbase + 4 * (lane & 15) + q;
                         nnext[q] = make_int2(-1, 0);
-                        const size_t at = p.list_stride ? (size_t)wn.e * p.list_stride + (wn.row0 - sh.offs[wn.e]) + r : (size_t)wn.row0 + r;
-                        if (r < wn.rows) nnext[q] = SAME_LAUNCH ? __ldcg(p.pair_gate + at) : __ldg(p.pair_gate + at);
+                        if (STAGED) {
+                            if (r < wn.rows) nnext[q] = make_int2(wn.row0 + r, __float_as_int(1.0f));
+                        } else {
+                            const size_t at = p.list_stride ? (size_t)wn.e * p.list_stride + (wn.row0 - sh.offs[wn.e]) + r : (size_t)wn.row0 + r;
+                            if (r < wn.rows) nnext[q] = SAME_LAUNCH ? __ldcg(p.pair_gate + at) : __ldg(p.pair_gate + at);
+                        }
                     }
                 }
+                const int cur_row0 = next_row0;
+                next_row0 = wn.row0;
                 if (ta < 0) continue;
                 // weights of a new run
                 const int want_run = cur_run, want_e = cur_e;
@@ -567,8 +578,13 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
                     if (warp == 2) mbar_arrive_expect_tx(pp_bar(sh, B::A_FULL + ab), kPpABytes);
                     else mbar_arrive(pp_bar(sh, B::A_FULL + ab));
                 }
-                if (lane < 16)
+                if (STAGED) {
+                    // (rows past the expert's last one belong to the next expert or lie past the matrix, where the
+                    // copy engine fills zeros: computed and never stored)
+                    if (lane == 0 && warp == 2) tma_load_2d(sA + ab * kPpABytes, tmXg_p, 0, cur_row0, pp_bar(sh, B::A_FULL + ab));
+                } else if (lane < 16) {
                     tma_gather4(sA + ab * kPpABytes + (rbase / 4 + lane) * 512, tmXg_p, 0, nrow[0], nrow[1], nrow[2], nrow[3], pp_bar(sh, B::A_FULL + ab));
+                }
             }
             if (!ok || *abort) {
                 // (bounded) let the copies in flight land before shared memory is reused
@@ -698,14 +714,18 @@ __device__ __forceinline__ void pp_ffn_body(const CUtensorMap* tmXg_p, const CUt
 #pragma unroll
             for (int c = 0; c < N2; c += 8) st_shared_v4(srow + c * 2, o[c / 2], o[c / 2 + 1], o[c / 2 + 2], o[c / 2 + 3]);
             __syncwarp();
-            const int n_own = live ? pair_to_row(sh.pair_gate_s[ta % kPpMetaRing][row].x, p.gather_magic, p.gather_shift) : -1;
+            const int n_own = !live ? -1 : STAGED ? sh.pair_gate_s[ta % kPpMetaRing][row].x
+                                                  : pair_to_row(sh.pair_gate_s[ta % kPpMetaRing][row].x, p.gather_magic, p.gather_shift);
             const int sub = lane >> 3, chunk = lane & 7;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int rl = 4 * i + sub;                                   // row of this warp's 32
                 const int n_i = __shfl_sync(0xffffffffu, n_own, rl);
                 const uint4 t = ld_shared_v4(swarp + rl * C::OUT_PITCH + chunk * 16);
-                if (n_i >= 0 && chunk < N2 / 8) red_add_bf16x8(p.scatter_out + (size_t)n_i * N2 + chunk * 8, t.x, t.y, t.z, t.w);
+                if (n_i >= 0 && chunk < N2 / 8) {
+                    if (STAGED) *reinterpret_cast<uint4*>(p.scatter_out + (size_t)n_i * N2 + chunk * 8) = t;
+                    else red_add_bf16x8(p.scatter_out + (size_t)n_i * N2 + chunk * 8, t.x, t.y, t.z, t.w);
+                }
             }
         }
     }
@@ -1056,7 +1076,7 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
                     p.topk_idx[at] = i1;
                     p.topk_p[at] = inv;
                 }
-                if (!lists) {
+                if (!lists && p.local_rank) {
                     p.local_rank[at] = r1;
                     if (p.k > 1) p.local_rank[at + 1] = r2;
                 }
@@ -1089,6 +1109,9 @@ __device__ __forceinline__ void pp_route_body(const CUtensorMap* tmX_p, const CU
     if (threadIdx.x == 0 && sh.abort_flag) atomicExch(p.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
     if (p.cta_hist)
         for (int i = threadIdx.x; i < p.experts_real; i += kPpThreads) p.cta_hist[(size_t)blockIdx.x * p.experts_real + i] = sh.hist[i];
+    if (p.assigned_out && ntiles > 0)
+        for (int i = threadIdx.x; i < p.experts_real; i += kPpThreads)
+            if (sh.hist[i] > 0) atomicAdd(p.assigned_out + i, sh.hist[i]);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();

@@ -147,7 +147,7 @@ pp_dispatch_kernel(const int32_t* topk_idx, const float* topk_p, const int32_t* 
                                         pairs_per_chunk, assigned, kept, offsets, dest, pair_gate, sm, offs);
 }
 
-template <int N2, int ACT>
+template <int N2, int ACT, bool STAGED = false>
 __global__ void __launch_bounds__(kPpThreads, 1)
 pp_ffn_kernel(const __grid_constant__ CUtensorMap tmXg, const __grid_constant__ CUtensorMap tmW1,
               const __grid_constant__ CUtensorMap tmW2, const PpParams p) {
@@ -158,7 +158,7 @@ pp_ffn_kernel(const __grid_constant__ CUtensorMap tmXg, const __grid_constant__ 
         tmem_alloc(smem_u32(&sh.tmem_base), 512);
         tmem_relinquish();
     }
-    pp_ffn_body<N2, ACT, false, false>(&tmXg, &tmW1, &tmW2, p, sh, smem_raw);
+    pp_ffn_body<N2, ACT, false, false, STAGED>(&tmXg, &tmW1, &tmW2, p, sh, smem_raw);
     if (warp == 1) {
         __syncwarp();
         tmem_dealloc(sh.tmem_base, 512);
@@ -342,6 +342,84 @@ bool pp_forward_supported(const Dims& D) {
     if (D.Hr % 128 || D.Hr < 128 || D.Hr > kPpMaxHr) return false;      // (the router takes its hidden layer in halves of 128)
     if (D.F != 128 && D.F != kPpMaxF) return false;                    // (the activation takes the hidden layer in turns of 64 or 128 columns per warpgroup)
     return pp_cooperative_launch_available();
+}
+
+// The router pass as the staged call's kernel (slicemoe_route without the full probability matrix): top-k ids
+// and probabilities, `assigned` by one atomic per expert and CTA.
+bool pp_route_supported(const Dims& D) {
+    if (D.dtype != SLICEMOE_BF16 || D.ds != 64 || D.N <= 0) return false;
+    if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
+    if (D.k > 2 || D.noise_sigma > 0.0f) return false;
+    return D.Hr % 128 == 0 && D.Hr >= 128 && D.Hr <= kPpMaxHr;
+}
+
+template <int EP>
+static int pp_launch_route_only(const Dims& D, const slicemoe_weights& w, const void* h, const PpParams& rp, cudaStream_t st) {
+    PpMaps m;      // (only the router's three maps: the expert weights may be absent in this call)
+    int rc;
+    if ((rc = make_tmap(&m.X, h, (uint64_t)D.N, (uint64_t)D.ds, 128))) return rc;
+    if ((rc = make_tmap(&m.Wr1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, kPpHC))) return rc;
+    if ((rc = make_tmap(&m.Wr2, w.Wr2, (uint64_t)D.E, (uint64_t)D.Hr, EP))) return rc;
+    const int tiles = (D.N + kTileM - 1) / kTileM;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    constexpr int slot_r = 6 + (EP == 16 ? 0 : EP == 32 ? 1 : 2);
+    auto kr = pp_route_kernel<EP>;
+    constexpr int smem_r = PpRouteCfg<EP>::SMEM_ALLOC > 120 * 1024 ? PpRouteCfg<EP>::SMEM_ALLOC : 120 * 1024;
+    if ((rc = pp_set_smem(kr, slot_r, smem_r))) return rc;
+    kr<<<grid, kPpThreads, smem_r, st>>>(m.X, m.Wr1, m.Wr2, rp);
+    SLICEMOE_LAUNCH_CHECK(1);
+    return SLICEMOE_OK;
+}
+
+int launch_route_pp(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx, float* topk_p,
+                    int32_t* assigned, int32_t* status, cudaStream_t st) {
+    if (assigned) SLICEMOE_CUDA_TRY(cudaMemsetAsync(assigned, 0, sizeof(int32_t) * D.E, st));
+    PpParams r{}, f{};
+    pp_fill_params(D, w, h, nullptr, topk_idx, topk_p, nullptr, nullptr, nullptr, nullptr, status, r, f);
+    r.zero_out = nullptr;
+    r.local_rank = nullptr;
+    r.assigned_out = assigned;
+    r.train_gates = 0;            // (the staged router returns the probabilities; slicemoe_gate_dropout is a call of its own)
+    switch (D.E) {
+        case 8:
+        case 16: return pp_launch_route_only<16>(D, w, h, r, st);
+        case 32: return pp_launch_route_only<32>(D, w, h, r, st);
+        case 64: return pp_launch_route_only<64>(D, w, h, r, st);
+        default: return SLICEMOE_ERR_UNSUPPORTED;
+    }
+}
+
+// The expert pass as the staged call's kernel (slicemoe_expert_ffn on stacked, already weighted rows).
+bool pp_ffn_supported(const Dims& D) {
+    if (D.dtype != SLICEMOE_BF16 || D.ds != 64 || D.R <= 0 || D.E > kMaxE) return false;
+    return D.F == 128 || D.F == kPpMaxF;
+}
+
+template <int ACT>
+static int pp_launch_ffn_only(const Dims& D, const slicemoe_weights& w, const void* xperm, const PpParams& fpar, cudaStream_t st) {
+    CUtensorMap mX, mW1, mW2;
+    int rc;
+    if ((rc = make_tmap(&mX, xperm, (uint64_t)D.R, (uint64_t)D.ds, 128))) return rc;
+    if ((rc = make_tmap(&mW1, w.W1, (uint64_t)D.E * D.F, (uint64_t)D.ds, kPpHC))) return rc;
+    if ((rc = make_tmap(&mW2, w.W2, (uint64_t)D.E * 64, (uint64_t)D.F, 64))) return rc;
+    auto kf = pp_ffn_kernel<64, ACT, true>;
+    constexpr int slot_f = 11 + (ACT == SLICEMOE_ACT_RELU ? 0 : 1);
+    if ((rc = pp_set_smem(kf, slot_f, PpFfnCfg<64>::SMEM_ALLOC))) return rc;
+    const int grid = max_tiles(D) < sm_count() ? max_tiles(D) : sm_count();
+    kf<<<grid, kPpThreads, PpFfnCfg<64>::SMEM_ALLOC, st>>>(mX, mW1, mW2, fpar);
+    SLICEMOE_LAUNCH_CHECK(1);
+    return SLICEMOE_OK;
+}
+
+int launch_ffn_pp(const Dims& D, const slicemoe_weights& w, const void* xperm, const int32_t* offsets, void* yperm,
+                  int32_t* status, cudaStream_t st) {
+    PpParams r{}, f{};
+    pp_fill_params(D, w, xperm, yperm, nullptr, nullptr, nullptr, const_cast<int32_t*>(offsets), nullptr, nullptr, status, r, f);
+    f.gather_src = nullptr;
+    f.pair_gate = nullptr;
+    f.list_stride = 0;
+    return D.act == SLICEMOE_ACT_GELU_TANH ? pp_launch_ffn_only<SLICEMOE_ACT_GELU_TANH>(D, w, xperm, f, st)
+                                           : pp_launch_ffn_only<SLICEMOE_ACT_RELU>(D, w, xperm, f, st);
 }
 
 int launch_forward_pp(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,

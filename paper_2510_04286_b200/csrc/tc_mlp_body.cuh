@@ -857,7 +857,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #pragma unroll
                         for (int i = 0; i < C::SUB; ++i)
                             convert_piece_bf16x2(v[i], gs, reinterpret_cast<const uint4*>(sb1 + (s0 + i) * C::PIECE * 2),
-                                                 true, z[s0 + i]);
+                                                 p.bias1 != nullptr, z[s0 + i]);      // (no shared-memory reads without a bias)
                     }
                     tc_fence_before_sync();
                     __syncwarp();

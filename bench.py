@@ -40,7 +40,7 @@ NCU_TRAFFIC = {
     ("forward_one_launch", 65536 * 16, 64, 2, 256): (613.103e6 + 342.652e6, "profiles/pp_forward_kernel_cfg1_cfg2.md (ncu, cfg2)"),
     ("forward_one_launch", 128 * 32, 128, 2, 512): (17.868e6, "profiles/decode_forward_kernel_cfg4.md (ncu, cfg4)"),
 }
-OTHER_CONFIGS = ("cfg2", "cfg3", "cfg3b", "cfg4")
+OTHER_CONFIGS = ("cfg2", "cfg3", "cfg3b", "cfg4", "paper768")     # paper768: the paper's own model shape (d = 768, S = 8, E = 16, k = 2)
 # dram__bytes_read + dram__bytes_write of the two backward kernels on cfg1 (profiles/backward_cfg1.md)
 NCU_TRAFFIC_BACKWARD_CFG1 = (43.363072e6 + 26.524160e6) + (87.232256e6 + 5.461248e6)
 NCU_TRAFFIC_ROWS_CFG1 = 16384 * 8

@@ -140,6 +140,8 @@ static int route_any(const Dims& D, const slicemoe_weights& w, const void* h, in
                      int32_t* assigned, float* probs, int32_t* status, cudaStream_t st) {
     // (64-wide slices without the full probability matrix: the whole-tile pipeline's router)
     if (!probs && pp_route_supported(D)) return launch_route_pp(D, w, h, idx, p, assigned, status, st);
+    // (wide slices, likewise: the router that keeps both weight matrices in shared memory)
+    if (!probs && wide_route_supported(D)) return launch_route_wide(D, w, h, idx, p, assigned, status, st);
     if (tc_route_supported(D)) return launch_route_tc(D, w, h, idx, p, assigned, probs, status, st);
     return launch_route_simt(D, w, h, idx, p, assigned, probs, st);
 }
@@ -181,9 +183,12 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     if (!events && !D.train_gates && decode_forward_supported(D))
         return launch_forward_decode(D, w, h, h_out, idx, p, assigned, kept, xperm, at<int32_t>(ws, W.status), clear_status, st);
     const bool one_launch = !events && !D.train_gates && fused_forward_supported(D);
+    // wide slices: the router is a launch of its own (its resident weights leave no shared memory for the other
+    // phases' state), the single kernel takes over at the dispatch
+    const bool wide = wide_route_supported(D);
     // (the single kernel clears the status word itself; a later chunk of one host-buffer call keeps
     // what an earlier chunk reported)
-    if (!one_launch && clear_status && (rc = reset_status(ws, W, st))) return rc;
+    if ((!one_launch || wide) && clear_status && (rc = reset_status(ws, W, st))) return rc;
     if ((rc = mark(0))) return rc;
     // With both tensor-core kernels available the stacked rows are never materialised: the router
     // leaves its per-CTA expert counts, one dispatch kernel ranks the pairs (dest, perm, gate) and
@@ -192,9 +197,13 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     float* gate = at<float>(ws, W.gate);
     // One cooperative launch does all of it; the stage-timed call keeps the three launches so that
     // the stages stay separable.
-    if (one_launch)
+    if (one_launch) {
+        if (wide && (rc = launch_route_wide(D, w, h, idx, p, nullptr, at<int32_t>(ws, W.status), st,
+                                            at<int32_t>(ws, W.cta_hist), h_out, fused_forward_grid()))) return rc;
         return launch_forward_fused(D, w, h, h_out, idx, p, assigned, kept, offsets, dest, perm, gate,
-                                    at<int32_t>(ws, W.cta_hist), at<int32_t>(ws, W.status), clear_status, st);
+                                    at<int32_t>(ws, W.cta_hist), at<int32_t>(ws, W.status), clear_status && !wide, st,
+                                    /*router_done=*/wide);
+    }
     if (fused) {
         int grid = 0, rows_per_cta = 0;
         tc_route_grid(D, &grid, &rows_per_cta);
@@ -202,8 +211,11 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
         // k <= 2: the experts add their rows straight into h' (zeroed by the router), so there is no
         // stacked output and no combine kernel; the two-term bf16 sum is order-independent.
         const bool scatter = D.k <= 2;
-        if ((rc = launch_route_tc(D, w, h, idx, p, nullptr, nullptr, at<int32_t>(ws, W.status), st, cta_hist,
-                                  scatter ? h_out : nullptr))) return rc;
+        if (wide) {
+            if ((rc = launch_route_wide(D, w, h, idx, p, nullptr, at<int32_t>(ws, W.status), st, cta_hist,
+                                        scatter ? h_out : nullptr))) return rc;
+        } else if ((rc = launch_route_tc(D, w, h, idx, p, nullptr, nullptr, at<int32_t>(ws, W.status), st, cta_hist,
+                                         scatter ? h_out : nullptr))) return rc;
         if ((rc = mark(1))) return rc;
         if (D.train_gates && (rc = launch_gate_dropout(D, p, D.drop_seed, D.drop_threshold, st))) return rc;
         if ((rc = launch_dispatch_fused(D, idx, p, cta_hist, grid, rows_per_cta, assigned, kept, offsets, dest, perm,

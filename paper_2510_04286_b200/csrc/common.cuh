@@ -105,6 +105,14 @@ bool tc_ffn_supported(const Dims& D);
 int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx,
                     float* topk_p, int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st,
                     int32_t* cta_hist = nullptr, void* zero_out = nullptr);
+// The router of wide slices (rows of 192 / 256 elements, router hidden width 256, k <= 2) with Wr1 and Wr2 resident
+// in shared memory; same outputs, grid and row partition as launch_route_tc without the probability matrix.
+// grid_rows: launch at least that many CTAs, so that cta_hist has that many rows (the single-kernel forward's
+// dispatch reads one row per CTA of ITS grid, the number of SMs).
+bool wide_route_supported(const Dims& D);
+int launch_route_wide(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx, float* topk_p,
+                      int32_t* assigned, int32_t* status, cudaStream_t st, int32_t* cta_hist = nullptr,
+                      void* zero_out = nullptr, int grid_rows = 0);
 // Grid of the tensor-core router and the rows each of its CTAs routes (CTA c: rows [c*rows_per_cta, ...)).
 void tc_route_grid(const Dims& D, int* grid, int* rows_per_cta);
 // Fused dispatch after the tensor-core router: one kernel that turns the router's per-CTA counts into
@@ -126,14 +134,17 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
 // barriers between them): bf16 shapes that both tensor-core kernels take, k <= 2.  The kernel clears
 // the status word itself (no memset before it).  topk_idx/topk_p/dest/perm/gate/cta_hist as in the
 // three-launch path; assigned/kept/offsets are written by CTA 0.
+// router_done: an earlier launch on the stream (launch_route_wide with cta_hist and zero_out) has routed the batch
+// over the same grid and row partition; the kernel starts at its dispatch phase.
 // fused_forward_reset_sync: puts the device's grid-barrier words back to zero (after a launch whose
 // bounded waits ran out).
 bool fused_forward_supported(const Dims& D);
 int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
                          float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
                          int32_t* perm, float* gate, int32_t* cta_hist, int32_t* status, bool clear_status,
-                         cudaStream_t st);
+                         cudaStream_t st, bool router_done = false);
 int fused_forward_reset_sync(cudaStream_t st);
+int fused_forward_grid();      // CTAs of the single kernel (one per SM)
 
 // The same forward on the two-stream pipeline (pp_body.cuh): 64-wide slices, k <= 2, no capacity limit.
 // one_launch: a single cooperative launch; otherwise one launch per phase with the stage events recorded.

@@ -2,6 +2,8 @@
 //
 //   phase 1  router       tc_body over this CTA's share of the row tiles: top-k ids and probabilities,
 //                         this CTA's per-expert counts (one row of the table), its rows of h' zeroed
+//                         (wide slices: a launch of its own before this one, route_wide.cu, and the kernel
+//                         starts at phase 2)
 //   -- grid barrier --    (the table is complete)
 //   phase 2  dispatch     this CTA ranks the pairs its own router phase produced: dest, perm, gate;
 //                         CTA 0 also writes assigned / kept / offsets
@@ -29,6 +31,7 @@ struct FusedParams {
     float* gate;
     int32_t* sync_words;      // g_grid_sync of this device
     int clear_status;         // set the status word to OK at entry
+    int router_done;          // phase 1 ran as a launch of its own before this one (same grid, same row partition)
 };
 
 // Grid barrier words (arrival count, generation), one pair per device, owned by the library: zero
@@ -91,9 +94,16 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     }
 
     // ---- phase 1: router -----------------------------------------------------------------------
-    tc_body<RC, false, false, true>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
-    bool ok = sh.abort_flag == 0;
-    ok = grid_barrier(fp.sync_words, gen0, sh) && ok;
+    bool ok = true;
+    if (!fp.router_done) {
+        tc_body<RC, false, false, true>(&tmX, &tmWr1, &tmWr2, fp.route, sh, smem_raw);
+        ok = sh.abort_flag == 0;
+        ok = grid_barrier(fp.sync_words, gen0, sh) && ok;
+        ++gen0;
+    } else {
+        if (threadIdx.x == 0) sh.abort_flag = 0;
+        __syncthreads();
+    }
 
     // ---- phase 2: dispatch of this CTA's own pairs -----------------------------------------------
     if (ok) {
@@ -102,7 +112,7 @@ fused_forward_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                                (int)blockIdx.x, fp.R, fp.E, fp.pairs_per_chunk, fp.capacity,
                                                fp.assigned, fp.kept, fp.offsets, fp.dest, fp.perm, fp.gate, dsm, sh.offs);
     }
-    ok = grid_barrier(fp.sync_words, gen0 + 1, sh) && ok;
+    ok = grid_barrier(fp.sync_words, gen0, sh) && ok;
 
     // ---- phase 3: experts ------------------------------------------------------------------------
     if (ok) tc_body<EC, true, true, true>(&tmX, &tmW1, &tmW2, fp.ffn, sh, smem_raw);
@@ -213,6 +223,8 @@ int fused_forward_reset_sync(cudaStream_t st) {
     return SLICEMOE_OK;
 }
 
+int fused_forward_grid() { return sm_count(); }
+
 bool fused_forward_supported(const Dims& D) {
     return tc_route_supported(D) && tc_ffn_supported(D) && D.N > 0 && D.k <= 2 && cooperative_launch_available();
 }
@@ -220,9 +232,10 @@ bool fused_forward_supported(const Dims& D) {
 int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h, void* h_out, int32_t* topk_idx,
                          float* topk_p, int32_t* assigned, int32_t* kept, int32_t* offsets, int32_t* dest,
                          int32_t* perm, float* gate, int32_t* cta_hist, int32_t* status, bool clear_status,
-                         cudaStream_t st) {
+                         cudaStream_t st, bool router_done) {
     FusedParams fp{};
     fp.clear_status = clear_status ? 1 : 0;
+    fp.router_done = router_done ? 1 : 0;
     int rc = grid_sync_address(&fp.sync_words);
     if (rc) return rc;
     const int grid = sm_count();

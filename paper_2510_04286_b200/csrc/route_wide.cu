@@ -1,0 +1,439 @@
+// Router of wide slices (Section 3.1: relu(X Wr1^T + br1) Wr2^T + br2 -> softmax -> top-k), bf16 storage, rows of
+// 192 or 256 elements, router hidden width 256, up to 64 experts, k <= 2 (sm_100a: tcgen05 + TMEM + TMA).
+//
+// The whole of Wr1 (128 KB) and Wr2 stay in shared memory for the life of the CTA, so a tile's GEMM-1 runs as
+// 128-wide MMAs against operands that are written to shared memory once per launch, not once per tile: what a tile
+// moves through shared memory is its own 64 KB of rows and the operand reads of its MMAs.  That leaves room for
+// exactly ONE row tile, held as four 64-column panels with a full / empty barrier pair each: a panel is handed back
+// as soon as the tile's last MMAs on it have completed and the next tile's panel is requested at once, so the row
+// loads run a whole tile ahead of their use although only one tile's worth of shared memory exists.
+//
+// One CTA of 768 threads per SM walks a contiguous range of 128-row tiles.  A tile is two units of 128 hidden
+// columns; three 128-column buffers of tensor memory take the units in turn (GEMM-1 runs up to two units ahead of
+// GEMM-2), the activation warps turn a buffer's fp32 values in place into a truncated bf16 and the rounded remainder
+// (GEMM-2 runs over both, so the logits keep fp32-level accuracy and the top-k decision does not hang on a bf16
+// rounding of the hidden layer), GEMM-2 reads them from tensor memory.  Warp roles:
+//   warp 0       row panels by TMA          warp 3  GEMM-1 issue        warp 1  GEMM-2 issue
+//   warp 2       zeroes this CTA's rows of h' (forward: the experts add into it)
+//   warps 4-19   activation (four warpgroups, 32 of a unit's 128 columns each; a thread owns one tile row)
+//   warps 20-23  softmax, top-k (ties to the lower id), this CTA's per-expert counts
+// All hand-offs are mbarriers with bounded waits; a run-out sets the status word and every role leaves.
+#include <mutex>
+
+#include "pp_body.cuh"
+
+namespace slicemoe {
+namespace {
+
+constexpr int kWrKP = 4;                      // 64-column panels of a row tile
+constexpr int kWrHr = 256;                    // router hidden width
+constexpr int kWrPanelA = kTileM * 128;       // bytes: 128 rows x 64 bf16
+constexpr int kWrPanelW1 = kWrHr * 128;       // bytes: 256 hidden units x 64 bf16
+constexpr int kWrMaxE = 64;
+
+struct WrShared {
+    __align__(8) uint64_t bars[32];
+    int hist[kWrMaxE];
+    uint32_t tmem_base;
+    int abort_flag;
+    __align__(16) float bias1_f32[kWrHr];
+    __align__(16) float bias2_f32[kWrMaxE];
+};
+
+struct WrBars {
+    static constexpr int A_FULL = 0;                        // [kWrKP]
+    static constexpr int A_EMPTY = A_FULL + kWrKP;          // [kWrKP]
+    static constexpr int W1_FULL = A_EMPTY + kWrKP;         // [kWrKP] one per K panel of Wr1
+    static constexpr int W2_FULL = W1_FULL + kWrKP;
+    static constexpr int ACC1_FULL = W2_FULL + 1;           // [3]
+    static constexpr int ACC1_EMPTY = ACC1_FULL + 3;        // [3]
+    static constexpr int HID_FULL = ACC1_EMPTY + 3;         // [3]
+    static constexpr int ACC2_FULL = HID_FULL + 3;          // [2]
+    static constexpr int ACC2_EMPTY = ACC2_FULL + 2;        // [2]
+    static constexpr int DRAIN = ACC2_EMPTY + 2;            // [2]
+    static constexpr int COUNT = DRAIN + 2;
+};
+static_assert(WrBars::COUNT <= 32, "barrier slots");
+
+template <int EP>
+struct WrCfg {
+    static constexpr int W2_CHUNK = EP * 128;               // bytes: EP experts x 64 hidden units
+    static constexpr int OFF_A = 0;
+    static constexpr int OFF_W1 = OFF_A + kWrKP * kWrPanelA;
+    static constexpr int OFF_W2 = OFF_W1 + kWrKP * kWrPanelW1;
+    static constexpr int SMEM_BYTES = OFF_W2 + (kWrHr / 64) * W2_CHUNK;
+    static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;
+    static constexpr int HB_COLS = 128, LOGIT_COL = 384;
+    static_assert(SMEM_ALLOC + sizeof(WrShared) + 64 <= 232448, "shared memory budget");
+    static_assert(EP % 16 == 0 && EP <= kWrMaxE, "expert count");
+};
+
+__device__ __forceinline__ uint32_t wr_bar(WrShared& sh, int i) { return smem_u32(&sh.bars[i]); }
+
+template <int EP>
+__global__ void __launch_bounds__(kPpThreads, 1)
+route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
+                  const __grid_constant__ CUtensorMap tmW2, const PpParams p) {
+    using C = WrCfg<EP>;
+    using B = WrBars;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ WrShared sh;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    volatile int* abort = &sh.abort_flag;
+
+    const int total_tiles = (p.n_rows + kTileM - 1) / kTileM;
+    const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
+    const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
+    const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
+    const int nunits = ntiles * 2;
+    const uint32_t sA = smem_base + C::OFF_A, sW1 = smem_base + C::OFF_W1, sW2 = smem_base + C::OFF_W2;
+
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh.tmem_base), 512);
+        tmem_relinquish();
+    }
+    if (threadIdx.x == 0) {
+        prefetch_tensormap(&tmX);
+        sh.abort_flag = 0;
+        for (int i = 0; i < kWrKP; ++i) { mbar_init(wr_bar(sh, B::A_FULL + i), 1); mbar_init(wr_bar(sh, B::A_EMPTY + i), 1); }
+        for (int i = 0; i < 3; ++i) {
+            mbar_init(wr_bar(sh, B::ACC1_FULL + i), 1);
+            mbar_init(wr_bar(sh, B::ACC1_EMPTY + i), 1);
+            mbar_init(wr_bar(sh, B::HID_FULL + i), 16);
+        }
+        for (int r = 0; r < 2; ++r) {
+            mbar_init(wr_bar(sh, B::ACC2_FULL + r), 1);
+            mbar_init(wr_bar(sh, B::ACC2_EMPTY + r), 4);
+            mbar_init(wr_bar(sh, B::DRAIN + r), 1);
+        }
+        fence_mbar_init();
+        // the first tile's panels come from DRAM and are what the pass waits for: requested right here
+        if (ntiles > 0)
+            for (int kp = 0; kp < kWrKP; ++kp) {
+                mbar_arrive_expect_tx(wr_bar(sh, B::A_FULL + kp), kWrPanelA);
+                tma_load_2d(sA + kp * kWrPanelA, &tmX, kp * 64, t_begin * kTileM, wr_bar(sh, B::A_FULL + kp));
+            }
+    } else if (threadIdx.x == 64) {
+        prefetch_tensormap(&tmW1);
+        prefetch_tensormap(&tmW2);
+        for (int i = 0; i < kWrKP; ++i) mbar_init(wr_bar(sh, B::W1_FULL + i), 1);
+        mbar_init(wr_bar(sh, B::W2_FULL), 1);
+        fence_mbar_init();
+        if (ntiles > 0) {
+            for (int kp = 0; kp < kWrKP; ++kp) {
+                mbar_arrive_expect_tx(wr_bar(sh, B::W1_FULL + kp), kWrPanelW1);
+                tma_load_2d(sW1 + kp * kWrPanelW1, &tmW1, kp * 64, 0, wr_bar(sh, B::W1_FULL + kp));
+            }
+            mbar_arrive_expect_tx(wr_bar(sh, B::W2_FULL), (uint32_t)((kWrHr / 64) * C::W2_CHUNK));
+            for (int c = 0; c < kWrHr / 64; ++c) tma_load_2d(sW2 + c * C::W2_CHUNK, &tmW2, c * 64, 0, wr_bar(sh, B::W2_FULL));
+        }
+    }
+    for (int e = threadIdx.x; e < kWrMaxE; e += kPpThreads) sh.hist[e] = 0;
+    for (int i = threadIdx.x; i < kWrHr; i += kPpThreads) sh.bias1_f32[i] = p.br1 ? __bfloat162float(p.br1[i]) : 0.0f;
+    for (int i = threadIdx.x; i < EP; i += kPpThreads)
+        sh.bias2_f32[i] = i >= p.experts_real ? -INFINITY : (p.br2 ? __bfloat162float(p.br2[i]) : 0.0f);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp == 0) {
+        // ================= row panels: tile ta's panel kp as soon as tile ta - 1 has let go of it ==========
+        if (lane == 0 && ntiles > 0) {
+            bool ok = true;
+            int requested = kWrKP;                     // panels requested so far (tile 0's: above)
+            for (int ta = 1; ta < ntiles && ok; ++ta) {
+                for (int kp = 0; kp < kWrKP; ++kp) {
+                    if (!mbar_wait(wr_bar(sh, B::A_EMPTY + kp), (uint32_t)(ta - 1) & 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    mbar_arrive_expect_tx(wr_bar(sh, B::A_FULL + kp), kWrPanelA);
+                    tma_load_2d(sA + kp * kWrPanelA, &tmX, kp * 64, (t_begin + ta) * kTileM, wr_bar(sh, B::A_FULL + kp));
+                    ++requested;
+                }
+            }
+            if (!ok || *abort) {
+                // giving up: the copies in flight still have to land before the CTA may leave
+                volatile int never = 0;
+                for (int kp = 0; kp < kWrKP; ++kp) {
+                    mbar_wait(wr_bar(sh, B::W1_FULL + kp), 0u, &never, 10000000ull);
+                    const int last_ta = (requested - 1 - kp) / kWrKP;          // last tile whose panel kp was requested
+                    mbar_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)last_ta & 1u, &never, 10000000ull);
+                }
+                mbar_wait(wr_bar(sh, B::W2_FULL), 0u, &never, 10000000ull);
+            }
+        }
+    } else if (warp == 3) {
+        // ================= GEMM-1 issue (up to two units ahead of GEMM-2: three hidden buffers) ============
+        if (nunits > 0) {
+            constexpr uint32_t idesc1 = make_idesc(128, 128, kFmtBF16, kFmtBF16);
+            const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1);
+            bool ok = true;
+#pragma unroll 1
+            for (int u = 0; u < nunits && ok; ++u) {
+                const int ta = u >> 1, hf = u & 1;
+                const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
+                // (the buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
+                if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b), (n & 1u) ^ 1u, abort)) { ok = false; break; }
+                const uint32_t d = tmem_base + b * C::HB_COLS;
+#pragma unroll
+                for (int kp = 0; kp < kWrKP; ++kp) {
+                    if (hf == 0) {
+                        if (u == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
+                        if (!pp_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)ta & 1u, abort)) { ok = false; break; }
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t a0 = dA + ((kp * kWrPanelA) >> 4);
+                    const uint32_t w0 = dW1 + ((kp * kWrPanelW1 + hf * (128 * 128)) >> 4);
+                    if (elect_one_sync()) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            if (kp == 0 && kk == 0) mma_ss<0>(d, a0, w0, idesc1);
+                            else mma_ss<1>(d, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
+                        }
+                        // the tile's second unit is the last reader of a panel
+                        if (hf == 1) mma_commit(wr_bar(sh, B::A_EMPTY + kp));
+                        if (kp == kWrKP - 1) mma_commit(wr_bar(sh, B::ACC1_FULL + b));
+                    }
+                    __syncwarp();
+                }
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                if (lane == 0) {
+                    mma_commit(wr_bar(sh, B::DRAIN));
+                    mbar_wait(wr_bar(sh, B::DRAIN), 0u, &never, 10000000ull);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 1) {
+        // ================= GEMM-2 issue: logits += hidden(hi) Wr2^T + hidden(lo) Wr2^T ========================
+        if (nunits > 0) {
+            constexpr uint32_t idesc2 = make_idesc(128, EP, kFmtBF16, kFmtBF16);
+            const uint32_t dW2 = desc_lo_sw128(sW2);
+            bool ok = pp_wait(wr_bar(sh, B::W2_FULL), 0u, abort);
+#pragma unroll 1
+            for (int u = 0; u < nunits && ok; ++u) {
+                const int ta = u >> 1, hf = u & 1;
+                const int r = ta & 1;
+                if (hf == 0 && !pp_wait(wr_bar(sh, B::ACC2_EMPTY + r), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
+                const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
+                if (!pp_wait(wr_bar(sh, B::HID_FULL + b), n & 1u, abort)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t w0 = dW2 + ((hf * 2 * C::W2_CHUNK) >> 4);
+                const uint32_t d = tmem_base + C::LOGIT_COL + r * 64, a = tmem_base + b * C::HB_COLS;
+                if (elect_one_sync()) {
+                    // K step kk of the unit: hi halves in columns 16 kk .. 16 kk + 7, lo halves in the next eight
+#pragma unroll
+                    for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t bd = w0 + (((kk >> 2) * C::W2_CHUNK + (kk & 3) * 32) >> 4);
+                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, hf > 0 ? 1u : 0u);
+                            else mma_ts<1>(d, a + kk * 16 + part * 8, bd, idesc2);
+                        }
+                    }
+                    mma_commit(wr_bar(sh, B::ACC1_EMPTY + b));
+                    if (hf == 1) mma_commit(wr_bar(sh, B::ACC2_FULL + r));
+                }
+                __syncwarp();
+            }
+            if (!ok || *abort) {
+                volatile int never = 0;
+                if (lane == 0) {
+                    mma_commit(wr_bar(sh, B::DRAIN + 1));
+                    mbar_wait(wr_bar(sh, B::DRAIN + 1), 0u, &never, 10000000ull);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 2) {
+        // ================= zero this CTA's rows of h' ========================================================
+        if (p.zero_out != nullptr && ntiles > 0) {
+            const long long row_lo = (long long)t_begin * kTileM;
+            long long row_hi = (long long)(t_begin + ntiles) * kTileM;
+            if (row_hi > p.n_rows) row_hi = p.n_rows;
+            uint4* dst = reinterpret_cast<uint4*>(p.zero_out + row_lo * p.row_elems);
+            const long long nvec = (row_hi - row_lo) * p.row_elems / 8;
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            for (long long i = lane; i < nvec; i += 32) dst[i] = z;
+        }
+    } else if (warp < 20) {
+        // ================= activation warps: warpgroup g, lane group lg ======================================
+        const int g = (warp - 4) >> 2;
+        const int lg = warp & 3;
+        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + 32 * g;
+        const bool has_br1 = p.br1 != nullptr;
+        bool ok = true;
+#pragma unroll 1
+        for (int u = 0; u < nunits && ok; ++u) {
+            const int hf = u & 1;
+            const uint32_t b = (uint32_t)u % 3u, par = ((uint32_t)u / 3u) & 1u;
+            ok = pp_wait(wr_bar(sh, B::ACC1_FULL + b), par, abort);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t acol = tlane + b * C::HB_COLS;
+            const float* bias = sh.bias1_f32 + hf * 128 + 32 * g;
+            // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu), lo = the
+            // rounded remainder (for a negative value the remainder is the value itself and its .relu is 0 too)
+            uint32_t acc32[32];
+            tmem_ld_x32(acol, acc32);
+            tmem_ld_wait();
+#pragma unroll
+            for (int pc = 0; pc < 2; ++pc) {
+                const uint32_t* acc = acc32 + 16 * pc;
+                float a[16];
+                if (has_br1) {
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        const float4 bb = *reinterpret_cast<const float4*>(bias + pc * 16 + i);
+                        add2(a[i], a[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), bb.x, bb.y);
+                        add2(a[i + 2], a[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), bb.z, bb.w);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) a[i] = __uint_as_float(acc[i]);
+                }
+                uint32_t hl[16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) hl[i] = cvt_rz_relu_bf16x2(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    hl[8 + i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hl[i] << 16), a[2 * i + 1] - __uint_as_float(hl[i] & 0xFFFF0000u));
+                tmem_st_x16(acol + 16 * pc, hl);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(wr_bar(sh, B::HID_FULL + b));
+        }
+    } else {
+        // ================= output warpgroup: softmax + top-k of a tile's logits ==============================
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + C::LOGIT_COL;
+        bool ok = true;
+#pragma unroll 1
+        for (int ta = 0; ta < ntiles && ok; ++ta) {
+            const int r = ta & 1;
+            ok = pp_wait(wr_bar(sh, B::ACC2_FULL + r), (uint32_t)(ta >> 1) & 1u, abort);
+            if (!ok) break;
+            tc_fence_after_sync();
+            uint32_t v[EP];
+#pragma unroll
+            for (int c = 0; c < EP; c += 16) tmem_ld_x16(tlane + r * 64 + c, v + c);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(wr_bar(sh, B::ACC2_EMPTY + r));
+            const int n = (t_begin + ta) * kTileM + row;
+            const bool valid = n < p.n_rows;
+            // one pass keeping the best two (strict comparisons in ascending id order: the picks of repeated
+            // arg-max with ties to the lower id); the logits stay in v as raw bits + bias
+            float b1 = -INFINITY, b2 = -INFINITY;
+            int i1 = 0, i2 = 0;
+#pragma unroll
+            for (int i = 0; i < EP; ++i) {
+                const float gl = __uint_as_float(v[i]) + sh.bias2_f32[i];
+                v[i] = __float_as_uint(gl);
+                const bool gt1 = gl > b1, gt2 = gl > b2;
+                b2 = gt1 ? b1 : (gt2 ? gl : b2);
+                i2 = gt1 ? i1 : (gt2 ? i : i2);
+                b1 = gt1 ? gl : b1;
+                i1 = gt1 ? i : i1;
+            }
+            const float sc = p.softmax_scale;
+            const float msc = b1 * sc;
+            float sum = 0.0f;
+#pragma unroll
+            for (int i = 0; i < EP; ++i) sum += ex2_approx(fmaf(__uint_as_float(v[i]), sc, -msc));
+            const float inv = 1.0f / sum;
+            const float p2 = ex2_approx(fmaf(b2, sc, -msc)) * inv;
+            if (valid) {
+                const size_t at = (size_t)n * p.k;
+                atomicAdd(&sh.hist[i1], 1);
+                if (p.k > 1) {
+                    *reinterpret_cast<int2*>(p.topk_idx + at) = make_int2(i1, i2);
+                    *reinterpret_cast<float2*>(p.topk_p + at) = make_float2(inv, p2);
+                    atomicAdd(&sh.hist[i2], 1);
+                } else {
+                    p.topk_idx[at] = i1;
+                    p.topk_p[at] = inv;
+                }
+            }
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh.abort_flag) atomicExch(p.status, (int)SLICEMOE_ERR_DEVICE_TIMEOUT);
+    if (p.cta_hist)
+        for (int i = threadIdx.x; i < p.experts_real; i += kPpThreads) p.cta_hist[(size_t)blockIdx.x * p.experts_real + i] = sh.hist[i];
+    if (p.assigned_out && ntiles > 0)
+        for (int i = threadIdx.x; i < p.experts_real; i += kPpThreads)
+            if (sh.hist[i] > 0) atomicAdd(p.assigned_out + i, sh.hist[i]);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(sh.tmem_base, 512);
+    }
+}
+
+template <int EP>
+int launch_wide(const Dims& D, const slicemoe_weights& w, const void* h, const PpParams& rp, int grid, cudaStream_t st) {
+    CUtensorMap mX, mW1, mW2;
+    int rc;
+    // (rows of 192 elements: the boxes reach past the tensors' edge and are zero-filled there)
+    if ((rc = make_tmap(&mX, h, (uint64_t)D.N, (uint64_t)D.ds, kTileM))) return rc;
+    if ((rc = make_tmap(&mW1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, kWrHr))) return rc;
+    if ((rc = make_tmap(&mW2, w.Wr2, (uint64_t)D.E, (uint64_t)D.Hr, EP))) return rc;      // (E = 8: zero-filled up to 16)
+    auto kern = route_wide_kernel<EP>;
+    static bool attr_set[kAttrMaxDevices] = {};
+    static std::mutex attr_mutex;
+    {
+        std::lock_guard<std::mutex> lock(attr_mutex);
+        if ((rc = set_smem_limit_once(kern, WrCfg<EP>::SMEM_ALLOC, attr_set))) return rc;
+    }
+    kern<<<grid, kPpThreads, WrCfg<EP>::SMEM_ALLOC, st>>>(mX, mW1, mW2, rp);
+    SLICEMOE_LAUNCH_CHECK(1);
+    return SLICEMOE_OK;
+}
+
+}  // namespace
+
+bool wide_route_supported(const Dims& D) {
+    if (D.dtype != SLICEMOE_BF16 || (D.ds != 256 && D.ds != 192) || D.N <= 0) return false;
+    if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
+    if (D.k > 2 || D.noise_sigma > 0.0f) return false;
+    return D.Hr == kWrHr;
+}
+
+int launch_route_wide(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx, float* topk_p,
+                      int32_t* assigned, int32_t* status, cudaStream_t st, int32_t* cta_hist, void* zero_out,
+                      int grid_rows) {
+    if (assigned) SLICEMOE_CUDA_TRY(cudaMemsetAsync(assigned, 0, sizeof(int32_t) * D.E, st));
+    PpParams r{};
+    r.status = status; r.n_rows = D.N; r.HID = D.Hr; r.experts_real = D.E; r.k = D.k;
+    r.softmax_scale = 1.4426950408889634f * D.inv_tau;
+    r.br1 = (const bf16*)w.br1; r.br2 = (const bf16*)w.br2;
+    r.topk_idx = topk_idx; r.topk_p = topk_p;
+    r.assigned_out = assigned; r.cta_hist = cta_hist;
+    r.zero_out = (bf16*)zero_out; r.row_elems = D.ds;
+    // The rows are split over the CTAs as tc_route_grid says (CTAs past the last tile have none); with grid_rows the
+    // launch has that many CTAs, each of which writes its row of cta_hist (zeros where it has no tile).
+    int grid = 0, rows_per_cta = 0;
+    tc_route_grid(D, &grid, &rows_per_cta);
+    if (grid_rows > grid) grid = grid_rows;
+    switch (D.E) {
+        case 8:
+        case 16: return launch_wide<16>(D, w, h, r, grid, st);
+        case 32: return launch_wide<32>(D, w, h, r, grid, st);
+        case 64: return launch_wide<64>(D, w, h, r, grid, st);
+        default: return SLICEMOE_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace slicemoe

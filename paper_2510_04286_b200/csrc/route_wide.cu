@@ -163,36 +163,53 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             }
         }
     } else if (warp == 3) {
-        // ================= GEMM-1 issue (up to two units ahead of GEMM-2: three hidden buffers) ============
+        // ================= GEMM-1 issue ======================================================================
+        // A tile's two units are issued panel by panel, both units on a panel before the next panel: the tile is
+        // then done with a panel -- and the next tile's copy of it can start -- eight MMAs after the panel has
+        // landed, while the tile's other panels are still on their way, so the row loads never pause.  (Unit by
+        // unit, all four panels would be released in a burst at the tile's end and requested in a burst.)
         if (nunits > 0) {
             constexpr uint32_t idesc1 = make_idesc(128, 128, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1);
             bool ok = true;
 #pragma unroll 1
-            for (int u = 0; u < nunits && ok; ++u) {
-                const int ta = u >> 1, hf = u & 1;
-                const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
-                // (the buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
-                if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b), (n & 1u) ^ 1u, abort)) { ok = false; break; }
-                const uint32_t d = tmem_base + b * C::HB_COLS;
+            for (int ta = 0; ta < ntiles && ok; ++ta) {
+                const uint32_t u0 = 2u * (uint32_t)ta, u1 = u0 + 1u;
+                const uint32_t b0 = u0 % 3u, b1 = u1 % 3u;
+                // (a buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
+                if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b0), ((u0 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
+                const uint32_t d0 = tmem_base + b0 * C::HB_COLS, d1 = tmem_base + b1 * C::HB_COLS;
 #pragma unroll
                 for (int kp = 0; kp < kWrKP; ++kp) {
-                    if (hf == 0) {
-                        if (u == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
-                        if (!pp_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)ta & 1u, abort)) { ok = false; break; }
-                    }
+                    if (ta == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
+                    if (!pp_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)ta & 1u, abort)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t a0 = dA + ((kp * kWrPanelA) >> 4);
-                    const uint32_t w0 = dW1 + ((kp * kWrPanelW1 + hf * (128 * 128)) >> 4);
+                    const uint32_t w0 = dW1 + ((kp * kWrPanelW1) >> 4), w1 = w0 + ((128 * 128) >> 4);
                     if (elect_one_sync()) {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk) {
-                            if (kp == 0 && kk == 0) mma_ss<0>(d, a0, w0, idesc1);
-                            else mma_ss<1>(d, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
+                            if (kp == 0 && kk == 0) mma_ss<0>(d0, a0, w0, idesc1);
+                            else mma_ss<1>(d0, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
                         }
-                        // the tile's second unit is the last reader of a panel
-                        if (hf == 1) mma_commit(wr_bar(sh, B::A_EMPTY + kp));
-                        if (kp == kWrKP - 1) mma_commit(wr_bar(sh, B::ACC1_FULL + b));
+                    }
+                    __syncwarp();
+                    // (the second unit's buffer is the one the previous tile's first unit is still in)
+                    if (kp == 0) {
+                        if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b1), ((u1 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
+                        tc_fence_after_sync();
+                    }
+                    if (elect_one_sync()) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            if (kp == 0 && kk == 0) mma_ss<0>(d1, a0, w1, idesc1);
+                            else mma_ss<1>(d1, a0 + ((kk * 32) >> 4), w1 + ((kk * 32) >> 4), idesc1);
+                        }
+                        mma_commit(wr_bar(sh, B::A_EMPTY + kp));
+                        if (kp == kWrKP - 1) {
+                            mma_commit(wr_bar(sh, B::ACC1_FULL + b0));
+                            mma_commit(wr_bar(sh, B::ACC1_FULL + b1));
+                        }
                     }
                     __syncwarp();
                 }

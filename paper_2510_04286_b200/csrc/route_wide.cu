@@ -36,6 +36,7 @@ struct WrShared {
     int hist[kWrMaxE];
     uint32_t tmem_base;
     int abort_flag;
+    int tiles_out;               // tiles whose top-k has been written (paces the zeroing of h')
     __align__(16) float bias1_f32[kWrHr];
     __align__(16) float bias2_f32[kWrMaxE];
 };
@@ -96,6 +97,7 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     if (threadIdx.x == 0) {
         prefetch_tensormap(&tmX);
         sh.abort_flag = 0;
+        sh.tiles_out = 0;
         for (int i = 0; i < kWrKP; ++i) { mbar_init(wr_bar(sh, B::A_FULL + i), 1); mbar_init(wr_bar(sh, B::A_EMPTY + i), 1); }
         for (int i = 0; i < 3; ++i) {
             mbar_init(wr_bar(sh, B::ACC1_FULL + i), 1);
@@ -266,14 +268,32 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         }
     } else if (warp == 2) {
         // ================= zero this CTA's rows of h' ========================================================
-        if (p.zero_out != nullptr && ntiles > 0) {
-            const long long row_lo = (long long)t_begin * kTileM;
-            long long row_hi = (long long)(t_begin + ntiles) * kTileM;
-            if (row_hi > p.n_rows) row_hi = p.n_rows;
-            uint4* dst = reinterpret_cast<uint4*>(p.zero_out + row_lo * p.row_elems);
-            const long long nvec = (row_hi - row_lo) * p.row_elems / 8;
+        // Tile by tile, at the pace of the tiles' results (two tiles ahead of the output warps): written in one
+        // burst at the start, the 2 x 64 KB per tile that this pass writes crowd out the row loads of the first
+        // tiles, whose latency is on the critical path of a pipeline with a single row-tile buffer.
+        if (p.zero_out != nullptr) {
             const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            for (long long i = lane; i < nvec; i += 32) dst[i] = z;
+            volatile int* done = &sh.tiles_out;
+            bool ok = true;
+#pragma unroll 1
+            for (int ta = 0; ta < ntiles && ok; ++ta) {
+                if (ta >= 2 && *done < ta - 1) {
+                    const uint64_t t0 = globaltimer_ns();
+                    while (*done < ta - 1) {
+                        __nanosleep(256);
+                        if (*abort || globaltimer_ns() - t0 > kWaitLimitNs) { ok = false; break; }
+                    }
+                    if (!ok) break;
+                }
+                const long long row_lo = (long long)(t_begin + ta) * kTileM;
+                long long row_hi = row_lo + kTileM;
+                if (row_hi > p.n_rows) row_hi = p.n_rows;
+                uint4* dst = reinterpret_cast<uint4*>(p.zero_out + row_lo * p.row_elems);
+                const int nvec = (int)(row_hi - row_lo) * p.row_elems / 8;
+#pragma unroll 4
+                for (int i = lane; i < nvec; i += 32) dst[i] = z;
+            }
+            // (a pass that gave up leaves its status word set; the rows not zeroed are then not results)
         }
     } else if (warp < 20) {
         // ================= activation warps: warpgroup g, lane group lg ======================================
@@ -366,6 +386,7 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             for (int i = 0; i < EP; ++i) sum += ex2_approx(fmaf(__uint_as_float(v[i]), sc, -msc));
             const float inv = 1.0f / sum;
             const float p2 = ex2_approx(fmaf(b2, sc, -msc)) * inv;
+            if (lane == 0 && lg == 0) sh.tiles_out = ta + 1;
             if (valid) {
                 const size_t at = (size_t)n * p.k;
                 atomicAdd(&sh.hist[i1], 1);

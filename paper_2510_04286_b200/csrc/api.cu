@@ -183,9 +183,11 @@ static int forward_impl(const Dims& D, const slicemoe_weights& w, const void* h,
     if (!events && !D.train_gates && decode_forward_supported(D))
         return launch_forward_decode(D, w, h, h_out, idx, p, assigned, kept, xperm, at<int32_t>(ws, W.status), clear_status, st);
     const bool one_launch = !events && !D.train_gates && fused_forward_supported(D);
-    // wide slices: the router is a launch of its own (its resident weights leave no shared memory for the other
-    // phases' state), the single kernel takes over at the dispatch
-    const bool wide = wide_route_supported(D);
+    // The router with resident weights is a launch of its own (its weights leave no shared memory for the other
+    // phases' state) and the single kernel then takes over at the dispatch.  Rows of 192 / 256: 15 % faster than
+    // the single kernel alone.  Rows of 96 / 128: the shorter router (31 -> 23 us on 131 072 rows of 96) and the
+    // second launch cancel, so the forward stays one launch there and only the stage-by-stage forms use it.
+    const bool wide = wide_route_supported(D) && (D.ds > 128 || !one_launch);
     // (the single kernel clears the status word itself; a later chunk of one host-buffer call keeps
     // what an earlier chunk reported)
     if ((!one_launch || wide) && clear_status && (rc = reset_status(ws, W, st))) return rc;

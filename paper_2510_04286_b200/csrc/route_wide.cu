@@ -1,18 +1,23 @@
-// Router of wide slices (Section 3.1: relu(X Wr1^T + br1) Wr2^T + br2 -> softmax -> top-k), bf16 storage, rows of
-// 192 or 256 elements, router hidden width 256, up to 64 experts, k <= 2 (sm_100a: tcgen05 + TMEM + TMA).
+// Router of slices of 96 to 256 elements (Section 3.1: relu(X Wr1^T + br1) Wr2^T + br2 -> softmax -> top-k), bf16
+// storage, router hidden width 256, up to 64 experts, k <= 2 (sm_100a: tcgen05 + TMEM + TMA).
 //
-// The whole of Wr1 (128 KB) and Wr2 stay in shared memory for the life of the CTA, so a tile's GEMM-1 runs as
+// The whole of Wr1 (up to 128 KB) and Wr2 stay in shared memory for the life of the CTA, so a tile's GEMM-1 runs as
 // 128-wide MMAs against operands that are written to shared memory once per launch, not once per tile: what a tile
-// moves through shared memory is its own 64 KB of rows and the operand reads of its MMAs.  That leaves room for
-// exactly ONE row tile, held as four 64-column panels with a full / empty barrier pair each: a panel is handed back
-// as soon as the tile's last MMAs on it have completed and the next tile's panel is requested at once, so the row
-// loads run a whole tile ahead of their use although only one tile's worth of shared memory exists.
+// moves through shared memory is its own rows and the operand reads of its MMAs.  Rows come as 64-column panels
+// with a full / empty barrier pair each:
+//   rows of 192 / 256 (four panels, Wr1 = 128 KB)   there is room for exactly ONE row tile.  A tile's two units are
+//       therefore issued panel by panel, both units on a panel before the next panel: the tile is done with a panel,
+//       and the next tile's copy of it is requested, eight MMAs after the panel has landed, while the tile's other
+//       panels are still on their way -- the row loads run a whole tile ahead although only one tile's worth of
+//       shared memory exists.
+//   rows of 96 / 128 (two panels, Wr1 = 64 KB)      three row tiles fit; the units are issued one after the other,
+//       GEMM-1 up to two units ahead of GEMM-2, and the loads run three tiles ahead.
 //
 // One CTA of 768 threads per SM walks a contiguous range of 128-row tiles.  A tile is two units of 128 hidden
-// columns; three 128-column buffers of tensor memory take the units in turn (GEMM-1 runs up to two units ahead of
-// GEMM-2), the activation warps turn a buffer's fp32 values in place into a truncated bf16 and the rounded remainder
-// (GEMM-2 runs over both, so the logits keep fp32-level accuracy and the top-k decision does not hang on a bf16
-// rounding of the hidden layer), GEMM-2 reads them from tensor memory.  Warp roles:
+// columns; three 128-column buffers of tensor memory take the units in turn, the activation warps turn a buffer's
+// fp32 values in place into a truncated bf16 and the rounded remainder (GEMM-2 runs over both, so the logits keep
+// fp32-level accuracy and the top-k decision does not hang on a bf16 rounding of the hidden layer), GEMM-2 reads them
+// from tensor memory.  Warp roles:
 //   warp 0       row panels by TMA          warp 3  GEMM-1 issue        warp 1  GEMM-2 issue
 //   warp 2       zeroes this CTA's rows of h' (forward: the experts add into it)
 //   warps 4-19   activation (four warpgroups, 32 of a unit's 128 columns each; a thread owns one tile row)
@@ -25,11 +30,12 @@
 namespace slicemoe {
 namespace {
 
-constexpr int kWrKP = 4;                      // 64-column panels of a row tile
 constexpr int kWrHr = 256;                    // router hidden width
 constexpr int kWrPanelA = kTileM * 128;       // bytes: 128 rows x 64 bf16
 constexpr int kWrPanelW1 = kWrHr * 128;       // bytes: 256 hidden units x 64 bf16
 constexpr int kWrMaxE = 64;
+constexpr int kWrMaxSlots = 6;                // row-panel slots: 1 tile x 4 panels or 3 tiles x 2 panels
+constexpr int kWrMaxKP = 4;
 
 struct WrShared {
     __align__(8) uint64_t bars[32];
@@ -42,10 +48,10 @@ struct WrShared {
 };
 
 struct WrBars {
-    static constexpr int A_FULL = 0;                        // [kWrKP]
-    static constexpr int A_EMPTY = A_FULL + kWrKP;          // [kWrKP]
-    static constexpr int W1_FULL = A_EMPTY + kWrKP;         // [kWrKP] one per K panel of Wr1
-    static constexpr int W2_FULL = W1_FULL + kWrKP;
+    static constexpr int A_FULL = 0;                        // [slots]
+    static constexpr int A_EMPTY = A_FULL + kWrMaxSlots;    // [slots]
+    static constexpr int W1_FULL = A_EMPTY + kWrMaxSlots;   // [KP] one per K panel of Wr1
+    static constexpr int W2_FULL = W1_FULL + kWrMaxKP;
     static constexpr int ACC1_FULL = W2_FULL + 1;           // [3]
     static constexpr int ACC1_EMPTY = ACC1_FULL + 3;        // [3]
     static constexpr int HID_FULL = ACC1_EMPTY + 3;         // [3]
@@ -56,27 +62,34 @@ struct WrBars {
 };
 static_assert(WrBars::COUNT <= 32, "barrier slots");
 
-template <int EP>
+// EP: experts (padded), KP: 64-column panels of a row tile
+template <int EP, int KP>
 struct WrCfg {
+    static constexpr int NT = KP == 4 ? 1 : 3;              // row tiles in shared memory
+    static constexpr int SLOTS = NT * KP;
     static constexpr int W2_CHUNK = EP * 128;               // bytes: EP experts x 64 hidden units
     static constexpr int OFF_A = 0;
-    static constexpr int OFF_W1 = OFF_A + kWrKP * kWrPanelA;
-    static constexpr int OFF_W2 = OFF_W1 + kWrKP * kWrPanelW1;
+    static constexpr int OFF_W1 = OFF_A + SLOTS * kWrPanelA;
+    static constexpr int OFF_W2 = OFF_W1 + KP * kWrPanelW1;
     static constexpr int SMEM_BYTES = OFF_W2 + (kWrHr / 64) * W2_CHUNK;
-    static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;
+    // (at least 120 KB so that two CTAs never share an SM: each allocates all of tensor memory)
+    static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024 > 120 * 1024 ? SMEM_BYTES + 1024 : 120 * 1024;
     static constexpr int HB_COLS = 128, LOGIT_COL = 384;
+    static_assert(KP == 2 || KP == 4, "row width");
+    static_assert(SLOTS <= kWrMaxSlots && KP <= kWrMaxKP, "barrier slots");
     static_assert(SMEM_ALLOC + sizeof(WrShared) + 64 <= 232448, "shared memory budget");
     static_assert(EP % 16 == 0 && EP <= kWrMaxE, "expert count");
 };
 
 __device__ __forceinline__ uint32_t wr_bar(WrShared& sh, int i) { return smem_u32(&sh.bars[i]); }
 
-template <int EP>
+template <int EP, int KP>
 __global__ void __launch_bounds__(kPpThreads, 1)
 route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
                   const __grid_constant__ CUtensorMap tmW2, const PpParams p) {
-    using C = WrCfg<EP>;
+    using C = WrCfg<EP, KP>;
     using B = WrBars;
+    constexpr int NT = C::NT;
     extern __shared__ uint8_t smem_raw[];
     __shared__ WrShared sh;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -98,7 +111,7 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         prefetch_tensormap(&tmX);
         sh.abort_flag = 0;
         sh.tiles_out = 0;
-        for (int i = 0; i < kWrKP; ++i) { mbar_init(wr_bar(sh, B::A_FULL + i), 1); mbar_init(wr_bar(sh, B::A_EMPTY + i), 1); }
+        for (int i = 0; i < C::SLOTS; ++i) { mbar_init(wr_bar(sh, B::A_FULL + i), 1); mbar_init(wr_bar(sh, B::A_EMPTY + i), 1); }
         for (int i = 0; i < 3; ++i) {
             mbar_init(wr_bar(sh, B::ACC1_FULL + i), 1);
             mbar_init(wr_bar(sh, B::ACC1_EMPTY + i), 1);
@@ -110,20 +123,20 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             mbar_init(wr_bar(sh, B::DRAIN + r), 1);
         }
         fence_mbar_init();
-        // the first tile's panels come from DRAM and are what the pass waits for: requested right here
-        if (ntiles > 0)
-            for (int kp = 0; kp < kWrKP; ++kp) {
-                mbar_arrive_expect_tx(wr_bar(sh, B::A_FULL + kp), kWrPanelA);
-                tma_load_2d(sA + kp * kWrPanelA, &tmX, kp * 64, t_begin * kTileM, wr_bar(sh, B::A_FULL + kp));
+        // the first tiles' panels come from DRAM and are what the pass waits for: requested right here
+        for (int ta = 0; ta < min(ntiles, NT); ++ta)
+            for (int kp = 0; kp < KP; ++kp) {
+                mbar_arrive_expect_tx(wr_bar(sh, B::A_FULL + ta * KP + kp), kWrPanelA);
+                tma_load_2d(sA + (ta * KP + kp) * kWrPanelA, &tmX, kp * 64, (t_begin + ta) * kTileM, wr_bar(sh, B::A_FULL + ta * KP + kp));
             }
     } else if (threadIdx.x == 64) {
         prefetch_tensormap(&tmW1);
         prefetch_tensormap(&tmW2);
-        for (int i = 0; i < kWrKP; ++i) mbar_init(wr_bar(sh, B::W1_FULL + i), 1);
+        for (int i = 0; i < KP; ++i) mbar_init(wr_bar(sh, B::W1_FULL + i), 1);
         mbar_init(wr_bar(sh, B::W2_FULL), 1);
         fence_mbar_init();
         if (ntiles > 0) {
-            for (int kp = 0; kp < kWrKP; ++kp) {
+            for (int kp = 0; kp < KP; ++kp) {
                 mbar_arrive_expect_tx(wr_bar(sh, B::W1_FULL + kp), kWrPanelW1);
                 tma_load_2d(sW1 + kp * kWrPanelW1, &tmW1, kp * 64, 0, wr_bar(sh, B::W1_FULL + kp));
             }
@@ -141,79 +154,115 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const uint32_t tmem_base = sh.tmem_base;
 
     if (warp == 0) {
-        // ================= row panels: tile ta's panel kp as soon as tile ta - 1 has let go of it ==========
+        // ================= row panels: a tile's panel as soon as the tile NT back has let go of its slot =====
         if (lane == 0 && ntiles > 0) {
             bool ok = true;
-            int requested = kWrKP;                     // panels requested so far (tile 0's: above)
-            for (int ta = 1; ta < ntiles && ok; ++ta) {
-                for (int kp = 0; kp < kWrKP; ++kp) {
-                    if (!mbar_wait(wr_bar(sh, B::A_EMPTY + kp), (uint32_t)(ta - 1) & 1u, abort, kWaitLimitNs)) { ok = false; break; }
-                    mbar_arrive_expect_tx(wr_bar(sh, B::A_FULL + kp), kWrPanelA);
-                    tma_load_2d(sA + kp * kWrPanelA, &tmX, kp * 64, (t_begin + ta) * kTileM, wr_bar(sh, B::A_FULL + kp));
+            int requested = min(ntiles, NT) * KP;             // panels requested so far (the first tiles': above)
+            for (int ta = NT; ta < ntiles && ok; ++ta) {
+                const int sb = (ta % NT) * KP;
+                for (int kp = 0; kp < KP; ++kp) {
+                    if (!mbar_wait(wr_bar(sh, B::A_EMPTY + sb + kp), ((uint32_t)(ta / NT) & 1u) ^ 1u, abort, kWaitLimitNs)) { ok = false; break; }
+                    mbar_arrive_expect_tx(wr_bar(sh, B::A_FULL + sb + kp), kWrPanelA);
+                    tma_load_2d(sA + (sb + kp) * kWrPanelA, &tmX, kp * 64, (t_begin + ta) * kTileM, wr_bar(sh, B::A_FULL + sb + kp));
                     ++requested;
                 }
             }
             if (!ok || *abort) {
-                // giving up: the copies in flight still have to land before the CTA may leave
+                // giving up: the copies in flight still have to land before the CTA may leave (the last SLOTS
+                // requests cover every slot once)
                 volatile int never = 0;
-                for (int kp = 0; kp < kWrKP; ++kp) {
-                    mbar_wait(wr_bar(sh, B::W1_FULL + kp), 0u, &never, 10000000ull);
-                    const int last_ta = (requested - 1 - kp) / kWrKP;          // last tile whose panel kp was requested
-                    mbar_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)last_ta & 1u, &never, 10000000ull);
-                }
+                for (int kp = 0; kp < KP; ++kp) mbar_wait(wr_bar(sh, B::W1_FULL + kp), 0u, &never, 10000000ull);
                 mbar_wait(wr_bar(sh, B::W2_FULL), 0u, &never, 10000000ull);
+                for (int q = requested - 1; q >= 0 && q >= requested - C::SLOTS; --q) {
+                    const int ta = q / KP;
+                    mbar_wait(wr_bar(sh, B::A_FULL + (ta % NT) * KP + q % KP), (uint32_t)(ta / NT) & 1u, &never, 10000000ull);
+                }
             }
         }
     } else if (warp == 3) {
         // ================= GEMM-1 issue ======================================================================
-        // A tile's two units are issued panel by panel, both units on a panel before the next panel: the tile is
-        // then done with a panel -- and the next tile's copy of it can start -- eight MMAs after the panel has
-        // landed, while the tile's other panels are still on their way, so the row loads never pause.  (Unit by
-        // unit, all four panels would be released in a burst at the tile's end and requested in a burst.)
         if (nunits > 0) {
             constexpr uint32_t idesc1 = make_idesc(128, 128, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1);
             bool ok = true;
+            if constexpr (NT == 1) {
+                // One row tile in shared memory: both units of a tile panel by panel, so that a panel is released
+                // eight MMAs after it has landed.  (Unit by unit, all panels would be released in a burst at the
+                // tile's end and requested in a burst: measured, 5 % slower.  Letting the first unit run ahead on
+                // the panels that are there while the second unit's buffer is busy: measured, slower too -- its
+                // MMAs queue in front of the GEMM-2 that frees that buffer.)
 #pragma unroll 1
-            for (int ta = 0; ta < ntiles && ok; ++ta) {
-                const uint32_t u0 = 2u * (uint32_t)ta, u1 = u0 + 1u;
-                const uint32_t b0 = u0 % 3u, b1 = u1 % 3u;
-                // (a buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
-                if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b0), ((u0 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
-                const uint32_t d0 = tmem_base + b0 * C::HB_COLS, d1 = tmem_base + b1 * C::HB_COLS;
+                for (int ta = 0; ta < ntiles && ok; ++ta) {
+                    const uint32_t u0 = 2u * (uint32_t)ta, u1 = u0 + 1u;
+                    const uint32_t b0 = u0 % 3u, b1 = u1 % 3u;
+                    // (a buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
+                    if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b0), ((u0 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
+                    const uint32_t d0 = tmem_base + b0 * C::HB_COLS, d1 = tmem_base + b1 * C::HB_COLS;
 #pragma unroll
-                for (int kp = 0; kp < kWrKP; ++kp) {
-                    if (ta == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
-                    if (!pp_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)ta & 1u, abort)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t a0 = dA + ((kp * kWrPanelA) >> 4);
-                    const uint32_t w0 = dW1 + ((kp * kWrPanelW1) >> 4), w1 = w0 + ((128 * 128) >> 4);
-                    if (elect_one_sync()) {
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            if (kp == 0 && kk == 0) mma_ss<0>(d0, a0, w0, idesc1);
-                            else mma_ss<1>(d0, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
-                        }
-                    }
-                    __syncwarp();
-                    // (the second unit's buffer is the one the previous tile's first unit is still in)
-                    if (kp == 0) {
-                        if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b1), ((u1 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
+                    for (int kp = 0; kp < KP; ++kp) {
+                        if (ta == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
+                        if (!pp_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)ta & 1u, abort)) { ok = false; break; }
                         tc_fence_after_sync();
-                    }
-                    if (elect_one_sync()) {
+                        const uint32_t a0 = dA + ((kp * kWrPanelA) >> 4);
+                        const uint32_t w0 = dW1 + ((kp * kWrPanelW1) >> 4), w1 = w0 + ((128 * 128) >> 4);
+                        if (elect_one_sync()) {
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            if (kp == 0 && kk == 0) mma_ss<0>(d1, a0, w1, idesc1);
-                            else mma_ss<1>(d1, a0 + ((kk * 32) >> 4), w1 + ((kk * 32) >> 4), idesc1);
+                            for (int kk = 0; kk < 4; ++kk) {
+                                if (kp == 0 && kk == 0) mma_ss<0>(d0, a0, w0, idesc1);
+                                else mma_ss<1>(d0, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
+                            }
                         }
-                        mma_commit(wr_bar(sh, B::A_EMPTY + kp));
-                        if (kp == kWrKP - 1) {
-                            mma_commit(wr_bar(sh, B::ACC1_FULL + b0));
-                            mma_commit(wr_bar(sh, B::ACC1_FULL + b1));
+                        __syncwarp();
+                        // (the second unit's buffer is the one the previous tile's first unit is still in)
+                        if (kp == 0) {
+                            if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b1), ((u1 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
+                            tc_fence_after_sync();
                         }
+                        if (elect_one_sync()) {
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) {
+                                if (kp == 0 && kk == 0) mma_ss<0>(d1, a0, w1, idesc1);
+                                else mma_ss<1>(d1, a0 + ((kk * 32) >> 4), w1 + ((kk * 32) >> 4), idesc1);
+                            }
+                            mma_commit(wr_bar(sh, B::A_EMPTY + kp));
+                            if (kp == KP - 1) {
+                                mma_commit(wr_bar(sh, B::ACC1_FULL + b0));
+                                mma_commit(wr_bar(sh, B::ACC1_FULL + b1));
+                            }
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
+                }
+            } else {
+                // Several row tiles in shared memory: unit by unit, up to two units ahead of GEMM-2.
+#pragma unroll 1
+                for (int u = 0; u < nunits && ok; ++u) {
+                    const int ta = u >> 1, hf = u & 1;
+                    const int sb = (ta % NT) * KP;
+                    const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
+                    if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b), (n & 1u) ^ 1u, abort)) { ok = false; break; }
+                    const uint32_t d = tmem_base + b * C::HB_COLS;
+#pragma unroll
+                    for (int kp = 0; kp < KP; ++kp) {
+                        if (hf == 0) {
+                            if (u == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
+                            if (!pp_wait(wr_bar(sh, B::A_FULL + sb + kp), (uint32_t)(ta / NT) & 1u, abort)) { ok = false; break; }
+                        }
+                        tc_fence_after_sync();
+                        const uint32_t a0 = dA + (((sb + kp) * kWrPanelA) >> 4);
+                        const uint32_t w0 = dW1 + ((kp * kWrPanelW1 + hf * (128 * 128)) >> 4);
+                        if (elect_one_sync()) {
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) {
+                                if (kp == 0 && kk == 0) mma_ss<0>(d, a0, w0, idesc1);
+                                else mma_ss<1>(d, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
+                            }
+                            // the tile's second unit is the last reader of a panel
+                            if (hf == 1) mma_commit(wr_bar(sh, B::A_EMPTY + sb + kp));
+                            if (kp == KP - 1) mma_commit(wr_bar(sh, B::ACC1_FULL + b));
+                        }
+                        __syncwarp();
+                    }
                 }
             }
             if (!ok || *abort) {
@@ -420,30 +469,35 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     }
 }
 
-template <int EP>
+template <int EP, int KP>
 int launch_wide(const Dims& D, const slicemoe_weights& w, const void* h, const PpParams& rp, int grid, cudaStream_t st) {
     CUtensorMap mX, mW1, mW2;
     int rc;
-    // (rows of 192 elements: the boxes reach past the tensors' edge and are zero-filled there)
+    // (rows of 96 / 192 elements: the boxes reach past the tensors' edge and are zero-filled there)
     if ((rc = make_tmap(&mX, h, (uint64_t)D.N, (uint64_t)D.ds, kTileM))) return rc;
     if ((rc = make_tmap(&mW1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, kWrHr))) return rc;
     if ((rc = make_tmap(&mW2, w.Wr2, (uint64_t)D.E, (uint64_t)D.Hr, EP))) return rc;      // (E = 8: zero-filled up to 16)
-    auto kern = route_wide_kernel<EP>;
+    auto kern = route_wide_kernel<EP, KP>;
     static bool attr_set[kAttrMaxDevices] = {};
     static std::mutex attr_mutex;
     {
         std::lock_guard<std::mutex> lock(attr_mutex);
-        if ((rc = set_smem_limit_once(kern, WrCfg<EP>::SMEM_ALLOC, attr_set))) return rc;
+        if ((rc = set_smem_limit_once(kern, WrCfg<EP, KP>::SMEM_ALLOC, attr_set))) return rc;
     }
-    kern<<<grid, kPpThreads, WrCfg<EP>::SMEM_ALLOC, st>>>(mX, mW1, mW2, rp);
+    kern<<<grid, kPpThreads, WrCfg<EP, KP>::SMEM_ALLOC, st>>>(mX, mW1, mW2, rp);
     SLICEMOE_LAUNCH_CHECK(1);
     return SLICEMOE_OK;
+}
+
+template <int EP>
+int launch_wide_e(const Dims& D, const slicemoe_weights& w, const void* h, const PpParams& rp, int grid, cudaStream_t st) {
+    return D.ds <= 128 ? launch_wide<EP, 2>(D, w, h, rp, grid, st) : launch_wide<EP, 4>(D, w, h, rp, grid, st);
 }
 
 }  // namespace
 
 bool wide_route_supported(const Dims& D) {
-    if (D.dtype != SLICEMOE_BF16 || (D.ds != 256 && D.ds != 192) || D.N <= 0) return false;
+    if (D.dtype != SLICEMOE_BF16 || (D.ds != 256 && D.ds != 192 && D.ds != 128 && D.ds != 96) || D.N <= 0) return false;
     if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
     if (D.k > 2 || D.noise_sigma > 0.0f) return false;
     return D.Hr == kWrHr;
@@ -467,9 +521,9 @@ int launch_route_wide(const Dims& D, const slicemoe_weights& w, const void* h, i
     if (grid_rows > grid) grid = grid_rows;
     switch (D.E) {
         case 8:
-        case 16: return launch_wide<16>(D, w, h, r, grid, st);
-        case 32: return launch_wide<32>(D, w, h, r, grid, st);
-        case 64: return launch_wide<64>(D, w, h, r, grid, st);
+        case 16: return launch_wide_e<16>(D, w, h, r, grid, st);
+        case 32: return launch_wide_e<32>(D, w, h, r, grid, st);
+        case 64: return launch_wide_e<64>(D, w, h, r, grid, st);
         default: return SLICEMOE_ERR_UNSUPPORTED;
     }
 }

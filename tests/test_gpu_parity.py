@@ -267,9 +267,9 @@ def test_profiled_forward_records_stage_times():
 @pytest.mark.parametrize("name", ["bf16_lm", "bf16_skew_cap", "bf16_decode", "bf16_single_row", "bf16_k3", "f32_cfg0",
                                   "bf16_paper_slice96", "bf16_paper_slice48", "bf16_paper_slice192", "bf16_e8"])
 def test_forward_launch_count_and_status(name):
-    """Supported bf16 shapes with k <= 2 run the whole forward as one launch (wide slices with a 256-wide router:
-    the router, whose weights fill the shared memory, and one launch for the rest); the others one launch per
-    step.  Either way the status word stays clear and repeated calls on two workspaces give the same bits."""
+    """Supported bf16 shapes with k <= 2 run the whole forward as one launch (slices of 192 / 256 elements with a
+    256-wide router: the router, whose weights fill the shared memory, and one launch for the rest); the others
+    one launch per step.  Either way the status word stays clear and repeated calls on two workspaces give the same bits."""
     import torch
     lc = SMALL[name]
     h, w = inputs(lc)

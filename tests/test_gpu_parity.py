@@ -69,6 +69,42 @@ def test_route(name):
     assert assigned.sum().item() == lc.R
 
 
+@pytest.mark.parametrize("T,d,S,E,k,init", [
+    (5000, 1024, 4, 64, 1, "normal"),     # 256-wide rows, 157 tiles: CTAs with two tiles and with one, ragged last tile
+    (2500, 1024, 4, 64, 2, "normal"),     # 256-wide rows, 79 tiles on 79 CTAs, ragged last tile; k = 2
+    (12000, 768, 4, 16, 2, "kaiming"),    # 192-wide rows (zero-filled fourth panel), three tiles per CTA, real biases
+    (30000, 512, 4, 32, 2, "normal"),     # 128-wide rows: two panels, three row tiles in shared memory, 7 tiles per CTA
+    (9000, 768, 8, 8, 1, "kaiming"),      # 96-wide rows (zero-filled second panel), E = 8 on the 16-wide instantiation
+    (100, 256, 1, 16, 2, "normal"),       # one ragged tile
+])
+def test_route_resident_weights(T, d, S, E, k, init):
+    """slicemoe_route without the probability matrix on slices of 96 to 256 elements (router hidden width 256):
+    the router that keeps both weight matrices in shared memory.  Routing on every row, the returned
+    probabilities and the per-expert counts against the oracle; the probability-matrix form (another kernel) must
+    pick the same experts wherever the gap is clear."""
+    import torch
+    lc = LC(f"rw_T{T}_d{d}_S{S}_E{E}_k{k}_{init}", T=T, d=d, S=S, E=E, k=k, F=2 * (d // S), init=init)
+    assert lc.Hr == 256 and lc.ds in (96, 128, 192, 256)
+    h, w = inputs(lc)
+    gpu = pu.GpuLayer(lc, h, w)
+    idx, p, assigned, _ = gpu.route(want_probs=False)
+    torch.cuda.synchronize()
+    assert gpu.status() == 0
+    ref = oracle.route(pu.oracle_config(lc), h, w)
+    idx_np = idx.cpu().numpy()
+    excluded = pu.check_routing(ref["probs"], ref["gap"], ref["topk_idx"], idx_np, p.cpu().numpy().astype(np.float64))
+    np.testing.assert_array_equal(assigned.cpu().numpy(), np.bincount(idx_np.ravel(), minlength=lc.E))
+    assert assigned.sum().item() == lc.R
+    idx2, p2, _, _ = gpu.route(want_probs=True)
+    torch.cuda.synchronize()
+    clear = ref["gap"] > pu.GAP_TOL
+    np.testing.assert_array_equal(np.sort(idx2.cpu().numpy(), axis=1)[clear], np.sort(idx_np, axis=1)[clear])
+    again = gpu.route(want_probs=False)
+    torch.cuda.synchronize()
+    assert torch.equal(again[0], idx) and torch.equal(again[1], p) and torch.equal(again[2], assigned)
+    print(lc.name, "excluded near-tie rows", excluded, "of", lc.N)
+
+
 @pytest.mark.parametrize("name", list(SMALL))
 def test_dispatch(name):
     import torch

@@ -2,25 +2,27 @@
 // storage, router hidden width 256, up to 64 experts, k <= 2 (sm_100a: tcgen05 + TMEM + TMA).
 //
 // The whole of Wr1 (up to 128 KB) and Wr2 stay in shared memory for the life of the CTA, so a tile's GEMM-1 runs as
-// 128-wide MMAs against operands that are written to shared memory once per launch, not once per tile: what a tile
+// wide MMAs against operands that are written to shared memory once per launch, not once per tile: what a tile
 // moves through shared memory is its own rows and the operand reads of its MMAs.  Rows come as 64-column panels
-// with a full / empty barrier pair each:
-//   rows of 192 / 256 (four panels, Wr1 = 128 KB)   there is room for exactly ONE row tile.  A tile's two units are
-//       therefore issued panel by panel, both units on a panel before the next panel: the tile is done with a panel,
-//       and the next tile's copy of it is requested, eight MMAs after the panel has landed, while the tile's other
-//       panels are still on their way -- the row loads run a whole tile ahead although only one tile's worth of
-//       shared memory exists.
-//   rows of 96 / 128 (two panels, Wr1 = 64 KB)      three row tiles fit; the units are issued one after the other,
-//       GEMM-1 up to two units ahead of GEMM-2, and the loads run three tiles ahead.
+// with a full / empty barrier pair each: rows of 192 / 256 (four panels, Wr1 = 128 KB) leave room for exactly ONE
+// row tile, rows of 96 / 128 (two panels, Wr1 = 64 KB) for three.  GEMM-1 is issued panel by panel, all of a tile's
+// MMAs on a panel before the next panel: the tile is done with a panel, and the next copy into its slot is
+// requested, eight MMAs after the panel has landed, while the tile's other panels are still on their way -- with one
+// row tile of shared memory the row loads still run a whole tile ahead.
 //
-// One CTA of 768 threads per SM walks a contiguous range of 128-row tiles.  A tile is two units of 128 hidden
-// columns; three 128-column buffers of tensor memory take the units in turn, the activation warps turn a buffer's
-// fp32 values in place into a truncated bf16 and the rounded remainder (GEMM-2 runs over both, so the logits keep
-// fp32-level accuracy and the top-k decision does not hang on a bf16 rounding of the hidden layer), GEMM-2 reads them
-// from tensor memory.  Warp roles:
+// One CTA of 768 threads per SM walks a contiguous range of 128-row tiles.  A tile's hidden layer is two units, a
+// narrow one (hidden 0 .. 63) and a wide one (64 .. 255): the wide unit has two buffers of tensor memory (the tile's
+// parity picks one), the narrow unit one -- it is the first through the activation and through GEMM-2, so its
+// buffer is free again by the time the next tile's first panel lands, and no tile waits for a buffer.  (Two units of
+// 128 columns on three buffers: the second unit of every tile waited ~1.2 k cycles for the previous tile's first.)
+// The activation warps turn a buffer's fp32 values in place into a truncated bf16 and the rounded remainder (GEMM-2
+// runs over both, so the logits keep fp32-level accuracy and the top-k decision does not hang on a bf16 rounding of
+// the hidden layer), GEMM-2 reads them from tensor memory into ONE logit accumulator, which the output warps have
+// long loaded when the next tile's GEMM-2 starts.  Warp roles:
 //   warp 0       row panels by TMA          warp 3  GEMM-1 issue        warp 1  GEMM-2 issue
 //   warp 2       zeroes this CTA's rows of h' (forward: the experts add into it)
-//   warps 4-19   activation (four warpgroups, 32 of a unit's 128 columns each; a thread owns one tile row)
+//   warps 4-19   activation (four warpgroups, 16 of the narrow and 48 of the wide unit's columns each; a thread
+//                owns one tile row)
 //   warps 20-23  softmax, top-k (ties to the lower id), this CTA's per-expert counts
 // All hand-offs are mbarriers with bounded waits; a run-out sets the status word and every role leaves.
 #include <mutex>
@@ -74,7 +76,11 @@ struct WrCfg {
     static constexpr int SMEM_BYTES = OFF_W2 + (kWrHr / 64) * W2_CHUNK;
     // (at least 120 KB so that two CTAs never share an SM: each allocates all of tensor memory)
     static constexpr int SMEM_ALLOC = SMEM_BYTES + 1024 > 120 * 1024 ? SMEM_BYTES + 1024 : 120 * 1024;
-    static constexpr int HB_COLS = 128, LOGIT_COL = 384;
+    // The hidden layer of a tile as two units: a narrow one (hidden 0 .. 63) and a wide one (64 .. 255).  Tensor
+    // memory: two wide buffers (the tile's parity picks one), one narrow buffer, one logit accumulator.
+    static constexpr int NARROW = 64, WIDE = kWrHr - NARROW;
+    static constexpr int WIDE_COL0 = 0, NARROW_COL = 2 * WIDE, LOGIT_COL = NARROW_COL + NARROW;
+    static_assert(LOGIT_COL + kWrMaxE <= 512, "tensor memory");
     static_assert(KP == 2 || KP == 4, "row width");
     static_assert(SLOTS <= kWrMaxSlots && KP <= kWrMaxKP, "barrier slots");
     static_assert(SMEM_ALLOC + sizeof(WrShared) + 64 <= 232448, "shared memory budget");
@@ -100,7 +106,6 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
     const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
     const int ntiles = min(total_tiles, t_begin + per_cta) - t_begin;
-    const int nunits = ntiles * 2;
     const uint32_t sA = smem_base + C::OFF_A, sW1 = smem_base + C::OFF_W1, sW2 = smem_base + C::OFF_W2;
 
     if (warp == 1) {
@@ -181,85 +186,60 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         }
     } else if (warp == 3) {
         // ================= GEMM-1 issue ======================================================================
-        if (nunits > 0) {
-            constexpr uint32_t idesc1 = make_idesc(128, 128, kFmtBF16, kFmtBF16);
+        // Panel by panel, both units on a panel before the next panel, so that a panel is released (and the next
+        // tile's copy of it requested) eight MMAs after it has landed.  The wide unit's buffer alternates with the
+        // tile and is long free; the narrow unit's single buffer is free once the previous tile's narrow unit
+        // -- first through the activation, 8 MMAs of GEMM-2 -- has been consumed, which is about when this tile's
+        // first panel lands.  From the second panel on the narrow unit goes first, so that it completes four
+        // MMAs before the tile does and its activation starts under them.
+        if (ntiles > 0) {
+            constexpr uint32_t idescW = make_idesc(128, C::WIDE, kFmtBF16, kFmtBF16);
+            constexpr uint32_t idescN = make_idesc(128, C::NARROW, kFmtBF16, kFmtBF16);
             const uint32_t dA = desc_lo_sw128(sA), dW1 = desc_lo_sw128(sW1);
             bool ok = true;
-            if constexpr (NT == 1) {
-                // One row tile in shared memory: both units of a tile panel by panel, so that a panel is released
-                // eight MMAs after it has landed.  (Unit by unit, all panels would be released in a burst at the
-                // tile's end and requested in a burst: measured, 5 % slower.  Letting the first unit run ahead on
-                // the panels that are there while the second unit's buffer is busy: measured, slower too -- its
-                // MMAs queue in front of the GEMM-2 that frees that buffer.)
 #pragma unroll 1
-                for (int ta = 0; ta < ntiles && ok; ++ta) {
-                    const uint32_t u0 = 2u * (uint32_t)ta, u1 = u0 + 1u;
-                    const uint32_t b0 = u0 % 3u, b1 = u1 % 3u;
-                    // (a buffer also held the hidden values of the unit three back: GEMM-2 must have read them)
-                    if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b0), ((u0 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
-                    const uint32_t d0 = tmem_base + b0 * C::HB_COLS, d1 = tmem_base + b1 * C::HB_COLS;
+            for (int ta = 0; ta < ntiles && ok; ++ta) {
+                const int wb = ta & 1;                  // wide buffer of this tile
+                const int sb = (ta % NT) * KP;
+                // (the buffer also held the hidden values of the tile two back: GEMM-2 must have read them)
+                if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + wb), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
+                const uint32_t dW = tmem_base + C::WIDE_COL0 + wb * C::WIDE, dN = tmem_base + C::NARROW_COL;
 #pragma unroll
-                    for (int kp = 0; kp < KP; ++kp) {
-                        if (ta == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
-                        if (!pp_wait(wr_bar(sh, B::A_FULL + kp), (uint32_t)ta & 1u, abort)) { ok = false; break; }
-                        tc_fence_after_sync();
-                        const uint32_t a0 = dA + ((kp * kWrPanelA) >> 4);
-                        const uint32_t w0 = dW1 + ((kp * kWrPanelW1) >> 4), w1 = w0 + ((128 * 128) >> 4);
+                for (int kp = 0; kp < KP; ++kp) {
+                    if (ta == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
+                    if (!pp_wait(wr_bar(sh, B::A_FULL + sb + kp), (uint32_t)(ta / NT) & 1u, abort)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a0 = dA + (((sb + kp) * kWrPanelA) >> 4);
+                    const uint32_t wN = dW1 + ((kp * kWrPanelW1) >> 4), wW = wN + ((C::NARROW * 128) >> 4);
+                    if (kp == 0) {
                         if (elect_one_sync()) {
 #pragma unroll
                             for (int kk = 0; kk < 4; ++kk) {
-                                if (kp == 0 && kk == 0) mma_ss<0>(d0, a0, w0, idesc1);
-                                else mma_ss<1>(d0, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
+                                if (kk == 0) mma_ss<0>(dW, a0, wW, idescW);
+                                else mma_ss<1>(dW, a0 + ((kk * 32) >> 4), wW + ((kk * 32) >> 4), idescW);
                             }
                         }
                         __syncwarp();
-                        // (the second unit's buffer is the one the previous tile's first unit is still in)
-                        if (kp == 0) {
-                            if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b1), ((u1 / 3u) & 1u) ^ 1u, abort)) { ok = false; break; }
-                            tc_fence_after_sync();
-                        }
+                        if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + 2), ((uint32_t)ta & 1u) ^ 1u, abort)) { ok = false; break; }
+                        tc_fence_after_sync();
                         if (elect_one_sync()) {
 #pragma unroll
                             for (int kk = 0; kk < 4; ++kk) {
-                                if (kp == 0 && kk == 0) mma_ss<0>(d1, a0, w1, idesc1);
-                                else mma_ss<1>(d1, a0 + ((kk * 32) >> 4), w1 + ((kk * 32) >> 4), idesc1);
+                                if (kk == 0) mma_ss<0>(dN, a0, wN, idescN);
+                                else mma_ss<1>(dN, a0 + ((kk * 32) >> 4), wN + ((kk * 32) >> 4), idescN);
                             }
-                            mma_commit(wr_bar(sh, B::A_EMPTY + kp));
-                            if (kp == KP - 1) {
-                                mma_commit(wr_bar(sh, B::ACC1_FULL + b0));
-                                mma_commit(wr_bar(sh, B::ACC1_FULL + b1));
-                            }
+                            mma_commit(wr_bar(sh, B::A_EMPTY + sb + kp));       // the tile is done with the panel
                         }
                         __syncwarp();
-                    }
-                }
-            } else {
-                // Several row tiles in shared memory: unit by unit, up to two units ahead of GEMM-2.
-#pragma unroll 1
-                for (int u = 0; u < nunits && ok; ++u) {
-                    const int ta = u >> 1, hf = u & 1;
-                    const int sb = (ta % NT) * KP;
-                    const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
-                    if (!pp_wait(wr_bar(sh, B::ACC1_EMPTY + b), (n & 1u) ^ 1u, abort)) { ok = false; break; }
-                    const uint32_t d = tmem_base + b * C::HB_COLS;
-#pragma unroll
-                    for (int kp = 0; kp < KP; ++kp) {
-                        if (hf == 0) {
-                            if (u == 0 && !pp_wait(wr_bar(sh, B::W1_FULL + kp), 0u, abort)) { ok = false; break; }
-                            if (!pp_wait(wr_bar(sh, B::A_FULL + sb + kp), (uint32_t)(ta / NT) & 1u, abort)) { ok = false; break; }
-                        }
-                        tc_fence_after_sync();
-                        const uint32_t a0 = dA + (((sb + kp) * kWrPanelA) >> 4);
-                        const uint32_t w0 = dW1 + ((kp * kWrPanelW1 + hf * (128 * 128)) >> 4);
+                    } else {
                         if (elect_one_sync()) {
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk) {
-                                if (kp == 0 && kk == 0) mma_ss<0>(d, a0, w0, idesc1);
-                                else mma_ss<1>(d, a0 + ((kk * 32) >> 4), w0 + ((kk * 32) >> 4), idesc1);
-                            }
-                            // the tile's second unit is the last reader of a panel
-                            if (hf == 1) mma_commit(wr_bar(sh, B::A_EMPTY + sb + kp));
-                            if (kp == KP - 1) mma_commit(wr_bar(sh, B::ACC1_FULL + b));
+                            for (int kk = 0; kk < 4; ++kk) mma_ss<1>(dN, a0 + ((kk * 32) >> 4), wN + ((kk * 32) >> 4), idescN);
+                            if (kp == KP - 1) mma_commit(wr_bar(sh, B::ACC1_FULL + 2));
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) mma_ss<1>(dW, a0 + ((kk * 32) >> 4), wW + ((kk * 32) >> 4), idescW);
+                            mma_commit(wr_bar(sh, B::A_EMPTY + sb + kp));
+                            if (kp == KP - 1) mma_commit(wr_bar(sh, B::ACC1_FULL + wb));
                         }
                         __syncwarp();
                     }
@@ -275,34 +255,51 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        // ================= GEMM-2 issue: logits += hidden(hi) Wr2^T + hidden(lo) Wr2^T ========================
-        if (nunits > 0) {
+        // ================= GEMM-2 issue: logits = hidden(hi) Wr2^T + hidden(lo) Wr2^T ==========================
+        // K step kk of a unit: hi halves in the unit's columns 16 kk .. 16 kk + 7, lo halves in the next eight.
+        // The narrow unit (hidden 0 .. 63, Wr2's first panel) first: its buffer is the one the next tile waits for.
+        if (ntiles > 0) {
             constexpr uint32_t idesc2 = make_idesc(128, EP, kFmtBF16, kFmtBF16);
             const uint32_t dW2 = desc_lo_sw128(sW2);
             bool ok = pp_wait(wr_bar(sh, B::W2_FULL), 0u, abort);
 #pragma unroll 1
-            for (int u = 0; u < nunits && ok; ++u) {
-                const int ta = u >> 1, hf = u & 1;
-                const int r = ta & 1;
-                if (hf == 0 && !pp_wait(wr_bar(sh, B::ACC2_EMPTY + r), ((uint32_t)(ta >> 1) & 1u) ^ 1u, abort)) { ok = false; break; }
-                const uint32_t b = (uint32_t)u % 3u, n = (uint32_t)u / 3u;
-                if (!pp_wait(wr_bar(sh, B::HID_FULL + b), n & 1u, abort)) { ok = false; break; }
+            for (int ta = 0; ta < ntiles && ok; ++ta) {
+                const int wb = ta & 1;
+                const uint32_t d = tmem_base + C::LOGIT_COL;
+                // (one logit accumulator: the output warps must have loaded the previous tile's)
+                if (!pp_wait(wr_bar(sh, B::ACC2_EMPTY), ((uint32_t)ta & 1u) ^ 1u, abort)) { ok = false; break; }
+                if (!pp_wait(wr_bar(sh, B::HID_FULL + 2), (uint32_t)ta & 1u, abort)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t w0 = dW2 + ((hf * 2 * C::W2_CHUNK) >> 4);
-                const uint32_t d = tmem_base + C::LOGIT_COL + r * 64, a = tmem_base + b * C::HB_COLS;
                 if (elect_one_sync()) {
-                    // K step kk of the unit: hi halves in columns 16 kk .. 16 kk + 7, lo halves in the next eight
+                    const uint32_t a = tmem_base + C::NARROW_COL;
 #pragma unroll
                     for (int part = 0; part < 2; ++part) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t bd = w0 + (((kk >> 2) * C::W2_CHUNK + (kk & 3) * 32) >> 4);
-                            if (part == 0 && kk == 0) mma_ts_dyn(d, a, bd, idesc2, hf > 0 ? 1u : 0u);
+                        for (int kk = 0; kk < C::NARROW / 16; ++kk) {
+                            const uint32_t bd = dW2 + ((kk * 32) >> 4);
+                            if (part == 0 && kk == 0) mma_ts<0>(d, a, bd, idesc2);
                             else mma_ts<1>(d, a + kk * 16 + part * 8, bd, idesc2);
                         }
                     }
-                    mma_commit(wr_bar(sh, B::ACC1_EMPTY + b));
-                    if (hf == 1) mma_commit(wr_bar(sh, B::ACC2_FULL + r));
+                    mma_commit(wr_bar(sh, B::ACC1_EMPTY + 2));
+                }
+                __syncwarp();
+                if (!pp_wait(wr_bar(sh, B::HID_FULL + wb), (uint32_t)(ta >> 1) & 1u, abort)) { ok = false; break; }
+                tc_fence_after_sync();
+                if (elect_one_sync()) {
+                    const uint32_t a = tmem_base + C::WIDE_COL0 + wb * C::WIDE;
+#pragma unroll
+                    for (int part = 0; part < 2; ++part) {
+#pragma unroll
+                        for (int kk = 0; kk < C::WIDE / 16; ++kk) {
+                            // hidden units NARROW + 16 kk ..: panel (NARROW + 16 kk) / 64 of Wr2
+                            constexpr int kk0 = C::NARROW / 16;
+                            const uint32_t bd = dW2 + (((((kk + kk0) >> 2) * C::W2_CHUNK) + ((kk + kk0) & 3) * 32) >> 4);
+                            mma_ts<1>(d, a + kk * 16 + part * 8, bd, idesc2);
+                        }
+                    }
+                    mma_commit(wr_bar(sh, B::ACC1_EMPTY + wb));
+                    mma_commit(wr_bar(sh, B::ACC2_FULL));
                 }
                 __syncwarp();
             }
@@ -346,52 +343,77 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         }
     } else if (warp < 20) {
         // ================= activation warps: warpgroup g, lane group lg ======================================
+        // relu(acc + bias) as hi + lo, in place: hi = the value truncated to bf16 (negative -> 0 by .relu), lo = the
+        // rounded remainder (for a negative value the remainder is the value itself and its .relu is 0 too).  A
+        // 16-column piece becomes 8 columns of hi pairs and 8 of lo pairs = one K step of GEMM-2.
         const int g = (warp - 4) >> 2;
         const int lg = warp & 3;
-        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16) + 32 * g;
+        const uint32_t tlane = tmem_base + ((uint32_t)(lg * 32) << 16);
         const bool has_br1 = p.br1 != nullptr;
+        auto split_piece = [&](const uint32_t* acc, const float* bias, uint32_t col) {
+            float a[16];
+            if (has_br1) {
+#pragma unroll
+                for (int i = 0; i < 16; i += 4) {
+                    const float4 bb = *reinterpret_cast<const float4*>(bias + i);
+                    add2(a[i], a[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), bb.x, bb.y);
+                    add2(a[i + 2], a[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), bb.z, bb.w);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) a[i] = __uint_as_float(acc[i]);
+            }
+            uint32_t hl[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) hl[i] = cvt_rz_relu_bf16x2(a[2 * i], a[2 * i + 1]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                hl[8 + i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hl[i] << 16), a[2 * i + 1] - __uint_as_float(hl[i] & 0xFFFF0000u));
+            tmem_st_x16(col, hl);
+        };
         bool ok = true;
 #pragma unroll 1
-        for (int u = 0; u < nunits && ok; ++u) {
-            const int hf = u & 1;
-            const uint32_t b = (uint32_t)u % 3u, par = ((uint32_t)u / 3u) & 1u;
-            ok = pp_wait(wr_bar(sh, B::ACC1_FULL + b), par, abort);
+        for (int ta = 0; ta < ntiles && ok; ++ta) {
+            const int wb = ta & 1;
+            // ---- the narrow unit (hidden 0 .. 63): 16 columns per warpgroup
+            ok = pp_wait(wr_bar(sh, B::ACC1_FULL + 2), (uint32_t)ta & 1u, abort);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t acol = tlane + b * C::HB_COLS;
-            const float* bias = sh.bias1_f32 + hf * 128 + 32 * g;
-            // relu(acc + bias) as hi + lo: hi = the value truncated to bf16 (negative -> 0 by .relu), lo = the
-            // rounded remainder (for a negative value the remainder is the value itself and its .relu is 0 too)
-            uint32_t acc32[32];
-            tmem_ld_x32(acol, acc32);
-            tmem_ld_wait();
-#pragma unroll
-            for (int pc = 0; pc < 2; ++pc) {
-                const uint32_t* acc = acc32 + 16 * pc;
-                float a[16];
-                if (has_br1) {
-#pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        const float4 bb = *reinterpret_cast<const float4*>(bias + pc * 16 + i);
-                        add2(a[i], a[i + 1], __uint_as_float(acc[i]), __uint_as_float(acc[i + 1]), bb.x, bb.y);
-                        add2(a[i + 2], a[i + 3], __uint_as_float(acc[i + 2]), __uint_as_float(acc[i + 3]), bb.z, bb.w);
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) a[i] = __uint_as_float(acc[i]);
-                }
-                uint32_t hl[16];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) hl[i] = cvt_rz_relu_bf16x2(a[2 * i], a[2 * i + 1]);
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    hl[8 + i] = cvt_rn_relu_bf16x2(a[2 * i] - __uint_as_float(hl[i] << 16), a[2 * i + 1] - __uint_as_float(hl[i] & 0xFFFF0000u));
-                tmem_st_x16(acol + 16 * pc, hl);
+            {
+                const uint32_t col = tlane + C::NARROW_COL + 16 * g;
+                uint32_t acc[16];
+                tmem_ld_x16(col, acc);
+                tmem_ld_wait();
+                split_piece(acc, sh.bias1_f32 + 16 * g, col);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(wr_bar(sh, B::HID_FULL + 2));
             }
-            tmem_st_wait();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(wr_bar(sh, B::HID_FULL + b));
+            // ---- the wide unit (hidden 64 .. 255): 48 columns per warpgroup
+            ok = pp_wait(wr_bar(sh, B::ACC1_FULL + wb), (uint32_t)(ta >> 1) & 1u, abort);
+            if (!ok) break;
+            tc_fence_after_sync();
+            {
+                const uint32_t col = tlane + C::WIDE_COL0 + wb * C::WIDE + 48 * g;
+                const float* bias = sh.bias1_f32 + C::NARROW + 48 * g;
+                // three pieces, each loaded under the arithmetic of the one before (16-column loads: the
+                // warpgroups' column offsets are multiples of 16 only)
+                uint32_t acc0[16], acc1[16];
+                tmem_ld_x16(col, acc0);
+                tmem_ld_wait();
+                tmem_ld_x16(col + 16, acc1);
+                split_piece(acc0, bias, col);
+                tmem_ld_wait();
+                tmem_ld_x16(col + 32, acc0);
+                split_piece(acc1, bias + 16, col + 16);
+                tmem_ld_wait();
+                split_piece(acc0, bias + 32, col + 32);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(wr_bar(sh, B::HID_FULL + wb));
+            }
         }
     } else {
         // ================= output warpgroup: softmax + top-k of a tile's logits ==============================
@@ -401,17 +423,16 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         bool ok = true;
 #pragma unroll 1
         for (int ta = 0; ta < ntiles && ok; ++ta) {
-            const int r = ta & 1;
-            ok = pp_wait(wr_bar(sh, B::ACC2_FULL + r), (uint32_t)(ta >> 1) & 1u, abort);
+            ok = pp_wait(wr_bar(sh, B::ACC2_FULL), (uint32_t)ta & 1u, abort);
             if (!ok) break;
             tc_fence_after_sync();
             uint32_t v[EP];
 #pragma unroll
-            for (int c = 0; c < EP; c += 16) tmem_ld_x16(tlane + r * 64 + c, v + c);
+            for (int c = 0; c < EP; c += 16) tmem_ld_x16(tlane + c, v + c);
             tmem_ld_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(wr_bar(sh, B::ACC2_EMPTY + r));
+            if (lane == 0) mbar_arrive(wr_bar(sh, B::ACC2_EMPTY));
             const int n = (t_begin + ta) * kTileM + row;
             const bool valid = n < p.n_rows;
             // one pass keeping the best two (strict comparisons in ascending id order: the picks of repeated

@@ -39,7 +39,7 @@ NCU_TRAFFIC = {
     ("forward_one_launch", 16384 * 8, 64, 2, 256): (17.9745e6 + 0.04e6, "profiles/pp_forward_kernel_cfg1_cfg2.md (ncu, cfg1)"),
     ("forward_one_launch", 65536 * 16, 64, 2, 256): (613.103e6 + 342.652e6, "profiles/pp_forward_kernel_cfg1_cfg2.md (ncu, cfg2)"),
     ("forward_one_launch", 128 * 32, 128, 2, 512): (17.868e6, "profiles/decode_forward_kernel_cfg4.md (ncu, cfg4)"),
-    ("route", 32768 * 8, 256, 1, 1024): (134.842e6 + 87.31e6, "profiles/route_wide_kernel_cfg3.md (ncu, cfg3; 134.8 MB read + 87.3 MB of the zero rows of h', which the "
+    ("route", 32768 * 8, 256, 1, 1024): (134.453e6 + 87.19e6, "profiles/route_wide_kernel_cfg3.md (ncu, cfg3; 134.5 MB read + 87.2 MB of the zero rows of h', which the "
                                          "forward's router writes for the combine step and the stage's compulsory bytes do not count)"),
 }
 OTHER_CONFIGS = ("cfg2", "cfg3", "cfg3b", "cfg4", "paper768")     # paper768: the paper's own model shape (d = 768, S = 8, E = 16, k = 2)

@@ -255,6 +255,7 @@ int launch_forward_fused(const Dims& D, const slicemoe_weights& w, const void* h
     f.yperm = nullptr; f.status = status;
     f.gather_src = (const bf16*)h; f.perm = perm; f.gate = gate; pair_to_row_magic(D.k, &f.gather_magic, &f.gather_shift);
     f.scatter_out = (bf16*)h_out;
+    f.split_hidden = D.k == 1 ? 1 : 0;     // (k = 1: a row of h' has one writer, two with the hidden layer in halves)
 
     fp.R = (int)D.R; fp.E = D.E; fp.pairs_per_chunk = rows_per_cta * D.k; fp.capacity = (int)D.capacity;
     fp.assigned = assigned; fp.kept = kept; fp.offsets = offsets; fp.dest = dest; fp.perm = perm; fp.gate = gate;

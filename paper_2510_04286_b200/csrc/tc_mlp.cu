@@ -136,6 +136,7 @@ int launch_ffn_tc(const Dims& D, const slicemoe_weights& w, const void* xperm, c
     p.yperm = (bf16*)yperm; p.status = status;
     p.gather_src = (const bf16*)gather_h; p.perm = perm; p.gate = gate; pair_to_row_magic(D.k, &p.gather_magic, &p.gather_shift);
     p.scatter_out = gather_h ? (bf16*)scatter_out : nullptr;
+    p.split_hidden = p.scatter_out && D.k == 1 ? 1 : 0;
     if (gather_h) xperm = gather_h;   // the A tensor map is not used in gather mode; any valid matrix will do
     p.row_elems = D.ds;
     const bool gelu = D.act == SLICEMOE_ACT_GELU_TANH;

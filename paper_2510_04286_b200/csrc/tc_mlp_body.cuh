@@ -77,6 +77,11 @@ struct TcParams {
     uint32_t gather_magic, gather_shift;   // row of pair i = (i * magic) >> shift = i / k (see pair_to_row)
     bf16* scatter_out;        // fused forward, k <= 2: h' viewed as Y[N, N2]; the row of pair (n, j) is added to
                               // Y[n, :] (h' zeroed beforehand) instead of being stored to yperm; or nullptr
+    // experts, scatter_out with k = 1: a batch that leaves more than half of the CTAs without a tile is run as two
+    // tiles per tile, each over one half of the hidden layer (two "virtual experts" per expert that share the
+    // expert's rows: W1 / b1 rows [half HID/2, ...), W2 columns likewise, b2 with the first half only); both add
+    // into the row of h', and a sum of two bf16 terms does not depend on their order
+    int split_hidden;
     // router, fused forward: this CTA also zeroes the rows of zero_out that it routes
     bf16* zero_out;           // h' viewed as Y[N, zero_cols], or nullptr
     int zero_cols;
@@ -230,11 +235,12 @@ struct Bars {
     static constexpr int COUNT = DRAIN + 2;
 };
 
+// (s: 0, or 1 when every expert is two virtual experts over the same rows; e counts virtual experts)
 __device__ __forceinline__ void locate_tile(const int* tile_start, const int* offs, int t, int& e,
-                                            int& row0, int& rows) {
+                                            int& row0, int& rows, int s = 0) {
     while (t >= tile_start[e + 1]) ++e;
-    row0 = offs[e] + (t - tile_start[e]) * kTileM;
-    rows = min(kTileM, offs[e + 1] - row0);
+    row0 = offs[e >> s] + (t - tile_start[e]) * kTileM;
+    rows = min(kTileM, offs[(e >> s) + 1] - row0);
 }
 
 // Row n = pair / k of a pair index, k = 1..8, without a division: (pair * magic) >> shift with
@@ -393,6 +399,7 @@ struct TcShared {
     int hist[kMaxE];
     uint32_t tmem_base;
     int abort_flag;
+    int split_shift;          // 1: two virtual experts per expert (TcParams::split_hidden), else 0
     // fused forward: per-row gate (Eq. 1) and pair index of the tiles in flight, copied in by the
     // gather warp with the rows themselves (ring over the CTA's tile counter)
     float gate_s[kMetaRing][kTileM];
@@ -427,8 +434,6 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     volatile int* abort = &sh.abort_flag;
-    const int nchunks = p.HID / C::HC;
-    const bool resident = nchunks <= C::W_STAGES;
     // FUSED (the single-kernel forward): what that caller always asks for is fixed at compile time --
     // rows gathered and results added into h' (experts); no probability matrix, no global counts, k <= 2,
     // h' zeroed (router) -- so that the other variants' code is not part of its hot loops
@@ -479,27 +484,44 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             sh.bias2_f32[i] = i >= p.experts_real ? -INFINITY : (p.bias2 ? __bfloat162float(p.bias2[i]) : 0.0f);
     __syncthreads();
     if (warp == 0) {
-        // first tile of every expert: exclusive scan of the tile counts, 32 experts at a time
-        int run = 0;
-        for (int e0 = 0; e0 < p.E; e0 += 32) {
-            const int e = e0 + lane;
-            const int nt = e < p.E ? (sh.offs[e + 1] - sh.offs[e] + kTileM - 1) / kTileM : 0;
-            int incl = nt;
+        // first tile of every (virtual) expert: exclusive scan of the tile counts, 32 experts at a time; a second
+        // time over two virtual experts per expert when that still leaves every CTA at most one tile
+        // (256-wide rows only: that is where a tile is long enough for the split to pay -- 29.7 -> 22.6 us for the 40
+        // tiles of the skewed benchmark batch -- and the narrower instantiations keep their register budget)
+        const bool may_split = !C::ROUTER && C::K1 == 256 && p.split_hidden && p.HID % (2 * C::HC) == 0 &&
+                               p.HID >= 4 * C::HC && 2 * p.E <= kMaxE;
+        int s = 0;
+        for (;;) {
+            const int EV = p.E << s;
+            int run = 0;
+            for (int e0 = 0; e0 < EV; e0 += 32) {
+                const int e = e0 + lane;
+                const int nt = e < EV ? (sh.offs[(e >> s) + 1] - sh.offs[e >> s] + kTileM - 1) / kTileM : 0;
+                int incl = nt;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, d);
-                if (lane >= d) incl += up;
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int up = __shfl_up_sync(0xffffffffu, incl, d);
+                    if (lane >= d) incl += up;
+                }
+                if (e < EV) sh.tile_start[e] = run + incl - nt;
+                run += __shfl_sync(0xffffffffu, incl, 31);
             }
-            if (e < p.E) sh.tile_start[e] = run + incl - nt;
-            run += __shfl_sync(0xffffffffu, incl, 31);
+            if (lane == 0) sh.tile_start[EV] = run;
+            __syncwarp();
+            if (s == 0 && may_split && run > 0 && 2 * run <= (int)gridDim.x) s = 1;
+            else break;
         }
-        if (lane == 0) sh.tile_start[p.E] = run;
+        if (lane == 0) sh.split_shift = s;
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = sh.tmem_base;
-    const int total_tiles = sh.tile_start[p.E];
+    const int vs = (C::ROUTER || C::K1 != 256) ? 0 : sh.split_shift;          // virtual-expert shift
+    const int hid = p.HID >> vs;                             // hidden units per (virtual) expert
+    const int nchunks = hid / C::HC;
+    const bool resident = nchunks <= C::W_STAGES;
+    const int total_tiles = sh.tile_start[p.E << vs];
     const int per_cta = (total_tiles + gridDim.x - 1) / gridDim.x;
     const int t_begin = min(total_tiles, (int)blockIdx.x * per_cta);
     const int t_end = min(total_tiles, t_begin + per_cta);
@@ -524,7 +546,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             bool ok = true;
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
                 int row0, rows;
-                locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
+                locate_tile(sh.tile_start, sh.offs, t, e, row0, rows, vs);
                 const int ab = ta % C::A_BUFS;
                 const uint32_t an = ta / C::A_BUFS;
                 if (!gather) {
@@ -548,10 +570,10 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                     mbar_arrive_expect_tx(bar(B::W1_FULL + slot), C::W1C_BYTES + (p.bias1 ? C::B1_BYTES : 0));
                     if (p.bias1)
                         bulk_load(smem_base + C::OFF_B1 + (wq % kBiasRing) * C::B1_BYTES,
-                                  p.bias1 + (size_t)e * p.HID + c * C::HC, C::B1_BYTES, bar(B::W1_FULL + slot));
+                                  p.bias1 + (size_t)e * hid + c * C::HC, C::B1_BYTES, bar(B::W1_FULL + slot));
 #pragma unroll
                     for (int kp = 0; kp < C::KP1; ++kp)
-                        tma_load_2d(sW + slot * C::W1C_BYTES + kp * C::W1_PANEL, &tmW1, kp * 64, e * p.HID + c * C::HC,
+                        tma_load_2d(sW + slot * C::W1C_BYTES + kp * C::W1_PANEL, &tmW1, kp * 64, e * hid + c * C::HC,
                                     bar(B::W1_FULL + slot));
                     last_bar[1] = bar(B::W1_FULL + slot);
                     last_par[1] = n & 1u;
@@ -561,7 +583,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #pragma unroll
                     for (int kp = 0; kp < C::KP2; ++kp)
                         tma_load_2d(smem_base + C::OFF_W2 + slot * C::W2C_BYTES + kp * C::W2_PANEL, &tmW2,
-                                    c * C::HC + kp * 64, e * C::N2, bar(B::W2_FULL + slot));
+                                    (e & vs) * hid + c * C::HC + kp * 64, (e >> vs) * C::N2, bar(B::W2_FULL + slot));
                     last_bar[2] = bar(B::W2_FULL + slot);
                     last_par[2] = n & 1u;
                 }
@@ -587,7 +609,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             uint32_t g = 0, reloads = 0;
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
                 int r0, rr;
-                locate_tile(sh.tile_start, sh.offs, t, e, r0, rr);
+                locate_tile(sh.tile_start, sh.offs, t, e, r0, rr, vs);
                 const bool reload = !resident || (e != prev_e);
                 prev_e = e;
                 const int ab = ta % C::A_BUFS;
@@ -643,14 +665,14 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
             uint32_t g = 0, reloads = 0;
             for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
                 int r0, rr;
-                locate_tile(sh.tile_start, sh.offs, t, e, r0, rr);
+                locate_tile(sh.tile_start, sh.offs, t, e, r0, rr, vs);
                 const bool reload = !resident || (e != prev_e);
                 prev_e = e;
                 // resident weights are handed back only when the next tile brings another expert
                 bool release = !resident;
                 if (resident && t + 1 < t_end) {
                     int e2 = e;
-                    locate_tile(sh.tile_start, sh.offs, t + 1, e2, r0, rr);
+                    locate_tile(sh.tile_start, sh.offs, t + 1, e2, r0, rr, vs);
                     release = (e2 != e);
                 }
                 const int buf = ta % C::ACC2_BUFS;
@@ -748,7 +770,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 for (int q = 0; q < QPW; ++q) nrow[q] = nnext[q] < 0 ? -1 : pair_to_row(nnext[q], p.gather_magic, p.gather_shift);
                 if (t + 1 < t_end) {
                     int row0, rows;
-                    locate_tile(sh.tile_start, sh.offs, t + 1, ge, row0, rows);
+                    locate_tile(sh.tile_start, sh.offs, t + 1, ge, row0, rows, vs);
 #pragma unroll
                     for (int q = 0; q < QPW; ++q) {
                         const int r = lane + 32 * (q0 + q);
@@ -791,7 +813,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
                 }
                 {
                     int row0, rows;
-                    locate_tile(sh.tile_start, sh.offs, t, gm, row0, rows);
+                    locate_tile(sh.tile_start, sh.offs, t, gm, row0, rows, vs);
 #pragma unroll
                     for (int q = 0; q < QPW; ++q) {
                         // rows past the tile's end take a neighbour's values: their A rows are zero and
@@ -819,7 +841,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         uint32_t q_tile = 0, q_next = 0;              // bias ring: W1 load count of this tile's chunk 0 / after it
         for (int t = t_begin; t < t_end && ok; ++t) {
             int row0, rows;
-            locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
+            locate_tile(sh.tile_start, sh.offs, t, e, row0, rows, vs);
             if (!resident || e != prev_e) {           // this tile's weights (and biases) were loaded for it
                 q_tile = q_next;
                 q_next += nchunks;
@@ -909,7 +931,7 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
         // added into row n of Y.
         for (int t = t_begin, ta = 0; t < t_end && ok; ++t, ++ta) {
             int row0, rows;
-            locate_tile(sh.tile_start, sh.offs, t, e, row0, rows);
+            locate_tile(sh.tile_start, sh.offs, t, e, row0, rows, vs);
             const int buf = ta % C::ACC2_BUFS;
             ok = mbar_wait(bar(B::ACC2_FULL + buf), (uint32_t)(ta / C::ACC2_BUFS) & 1u, abort, kWaitLimitNs);
             ok = __all_sync(0xffffffffu, ok);
@@ -1021,8 +1043,8 @@ __device__ __forceinline__ void tc_body(const CUtensorMap* tmA_p, const CUtensor
 #pragma unroll
                     for (int q = 0; q < OB / 8; ++q) {
                         float bb[8];
-                        if (p.bias2) {
-                            unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.bias2 + (size_t)e * C::N2 + cb + q * 8)), bb);
+                        if (p.bias2 && (e & vs) == 0) {
+                            unpack16<bf16>(__ldg(reinterpret_cast<const uint4*>(p.bias2 + (size_t)(e >> vs) * C::N2 + cb + q * 8)), bb);
                         } else {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) bb[i] = 0.0f;

@@ -36,6 +36,9 @@ SMALL = {
     "bf16_gelu_biased": LC("gelub", T=130, d=512, S=4, E=16, k=1, F=512, init="kaiming"),
     "bf16_e64_ds64": LC("e64", T=260, d=128, S=2, E=64, k=2, F=128),
     "bf16_ds256_k2": LC("w256", T=70, d=512, S=2, E=16, k=2, F=512, Hr=128),
+    # 256-wide slices, k = 1, few tiles: the expert pass runs every tile as two tiles over halves of the hidden layer
+    # (W2's column halves, b2 added once); real biases
+    "bf16_ds256_k1_split": LC("w256k1", T=300, d=512, S=2, E=16, k=1, F=512, init="kaiming"),
     # the paper's d = 768 at S = 16 and S = 4: 48- and 192-wide slices on zero-filled 64 / 256-wide tiles
     # eight experts on the 16-wide router instantiation (padded experts masked out)
     "bf16_e8": LC("e8", T=150, d=512, S=4, E=8, k=2, F=512),

@@ -489,3 +489,37 @@ def test_forward_64wide_list_dispatch_shapes(T, E, k, init):
     torch.cuda.synchronize()
     for a, b in zip(first, again):
         assert torch.equal(a, b)
+
+
+def test_forward_random_wide_slice_shapes():
+    """Sixteen seeded random shapes with slices of 96 to 256 elements (E, k, S, F, batch size, activation, bias
+    init and capacity limit drawn at random): the forward against the oracle, the staged route without the
+    probability matrix against the oracle's routing, and two forwards on the same workspace bit for bit.  Covers
+    the router with resident weights, its hand-over to the single kernel and the split expert tiles on shapes
+    nobody picked by hand."""
+    import torch
+    rng = np.random.default_rng(20251004286)
+    for i in range(16):
+        E = int(rng.choice([8, 16, 32, 64]))
+        k = int(rng.choice([1, 1, 2]))
+        ds = int(rng.choice([96, 128, 192, 256, 256]))
+        S = int(rng.choice([1, 2, 4]))
+        F = int(rng.choice([2, 4])) * ds
+        T = max(1, int(rng.choice([1, 17, 129, 500, 1111, 2500, 6000, 12000])) // S)
+        init = str(rng.choice(["normal", "kaiming"]))
+        act = int(rng.choice([0, 1]))
+        cap = int(rng.choice([0, 0, 1])) * max(1, int(1.25 * T * S * k / E) // int(rng.choice([1, 4, 40])))
+        lc = LC(f"rw{i}", T=T, d=ds * S, S=S, E=E, k=k, F=F, act=act, init=init, capacity=cap)
+        rep = pu.check_forward_against_oracle(lc, seed=int(rng.integers(1 << 30)), sample_rows=2048,
+                                              one_ulp_of_element=True)
+        h, w = inputs(lc)
+        gpu = pu.GpuLayer(lc, h, w)
+        idx, p, _, _ = gpu.route(want_probs=False)
+        torch.cuda.synchronize()
+        ref = oracle.route(pu.oracle_config(lc), h, w)
+        pu.check_routing(ref["probs"], ref["gap"], ref["topk_idx"], idx.cpu().numpy(), p.cpu().numpy().astype(np.float64))
+        a, b = gpu.forward(), gpu.forward()
+        torch.cuda.synchronize()
+        assert all(torch.equal(x, y) for x, y in zip(a, b)) and gpu.status() == 0
+        print(lc.name, dict(T=T, S=S, ds=ds, E=E, k=k, F=F, act=act, init=init, capacity=cap), rep)
+

@@ -105,7 +105,7 @@ bool tc_ffn_supported(const Dims& D);
 int launch_route_tc(const Dims& D, const slicemoe_weights& w, const void* h, int32_t* topk_idx,
                     float* topk_p, int32_t* assigned, float* probs_opt, int32_t* status, cudaStream_t st,
                     int32_t* cta_hist = nullptr, void* zero_out = nullptr);
-// The router of wide slices (rows of 192 / 256 elements, router hidden width 256, k <= 2) with Wr1 and Wr2 resident
+// The router of slices of 96 / 128 / 192 / 256 elements (router hidden width 256, k <= 8) with Wr1 and Wr2 resident
 // in shared memory; same outputs, grid and row partition as launch_route_tc without the probability matrix.
 // grid_rows: launch at least that many CTAs, so that cta_hist has that many rows (the single-kernel forward's
 // dispatch reads one row per CTA of ITS grid, the number of SMs).

@@ -1,5 +1,5 @@
 // Router of slices of 96 to 256 elements (Section 3.1: relu(X Wr1^T + br1) Wr2^T + br2 -> softmax -> top-k), bf16
-// storage, router hidden width 256, up to 64 experts, k <= 2 (sm_100a: tcgen05 + TMEM + TMA).
+// storage, router hidden width 256, up to 64 experts, k <= 8 (sm_100a: tcgen05 + TMEM + TMA).
 //
 // The whole of Wr1 (up to 128 KB) and Wr2 stay in shared memory for the life of the CTA, so a tile's GEMM-1 runs as
 // wide MMAs against operands that are written to shared memory once per launch, not once per tile: what a tile
@@ -89,7 +89,9 @@ struct WrCfg {
 
 __device__ __forceinline__ uint32_t wr_bar(WrShared& sh, int i) { return smem_u32(&sh.bars[i]); }
 
-template <int EP, int KP>
+// KBIG: k may exceed 2 (a kernel of its own: the extra picks' code and registers cost the k <= 2 kernel 4 % of its
+// time on 64 experts when they share one)
+template <int EP, int KP, bool KBIG>
 __global__ void __launch_bounds__(kPpThreads, 1)
 route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW1,
                   const __grid_constant__ CUtensorMap tmW2, const PpParams p) {
@@ -460,13 +462,34 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             if (valid) {
                 const size_t at = (size_t)n * p.k;
                 atomicAdd(&sh.hist[i1], 1);
-                if (p.k > 1) {
-                    *reinterpret_cast<int2*>(p.topk_idx + at) = make_int2(i1, i2);
-                    *reinterpret_cast<float2*>(p.topk_p + at) = make_float2(inv, p2);
-                    atomicAdd(&sh.hist[i2], 1);
-                } else {
+                if (p.k == 1) {
                     p.topk_idx[at] = i1;
                     p.topk_p[at] = inv;
+                } else {
+                    if (!KBIG || p.k == 2) {
+                        *reinterpret_cast<int2*>(p.topk_idx + at) = make_int2(i1, i2);
+                        *reinterpret_cast<float2*>(p.topk_p + at) = make_float2(inv, p2);
+                    } else {
+                        p.topk_idx[at] = i1;     p.topk_p[at] = inv;
+                        p.topk_idx[at + 1] = i2; p.topk_p[at + 1] = p2;
+                    }
+                    atomicAdd(&sh.hist[i2], 1);
+                    // k > 2: the rest by repeated arg-max over what is left (ties to the lower id)
+                    unsigned long long taken = (1ull << i1) | (1ull << i2);
+                    for (int j = 2; KBIG && j < p.k; ++j) {
+                        int best = -1;
+                        float bv = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < EP; ++i) {
+                            const float gl = __uint_as_float(v[i]);
+                            const bool free_i = !((taken >> i) & 1ull);
+                            if (free_i && (best < 0 || gl > bv)) { best = i; bv = gl; }
+                        }
+                        taken |= 1ull << best;
+                        p.topk_idx[at + j] = best;
+                        p.topk_p[at + j] = ex2_approx(fmaf(bv, sc, -msc)) * inv;
+                        atomicAdd(&sh.hist[best], 1);
+                    }
                 }
             }
         }
@@ -490,7 +513,7 @@ route_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     }
 }
 
-template <int EP, int KP>
+template <int EP, int KP, bool KBIG>
 int launch_wide(const Dims& D, const slicemoe_weights& w, const void* h, const PpParams& rp, int grid, cudaStream_t st) {
     CUtensorMap mX, mW1, mW2;
     int rc;
@@ -498,7 +521,7 @@ int launch_wide(const Dims& D, const slicemoe_weights& w, const void* h, const P
     if ((rc = make_tmap(&mX, h, (uint64_t)D.N, (uint64_t)D.ds, kTileM))) return rc;
     if ((rc = make_tmap(&mW1, w.Wr1, (uint64_t)D.Hr, (uint64_t)D.ds, kWrHr))) return rc;
     if ((rc = make_tmap(&mW2, w.Wr2, (uint64_t)D.E, (uint64_t)D.Hr, EP))) return rc;      // (E = 8: zero-filled up to 16)
-    auto kern = route_wide_kernel<EP, KP>;
+    auto kern = route_wide_kernel<EP, KP, KBIG>;
     static bool attr_set[kAttrMaxDevices] = {};
     static std::mutex attr_mutex;
     {
@@ -512,7 +535,8 @@ int launch_wide(const Dims& D, const slicemoe_weights& w, const void* h, const P
 
 template <int EP>
 int launch_wide_e(const Dims& D, const slicemoe_weights& w, const void* h, const PpParams& rp, int grid, cudaStream_t st) {
-    return D.ds <= 128 ? launch_wide<EP, 2>(D, w, h, rp, grid, st) : launch_wide<EP, 4>(D, w, h, rp, grid, st);
+    if (D.k > 2) return D.ds <= 128 ? launch_wide<EP, 2, true>(D, w, h, rp, grid, st) : launch_wide<EP, 4, true>(D, w, h, rp, grid, st);
+    return D.ds <= 128 ? launch_wide<EP, 2, false>(D, w, h, rp, grid, st) : launch_wide<EP, 4, false>(D, w, h, rp, grid, st);
 }
 
 }  // namespace
@@ -520,7 +544,7 @@ int launch_wide_e(const Dims& D, const slicemoe_weights& w, const void* h, const
 bool wide_route_supported(const Dims& D) {
     if (D.dtype != SLICEMOE_BF16 || (D.ds != 256 && D.ds != 192 && D.ds != 128 && D.ds != 96) || D.N <= 0) return false;
     if (D.E != 8 && D.E != 16 && D.E != 32 && D.E != 64) return false;
-    if (D.k > 2 || D.noise_sigma > 0.0f) return false;
+    if (D.k > 8 || D.k > D.E || D.noise_sigma > 0.0f) return false;
     return D.Hr == kWrHr;
 }
 

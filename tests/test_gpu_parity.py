@@ -44,6 +44,7 @@ SMALL = {
     "bf16_e8": LC("e8", T=150, d=512, S=4, E=8, k=2, F=512),
     # k = 3 (the paper's Table 4) on the tensor-core kernels: stacked outputs + combine kernel
     "bf16_k3_tc": LC("k3tc", T=200, d=512, S=8, E=16, k=3, F=256),
+    "bf16_k3_slice96": LC("k3s96", T=300, d=768, S=8, E=16, k=3, F=384),   # k = 3 at the paper's own width: four launches + combine
     "bf16_paper_slice48": LC("s48", T=50, d=768, S=16, E=16, k=2, F=192),
     "bf16_paper_slice192": LC("s192", T=60, d=768, S=4, E=16, k=2, F=768),
     # S = 2 and S = 32 of the same sweep: 384- and 24-wide slices, CUDA-core kernels
@@ -79,6 +80,8 @@ def test_route(name):
     (30000, 512, 4, 32, 2, "normal"),     # 128-wide rows: two panels, three row tiles in shared memory, 7 tiles per CTA
     (9000, 768, 8, 8, 1, "kaiming"),      # 96-wide rows (zero-filled second panel), E = 8 on the 16-wide instantiation
     (100, 256, 1, 16, 2, "normal"),       # one ragged tile
+    (9000, 768, 8, 16, 3, "normal"),      # k = 3 (the paper's Table 4 shape): the third pick by repeated arg-max
+    (3000, 1024, 4, 64, 5, "kaiming"),    # k = 5 of 64 experts on 256-wide rows
 ])
 def test_route_resident_weights(T, d, S, E, k, init):
     """slicemoe_route without the probability matrix on slices of 96 to 256 elements (router hidden width 256):
